@@ -1,0 +1,553 @@
+/*
+ * ppo_oracle.c -- TEST INFRASTRUCTURE, NOT PRODUCT CODE.
+ *
+ * A plain, slow, CPU-only restatement of one PPO learner step over a rollout
+ * buffer D (Algorithm 2: D <- D U {(obs, actions, rew, done)}; TrainPPO(pi, D)).
+ * It exists so that the CUDA library can be checked against something that can
+ * be read by eye.  It shares no code, header, table or constant generator with
+ * the CUDA path, and nothing in the product may call it.
+ *
+ * Arithmetic is fp64 throughout.  The only places where a narrower precision is
+ * part of the definition are: weight matrices are rounded to bf16 (round to
+ * nearest even) before use; depth pixels arrive as fp16 values (exactly
+ * representable in fp64); the outputs of Adam are rounded to fp32.
+ *
+ * Every function states the passage it follows.  The paper itself gives
+ * TrainPPO only by name (Algorithm 2; Section III-C: "PPO", "CNN ... ReLU");
+ * the formulas are the textbook definitions of GAE(gamma, lambda), PPO-clip,
+ * the diagonal Gaussian policy and Adam that it cites.
+ *
+ * Pinned by tests/test_oracle_*.py (worked 2-env x 3-step example, closed
+ * forms, finite differences, brute force permutation checks, textbook special
+ * cases).  No function here is "parity unpinned".
+ *
+ * Build: gcc -O2 -fopenmp -shared -fPIC (see oracle/build.py).
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+#define ORC_MAX_CONV 8
+#define ORC_MAX_FC 4
+
+/* Network shape.  Section III-C: a CNN with ReLU on the depth image, combined
+ * with proprioception, then fully connected layers.  Every conv has stride 2
+ * and zero padding k/2; widths come from the workload description. */
+typedef struct {
+    int32_t H, W;                 /* depth image */
+    int32_t n_conv;
+    int32_t conv_c[ORC_MAX_CONV]; /* output channels */
+    int32_t conv_k[ORC_MAX_CONV]; /* square kernel size (odd) */
+    int32_t n_fc;
+    int32_t fc[ORC_MAX_FC];       /* hidden widths */
+    int32_t P, A;                 /* proprio width, action width */
+} orc_model;
+
+int orc_num_threads(void) {
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}
+
+/* ---------------------------------------------------------------- buffer -- */
+
+/* Section III-B: the buffer holds, per env and per step of the horizon, one
+ * depth frame; its size is N*T*H*W*elem bytes (the text's example: 512 envs,
+ * 320x240, 16 steps, fp32 = "2.5GB"). */
+uint64_t orc_depth_bytes(uint64_t N, uint64_t T, uint64_t H, uint64_t W, uint64_t elem) {
+    return N * T * H * W * elem;
+}
+
+/* ------------------------------------------------------------------- GAE -- */
+
+/* GAE(gamma, lambda) for TrainPPO (Algorithm 2).  Time-major arrays [T][N].
+ * done[t][n] was returned by the same Env.Step as reward[t][n], so it cuts
+ * the bootstrap from step t to step t+1.
+ *   delta_t = r_t + gamma * V_{t+1} * (1 - d_t) - V_t
+ *   A_t     = delta_t + gamma * lambda * (1 - d_t) * A_{t+1}
+ *   R_t     = A_t + V_t,      V_T = last_value, A_T = 0 */
+void orc_gae(int T, int N, const float *reward, const float *value, const uint8_t *done,
+             const float *last_value, double gamma, double lambda, double *adv, double *ret) {
+    for (int n = 0; n < N; ++n) {
+        double v_next = (double)last_value[n];
+        double a_next = 0.0;
+        for (int t = T - 1; t >= 0; --t) {
+            size_t i = (size_t)t * N + n;
+            double not_done = done[i] ? 0.0 : 1.0;
+            double v = (double)value[i];
+            double delta = (double)reward[i] + gamma * v_next * not_done - v;
+            double a = delta + gamma * lambda * not_done * a_next;
+            adv[i] = a;
+            ret[i] = a + v;
+            v_next = v;
+            a_next = a;
+        }
+    }
+}
+
+/* Advantage normalisation over the whole buffer, once, before minibatching:
+ * mu = mean, sigma = unbiased (M-1) standard deviation, a <- (a-mu)/(sigma+1e-8). */
+void orc_adv_normalize(size_t M, double *adv, double *mean_out, double *std_out) {
+    double s = 0.0;
+    for (size_t i = 0; i < M; ++i) s += adv[i];
+    double mu = s / (double)M;
+    double q = 0.0;
+    for (size_t i = 0; i < M; ++i) q += (adv[i] - mu) * (adv[i] - mu);
+    double sigma = (M > 1) ? sqrt(q / (double)(M - 1)) : 0.0;
+    for (size_t i = 0; i < M; ++i) adv[i] = (adv[i] - mu) / (sigma + 1e-8);
+    if (mean_out) *mean_out = mu;
+    if (std_out) *std_out = sigma;
+}
+
+/* ----------------------------------------------------------- permutation -- */
+
+/* Seeded bijection on [0, M): a 6-round balanced Feistel network on 2h bits
+ * (2^(2h) >= M) with cycle walking.  All arithmetic is uint32 with wrap-around. */
+uint32_t orc_mix32(uint32_t x) {
+    x ^= x >> 16;
+    x *= 0x9E3779B9u;
+    x ^= x >> 15;
+    x *= 0x6A09E667u;
+    x ^= x >> 16;
+    return x;
+}
+
+void orc_perm_keys(uint64_t seed, uint32_t epoch, uint32_t key[6]) {
+    uint32_t lo = (uint32_t)(seed & 0xFFFFFFFFu), hi = (uint32_t)(seed >> 32);
+    for (uint32_t j = 0; j < 6; ++j) {
+        uint32_t a = orc_mix32(hi + 0x9E3779B9u * (j + 1));
+        uint32_t b = orc_mix32(epoch + 0xBB67AE85u * (j + 1));
+        key[j] = orc_mix32(lo ^ a ^ b);
+    }
+}
+
+int orc_perm_half_bits(uint32_t M) {
+    int bits = 0; /* smallest bits with 2^bits >= M */
+    while (((uint64_t)1 << bits) < (uint64_t)M) ++bits;
+    int h = (bits + 1) / 2;
+    return h < 1 ? 1 : h;
+}
+
+uint32_t orc_perm(uint64_t seed, uint32_t epoch, uint32_t M, uint32_t i) {
+    uint32_t key[6];
+    orc_perm_keys(seed, epoch, key);
+    int h = orc_perm_half_bits(M);
+    uint32_t mask = ((uint32_t)1 << h) - 1u;
+    uint32_t x = i;
+    do {
+        uint32_t L = x >> h, R = x & mask;
+        for (int j = 0; j < 6; ++j) {
+            uint32_t newR = L ^ (orc_mix32(R ^ key[j]) & mask);
+            L = R;
+            R = newR;
+        }
+        x = (L << h) | R;
+    } while (x >= M);
+    return x;
+}
+
+/* Minibatch k of K (B = M/K rows): row j holds sample orc_perm(k*B + j). */
+void orc_perm_fill(uint64_t seed, uint32_t epoch, uint32_t M, uint32_t start, uint32_t count, uint32_t *out) {
+    for (uint32_t j = 0; j < count; ++j) out[j] = orc_perm(seed, epoch, M, start + j);
+}
+
+/* ---------------------------------------------------------------- layout -- */
+
+double orc_round_bf16(double x) {
+    float f = (float)x;
+    uint32_t u;
+    memcpy(&u, &f, 4);
+    if ((u & 0x7F800000u) == 0x7F800000u) return (double)f; /* inf / nan unchanged */
+    uint32_t lsb = (u >> 16) & 1u;
+    u += 0x7FFFu + lsb; /* round to nearest, ties to even */
+    u &= 0xFFFF0000u;
+    memcpy(&f, &u, 4);
+    return (double)f;
+}
+
+static int conv_out(int in, int k) { return (in + 2 * (k / 2) - k) / 2 + 1; }
+
+void orc_conv_shapes(const orc_model *m, int32_t *Ho, int32_t *Wo) {
+    int h = m->H, w = m->W;
+    for (int l = 0; l < m->n_conv; ++l) {
+        h = conv_out(h, m->conv_k[l]);
+        w = conv_out(w, m->conv_k[l]);
+        Ho[l] = h;
+        Wo[l] = w;
+    }
+}
+
+/* Parameter vector layout (an interface shared with the caller, restated here):
+ * tensors in the order conv W_l [Cout][k][k][Cin], conv b_l, ..., fc W [out][in],
+ * fc b, ..., head W [A+1][hid] (rows 0..A-1 mean, row A value), head b [A+1],
+ * log-sigma [A]; each tensor starts at a multiple of 64 elements.
+ * offsets/sizes must have room for 2*n_conv + 2*n_fc + 3 entries.
+ * Returns the total length of the vector; *n_tensors gets the tensor count. */
+int64_t orc_param_layout(const orc_model *m, int64_t *offsets, int64_t *sizes, int32_t *is_matrix, int32_t *n_tensors) {
+    int64_t off = 0;
+    int n = 0;
+    int cin = 1;
+#define PUSH(sz, mat)                        \
+    do {                                     \
+        offsets[n] = off;                    \
+        sizes[n] = (sz);                     \
+        is_matrix[n] = (mat);                \
+        off += ((int64_t)(sz) + 63) / 64 * 64; \
+        ++n;                                 \
+    } while (0)
+    for (int l = 0; l < m->n_conv; ++l) {
+        PUSH((int64_t)m->conv_c[l] * m->conv_k[l] * m->conv_k[l] * cin, 1);
+        PUSH(m->conv_c[l], 0);
+        cin = m->conv_c[l];
+    }
+    int in = cin + m->P;
+    for (int l = 0; l < m->n_fc; ++l) {
+        PUSH((int64_t)m->fc[l] * in, 1);
+        PUSH(m->fc[l], 0);
+        in = m->fc[l];
+    }
+    PUSH((int64_t)(m->A + 1) * in, 1);
+    PUSH(m->A + 1, 0);
+    PUSH(m->A, 0);
+#undef PUSH
+    *n_tensors = n;
+    return off;
+}
+
+/* Weight matrices are used as bf16-rounded copies of the fp32 master; biases
+ * and log-sigma are used as they are. */
+void orc_round_weights(const orc_model *m, const double *theta, double *theta_used) {
+    int64_t offs[2 * ORC_MAX_CONV + 2 * ORC_MAX_FC + 3], szs[2 * ORC_MAX_CONV + 2 * ORC_MAX_FC + 3];
+    int32_t mat[2 * ORC_MAX_CONV + 2 * ORC_MAX_FC + 3], n;
+    int64_t total = orc_param_layout(m, offs, szs, mat, &n);
+    for (int64_t i = 0; i < total; ++i) theta_used[i] = theta[i];
+    for (int t = 0; t < n; ++t)
+        if (mat[t])
+            for (int64_t i = 0; i < szs[t]; ++i) theta_used[offs[t] + i] = orc_round_bf16(theta[offs[t] + i]);
+}
+
+/* Per-sample activation record: [image H*W | a_1 | ... | a_L | h_0 = pooled ++ proprio | h_1 | ... | h_F]. */
+int64_t orc_act_stride(const orc_model *m) {
+    int32_t Ho[ORC_MAX_CONV], Wo[ORC_MAX_CONV];
+    orc_conv_shapes(m, Ho, Wo);
+    int64_t s = (int64_t)m->H * m->W;
+    for (int l = 0; l < m->n_conv; ++l) s += (int64_t)Ho[l] * Wo[l] * m->conv_c[l];
+    s += m->conv_c[m->n_conv - 1] + m->P;
+    for (int l = 0; l < m->n_fc; ++l) s += m->fc[l];
+    return s;
+}
+
+/* --------------------------------------------------------------- encoder -- */
+
+/* Forward of one sample (Section III-C: CNN + ReLU on depth, concatenated with
+ * proprioception, fully connected layers; heads give the Gaussian mean and the value).
+ *   conv: y[oh][ow][co] = ReLU(b[co] + sum_{kh,kw,ci} W[co][kh][kw][ci] * x[2*oh+kh-p][2*ow+kw-p][ci])
+ *         (cross-correlation, zero outside the image, p = k/2)
+ *   g = mean of the last conv output over its pixels; h_0 = [g, proprio]
+ *   h_l = ReLU(W_l h_{l-1} + b_l);  out = W_head h_F + b_head; mu = out[0..A), V = out[A]. */
+static void fwd_one(const orc_model *m, const double *th, const int64_t *offs, const double *depth,
+                    const double *proprio, double *act, double *mu, double *V) {
+    int32_t Ho[ORC_MAX_CONV], Wo[ORC_MAX_CONV];
+    orc_conv_shapes(m, Ho, Wo);
+    double *x = act;
+    for (int64_t i = 0; i < (int64_t)m->H * m->W; ++i) x[i] = depth[i];
+    int hin = m->H, win = m->W, cin = 1;
+    int ti = 0;
+    for (int l = 0; l < m->n_conv; ++l) {
+        int k = m->conv_k[l], p = k / 2, co_n = m->conv_c[l];
+        const double *Wt = th + offs[ti], *b = th + offs[ti + 1];
+        ti += 2;
+        double *y = x + (int64_t)hin * win * cin;
+        for (int oh = 0; oh < Ho[l]; ++oh)
+            for (int ow = 0; ow < Wo[l]; ++ow)
+                for (int co = 0; co < co_n; ++co) {
+                    double acc = b[co];
+                    for (int kh = 0; kh < k; ++kh) {
+                        int ih = 2 * oh + kh - p;
+                        if (ih < 0 || ih >= hin) continue;
+                        for (int kw = 0; kw < k; ++kw) {
+                            int iw = 2 * ow + kw - p;
+                            if (iw < 0 || iw >= win) continue;
+                            const double *wp = Wt + (((int64_t)co * k + kh) * k + kw) * cin;
+                            const double *xp = x + ((int64_t)ih * win + iw) * cin;
+                            for (int ci = 0; ci < cin; ++ci) acc += wp[ci] * xp[ci];
+                        }
+                    }
+                    y[((int64_t)oh * Wo[l] + ow) * co_n + co] = acc > 0.0 ? acc : 0.0;
+                }
+        x = y;
+        hin = Ho[l];
+        win = Wo[l];
+        cin = co_n;
+    }
+    /* global average pool, then concatenate proprio */
+    double *h = x + (int64_t)hin * win * cin;
+    for (int c = 0; c < cin; ++c) {
+        double s = 0.0;
+        for (int px = 0; px < hin * win; ++px) s += x[(int64_t)px * cin + c];
+        h[c] = s / (double)(hin * win);
+    }
+    for (int j = 0; j < m->P; ++j) h[cin + j] = proprio[j];
+    int in = cin + m->P;
+    for (int l = 0; l < m->n_fc; ++l) {
+        const double *Wt = th + offs[ti], *b = th + offs[ti + 1];
+        ti += 2;
+        double *y = h + in;
+        for (int o = 0; o < m->fc[l]; ++o) {
+            double acc = b[o];
+            for (int i = 0; i < in; ++i) acc += Wt[(int64_t)o * in + i] * h[i];
+            y[o] = acc > 0.0 ? acc : 0.0;
+        }
+        h = y;
+        in = m->fc[l];
+    }
+    const double *Wh = th + offs[ti], *bh = th + offs[ti + 1];
+    for (int o = 0; o <= m->A; ++o) {
+        double acc = bh[o];
+        for (int i = 0; i < in; ++i) acc += Wh[(int64_t)o * in + i] * h[i];
+        if (o < m->A) mu[o] = acc; else *V = acc;
+    }
+}
+
+/* Chain rule through fwd_one for one sample; adds this sample's gradient into g
+ * (same layout as the parameter vector).  ReLU' = 1 where the stored output is
+ * > 0 (equivalently the pre-activation is > 0), else 0.  The log-sigma slot of g
+ * is not touched here (it has no path through the network). */
+static void bwd_one(const orc_model *m, const double *th, const int64_t *offs, int n_tensors, const double *act,
+                    const double *dmu, double dV, double *g, double *scratch) {
+    int32_t Ho[ORC_MAX_CONV], Wo[ORC_MAX_CONV];
+    orc_conv_shapes(m, Ho, Wo);
+    /* locate activations */
+    const double *a[ORC_MAX_CONV + 1];
+    int hs[ORC_MAX_CONV + 1], ws[ORC_MAX_CONV + 1], cs[ORC_MAX_CONV + 1];
+    a[0] = act; hs[0] = m->H; ws[0] = m->W; cs[0] = 1;
+    for (int l = 0; l < m->n_conv; ++l) {
+        a[l + 1] = a[l] + (int64_t)hs[l] * ws[l] * cs[l];
+        hs[l + 1] = Ho[l]; ws[l + 1] = Wo[l]; cs[l + 1] = m->conv_c[l];
+    }
+    int L = m->n_conv, F = m->n_fc;
+    const double *hv[ORC_MAX_FC + 1];
+    int hn[ORC_MAX_FC + 1];
+    hv[0] = a[L] + (int64_t)hs[L] * ws[L] * cs[L];
+    hn[0] = cs[L] + m->P;
+    for (int l = 0; l < F; ++l) { hv[l + 1] = hv[l] + hn[l]; hn[l + 1] = m->fc[l]; }
+
+    /* scratch: two ping-pong gradient buffers large enough for any activation */
+    int64_t big = (int64_t)m->H * m->W;
+    for (int l = 1; l <= L; ++l) { int64_t s = (int64_t)hs[l] * ws[l] * cs[l]; if (s > big) big = s; }
+    for (int l = 0; l <= F; ++l) if (hn[l] > big) big = hn[l];
+    double *d_cur = scratch, *d_prev = scratch + big;
+
+    /* head */
+    int ti = n_tensors - 3; /* head W, head b, log-sigma */
+    {
+        const double *Wh = th + offs[ti];
+        double *gW = g + offs[ti], *gb = g + offs[ti + 1];
+        int in = hn[F];
+        for (int i = 0; i < in; ++i) d_cur[i] = 0.0;
+        for (int o = 0; o <= m->A; ++o) {
+            double d = (o < m->A) ? dmu[o] : dV;
+            gb[o] += d;
+            for (int i = 0; i < in; ++i) {
+                gW[(int64_t)o * in + i] += d * hv[F][i];
+                d_cur[i] += Wh[(int64_t)o * in + i] * d;
+            }
+        }
+    }
+    /* hidden fc layers, last to first; d_cur holds dL/dh_l (post-ReLU) */
+    for (int l = F; l >= 1; --l) {
+        ti -= 2;
+        const double *Wt = th + offs[ti];
+        double *gW = g + offs[ti], *gb = g + offs[ti + 1];
+        int in = hn[l - 1], out = hn[l];
+        for (int i = 0; i < in; ++i) d_prev[i] = 0.0;
+        for (int o = 0; o < out; ++o) {
+            double dz = hv[l][o] > 0.0 ? d_cur[o] : 0.0;
+            gb[o] += dz;
+            for (int i = 0; i < in; ++i) {
+                gW[(int64_t)o * in + i] += dz * hv[l - 1][i];
+                d_prev[i] += Wt[(int64_t)o * in + i] * dz;
+            }
+        }
+        double *tmp = d_cur; d_cur = d_prev; d_prev = tmp;
+    }
+    /* un-pool: every pixel of the last conv output gets dg[c] / (Ho*Wo); the proprio part ends here */
+    {
+        int npx = hs[L] * ws[L], c_n = cs[L];
+        for (int px = 0; px < npx; ++px)
+            for (int c = 0; c < c_n; ++c) d_prev[(int64_t)px * c_n + c] = d_cur[c] / (double)npx;
+        double *tmp = d_cur; d_cur = d_prev; d_prev = tmp;
+    }
+    /* conv layers, last to first; d_cur holds dL/da_l (post-ReLU) */
+    for (int l = L; l >= 1; --l) {
+        ti -= 2;
+        int k = m->conv_k[l - 1], p = k / 2, co_n = cs[l], cin = cs[l - 1];
+        int hin = hs[l - 1], win = ws[l - 1];
+        const double *Wt = th + offs[ti];
+        double *gW = g + offs[ti], *gb = g + offs[ti + 1];
+        const double *x = a[l - 1], *y = a[l];
+        if (l > 1) for (int64_t i = 0; i < (int64_t)hin * win * cin; ++i) d_prev[i] = 0.0;
+        for (int oh = 0; oh < hs[l]; ++oh)
+            for (int ow = 0; ow < ws[l]; ++ow)
+                for (int co = 0; co < co_n; ++co) {
+                    int64_t oi = ((int64_t)oh * ws[l] + ow) * co_n + co;
+                    double dz = y[oi] > 0.0 ? d_cur[oi] : 0.0;
+                    if (dz == 0.0) continue;
+                    gb[co] += dz;
+                    for (int kh = 0; kh < k; ++kh) {
+                        int ih = 2 * oh + kh - p;
+                        if (ih < 0 || ih >= hin) continue;
+                        for (int kw = 0; kw < k; ++kw) {
+                            int iw = 2 * ow + kw - p;
+                            if (iw < 0 || iw >= win) continue;
+                            int64_t wi = (((int64_t)co * k + kh) * k + kw) * cin;
+                            int64_t xi = ((int64_t)ih * win + iw) * cin;
+                            for (int ci = 0; ci < cin; ++ci) {
+                                gW[wi + ci] += dz * x[xi + ci];
+                                if (l > 1) d_prev[xi + ci] += Wt[wi + ci] * dz;
+                            }
+                        }
+                    }
+                }
+        double *tmp = d_cur; d_cur = d_prev; d_prev = tmp;
+    }
+}
+
+int64_t orc_bwd_scratch_len(const orc_model *m) {
+    int32_t Ho[ORC_MAX_CONV], Wo[ORC_MAX_CONV];
+    orc_conv_shapes(m, Ho, Wo);
+    int64_t big = (int64_t)m->H * m->W;
+    for (int l = 0; l < m->n_conv; ++l) { int64_t s = (int64_t)Ho[l] * Wo[l] * m->conv_c[l]; if (s > big) big = s; }
+    int64_t h0 = m->conv_c[m->n_conv - 1] + m->P;
+    if (h0 > big) big = h0;
+    for (int l = 0; l < m->n_fc; ++l) if (m->fc[l] > big) big = m->fc[l];
+    return 2 * big;
+}
+
+/* Forward of B samples.  theta_used: parameter vector with weight matrices already
+ * bf16-rounded (orc_round_weights).  acts: B * orc_act_stride doubles (kept for backward). */
+void orc_encoder_fwd(const orc_model *m, const double *theta_used, int B, const double *depth, const double *proprio,
+                     double *acts, double *mu, double *V) {
+    int64_t offs[2 * ORC_MAX_CONV + 2 * ORC_MAX_FC + 3], szs[2 * ORC_MAX_CONV + 2 * ORC_MAX_FC + 3];
+    int32_t mat[2 * ORC_MAX_CONV + 2 * ORC_MAX_FC + 3], n;
+    orc_param_layout(m, offs, szs, mat, &n);
+    int64_t stride = orc_act_stride(m);
+#pragma omp parallel for schedule(dynamic)
+    for (int b = 0; b < B; ++b)
+        fwd_one(m, theta_used, offs, depth + (int64_t)b * m->H * m->W, proprio + (int64_t)b * m->P,
+                acts + b * stride, mu + (int64_t)b * m->A, V + b);
+}
+
+/* Backward of B samples: grad (length = parameter vector) += sum over samples of the
+ * per-sample gradient, given dL/dmu [B][A] and dL/dV [B]. */
+void orc_encoder_bwd(const orc_model *m, const double *theta_used, int B, const double *acts, const double *dmu,
+                     const double *dV, double *grad) {
+    int64_t offs[2 * ORC_MAX_CONV + 2 * ORC_MAX_FC + 3], szs[2 * ORC_MAX_CONV + 2 * ORC_MAX_FC + 3];
+    int32_t mat[2 * ORC_MAX_CONV + 2 * ORC_MAX_FC + 3], n;
+    int64_t total = orc_param_layout(m, offs, szs, mat, &n);
+    int64_t stride = orc_act_stride(m);
+    int64_t slen = orc_bwd_scratch_len(m);
+#pragma omp parallel
+    {
+        double *g_local = (double *)calloc((size_t)total, sizeof(double));
+        double *scratch = (double *)malloc((size_t)slen * sizeof(double));
+#pragma omp for schedule(dynamic)
+        for (int b = 0; b < B; ++b)
+            bwd_one(m, theta_used, offs, n, acts + b * stride, dmu + (int64_t)b * m->A, dV[b], g_local, scratch);
+#pragma omp critical
+        for (int64_t i = 0; i < total; ++i) grad[i] += g_local[i];
+        free(g_local);
+        free(scratch);
+    }
+}
+
+/* ------------------------------------------------------------------ loss -- */
+
+/* PPO-clip loss with a diagonal Gaussian policy (state-independent log-sigma), an
+ * unclipped squared-error value loss and an entropy bonus, and its gradient with
+ * respect to mu, V and log-sigma.  Rows i < B, means over B_total rows.
+ *   z = (a - mu)/sigma, sigma = exp(logsigma)
+ *   logp = sum_j [ -z_j^2/2 - logsigma_j - ln(2 pi)/2 ]
+ *   r = exp(logp - logp_old);  s = min(r*Adv, clamp(r, 1-eps, 1+eps)*Adv)
+ *   L_pi = -mean(s);  L_V = mean((V - R)^2);  H = sum_j logsigma_j + (A/2)(1 + ln(2 pi))
+ *   L = L_pi + c_v L_V - c_e H
+ * out[0..4] += {L_pi, L_V, H * B/B_total, mean(logp_old - logp), mean(|r-1| > eps)} contributions
+ * of these B rows (so that micro-batches sum to the minibatch value; H is a constant of the
+ * parameters and is reported weighted by the share of rows).
+ * dlogsigma[j] += sum_i dL/dlogp_i * (z_ij^2 - 1) - c_e * B/B_total. */
+void orc_loss(int B, int B_total, int A, const double *mu, const double *V, const double *logsigma,
+              const double *action, const double *logp_old, const double *adv, const double *ret, double clip,
+              double c_v, double c_e, double *out, double *dmu, double *dV, double *dlogsigma) {
+    const double half_log_2pi = 0.5 * log(2.0 * M_PI);
+    double Bt = (double)B_total;
+    double H = 0.0;
+    for (int j = 0; j < A; ++j) H += logsigma[j];
+    H += 0.5 * A * (1.0 + 2.0 * half_log_2pi);
+    for (int i = 0; i < B; ++i) {
+        double logp = 0.0;
+        for (int j = 0; j < A; ++j) {
+            double sg = exp(logsigma[j]);
+            double z = (action[(int64_t)i * A + j] - mu[(int64_t)i * A + j]) / sg;
+            logp += -0.5 * z * z - logsigma[j] - half_log_2pi;
+        }
+        double r = exp(logp - logp_old[i]);
+        double rc = r < 1.0 - clip ? 1.0 - clip : (r > 1.0 + clip ? 1.0 + clip : r);
+        double s_un = r * adv[i], s_cl = rc * adv[i];
+        double s, gs;
+        if (s_un <= s_cl) { s = s_un; gs = adv[i]; } else { s = s_cl; gs = 0.0; }
+        out[0] += -s / Bt;
+        double verr = V[i] - ret[i];
+        out[1] += verr * verr / Bt;
+        out[3] += (logp_old[i] - logp) / Bt;
+        out[4] += (fabs(r - 1.0) > clip ? 1.0 : 0.0) / Bt;
+        double dlogp = -gs * r / Bt;
+        for (int j = 0; j < A; ++j) {
+            double sg = exp(logsigma[j]);
+            double z = (action[(int64_t)i * A + j] - mu[(int64_t)i * A + j]) / sg;
+            dmu[(int64_t)i * A + j] = dlogp * z / sg;
+            dlogsigma[j] += dlogp * (z * z - 1.0);
+        }
+        dV[i] = 2.0 * c_v * verr / Bt;
+    }
+    out[2] += H * (double)B / Bt;
+    for (int j = 0; j < A; ++j) dlogsigma[j] += -c_e * (double)B / Bt;
+}
+
+/* Rollout-time action of the policy (Algorithm 2, actions <- pi(obs)):
+ * a = mu + sigma * eps with eps ~ N(0, I) supplied by the caller, and its log-probability. */
+void orc_sample_action(int B, int A, const double *mu, const double *logsigma, const double *eps, double *action,
+                       double *logp) {
+    const double half_log_2pi = 0.5 * log(2.0 * M_PI);
+    for (int i = 0; i < B; ++i) {
+        double lp = 0.0;
+        for (int j = 0; j < A; ++j) {
+            double e = eps[(int64_t)i * A + j];
+            action[(int64_t)i * A + j] = mu[(int64_t)i * A + j] + exp(logsigma[j]) * e;
+            lp += -0.5 * e * e - logsigma[j] - half_log_2pi;
+        }
+        logp[i] = lp;
+    }
+}
+
+/* ------------------------------------------------------------------ Adam -- */
+
+/* Adam with bias correction, epsilon outside the square root and after the
+ * correction, no weight decay; step is 1-based.  theta is rounded to fp32 on output
+ * (the master copy is fp32); m and v are kept in fp64 here. */
+void orc_adam(int64_t n, double *theta, double *m, double *v, const double *g, double lr, double beta1, double beta2,
+              double eps, int64_t step) {
+    double c1 = 1.0 - pow(beta1, (double)step), c2 = 1.0 - pow(beta2, (double)step);
+    for (int64_t i = 0; i < n; ++i) {
+        m[i] = beta1 * m[i] + (1.0 - beta1) * g[i];
+        v[i] = beta2 * v[i] + (1.0 - beta2) * g[i] * g[i];
+        double mhat = m[i] / c1, vhat = v[i] / c2;
+        theta[i] = (double)(float)(theta[i] - lr * mhat / (sqrt(vhat) + eps));
+    }
+}

@@ -1,0 +1,161 @@
+"""Seeded synthetic inputs for the PPO learner step.
+
+This module holds workload shapes and random input generators only; none of the
+learner's arithmetic lives here.  The frames stand in for a simulator's tiled
+depth rendering at 160x120 / 320x240 with a horizon of 16 (Section III-B,
+Table I): depth is uniform in [0.1, 2.0] m stored as fp16 with 10 % of the pixels
+zeroed (missing returns), proprioception is 32 standard normals, rewards and old
+values are standard normals, dones are Bernoulli.
+
+Two back ends produce the same distributions: numpy (Philox, for parity-sized
+cases that also feed the CPU checker) and torch on the device (for buffers of
+many GB that never visit the host).
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass, field
+from typing import Dict, List, Sequence
+
+import numpy as np
+
+
+@dataclass(frozen=True)
+class Workload:
+    name: str
+    N: int
+    T: int
+    H: int
+    W: int
+    conv_c: Sequence[int]
+    conv_k: Sequence[int]
+    fc: Sequence[int]
+    epochs: int
+    minibatches: int
+    done_rate: float = 0.01
+    P: int = 32
+    A: int = 12
+    gamma: float = 0.99
+    lam: float = 0.95
+    clip: float = 0.2
+    seed: int = 0
+
+    @property
+    def M(self) -> int:
+        return self.N * self.T
+
+    @property
+    def B(self) -> int:
+        return self.M // self.minibatches
+
+    def scaled(self, N: int, **kw) -> "Workload":
+        d = dict(self.__dict__)
+        d.update(N=N, **kw)
+        return Workload(**d)
+
+
+WORKLOADS: Dict[str, Workload] = {
+    "cfg1": Workload("cfg1", 256, 16, 64, 64, (16, 32, 64), (3, 3, 3), (256,), 1, 4),
+    "cfg2": Workload("cfg2", 1024, 16, 120, 160, (32, 64, 128, 256), (3, 3, 3, 3), (512, 512), 1, 4),
+    "cfg3": Workload("cfg3", 4096, 16, 120, 160, (32, 64, 128, 256), (3, 3, 3, 3), (512, 512), 5, 4),
+    "cfg4": Workload("cfg4", 8192, 16, 240, 320, (32, 64, 128, 256, 256), (5, 3, 3, 3, 3), (512, 512), 5, 8,
+                     done_rate=0.005),
+    "cfg5_1k": Workload("cfg5_1k", 1024, 32, 120, 160, (32, 64, 128, 256), (3, 3, 3, 3), (512, 512), 1, 4),
+    "cfg5_4k": Workload("cfg5_4k", 4096, 32, 120, 160, (32, 64, 128, 256), (3, 3, 3, 3), (512, 512), 1, 4),
+    "cfg5_16k": Workload("cfg5_16k", 16384, 32, 120, 160, (32, 64, 128, 256), (3, 3, 3, 3), (512, 512), 1, 4),
+}
+
+_FIELDS = ("depth", "proprio", "reward", "value", "done", "last_value", "eps", "logp_jitter")
+
+
+def _rng(seed: int, name: str) -> np.random.Generator:
+    return np.random.Generator(np.random.Philox(key=[seed, _FIELDS.index(name) + 1]))
+
+
+def rollout_numpy(w: Workload, seed: int | None = None) -> Dict[str, np.ndarray]:
+    """One rollout's worth of inputs, time-major [T, N, ...], one Philox stream per field.
+
+    `eps` is the standard-normal action noise the rollout policy consumed (the caller turns it into
+    actions and old log-probs with its own forward pass); `logp_jitter` is N(0, 0.3^2) noise a test may
+    add to the old log-probs so that both branches of the clip are exercised.
+    """
+    seed = w.seed if seed is None else seed
+    T, N = w.T, w.N
+    g = _rng(seed, "depth")
+    depth = g.uniform(0.1, 2.0, size=(T, N, w.H, w.W)).astype(np.float16)
+    depth[g.random(size=depth.shape) < 0.10] = 0
+    out = {
+        "depth": depth,
+        "proprio": _rng(seed, "proprio").standard_normal((T, N, w.P)).astype(np.float32),
+        "reward": _rng(seed, "reward").standard_normal((T, N)).astype(np.float32),
+        "value": _rng(seed, "value").standard_normal((T, N)).astype(np.float32),
+        "done": (_rng(seed, "done").random((T, N)) < w.done_rate).astype(np.uint8),
+        "last_value": _rng(seed, "last_value").standard_normal((N,)).astype(np.float32),
+        "eps": _rng(seed, "eps").standard_normal((T, N, w.A)).astype(np.float32),
+        "logp_jitter": (0.3 * _rng(seed, "logp_jitter").standard_normal((T, N))).astype(np.float32),
+    }
+    return out
+
+
+def rollout_torch(w: Workload, device, seed: int | None = None, chunk_t: int = 1):
+    """Same distributions generated on `device` with torch's generator (one seed per field and step).
+
+    Returns a dict of device tensors [T, N, ...].  Depth is produced step by step so that the fp32
+    temporaries stay small next to a buffer of tens of GB.
+    """
+    import torch
+
+    seed = w.seed if seed is None else seed
+    T, N = w.T, w.N
+    gen = torch.Generator(device=device)
+    depth = torch.empty((T, N, w.H, w.W), dtype=torch.float16, device=device)
+    # generate in slabs of at most ~64M pixels to bound the fp32 temporaries
+    rows = max(1, min(N, (64 << 20) // (w.H * w.W)))
+    for t in range(T):
+        gen.manual_seed(1_000_003 * (seed + 1) + t)
+        for n0 in range(0, N, rows):
+            n1 = min(N, n0 + rows)
+            u = torch.rand((n1 - n0, w.H, w.W), generator=gen, device=device)
+            d = (0.1 + 1.9 * u).to(torch.float16)
+            z = torch.rand((n1 - n0, w.H, w.W), generator=gen, device=device) < 0.10
+            d[z] = 0
+            depth[t, n0:n1] = d
+            del u, d, z
+
+    def normal(name, shape, scale=1.0):
+        gen.manual_seed(7_000_003 * (seed + 1) + _FIELDS.index(name))
+        return scale * torch.randn(shape, generator=gen, device=device, dtype=torch.float32)
+
+    gen.manual_seed(7_000_003 * (seed + 1) + _FIELDS.index("done"))
+    done = (torch.rand((T, N), generator=gen, device=device) < w.done_rate).to(torch.uint8)
+    return {
+        "depth": depth,
+        "proprio": normal("proprio", (T, N, w.P)),
+        "reward": normal("reward", (T, N)),
+        "value": normal("value", (T, N)),
+        "done": done,
+        "last_value": normal("last_value", (N,)),
+        "eps": normal("eps", (T, N, w.A)),
+        "logp_jitter": normal("logp_jitter", (T, N), 0.3),
+    }
+
+
+def init_params(total: int, offsets: List[int], shapes: List[tuple], seed: int) -> np.ndarray:
+    """Random initial fp32 parameter vector for a given tensor layout.
+
+    Weight tensors (rank >= 2) ~ U(+-sqrt(6 / fan_in)); the last weight tensor (the mean/value head) is
+    scaled by 0.01 so that the initial policy mean is near zero; rank-1 tensors (biases, log-sigma) are 0.
+    Gaps between tensors stay 0.
+    """
+    theta = np.zeros(total, np.float32)
+    g = np.random.Generator(np.random.Philox(key=[seed + 1, 99]))
+    mats = [i for i, s in enumerate(shapes) if len(s) >= 2]
+    for i in mats:
+        shp = shapes[i]
+        fan_in = int(np.prod(shp[1:]))
+        bound = np.sqrt(6.0 / fan_in)
+        n = int(np.prod(shp))
+        wts = g.uniform(-bound, bound, size=n).astype(np.float32)
+        if i == mats[-1]:
+            wts *= np.float32(0.01)
+        theta[offsets[i]: offsets[i] + n] = wts
+    return theta
