@@ -1,0 +1,439 @@
+#!/usr/bin/env python
+"""Benchmark of the PPO learner step (TrainPPO over an on-device rollout buffer) on B200.
+
+One "step" is one pass of the whole hot path over one buffer of synthetic rollouts:
+GAE + advantage normalisation, then for every epoch and minibatch the permutation gather,
+encoder forward, fused loss, encoder backward and Adam.  The metric is env-steps trained
+per second = M * epochs / time, with the buffer resident in HBM (`value`) and with the
+rollout arriving from pinned host memory every step (`e2e`).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg2] [--impl reference]
+
+With N > 1 (torchrun) every rank trains an independent replica on its own buffer: the
+path has no exchange step on one learner GPU, so there is no collective on the data path.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "ppo_learner_env_steps_trained_per_sec"
+UNIT = "env-steps/s"
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return {"hbm_gbs": d["hbm_gbs"], "bf16_tflops": d["bf16_tflops"],
+                "bf16_tflops_sustained": d.get("bf16_tflops_sustained", d["bf16_tflops"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+# ----------------------------------------------------------------- work model ----
+
+def conv_dims(w):
+    hs, ws, cs = [w.H], [w.W], [1]
+    for c, k in zip(w.conv_c, w.conv_k):
+        hs.append((hs[-1] + 2 * (k // 2) - k) // 2 + 1)
+        ws.append((ws[-1] + 2 * (k // 2) - k) // 2 + 1)
+        cs.append(c)
+    return hs, ws, cs
+
+
+def fwd_flops_per_sample(w, skip_conv1=False):
+    """Algorithmic flops of the network's own MACs (2 * Cout * Ho * Wo * Cin * k^2 per conv, 2 * in * out per FC)."""
+    hs, ws, cs = conv_dims(w)
+    f = 0
+    for l, k in enumerate(w.conv_k):
+        if skip_conv1 and l == 0:
+            continue
+        f += 2 * cs[l + 1] * hs[l + 1] * ws[l + 1] * cs[l] * k * k
+    i = cs[-1] + w.P
+    for o in list(w.fc) + [w.A + 1]:
+        f += 2 * i * o
+        i = o
+    return f
+
+
+def bwd_flops_per_sample(w):
+    """dgrad + wgrad = 2x the forward for every layer except conv1, which has no dgrad."""
+    hs, ws, cs = conv_dims(w)
+    conv1 = 2 * cs[1] * hs[1] * ws[1] * w.conv_k[0] ** 2
+    return 2 * fwd_flops_per_sample(w) - conv1
+
+
+def record_bytes(w):
+    return w.H * w.W * 2 + w.P * 4 + w.A * 4 + 4 * 4
+
+
+# --------------------------------------------------------------------- clocks ----
+
+class ClockSampler:
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, device_index):
+        self.idx = device_index
+        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.p = None
+
+    def start(self):
+        try:
+            self.p = subprocess.Popen(["nvidia-smi", "-i", str(self.idx), f"--query-gpu={self.Q}",
+                                       "--format=csv,noheader,nounits", "-lms", "100"], stdout=self.f,
+                                      stderr=subprocess.DEVNULL)
+        except OSError:
+            self.p = None
+
+    def stop(self):
+        if self.p is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.p.terminate()
+        try:
+            self.p.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.p.kill()
+        self.f.flush()
+        rows = [r.split(",") for r in open(self.f.name).read().strip().splitlines() if r.count(",") >= 8]
+        os.unlink(self.f.name)
+        if not rows:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        sm = sorted(float(r[1]) for r in rows)
+        reasons = set()
+        for r in rows:
+            for name, col in (("hw_slowdown", 5), ("hw_thermal_slowdown", 6), ("sw_thermal_slowdown", 7),
+                              ("sw_power_cap", 8)):
+                if r[col].strip().lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": sm[len(sm) // 2], "sm_max_mhz": float(rows[0][2]), "samples": len(rows),
+                "power_w_max": max(float(r[3]) for r in rows), "reasons": sorted(reasons)}
+
+
+# ------------------------------------------------------------------ our arm ------
+
+def make_learner(w, microbatch, device):
+    """Seeded parameters, a device-generated rollout, actions/log-probs from the rollout policy, buffer filled."""
+    import torch
+    from paper_2509_16434_b200 import synth
+    from paper_2509_16434_b200.learner import Learner
+    L = Learner(w, microbatch, device)
+    offs = L.model.tensors()
+    shapes = []
+    cin = 1
+    for c, k in zip(w.conv_c, w.conv_k):
+        shapes += [(c, k, k, cin), (c,)]
+        cin = c
+    i = cin + w.P
+    for o in w.fc:
+        shapes += [(o, i), (o,)]
+        i = o
+    shapes += [(w.A + 1, i), (w.A + 1,), (w.A,)]
+    theta = synth.init_params(L.model.arena, [o for o, _ in offs], shapes, w.seed)
+    L.model.load(theta)
+    roll = synth.rollout_torch(w, device, w.seed)
+    action = torch.empty((w.T, w.N, w.A), dtype=torch.float32, device=device)
+    logp = torch.empty((w.T, w.N), dtype=torch.float32, device=device)
+    for t in range(w.T):
+        a, lp, _ = L.act(roll["depth"][t], roll["proprio"][t], roll["eps"][t])
+        action[t], logp[t] = a, lp
+    # jitter the old log-probs so that both branches of the clip do work, as after the first update of an epoch
+    logp += roll["logp_jitter"]
+    roll["action"], roll["logp"] = action, logp
+    L.write_rollout(roll, action, logp)
+    torch.cuda.synchronize()
+    return L, roll
+
+
+class CallTimer:
+    """CUDA-event pairs around C-ABI calls on the current stream."""
+
+    def __init__(self):
+        self.ev = {}
+
+    def wrap(self, name, fn):
+        import torch
+
+        def inner(*a, **k):
+            s, e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            s.record()
+            r = fn(*a, **k)
+            e.record()
+            self.ev.setdefault(name, []).append((s, e))
+            return r
+        return inner
+
+    def mean_ms(self, name):
+        xs = [s.elapsed_time(e) for s, e in self.ev.get(name, [])]
+        return (sum(xs) / len(xs), len(xs)) if xs else (None, 0)
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2509_16434_b200 import binding as ppo
+    from paper_2509_16434_b200 import synth
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    device = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=device)
+    w = synth.WORKLOADS[args.workload]
+    peaks = load_peaks()
+    L, roll = make_learner(w, args.microbatch, device)
+
+    timer = CallTimer()
+    names = ["ppo_compute_gae", "ppo_shuffle_gather_minibatch", "ppo_encoder_fwd", "ppo_loss_fwd_bwd",
+             "ppo_encoder_bwd", "ppo_adam_step"]
+    originals = {n: getattr(ppo, n) for n in names}
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def one_step(seed):
+        L.train(roll["last_value"], seed=seed)
+
+    for i in range(args.warmup):
+        one_step(i)
+    barrier()
+    for n in names:
+        setattr(ppo, n, timer.wrap(n, originals[n]))
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES", "").split(",")
+    sampler = ClockSampler(vis[local] if local < len(vis) and vis[local].strip().isdigit() else local)
+    launches0 = L.launches
+    if rank == 0:
+        sampler.start()
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    t0.record()
+    for i in range(args.steps):
+        one_step(100 + i)
+    t1.record()
+    barrier()
+    clocks = sampler.stop() if rank == 0 else None
+    for n in names:
+        setattr(ppo, n, originals[n])
+    ms = t0.elapsed_time(t1)
+    status = ppo.ppo_poll_status()
+    if status != 0:
+        raise RuntimeError(f"device status {status} ({ppo.ppo_status_string(status)})")
+    launches = L.launches - launches0
+    loss = L.loss.cpu().numpy().tolist()
+
+    # ---- end to end: rollout arrives from pinned host memory every step, loss read back
+    host = {k: torch.empty(v.shape, dtype=v.dtype, pin_memory=True) for k, v in roll.items()
+            if k in ("depth", "proprio", "action", "logp", "value", "reward", "done", "last_value")}
+    for k in host:
+        host[k].copy_(roll[k])
+    stage = {k: torch.empty_like(roll[k][0]) for k in host if k != "last_value"}
+    lastv = torch.empty_like(roll["last_value"])
+    h2d = sum(v.numel() * v.element_size() for v in host.values())
+    loss_host = torch.empty(5, dtype=torch.float32, pin_memory=True)
+
+    def e2e_step(seed):
+        for t in range(w.T):
+            for k in stage:
+                stage[k].copy_(host[k][t], non_blocking=True)
+            ppo.ppo_buffer_write_step(L.buffer, t, stage["depth"], stage["proprio"], stage["action"], stage["logp"],
+                                      stage["value"], stage["reward"], stage["done"])
+        lastv.copy_(host["last_value"], non_blocking=True)
+        L.train(lastv, seed=seed)
+        loss_host.copy_(L.loss, non_blocking=True)
+        torch.cuda.current_stream().synchronize()
+
+    e2e_steps = max(1, min(args.steps, 3))
+    e2e_step(7)
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(e2e_steps):
+        e2e_step(200 + i)
+    e1.record()
+    barrier()
+    e2e_ms = e0.elapsed_time(e1)
+
+    if world > 1:
+        t = torch.tensor([ms, e2e_ms], device=device, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms, e2e_ms = t.tolist()
+    env_steps = w.M * w.epochs
+    value = world * env_steps * args.steps / (ms * 1e-3)
+    e2e_value = world * env_steps * e2e_steps / (e2e_ms * 1e-3)
+
+    if rank == 0:
+        # roofline of the dominant calls: encoder forward+backward (tensor-bound), beside the HBM-bound ones
+        rows = L.microbatch
+        fwd_ms, n_fwd = timer.mean_ms("ppo_encoder_fwd")
+        bwd_ms, _ = timer.mean_ms("ppo_encoder_bwd")
+        gat_ms, _ = timer.mean_ms("ppo_shuffle_gather_minibatch")
+        gae_ms, _ = timer.mean_ms("ppo_compute_gae")
+        adam_ms, _ = timer.mean_ms("ppo_adam_step")
+        # a trailing micro-batch may be smaller; use the true mean rows per call
+        calls_per_mb = -(-w.B // rows)
+        mean_rows = w.B / calls_per_mb
+        enc_flops = (fwd_flops_per_sample(w) + bwd_flops_per_sample(w)) * mean_rows
+        enc_tf = enc_flops / ((fwd_ms + bwd_ms) * 1e-3) / 1e12
+        peak_tf = peaks["bf16_tflops_sustained"]
+        gather_gbs = 2 * w.B * record_bytes(w) / (gat_ms * 1e-3) / 1e9
+        gae_gbs = (17 + 8) * w.M / (gae_ms * 1e-3) / 1e9
+        adam_gbs = 30 * L.model.arena / (adam_ms * 1e-3) / 1e9
+        roofline = {"bound": "tensor", "kernel": "ppo_encoder_fwd + ppo_encoder_bwd (implicit-GEMM convolutions)",
+                    "achieved": round(enc_tf, 2), "peak": peak_tf, "unit": "TFLOP/s",
+                    "frac": round(enc_tf / peak_tf, 4), "traffic": None,
+                    "peak_source": peaks["source"] + " (sustained bf16)",
+                    "ms_per_call": {"fwd": round(fwd_ms, 4), "bwd": round(bwd_ms, 4), "rows": mean_rows}}
+        others = {
+            "gather": {"bound": "hbm", "achieved": round(gather_gbs, 1), "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                       "frac": round(gather_gbs / peaks["hbm_gbs"], 4), "ms": round(gat_ms, 4)},
+            "gae_norm": {"bound": "hbm", "achieved": round(gae_gbs, 1), "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                         "frac": round(gae_gbs / peaks["hbm_gbs"], 4), "ms": round(gae_ms, 4),
+                         "note": "working set fits L2; launch-latency bound at this size"},
+            "adam": {"bound": "hbm", "achieved": round(adam_gbs, 1), "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                     "frac": round(adam_gbs / peaks["hbm_gbs"], 4), "ms": round(adam_ms, 4),
+                     "note": "working set fits L2; launch-latency bound at this size"},
+        }
+        cpu = cpu_baseline(w, roll, L) if world == 1 and not args.no_cpu_baseline else None
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": f"{w.name}: {w.N} envs x T={w.T}, depth 1x{w.H}x{w.W} fp16, conv "
+                                   f"{'-'.join(map(str, w.conv_c))}, fc {'-'.join(map(str, w.fc))}, "
+                                   f"{w.epochs} epoch(s) x {w.minibatches} minibatches",
+                       "env_steps_per_step": env_steps, "minibatch": w.B, "microbatch": L.microbatch,
+                       "l2_policy": "inputs_larger_than_l2 (buffer %.0f MB, minibatch activations %.0f MB)" % (
+                           w.M * record_bytes(w) / 1e6, L.model.workspace.numel() / 1e6),
+                       "parallelism": "replicas only" if world > 1 else "single GPU"},
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": 20,
+                    "steps": e2e_steps, "ms_per_step": e2e_ms / e2e_steps},
+            "gpu_launches": launches, "clocks": clocks, "roofline": roofline, "roofline_other_kernels": others,
+            "cpu_baseline": cpu, "loss_last_minibatch": loss,
+        }
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+# ---------------------------------------------------------------- CPU baseline ----
+
+def oracle_sample_step(w, fields, theta, n_samples):
+    """The oracle's learner step on a bounded sample: GAE + normalisation at full size, then one minibatch of
+    n_samples rows (permutation, gather, forward, loss, backward, Adam).  Returns seconds and samples trained."""
+    from oracle import oracle as orc
+    md = orc.ModelDesc(w.H, w.W, tuple(w.conv_c), tuple(w.conv_k), tuple(w.fc), w.P, w.A)
+    t0 = time.perf_counter()
+    adv, ret = orc.gae(fields["reward"], fields["value"], fields["done"], fields["last_value"], w.gamma, w.lam)
+    adv, _, _ = orc.adv_normalize(adv)
+    t_gae = time.perf_counter() - t0
+    t0 = time.perf_counter()
+    idx = orc.perm(w.seed, 0, w.M, 0, n_samples)
+    tt, nn = np.divmod(idx.astype(np.int64), w.N)
+    depth = fields["depth_rows"]            # the sampled rows' frames, gathered on the device side of the bench
+    g = {"proprio": fields["proprio"][tt, nn], "action": fields["action"][tt, nn], "logp": fields["logp"][tt, nn],
+         "adv": adv[tt, nn], "ret": ret[tt, nn]}
+    _, out, grad, _, _ = orc.total_loss_and_grad(md, theta, depth, g["proprio"], g["action"], g["logp"], g["adv"],
+                                                 g["ret"], w.clip, 0.5, 0.01)
+    th = np.asarray(theta, np.float64).copy()
+    orc.adam(th, np.zeros_like(th), np.zeros_like(th), grad, 3e-4, 0.9, 0.999, 1e-8, 1)
+    t_mb = time.perf_counter() - t0
+    return t_gae, t_mb, out
+
+
+def cpu_baseline(w, roll, L, n_samples=None):
+    """Times the oracle, as it stands, on this machine's host cores over a bounded sample of the same workload."""
+    from oracle import oracle as orc
+    import torch
+    n_samples = n_samples or (256 if w.H * w.W <= 64 * 64 else 48 if w.H * w.W <= 120 * 160 else 12)
+    idx = orc.perm(w.seed, 0, w.M, 0, n_samples).astype(np.int64)
+    flat = roll["depth"].view(w.M, w.H, w.W)
+    fields = {k: roll[k].cpu().numpy() for k in ("proprio", "action", "logp", "value", "reward", "done",
+                                                 "last_value")}
+    fields["depth_rows"] = flat[torch.as_tensor(idx, device=flat.device)].cpu().numpy()
+    theta = L.model.master.cpu().numpy()
+    t_gae, t_mb, _ = oracle_sample_step(w, fields, theta, n_samples)
+    # whole step = GAE once + M*E sample-passes at the measured per-sample minibatch cost
+    per_step = t_gae + t_mb / n_samples * w.M * w.epochs
+    return {"value": w.M * w.epochs / per_step, "unit": UNIT, "cores": orc.num_threads(), "kind": "oracle",
+            "sample": f"GAE+normalisation at full size ({w.M} env-steps, {t_gae:.3f} s) + one minibatch of "
+                      f"{n_samples} rows gather/fwd/loss/bwd/Adam ({t_mb:.2f} s), extrapolated linearly to "
+                      f"{w.M * w.epochs} sample-passes"}
+
+
+def run_reference(args):
+    """The reference arm of this build is the CPU oracle: timed as it stands on the host cores."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import oracle as orc
+    from paper_2509_16434_b200 import synth
+    w = synth.WORKLOADS[args.workload]
+    n_samples = 256 if w.H * w.W <= 64 * 64 else 32 if w.H * w.W <= 120 * 160 else 8
+    # a host-generated slice of the workload: all small fields at full size, frames only for the sampled rows
+    small = w.scaled(w.N, H=2, W=2)
+    roll = synth.rollout_numpy(small, w.seed)
+    g = np.random.Generator(np.random.Philox(key=[w.seed, 1234]))
+    depth = g.uniform(0.1, 2.0, (n_samples, w.H, w.W)).astype(np.float16)
+    depth[g.random(depth.shape) < 0.1] = 0
+    md = orc.ModelDesc(w.H, w.W, tuple(w.conv_c), tuple(w.conv_k), tuple(w.fc), w.P, w.A)
+    lay = orc.param_layout(md)
+    theta = synth.init_params(lay.total, lay.offsets, lay.shapes, w.seed)
+    fields = {k: roll[k] for k in ("proprio", "value", "reward", "done", "last_value")}
+    fields["action"] = roll["eps"]
+    fields["logp"] = (-0.5 * (roll["eps"].astype(np.float64) ** 2).sum(-1) - 0.5 * w.A * np.log(2 * np.pi)
+                      + roll["logp_jitter"]).astype(np.float32)
+    fields["depth_rows"] = depth
+    times = []
+    for i in range(args.warmup + args.steps):
+        t_gae, t_mb, _ = oracle_sample_step(w, fields, theta, n_samples)
+        if i >= args.warmup:
+            times.append(t_gae + t_mb / n_samples * w.M * w.epochs)
+    per_step = float(np.mean(times))
+    value = w.M * w.epochs / per_step
+    sample = (f"per step: GAE+normalisation at full size + one minibatch of {n_samples} rows "
+              f"(gather/fwd/loss/bwd/Adam), extrapolated linearly to {w.M * w.epochs} sample-passes")
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": int(args.gpus),
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": per_step * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": f"{w.name}: {w.N} envs x T={w.T}, depth 1x{w.H}x{w.W}", "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": orc.num_threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="cfg2")
+    ap.add_argument("--microbatch", type=int, default=512)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

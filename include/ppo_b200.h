@@ -1,0 +1,235 @@
+/*
+ * ppo_b200.h -- C ABI of libppo_b200.so: one PPO learner step over an on-device
+ * rollout buffer of depth-image observations, for NVIDIA B200 (sm_100a).
+ *
+ * The library is the learner side of a disaggregated simulator/learner split
+ * (Section III-B, Algorithm 2): it keeps the trajectory buffer D of one horizon
+ * on the learner GPU (D <- {} ; D <- D U {(obs, actions, rew, done)}) and runs
+ * TrainPPO(pi, D) on it.
+ *
+ * Conventions
+ *  - Every function that can fail returns an int status (PPO_OK == 0).  Argument
+ *    and state errors are found on the host and nothing is launched.  No function
+ *    throws, exits or traps the device.
+ *  - "dev" pointers are CUDA device pointers owned by the caller.  The library
+ *    never allocates or frees device memory; size queries say how much the caller
+ *    must provide.  *_create / *_alloc allocate only small host-side handles.
+ *  - `stream` is a cudaStream_t passed as void*.  Calls only enqueue work on it and
+ *    do not synchronise (ppo_poll_status is the exception).
+ *  - Device pointers must be 16-byte aligned; storage handed to ppo_buffer_alloc
+ *    and ppo_model_bind's workspace must be 256-byte aligned.
+ *  - Samples of the buffer are numbered time-major: s = t * N + n.
+ *  - Not thread-safe per handle; different handles may be used from different threads.
+ */
+#ifndef PPO_B200_H
+#define PPO_B200_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum {
+    PPO_OK = 0,
+    PPO_ERR_INVALID_ARG = 1, /* NULL pointer, value out of range */
+    PPO_ERR_SHAPE = 2,       /* sizes inconsistent with the descriptor */
+    PPO_ERR_ALIGN = 3,       /* pointer not aligned as required */
+    PPO_ERR_STATE = 4,       /* call out of order (e.g. gather before GAE) */
+    PPO_ERR_CUDA = 5,        /* a CUDA runtime call failed */
+    PPO_ERR_TIMEOUT = 6,     /* a bounded device-side wait gave up */
+    PPO_ERR_UNSUPPORTED = 7  /* shape outside what the kernels implement */
+};
+
+const char *ppo_status_string(int status);
+
+/* ------------------------------------------------------------------ buffer -- */
+
+/* Shape of the trajectory buffer D (Algorithm 2): N envs, horizon T, depth frames
+ * H x W (fp16), P proprioceptive floats and A action floats per env-step. */
+typedef struct {
+    int32_t N, T, H, W, P, A;
+} ppo_buffer_desc;
+
+typedef struct ppo_buffer ppo_buffer;
+
+/* Slabs of the buffer, each time-major [T][N][...] and 256-byte aligned. */
+enum {
+    PPO_FIELD_DEPTH = 0,  /* fp16  [T][N][H][W] */
+    PPO_FIELD_PROPRIO,    /* fp32  [T][N][P]    */
+    PPO_FIELD_ACTION,     /* fp32  [T][N][A]    */
+    PPO_FIELD_LOGP,       /* fp32  [T][N]  log-prob of the action under the rollout policy */
+    PPO_FIELD_VALUE,      /* fp32  [T][N]  value estimate at rollout time */
+    PPO_FIELD_REWARD,     /* fp32  [T][N]  */
+    PPO_FIELD_DONE,       /* uint8 [T][N]  returned by the same env step as the reward */
+    PPO_FIELD_ADV,        /* fp32  [T][N]  written by ppo_compute_gae */
+    PPO_FIELD_RET,        /* fp32  [T][N]  written by ppo_compute_gae */
+    PPO_FIELD_SCRATCH,    /* internal reduction scratch */
+    PPO_NUM_FIELDS
+};
+
+/* Bytes of one slab (unpadded) for a depth element of `depth_elem_bytes` (the kernels
+ * use 2; 4 reproduces the fp32 sizing example of Section III-B: 512 envs x 320x240 x
+ * 16 steps = 2.5 GB).  Returns 0 for a bad descriptor or field. */
+size_t ppo_buffer_field_bytes(const ppo_buffer_desc *desc, int field, int depth_elem_bytes);
+
+/* Total device bytes ppo_buffer_alloc needs (fp16 depth, every slab padded to 256 B).
+ * Returns 0 for a bad descriptor. */
+size_t ppo_buffer_bytes(const ppo_buffer_desc *desc);
+
+/* D <- {} (Algorithm 2): carves the slabs out of caller-owned device storage of at
+ * least ppo_buffer_bytes(desc) bytes, 256-byte aligned.  The storage must outlive the
+ * handle.  Nothing is written to the device. */
+int ppo_buffer_alloc(const ppo_buffer_desc *desc, void *dev_storage, size_t bytes, ppo_buffer **out);
+
+/* Frees the host handle only. */
+int ppo_buffer_free(ppo_buffer *buf);
+
+/* Device address of a slab (NULL on error); for callers that fill or read slabs directly. */
+void *ppo_buffer_field_ptr(const ppo_buffer *buf, int field);
+
+/* D <- D U {(obs, actions, rew, done)} for step t in [0, T) (Algorithm 2): copies one
+ * step of all N envs from caller device arrays into slab row t.
+ *   depth_f16 [N][H][W] fp16, proprio [N][P], action [N][A], logp [N], value [N],
+ *   reward [N] (fp32), done [N] uint8.
+ * Invalidates advantages computed earlier.  Errors: t outside [0,T) -> INVALID_ARG. */
+int ppo_buffer_write_step(ppo_buffer *buf, int t, const void *dev_depth_f16, const float *dev_proprio,
+                          const float *dev_action, const float *dev_logp, const float *dev_value,
+                          const float *dev_reward, const uint8_t *dev_done, void *stream);
+
+/* First stage of TrainPPO (Algorithm 2): generalised advantage estimation per env by a
+ * reverse scan over t,
+ *   delta_t = r_t + gamma V_{t+1} (1 - d_t) - V_t,  A_t = delta_t + gamma lambda (1 - d_t) A_{t+1},
+ *   R_t = A_t + V_t,  V_T = dev_last_value[n],  A_T = 0,
+ * written to the ADV and RET slabs; then, if normalize != 0, the advantages of the whole
+ * buffer are replaced by (A - mean) / (std + 1e-8) with the unbiased (M-1) standard
+ * deviation.  dev_stats_out (may be NULL) receives {mean, std} of the raw advantages as
+ * fp32 when normalize != 0.  fp32 arithmetic, fp64 accumulation of the moments. */
+int ppo_compute_gae(ppo_buffer *buf, const float *dev_last_value, float gamma, float lambda, int normalize,
+                    float *dev_stats_out, void *stream);
+
+/* One gathered minibatch: caller-allocated device arrays of B rows. */
+typedef struct {
+    void *depth_f16;  /* [B][H][W] fp16 */
+    float *proprio;   /* [B][P] */
+    float *action;    /* [B][A] */
+    float *logp_old;  /* [B] */
+    float *value_old; /* [B] */
+    float *adv;       /* [B] */
+    float *ret;       /* [B] */
+    uint32_t *index;  /* [B] sample numbers s of the rows; may be NULL */
+    int32_t B;
+} ppo_minibatch;
+
+/* Minibatch mb_index of num_minibatches for (seed, epoch): row j receives an exact copy
+ * of sample s = pi(mb_index * B + j), where pi is the seeded bijection on [0, M), M = N*T:
+ * a 6-round balanced Feistel network on 2h bits, h = max(1, ceil(ceil_log2(M) / 2)), with
+ * cycle walking; round function mix32(R ^ key_j) & (2^h - 1); all arithmetic uint32.
+ *   mix32(x): x ^= x>>16; x *= 0x9E3779B9; x ^= x>>15; x *= 0x6A09E667; x ^= x>>16
+ *   key_j = mix32(lo32(seed) ^ mix32(hi32(seed) + 0x9E3779B9*(j+1)) ^ mix32(epoch + 0xBB67AE85*(j+1)))
+ * Requires M % num_minibatches == 0 and out->B == M / num_minibatches (else SHAPE), and
+ * a prior ppo_compute_gae since the last write_step (else STATE). */
+int ppo_shuffle_gather_minibatch(const ppo_buffer *buf, uint64_t seed, uint32_t epoch, int mb_index,
+                                 int num_minibatches, const ppo_minibatch *out, void *stream);
+
+/* ------------------------------------------------------------------- model -- */
+
+#define PPO_MAX_CONV 8
+#define PPO_MAX_FC 4
+
+/* Policy/value network (Section III-C: CNN with ReLU on the depth image, joined with
+ * proprioception, fully connected layers).  Conv l: k x k cross-correlation, stride 2,
+ * zero padding k/2, ReLU; global average pool; concat [pooled, proprio]; hidden FC layers
+ * with ReLU; one linear head giving the Gaussian mean (A) and the value (1); log-sigma is a
+ * free A-vector.  Channel counts of conv layers >= 1 and FC widths must be multiples of 8. */
+typedef struct {
+    int32_t H, W;
+    int32_t n_conv;
+    int32_t conv_c[PPO_MAX_CONV];
+    int32_t conv_k[PPO_MAX_CONV];
+    int32_t n_fc;
+    int32_t fc[PPO_MAX_FC];
+    int32_t P, A;
+} ppo_model_desc;
+
+typedef struct ppo_model ppo_model;
+
+int ppo_model_create(const ppo_model_desc *desc, ppo_model **out);
+int ppo_model_destroy(ppo_model *m);
+
+/* Parameter vector ("arena") layout: tensors in the order conv W_l [Cout][k][k][Cin],
+ * conv b_l [Cout], ..., fc W [out][in], fc b [out], ..., head W [A+1][hid] (rows 0..A-1
+ * mean, row A value), head b [A+1], log-sigma [A]; every tensor starts at a multiple of 64
+ * elements; gaps are zero and stay zero.  The same offsets index master, shadow, gradient
+ * and Adam moment arrays. */
+size_t ppo_model_param_count(const ppo_model *m); /* sum of tensor sizes, without gaps */
+size_t ppo_model_arena_elems(const ppo_model *m); /* length of the arrays, with gaps */
+int ppo_model_num_tensors(const ppo_model *m);
+int ppo_model_tensor_info(const ppo_model *m, int index, int64_t *offset, int64_t *size);
+
+/* Device bytes of workspace for forward+backward of up to `microbatch` rows at a time. */
+size_t ppo_model_workspace_bytes(const ppo_model *m, int microbatch);
+
+/* Attaches caller-owned device arrays: master/grad/adam_m/adam_v fp32 [arena_elems],
+ * shadow_bf16 bf16 [arena_elems] (weights as the GEMMs read them; refreshed by
+ * ppo_adam_step and ppo_model_sync_shadow), workspace of ws_bytes >=
+ * ppo_model_workspace_bytes(m, microbatch). */
+int ppo_model_bind(ppo_model *m, float *dev_master, void *dev_shadow_bf16, float *dev_grad, float *dev_adam_m,
+                   float *dev_adam_v, void *dev_workspace, size_t ws_bytes, int microbatch);
+
+/* shadow <- bf16(master) (round to nearest even); call after writing master from outside. */
+int ppo_model_sync_shadow(ppo_model *m, void *stream);
+
+/* Forward of rows [row0, row0+rows) of a minibatch (rows <= bound microbatch): writes the
+ * Gaussian mean dev_mean [rows][A] and the value dev_value [rows] (fp32) and keeps the
+ * activations in the workspace for ppo_encoder_bwd.  bf16 operands (weights from the
+ * shadow, activations rounded to bf16 between layers), fp32 accumulation; the depth
+ * frame enters as fp16. */
+int ppo_encoder_fwd(ppo_model *m, const ppo_minibatch *mb, int row0, int rows, float *dev_mean, float *dev_value,
+                    void *stream);
+
+/* PPO-clip loss of rows [row0, row0+rows) fused with its gradient (TrainPPO, Algorithm 2):
+ *   z = (a - mu)/sigma, sigma = exp(logsigma);  logp = sum_j [-z_j^2/2 - logsigma_j - ln(2 pi)/2]
+ *   r = exp(logp - logp_old);  s = min(r Adv, clamp(r, 1-clip, 1+clip) Adv)
+ *   L = -mean(s) + vf_coef mean((V - R)^2) - ent_coef H,  H = sum_j logsigma_j + (A/2)(1 + ln 2 pi)
+ * with means over B_total rows (so micro-batches add up to the minibatch).  Writes
+ * dL/dmu to dev_dmean [rows][A] and dL/dV to dev_dvalue [rows]; ADDS dL/dlogsigma into the
+ * log-sigma slot of the bound gradient array and ADDS this call's share of
+ * {L_pi, L_V, H, approx_kl = mean(logp_old - logp), clip_fraction} into dev_loss_out[5]
+ * (the caller zeroes both at the start of a minibatch).  At a tie of the min the unclipped
+ * branch is taken. */
+int ppo_loss_fwd_bwd(ppo_model *m, const ppo_minibatch *mb, int row0, int rows, int B_total, const float *dev_mean,
+                     const float *dev_value, float clip, float vf_coef, float ent_coef, float *dev_loss_out,
+                     float *dev_dmean, float *dev_dvalue, void *stream);
+
+/* Backward of the rows of the latest ppo_encoder_fwd (same row0/rows, else STATE): adds
+ * (accumulate != 0) or writes (accumulate == 0, the log-sigma slot is left as it is)
+ * dL/dtheta into the bound gradient array, with respect to the fp32 master (straight
+ * through the bf16 rounding). */
+int ppo_encoder_bwd(ppo_model *m, const ppo_minibatch *mb, int row0, int rows, const float *dev_dmean,
+                    const float *dev_dvalue, int accumulate, void *stream);
+
+/* Zeroes the bound gradient array (start of a minibatch). */
+int ppo_model_zero_grad(ppo_model *m, void *stream);
+
+/* Adam over the whole arena in one pass (bias-corrected, eps outside the square root, no
+ * weight decay), step >= 1:  m <- b1 m + (1-b1) g;  v <- b2 v + (1-b2) g^2;
+ * theta <- theta - lr (m/(1-b1^step)) / (sqrt(v/(1-b2^step)) + eps); shadow <- bf16(theta). */
+int ppo_adam_step(ppo_model *m, float lr, float beta1, float beta2, float eps, int64_t step, void *stream);
+
+/* Rollout-time action of the policy (Algorithm 2, actions <- pi(obs)) given the mean from
+ * ppo_encoder_fwd and caller-supplied standard-normal noise dev_eps [rows][A]:
+ * action = mu + exp(logsigma) * eps, logp = its log-density.  Outputs fp32 [rows][A], [rows]. */
+int ppo_policy_sample(const ppo_model *m, int rows, const float *dev_mean, const float *dev_eps, float *dev_action,
+                      float *dev_logp, void *stream);
+
+/* Synchronises `stream`, then returns the first error a kernel recorded in the library's
+ * device status word since the last poll (PPO_OK if none), or PPO_ERR_CUDA if the stream
+ * reports a CUDA error. */
+int ppo_poll_status(void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PPO_B200_H */

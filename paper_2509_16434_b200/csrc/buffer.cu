@@ -1,0 +1,498 @@
+// Rollout buffer D on the learner GPU (Algorithm 2): slab carving, write_step, GAE with
+// advantage normalisation, and the seeded permutation gather.
+#include <new>
+
+#include "common.cuh"
+
+// ------------------------------------------------------------------ status ----
+
+static __device__ int32_t g_ppo_status;
+
+int32_t *ppo_device_status_ptr() {
+    static int32_t *ptrs[64] = {nullptr};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    if (!ptrs[dev]) {
+        void *p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_ppo_status) != cudaSuccess) return nullptr;
+        ptrs[dev] = static_cast<int32_t *>(p);
+    }
+    return ptrs[dev];
+}
+
+int ppo_num_sms() {
+    static int sms[64] = {0};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 148;
+    if (!sms[dev]) {
+        int n = 0;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
+        sms[dev] = n;
+    }
+    return sms[dev];
+}
+
+extern "C" const char *ppo_status_string(int s) {
+    switch (s) {
+        case PPO_OK: return "ok";
+        case PPO_ERR_INVALID_ARG: return "invalid argument";
+        case PPO_ERR_SHAPE: return "shape mismatch";
+        case PPO_ERR_ALIGN: return "misaligned pointer";
+        case PPO_ERR_STATE: return "call out of order";
+        case PPO_ERR_CUDA: return "CUDA error";
+        case PPO_ERR_TIMEOUT: return "device-side wait timed out";
+        case PPO_ERR_UNSUPPORTED: return "unsupported shape";
+        default: return "unknown status";
+    }
+}
+
+extern "C" int ppo_poll_status(void *stream) {
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    int32_t *p = ppo_device_status_ptr();
+    if (!p) return PPO_ERR_CUDA;
+    int32_t host = 0;
+    if (cudaMemcpyAsync(&host, p, sizeof(host), cudaMemcpyDeviceToHost, st) != cudaSuccess) return PPO_ERR_CUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return PPO_ERR_CUDA;
+    if (host != 0) {
+        if (cudaMemsetAsync(p, 0, sizeof(host), st) != cudaSuccess) return PPO_ERR_CUDA;
+        if (cudaStreamSynchronize(st) != cudaSuccess) return PPO_ERR_CUDA;
+    }
+    return host;
+}
+
+// ------------------------------------------------------------------ layout ----
+
+static const int kMaxGaeBlocks = 4096;
+
+static bool desc_ok(const ppo_buffer_desc *d) {
+    return d && d->N > 0 && d->T > 0 && d->H > 0 && d->W > 0 && d->P > 0 && d->A > 0 &&
+           (long long)d->N * d->T < (1ll << 31);
+}
+
+static size_t field_bytes(const ppo_buffer_desc *d, int field, int depth_elem) {
+    size_t M = (size_t)d->N * d->T;
+    switch (field) {
+        case PPO_FIELD_DEPTH: return M * d->H * d->W * (size_t)depth_elem;
+        case PPO_FIELD_PROPRIO: return M * d->P * 4;
+        case PPO_FIELD_ACTION: return M * d->A * 4;
+        case PPO_FIELD_LOGP:
+        case PPO_FIELD_VALUE:
+        case PPO_FIELD_REWARD:
+        case PPO_FIELD_ADV:
+        case PPO_FIELD_RET: return M * 4;
+        case PPO_FIELD_DONE: return M;
+        case PPO_FIELD_SCRATCH: return (size_t)kMaxGaeBlocks * 2 * sizeof(double);
+        default: return 0;
+    }
+}
+
+extern "C" size_t ppo_buffer_field_bytes(const ppo_buffer_desc *d, int field, int depth_elem_bytes) {
+    if (!desc_ok(d) || field < 0 || field >= PPO_NUM_FIELDS) return 0;
+    if (depth_elem_bytes != 2 && depth_elem_bytes != 4) return 0;
+    return field_bytes(d, field, depth_elem_bytes);
+}
+
+extern "C" size_t ppo_buffer_bytes(const ppo_buffer_desc *d) {
+    if (!desc_ok(d)) return 0;
+    size_t total = 0;
+    for (int f = 0; f < PPO_NUM_FIELDS; ++f) total += ppo_align_up(field_bytes(d, f, 2), 256);
+    return total;
+}
+
+extern "C" int ppo_buffer_alloc(const ppo_buffer_desc *d, void *dev_storage, size_t bytes, ppo_buffer **out) {
+    if (!out) return PPO_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (!desc_ok(d) || !dev_storage) return PPO_ERR_INVALID_ARG;
+    if (!ppo_aligned(dev_storage, 256)) return PPO_ERR_ALIGN;
+    if (bytes < ppo_buffer_bytes(d)) return PPO_ERR_SHAPE;
+    ppo_buffer *b = new (std::nothrow) ppo_buffer();
+    if (!b) return PPO_ERR_INVALID_ARG;
+    b->d = *d;
+    b->base = static_cast<char *>(dev_storage);
+    b->bytes = bytes;
+    size_t off = 0;
+    for (int f = 0; f < PPO_NUM_FIELDS; ++f) {
+        b->field_off[f] = off;
+        off += ppo_align_up(field_bytes(d, f, 2), 256);
+    }
+    b->gae_valid = false;
+    b->gae_blocks = 0;
+    *out = b;
+    return PPO_OK;
+}
+
+extern "C" int ppo_buffer_free(ppo_buffer *b) {
+    if (!b) return PPO_ERR_INVALID_ARG;
+    delete b;
+    return PPO_OK;
+}
+
+extern "C" void *ppo_buffer_field_ptr(const ppo_buffer *b, int field) {
+    if (!b || field < 0 || field >= PPO_NUM_FIELDS) return nullptr;
+    return b->base + b->field_off[field];
+}
+
+template <typename T>
+static T *slab(const ppo_buffer *b, int field) {
+    return reinterpret_cast<T *>(b->base + b->field_off[field]);
+}
+
+// -------------------------------------------------------------- write_step ----
+
+struct CopySeg {
+    const char *src;
+    char *dst;
+    unsigned long long bytes;
+    int vec;  // 16 when both ends and the size allow 128-bit accesses, else 1
+};
+struct CopySegs {
+    CopySeg s[7];
+};
+
+// blockIdx.y selects the segment; blocks stride over it with 128-bit (or byte) accesses.
+__global__ void __launch_bounds__(256) write_step_kernel(CopySegs segs) {
+    const CopySeg sg = segs.s[blockIdx.y];
+    const unsigned long long tid = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x;
+    const unsigned long long nth = (unsigned long long)gridDim.x * blockDim.x;
+    if (sg.vec == 16) {
+        const uint4 *s = reinterpret_cast<const uint4 *>(sg.src);
+        uint4 *d = reinterpret_cast<uint4 *>(sg.dst);
+        const unsigned long long n = sg.bytes >> 4;
+        unsigned long long i = tid;
+        for (; i + 3 * nth < n; i += 4 * nth) {
+            uint4 a = __ldcs(s + i), b = __ldcs(s + i + nth), c = __ldcs(s + i + 2 * nth), e = __ldcs(s + i + 3 * nth);
+            d[i] = a;
+            d[i + nth] = b;
+            d[i + 2 * nth] = c;
+            d[i + 3 * nth] = e;
+        }
+        for (; i < n; i += nth) d[i] = __ldcs(s + i);
+    } else {
+        for (unsigned long long i = tid; i < sg.bytes; i += nth) sg.dst[i] = sg.src[i];
+    }
+}
+
+extern "C" int ppo_buffer_write_step(ppo_buffer *b, int t, const void *depth, const float *proprio,
+                                     const float *action, const float *logp, const float *value, const float *reward,
+                                     const uint8_t *done, void *stream) {
+    if (!b || !depth || !proprio || !action || !logp || !value || !reward || !done) return PPO_ERR_INVALID_ARG;
+    if (t < 0 || t >= b->d.T) return PPO_ERR_INVALID_ARG;
+    const ppo_buffer_desc &d = b->d;
+    const size_t N = d.N;
+    const void *srcs[7] = {depth, proprio, action, logp, value, reward, done};
+    const int fields[7] = {PPO_FIELD_DEPTH, PPO_FIELD_PROPRIO, PPO_FIELD_ACTION, PPO_FIELD_LOGP,
+                           PPO_FIELD_VALUE, PPO_FIELD_REWARD, PPO_FIELD_DONE};
+    const size_t per_env[7] = {(size_t)d.H * d.W * 2, (size_t)d.P * 4, (size_t)d.A * 4, 4, 4, 4, 1};
+    CopySegs segs;
+    for (int i = 0; i < 7; ++i) {
+        size_t bytes = N * per_env[i];
+        char *dst = b->base + b->field_off[fields[i]] + (size_t)t * bytes;
+        segs.s[i].src = static_cast<const char *>(srcs[i]);
+        segs.s[i].dst = dst;
+        segs.s[i].bytes = bytes;
+        segs.s[i].vec = (ppo_aligned(srcs[i], 16) && ppo_aligned(dst, 16) && bytes % 16 == 0) ? 16 : 1;
+    }
+    b->gae_valid = false;
+    // enough blocks to cover the depth segment with ~4 x 16 B per thread, capped at a few waves
+    long long units = (long long)(segs.s[0].bytes / 16 / 4 / 256) + 1;
+    int gx = (int)(units < (long long)ppo_num_sms() * 16 ? units : (long long)ppo_num_sms() * 16);
+    dim3 grid(gx, 7);
+    write_step_kernel<<<grid, 256, 0, static_cast<cudaStream_t>(stream)>>>(segs);
+    PPO_LAUNCH_CHECK();
+    return PPO_OK;
+}
+
+// --------------------------------------------------------------------- GAE ----
+
+__device__ __forceinline__ double warp_sum(double v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_down_sync(0xffffffffu, v, o);
+    return v;
+}
+
+// Sum over the block; the result is valid in thread 0.  Fixed reduction order.
+__device__ __forceinline__ double block_sum(double v, double *sh /*[32]*/) {
+    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+    v = warp_sum(v);
+    __syncthreads();
+    if (lane == 0) sh[wid] = v;
+    __syncthreads();
+    if (wid == 0) {
+        v = (lane < (int)((blockDim.x + 31) >> 5)) ? sh[lane] : 0.0;
+        v = warp_sum(v);
+    }
+    return v;
+}
+
+// One thread per env: reverse scan over t with the loads of UNR steps issued together.
+// Reads r, V (fp32) and d (u8), writes A and R: 17 B per env-step.  Each block leaves the
+// fp64 sums of A and A^2 of its envs in partials[2*blockIdx.x .. +1].
+template <int UNR>
+__global__ void __launch_bounds__(128) gae_scan_kernel(const float *__restrict__ reward,
+                                                       const float *__restrict__ value,
+                                                       const uint8_t *__restrict__ done,
+                                                       const float *__restrict__ last_value, float gamma,
+                                                       float gamma_lambda, float *__restrict__ adv,
+                                                       float *__restrict__ ret, int T, int N,
+                                                       double *__restrict__ partials) {
+    __shared__ double sh[32];
+    const int n = blockIdx.x * blockDim.x + threadIdx.x;
+    double s1 = 0.0, s2 = 0.0;
+    if (n < N) {
+        float v_next = last_value[n];
+        float a_next = 0.f;
+        int t = T - 1;
+        for (; t >= UNR - 1; t -= UNR) {
+            float r[UNR], v[UNR];
+            uint8_t d[UNR];
+#pragma unroll
+            for (int u = 0; u < UNR; ++u) {
+                size_t i = (size_t)(t - u) * N + n;
+                r[u] = __ldcs(reward + i);
+                v[u] = __ldcs(value + i);
+                d[u] = __ldcs(done + i);
+            }
+#pragma unroll
+            for (int u = 0; u < UNR; ++u) {
+                size_t i = (size_t)(t - u) * N + n;
+                float nd = d[u] ? 0.f : 1.f;
+                float delta = r[u] + gamma * v_next * nd - v[u];
+                float a = delta + gamma_lambda * nd * a_next;
+                __stcs(adv + i, a);
+                __stcs(ret + i, a + v[u]);
+                s1 += (double)a;
+                s2 += (double)a * (double)a;
+                v_next = v[u];
+                a_next = a;
+            }
+        }
+        for (; t >= 0; --t) {
+            size_t i = (size_t)t * N + n;
+            float r = reward[i], v = value[i];
+            float nd = done[i] ? 0.f : 1.f;
+            float delta = r + gamma * v_next * nd - v;
+            float a = delta + gamma_lambda * nd * a_next;
+            adv[i] = a;
+            ret[i] = a + v;
+            s1 += (double)a;
+            s2 += (double)a * (double)a;
+            v_next = v;
+            a_next = a;
+        }
+    }
+    s1 = block_sum(s1, sh);
+    s2 = block_sum(s2, sh);
+    if (threadIdx.x == 0) {
+        partials[2 * blockIdx.x] = s1;
+        partials[2 * blockIdx.x + 1] = s2;
+    }
+}
+
+// Every block reduces the per-block partial sums in the same fixed order (deterministic),
+// then normalises its share of the advantages in place with 128-bit accesses.
+__global__ void __launch_bounds__(256) adv_normalize_kernel(float *__restrict__ adv, long long M,
+                                                            const double *__restrict__ partials, int nparts,
+                                                            float *__restrict__ stats_out) {
+    __shared__ double sh[32];
+    __shared__ float s_mean, s_inv;
+    double s1 = 0.0, s2 = 0.0;
+    for (int i = threadIdx.x; i < nparts; i += blockDim.x) {
+        s1 += partials[2 * i];
+        s2 += partials[2 * i + 1];
+    }
+    s1 = block_sum(s1, sh);
+    s2 = block_sum(s2, sh);
+    if (threadIdx.x == 0) {
+        double mean = s1 / (double)M;
+        double var = (M > 1) ? (s2 - s1 * mean) / (double)(M - 1) : 0.0;
+        double sd = sqrt(var > 0.0 ? var : 0.0);
+        s_mean = (float)mean;
+        s_inv = (float)(1.0 / (sd + 1e-8));
+        if (blockIdx.x == 0 && stats_out) {
+            stats_out[0] = (float)mean;
+            stats_out[1] = (float)sd;
+        }
+    }
+    __syncthreads();
+    const float mean = s_mean, inv = s_inv;
+    const long long tid = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    const long long nth = (long long)gridDim.x * blockDim.x;
+    const long long n4 = M >> 2;
+    float4 *a4 = reinterpret_cast<float4 *>(adv);
+    for (long long i = tid; i < n4; i += nth) {
+        float4 x = a4[i];
+        x.x = (x.x - mean) * inv;
+        x.y = (x.y - mean) * inv;
+        x.z = (x.z - mean) * inv;
+        x.w = (x.w - mean) * inv;
+        a4[i] = x;
+    }
+    for (long long i = (n4 << 2) + tid; i < M; i += nth) adv[i] = (adv[i] - mean) * inv;
+}
+
+extern "C" int ppo_compute_gae(ppo_buffer *b, const float *last_value, float gamma, float lambda, int normalize,
+                               float *stats_out, void *stream) {
+    if (!b || !last_value) return PPO_ERR_INVALID_ARG;
+    if (!(gamma >= 0.f && gamma <= 1.f) || !(lambda >= 0.f && lambda <= 1.f)) return PPO_ERR_INVALID_ARG;
+    const int N = b->d.N, T = b->d.T;
+    const int threads = 128;
+    const int blocks = ppo_cdiv(N, threads);
+    if (blocks > kMaxGaeBlocks) return PPO_ERR_UNSUPPORTED;  // N <= 524288 envs
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    double *partials = slab<double>(b, PPO_FIELD_SCRATCH);
+    gae_scan_kernel<8><<<blocks, threads, 0, st>>>(slab<float>(b, PPO_FIELD_REWARD), slab<float>(b, PPO_FIELD_VALUE),
+                                                   slab<uint8_t>(b, PPO_FIELD_DONE), last_value, gamma,
+                                                   gamma * lambda, slab<float>(b, PPO_FIELD_ADV),
+                                                   slab<float>(b, PPO_FIELD_RET), T, N, partials);
+    PPO_LAUNCH_CHECK();
+    if (normalize) {
+        const long long M = (long long)N * T;
+        int nb = ppo_cdiv(M, 256 * 4 * 4);
+        int cap = ppo_num_sms() * 8;
+        if (nb > cap) nb = cap;
+        if (nb < 1) nb = 1;
+        adv_normalize_kernel<<<nb, 256, 0, st>>>(slab<float>(b, PPO_FIELD_ADV), M, partials, blocks, stats_out);
+        PPO_LAUNCH_CHECK();
+    }
+    b->gae_valid = true;
+    b->gae_blocks = blocks;
+    return PPO_OK;
+}
+
+// ------------------------------------------------------------------ gather ----
+
+struct PermParams {
+    uint32_t key[6];
+    uint32_t M;
+    int h;
+    uint32_t mask;
+};
+
+__host__ __device__ __forceinline__ uint32_t perm_mix(uint32_t x) {
+    x ^= x >> 16;
+    x *= 0x9E3779B9u;
+    x ^= x >> 15;
+    x *= 0x6A09E667u;
+    x ^= x >> 16;
+    return x;
+}
+
+static PermParams make_perm(uint64_t seed, uint32_t epoch, uint32_t M) {
+    PermParams p;
+    const uint32_t lo = (uint32_t)seed, hi = (uint32_t)(seed >> 32);
+    for (uint32_t j = 0; j < 6; ++j)
+        p.key[j] = perm_mix(lo ^ perm_mix(hi + 0x9E3779B9u * (j + 1)) ^ perm_mix(epoch + 0xBB67AE85u * (j + 1)));
+    int bits = 0;
+    while ((1ull << bits) < (unsigned long long)M) ++bits;
+    p.h = (bits + 1) / 2 < 1 ? 1 : (bits + 1) / 2;
+    p.mask = (1u << p.h) - 1u;
+    p.M = M;
+    return p;
+}
+
+__device__ __forceinline__ uint32_t perm_apply(const PermParams &p, uint32_t i) {
+    uint32_t x = i;
+    do {
+        uint32_t L = x >> p.h, R = x & p.mask;
+#pragma unroll
+        for (int j = 0; j < 6; ++j) {
+            uint32_t nr = L ^ (perm_mix(R ^ p.key[j]) & p.mask);
+            L = R;
+            R = nr;
+        }
+        x = (L << p.h) | R;
+    } while (x >= p.M);
+    return x;
+}
+
+struct GatherArgs {
+    const char *depth;
+    const float *proprio, *action, *logp, *value, *adv, *ret;
+    char *o_depth;
+    float *o_proprio, *o_action, *o_logp, *o_value, *o_adv, *o_ret;
+    uint32_t *o_index;
+    uint32_t start;      // first position of this minibatch in the permuted order
+    uint32_t rows;       // B
+    uint32_t frame16;    // frame bytes / 16
+    uint32_t chunks;     // CTAs per row
+    int P, A;
+};
+
+// One CTA copies one chunk of one row's depth frame with 128-bit loads (no L1 allocation,
+// evict-first) and streaming stores; chunk 0 also copies the row's small fields.
+__global__ void __launch_bounds__(256) gather_kernel(GatherArgs g, PermParams p) {
+    const uint32_t row = blockIdx.x / g.chunks;
+    const uint32_t chunk = blockIdx.x - row * g.chunks;
+    const uint32_t s = perm_apply(p, g.start + row);
+    const uint4 *src = reinterpret_cast<const uint4 *>(g.depth) + (size_t)s * g.frame16;
+    uint4 *dst = reinterpret_cast<uint4 *>(g.o_depth) + (size_t)row * g.frame16;
+    const uint32_t per = (g.frame16 + g.chunks - 1) / g.chunks;
+    const uint32_t lo = chunk * per;
+    const uint32_t hi = min(lo + per, g.frame16);
+    uint32_t i = lo + threadIdx.x;
+    for (; i + 3 * 256 < hi; i += 4 * 256) {
+        uint4 a = __ldcs(src + i), b = __ldcs(src + i + 256), c = __ldcs(src + i + 512), d = __ldcs(src + i + 768);
+        __stcs(dst + i, a);
+        __stcs(dst + i + 256, b);
+        __stcs(dst + i + 512, c);
+        __stcs(dst + i + 768, d);
+    }
+    for (; i < hi; i += 256) __stcs(dst + i, __ldcs(src + i));
+    if (chunk == 0) {
+        const int t = threadIdx.x;
+        if (t < g.P) g.o_proprio[(size_t)row * g.P + t] = g.proprio[(size_t)s * g.P + t];
+        if (t >= 64 && t < 64 + g.A) g.o_action[(size_t)row * g.A + (t - 64)] = g.action[(size_t)s * g.A + (t - 64)];
+        if (t == 128) g.o_logp[row] = g.logp[s];
+        if (t == 129) g.o_value[row] = g.value[s];
+        if (t == 130) g.o_adv[row] = g.adv[s];
+        if (t == 131) g.o_ret[row] = g.ret[s];
+        if (t == 132 && g.o_index) g.o_index[row] = s;
+    }
+}
+
+extern "C" int ppo_shuffle_gather_minibatch(const ppo_buffer *b, uint64_t seed, uint32_t epoch, int mb_index,
+                                            int num_minibatches, const ppo_minibatch *out, void *stream) {
+    if (!b || !out) return PPO_ERR_INVALID_ARG;
+    if (num_minibatches <= 0 || mb_index < 0 || mb_index >= num_minibatches) return PPO_ERR_INVALID_ARG;
+    const long long M = (long long)b->d.N * b->d.T;
+    if (M % num_minibatches != 0) return PPO_ERR_SHAPE;
+    const long long B = M / num_minibatches;
+    if (out->B != B) return PPO_ERR_SHAPE;
+    if (!out->depth_f16 || !out->proprio || !out->action || !out->logp_old || !out->value_old || !out->adv ||
+        !out->ret)
+        return PPO_ERR_INVALID_ARG;
+    if (!ppo_aligned(out->depth_f16, 16)) return PPO_ERR_ALIGN;
+    if (!b->gae_valid) return PPO_ERR_STATE;
+    const size_t frame = (size_t)b->d.H * b->d.W * 2;
+    if (frame % 16 != 0) return PPO_ERR_UNSUPPORTED;
+    if (b->d.P > 64 || b->d.A > 64) return PPO_ERR_UNSUPPORTED;
+    GatherArgs g;
+    g.depth = b->base + b->field_off[PPO_FIELD_DEPTH];
+    g.proprio = slab<float>(b, PPO_FIELD_PROPRIO);
+    g.action = slab<float>(b, PPO_FIELD_ACTION);
+    g.logp = slab<float>(b, PPO_FIELD_LOGP);
+    g.value = slab<float>(b, PPO_FIELD_VALUE);
+    g.adv = slab<float>(b, PPO_FIELD_ADV);
+    g.ret = slab<float>(b, PPO_FIELD_RET);
+    g.o_depth = static_cast<char *>(out->depth_f16);
+    g.o_proprio = out->proprio;
+    g.o_action = out->action;
+    g.o_logp = out->logp_old;
+    g.o_value = out->value_old;
+    g.o_adv = out->adv;
+    g.o_ret = out->ret;
+    g.o_index = out->index;
+    g.start = (uint32_t)(mb_index * B);
+    g.rows = (uint32_t)B;
+    g.frame16 = (uint32_t)(frame / 16);
+    // 16 KB per CTA: 4 x 128-bit per thread, so a frame of 38 400 B becomes 3 CTAs
+    g.chunks = (uint32_t)((frame + 16383) / 16384);
+    g.P = b->d.P;
+    g.A = b->d.A;
+    const long long ctas = B * g.chunks;
+    if (ctas > 0x7fffffffll) return PPO_ERR_UNSUPPORTED;
+    PermParams p = make_perm(seed, epoch, (uint32_t)M);
+    gather_kernel<<<(unsigned)ctas, 256, 0, static_cast<cudaStream_t>(stream)>>>(g, p);
+    PPO_LAUNCH_CHECK();
+    return PPO_OK;
+}

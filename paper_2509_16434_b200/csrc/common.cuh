@@ -1,0 +1,85 @@
+// Shared declarations of the CUDA library: status codes, handles, small device helpers.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <vector>
+
+#include "../../include/ppo_b200.h"
+
+typedef __nv_bfloat16 bf16;
+
+#define PPO_CUDA_CHECK(expr)                    \
+    do {                                        \
+        cudaError_t _e = (expr);                \
+        if (_e != cudaSuccess) return PPO_ERR_CUDA; \
+    } while (0)
+
+#define PPO_LAUNCH_CHECK() PPO_CUDA_CHECK(cudaGetLastError())
+
+static inline bool ppo_aligned(const void *p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+static inline size_t ppo_align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+static inline int ppo_cdiv(long long a, long long b) { return (int)((a + b - 1) / b); }
+
+// Device status word shared by all kernels (first error wins); lives in status.cu.
+int32_t *ppo_device_status_ptr();
+int ppo_num_sms();
+
+struct ppo_buffer {
+    ppo_buffer_desc d;
+    char *base;
+    size_t bytes;
+    size_t field_off[PPO_NUM_FIELDS];
+    bool gae_valid;
+    int gae_blocks;  // partial sums held in the scratch slab
+};
+
+// Geometry of one stride-2 convolution (an FC layer is the 1x1 image, k = 1 case).
+struct ConvGeom {
+    int B, Hi, Wi, Ci, Ho, Wo, Co, k, pad;
+    __host__ __device__ int taps() const { return k * k; }
+    __host__ __device__ long long M() const { return (long long)B * Ho * Wo; }
+    __host__ __device__ int K() const { return k * k * Ci; }
+};
+
+struct ppo_tensor {
+    int64_t off, size;
+};
+
+struct ppo_model {
+    ppo_model_desc d;
+    int L, F;
+    int Hs[PPO_MAX_CONV + 1], Ws[PPO_MAX_CONV + 1], Cs[PPO_MAX_CONV + 1];  // index 0 = input image
+    int hw[PPO_MAX_FC + 1];                                                // widths of h_0..h_F
+    std::vector<ppo_tensor> tensors;
+    size_t arena, nparams;
+    // bound arrays
+    float *master, *grad, *adam_m, *adam_v;
+    bf16 *shadow;
+    char *ws;
+    size_t ws_bytes;
+    int mbmax;
+    // workspace carve
+    bf16 *act[PPO_MAX_CONV + 1];   // act[l], l >= 1: [mb][Ho][Wo][C] post-ReLU
+    bf16 *dact[PPO_MAX_CONV + 1];  // gradient w.r.t. the pre-activation of act[l]
+    bf16 *h[PPO_MAX_FC + 1];       // h[0] = [pooled, proprio]; h[l] post-ReLU
+    bf16 *dh[PPO_MAX_FC + 2];      // dh[l]: gradient w.r.t. pre-activation of h[l]; dh[F+1]: head dout padded to 16
+    float *dh0_f32;                // gradient w.r.t. h[0] (pooled part feeds the un-pool)
+    bf16 *wT;                      // transposed bf16 weights Wt[ci][tap][co padded to 8] for the dgrad GEMMs
+    int64_t wT_off[2 * PPO_MAX_CONV + 2 * PPO_MAX_FC + 3];  // per tensor index (matrices only)
+    size_t wT_elems;
+    float *loss_partials;
+    int loss_partial_blocks;
+    bool wT_valid;
+    // forward/backward pairing
+    int last_row0, last_rows;
+    bool fwd_valid;
+    int impl;  // 0 = tensor-core GEMMs, 1 = CUDA-core reference GEMMs
+};
+
+__device__ __forceinline__ float bf2f(bf16 x) { return __bfloat162float(x); }
+
+__device__ __forceinline__ void ppo_report(int32_t *status, int code) { atomicCAS(status, 0, code); }

@@ -1,0 +1,37 @@
+// The three GEMM-shaped operations of the encoder, as implicit GEMMs over NHWC bf16
+// activations.  A fully connected layer is the case Hi = Wi = Ho = Wo = 1, k = 1, pad = 0.
+//   fwd   : Y[m][co]  = act( bias[co] + sum_{tap,ci} X[b, 2oh+kh-p, 2ow+kw-p, ci] * W[co][tap][ci] )
+//   dgrad : dX[m'][ci] = mask( sum_{tap,co} dY[b, (ih+p-kh)/2, (iw+p-kw)/2, co] * W[co][tap][ci] )
+//   wgrad : dW[co][tap][ci] += sum_m dY[m][co] * X[b, 2oh+kh-p, 2ow+kw-p, ci]
+// m = (b, oh, ow) over output pixels, m' = (b, ih, iw) over input pixels; fp32 accumulation.
+#pragma once
+#include "common.cuh"
+
+struct FwdEpilogue {
+    const float *bias;  // [Co] fp32
+    int relu;
+    bf16 *out;          // [M][Co] bf16, or nullptr when the head outputs below are used
+    float *out_mean;    // head: columns 0..A-1 -> [M][A]
+    float *out_value;   // head: column A -> [M]
+    int A;
+};
+
+struct DgradEpilogue {
+    const bf16 *mask_act;  // [M'][Ci]: output is zeroed where this is <= 0; may be nullptr
+    bf16 *out;             // [M'][Ci] bf16, or nullptr
+    float *out_f32;        // [M'][Ci] fp32, or nullptr
+};
+
+// ldy: row stride (elements) of Y / dY (>= Co).  wt_ld: row stride of the innermost (co)
+// dimension of the transposed weights Wt[ci][tap][wt_ld].
+int simt_gemm_fwd(const ConvGeom &g, const bf16 *X, const bf16 *W, const FwdEpilogue &e, cudaStream_t st);
+int simt_gemm_dgrad(const ConvGeom &g, const bf16 *dY, int ldy, const bf16 *W, const DgradEpilogue &e,
+                    cudaStream_t st);
+int simt_gemm_wgrad(const ConvGeom &g, const bf16 *dY, int ldy, const bf16 *X, float *dW, cudaStream_t st);
+
+int tc_gemm_fwd(const ConvGeom &g, const bf16 *X, const bf16 *W, const FwdEpilogue &e, int32_t *status,
+                cudaStream_t st);
+int tc_gemm_dgrad(const ConvGeom &g, const bf16 *dY, int ldy, const bf16 *Wt, int wt_ld, const DgradEpilogue &e,
+                  int32_t *status, cudaStream_t st);
+int tc_gemm_wgrad(const ConvGeom &g, const bf16 *dY, int ldy, const bf16 *X, float *dW, int32_t *status,
+                  cudaStream_t st);

@@ -1,0 +1,388 @@
+// Model handle (parameter arena layout, workspace carve), fused PPO loss + gradient,
+// Gaussian action sampling and the fused Adam pass.
+#include <math.h>
+
+#include <new>
+
+#include "common.cuh"
+
+static int conv_out(int in, int k) { return (in + 2 * (k / 2) - k) / 2 + 1; }
+
+extern "C" int ppo_model_create(const ppo_model_desc *d, ppo_model **out) {
+    if (!out) return PPO_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (!d) return PPO_ERR_INVALID_ARG;
+    if (d->H <= 0 || d->W <= 0 || d->n_conv < 1 || d->n_conv > PPO_MAX_CONV || d->n_fc < 0 || d->n_fc > PPO_MAX_FC ||
+        d->P <= 0 || d->A <= 0 || d->A > 15)
+        return PPO_ERR_INVALID_ARG;
+    for (int l = 0; l < d->n_conv; ++l) {
+        if (d->conv_c[l] <= 0 || d->conv_c[l] % 8 != 0 || d->conv_c[l] > 512) return PPO_ERR_UNSUPPORTED;
+        if (d->conv_k[l] < 1 || d->conv_k[l] % 2 == 0 || d->conv_k[l] > 7) return PPO_ERR_UNSUPPORTED;
+    }
+    if (d->conv_c[0] > 64) return PPO_ERR_UNSUPPORTED;  // first layer runs as a direct convolution
+    if (d->conv_c[0] * (d->conv_k[0] * d->conv_k[0] + 1) > 2048) return PPO_ERR_UNSUPPORTED;
+    for (int l = 0; l < d->n_fc; ++l)
+        if (d->fc[l] <= 0 || d->fc[l] % 8 != 0) return PPO_ERR_UNSUPPORTED;
+    if ((d->conv_c[d->n_conv - 1] + d->P) % 8 != 0) return PPO_ERR_UNSUPPORTED;
+    ppo_model *m = new (std::nothrow) ppo_model();
+    if (!m) return PPO_ERR_INVALID_ARG;
+    m->d = *d;
+    m->L = d->n_conv;
+    m->F = d->n_fc;
+    m->Hs[0] = d->H;
+    m->Ws[0] = d->W;
+    m->Cs[0] = 1;
+    for (int l = 0; l < m->L; ++l) {
+        m->Hs[l + 1] = conv_out(m->Hs[l], d->conv_k[l]);
+        m->Ws[l + 1] = conv_out(m->Ws[l], d->conv_k[l]);
+        m->Cs[l + 1] = d->conv_c[l];
+    }
+    m->hw[0] = m->Cs[m->L] + d->P;
+    for (int l = 0; l < m->F; ++l) m->hw[l + 1] = d->fc[l];
+    int64_t off = 0;
+    size_t count = 0;
+    auto push = [&](int64_t sz) {
+        m->tensors.push_back({off, sz});
+        off += (sz + 63) / 64 * 64;
+        count += (size_t)sz;
+    };
+    for (int l = 0; l < m->L; ++l) {
+        push((int64_t)m->Cs[l + 1] * d->conv_k[l] * d->conv_k[l] * m->Cs[l]);
+        push(m->Cs[l + 1]);
+    }
+    for (int l = 0; l < m->F; ++l) {
+        push((int64_t)m->hw[l + 1] * m->hw[l]);
+        push(m->hw[l + 1]);
+    }
+    push((int64_t)(d->A + 1) * m->hw[m->F]);
+    push(d->A + 1);
+    push(d->A);
+    m->arena = (size_t)off;
+    m->nparams = count;
+    {   // transposed copies of the weight matrices (conv layers >= 2, FC layers, head)
+        int64_t toff = 0;
+        for (size_t i = 0; i < m->tensors.size(); ++i) m->wT_off[i] = 0;
+        auto tpush = [&](int ti, int64_t Ci, int64_t taps, int64_t Co) {
+            m->wT_off[ti] = toff;
+            toff += (Ci * taps * ((Co + 7) / 8 * 8) + 63) / 64 * 64;
+        };
+        for (int l = 2; l <= m->L; ++l) tpush(2 * (l - 1), m->Cs[l - 1], d->conv_k[l - 1] * d->conv_k[l - 1], m->Cs[l]);
+        for (int l = 1; l <= m->F + 1; ++l)
+            tpush(2 * m->L + 2 * (l - 1), m->hw[l - 1], 1, l <= m->F ? m->hw[l] : d->A + 1);
+        m->wT_elems = (size_t)toff;
+    }
+    m->master = m->grad = m->adam_m = m->adam_v = nullptr;
+    m->shadow = nullptr;
+    m->ws = nullptr;
+    m->ws_bytes = 0;
+    m->mbmax = 0;
+    m->fwd_valid = false;
+    m->wT_valid = false;
+    m->last_row0 = m->last_rows = -1;
+    m->impl = 0;
+    const char *e = getenv("PPO_B200_ENCODER");
+    if (e && e[0] == 's') m->impl = 1;  // "simt": CUDA-core reference GEMMs (debugging aid)
+    *out = m;
+    return PPO_OK;
+}
+
+extern "C" int ppo_model_destroy(ppo_model *m) {
+    if (!m) return PPO_ERR_INVALID_ARG;
+    delete m;
+    return PPO_OK;
+}
+
+extern "C" size_t ppo_model_param_count(const ppo_model *m) { return m ? m->nparams : 0; }
+extern "C" size_t ppo_model_arena_elems(const ppo_model *m) { return m ? m->arena : 0; }
+extern "C" int ppo_model_num_tensors(const ppo_model *m) { return m ? (int)m->tensors.size() : 0; }
+extern "C" int ppo_model_tensor_info(const ppo_model *m, int i, int64_t *off, int64_t *size) {
+    if (!m || i < 0 || i >= (int)m->tensors.size() || !off || !size) return PPO_ERR_INVALID_ARG;
+    *off = m->tensors[i].off;
+    *size = m->tensors[i].size;
+    return PPO_OK;
+}
+
+static const int kLossThreads = 128;
+
+// Walks the workspace carve; with base == nullptr only sizes are computed.
+static size_t carve(ppo_model *m, const ppo_model *shape, int mb, char *base) {
+    size_t off = 0;
+    auto take = [&](size_t bytes) -> char * {
+        char *p = base ? base + off : nullptr;
+        off += ppo_align_up(bytes, 256);
+        return p;
+    };
+    for (int l = 1; l <= shape->L; ++l) {
+        size_t bytes = (size_t)mb * shape->Hs[l] * shape->Ws[l] * shape->Cs[l] * sizeof(bf16);
+        char *a = take(bytes), *g = take(bytes);
+        if (m) { m->act[l] = (bf16 *)a; m->dact[l] = (bf16 *)g; }
+    }
+    for (int l = 0; l <= shape->F; ++l) {
+        size_t bytes = (size_t)mb * shape->hw[l] * sizeof(bf16);
+        char *a = take(bytes), *g = take(bytes);
+        if (m) { m->h[l] = (bf16 *)a; m->dh[l] = (bf16 *)g; }
+    }
+    {
+        char *g = take((size_t)mb * 16 * sizeof(bf16));
+        if (m) m->dh[shape->F + 1] = (bf16 *)g;
+        char *f = take((size_t)mb * shape->hw[0] * sizeof(float));
+        if (m) m->dh0_f32 = (float *)f;
+        char *w = take(shape->wT_elems * sizeof(bf16));
+        if (m) m->wT = (bf16 *)w;
+        int blocks = ppo_cdiv(mb, kLossThreads);
+        char *lp = take((size_t)blocks * 32 * sizeof(float));
+        if (m) { m->loss_partials = (float *)lp; m->loss_partial_blocks = blocks; }
+    }
+    return off;
+}
+
+extern "C" size_t ppo_model_workspace_bytes(const ppo_model *m, int microbatch) {
+    if (!m || microbatch <= 0) return 0;
+    return carve(nullptr, m, microbatch, nullptr);
+}
+
+extern "C" int ppo_model_bind(ppo_model *m, float *master, void *shadow, float *grad, float *am, float *av, void *ws,
+                              size_t ws_bytes, int microbatch) {
+    if (!m || !master || !shadow || !grad || !am || !av || !ws || microbatch <= 0) return PPO_ERR_INVALID_ARG;
+    if (!ppo_aligned(master, 16) || !ppo_aligned(shadow, 16) || !ppo_aligned(grad, 16) || !ppo_aligned(am, 16) ||
+        !ppo_aligned(av, 16) || !ppo_aligned(ws, 256))
+        return PPO_ERR_ALIGN;
+    if (ws_bytes < ppo_model_workspace_bytes(m, microbatch)) return PPO_ERR_SHAPE;
+    m->master = master;
+    m->shadow = static_cast<bf16 *>(shadow);
+    m->grad = grad;
+    m->adam_m = am;
+    m->adam_v = av;
+    m->ws = static_cast<char *>(ws);
+    m->ws_bytes = ws_bytes;
+    m->mbmax = microbatch;
+    carve(m, m, microbatch, m->ws);
+    m->fwd_valid = false;
+    m->wT_valid = false;
+    return PPO_OK;
+}
+
+// ------------------------------------------------------------ shadow / zero ----
+
+__global__ void __launch_bounds__(256) shadow_kernel(const float4 *__restrict__ master, uint2 *__restrict__ shadow,
+                                                     size_t n4) {
+    size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n4) return;
+    float4 x = master[i];
+    __nv_bfloat162 lo = __floats2bfloat162_rn(x.x, x.y), hi = __floats2bfloat162_rn(x.z, x.w);
+    uint2 o;
+    o.x = *reinterpret_cast<uint32_t *>(&lo);
+    o.y = *reinterpret_cast<uint32_t *>(&hi);
+    shadow[i] = o;
+}
+
+extern "C" int ppo_model_sync_shadow(ppo_model *m, void *stream) {
+    if (!m || !m->master) return PPO_ERR_STATE;
+    size_t n4 = m->arena / 4;
+    shadow_kernel<<<ppo_cdiv(n4, 256), 256, 0, static_cast<cudaStream_t>(stream)>>>(
+        reinterpret_cast<const float4 *>(m->master), reinterpret_cast<uint2 *>(m->shadow), n4);
+    PPO_LAUNCH_CHECK();
+    m->wT_valid = false;
+    return PPO_OK;
+}
+
+extern "C" int ppo_model_zero_grad(ppo_model *m, void *stream) {
+    if (!m || !m->grad) return PPO_ERR_STATE;
+    PPO_CUDA_CHECK(cudaMemsetAsync(m->grad, 0, m->arena * sizeof(float), static_cast<cudaStream_t>(stream)));
+    return PPO_OK;
+}
+
+// -------------------------------------------------------------------- Adam ----
+
+// One 128-bit lane per thread over the whole arena: reads theta, m, v, g (16 B/param),
+// writes theta, m, v (12 B/param) and the bf16 shadow (2 B/param).
+__global__ void __launch_bounds__(256) adam_kernel(float4 *__restrict__ theta, float4 *__restrict__ m,
+                                                   float4 *__restrict__ v, const float4 *__restrict__ g,
+                                                   uint2 *__restrict__ shadow, size_t n4, float lr, float b1,
+                                                   float b2, float eps, float inv_c1, float inv_c2) {
+    const size_t nth = (size_t)gridDim.x * blockDim.x;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += nth) {
+        float4 th = theta[i], mm = m[i], vv = v[i];
+        const float4 gg = g[i];
+        float *pt = &th.x, *pm = &mm.x, *pv = &vv.x;
+        const float *pg = &gg.x;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            pm[j] = b1 * pm[j] + (1.f - b1) * pg[j];
+            pv[j] = b2 * pv[j] + (1.f - b2) * pg[j] * pg[j];
+            const float mhat = pm[j] * inv_c1, vhat = pv[j] * inv_c2;
+            pt[j] = pt[j] - lr * mhat / (sqrtf(vhat) + eps);
+        }
+        theta[i] = th;
+        m[i] = mm;
+        v[i] = vv;
+        __nv_bfloat162 lo = __floats2bfloat162_rn(th.x, th.y), hi = __floats2bfloat162_rn(th.z, th.w);
+        uint2 o;
+        o.x = *reinterpret_cast<uint32_t *>(&lo);
+        o.y = *reinterpret_cast<uint32_t *>(&hi);
+        shadow[i] = o;
+    }
+}
+
+extern "C" int ppo_adam_step(ppo_model *m, float lr, float beta1, float beta2, float eps, int64_t step,
+                             void *stream) {
+    if (!m || !m->master) return PPO_ERR_STATE;
+    if (step < 1 || !(beta1 >= 0.f && beta1 < 1.f) || !(beta2 >= 0.f && beta2 < 1.f) || !(eps > 0.f))
+        return PPO_ERR_INVALID_ARG;
+    const double c1 = 1.0 - pow((double)beta1, (double)step), c2 = 1.0 - pow((double)beta2, (double)step);
+    const size_t n4 = m->arena / 4;
+    int blocks = ppo_cdiv(n4, 256);
+    const int cap = ppo_num_sms() * 8;
+    if (blocks > cap) blocks = cap;
+    adam_kernel<<<blocks, 256, 0, static_cast<cudaStream_t>(stream)>>>(
+        reinterpret_cast<float4 *>(m->master), reinterpret_cast<float4 *>(m->adam_m),
+        reinterpret_cast<float4 *>(m->adam_v), reinterpret_cast<const float4 *>(m->grad),
+        reinterpret_cast<uint2 *>(m->shadow), n4, lr, beta1, beta2, eps, (float)(1.0 / c1), (float)(1.0 / c2));
+    PPO_LAUNCH_CHECK();
+    m->wT_valid = false;
+    m->fwd_valid = false;
+    return PPO_OK;
+}
+
+// -------------------------------------------------------------------- loss ----
+
+#define PPO_MAX_A 16
+#define PPO_HALF_LOG_2PI 0.91893853320467274178f
+
+__device__ __forceinline__ float warp_sum_f(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_down_sync(0xffffffffu, v, o);
+    return v;
+}
+
+// One thread per row: log-prob, ratio, clipped surrogate, value error and their gradients.
+// Block sums of {L_pi, L_V, kl, clipfrac, dlogsigma[A]} go to partials[blockIdx.x][32].
+__global__ void __launch_bounds__(kLossThreads) loss_kernel(
+    int rows, int A, float inv_Bt, const float *__restrict__ mean, const float *__restrict__ value,
+    const float *__restrict__ logsigma, const float *__restrict__ action, const float *__restrict__ logp_old,
+    const float *__restrict__ adv, const float *__restrict__ ret, float clip, float vf_coef,
+    float *__restrict__ dmean, float *__restrict__ dvalue, float *__restrict__ partials) {
+    __shared__ float sh[kLossThreads / 32][4 + PPO_MAX_A];
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    float acc[4 + PPO_MAX_A];
+#pragma unroll
+    for (int j = 0; j < 4 + PPO_MAX_A; ++j) acc[j] = 0.f;
+    if (i < rows) {
+        float z[PPO_MAX_A], inv_sg[PPO_MAX_A];
+        float logp = 0.f;
+#pragma unroll
+        for (int j = 0; j < PPO_MAX_A; ++j) {
+            if (j < A) {
+                const float ls = logsigma[j];
+                inv_sg[j] = expf(-ls);
+                z[j] = (action[(size_t)i * A + j] - mean[(size_t)i * A + j]) * inv_sg[j];
+                logp += -0.5f * z[j] * z[j] - ls - PPO_HALF_LOG_2PI;
+            }
+        }
+        const float lpo = logp_old[i];
+        const float r = expf(logp - lpo);
+        const float rc = fminf(fmaxf(r, 1.f - clip), 1.f + clip);
+        const float a = adv[i];
+        const float s_un = r * a, s_cl = rc * a;
+        const bool unclipped = s_un <= s_cl;
+        const float s = unclipped ? s_un : s_cl;
+        const float gs = unclipped ? a : 0.f;
+        const float verr = value[i] - ret[i];
+        acc[0] = -s * inv_Bt;
+        acc[1] = verr * verr * inv_Bt;
+        acc[2] = (lpo - logp) * inv_Bt;
+        acc[3] = (fabsf(r - 1.f) > clip ? 1.f : 0.f) * inv_Bt;
+        const float dlogp = -gs * r * inv_Bt;
+#pragma unroll
+        for (int j = 0; j < PPO_MAX_A; ++j) {
+            if (j < A) {
+                dmean[(size_t)i * A + j] = dlogp * z[j] * inv_sg[j];
+                acc[4 + j] = dlogp * (z[j] * z[j] - 1.f);
+            }
+        }
+        dvalue[i] = 2.f * vf_coef * verr * inv_Bt;
+    }
+    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+#pragma unroll
+    for (int j = 0; j < 4 + PPO_MAX_A; ++j) {
+        float v = warp_sum_f(acc[j]);
+        if (lane == 0) sh[wid][j] = v;
+    }
+    __syncthreads();
+    if (threadIdx.x < 4 + PPO_MAX_A) {
+        float v = 0.f;
+#pragma unroll
+        for (int w = 0; w < kLossThreads / 32; ++w) v += sh[w][threadIdx.x];
+        partials[(size_t)blockIdx.x * 32 + threadIdx.x] = v;
+    }
+}
+
+// Single block: fixed-order sum of the per-block partials (fp64), added into the loss
+// scalars and the log-sigma gradient.
+__global__ void __launch_bounds__(32) loss_finalize_kernel(const float *__restrict__ partials, int nblocks, int A,
+                                                           const float *__restrict__ logsigma, float share,
+                                                           float ent_coef, float *__restrict__ loss_out,
+                                                           float *__restrict__ grad_logsigma) {
+    const int j = threadIdx.x;
+    if (j >= 4 + A) return;
+    double s = 0.0;
+    for (int b = 0; b < nblocks; ++b) s += (double)partials[(size_t)b * 32 + j];
+    if (j == 0) loss_out[0] += (float)s;
+    if (j == 1) loss_out[1] += (float)s;
+    if (j == 2) loss_out[3] += (float)s;
+    if (j == 3) loss_out[4] += (float)s;
+    if (j >= 4) grad_logsigma[j - 4] += (float)s - ent_coef * share;
+    if (j == 0) {
+        float H = 0.5f * A * (1.f + 2.f * PPO_HALF_LOG_2PI);
+        for (int k = 0; k < A; ++k) H += logsigma[k];
+        loss_out[2] += H * share;
+    }
+}
+
+extern "C" int ppo_loss_fwd_bwd(ppo_model *m, const ppo_minibatch *mb, int row0, int rows, int B_total,
+                                const float *mean, const float *value, float clip, float vf_coef, float ent_coef,
+                                float *loss_out, float *dmean, float *dvalue, void *stream) {
+    if (!m || !mb || !mean || !value || !loss_out || !dmean || !dvalue) return PPO_ERR_INVALID_ARG;
+    if (!m->master) return PPO_ERR_STATE;
+    if (row0 < 0 || rows <= 0 || row0 + rows > mb->B || B_total < rows || rows > m->mbmax) return PPO_ERR_SHAPE;
+    if (!(clip > 0.f)) return PPO_ERR_INVALID_ARG;
+    const int A = m->d.A;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const float *logsigma = m->master + m->tensors.back().off;
+    const int blocks = ppo_cdiv(rows, kLossThreads);
+    loss_kernel<<<blocks, kLossThreads, 0, st>>>(rows, A, 1.f / (float)B_total, mean, value, logsigma,
+                                                 mb->action + (size_t)row0 * A, mb->logp_old + row0, mb->adv + row0,
+                                                 mb->ret + row0, clip, vf_coef, dmean, dvalue, m->loss_partials);
+    PPO_LAUNCH_CHECK();
+    loss_finalize_kernel<<<1, 32, 0, st>>>(m->loss_partials, blocks, A, logsigma, (float)rows / (float)B_total,
+                                           ent_coef, loss_out, m->grad + m->tensors.back().off);
+    PPO_LAUNCH_CHECK();
+    return PPO_OK;
+}
+
+// ------------------------------------------------------------------ sample ----
+
+__global__ void __launch_bounds__(128) sample_kernel(int rows, int A, const float *__restrict__ mean,
+                                                     const float *__restrict__ logsigma,
+                                                     const float *__restrict__ eps, float *__restrict__ action,
+                                                     float *__restrict__ logp) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= rows) return;
+    float lp = 0.f;
+    for (int j = 0; j < A; ++j) {
+        const float ls = logsigma[j], e = eps[(size_t)i * A + j];
+        action[(size_t)i * A + j] = mean[(size_t)i * A + j] + expf(ls) * e;
+        lp += -0.5f * e * e - ls - PPO_HALF_LOG_2PI;
+    }
+    logp[i] = lp;
+}
+
+extern "C" int ppo_policy_sample(const ppo_model *m, int rows, const float *mean, const float *eps, float *action,
+                                 float *logp, void *stream) {
+    if (!m || !mean || !eps || !action || !logp || rows <= 0) return PPO_ERR_INVALID_ARG;
+    if (!m->master) return PPO_ERR_STATE;
+    sample_kernel<<<ppo_cdiv(rows, 128), 128, 0, static_cast<cudaStream_t>(stream)>>>(
+        rows, m->d.A, mean, m->master + m->tensors.back().off, eps, action, logp);
+    PPO_LAUNCH_CHECK();
+    return PPO_OK;
+}

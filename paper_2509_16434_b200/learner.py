@@ -1,0 +1,109 @@
+"""TrainPPO (Algorithm 2) as a sequence of C-ABI calls: GAE once, then for every epoch and
+minibatch gather -> forward -> loss -> backward -> Adam, in micro-batches.
+
+Call sequencing and buffer ownership only; all arithmetic happens in libppo_b200.so.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass
+from typing import Dict, Optional
+
+import torch
+
+from . import binding as ppo
+from .synth import Workload
+
+
+@dataclass
+class Hyper:
+    gamma: float = 0.99
+    lam: float = 0.95
+    clip: float = 0.2
+    vf_coef: float = 0.5
+    ent_coef: float = 0.01
+    lr: float = 3e-4
+    beta1: float = 0.9
+    beta2: float = 0.999
+    eps: float = 1e-8
+
+
+class Learner:
+    def __init__(self, w: Workload, microbatch: int, device="cuda", hyper: Optional[Hyper] = None,
+                 with_index: bool = False):
+        self.w = w
+        self.device = device
+        self.hyper = hyper or Hyper(gamma=w.gamma, lam=w.lam, clip=w.clip)
+        self.bdesc = ppo.buffer_desc(w.N, w.T, w.H, w.W, w.P, w.A)
+        self.buffer = ppo.Buffer(self.bdesc, device)
+        self.mdesc = ppo.model_desc(w.H, w.W, w.conv_c, w.conv_k, w.fc, w.P, w.A)
+        self.microbatch = min(microbatch, w.B)
+        self.model = ppo.Model(self.mdesc, self.microbatch, device)
+        self.mb = ppo.MinibatchArrays(self.bdesc, w.B, device, with_index=with_index)
+        mbs = self.microbatch
+        self.mean = torch.empty((mbs, w.A), dtype=torch.float32, device=device)
+        self.value = torch.empty(mbs, dtype=torch.float32, device=device)
+        self.dmean = torch.empty((mbs, w.A), dtype=torch.float32, device=device)
+        self.dvalue = torch.empty(mbs, dtype=torch.float32, device=device)
+        self.loss = torch.zeros(5, dtype=torch.float32, device=device)
+        self.stats = torch.zeros(2, dtype=torch.float32, device=device)
+        self.adam_t = 0
+        self.launches = 0  # kernels and memsets enqueued by the library, by this object's count
+
+    # ------------------------------------------------------------------ buffer fill
+
+    def write_rollout(self, r: Dict[str, torch.Tensor], action: torch.Tensor, logp: torch.Tensor):
+        """D <- D U {...} for t = 0..T-1 from device tensors shaped [T, N, ...]."""
+        for t in range(self.w.T):
+            ppo.ppo_buffer_write_step(self.buffer, t, r["depth"][t], r["proprio"][t], action[t], logp[t],
+                                      r["value"][t], r["reward"][t], r["done"][t])
+
+    def act(self, depth: torch.Tensor, proprio: torch.Tensor, eps: torch.Tensor):
+        """Rollout-time policy: mean/value from the encoder, action = mean + sigma * eps and its log-prob.
+        depth [n,H,W] fp16, proprio [n,P], eps [n,A]; processed in micro-batches.  Returns (action, logp, value)."""
+        n = depth.shape[0]
+        action = torch.empty((n, self.w.A), dtype=torch.float32, device=self.device)
+        logp = torch.empty(n, dtype=torch.float32, device=self.device)
+        value = torch.empty(n, dtype=torch.float32, device=self.device)
+        obs = ppo.Minibatch(depth.data_ptr(), proprio.data_ptr(), None, None, None, None, None, None, n)
+        for r0 in range(0, n, self.microbatch):
+            rows = min(self.microbatch, n - r0)
+            ppo.ppo_encoder_fwd(self.model, obs, r0, rows, self.mean, value[r0:r0 + rows])
+            ppo.ppo_policy_sample(self.model, rows, self.mean, eps[r0:r0 + rows], action[r0:r0 + rows],
+                                  logp[r0:r0 + rows])
+        return action, logp, value
+
+    # ------------------------------------------------------------------ TrainPPO
+
+    def compute_gae(self, last_value: torch.Tensor, normalize: bool = True):
+        h = self.hyper
+        ppo.ppo_compute_gae(self.buffer, last_value, h.gamma, h.lam, normalize, self.stats)
+        self.launches += 2 if normalize else 1
+
+    def minibatch_step(self, seed: int, epoch: int, k: int, num_minibatches: Optional[int] = None):
+        """gather -> (fwd -> loss -> bwd) per micro-batch -> Adam for minibatch k of this epoch."""
+        w, h = self.w, self.hyper
+        K = num_minibatches or w.minibatches
+        B = w.M // K
+        n_layers_gemm = (len(w.conv_c) - 1) + len(w.fc) + 1
+        ppo.ppo_shuffle_gather_minibatch(self.buffer, seed, epoch, k, K, self.mb)
+        ppo.ppo_model_zero_grad(self.model)
+        self.loss.zero_()
+        self.launches += 3
+        for r0 in range(0, B, self.microbatch):
+            rows = min(self.microbatch, B - r0)
+            ppo.ppo_encoder_fwd(self.model, self.mb, r0, rows, self.mean, self.value)
+            ppo.ppo_loss_fwd_bwd(self.model, self.mb, r0, rows, B, self.mean, self.value, h.clip, h.vf_coef,
+                                 h.ent_coef, self.loss, self.dmean, self.dvalue)
+            ppo.ppo_encoder_bwd(self.model, self.mb, r0, rows, self.dmean, self.dvalue, True)
+            # fwd: conv1 + GEMMs + pool; loss: 2; bwd: pack + 3 per GEMM layer + unpool + conv1 wgrad
+            self.launches += (1 + n_layers_gemm + 1) + 2 + (1 + 3 * n_layers_gemm + 1 + 1)
+        self.adam_t += 1
+        ppo.ppo_adam_step(self.model, h.lr, h.beta1, h.beta2, h.eps, self.adam_t)
+        self.launches += 1
+
+    def train(self, last_value: torch.Tensor, seed: int = 0):
+        """One TrainPPO call over the current buffer."""
+        self.compute_gae(last_value)
+        for e in range(self.w.epochs):
+            for k in range(self.w.minibatches):
+                self.minibatch_step(seed, e, k)

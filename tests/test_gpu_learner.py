@@ -1,0 +1,220 @@
+"""GPU parity: encoder forward/backward, PPO loss + gradient, Adam and whole minibatch steps against the CPU oracle."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import oracle as orc
+from paper_2509_16434_b200 import binding as ppo
+from paper_2509_16434_b200 import synth
+from paper_2509_16434_b200.learner import Hyper, Learner
+from helpers import oracle_model, oracle_rollout_actions, rel_l2
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+ENC_TOL = 2e-2    # relative L2: bf16 operands / activations with fp32 accumulation vs fp64
+LOSS_TOL = 1e-3   # relative error of the loss scalars
+ADAM_TOL = 1e-3   # relative L2 of the parameters after one step
+
+
+def _setup(w, microbatch, seed=0, jitter=True, theta_scale_head=1.0):
+    """Learner with seeded parameters and a buffer filled from the oracle-side rollout policy."""
+    md = oracle_model(w)
+    lay = orc.param_layout(md)
+    theta = synth.init_params(lay.total, lay.offsets, lay.shapes, seed)
+    if theta_scale_head != 1.0:
+        hw = len(lay.offsets) - 3
+        theta[lay.offsets[hw]:lay.offsets[hw] + lay.sizes[hw]] *= theta_scale_head
+    g = np.random.default_rng(seed + 7)
+    for off, sz, shp in zip(lay.offsets, lay.sizes, lay.shapes):
+        if len(shp) == 1:
+            theta[off:off + sz] = (0.05 * g.standard_normal(sz)).astype(np.float32)
+    roll = synth.rollout_numpy(w, seed)
+    action, logp = oracle_rollout_actions(md, theta, roll)
+    if jitter:
+        logp = (logp + roll["logp_jitter"]).astype(np.float32)
+    L = Learner(w, microbatch, DEV, with_index=True)
+    L.model.load(theta)
+    dev = {k: torch.as_tensor(v).to(DEV) for k, v in roll.items()}
+    L.write_rollout(dev, torch.as_tensor(action).to(DEV), torch.as_tensor(logp).to(DEV))
+    return L, md, lay, theta, roll, action, logp, dev
+
+
+def _oracle_minibatch(md, lay, theta, roll, action, logp, w, hyper, seed, epoch, k, K):
+    adv, ret = orc.gae(roll["reward"], roll["value"], roll["done"], roll["last_value"], np.float32(hyper.gamma),
+                       np.float32(hyper.lam))
+    adv, _, _ = orc.adv_normalize(adv)
+    M = w.N * w.T
+    B = M // K
+    idx = orc.perm(seed, epoch, M, k * B, B)
+    f = orc.gather({"depth": roll["depth"], "proprio": roll["proprio"], "action": action, "logp": logp,
+                    "adv": adv.astype(np.float32), "ret": ret.astype(np.float32)}, idx, w.N)
+    Ltot, out, grad, mu, V = orc.total_loss_and_grad(md, theta, f["depth"], f["proprio"], f["action"], f["logp"],
+                                                     f["adv"], f["ret"], np.float32(hyper.clip),
+                                                     np.float32(hyper.vf_coef), np.float32(hyper.ent_coef))
+    return f, out, grad, mu, V
+
+
+def _check_grads(lay, got, want, tol=ENC_TOL):
+    for i, (off, sz) in enumerate(zip(lay.offsets, lay.sizes)):
+        e = rel_l2(got[off:off + sz], want[off:off + sz])
+        assert e <= tol, f"tensor {i}: rel L2 {e:.3e}"
+    assert rel_l2(got, want) <= tol
+
+
+SHAPES = {
+    "tiny": synth.Workload("tiny", 8, 4, 16, 24, (8, 16), (3, 3), (32,), 1, 2, P=8, A=3),
+    "odd": synth.Workload("odd", 6, 5, 17, 23, (8, 16, 24), (5, 3, 3), (40, 24), 1, 3, P=16, A=5),
+    "cfg1_twin": synth.WORKLOADS["cfg1"].scaled(16, T=4),
+    "cfg2_twin": synth.WORKLOADS["cfg2"].scaled(8, T=2, minibatches=2),
+    "cfg4_twin": synth.WORKLOADS["cfg4"].scaled(2, T=2, minibatches=2),
+}
+
+
+@pytest.mark.parametrize("name,microbatch", [("tiny", 16), ("tiny", 5), ("odd", 10), ("cfg1_twin", 16),
+                                             ("cfg2_twin", 8), ("cfg2_twin", 3), ("cfg4_twin", 2)])
+def test_minibatch_forward_loss_backward_match_oracle(name, microbatch):
+    w = SHAPES[name]
+    L, md, lay, theta, roll, action, logp, dev = _setup(w, microbatch, theta_scale_head=20.0)
+    h = L.hyper
+    K = w.minibatches
+    B = w.M // K
+    L.compute_gae(dev["last_value"])
+    k = K - 1
+    f, out_o, grad_o, mu_o, V_o = _oracle_minibatch(md, lay, theta, roll, action, logp, w, h, 3, 1, k, K)
+    ppo.ppo_shuffle_gather_minibatch(L.buffer, 3, 1, k, K, L.mb)
+    ppo.ppo_model_zero_grad(L.model)
+    L.loss.zero_()
+    mus, Vs = [], []
+    for r0 in range(0, B, L.microbatch):
+        rows = min(L.microbatch, B - r0)
+        ppo.ppo_encoder_fwd(L.model, L.mb, r0, rows, L.mean, L.value)
+        mus.append(L.mean[:rows].cpu().numpy().copy())
+        Vs.append(L.value[:rows].cpu().numpy().copy())
+        ppo.ppo_loss_fwd_bwd(L.model, L.mb, r0, rows, B, L.mean, L.value, h.clip, h.vf_coef, h.ent_coef, L.loss,
+                             L.dmean, L.dvalue)
+        ppo.ppo_encoder_bwd(L.model, L.mb, r0, rows, L.dmean, L.dvalue, True)
+    assert ppo.ppo_poll_status() == 0
+    mu, V = np.concatenate(mus), np.concatenate(Vs)
+    assert rel_l2(mu, mu_o) <= ENC_TOL, rel_l2(mu, mu_o)
+    assert rel_l2(V, V_o) <= ENC_TOL, rel_l2(V, V_o)
+    out = L.loss.cpu().numpy()
+    assert 0.0 < out_o[4] < 1.0, "both clip branches must be exercised"
+    # entropy is exact arithmetic on log-sigma; the others inherit the encoder's bf16 error through mu and V
+    assert abs(out[2] - out_o[2]) <= LOSS_TOL * abs(out_o[2])
+    for j, tol in [(0, 2e-2), (1, 2e-2), (3, 2e-2)]:
+        assert abs(out[j] - out_o[j]) <= tol * max(abs(out_o[j]), 0.05), (j, out[j], out_o[j])
+    assert abs(out[4] - out_o[4]) <= 2.0 / B + 1e-6
+    _check_grads(lay, L.model.grad.cpu().numpy(), grad_o, tol=3e-2)
+
+
+def test_loss_kernel_alone_matches_oracle_to_1e3():
+    """Same mu and V on both sides: isolates the fused loss/gradient kernel (fp32 vs fp64)."""
+    w = SHAPES["cfg1_twin"]
+    L, md, lay, theta, roll, action, logp, dev = _setup(w, 64)
+    g = np.random.default_rng(0)
+    B, A = 64, w.A
+    mu = (0.3 * g.standard_normal((B, A))).astype(np.float32)
+    V = g.standard_normal(B).astype(np.float32)
+    ls = (0.2 * g.standard_normal(A)).astype(np.float32)
+    act = (mu + np.exp(ls) * g.standard_normal((B, A))).astype(np.float32)
+    z = (act - mu) / np.exp(ls)
+    lpo = ((-0.5 * z ** 2 - ls - 0.5 * np.log(2 * np.pi)).sum(1) + 0.3 * g.standard_normal(B)).astype(np.float32)
+    adv, ret = g.standard_normal(B).astype(np.float32), g.standard_normal(B).astype(np.float32)
+    L.model.master[lay.offsets[-1]:lay.offsets[-1] + A] = torch.as_tensor(ls).to(DEV)
+    mb = ppo.MinibatchArrays(L.bdesc, B)
+    mb.action.copy_(torch.as_tensor(act))
+    mb.logp_old.copy_(torch.as_tensor(lpo))
+    mb.adv.copy_(torch.as_tensor(adv))
+    mb.ret.copy_(torch.as_tensor(ret))
+    out_o, dmu_o, dV_o, dls_o = orc.loss(mu, V, ls, act, lpo, adv, ret, np.float32(0.2), 0.5, np.float32(0.01))
+    ppo.ppo_model_zero_grad(L.model)
+    L.loss.zero_()
+    dmean = torch.empty((B, A), device=DEV)
+    dvalue = torch.empty(B, device=DEV)
+    # two micro-batches of uneven size must add up to the minibatch
+    mean_d, value_d = torch.as_tensor(mu).to(DEV), torch.as_tensor(V).to(DEV)
+    for r0, rows in [(0, 40), (40, 24)]:
+        ppo.ppo_loss_fwd_bwd(L.model, mb, r0, rows, B, mean_d[r0:], value_d[r0:], 0.2, 0.5, 0.01, L.loss,
+                             dmean[r0:], dvalue[r0:])
+    out = L.loss.cpu().numpy()
+    assert 0 < out_o[4] < 1
+    for j in range(5):
+        assert abs(out[j] - out_o[j]) <= LOSS_TOL * max(abs(out_o[j]), 1e-3), (j, out[j], out_o[j])
+    assert rel_l2(dmean.cpu().numpy(), dmu_o) <= LOSS_TOL
+    assert rel_l2(dvalue.cpu().numpy(), dV_o) <= LOSS_TOL
+    dls = L.model.grad[lay.offsets[-1]:lay.offsets[-1] + A].cpu().numpy()
+    assert rel_l2(dls, dls_o) <= LOSS_TOL
+    assert ppo.ppo_poll_status() == 0
+
+
+def test_ratio_is_one_on_the_rollout_policy():
+    """Old log-probs from the same weights: r = 1 up to the encoder's rounding, so nothing is clipped."""
+    w = SHAPES["cfg1_twin"]
+    L, md, lay, theta, roll, action, logp, dev = _setup(w, 32, jitter=False)
+    L.compute_gae(dev["last_value"])
+    ppo.ppo_shuffle_gather_minibatch(L.buffer, 0, 0, 0, 2, L.mb)
+    L.loss.zero_()
+    ppo.ppo_model_zero_grad(L.model)
+    B = w.M // 2
+    ppo.ppo_encoder_fwd(L.model, L.mb, 0, B, L.mean, L.value)
+    ppo.ppo_loss_fwd_bwd(L.model, L.mb, 0, B, B, L.mean, L.value, 0.2, 0.5, 0.01, L.loss, L.dmean, L.dvalue)
+    out = L.loss.cpu().numpy()
+    assert out[4] == 0.0 and abs(out[3]) < 5e-3
+    assert abs(out[0] + L.mb.adv[:B].mean().item()) < 5e-3
+
+
+def test_adam_step_matches_oracle():
+    w = SHAPES["cfg1_twin"]
+    L, md, lay, theta, *_ = _setup(w, 16)
+    n = lay.total
+    g = np.random.default_rng(5)
+    grad = (g.standard_normal(n) * (g.random(n) < 0.9)).astype(np.float32)
+    m0 = (0.1 * g.standard_normal(n)).astype(np.float32)
+    v0 = (0.01 * g.random(n)).astype(np.float32)
+    L.model.grad.copy_(torch.as_tensor(grad))
+    L.model.adam_m.copy_(torch.as_tensor(m0))
+    L.model.adam_v.copy_(torch.as_tensor(v0))
+    th, m, v = theta.astype(np.float64), m0.astype(np.float64), v0.astype(np.float64)
+    for step in (1, 2, 7):
+        orc.adam(th, m, v, grad, np.float32(3e-4), np.float32(0.9), np.float32(0.999), np.float32(1e-8), step)
+        ppo.ppo_adam_step(L.model, 3e-4, 0.9, 0.999, 1e-8, step)
+        got = L.model.master.cpu().numpy()
+        assert rel_l2(got, th) <= ADAM_TOL
+        assert rel_l2(got - theta, th - theta) <= ADAM_TOL, "the update itself, not just theta"
+        assert rel_l2(L.model.adam_m.cpu().numpy(), m) <= 1e-5
+        assert rel_l2(L.model.adam_v.cpu().numpy(), v) <= 1e-5
+        sh = L.model.shadow.float().cpu().numpy()
+        want = torch.as_tensor(got).to(torch.bfloat16).float().numpy()
+        assert np.array_equal(sh, want), "shadow must be the bf16 rounding of the new master"
+    assert ppo.ppo_poll_status() == 0
+
+
+@pytest.mark.parametrize("name,microbatch", [("cfg1_twin", 16), ("cfg2_twin", 8)])
+def test_whole_learner_step_parameters_match_oracle(name, microbatch):
+    """GAE -> every minibatch of one epoch (gather, fwd, loss, bwd, Adam): parameters after the last Adam step."""
+    w = SHAPES[name]
+    L, md, lay, theta, roll, action, logp, dev = _setup(w, microbatch, theta_scale_head=20.0)
+    h = L.hyper
+    L.train(dev["last_value"], seed=11)
+    assert ppo.ppo_poll_status() == 0
+    th = theta.astype(np.float64)
+    m, v = np.zeros_like(th), np.zeros_like(th)
+    step = 0
+    for k in range(w.minibatches):
+        _, _, grad, _, _ = _oracle_minibatch(md, lay, th.astype(np.float32), roll, action, logp, w, h, 11, 0, k,
+                                             w.minibatches)
+        step += 1
+        orc.adam(th, m, v, grad, np.float32(h.lr), np.float32(h.beta1), np.float32(h.beta2), np.float32(h.eps), step)
+    got = L.model.master.cpu().numpy()
+    assert rel_l2(got, th) <= ADAM_TOL, rel_l2(got, th)
+    # the first Adam step moves every parameter by ~lr * sign(g): compare the displacement too, loosely
+    assert rel_l2(got - theta, th - theta) <= 0.25, rel_l2(got - theta, th - theta)
+
+
+def test_policy_act_matches_oracle():
+    w = SHAPES["cfg1_twin"]
+    L, md, lay, theta, roll, action, logp, dev = _setup(w, 16, jitter=False)
+    a, lp, val = L.act(dev["depth"][0], dev["proprio"][0], dev["eps"][0])
+    assert rel_l2(a.cpu().numpy(), action[0]) <= ENC_TOL
+    assert np.abs(lp.cpu().numpy() - logp[0]).max() <= 1e-4  # log-prob depends on eps and log-sigma only
+    assert ppo.ppo_poll_status() == 0
