@@ -350,7 +350,7 @@ def oracle_sample_step(w, fields, theta, n_samples):
     g = {"proprio": fields["proprio"][tt, nn], "action": fields["action"][tt, nn], "logp": fields["logp"][tt, nn],
          "adv": adv[tt, nn], "ret": ret[tt, nn]}
     _, out, grad, _, _ = orc.total_loss_and_grad(md, theta, depth, g["proprio"], g["action"], g["logp"], g["adv"],
-                                                 g["ret"], w.clip, 0.5, 0.01)
+                                                 g["ret"], w.clip, 0.5, 0.01, act_bf16=True)
     th = np.asarray(theta, np.float64).copy()
     orc.adam(th, np.zeros_like(th), np.zeros_like(th), grad, 3e-4, 0.9, 0.999, 1e-8, 1)
     t_mb = time.perf_counter() - t0

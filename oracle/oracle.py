@@ -200,8 +200,9 @@ def round_weights(md: ModelDesc, theta) -> np.ndarray:
     return out
 
 
-def encoder_fwd(md: ModelDesc, theta_used, depth, proprio):
-    """depth [B,H,W] (any float type, values exactly representable), proprio [B,P] -> mu [B,A], V [B], acts."""
+def encoder_fwd(md: ModelDesc, theta_used, depth, proprio, act_bf16: bool = False):
+    """depth [B,H,W] (any float type, values exactly representable), proprio [B,P] -> mu [B,A], V [B], acts.
+    act_bf16: round every layer's stored output to bf16 (the next contraction's operand)."""
     depth = _f64(depth)
     proprio = _f64(proprio)
     theta_used = _f64(theta_used)
@@ -210,7 +211,8 @@ def encoder_fwd(md: ModelDesc, theta_used, depth, proprio):
     mu = np.empty((B, md.A), np.float64)
     V = np.empty((B,), np.float64)
     m = md.c()
-    lib().orc_encoder_fwd(C.byref(m), _p(theta_used), C.c_int(B), _p(depth), _p(proprio), _p(acts), _p(mu), _p(V))
+    lib().orc_encoder_fwd(C.byref(m), _p(theta_used), C.c_int(B), _p(depth), _p(proprio), _p(acts), _p(mu), _p(V),
+                          C.c_int(int(act_bf16)))
     return mu, V, acts
 
 
@@ -267,14 +269,15 @@ def adam(theta, m, v, g, lr, beta1, beta2, eps, step):
 
 # ----------------------------------------------------- composed learner ----
 
-def total_loss_and_grad(md: ModelDesc, theta, depth, proprio, action, logp_old, adv, ret, clip, c_v, c_e):
+def total_loss_and_grad(md: ModelDesc, theta, depth, proprio, action, logp_old, adv, ret, clip, c_v, c_e,
+                        act_bf16: bool = False):
     """One minibatch: L = L_pi + c_v L_V - c_e H and dL/dtheta (w.r.t. the fp32 master, straight through the
-    bf16 rounding of the weight matrices).  Returns (L, out[5], grad, mu, V)."""
+    bf16 rounding of the weight matrices and, with act_bf16, of the activations).  Returns (L, out[5], grad, mu, V)."""
     lay = param_layout(md)
     theta = _f64(theta)
     used = round_weights(md, theta)
     logsigma = theta[lay.offsets[-1]: lay.offsets[-1] + md.A]
-    mu, V, acts = encoder_fwd(md, used, depth, proprio)
+    mu, V, acts = encoder_fwd(md, used, depth, proprio, act_bf16)
     out, dmu, dV, dls = loss(mu, V, logsigma, action, logp_old, adv, ret, clip, c_v, c_e)
     grad = encoder_bwd(md, used, acts, dmu, dV)
     grad[lay.offsets[-1]: lay.offsets[-1] + md.A] += dls

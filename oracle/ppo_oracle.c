@@ -8,9 +8,15 @@
  * the CUDA path, and nothing in the product may call it.
  *
  * Arithmetic is fp64 throughout.  The only places where a narrower precision is
- * part of the definition are: weight matrices are rounded to bf16 (round to
- * nearest even) before use; depth pixels arrive as fp16 values (exactly
- * representable in fp64); the outputs of Adam are rounded to fp32.
+ * part of the definition are: the operands of every layer's contraction are bf16
+ * values (weight matrices are rounded to bf16, round to nearest even, and with
+ * act_bf16 != 0 every layer's output is rounded to bf16 before the next layer
+ * reads it), while sums are kept in fp64; depth pixels arrive as fp16 values
+ * (exactly representable in fp64); the outputs of Adam are rounded to fp32.
+ * Rounding the activations matters for more than accuracy: the ReLU gate
+ * (output > 0) is a discrete decision, and it has to be taken on the same values
+ * on both sides of a comparison.  The backward pass treats every rounding as the
+ * identity (straight through) and rounds nothing itself.
  *
  * Every function states the passage it follows.  The paper itself gives
  * TrainPPO only by name (Algorithm 2; Section III-C: "PPO", "CNN ... ReLU");
@@ -251,9 +257,11 @@ int64_t orc_act_stride(const orc_model *m) {
  *   conv: y[oh][ow][co] = ReLU(b[co] + sum_{kh,kw,ci} W[co][kh][kw][ci] * x[2*oh+kh-p][2*ow+kw-p][ci])
  *         (cross-correlation, zero outside the image, p = k/2)
  *   g = mean of the last conv output over its pixels; h_0 = [g, proprio]
- *   h_l = ReLU(W_l h_{l-1} + b_l);  out = W_head h_F + b_head; mu = out[0..A), V = out[A]. */
+ *   h_l = ReLU(W_l h_{l-1} + b_l);  out = W_head h_F + b_head; mu = out[0..A), V = out[A].
+ * With act_bf16 != 0 every conv output, h_0 and every hidden h_l is rounded to bf16 where it
+ * is stored (the next layer's operand); the head output is not rounded. */
 static void fwd_one(const orc_model *m, const double *th, const int64_t *offs, const double *depth,
-                    const double *proprio, double *act, double *mu, double *V) {
+                    const double *proprio, double *act, double *mu, double *V, int act_bf16) {
     int32_t Ho[ORC_MAX_CONV], Wo[ORC_MAX_CONV];
     orc_conv_shapes(m, Ho, Wo);
     double *x = act;
@@ -280,7 +288,8 @@ static void fwd_one(const orc_model *m, const double *th, const int64_t *offs, c
                             for (int ci = 0; ci < cin; ++ci) acc += wp[ci] * xp[ci];
                         }
                     }
-                    y[((int64_t)oh * Wo[l] + ow) * co_n + co] = acc > 0.0 ? acc : 0.0;
+                    acc = acc > 0.0 ? acc : 0.0;
+                    y[((int64_t)oh * Wo[l] + ow) * co_n + co] = act_bf16 ? orc_round_bf16(acc) : acc;
                 }
         x = y;
         hin = Ho[l];
@@ -293,8 +302,9 @@ static void fwd_one(const orc_model *m, const double *th, const int64_t *offs, c
         double s = 0.0;
         for (int px = 0; px < hin * win; ++px) s += x[(int64_t)px * cin + c];
         h[c] = s / (double)(hin * win);
+        if (act_bf16) h[c] = orc_round_bf16(h[c]);
     }
-    for (int j = 0; j < m->P; ++j) h[cin + j] = proprio[j];
+    for (int j = 0; j < m->P; ++j) h[cin + j] = act_bf16 ? orc_round_bf16(proprio[j]) : proprio[j];
     int in = cin + m->P;
     for (int l = 0; l < m->n_fc; ++l) {
         const double *Wt = th + offs[ti], *b = th + offs[ti + 1];
@@ -303,7 +313,8 @@ static void fwd_one(const orc_model *m, const double *th, const int64_t *offs, c
         for (int o = 0; o < m->fc[l]; ++o) {
             double acc = b[o];
             for (int i = 0; i < in; ++i) acc += Wt[(int64_t)o * in + i] * h[i];
-            y[o] = acc > 0.0 ? acc : 0.0;
+            acc = acc > 0.0 ? acc : 0.0;
+            y[o] = act_bf16 ? orc_round_bf16(acc) : acc;
         }
         h = y;
         in = m->fc[l];
@@ -434,7 +445,7 @@ int64_t orc_bwd_scratch_len(const orc_model *m) {
 /* Forward of B samples.  theta_used: parameter vector with weight matrices already
  * bf16-rounded (orc_round_weights).  acts: B * orc_act_stride doubles (kept for backward). */
 void orc_encoder_fwd(const orc_model *m, const double *theta_used, int B, const double *depth, const double *proprio,
-                     double *acts, double *mu, double *V) {
+                     double *acts, double *mu, double *V, int act_bf16) {
     int64_t offs[2 * ORC_MAX_CONV + 2 * ORC_MAX_FC + 3], szs[2 * ORC_MAX_CONV + 2 * ORC_MAX_FC + 3];
     int32_t mat[2 * ORC_MAX_CONV + 2 * ORC_MAX_FC + 3], n;
     orc_param_layout(m, offs, szs, mat, &n);
@@ -442,7 +453,7 @@ void orc_encoder_fwd(const orc_model *m, const double *theta_used, int B, const 
 #pragma omp parallel for schedule(dynamic)
     for (int b = 0; b < B; ++b)
         fwd_one(m, theta_used, offs, depth + (int64_t)b * m->H * m->W, proprio + (int64_t)b * m->P,
-                acts + b * stride, mu + (int64_t)b * m->A, V + b);
+                acts + b * stride, mu + (int64_t)b * m->A, V + b, act_bf16);
 }
 
 /* Backward of B samples: grad (length = parameter vector) += sum over samples of the

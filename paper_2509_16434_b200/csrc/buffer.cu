@@ -413,25 +413,27 @@ struct GatherArgs {
     uint32_t *o_index;
     uint32_t start;      // first position of this minibatch in the permuted order
     uint32_t rows;       // B
-    uint32_t frame16;    // frame bytes / 16
+    uint32_t frame16;    // frame length in copy units (16 B, or 2 B for odd frame sizes)
     uint32_t chunks;     // CTAs per row
     int P, A;
 };
 
 // One CTA copies one chunk of one row's depth frame with 128-bit loads (no L1 allocation,
-// evict-first) and streaming stores; chunk 0 also copies the row's small fields.
+// evict-first) and streaming stores; chunk 0 also copies the row's small fields.  VecT is
+// uint4 when the frame size is a multiple of 16 bytes, else uint16_t (one fp16 pixel).
+template <typename VecT>
 __global__ void __launch_bounds__(256) gather_kernel(GatherArgs g, PermParams p) {
     const uint32_t row = blockIdx.x / g.chunks;
     const uint32_t chunk = blockIdx.x - row * g.chunks;
     const uint32_t s = perm_apply(p, g.start + row);
-    const uint4 *src = reinterpret_cast<const uint4 *>(g.depth) + (size_t)s * g.frame16;
-    uint4 *dst = reinterpret_cast<uint4 *>(g.o_depth) + (size_t)row * g.frame16;
+    const VecT *src = reinterpret_cast<const VecT *>(g.depth) + (size_t)s * g.frame16;
+    VecT *dst = reinterpret_cast<VecT *>(g.o_depth) + (size_t)row * g.frame16;
     const uint32_t per = (g.frame16 + g.chunks - 1) / g.chunks;
     const uint32_t lo = chunk * per;
     const uint32_t hi = min(lo + per, g.frame16);
     uint32_t i = lo + threadIdx.x;
     for (; i + 3 * 256 < hi; i += 4 * 256) {
-        uint4 a = __ldcs(src + i), b = __ldcs(src + i + 256), c = __ldcs(src + i + 512), d = __ldcs(src + i + 768);
+        VecT a = __ldcs(src + i), b = __ldcs(src + i + 256), c = __ldcs(src + i + 512), d = __ldcs(src + i + 768);
         __stcs(dst + i, a);
         __stcs(dst + i + 256, b);
         __stcs(dst + i + 512, c);
@@ -464,7 +466,7 @@ extern "C" int ppo_shuffle_gather_minibatch(const ppo_buffer *b, uint64_t seed, 
     if (!ppo_aligned(out->depth_f16, 16)) return PPO_ERR_ALIGN;
     if (!b->gae_valid) return PPO_ERR_STATE;
     const size_t frame = (size_t)b->d.H * b->d.W * 2;
-    if (frame % 16 != 0) return PPO_ERR_UNSUPPORTED;
+    const bool vec16 = frame % 16 == 0;
     if (b->d.P > 64 || b->d.A > 64) return PPO_ERR_UNSUPPORTED;
     GatherArgs g;
     g.depth = b->base + b->field_off[PPO_FIELD_DEPTH];
@@ -484,7 +486,7 @@ extern "C" int ppo_shuffle_gather_minibatch(const ppo_buffer *b, uint64_t seed, 
     g.o_index = out->index;
     g.start = (uint32_t)(mb_index * B);
     g.rows = (uint32_t)B;
-    g.frame16 = (uint32_t)(frame / 16);
+    g.frame16 = (uint32_t)(vec16 ? frame / 16 : frame / 2);
     // 16 KB per CTA: 4 x 128-bit per thread, so a frame of 38 400 B becomes 3 CTAs
     g.chunks = (uint32_t)((frame + 16383) / 16384);
     g.P = b->d.P;
@@ -492,7 +494,8 @@ extern "C" int ppo_shuffle_gather_minibatch(const ppo_buffer *b, uint64_t seed, 
     const long long ctas = B * g.chunks;
     if (ctas > 0x7fffffffll) return PPO_ERR_UNSUPPORTED;
     PermParams p = make_perm(seed, epoch, (uint32_t)M);
-    gather_kernel<<<(unsigned)ctas, 256, 0, static_cast<cudaStream_t>(stream)>>>(g, p);
+    if (vec16) gather_kernel<uint4><<<(unsigned)ctas, 256, 0, static_cast<cudaStream_t>(stream)>>>(g, p);
+    else gather_kernel<uint16_t><<<(unsigned)ctas, 256, 0, static_cast<cudaStream_t>(stream)>>>(g, p);
     PPO_LAUNCH_CHECK();
     return PPO_OK;
 }

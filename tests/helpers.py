@@ -29,7 +29,7 @@ def oracle_rollout_actions(md, theta, roll):
     T, N = roll["reward"].shape
     depth = roll["depth"].reshape(T * N, md.H, md.W)
     proprio = roll["proprio"].reshape(T * N, md.P)
-    mu, V, _ = orc.encoder_fwd(md, used, depth, proprio)
+    mu, V, _ = orc.encoder_fwd(md, used, depth, proprio, True)
     ls = np.asarray(theta, np.float64)[lay.offsets[-1]:lay.offsets[-1] + md.A]
     action, logp = orc.sample_action(mu, ls, roll["eps"].reshape(T * N, md.A))
     return (action.astype(np.float32).reshape(T, N, md.A), logp.astype(np.float32).reshape(T, N))

@@ -50,7 +50,8 @@ def _oracle_minibatch(md, lay, theta, roll, action, logp, w, hyper, seed, epoch,
                     "adv": adv.astype(np.float32), "ret": ret.astype(np.float32)}, idx, w.N)
     Ltot, out, grad, mu, V = orc.total_loss_and_grad(md, theta, f["depth"], f["proprio"], f["action"], f["logp"],
                                                      f["adv"], f["ret"], np.float32(hyper.clip),
-                                                     np.float32(hyper.vf_coef), np.float32(hyper.ent_coef))
+                                                     np.float32(hyper.vf_coef), np.float32(hyper.ent_coef),
+                                                     act_bf16=True)
     return f, out, grad, mu, V
 
 
@@ -104,7 +105,7 @@ def test_minibatch_forward_loss_backward_match_oracle(name, microbatch):
     for j, tol in [(0, 2e-2), (1, 2e-2), (3, 2e-2)]:
         assert abs(out[j] - out_o[j]) <= tol * max(abs(out_o[j]), 0.05), (j, out[j], out_o[j])
     assert abs(out[4] - out_o[4]) <= 2.0 / B + 1e-6
-    _check_grads(lay, L.model.grad.cpu().numpy(), grad_o, tol=3e-2)
+    _check_grads(lay, L.model.grad.cpu().numpy(), grad_o)
 
 
 def test_loss_kernel_alone_matches_oracle_to_1e3():

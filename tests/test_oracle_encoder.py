@@ -24,7 +24,14 @@ def _theta(md, seed, bias_scale=0.1):
     return th, lay
 
 
-def _torch_forward(md, lay, th, depth, proprio):
+def _rnd(x, on):
+    """bf16 rounding with a straight-through gradient."""
+    if not on:
+        return x
+    return x + (x.detach().to(torch.float32).to(torch.bfloat16).to(torch.float64) - x.detach())
+
+
+def _torch_forward(md, lay, th, depth, proprio, act_bf16=False):
     """The same network written with torch library ops in fp64 (conv2d is cross-correlation)."""
     t = torch.tensor(th, dtype=torch.float64, requires_grad=True)
     x = torch.tensor(depth, dtype=torch.float64)[:, None]  # NCHW
@@ -33,13 +40,13 @@ def _torch_forward(md, lay, th, depth, proprio):
         shp = lay.shapes[i]
         Wt = t[lay.offsets[i]:lay.offsets[i] + lay.sizes[i]].reshape(shp).permute(0, 3, 1, 2)  # [Co,kh,kw,Ci] -> OIHW
         b = t[lay.offsets[i + 1]:lay.offsets[i + 1] + co]
-        x = F.relu(F.conv2d(x, Wt, b, stride=2, padding=k // 2))
+        x = _rnd(F.relu(F.conv2d(x, Wt, b, stride=2, padding=k // 2)), act_bf16)
         i += 2
-    h = torch.cat([x.mean(dim=(2, 3)), torch.tensor(proprio, dtype=torch.float64)], 1)
+    h = _rnd(torch.cat([x.mean(dim=(2, 3)), torch.tensor(proprio, dtype=torch.float64)], 1), act_bf16)
     for o in md.fc:
         Wt = t[lay.offsets[i]:lay.offsets[i] + lay.sizes[i]].reshape(lay.shapes[i])
         b = t[lay.offsets[i + 1]:lay.offsets[i + 1] + o]
-        h = F.relu(F.linear(h, Wt, b))
+        h = _rnd(F.relu(F.linear(h, Wt, b)), act_bf16)
         i += 2
     Wt = t[lay.offsets[i]:lay.offsets[i] + lay.sizes[i]].reshape(lay.shapes[i])
     b = t[lay.offsets[i + 1]:lay.offsets[i + 1] + md.A + 1]
@@ -47,8 +54,9 @@ def _torch_forward(md, lay, th, depth, proprio):
     return t, out[:, :md.A], out[:, md.A]
 
 
+@pytest.mark.parametrize("act_bf16", [False, True])
 @pytest.mark.parametrize("md", [TINY, TINY5, orc.ModelDesc(16, 16, (4, 8, 8), (3, 3, 3), (16,), 4, 3)])
-def test_forward_and_backward_match_torch_autograd(md):
+def test_forward_and_backward_match_torch_autograd(md, act_bf16):
     """Catches: kernel flip, wrong padding/stride/output size, wrong weight index order, wrong pool divisor,
     concat order, transposed FC weights, missing ReLU mask in the backward."""
     th, lay = _theta(md, 3)
@@ -56,8 +64,14 @@ def test_forward_and_backward_match_torch_autograd(md):
     B = 3
     depth = g.uniform(0.1, 2.0, (B, md.H, md.W))
     proprio = g.standard_normal((B, md.P))
-    mu, V, acts = orc.encoder_fwd(md, th, depth, proprio)
-    t, mu_t, V_t = _torch_forward(md, lay, th, depth, proprio)
+    mu, V, acts = orc.encoder_fwd(md, th, depth, proprio, act_bf16)
+    t, mu_t, V_t = _torch_forward(md, lay, th, depth, proprio, act_bf16)
+    if act_bf16:  # rounding is on: the stored activations are bf16 values and differ from the unrounded run
+        mu_u, _, acts_u = orc.encoder_fwd(md, th, depth, proprio, False)
+        n_img = md.H * md.W
+        a = acts[:, n_img:]
+        assert np.array_equal(a, torch.tensor(a).to(torch.bfloat16).to(torch.float64).numpy())
+        assert not np.array_equal(acts, acts_u) and 0 < np.abs(mu - mu_u).max() < 0.05 * np.abs(mu_u).max()
     assert np.allclose(mu, mu_t.detach().numpy(), atol=1e-12)
     assert np.allclose(V, V_t.detach().numpy(), atol=1e-12)
     dmu = g.standard_normal(mu.shape)
