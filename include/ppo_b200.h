@@ -210,6 +210,13 @@ int ppo_loss_fwd_bwd(ppo_model *m, const ppo_minibatch *mb, int row0, int rows, 
 int ppo_encoder_bwd(ppo_model *m, const ppo_minibatch *mb, int row0, int rows, const float *dev_dmean,
                     const float *dev_dvalue, int accumulate, void *stream);
 
+/* Where the forward keeps what the backward reads (inside the bound workspace): kind 0 =
+ * conv activation of layer `index` in 1..n_conv, NHWC bf16 [rows][Ho][Wo][C]; kind 1 = h_index
+ * for index in 0..n_fc, bf16 [rows][width] (h_0 = [pooled, proprio]).  *elems is the capacity
+ * for the bound micro-batch.  For inspection and for tests that substitute the saved
+ * activations between ppo_encoder_fwd and ppo_encoder_bwd. */
+int ppo_model_activation_ptr(const ppo_model *m, int kind, int index, void **dev_ptr, size_t *elems);
+
 /* Zeroes the bound gradient array (start of a minibatch). */
 int ppo_model_zero_grad(ppo_model *m, void *stream);
 

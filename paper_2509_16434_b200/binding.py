@@ -26,7 +26,7 @@ EXPORTS = [
     "ppo_model_create", "ppo_model_destroy", "ppo_model_param_count", "ppo_model_arena_elems",
     "ppo_model_num_tensors", "ppo_model_tensor_info", "ppo_model_workspace_bytes", "ppo_model_bind",
     "ppo_model_sync_shadow", "ppo_encoder_fwd", "ppo_loss_fwd_bwd", "ppo_encoder_bwd", "ppo_model_zero_grad",
-    "ppo_adam_step", "ppo_policy_sample", "ppo_poll_status",
+    "ppo_adam_step", "ppo_policy_sample", "ppo_poll_status", "ppo_model_activation_ptr",
 ]
 
 
@@ -98,6 +98,8 @@ def lib():
         L.ppo_policy_sample.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
                                         C.c_void_p]
         L.ppo_poll_status.argtypes = [C.c_void_p]
+        L.ppo_model_activation_ptr.argtypes = [C.c_void_p, C.c_int, C.c_int, C.POINTER(C.c_void_p),
+                                               C.POINTER(C.c_size_t)]
         _lib = L
     return _lib
 
@@ -273,6 +275,14 @@ class Model:
             _check(lib().ppo_model_tensor_info(self.handle, i, C.byref(off), C.byref(sz)), "ppo_model_tensor_info")
             out.append((off.value, sz.value))
         return out
+
+    def activation(self, kind: int, index: int) -> torch.Tensor:
+        """A flat bf16 torch view of a saved activation inside the workspace (see ppo_model_activation_ptr)."""
+        p, n = C.c_void_p(), C.c_size_t()
+        _check(lib().ppo_model_activation_ptr(self.handle, kind, index, C.byref(p), C.byref(n)),
+               "ppo_model_activation_ptr")
+        off = p.value - self.workspace.data_ptr()
+        return self.workspace[off:off + 2 * n.value].view(torch.bfloat16)
 
     def load(self, theta, stream=None):
         """Copies an fp32 parameter vector (numpy or torch, arena layout) into master and refreshes the shadow."""

@@ -162,6 +162,22 @@ extern "C" int ppo_model_bind(ppo_model *m, float *master, void *shadow, float *
     return PPO_OK;
 }
 
+extern "C" int ppo_model_activation_ptr(const ppo_model *m, int kind, int index, void **ptr, size_t *elems) {
+    if (!m || !ptr || !elems) return PPO_ERR_INVALID_ARG;
+    if (!m->ws) return PPO_ERR_STATE;
+    if (kind == 0 && index >= 1 && index <= m->L) {
+        *ptr = m->act[index];
+        *elems = (size_t)m->mbmax * m->Hs[index] * m->Ws[index] * m->Cs[index];
+        return PPO_OK;
+    }
+    if (kind == 1 && index >= 0 && index <= m->F) {
+        *ptr = m->h[index];
+        *elems = (size_t)m->mbmax * m->hw[index];
+        return PPO_OK;
+    }
+    return PPO_ERR_INVALID_ARG;
+}
+
 // ------------------------------------------------------------ shadow / zero ----
 
 __global__ void __launch_bounds__(256) shadow_kernel(const float4 *__restrict__ master, uint2 *__restrict__ shadow,

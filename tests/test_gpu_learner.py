@@ -14,6 +14,14 @@ DEV = "cuda"
 ENC_TOL = 2e-2    # relative L2: bf16 operands / activations with fp32 accumulation vs fp64
 LOSS_TOL = 1e-3   # relative error of the loss scalars
 ADAM_TOL = 1e-3   # relative L2 of the parameters after one step
+# End-to-end gradients (GPU forward feeding GPU backward) against the oracle's own forward+backward: a stored activation
+# that lands on the other side of a bf16 rounding boundary (fp32 vs fp64 sums) moves downstream pre-activations by
+# ~1e-4 relative, which flips the ReLU gate of the ~1e-4 fraction of units sitting that close to zero; each flipped
+# gate changes that unit's gradient by its full size, so the relative L2 error of a gradient is ~sqrt(flipped
+# fraction / active fraction) ~ 1-2 % per layer it passes through, not ~eps.  The backward operator itself is
+# held to ENC_TOL in the test that gives both sides identical saved activations.
+E2E_GRAD_TOL_TOTAL = 1e-1
+E2E_GRAD_TOL_TENSOR = 2e-1
 
 
 def _setup(w, microbatch, seed=0, jitter=True, theta_scale_head=1.0):
@@ -55,11 +63,54 @@ def _oracle_minibatch(md, lay, theta, roll, action, logp, w, hyper, seed, epoch,
     return f, out, grad, mu, V
 
 
-def _check_grads(lay, got, want, tol=ENC_TOL):
+def _check_grads(lay, got, want, tol=ENC_TOL, tol_total=None):
     for i, (off, sz) in enumerate(zip(lay.offsets, lay.sizes)):
         e = rel_l2(got[off:off + sz], want[off:off + sz])
         assert e <= tol, f"tensor {i}: rel L2 {e:.3e}"
-    assert rel_l2(got, want) <= tol
+    assert rel_l2(got, want) <= (tol if tol_total is None else tol_total)
+
+
+def _upload_oracle_activations(L, md, acts, B):
+    """Replaces the activations the GPU forward saved by the oracle's (bf16 values), layer by layer."""
+    Ho, Wo = orc.conv_shapes(md)
+    off = md.H * md.W
+    for l, (h, w_, c) in enumerate(zip(Ho, Wo, md.conv_c), start=1):
+        n = h * w_ * c
+        L.model.activation(0, l)[:B * n].copy_(torch.as_tensor(acts[:, off:off + n].reshape(-1)).to(torch.bfloat16))
+        off += n
+    widths = [md.conv_c[-1] + md.P] + list(md.fc)
+    for l, n in enumerate(widths):
+        L.model.activation(1, l)[:B * n].copy_(torch.as_tensor(acts[:, off:off + n].reshape(-1)).to(torch.bfloat16))
+        off += n
+    assert off == acts.shape[1]
+
+
+@pytest.mark.parametrize("name", ["tiny", "odd", "cfg1_twin", "cfg2_twin", "cfg4_twin"])
+def test_backward_matches_oracle_on_identical_activations(name):
+    """The backward operator alone: both sides start from the oracle's saved activations, mean and value."""
+    w = SHAPES[name]
+    B = w.M // w.minibatches
+    L, md, lay, theta, roll, action, logp, dev = _setup(w, B, theta_scale_head=20.0)
+    h = L.hyper
+    K = w.minibatches
+    L.compute_gae(dev["last_value"])
+    f, out_o, grad_o, mu_o, V_o = _oracle_minibatch(md, lay, theta, roll, action, logp, w, h, 5, 0, 0, K)
+    _, _, acts = orc.encoder_fwd(md, orc.round_weights(md, theta), f["depth"], f["proprio"], True)
+    ppo.ppo_shuffle_gather_minibatch(L.buffer, 5, 0, 0, K, L.mb)
+    ppo.ppo_model_zero_grad(L.model)
+    L.loss.zero_()
+    ppo.ppo_encoder_fwd(L.model, L.mb, 0, B, L.mean, L.value)
+    _upload_oracle_activations(L, md, acts, B)
+    L.mean[:B].copy_(torch.as_tensor(mu_o, dtype=torch.float32))
+    L.value[:B].copy_(torch.as_tensor(V_o, dtype=torch.float32))
+    ppo.ppo_loss_fwd_bwd(L.model, L.mb, 0, B, B, L.mean, L.value, h.clip, h.vf_coef, h.ent_coef, L.loss, L.dmean,
+                         L.dvalue)
+    ppo.ppo_encoder_bwd(L.model, L.mb, 0, B, L.dmean, L.dvalue, True)
+    assert ppo.ppo_poll_status() == 0
+    out = L.loss.cpu().numpy()
+    for j in range(5):
+        assert abs(out[j] - out_o[j]) <= LOSS_TOL * max(abs(out_o[j]), 1e-2), (j, out[j], out_o[j])
+    _check_grads(lay, L.model.grad.cpu().numpy(), grad_o)
 
 
 SHAPES = {
@@ -105,7 +156,7 @@ def test_minibatch_forward_loss_backward_match_oracle(name, microbatch):
     for j, tol in [(0, 2e-2), (1, 2e-2), (3, 2e-2)]:
         assert abs(out[j] - out_o[j]) <= tol * max(abs(out_o[j]), 0.05), (j, out[j], out_o[j])
     assert abs(out[4] - out_o[4]) <= 2.0 / B + 1e-6
-    _check_grads(lay, L.model.grad.cpu().numpy(), grad_o)
+    _check_grads(lay, L.model.grad.cpu().numpy(), grad_o, E2E_GRAD_TOL_TENSOR, E2E_GRAD_TOL_TOTAL)
 
 
 def test_loss_kernel_alone_matches_oracle_to_1e3():
