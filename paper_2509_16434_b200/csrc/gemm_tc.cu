@@ -1,12 +1,651 @@
-// placeholder: tensor-core GEMMs (forwarding to the CUDA-core kernels until they land)
+// Tensor-core versions of the encoder's implicit GEMMs for sm_100a: tcgen05.mma with the
+// accumulator in tensor memory (TMEM), operands gathered into 128-byte-swizzled shared
+// memory by cp.async, an mbarrier ring between the gather warps and the MMA-issuing warp,
+// and a tcgen05.ld epilogue.  Every wait is bounded: on a time-out the kernel records
+// PPO_ERR_TIMEOUT, drains its copies, frees its TMEM and returns.
+//
+//  igemm_kmajor_kernel : D[m][n] = sum_k A[m][k] B[n][k], both operands K-major.
+//      forward  A = im2col(X) (row m = output pixel), B = W[co][tap][ci]
+//      dgrad    A = gathered dY (row m = input pixel of one stride-parity class), B = Wt[ci][tap][co]
+//  igemm_wgrad_kernel  : D[j][co] = sum_m A[m][j] B[m][co], both operands MN-major (the reduction
+//      index m is the slow one in memory), split over m across CTAs, fp32 atomics into dW.
+//
+// Shared-memory operand image (both kernels): rows of 128 bytes (64 bf16), the 16-byte chunk c
+// of row r stored at chunk position c ^ (r & 7) -- the SWIZZLE_128B pattern the UMMA shared
+// memory descriptors name.  Read K-major, a row is one M/N index and its 64 columns are K; read
+// MN-major, a row is one K index and its 64 columns are M/N.
 #include "gemm.cuh"
-int tc_gemm_fwd(const ConvGeom &g, const bf16 *X, const bf16 *W, const FwdEpilogue &e, int32_t *, cudaStream_t st) {
-    return simt_gemm_fwd(g, X, W, e, st);
+
+namespace {
+
+constexpr int kStages = 4;
+constexpr int kLag = 2;               // cp.async groups in flight per producer thread
+constexpr int kProducers = 128;       // 4 warps: gather, then epilogue
+constexpr int kThreads = 160;         // + 1 warp issuing the MMAs
+constexpr int kMaxTaps = 49;
+constexpr long long kWaitCycles = 4000000000ll;  // ~2 s at 2 GHz
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint64_t *bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
 }
-int tc_gemm_dgrad(const ConvGeom &, const bf16 *, int, const bf16 *, int, const DgradEpilogue &, int32_t *,
-                  cudaStream_t) {
-    return PPO_ERR_UNSUPPORTED;
+__device__ __forceinline__ void mbar_arrive(uint64_t *bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
-int tc_gemm_wgrad(const ConvGeom &g, const bf16 *dY, int ldy, const bf16 *X, float *dW, int32_t *, cudaStream_t st) {
-    return simt_gemm_wgrad(g, dY, ldy, X, dW, st);
+__device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Bounded wait; returns false when this or another thread of the CTA gave up.
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag, int32_t *status) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    while (!mbar_try_wait(bar, parity)) {
+        if (*abort_flag) return false;
+        if (clock64() - t0 > kWaitCycles) {
+            *abort_flag = 1;
+            ppo_report(status, PPO_ERR_TIMEOUT);
+            return false;
+        }
+    }
+    return true;
+}
+
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void *src, bool valid) {
+    const uint32_t n = valid ? 16u : 0u;  // 0 source bytes: the 16 destination bytes are zero-filled
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(n) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() {
+    asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
+}
+// Makes this thread's completed generic-proxy writes to shared memory visible to the async
+// proxy (the tensor core reads operands through it).
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tmem_alloc(uint32_t *slot, uint32_t ncols) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(slot)), "r"(ncols)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t addr, uint32_t ncols) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(addr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint64_t *bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
+                 : "memory");
+}
+// D[tmem] (+)= A[smem desc] * B[smem desc], bf16 operands, fp32 accumulate.
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                          uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// 16 consecutive fp32 columns of this thread's TMEM lane.
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float *v) {
+    uint32_t r[16];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, "
+        "%15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr)
+        : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+// Shared-memory matrix descriptor for the SWIZZLE_128B image: start address, leading and
+// stride byte offsets (each >> 4), descriptor version 1 (bit 46), layout type 2 (bits 61-63).
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+    return (uint64_t)((addr >> 4) & 0x3FFFu) | ((uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16) |
+           ((uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32) | (1ull << 46) | (2ull << 61);
+}
+// Instruction descriptor, kind::f16: D fp32 (bits 4-5 = 1), A and B bf16 (bits 7-9, 10-12 = 1),
+// operand majors (bit 15, 16: 0 = K-major, 1 = MN-major), N >> 3 (bits 17-22), M >> 4 (bits 24-28).
+__host__ __device__ constexpr uint32_t instr_desc(int M, int N, int a_mn, int b_mn) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)a_mn << 15) | ((uint32_t)b_mn << 16) |
+           ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
+}
+
+struct Pipe {  // barrier block at the end of dynamic shared memory
+    uint64_t full[kStages];
+    uint64_t empty[kStages];
+    uint64_t accum;
+    uint32_t tmem_slot;
+    int abort_flag;
+};
+
+__device__ __forceinline__ uint32_t tmem_cols_for(int bn) {
+    uint32_t c = 32;
+    while ((int)c < bn) c <<= 1;
+    return c;
+}
+
+// ------------------------------------------------------------------ K-major ----
+
+struct Taps {
+    int n;                 // taps walked along K
+    int ck;                // 16-byte chunks (8 elements) per tap
+    signed char dy[kMaxTaps], dx[kMaxTaps];
+    short wt[kMaxTaps];    // index of the tap inside the weight tensor
+};
+
+enum { EPI_FWD = 0, EPI_HEAD = 1, EPI_DGRAD = 2 };
+
+struct KArgs {
+    const bf16 *S;         // source [B][Hs][Ws][lds]
+    int Hs, Ws, lds;
+    const bf16 *Wm;        // weights: element (n, tap t, c) at n * w_row + wt[t] * w_tap + c
+    int w_row, w_tap;
+    int Hr, Wr;            // row grid: m = (b * Hr + y) * Wr + x
+    long long Mrows;
+    int s_mul, s_oy, s_ox;  // source pixel of tap t: (y * s_mul + s_oy + dy[t], x * s_mul + s_ox + dx[t])
+    int o_mul, o_oy, o_ox, Hout, Wout;  // output row = (b * Hout + y * o_mul + o_oy) * Wout + x * o_mul + o_ox
+    int N, BN, ldo;
+    int mode, relu, A;
+    const float *bias;
+    bf16 *out;
+    float *out_f32;
+    const bf16 *mask;
+    float *mean, *value;
+    int kchunks;           // taps.n * taps.ck
+    int32_t *status;
+    Taps taps;
+};
+
+__global__ void __launch_bounds__(kThreads) igemm_kmajor_kernel(const __grid_constant__ KArgs a) {
+    extern __shared__ __align__(1024) uint8_t smem_raw[];
+    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    const int BN = a.BN;
+    const uint32_t stage_bytes = 16384u + (uint32_t)BN * 128u;
+    Pipe *pipe = reinterpret_cast<Pipe *>(smem + kStages * stage_bytes);
+    volatile int *abort_flag = &pipe->abort_flag;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t ncols = tmem_cols_for(BN);
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(&pipe->full[s], kProducers);
+            mbar_init(&pipe->empty[s], 1);
+        }
+        mbar_init(&pipe->accum, 1);
+        pipe->abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 4) tmem_alloc(&pipe->tmem_slot, ncols);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_d = pipe->tmem_slot;
+
+    const long long m0 = (long long)blockIdx.x * 128;
+    const int n0 = blockIdx.y * BN;
+    const int nkb = (a.kchunks + 7) >> 3;
+    const uint32_t smem_base = smem_u32(smem);
+
+    if (warp < 4) {
+        // ---------------- gather: thread p owns row p of the A tile and column slot p % 8 of B rows p/8 + 16 i
+        const int p = threadIdx.x;
+        const long long m = m0 + p;
+        const bool row_ok = m < a.Mrows;
+        int y = 0, x = 0;
+        long long b = 0;
+        if (row_ok) {
+            x = (int)(m % a.Wr);
+            const long long t = m / a.Wr;
+            y = (int)(t % a.Hr);
+            b = t / a.Hr;
+        }
+        const int sy0 = y * a.s_mul + a.s_oy, sx0 = x * a.s_mul + a.s_ox;
+        const bf16 *src_img = a.S + b * a.Hs * a.Ws * a.lds;
+        int tA = 0, cA = 0;                 // walk of the A chunks: tap, chunk inside tap
+        const int jB = p & 7;
+        int tB = jB / a.taps.ck, cB = jB % a.taps.ck;
+        const int nB = BN >> 4;             // B chunks per thread per K block
+        bool ok = true;
+        for (int kb = 0; kb < nkb && ok; ++kb) {
+            const int s = kb % kStages;
+            if (kb >= kStages) ok = mbar_wait(&pipe->empty[s], ((kb / kStages) - 1) & 1, abort_flag, a.status);
+            if (!ok) break;
+            const uint32_t sa = smem_base + s * stage_bytes, sb = sa + 16384u;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                bool v = row_ok && tA < a.taps.n;
+                const bf16 *src = a.S;
+                if (v) {
+                    const int yy = sy0 + a.taps.dy[tA], xx = sx0 + a.taps.dx[tA];
+                    v = yy >= 0 && yy < a.Hs && xx >= 0 && xx < a.Ws;
+                    if (v) src = src_img + ((long long)yy * a.Ws + xx) * a.lds + cA * 8;
+                }
+                cp_async16(sa + p * 128 + ((j ^ (p & 7)) << 4), src, v);
+                if (++cA == a.taps.ck) { cA = 0; ++tA; }
+            }
+            {
+                const bool kv = tB < a.taps.n;
+                const long long koff = kv ? (long long)a.taps.wt[tB] * a.w_tap + cB * 8 : 0;
+                for (int i = 0; i < nB; ++i) {
+                    const int n = (p >> 3) + i * 16;
+                    const bool v = kv && (n0 + n) < a.N;
+                    const bf16 *src = v ? a.Wm + (long long)(n0 + n) * a.w_row + koff : a.Wm;
+                    cp_async16(sb + n * 128 + ((jB ^ (n & 7)) << 4), src, v);
+                }
+                cB += 8;
+                while (cB >= a.taps.ck) { cB -= a.taps.ck; ++tB; }
+            }
+            cp_async_commit();
+            if (kb >= kLag) {
+                cp_async_wait<kLag>();
+                fence_async_smem();
+                mbar_arrive(&pipe->full[(kb - kLag) % kStages]);
+            }
+        }
+        cp_async_wait<0>();
+        fence_async_smem();
+        if (ok)
+            for (int kb = (nkb > kLag ? nkb - kLag : 0); kb < nkb; ++kb) mbar_arrive(&pipe->full[kb % kStages]);
+
+        // ---------------- epilogue: thread p reads TMEM lane p
+        if (ok) ok = mbar_wait(&pipe->accum, 0, abort_flag, a.status);
+        tc_fence_after();
+        if (ok) {
+            const long long orow = (b * a.Hout + (long long)y * a.o_mul + a.o_oy) * a.Wout + (long long)x * a.o_mul + a.o_ox;
+            const uint32_t lane_base = tmem_d + ((uint32_t)(warp * 32) << 16);
+            for (int c0 = 0; c0 < BN; c0 += 16) {
+                if (n0 + c0 >= a.N) break;  // uniform across the warp
+                float v[16];
+                if (nkb > 0) {
+                    tmem_ld16(lane_base + (uint32_t)c0, v);
+                } else {  // empty reduction: the accumulator was never written
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) v[i] = 0.f;
+                }
+                if (!row_ok) continue;
+                const int n = n0 + c0;
+                if (a.mode == EPI_HEAD) {
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) {
+                        if (n + i < a.A) a.mean[m * a.A + n + i] = v[i] + a.bias[n + i];
+                        else if (n + i == a.A) a.value[m] = v[i] + a.bias[n + i];
+                    }
+                    continue;
+                }
+                if (a.mode == EPI_FWD) {
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) {
+                        const float bv = (n + i < a.N) ? a.bias[n + i] : 0.f;
+                        v[i] += bv;
+                        if (a.relu) v[i] = fmaxf(v[i], 0.f);
+                    }
+                } else if (a.mask) {
+                    const uint4 *mp = reinterpret_cast<const uint4 *>(a.mask + orow * a.ldo + n);
+#pragma unroll
+                    for (int hlf = 0; hlf < 2; ++hlf) {
+                        if (n + hlf * 8 < a.N) {
+                            const uint4 mk = mp[hlf];
+                            const __nv_bfloat162 *m2 = reinterpret_cast<const __nv_bfloat162 *>(&mk);
+#pragma unroll
+                            for (int i = 0; i < 4; ++i) {
+                                const float2 f = __bfloat1622float2(m2[i]);
+                                if (!(f.x > 0.f)) v[hlf * 8 + 2 * i] = 0.f;
+                                if (!(f.y > 0.f)) v[hlf * 8 + 2 * i + 1] = 0.f;
+                            }
+                        }
+                    }
+                }
+                if (a.out) {
+                    uint4 *op = reinterpret_cast<uint4 *>(a.out + orow * a.ldo + n);
+#pragma unroll
+                    for (int hlf = 0; hlf < 2; ++hlf) {
+                        if (n + hlf * 8 < a.N) {
+                            __nv_bfloat162 pk[4];
+#pragma unroll
+                            for (int i = 0; i < 4; ++i)
+                                pk[i] = __floats2bfloat162_rn(v[hlf * 8 + 2 * i], v[hlf * 8 + 2 * i + 1]);
+                            op[hlf] = *reinterpret_cast<uint4 *>(pk);
+                        }
+                    }
+                }
+                if (a.out_f32) {
+                    float4 *op = reinterpret_cast<float4 *>(a.out_f32 + orow * a.ldo + n);
+#pragma unroll
+                    for (int q = 0; q < 4; ++q)
+                        if (n + q * 4 < a.N) op[q] = make_float4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
+                }
+            }
+        }
+    } else {
+        // ---------------- MMA issue: one thread feeds the tensor core
+        const uint32_t idesc = instr_desc(128, BN, 0, 0);
+        bool ok = true;
+        for (int kb = 0; kb < nkb && ok; ++kb) {
+            const int s = kb % kStages;
+            ok = mbar_wait(&pipe->full[s], (kb / kStages) & 1, abort_flag, a.status);
+            if (!ok) break;
+            tc_fence_after();
+            if (lane == 0) {
+                const uint32_t sa = smem_base + s * stage_bytes, sb = sa + 16384u;
+#pragma unroll
+                for (int k = 0; k < 4; ++k)  // 4 x (K = 16 elements = 32 bytes along the swizzled row)
+                    umma_bf16(tmem_d, smem_desc(sa + k * 32, 16, 1024), smem_desc(sb + k * 32, 16, 1024), idesc,
+                              (kb > 0 || k > 0) ? 1u : 0u);
+                umma_commit(&pipe->empty[s]);
+            }
+            __syncwarp();
+        }
+        if (ok && lane == 0) umma_commit(&pipe->accum);
+        __syncwarp();
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 4) {
+        tc_fence_after();
+        tmem_dealloc(tmem_d, ncols);
+    }
+}
+
+// -------------------------------------------------------------------- wgrad ----
+
+struct WArgs {
+    const bf16 *X;         // [B][Hi][Wi][Ci]
+    int Hi, Wi, Ci, Ho, Wo, ksz, pad;
+    const bf16 *dY;        // [M][ldy]
+    int ldy, Co;
+    long long Mtot;        // B * Ho * Wo
+    long long m_per_split; // multiple of 64
+    int Kfwd;              // ksz * ksz * Ci
+    int BN;
+    float *dW;             // [Co][Kfwd], accumulated with atomics
+    int32_t *status;
+};
+
+__global__ void __launch_bounds__(kThreads) igemm_wgrad_kernel(const __grid_constant__ WArgs a) {
+    extern __shared__ __align__(1024) uint8_t smem_raw[];
+    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    const int BN = a.BN;
+    const int nblkB = (BN + 63) >> 6;
+    const uint32_t stage_bytes = 16384u + (uint32_t)nblkB * 8192u;
+    Pipe *pipe = reinterpret_cast<Pipe *>(smem + kStages * stage_bytes);
+    volatile int *abort_flag = &pipe->abort_flag;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t ncols = tmem_cols_for(BN);
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(&pipe->full[s], kProducers);
+            mbar_init(&pipe->empty[s], 1);
+        }
+        mbar_init(&pipe->accum, 1);
+        pipe->abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 4) tmem_alloc(&pipe->tmem_slot, ncols);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_d = pipe->tmem_slot;
+
+    const int j0 = blockIdx.x * 128;       // tile of the (tap, ci) index
+    const int co0 = blockIdx.y * BN;
+    const long long m_lo = (long long)blockIdx.z * a.m_per_split;
+    const long long m_hi = min(a.Mtot, m_lo + a.m_per_split);
+    const int nkb = (int)((m_hi - m_lo + 63) >> 6);
+    const uint32_t smem_base = smem_u32(smem);
+
+    if (warp < 4) {
+        const int p = threadIdx.x;
+        const int r = p & 63, half = p >> 6;
+        // this thread's 8 A chunks: columns j0 + half*64 + 8 q, fixed for the whole kernel
+        int a_off[8];       // element offset of the chunk inside a source pixel, or -1 when past Kfwd
+        signed char a_dy[8], a_dx[8];
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            const int jj = j0 + half * 64 + q * 8;
+            if (jj < a.Kfwd) {
+                const int t = jj / a.Ci;
+                a_off[q] = jj - t * a.Ci;
+                a_dy[q] = (signed char)(t / a.ksz);
+                a_dx[q] = (signed char)(t % a.ksz);
+            } else {
+                a_off[q] = -1;
+                a_dy[q] = a_dx[q] = 0;
+            }
+        }
+        const int co_lim = min(a.ldy, co0 + BN);  // dY columns that exist in memory for this tile
+        bool ok = true;
+        for (int kb = 0; kb < nkb && ok; ++kb) {
+            const int s = kb % kStages;
+            if (kb >= kStages) ok = mbar_wait(&pipe->empty[s], ((kb / kStages) - 1) & 1, abort_flag, a.status);
+            if (!ok) break;
+            const uint32_t sa = smem_base + s * stage_bytes, sb = sa + 16384u;
+            const long long m = m_lo + (long long)kb * 64 + r;
+            const bool row_ok = m < m_hi;
+            int oh = 0, ow = 0;
+            long long b = 0;
+            if (row_ok) {
+                ow = (int)(m % a.Wo);
+                const long long t = m / a.Wo;
+                oh = (int)(t % a.Ho);
+                b = t / a.Ho;
+            }
+            const int y0 = 2 * oh - a.pad, x0 = 2 * ow - a.pad;
+            const bf16 *img = a.X + b * a.Hi * a.Wi * a.Ci;
+            const uint32_t arow = sa + half * 8192 + r * 128;
+#pragma unroll
+            for (int q = 0; q < 8; ++q) {
+                const int yy = y0 + a_dy[q], xx = x0 + a_dx[q];
+                const bool v = row_ok && a_off[q] >= 0 && yy >= 0 && yy < a.Hi && xx >= 0 && xx < a.Wi;
+                const bf16 *src = v ? img + ((long long)yy * a.Wi + xx) * a.Ci + a_off[q] : a.X;
+                cp_async16(arow + ((q ^ (r & 7)) << 4), src, v);
+            }
+            const bf16 *dyrow = a.dY + m * a.ldy;
+            for (int blk = half; blk < nblkB; blk += 2) {
+                const uint32_t brow = sb + blk * 8192 + r * 128;
+#pragma unroll
+                for (int q = 0; q < 8; ++q) {
+                    const int co = co0 + blk * 64 + q * 8;
+                    const bool v = row_ok && co < co_lim;
+                    cp_async16(brow + ((q ^ (r & 7)) << 4), v ? dyrow + co : a.dY, v);
+                }
+            }
+            cp_async_commit();
+            if (kb >= kLag) {
+                cp_async_wait<kLag>();
+                fence_async_smem();
+                mbar_arrive(&pipe->full[(kb - kLag) % kStages]);
+            }
+        }
+        cp_async_wait<0>();
+        fence_async_smem();
+        if (ok)
+            for (int kb = (nkb > kLag ? nkb - kLag : 0); kb < nkb; ++kb) mbar_arrive(&pipe->full[kb % kStages]);
+
+        // ---------------- epilogue: TMEM lane p is column j0 + p of dW^T
+        if (ok && nkb > 0) ok = mbar_wait(&pipe->accum, 0, abort_flag, a.status);
+        tc_fence_after();
+        if (ok && nkb > 0) {
+            const int jj = j0 + p;
+            const uint32_t lane_base = tmem_d + ((uint32_t)(warp * 32) << 16);
+            for (int c0 = 0; c0 < BN; c0 += 16) {
+                if (co0 + c0 >= a.Co) break;
+                float v[16];
+                tmem_ld16(lane_base + (uint32_t)c0, v);
+                if (jj >= a.Kfwd) continue;
+#pragma unroll
+                for (int i = 0; i < 16; ++i) {
+                    const int co = co0 + c0 + i;
+                    if (co < a.Co) atomicAdd(a.dW + (long long)co * a.Kfwd + jj, v[i]);
+                }
+            }
+        }
+    } else {
+        const uint32_t idesc = instr_desc(128, BN, 1, 1);
+        bool ok = true;
+        for (int kb = 0; kb < nkb && ok; ++kb) {
+            const int s = kb % kStages;
+            ok = mbar_wait(&pipe->full[s], (kb / kStages) & 1, abort_flag, a.status);
+            if (!ok) break;
+            tc_fence_after();
+            if (lane == 0) {
+                const uint32_t sa = smem_base + s * stage_bytes, sb = sa + 16384u;
+#pragma unroll
+                for (int k = 0; k < 4; ++k)  // 4 x (K = 16 reduction rows = 2048 bytes)
+                    umma_bf16(tmem_d, smem_desc(sa + k * 2048, 8192, 1024), smem_desc(sb + k * 2048, 8192, 1024),
+                              idesc, (kb > 0 || k > 0) ? 1u : 0u);
+                umma_commit(&pipe->empty[s]);
+            }
+            __syncwarp();
+        }
+        if (ok && nkb > 0 && lane == 0) umma_commit(&pipe->accum);
+        __syncwarp();
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 4) {
+        tc_fence_after();
+        tmem_dealloc(tmem_d, ncols);
+    }
+}
+
+// --------------------------------------------------------------------- host ----
+
+int pick_bn(int N) {  // tile width: N split evenly into tiles of at most 256, rounded up to 16
+    const int tiles = (N + 255) / 256;
+    int bn = ((N + tiles - 1) / tiles + 15) / 16 * 16;
+    return bn < 16 ? 16 : bn;
+}
+
+size_t kmajor_smem(int BN) { return (size_t)kStages * (16384 + (size_t)BN * 128) + sizeof(Pipe) + 1024; }
+size_t wgrad_smem(int BN) { return (size_t)kStages * (16384 + (size_t)((BN + 63) / 64) * 8192) + sizeof(Pipe) + 1024; }
+
+// Opts both kernels into their largest dynamic shared memory footprint, once per device.
+int ensure_smem_attrs() {
+    static bool attr_set[64] = {false};
+    int dev = 0;
+    PPO_CUDA_CHECK(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) return PPO_ERR_CUDA;
+    if (!attr_set[dev]) {
+        PPO_CUDA_CHECK(cudaFuncSetAttribute(igemm_kmajor_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                            (int)kmajor_smem(256)));
+        PPO_CUDA_CHECK(cudaFuncSetAttribute(igemm_wgrad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                            (int)wgrad_smem(256)));
+        attr_set[dev] = true;
+    }
+    return PPO_OK;
+}
+
+int launch_kmajor(const KArgs &a, cudaStream_t st) {
+    int s = ensure_smem_attrs();
+    if (s != PPO_OK) return s;
+    if (a.Mrows <= 0) return PPO_OK;
+    dim3 grid((unsigned)((a.Mrows + 127) / 128), (unsigned)((a.N + a.BN - 1) / a.BN));
+    igemm_kmajor_kernel<<<grid, kThreads, kmajor_smem(a.BN), st>>>(a);
+    PPO_LAUNCH_CHECK();
+    return PPO_OK;
+}
+
+}  // namespace
+
+int tc_gemm_fwd(const ConvGeom &g, const bf16 *X, const bf16 *W, const FwdEpilogue &e, int32_t *status,
+                cudaStream_t st) {
+    if (g.Ci % 8 != 0 || g.taps() > kMaxTaps || !status) return PPO_ERR_UNSUPPORTED;
+    KArgs a = {};
+    a.S = X; a.Hs = g.Hi; a.Ws = g.Wi; a.lds = g.Ci;
+    a.Wm = W; a.w_row = g.K(); a.w_tap = g.Ci;
+    a.Hr = g.Ho; a.Wr = g.Wo; a.Mrows = g.M();
+    a.s_mul = 2; a.s_oy = a.s_ox = -g.pad;
+    a.o_mul = 1; a.o_oy = a.o_ox = 0; a.Hout = g.Ho; a.Wout = g.Wo;
+    a.N = g.Co; a.BN = pick_bn(g.Co); a.ldo = g.Co;
+    a.mode = e.out ? EPI_FWD : EPI_HEAD; a.relu = e.relu; a.A = e.A;
+    a.bias = e.bias; a.out = e.out; a.out_f32 = nullptr; a.mask = nullptr; a.mean = e.out_mean; a.value = e.out_value;
+    a.taps.n = g.taps(); a.taps.ck = g.Ci / 8;
+    for (int t = 0; t < g.taps(); ++t) {
+        a.taps.dy[t] = (signed char)(t / g.k);
+        a.taps.dx[t] = (signed char)(t % g.k);
+        a.taps.wt[t] = (short)t;
+    }
+    a.kchunks = a.taps.n * a.taps.ck;
+    a.status = status;
+    if (a.mode == EPI_FWD && g.Co % 8 != 0) return PPO_ERR_UNSUPPORTED;
+    return launch_kmajor(a, st);
+}
+
+int tc_gemm_dgrad(const ConvGeom &g, const bf16 *dY, int ldy, const bf16 *Wt, int wt_ld, const DgradEpilogue &e,
+                  int32_t *status, cudaStream_t st) {
+    if (g.Ci % 8 != 0 || ldy % 8 != 0 || wt_ld % 8 != 0 || !status) return PPO_ERR_UNSUPPORTED;
+    // One launch per stride-parity class (ih % 2, iw % 2): inside a class every input pixel sees the
+    // same set of kernel taps, kh = (ph + pad) mod 2, +2, ..., reading output row (ih + pad - kh) / 2.
+    for (int ph = 0; ph < 2; ++ph)
+        for (int pw = 0; pw < 2; ++pw) {
+            const int Hr = (g.Hi - ph + 1) / 2, Wr = (g.Wi - pw + 1) / 2;
+            if (Hr <= 0 || Wr <= 0) continue;
+            KArgs a = {};
+            a.S = dY; a.Hs = g.Ho; a.Ws = g.Wo; a.lds = ldy;
+            a.Wm = Wt; a.w_row = g.taps() * wt_ld; a.w_tap = wt_ld;
+            a.Hr = Hr; a.Wr = Wr; a.Mrows = (long long)g.B * Hr * Wr;
+            a.s_mul = 1; a.s_oy = a.s_ox = 0;
+            a.o_mul = 2; a.o_oy = ph; a.o_ox = pw; a.Hout = g.Hi; a.Wout = g.Wi;
+            a.N = g.Ci; a.BN = pick_bn(g.Ci); a.ldo = g.Ci;
+            a.mode = EPI_DGRAD; a.relu = 0; a.A = 0;
+            a.bias = nullptr; a.out = e.out; a.out_f32 = e.out_f32; a.mask = e.mask_act;
+            int nt = 0;
+            for (int kh = (ph + g.pad) & 1; kh < g.k; kh += 2)
+                for (int kw = (pw + g.pad) & 1; kw < g.k; kw += 2) {
+                    if (nt >= kMaxTaps) return PPO_ERR_UNSUPPORTED;
+                    a.taps.dy[nt] = (signed char)((ph + g.pad - kh) / 2);
+                    a.taps.dx[nt] = (signed char)((pw + g.pad - kw) / 2);
+                    a.taps.wt[nt] = (short)(kh * g.k + kw);
+                    ++nt;
+                }
+            a.taps.n = nt; a.taps.ck = wt_ld / 8;
+            a.kchunks = nt * a.taps.ck;
+            a.status = status;
+            // nt == 0 (k = 1, odd pixels): no tap reaches this class and the kernel writes zeros
+            int s = launch_kmajor(a, st);
+            if (s != PPO_OK) return s;
+        }
+    return PPO_OK;
+}
+
+int tc_gemm_wgrad(const ConvGeom &g, const bf16 *dY, int ldy, const bf16 *X, float *dW, int32_t *status,
+                  cudaStream_t st) {
+    if (g.Ci % 8 != 0 || ldy % 8 != 0 || !status) return PPO_ERR_UNSUPPORTED;
+    WArgs a = {};
+    a.X = X; a.Hi = g.Hi; a.Wi = g.Wi; a.Ci = g.Ci; a.Ho = g.Ho; a.Wo = g.Wo; a.ksz = g.k; a.pad = g.pad;
+    a.dY = dY; a.ldy = ldy; a.Co = g.Co;
+    a.Mtot = g.M();
+    a.Kfwd = g.K();
+    a.BN = pick_bn(g.Co);
+    a.dW = dW;
+    a.status = status;
+    int s = ensure_smem_attrs();
+    if (s != PPO_OK) return s;
+    const int tiles = ((a.Kfwd + 127) / 128) * ((g.Co + a.BN - 1) / a.BN);
+    long long splits = (long long)ppo_num_sms() * 2 / tiles;
+    if (splits < 1) splits = 1;
+    long long per = ((a.Mtot + splits - 1) / splits + 63) / 64 * 64;
+    if (per < 256) per = 256;
+    splits = (a.Mtot + per - 1) / per;
+    a.m_per_split = per;
+    dim3 grid((unsigned)((a.Kfwd + 127) / 128), (unsigned)((g.Co + a.BN - 1) / a.BN), (unsigned)splits);
+    igemm_wgrad_kernel<<<grid, kThreads, wgrad_smem(a.BN), st>>>(a);
+    PPO_LAUNCH_CHECK();
+    return PPO_OK;
 }

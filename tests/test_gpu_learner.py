@@ -161,7 +161,7 @@ def test_minibatch_forward_loss_backward_match_oracle(name, microbatch):
 
 def test_loss_kernel_alone_matches_oracle_to_1e3():
     """Same mu and V on both sides: isolates the fused loss/gradient kernel (fp32 vs fp64)."""
-    w = SHAPES["cfg1_twin"]
+    w = SHAPES["cfg1_twin"].scaled(16, minibatches=1)  # one minibatch of 64 rows
     L, md, lay, theta, roll, action, logp, dev = _setup(w, 64)
     g = np.random.default_rng(0)
     B, A = 64, w.A
@@ -201,7 +201,7 @@ def test_loss_kernel_alone_matches_oracle_to_1e3():
 
 def test_ratio_is_one_on_the_rollout_policy():
     """Old log-probs from the same weights: r = 1 up to the encoder's rounding, so nothing is clipped."""
-    w = SHAPES["cfg1_twin"]
+    w = SHAPES["cfg1_twin"].scaled(16, minibatches=2)
     L, md, lay, theta, roll, action, logp, dev = _setup(w, 32, jitter=False)
     L.compute_gae(dev["last_value"])
     ppo.ppo_shuffle_gather_minibatch(L.buffer, 0, 0, 0, 2, L.mb)
