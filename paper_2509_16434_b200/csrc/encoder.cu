@@ -55,98 +55,148 @@ __global__ void __launch_bounds__(128) conv1_fwd_kernel(const __half *__restrict
 }
 
 // dW1[co][tap] += sum_m dZ1[m][co] * x(m, tap);  db1[co] += sum_m dZ1[m][co].
-// A block stages TM output pixels (their gradients and input patches) in shared memory,
-// then each thread owns a few (co, tap) pairs and reduces over the staged pixels.
-template <int KS>
+// Register tiling: C1 / CPT threads share one output pixel, each owning CPT channels and all k*k
+// taps (CPT * k*k accumulators); the pixel's gradient row is read once, coalesced, straight from
+// global memory and its input patch through L1.  Partial sums are folded across the pixel groups
+// of a warp by shuffles, across warps through shared memory, then added with one atomic each.
+template <int KS, int CPT>
 __global__ void __launch_bounds__(256) conv1_wgrad_kernel(const __half *__restrict__ depth,
                                                           const bf16 *__restrict__ dZ, float *__restrict__ dW,
                                                           float *__restrict__ db, int rows, int Hi, int Wi, int Ho,
                                                           int Wo, int C1) {
-    constexpr int TM = 64, K2 = KS * KS, MAXP = 8;
-    extern __shared__ float sm[];
-    float *dz = sm;             // [TM][C1]
-    float *px = sm + TM * C1;   // [TM][K2]
-    const int npairs = C1 * K2 + C1;
-    float acc[MAXP];
+    constexpr int K2 = KS * KS, P = KS / 2;
+    extern __shared__ float sm[];  // [8 warps][C1 * (K2 + 1)]
+    const int tpp = C1 / CPT;                  // threads per pixel (a power of two <= 32)
+    const int cq = threadIdx.x % tpp;          // channel group
+    const int pg = threadIdx.x / tpp;          // pixel group inside the block
+    const int groups = 256 / tpp;
+    float acc[CPT][K2 + 1];
 #pragma unroll
-    for (int j = 0; j < MAXP; ++j) acc[j] = 0.f;
+    for (int c = 0; c < CPT; ++c)
+#pragma unroll
+        for (int t = 0; t <= K2; ++t) acc[c][t] = 0.f;
     const long long M = (long long)rows * Ho * Wo;
-    constexpr int P = KS / 2;
-    for (long long m0 = (long long)blockIdx.x * TM; m0 < M; m0 += (long long)gridDim.x * TM) {
-        __syncthreads();
-        for (int i = threadIdx.x; i < TM * C1; i += blockDim.x) {
-            const long long m = m0 + i / C1;
-            dz[i] = (m < M) ? bf2f(dZ[m * C1 + i % C1]) : 0.f;
+    for (long long m = (long long)blockIdx.x * groups + pg; m < M; m += (long long)gridDim.x * groups) {
+        float dz[CPT];
+        if (CPT == 4) {
+            const uint2 raw = *reinterpret_cast<const uint2 *>(dZ + m * C1 + cq * 4);
+            const float2 lo = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&raw.x));
+            const float2 hi = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&raw.y));
+            dz[0] = lo.x; dz[1 % CPT] = lo.y; dz[2 % CPT] = hi.x; dz[3 % CPT] = hi.y;
+        } else if (CPT == 2) {
+            const float2 v = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(dZ + m * C1 + cq * 2));
+            dz[0] = v.x; dz[1 % CPT] = v.y;
+        } else {
+            dz[0] = bf2f(dZ[m * C1 + cq]);
         }
-        for (int i = threadIdx.x; i < TM * K2; i += blockDim.x) {
-            const int mm = i / K2, tap = i % K2;
-            const long long m = m0 + mm;
-            float v = 0.f;
-            if (m < M) {
-                const int ow = (int)(m % Wo);
-                const long long t = m / Wo;
-                const int oh = (int)(t % Ho);
-                const long long b = t / Ho;
-                const int ih = 2 * oh + tap / KS - P, iw = 2 * ow + tap % KS - P;
-                if (ih >= 0 && ih < Hi && iw >= 0 && iw < Wi) v = __half2float(depth[(b * Hi + ih) * Wi + iw]);
-            }
-            px[i] = v;
-        }
-        __syncthreads();
+        bool any = false;
 #pragma unroll
-        for (int j = 0; j < MAXP; ++j) {
-            const int p = threadIdx.x + j * 256;
-            if (p < npairs) {
-                float s = 0.f;
-                if (p < C1 * K2) {
-                    const int co = p % C1, tap = p / C1;
-#pragma unroll 8
-                    for (int mm = 0; mm < TM; ++mm) s = fmaf(dz[mm * C1 + co], px[mm * K2 + tap], s);
-                } else {
-                    const int co = p - C1 * K2;
-#pragma unroll 8
-                    for (int mm = 0; mm < TM; ++mm) s += dz[mm * C1 + co];
-                }
-                acc[j] += s;
+        for (int c = 0; c < CPT; ++c) any |= dz[c] != 0.f;
+        if (!any) continue;  // ReLU-masked gradient rows are frequent
+        const int ow = (int)(m % Wo);
+        const long long t = m / Wo;
+        const int oh = (int)(t % Ho);
+        const long long b = t / Ho;
+        const __half *img = depth + b * Hi * Wi;
+#pragma unroll
+        for (int kh = 0; kh < KS; ++kh) {
+            const int ih = 2 * oh + kh - P;
+            if (ih < 0 || ih >= Hi) continue;
+#pragma unroll
+            for (int kw = 0; kw < KS; ++kw) {
+                const int iw = 2 * ow + kw - P;
+                if (iw < 0 || iw >= Wi) continue;
+                const float xv = __half2float(img[ih * Wi + iw]);
+#pragma unroll
+                for (int c = 0; c < CPT; ++c) acc[c][kh * KS + kw] = fmaf(dz[c], xv, acc[c][kh * KS + kw]);
             }
         }
+#pragma unroll
+        for (int c = 0; c < CPT; ++c) acc[c][K2] += dz[c];
     }
+    // fold the pixel groups that live in one warp (lanes that differ in bits >= log2(tpp))
 #pragma unroll
-    for (int j = 0; j < MAXP; ++j) {
-        const int p = threadIdx.x + j * 256;
-        if (p < C1 * K2) atomicAdd(dW + (p % C1) * K2 + p / C1, acc[j]);
-        else if (p < npairs) atomicAdd(db + (p - C1 * K2), acc[j]);
+    for (int c = 0; c < CPT; ++c)
+#pragma unroll
+        for (int t = 0; t <= K2; ++t) {
+            float v = acc[c][t];
+            for (int o = tpp; o < 32; o <<= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+            acc[c][t] = v;
+        }
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int per = C1 * (K2 + 1);
+    if (lane < tpp) {
+#pragma unroll
+        for (int c = 0; c < CPT; ++c)
+#pragma unroll
+            for (int t = 0; t <= K2; ++t) sm[warp * per + (cq * CPT + c) * (K2 + 1) + t] = acc[c][t];
+    }
+    __syncthreads();
+    const int nw = 8;  // every warp holds a full set of channel groups (tpp <= 32)
+    for (int i = threadIdx.x; i < per; i += 256) {
+        float v = 0.f;
+        for (int w = 0; w < nw; ++w) v += sm[w * per + i];
+        const int co = i / (K2 + 1), t = i % (K2 + 1);
+        if (t < K2) atomicAdd(dW + co * K2 + t, v);
+        else atomicAdd(db + co, v);
     }
 }
 
 // ------------------------------------------------------------- small kernels ----
 
-// h0[b] = [mean over pixels of act[b][px][c], proprio[b]] as bf16.  One block per row b.
+// h0[b] = [mean over pixels of act[b][px][c], proprio[b]] as bf16.  One warp per row b; a lane
+// owns 8 channels at a time so that every pixel is read with 128-bit loads.
 __global__ void __launch_bounds__(256) pool_concat_kernel(const bf16 *__restrict__ act,
                                                           const float *__restrict__ proprio, bf16 *__restrict__ h0,
-                                                          int npx, int C, int P) {
-    const int b = blockIdx.x;
+                                                          int rows, int npx, int C, int P) {
+    const int b = blockIdx.x * 8 + (threadIdx.x >> 5);
+    const int lane = threadIdx.x & 31;
+    if (b >= rows) return;
     const float inv = 1.f / (float)npx;
-    for (int c = threadIdx.x; c < C; c += blockDim.x) {
-        const bf16 *p = act + (size_t)b * npx * C + c;
-        float s = 0.f;
-        for (int px = 0; px < npx; ++px) s += bf2f(p[(size_t)px * C]);
-        h0[(size_t)b * (C + P) + c] = __float2bfloat16_rn(s * inv);
+    const bf16 *base = act + (size_t)b * npx * C;
+    bf16 *out = h0 + (size_t)b * (C + P);
+    for (int c8 = lane * 8; c8 < C; c8 += 256) {
+        float s[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) s[i] = 0.f;
+        for (int px = 0; px < npx; ++px) {
+            const uint4 raw = *reinterpret_cast<const uint4 *>(base + (size_t)px * C + c8);
+            const __nv_bfloat162 *p2 = reinterpret_cast<const __nv_bfloat162 *>(&raw);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const float2 f = __bfloat1622float2(p2[i]);
+                s[2 * i] += f.x;
+                s[2 * i + 1] += f.y;
+            }
+        }
+#pragma unroll
+        for (int i = 0; i < 8; ++i) out[c8 + i] = __float2bfloat16_rn(s[i] * inv);
     }
-    for (int j = threadIdx.x; j < P; j += blockDim.x)
-        h0[(size_t)b * (C + P) + C + j] = __float2bfloat16_rn(proprio[(size_t)b * P + j]);
+    for (int j = lane; j < P; j += 32) out[C + j] = __float2bfloat16_rn(proprio[(size_t)b * P + j]);
 }
 
-// dact[b][px][c] = dh0[b][c] / npx where act > 0, else 0.
+// dact[b][px][c] = dh0[b][c] / npx where act > 0, else 0; 8 channels per thread.
 __global__ void __launch_bounds__(256) unpool_kernel(const float *__restrict__ dh0, const bf16 *__restrict__ act,
-                                                     bf16 *__restrict__ dact, long long total, int npx, int C,
+                                                     bf16 *__restrict__ dact, long long total8, int npx, int C,
                                                      int ld_h0) {
     const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-    if (i >= total) return;
-    const int c = (int)(i % C);
-    const long long b = i / ((long long)npx * C);
-    const float g = dh0[b * ld_h0 + c] / (float)npx;
-    dact[i] = __float2bfloat16_rn(bf2f(act[i]) > 0.f ? g : 0.f);
+    if (i >= total8) return;
+    const int c8n = C >> 3;
+    const int c8 = (int)(i % c8n) * 8;
+    const long long b = i / ((long long)npx * c8n);
+    const float inv = 1.f / (float)npx;
+    const float4 g0 = *reinterpret_cast<const float4 *>(dh0 + b * ld_h0 + c8);
+    const float4 g1 = *reinterpret_cast<const float4 *>(dh0 + b * ld_h0 + c8 + 4);
+    const float g[8] = {g0.x, g0.y, g0.z, g0.w, g1.x, g1.y, g1.z, g1.w};
+    const uint4 raw = *reinterpret_cast<const uint4 *>(act + i * 8);
+    const __nv_bfloat162 *a2 = reinterpret_cast<const __nv_bfloat162 *>(&raw);
+    __nv_bfloat162 o[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        const float2 f = __bfloat1622float2(a2[k]);
+        o[k] = __floats2bfloat162_rn(f.x > 0.f ? g[2 * k] * inv : 0.f, f.y > 0.f ? g[2 * k + 1] * inv : 0.f);
+    }
+    *reinterpret_cast<uint4 *>(dact + i * 8) = *reinterpret_cast<uint4 *>(o);
 }
 
 // Head gradient as a bf16 GEMM operand: [rows][16] = [dmean (A), dvalue, zeros].
@@ -162,26 +212,56 @@ __global__ void __launch_bounds__(256) pack_dout_kernel(const float *__restrict_
     out[i] = __float2bfloat16_rn(v);
 }
 
-// db[n] += sum_m dZ[m][n]  (bias gradients).  32 columns x 8 row groups per block.
+// db[n] += sum_m dZ[m][n]  (bias gradients), N a multiple of 8.  Threads walk (row, 8-column chunk)
+// pairs with 128-bit loads; threads that share a chunk are folded through shared memory.
 __global__ void __launch_bounds__(256) colsum_kernel(const bf16 *__restrict__ dZ, int ld, long long M, int N,
-                                                     float *__restrict__ db, int rows_per_block) {
-    __shared__ float sh[8][33];
-    const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
-    const long long m_lo = (long long)blockIdx.x * rows_per_block;
-    const long long m_hi = min(M, m_lo + rows_per_block);
-    for (int n0 = 0; n0 < N; n0 += 32) {
-        const int n = n0 + tx;
-        float s = 0.f;
-        if (n < N)
-            for (long long m = m_lo + ty; m < m_hi; m += 8) s += bf2f(dZ[m * ld + n]);
-        sh[ty][tx] = s;
-        __syncthreads();
-        if (ty == 0 && n < N) {
-            float t = 0.f;
+                                                     float *__restrict__ db) {
+    __shared__ float sh[256][9];
+    const int chunks = N >> 3;                    // 16-byte chunks per row
+    const int rows_per_pass = 256 / chunks;       // whole rows covered by one pass of the block
+    const int tc = threadIdx.x % chunks, tr = threadIdx.x / chunks;
+    float acc[8];
 #pragma unroll
-            for (int j = 0; j < 8; ++j) t += sh[j][tx];
-            atomicAdd(db + n, t);
+    for (int i = 0; i < 8; ++i) acc[i] = 0.f;
+    if (tr < rows_per_pass) {
+        for (long long m = (long long)blockIdx.x * rows_per_pass + tr; m < M;
+             m += (long long)gridDim.x * rows_per_pass) {
+            const uint4 raw = *reinterpret_cast<const uint4 *>(dZ + m * ld + tc * 8);
+            const __nv_bfloat162 *p2 = reinterpret_cast<const __nv_bfloat162 *>(&raw);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const float2 f = __bfloat1622float2(p2[i]);
+                acc[2 * i] += f.x;
+                acc[2 * i + 1] += f.y;
+            }
         }
+    }
+#pragma unroll
+    for (int i = 0; i < 8; ++i) sh[threadIdx.x][i] = acc[i];
+    __syncthreads();
+    if (threadIdx.x < N) {
+        const int c = threadIdx.x >> 3, e = threadIdx.x & 7;
+        float v = 0.f;
+        for (int r = 0; r < rows_per_pass; ++r) v += sh[r * chunks + c][e];
+        atomicAdd(db + threadIdx.x, v);
+    }
+}
+
+// db[n] += sum_m dZ[m][n] for any N <= ld (used for the head, whose 13 columns sit in rows of 16).
+__global__ void __launch_bounds__(256) colsum_small_kernel(const bf16 *__restrict__ dZ, int ld, long long M, int N,
+                                                           float *__restrict__ db) {
+    __shared__ float sh[256];
+    for (int n = 0; n < N; ++n) {
+        float v = 0.f;
+        for (long long m = (long long)blockIdx.x * 256 + threadIdx.x; m < M; m += (long long)gridDim.x * 256)
+            v += bf2f(dZ[m * ld + n]);
+        sh[threadIdx.x] = v;
+        __syncthreads();
+        for (int o = 128; o > 0; o >>= 1) {
+            if (threadIdx.x < o) sh[threadIdx.x] += sh[threadIdx.x + o];
+            __syncthreads();
+        }
+        if (threadIdx.x == 0) atomicAdd(db + n, sh[0]);
         __syncthreads();
     }
 }
@@ -244,8 +324,25 @@ static int run_wgrad(const ppo_model *m, const ConvGeom &g, const bf16 *dY, int 
 }
 
 static int run_colsum(const bf16 *dZ, int ld, long long M, int N, float *db, cudaStream_t st) {
-    const int rpb = 512;
-    colsum_kernel<<<ppo_cdiv(M, rpb), 256, 0, st>>>(dZ, ld, M, N, db, rpb);
+    if (N % 8 == 0 && N <= 256 && ld % 8 == 0) {
+        const int rows_per_pass = 256 / (N / 8);
+        int blocks = ppo_cdiv(M, (long long)rows_per_pass * 8);
+        const int cap = ppo_num_sms() * 4;
+        blocks = blocks > cap ? cap : (blocks < 1 ? 1 : blocks);
+        colsum_kernel<<<blocks, 256, 0, st>>>(dZ, ld, M, N, db);
+    } else if (N > 256 && N % 256 == 0) {
+        // wide FC layers: one launch per 256-column slab
+        for (int n0 = 0; n0 < N; n0 += 256) {
+            int blocks = ppo_cdiv(M, 64);
+            const int cap = ppo_num_sms() * 4;
+            blocks = blocks > cap ? cap : (blocks < 1 ? 1 : blocks);
+            colsum_kernel<<<blocks, 256, 0, st>>>(dZ + n0, ld, M, 256, db + n0);
+        }
+    } else {
+        int blocks = ppo_cdiv(M, 2048);
+        blocks = blocks > 64 ? 64 : (blocks < 1 ? 1 : blocks);
+        colsum_small_kernel<<<blocks, 256, 0, st>>>(dZ, ld, M, N, db);
+    }
     PPO_LAUNCH_CHECK();
     return PPO_OK;
 }
@@ -293,8 +390,8 @@ extern "C" int ppo_encoder_fwd(ppo_model *m, const ppo_minibatch *mb, int row0, 
         FwdEpilogue e = {m->master + m->tensors[2 * (l - 1) + 1].off, 1, m->act[l], nullptr, nullptr, 0};
         PPO_TRY(run_fwd(m, g, m->act[l - 1], m->shadow + m->tensors[2 * (l - 1)].off, e, st));
     }
-    pool_concat_kernel<<<rows, 256, 0, st>>>(m->act[m->L], mb->proprio + (size_t)row0 * d.P, m->h[0],
-                                             m->Hs[m->L] * m->Ws[m->L], m->Cs[m->L], d.P);
+    pool_concat_kernel<<<ppo_cdiv(rows, 8), 256, 0, st>>>(m->act[m->L], mb->proprio + (size_t)row0 * d.P, m->h[0], rows,
+                                                          m->Hs[m->L] * m->Ws[m->L], m->Cs[m->L], d.P);
     PPO_LAUNCH_CHECK();
     int ti = 2 * m->L;
     for (int l = 1; l <= m->F; ++l, ti += 2) {
@@ -367,9 +464,9 @@ extern "C" int ppo_encoder_bwd(ppo_model *m, const ppo_minibatch *mb, int row0, 
     }
     {
         const int npx = m->Hs[L] * m->Ws[L], C = m->Cs[L];
-        const long long total = (long long)rows * npx * C;
-        unpool_kernel<<<ppo_cdiv(total, 256), 256, 0, st>>>(m->dh0_f32, m->act[L], m->dact[L], total, npx, C,
-                                                          m->hw[0]);
+        const long long total8 = (long long)rows * npx * C / 8;
+        unpool_kernel<<<ppo_cdiv(total8, 256), 256, 0, st>>>(m->dh0_f32, m->act[L], m->dact[L], total8, npx, C,
+                                                           m->hw[0]);
         PPO_LAUNCH_CHECK();
     }
     for (int l = L; l >= 2; --l) {
@@ -385,18 +482,27 @@ extern "C" int ppo_encoder_bwd(ppo_model *m, const ppo_minibatch *mb, int row0, 
         const __half *depth = static_cast<const __half *>(mb->depth_f16) + (size_t)row0 * d.H * d.W;
         const int C1 = m->Cs[1], KS = d.conv_k[0];
         const long long M = (long long)rows * m->Hs[1] * m->Ws[1];
-        const size_t smem = (size_t)64 * (C1 + KS * KS) * sizeof(float);
-        int blocks = ppo_cdiv(M, 64);
+        const int cpt = KS <= 3 ? 4 : (KS == 5 ? 2 : 1);
+        const int tpp = C1 / cpt;
+        if (C1 % cpt != 0 || tpp > 32 || (tpp & (tpp - 1)) != 0) return PPO_ERR_UNSUPPORTED;
+        const size_t smem = (size_t)8 * C1 * (KS * KS + 1) * sizeof(float);
+        int blocks = ppo_cdiv(M, (256 / tpp) * 16);
         const int cap = ppo_num_sms() * 4;
-        if (blocks > cap) blocks = cap;
+        blocks = blocks > cap ? cap : (blocks < 1 ? 1 : blocks);
         float *dW = m->grad + m->tensors[0].off, *db = m->grad + m->tensors[1].off;
-#define PPO_CONV1W(KS_)                                                                                       \
-    conv1_wgrad_kernel<KS_><<<blocks, 256, smem, st>>>(depth, m->dact[1], dW, db, rows, d.H, d.W, m->Hs[1], \
-                                                       m->Ws[1], C1)
-        if (KS == 1) PPO_CONV1W(1);
-        else if (KS == 3) PPO_CONV1W(3);
-        else if (KS == 5) PPO_CONV1W(5);
-        else PPO_CONV1W(7);
+#define PPO_CONV1W(KS_, CPT_)                                                                                     \
+    conv1_wgrad_kernel<KS_, CPT_><<<blocks, 256, smem, st>>>(depth, m->dact[1], dW, db, rows, d.H, d.W, m->Hs[1], \
+                                                             m->Ws[1], C1)
+        if (smem > 48 * 1024) {
+            if (KS == 5) PPO_CUDA_CHECK(cudaFuncSetAttribute(conv1_wgrad_kernel<5, 2>,
+                                                             cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+            if (KS == 7) PPO_CUDA_CHECK(cudaFuncSetAttribute(conv1_wgrad_kernel<7, 1>,
+                                                             cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        }
+        if (KS == 1) PPO_CONV1W(1, 4);
+        else if (KS == 3) PPO_CONV1W(3, 4);
+        else if (KS == 5) PPO_CONV1W(5, 2);
+        else PPO_CONV1W(7, 1);
 #undef PPO_CONV1W
         PPO_LAUNCH_CHECK();
     }

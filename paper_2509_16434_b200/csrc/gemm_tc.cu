@@ -66,8 +66,14 @@ template <int N>
 __device__ __forceinline__ void cp_async_wait() {
     asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
 }
-// Makes this thread's completed generic-proxy writes to shared memory visible to the async
-// proxy (the tensor core reads operands through it).
+// The mbarrier receives one arrival from this thread once all cp.async it has issued so far have
+// landed (the arrival counts against the barrier's expected count).
+__device__ __forceinline__ void cp_async_arrive(uint64_t *bar) {
+    asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+// Orders generic-proxy writes to shared memory that this thread has observed (here: the gather
+// warps' cp.async data, observed through the full barrier) before its later async-proxy
+// operations (the tensor core reads operands through the async proxy).
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
@@ -132,7 +138,8 @@ __device__ __forceinline__ uint32_t tmem_cols_for(int bn) {
 // ------------------------------------------------------------------ K-major ----
 
 constexpr int kMaxStagesK = 8;
-constexpr int kKThreads = 288;  // warps 0-3 gather, warp 4 issues MMAs, warps 5-8 run the epilogue
+constexpr int kGatherWarps = 8;
+constexpr int kKThreads = (kGatherWarps + 5) * 32;  // gather warps, one MMA-issuing warp, 4 epilogue warps
 
 struct Taps {
     int n;                 // taps walked along K
@@ -161,7 +168,7 @@ struct KArgs {
     int s_mul, s_oy, s_ox; // source pixel of tap t: (y * s_mul + s_oy + dy[t], x * s_mul + s_ox + dx[t])
     int o_mul, Hout, Wout; // output row = (b * Hout + oy) * Wout + ox
     int N, BN, ldo, tiles_n;
-    int stages, lag;
+    int stages, dbg;
     int mode, relu, A;
     const float *bias;
     bf16 *out;
@@ -182,17 +189,6 @@ struct PipeK {
     int abort_flag;
 };
 
-__device__ __forceinline__ void cp_async_wait_dyn(int lag) {
-    switch (lag) {
-        case 1: cp_async_wait<1>(); break;
-        case 2: cp_async_wait<2>(); break;
-        case 3: cp_async_wait<3>(); break;
-        case 4: cp_async_wait<4>(); break;
-        case 5: cp_async_wait<5>(); break;
-        default: cp_async_wait<6>(); break;
-    }
-}
-
 // Persistent: CTA c works on tiles c, c + gridDim.x, ...  The gather warps run ahead across tile
 // boundaries, the accumulator is double-buffered in TMEM so that the epilogue of one tile overlaps
 // the MMAs of the next.
@@ -209,7 +205,7 @@ __global__ void __launch_bounds__(kKThreads, 1) igemm_kmajor_kernel(const __grid
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < S; ++s) {
-            mbar_init(&pipe->full[s], kProducers);
+            mbar_init(&pipe->full[s], kGatherWarps * 32);
             mbar_init(&pipe->empty[s], 1);
         }
         for (int i = 0; i < 2; ++i) {
@@ -219,30 +215,34 @@ __global__ void __launch_bounds__(kKThreads, 1) igemm_kmajor_kernel(const __grid
         pipe->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (warp == 4) tmem_alloc(&pipe->tmem_slot, ncols);
+    if (warp == kGatherWarps) tmem_alloc(&pipe->tmem_slot, ncols);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = pipe->tmem_slot;
     const uint32_t smem_base = smem_u32(smem);
 
-    if (warp < 4) {
-        // ---------------- gather: thread p owns row p of the A tile and chunk slot p % 8 of B rows p/8 + 16 i
+    if (warp < kGatherWarps) {
+        // ---------------- gather: thread p fills half h = p / 128 (4 of the 8 chunks) of row p % 128 of the
+        // A tile, and chunk slot p % 8 of B rows p/8, p/8 + 32, ...
         const int p = threadIdx.x;
-        const int jB = p & 7;
-        const int nB = BN >> 4;
+        const int r = p & 127, h = p >> 7;
+        const int jB = p & 7, rB = p >> 3;
+        const uint32_t sw = (uint32_t)(r & 7);
+        const uint32_t a_dst0 = (uint32_t)r * 128u;
+        const uint32_t b_dst0 = 16384u + (uint32_t)rB * 128u + (((uint32_t)jB ^ ((uint32_t)rB & 7u)) << 4);
+        const bool fast = (a.ck & 3) == 0;   // a group of 4 chunks never straddles two taps
         int it = 0;          // K blocks issued so far (all tiles)
-        int arrived = 0;     // K blocks whose full barrier this thread has arrived on
         bool ok = true;
         for (int g = blockIdx.x; g < a.total_tiles && ok; g += gridDim.x) {
             int c = 0;
             while (c + 1 < a.ncls && g >= a.cls[c + 1].tile0) ++c;
             const KClass &k = a.cls[c];
             const int local = g - k.tile0;
-            const long long m = (long long)(local / a.tiles_n) * 128 + p;
+            const long long m = (long long)(local / a.tiles_n) * 128 + r;
             const int n0 = (local % a.tiles_n) * BN;
-            const int kchunks = k.taps.n * a.ck;
-            const int nkb = (kchunks + 7) >> 3;
+            const int ntaps = k.taps.n;
+            const int nkb = (ntaps * a.ck + 7) >> 3;
             const bool row_ok = m < k.Mrows;
             int y = 0, x = 0;
             long long b = 0;
@@ -254,51 +254,68 @@ __global__ void __launch_bounds__(kKThreads, 1) igemm_kmajor_kernel(const __grid
             }
             const int sy0 = y * a.s_mul + a.s_oy, sx0 = x * a.s_mul + a.s_ox;
             const bf16 *src_img = a.S + b * a.Hs * a.Ws * a.lds;
-            int tA = 0, cA = 0;
+            // A walk: flattened chunk index of this thread's group is kb * 8 + 4 h
+            int tA = (4 * h) / a.ck, cA = (4 * h) % a.ck;
+            // B walk: flattened chunk index kb * 8 + jB
             int tB = jB / a.ck, cB = jB % a.ck;
+            const bf16 *b_src0 = a.Wm + (long long)(n0 + rB) * a.w_row;
+            int nBv = (a.N - n0 - rB + 31) / 32;          // B rows of this thread that exist
+            const int nBt = (BN - rB + 31) / 32;          // B rows of this thread inside the tile
+            nBv = nBv < 0 ? 0 : (nBv > nBt ? nBt : nBv);
             for (int kb = 0; kb < nkb; ++kb, ++it) {
                 const int s = it % S;
                 ok = mbar_wait(&pipe->empty[s], ((it / S) & 1) ^ 1, abort_flag, a.status);
                 if (!ok) break;
-                const uint32_t sa = smem_base + s * stage_bytes, sb = sa + 16384u;
-#pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                    bool v = row_ok && tA < k.taps.n;
+                const uint32_t st = smem_base + s * stage_bytes;
+                if (fast) {
+                    bool v = row_ok && tA < ntaps;
                     const bf16 *src = a.S;
                     if (v) {
                         const int yy = sy0 + k.taps.dy[tA], xx = sx0 + k.taps.dx[tA];
-                        v = yy >= 0 && yy < a.Hs && xx >= 0 && xx < a.Ws;
-                        if (v) src = src_img + ((long long)yy * a.Ws + xx) * a.lds + cA * 8;
+                        v = (unsigned)yy < (unsigned)a.Hs && (unsigned)xx < (unsigned)a.Ws;
+                        if (v) src = src_img + ((yy * a.Ws + xx) * a.lds + cA * 8);
                     }
-                    cp_async16(sa + p * 128 + ((j ^ (p & 7)) << 4), src, v);
-                    if (++cA == a.ck) { cA = 0; ++tA; }
+                    const uint32_t d = st + a_dst0;
+#pragma unroll
+                    for (int j = 0; j < 4; ++j)
+                        cp_async16(d + ((((uint32_t)(4 * h + j)) ^ sw) << 4), src + j * 8, v);
+                    cA += 8;
+                    while (cA >= a.ck) { cA -= a.ck; ++tA; }
+                } else {
+                    int t = tA, cc = cA;
+                    for (int j = 0; j < 4; ++j) {
+                        while (cc >= a.ck) { cc -= a.ck; ++t; }
+                        bool v = row_ok && t < ntaps;
+                        const bf16 *src = a.S;
+                        if (v) {
+                            const int yy = sy0 + k.taps.dy[t], xx = sx0 + k.taps.dx[t];
+                            v = (unsigned)yy < (unsigned)a.Hs && (unsigned)xx < (unsigned)a.Ws;
+                            if (v) src = src_img + ((yy * a.Ws + xx) * a.lds + cc * 8);
+                        }
+                        cp_async16(st + a_dst0 + ((((uint32_t)(4 * h + j)) ^ sw) << 4), src, v);
+                        ++cc;
+                    }
+                    cA += 8;
+                    while (cA >= a.ck) { cA -= a.ck; ++tA; }
                 }
                 {
-                    const bool kv = tB < k.taps.n;
-                    const long long koff = kv ? (long long)k.taps.wt[tB] * a.w_tap + cB * 8 : 0;
-                    for (int i = 0; i < nB; ++i) {
-                        const int n = (p >> 3) + i * 16;
-                        const bool v = kv && (n0 + n) < a.N;
-                        const bf16 *src = v ? a.Wm + (long long)(n0 + n) * a.w_row + koff : a.Wm;
-                        cp_async16(sb + n * 128 + ((jB ^ (n & 7)) << 4), src, v);
+                    const bool kv = tB < ntaps;
+                    const bf16 *src = b_src0 + (kv ? (int)k.taps.wt[tB] * a.w_tap + cB * 8 : 0);
+                    const uint32_t d = st + b_dst0;
+                    const long long rstep = 32ll * a.w_row;
+                    for (int i = 0; i < nBt; ++i) {
+                        const bool v = kv && i < nBv;
+                        cp_async16(d + (uint32_t)i * 4096u, v ? src + i * rstep : a.Wm, v);
                     }
                     cB += 8;
                     while (cB >= a.ck) { cB -= a.ck; ++tB; }
                 }
-                cp_async_commit();
-                if (it - arrived >= a.lag) {  // the group issued `lag` blocks ago has landed
-                    cp_async_wait_dyn(a.lag);
-                    fence_async_smem();
-                    mbar_arrive(&pipe->full[arrived % S]);
-                    ++arrived;
-                }
+                cp_async_arrive(&pipe->full[s]);
             }
         }
+        cp_async_commit();
         cp_async_wait<0>();
-        fence_async_smem();
-        if (ok)
-            for (; arrived < it; ++arrived) mbar_arrive(&pipe->full[arrived % S]);
-    } else if (warp == 4) {
+    } else if (warp == kGatherWarps) {
         // ---------------- MMA issue: one thread feeds the tensor core
         const uint32_t idesc = instr_desc(128, BN, 0, 0);
         int it = 0, ti = 0;
@@ -316,6 +333,7 @@ __global__ void __launch_bounds__(kKThreads, 1) igemm_kmajor_kernel(const __grid
                 const int s = it % S;
                 ok = mbar_wait(&pipe->full[s], (it / S) & 1, abort_flag, a.status);
                 if (!ok) break;
+                if (!(a.dbg & 1)) fence_async_smem();
                 tc_fence_after();
                 if (lane == 0) {
                     const uint32_t sa = smem_base + s * stage_bytes, sb = sa + 16384u;
@@ -426,7 +444,7 @@ __global__ void __launch_bounds__(kKThreads, 1) igemm_kmajor_kernel(const __grid
     }
     tc_fence_before();
     __syncthreads();
-    if (warp == 4) {
+    if (warp == kGatherWarps) {
         tc_fence_after();
         tmem_dealloc(tmem_base, ncols);
     }
@@ -443,7 +461,7 @@ struct WArgs {
     long long m_per_split; // multiple of 64
     int Kfwd;              // ksz * ksz * Ci
     int BN;
-    int stages, lag;
+    int stages;
     float *dW;             // [Co][Kfwd], accumulated with atomics
     int32_t *status;
 };
@@ -538,17 +556,10 @@ __global__ void __launch_bounds__(kThreads) igemm_wgrad_kernel(const __grid_cons
                     cp_async16(brow + ((q ^ (r & 7)) << 4), v ? dyrow + co : a.dY, v);
                 }
             }
-            cp_async_commit();
-            if (kb >= a.lag) {
-                cp_async_wait_dyn(a.lag);
-                fence_async_smem();
-                mbar_arrive(&pipe->full[(kb - a.lag) % S]);
-            }
+            cp_async_arrive(&pipe->full[s]);
         }
+        cp_async_commit();
         cp_async_wait<0>();
-        fence_async_smem();
-        if (ok)
-            for (int kb = (nkb > a.lag ? nkb - a.lag : 0); kb < nkb; ++kb) mbar_arrive(&pipe->full[kb % S]);
 
         // ---------------- epilogue: TMEM lane p is column j0 + p of dW^T
         if (ok && nkb > 0) ok = mbar_wait(&pipe->tfull[0], 0, abort_flag, a.status);
@@ -575,6 +586,7 @@ __global__ void __launch_bounds__(kThreads) igemm_wgrad_kernel(const __grid_cons
             const int s = kb % S;
             ok = mbar_wait(&pipe->full[s], (kb / S) & 1, abort_flag, a.status);
             if (!ok) break;
+            fence_async_smem();
             tc_fence_after();
             if (lane == 0) {
                 const uint32_t sa = smem_base + s * stage_bytes, sb = sa + 16384u;
@@ -650,7 +662,7 @@ int launch_kmajor(KArgs &a, cudaStream_t st) {
     if (tiles > 0x7fffffffll) return PPO_ERR_UNSUPPORTED;
     a.total_tiles = (int)tiles;
     a.stages = kmajor_stages(a.BN);
-    a.lag = a.stages - 2 > 6 ? 6 : a.stages - 2;
+    { const char *e = getenv("PPO_DBG"); a.dbg = e ? atoi(e) : 0; }
     const int sms = ppo_num_sms();
     const unsigned grid = (unsigned)(tiles < sms ? tiles : sms);
     igemm_kmajor_kernel<<<grid, kKThreads, kmajor_smem(a.BN), st>>>(a);
@@ -732,7 +744,6 @@ int tc_gemm_wgrad(const ConvGeom &g, const bf16 *dY, int ldy, const bf16 *X, flo
     a.Kfwd = g.K();
     a.BN = pick_bn(g.Co);
     a.stages = wgrad_stages(a.BN);
-    a.lag = a.stages - 2 > 6 ? 6 : a.stages - 2;
     a.dW = dW;
     a.status = status;
     int s = ensure_smem_attrs();
