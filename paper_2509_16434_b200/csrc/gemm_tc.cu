@@ -168,7 +168,7 @@ struct KArgs {
     int s_mul, s_oy, s_ox; // source pixel of tap t: (y * s_mul + s_oy + dy[t], x * s_mul + s_ox + dx[t])
     int o_mul, Hout, Wout; // output row = (b * Hout + oy) * Wout + ox
     int N, BN, ldo, tiles_n;
-    int stages, dbg;
+    int stages;
     int mode, relu, A;
     const float *bias;
     bf16 *out;
@@ -333,7 +333,7 @@ __global__ void __launch_bounds__(kKThreads, 1) igemm_kmajor_kernel(const __grid
                 const int s = it % S;
                 ok = mbar_wait(&pipe->full[s], (it / S) & 1, abort_flag, a.status);
                 if (!ok) break;
-                if (!(a.dbg & 1)) fence_async_smem();
+                fence_async_smem();
                 tc_fence_after();
                 if (lane == 0) {
                     const uint32_t sa = smem_base + s * stage_bytes, sb = sa + 16384u;
@@ -662,7 +662,6 @@ int launch_kmajor(KArgs &a, cudaStream_t st) {
     if (tiles > 0x7fffffffll) return PPO_ERR_UNSUPPORTED;
     a.total_tiles = (int)tiles;
     a.stages = kmajor_stages(a.BN);
-    { const char *e = getenv("PPO_DBG"); a.dbg = e ? atoi(e) : 0; }
     const int sms = ppo_num_sms();
     const unsigned grid = (unsigned)(tiles < sms ? tiles : sms);
     igemm_kmajor_kernel<<<grid, kKThreads, kmajor_smem(a.BN), st>>>(a);
