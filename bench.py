@@ -223,11 +223,13 @@ def run_ours(args):
         sampler.start()
     t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
+    torch.cuda.nvtx.range_push("timed")
     t0.record()
     for i in range(args.steps):
         one_step(100 + i)
     t1.record()
     barrier()
+    torch.cuda.nvtx.range_pop()
     clocks = sampler.stop() if rank == 0 else None
     for n in names:
         setattr(ppo, n, originals[n])
