@@ -308,18 +308,24 @@ static ConvGeom fc_geom(int rows, int in, int out) {
 static int run_fwd(const ppo_model *m, const ConvGeom &g, const bf16 *X, const bf16 *W, const FwdEpilogue &e,
                    cudaStream_t st) {
     if (m->impl == 1) return simt_gemm_fwd(g, X, W, e, st);
+    const int s = tma_gemm_fwd(g, X, W, e, ppo_device_status_ptr(), st);
+    if (s != PPO_ERR_UNSUPPORTED) return s;
     return tc_gemm_fwd(g, X, W, e, ppo_device_status_ptr(), st);
 }
 
 static int run_dgrad(const ppo_model *m, const ConvGeom &g, const bf16 *dY, int ldy, const bf16 *W, const bf16 *Wt,
                      int wt_ld, const DgradEpilogue &e, cudaStream_t st) {
     if (m->impl == 1) return simt_gemm_dgrad(g, dY, ldy, W, e, st);
+    const int s = tma_gemm_dgrad(g, dY, ldy, Wt, wt_ld, e, ppo_device_status_ptr(), st);
+    if (s != PPO_ERR_UNSUPPORTED) return s;
     return tc_gemm_dgrad(g, dY, ldy, Wt, wt_ld, e, ppo_device_status_ptr(), st);
 }
 
 static int run_wgrad(const ppo_model *m, const ConvGeom &g, const bf16 *dY, int ldy, const bf16 *X, float *dW,
                      cudaStream_t st) {
     if (m->impl == 1) return simt_gemm_wgrad(g, dY, ldy, X, dW, st);
+    const int s = tma_gemm_wgrad(g, dY, ldy, X, dW, ppo_device_status_ptr(), st);
+    if (s != PPO_ERR_UNSUPPORTED) return s;
     return tc_gemm_wgrad(g, dY, ldy, X, dW, ppo_device_status_ptr(), st);
 }
 

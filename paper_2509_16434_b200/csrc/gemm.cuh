@@ -35,3 +35,13 @@ int tc_gemm_dgrad(const ConvGeom &g, const bf16 *dY, int ldy, const bf16 *Wt, in
                   int32_t *status, cudaStream_t st);
 int tc_gemm_wgrad(const ConvGeom &g, const bf16 *dY, int ldy, const bf16 *X, float *dW, int32_t *status,
                   cudaStream_t st);
+
+// TMA-fed versions of the same three operations (operand tiles moved by cp.async.bulk.tensor).  They cover
+// channel counts that are multiples of 32 (any multiple of 8 that is at least 64 for a fully connected layer);
+// for anything else they return PPO_ERR_UNSUPPORTED without launching and the caller uses the tc_ versions.
+int tma_gemm_fwd(const ConvGeom &g, const bf16 *X, const bf16 *W, const FwdEpilogue &e, int32_t *status,
+                 cudaStream_t st);
+int tma_gemm_dgrad(const ConvGeom &g, const bf16 *dY, int ldy, const bf16 *Wt, int wt_ld, const DgradEpilogue &e,
+                   int32_t *status, cudaStream_t st);
+int tma_gemm_wgrad(const ConvGeom &g, const bf16 *dY, int ldy, const bf16 *X, float *dW, int32_t *status,
+                   cudaStream_t st);

@@ -15,126 +15,15 @@
 // memory descriptors name.  Read K-major, a row is one M/N index and its 64 columns are K; read
 // MN-major, a row is one K index and its 64 columns are M/N.
 #include "gemm.cuh"
+#include "tcgen05.cuh"
 
 namespace {
+
+using namespace tc;
 
 constexpr int kProducers = 128;       // 4 warps: gather, then epilogue
 constexpr int kThreads = 160;         // wgrad kernel: + 1 warp issuing the MMAs
 constexpr int kMaxTaps = 49;
-constexpr long long kWaitCycles = 4000000000ll;  // ~2 s at 2 GHz
-
-__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint64_t *bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint64_t *bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(smem_u32(bar)), "r"(parity)
-        : "memory");
-    return ok != 0;
-}
-// Bounded wait; returns false when this or another thread of the CTA gave up.
-__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag, int32_t *status) {
-    if (mbar_try_wait(bar, parity)) return true;
-    const long long t0 = clock64();
-    while (!mbar_try_wait(bar, parity)) {
-        if (*abort_flag) return false;
-        if (clock64() - t0 > kWaitCycles) {
-            *abort_flag = 1;
-            ppo_report(status, PPO_ERR_TIMEOUT);
-            return false;
-        }
-    }
-    return true;
-}
-
-__device__ __forceinline__ void cp_async16(uint32_t dst, const void *src, bool valid) {
-    const uint32_t n = valid ? 16u : 0u;  // 0 source bytes: the 16 destination bytes are zero-filled
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(n) : "memory");
-}
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-template <int N>
-__device__ __forceinline__ void cp_async_wait() {
-    asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
-}
-// The mbarrier receives one arrival from this thread once all cp.async it has issued so far have
-// landed (the arrival counts against the barrier's expected count).
-__device__ __forceinline__ void cp_async_arrive(uint64_t *bar) {
-    asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-// Orders generic-proxy writes to shared memory that this thread has observed (here: the gather
-// warps' cp.async data, observed through the full barrier) before its later async-proxy
-// operations (the tensor core reads operands through the async proxy).
-__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
-
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-
-__device__ __forceinline__ void tmem_alloc(uint32_t *slot, uint32_t ncols) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(slot)), "r"(ncols)
-                 : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-}
-__device__ __forceinline__ void tmem_dealloc(uint32_t addr, uint32_t ncols) {
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(addr), "r"(ncols) : "memory");
-}
-__device__ __forceinline__ void umma_commit(uint64_t *bar) {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
-                 : "memory");
-}
-// D[tmem] (+)= A[smem desc] * B[smem desc], bf16 operands, fp32 accumulate.
-__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
-                                          uint32_t accumulate) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
-        : "memory");
-}
-// 16 consecutive fp32 columns of this thread's TMEM lane.
-__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float *v) {
-    uint32_t r[16];
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, "
-        "%15}, [%16];"
-        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
-          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
-        : "r"(taddr)
-        : "memory");
-    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-#pragma unroll
-    for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
-}
-
-// Shared-memory matrix descriptor for the SWIZZLE_128B image: start address, leading and
-// stride byte offsets (each >> 4), descriptor version 1 (bit 46), layout type 2 (bits 61-63).
-__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
-    return (uint64_t)((addr >> 4) & 0x3FFFu) | ((uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16) |
-           ((uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32) | (1ull << 46) | (2ull << 61);
-}
-// Instruction descriptor, kind::f16: D fp32 (bits 4-5 = 1), A and B bf16 (bits 7-9, 10-12 = 1),
-// operand majors (bit 15, 16: 0 = K-major, 1 = MN-major), N >> 3 (bits 17-22), M >> 4 (bits 24-28).
-__host__ __device__ constexpr uint32_t instr_desc(int M, int N, int a_mn, int b_mn) {
-    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)a_mn << 15) | ((uint32_t)b_mn << 16) |
-           ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
-}
-
-__device__ __forceinline__ uint32_t tmem_cols_for(int bn) {
-    uint32_t c = 32;
-    while ((int)c < bn) c <<= 1;
-    return c;
-}
-
 // ------------------------------------------------------------------ K-major ----
 
 constexpr int kMaxStagesK = 8;
@@ -223,93 +112,73 @@ __global__ void __launch_bounds__(kKThreads, 1) igemm_kmajor_kernel(const __grid
     const uint32_t smem_base = smem_u32(smem);
 
     if (warp < kGatherWarps) {
-        // ---------------- gather: thread p fills half h = p / 128 (4 of the 8 chunks) of row p % 128 of the
-        // A tile, and chunk slot p % 8 of B rows p/8, p/8 + 32, ...
+        // ---------------- gather: thread p owns 16-byte chunk column c = p % 8 of the K block and rows
+        // p / 8 + 32 i of both tiles, so that the 8 lanes of a row read up to 128 contiguous bytes (whole
+        // 32-byte sectors) and a warp writes four complete swizzled rows (no bank conflicts).
         const int p = threadIdx.x;
-        const int r = p & 127, h = p >> 7;
-        const int jB = p & 7, rB = p >> 3;
-        const uint32_t sw = (uint32_t)(r & 7);
-        const uint32_t a_dst0 = (uint32_t)r * 128u;
-        const uint32_t b_dst0 = 16384u + (uint32_t)rB * 128u + (((uint32_t)jB ^ ((uint32_t)rB & 7u)) << 4);
-        const bool fast = (a.ck & 3) == 0;   // a group of 4 chunks never straddles two taps
+        const int c = p & 7, rg = p >> 3;
+        const uint32_t dst0 = (uint32_t)rg * 128u + (((uint32_t)c ^ ((uint32_t)rg & 7u)) << 4);
         int it = 0;          // K blocks issued so far (all tiles)
         bool ok = true;
         for (int g = blockIdx.x; g < a.total_tiles && ok; g += gridDim.x) {
-            int c = 0;
-            while (c + 1 < a.ncls && g >= a.cls[c + 1].tile0) ++c;
-            const KClass &k = a.cls[c];
+            int cl = 0;
+            while (cl + 1 < a.ncls && g >= a.cls[cl + 1].tile0) ++cl;
+            const KClass &k = a.cls[cl];
             const int local = g - k.tile0;
-            const long long m = (long long)(local / a.tiles_n) * 128 + r;
+            const long long m0 = (long long)(local / a.tiles_n) * 128 + rg;
             const int n0 = (local % a.tiles_n) * BN;
             const int ntaps = k.taps.n;
             const int nkb = (ntaps * a.ck + 7) >> 3;
-            const bool row_ok = m < k.Mrows;
-            int y = 0, x = 0;
-            long long b = 0;
-            if (row_ok) {
-                x = (int)(m % k.Wr);
-                const long long t = m / k.Wr;
-                y = (int)(t % k.Hr);
-                b = t / k.Hr;
+            // the four A rows of this thread: source pixel of tap (0, 0) and image base, or sy = INT_MIN / 2
+            // for rows past the end (every tap then fails the bounds test)
+            int sy[4], sx[4];
+            const bf16 *img[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const long long m = m0 + 32 * i;
+                if (m < k.Mrows) {
+                    const int x = (int)(m % k.Wr);
+                    const long long t = m / k.Wr;
+                    const int y = (int)(t % k.Hr);
+                    sy[i] = y * a.s_mul + a.s_oy;
+                    sx[i] = x * a.s_mul + a.s_ox;
+                    img[i] = a.S + (t / k.Hr) * a.Hs * a.Ws * a.lds;
+                } else {
+                    sy[i] = -(1 << 30);
+                    sx[i] = 0;
+                    img[i] = a.S;
+                }
             }
-            const int sy0 = y * a.s_mul + a.s_oy, sx0 = x * a.s_mul + a.s_ox;
-            const bf16 *src_img = a.S + b * a.Hs * a.Ws * a.lds;
-            // A walk: flattened chunk index of this thread's group is kb * 8 + 4 h
-            int tA = (4 * h) / a.ck, cA = (4 * h) % a.ck;
-            // B walk: flattened chunk index kb * 8 + jB
-            int tB = jB / a.ck, cB = jB % a.ck;
-            const bf16 *b_src0 = a.Wm + (long long)(n0 + rB) * a.w_row;
-            int nBv = (a.N - n0 - rB + 31) / 32;          // B rows of this thread that exist
-            const int nBt = (BN - rB + 31) / 32;          // B rows of this thread inside the tile
+            int tK = c / a.ck, cK = c % a.ck;   // tap and chunk inside the tap of flattened chunk kb * 8 + c
+            const bf16 *b_src0 = a.Wm + (long long)(n0 + rg) * a.w_row;
+            int nBv = (a.N - n0 - rg + 31) / 32;          // B rows of this thread that exist
+            const int nBt = (BN - rg + 31) / 32;          // B rows of this thread inside the tile
             nBv = nBv < 0 ? 0 : (nBv > nBt ? nBt : nBv);
+            const long long rstep = 32ll * a.w_row;
             for (int kb = 0; kb < nkb; ++kb, ++it) {
                 const int s = it % S;
                 ok = mbar_wait(&pipe->empty[s], ((it / S) & 1) ^ 1, abort_flag, a.status);
                 if (!ok) break;
-                const uint32_t st = smem_base + s * stage_bytes;
-                if (fast) {
-                    bool v = row_ok && tA < ntaps;
-                    const bf16 *src = a.S;
-                    if (v) {
-                        const int yy = sy0 + k.taps.dy[tA], xx = sx0 + k.taps.dx[tA];
-                        v = (unsigned)yy < (unsigned)a.Hs && (unsigned)xx < (unsigned)a.Ws;
-                        if (v) src = src_img + ((yy * a.Ws + xx) * a.lds + cA * 8);
-                    }
-                    const uint32_t d = st + a_dst0;
+                const uint32_t d = smem_base + s * stage_bytes + dst0;
+                const bool kv = tK < ntaps;
+                const int dy = kv ? k.taps.dy[tK] : 0, dx = kv ? k.taps.dx[tK] : 0;
 #pragma unroll
-                    for (int j = 0; j < 4; ++j)
-                        cp_async16(d + ((((uint32_t)(4 * h + j)) ^ sw) << 4), src + j * 8, v);
-                    cA += 8;
-                    while (cA >= a.ck) { cA -= a.ck; ++tA; }
-                } else {
-                    int t = tA, cc = cA;
-                    for (int j = 0; j < 4; ++j) {
-                        while (cc >= a.ck) { cc -= a.ck; ++t; }
-                        bool v = row_ok && t < ntaps;
-                        const bf16 *src = a.S;
-                        if (v) {
-                            const int yy = sy0 + k.taps.dy[t], xx = sx0 + k.taps.dx[t];
-                            v = (unsigned)yy < (unsigned)a.Hs && (unsigned)xx < (unsigned)a.Ws;
-                            if (v) src = src_img + ((yy * a.Ws + xx) * a.lds + cc * 8);
-                        }
-                        cp_async16(st + a_dst0 + ((((uint32_t)(4 * h + j)) ^ sw) << 4), src, v);
-                        ++cc;
-                    }
-                    cA += 8;
-                    while (cA >= a.ck) { cA -= a.ck; ++tA; }
+                for (int i = 0; i < 4; ++i) {
+                    const int yy = sy[i] + dy, xx = sx[i] + dx;
+                    const bool v = kv && (unsigned)yy < (unsigned)a.Hs && (unsigned)xx < (unsigned)a.Ws;
+                    const bf16 *src = v ? img[i] + ((yy * a.Ws + xx) * a.lds + cK * 8) : a.S;
+                    cp_async16_ca(d + (uint32_t)i * 4096u, src, v);
                 }
                 {
-                    const bool kv = tB < ntaps;
-                    const bf16 *src = b_src0 + (kv ? (int)k.taps.wt[tB] * a.w_tap + cB * 8 : 0);
-                    const uint32_t d = st + b_dst0;
-                    const long long rstep = 32ll * a.w_row;
+                    const bf16 *src = b_src0 + (kv ? (int)k.taps.wt[tK] * a.w_tap + cK * 8 : 0);
+                    const uint32_t db = d + 16384u;
                     for (int i = 0; i < nBt; ++i) {
                         const bool v = kv && i < nBv;
-                        cp_async16(d + (uint32_t)i * 4096u, v ? src + i * rstep : a.Wm, v);
+                        cp_async16(db + (uint32_t)i * 4096u, v ? src + i * rstep : a.Wm, v);
                     }
-                    cB += 8;
-                    while (cB >= a.ck) { cB -= a.ck; ++tB; }
                 }
+                cK += 8;
+                while (cK >= a.ck) { cK -= a.ck; ++tK; }
                 cp_async_arrive(&pipe->full[s]);
             }
         }
@@ -459,6 +328,7 @@ struct WArgs {
     int ldy, Co;
     long long Mtot;        // B * Ho * Wo
     long long m_per_split; // multiple of 64
+    int db64, doh64, dow64; // 64 rows = db64 images + doh64 output rows + dow64 pixels
     int Kfwd;              // ksz * ksz * Ci
     int BN;
     int stages;
@@ -501,23 +371,30 @@ __global__ void __launch_bounds__(kThreads) igemm_wgrad_kernel(const __grid_cons
     const uint32_t smem_base = smem_u32(smem);
 
     if (warp < 4) {
+        // Thread p owns 16-byte chunk column c16 = p % 16 of the 128-column A tile (and of each pair of
+        // 64-column B blocks) and rows p / 16 + 8 i, so that the lanes of a row read contiguous bytes.
         const int p = threadIdx.x;
-        const int r = p & 63, half = p >> 6;
-        // this thread's 8 A chunks: columns j0 + half*64 + 8 q, fixed for the whole kernel
-        int a_off[8];       // element offset of the chunk inside a source pixel, or -1 when past Kfwd
-        signed char a_dy[8], a_dx[8];
-#pragma unroll
-        for (int q = 0; q < 8; ++q) {
+        const int c16 = p & 15, rg = p >> 4, half = c16 >> 3, q = c16 & 7;
+        int a_off = -1, a_dy = 0, a_dx = 0;   // this thread's column: offset inside a source pixel and its tap
+        {
             const int jj = j0 + half * 64 + q * 8;
             if (jj < a.Kfwd) {
                 const int t = jj / a.Ci;
-                a_off[q] = jj - t * a.Ci;
-                a_dy[q] = (signed char)(t / a.ksz);
-                a_dx[q] = (signed char)(t % a.ksz);
-            } else {
-                a_off[q] = -1;
-                a_dy[q] = a_dx[q] = 0;
+                a_off = jj - t * a.Ci;
+                a_dy = t / a.ksz - a.pad;
+                a_dx = t % a.ksz - a.pad;
             }
+        }
+        const uint32_t dst0 = (uint32_t)half * 8192u + (uint32_t)rg * 128u + (((uint32_t)q ^ ((uint32_t)rg & 7u)) << 4);
+        // output pixel of each of the 8 rows, advanced by 64 rows per K block without divisions
+        int ow[8], oh[8], ob[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const long long m = m_lo + rg + 8 * i;
+            ow[i] = (int)(m % a.Wo);
+            const long long t = m / a.Wo;
+            oh[i] = (int)(t % a.Ho);
+            ob[i] = (int)(t / a.Ho);
         }
         const int co_lim = min(a.ldy, co0 + BN);  // dY columns that exist in memory for this tile
         bool ok = true;
@@ -525,36 +402,28 @@ __global__ void __launch_bounds__(kThreads) igemm_wgrad_kernel(const __grid_cons
             const int s = kb % S;
             ok = mbar_wait(&pipe->empty[s], ((kb / S) & 1) ^ 1, abort_flag, a.status);
             if (!ok) break;
-            const uint32_t sa = smem_base + s * stage_bytes, sb = sa + 16384u;
-            const long long m = m_lo + (long long)kb * 64 + r;
-            const bool row_ok = m < m_hi;
-            int oh = 0, ow = 0;
-            long long b = 0;
-            if (row_ok) {
-                ow = (int)(m % a.Wo);
-                const long long t = m / a.Wo;
-                oh = (int)(t % a.Ho);
-                b = t / a.Ho;
-            }
-            const int y0 = 2 * oh - a.pad, x0 = 2 * ow - a.pad;
-            const bf16 *img = a.X + b * a.Hi * a.Wi * a.Ci;
-            const uint32_t arow = sa + half * 8192 + r * 128;
+            const uint32_t sa = smem_base + s * stage_bytes + dst0, sb = sa + 16384u - (uint32_t)half * 8192u;
+            const long long mb = m_lo + (long long)kb * 64 + rg;
 #pragma unroll
-            for (int q = 0; q < 8; ++q) {
-                const int yy = y0 + a_dy[q], xx = x0 + a_dx[q];
-                const bool v = row_ok && a_off[q] >= 0 && yy >= 0 && yy < a.Hi && xx >= 0 && xx < a.Wi;
-                const bf16 *src = v ? img + ((long long)yy * a.Wi + xx) * a.Ci + a_off[q] : a.X;
-                cp_async16(arow + ((q ^ (r & 7)) << 4), src, v);
-            }
-            const bf16 *dyrow = a.dY + m * a.ldy;
-            for (int blk = half; blk < nblkB; blk += 2) {
-                const uint32_t brow = sb + blk * 8192 + r * 128;
-#pragma unroll
-                for (int q = 0; q < 8; ++q) {
+            for (int i = 0; i < 8; ++i) {
+                const long long m = mb + 8 * i;
+                const bool row_ok = m < m_hi;
+                const int yy = 2 * oh[i] + a_dy, xx = 2 * ow[i] + a_dx;
+                const bool v = row_ok && a_off >= 0 && (unsigned)yy < (unsigned)a.Hi && (unsigned)xx < (unsigned)a.Wi;
+                const bf16 *src = v ? a.X + (((long long)ob[i] * a.Hi + yy) * a.Wi + xx) * a.Ci + a_off : a.X;
+                cp_async16_ca(sa + (uint32_t)i * 1024u, src, v);
+                const bf16 *dyrow = a.dY + m * a.ldy;
+                for (int blk = half; blk < nblkB; blk += 2) {
                     const int co = co0 + blk * 64 + q * 8;
-                    const bool v = row_ok && co < co_lim;
-                    cp_async16(brow + ((q ^ (r & 7)) << 4), v ? dyrow + co : a.dY, v);
+                    const bool vb = row_ok && co < co_lim;
+                    cp_async16(sb + (uint32_t)blk * 8192u + (uint32_t)i * 1024u, vb ? dyrow + co : a.dY, vb);
                 }
+                // next K block: 64 rows further
+                ow[i] += a.dow64;
+                if (ow[i] >= a.Wo) { ow[i] -= a.Wo; ++oh[i]; }
+                oh[i] += a.doh64;
+                if (oh[i] >= a.Ho) { oh[i] -= a.Ho; ++ob[i]; }
+                ob[i] += a.db64;
             }
             cp_async_arrive(&pipe->full[s]);
         }
@@ -754,6 +623,9 @@ int tc_gemm_wgrad(const ConvGeom &g, const bf16 *dY, int ldy, const bf16 *X, flo
     if (per < 256) per = 256;
     splits = (a.Mtot + per - 1) / per;
     a.m_per_split = per;
+    a.db64 = 64 / (g.Ho * g.Wo);
+    a.doh64 = (64 % (g.Ho * g.Wo)) / g.Wo;
+    a.dow64 = 64 % g.Wo;
     dim3 grid((unsigned)((a.Kfwd + 127) / 128), (unsigned)((g.Co + a.BN - 1) / a.BN), (unsigned)splits);
     igemm_wgrad_kernel<<<grid, kThreads, wgrad_smem(a.BN), st>>>(a);
     PPO_LAUNCH_CHECK();

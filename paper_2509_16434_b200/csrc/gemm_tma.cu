@@ -1,0 +1,798 @@
+// TMA-fed tensor-core versions of the encoder's implicit GEMMs for sm_100a.
+//
+// One elected thread moves whole operand tiles with cp.async.bulk.tensor (TMA): a box of the NHWC
+// activation tensor with a traversal stride of 2 along W and H *is* the im2col tile of one kernel tap
+// of a stride-2 convolution, zero padding included (out-of-range parts of a box arrive as zeros), and
+// it lands in shared memory already in the swizzled image the UMMA descriptors name.  A second thread
+// issues tcgen05.mma into a double-buffered accumulator in tensor memory; four warps read it back with
+// tcgen05.ld for the epilogue.  No thread computes an address per element.
+//
+//  tma_kmajor_kernel : D[m][n] = sum_k A[m][k] B[n][k], both operands K-major.
+//      forward  A = tap boxes of X (row m = output pixel), B = W[co][tap][ci]
+//      dgrad    A = shifted boxes of dY (row m = input pixel of one stride-parity class), B = Wt[ci][tap][co]
+//  tma_wgrad_kernel  : D[j][co] = sum_m A[m][j] B[m][co], both operands MN-major: the same tap boxes of X
+//      and plain boxes of dY, read with the pixel index as the reduction; split over pixel tiles across
+//      CTAs, fp32 atomics into dW.
+//
+// Tiles follow the pixel grid instead of cutting the flattened pixel index every 128: a tile is R whole
+// rows of the (image, row) sequence (R * width <= 128), fetched as a few boxes of 1, 2, 4, ... rows that
+// never straddle an image, or a 128-pixel segment of one row when rows are longer than 128 (the fully
+// connected layers, whose "row" is the batch).  Rows of the 128-row MMA tile beyond R * width are not
+// written and their results are ignored.
+//
+// Shared-memory rows are 128 bytes (64 channels, SWIZZLE_128B) or 64 bytes (32 channels, SWIZZLE_64B).
+// Every wait is bounded: on a time-out the kernel records PPO_ERR_TIMEOUT, waits (bounded) for the
+// copies it has in flight, frees its tensor memory and returns.
+#include <cuda.h>  // CUtensorMap and its enums; the encoder is reached through the runtime's entry-point query
+
+#include "gemm.cuh"
+#include "tcgen05.cuh"
+
+namespace {
+
+using namespace tc;
+
+constexpr int kMaxTaps = 49;
+constexpr int kMaxBoxes = 32;    // boxes per tile; rows per tile are capped at 32 so that this always holds
+constexpr int kMaxHeights = 6;   // box heights 1, 2, 4, 8, 16, 32 rows
+constexpr int kMaxStages = 8;
+constexpr int kThreads = 192;    // warp 0: TMA producer, warp 1: MMA issue and TMEM owner, warps 2-5: epilogue
+constexpr size_t kSmemBudget = 200 * 1024;
+
+struct Taps {
+    int n;
+    signed char dy[kMaxTaps], dx[kMaxTaps];
+    short wt[kMaxTaps];  // index of the tap inside the weight tensor
+};
+
+// Pixel grid the rows of a GEMM walk: Nimg images of Hr rows of Wr pixels.
+struct RowGrid {
+    int Wr, Hr, Nimg;
+    int R;      // grid rows per tile when Wr <= 128, else 0: a tile is a 128-pixel segment of one row
+    int xsegs;  // segments per row when R == 0
+    int tiles;  // tiles over the whole grid
+    int arows;  // pixel rows a tile fills in shared memory: R * Wr, or 128
+};
+
+struct Box {
+    int n, y, x;  // image, first row, first pixel
+    int hl;       // log2 of the box height in rows
+    int rowoff;   // first shared-memory row of the box
+};
+
+struct Pipe {
+    uint64_t full[kMaxStages];
+    uint64_t empty[kMaxStages];
+    uint64_t tfull[2];
+    uint64_t tempty[2];
+    uint32_t tmem_slot;
+    int abort_flag;
+    Box boxes[kMaxBoxes];
+};
+
+// Boxes of tile `tile`, in shared-memory row order.  Rows past the last image get an image index >= Nimg,
+// which the copy engine answers with zeros.  Called by one thread.
+__device__ int build_boxes(const RowGrid &g, int tile, Box *out) {
+    if (g.R == 0) {
+        const int frow = tile / g.xsegs, xs = tile - frow * g.xsegs;
+        const int n = frow / g.Hr;
+        out[0] = {n, frow - n * g.Hr, xs * 128, 0, 0};
+        return 1;
+    }
+    int f = tile * g.R, nb = 0, off = 0;
+    const int fend = f + g.R;
+    while (f < fend) {
+        const int n = f / g.Hr;
+        int y = f - n * g.Hr;
+        int seg = min(g.Hr - y, fend - f);
+        while (seg > 0) {
+            const int hl = 31 - __clz(seg), h = 1 << hl;
+            out[nb++] = {n, y, 0, hl, off};
+            y += h;
+            f += h;
+            off += h * g.Wr;
+            seg -= h;
+        }
+    }
+    return nb;
+}
+
+// After a time-out: bounded wait for the copies of the last `S` armed stages (iterations it-S .. it-1).
+__device__ void drain_copies(Pipe *pipe, int it, int S) {
+    for (int i = max(0, it - S); i < it; ++i) {
+        const long long t0 = clock64();
+        while (!mbar_try_wait(&pipe->full[i % S], (i / S) & 1))
+            if (clock64() - t0 > kWaitCycles / 4) break;
+    }
+}
+
+// ------------------------------------------------------------------ K-major ----
+
+struct KClass {
+    int o_oy, o_ox;  // output pixel = (y * o_mul + o_oy, x * o_mul + o_ox)
+    Taps taps;
+};
+
+enum { EPI_FWD = 0, EPI_HEAD = 1, EPI_DGRAD = 2 };
+
+struct KArgs {
+    CUtensorMap mapA[kMaxHeights];
+    CUtensorMap mapB;
+    RowGrid grid;
+    int s_mul, s_oy, s_ox;  // source pixel of tap t: (y * s_mul + s_oy + dy[t], x * s_mul + s_ox + dx[t])
+    int CB, row_bytes;      // channels per box (64 or 32) and bytes of a shared-memory row
+    int kchunks;            // boxes along the channels of one tap
+    int w_tap;              // elements between taps in a weight row
+    int N, BN, tiles_n, tiles_per_cls, total_tiles, ncls, stages;
+    uint32_t tx_bytes;      // bytes one K block brings in
+    int o_mul, Hout, Wout, ldo;
+    int mode, relu, A;
+    const float *bias;
+    bf16 *out;
+    float *out_f32;
+    const bf16 *mask;
+    float *mean, *value;
+    int32_t *status;
+    KClass cls[4];
+};
+
+__global__ void __launch_bounds__(kThreads, 1) tma_kmajor_kernel(const __grid_constant__ KArgs a) {
+    extern __shared__ __align__(1024) uint8_t smem_raw[];
+    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    const int BN = a.BN, S = a.stages;
+    const uint32_t rb = (uint32_t)a.row_bytes;
+    const uint32_t a_bytes = 128u * rb;
+    const uint32_t stage_bytes = a_bytes + (uint32_t)BN * rb;
+    Pipe *pipe = reinterpret_cast<Pipe *>(smem + (size_t)S * stage_bytes);
+    volatile int *abort_flag = &pipe->abort_flag;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t acc_cols = tmem_cols_for(BN);
+    const uint32_t ncols = acc_cols * 2;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < S; ++s) {
+            mbar_init(&pipe->full[s], 1);
+            mbar_init(&pipe->empty[s], 1);
+        }
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(&pipe->tfull[i], 1);
+            mbar_init(&pipe->tempty[i], 128);
+        }
+        pipe->abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) tmem_alloc(&pipe->tmem_slot, ncols);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = pipe->tmem_slot;
+    const uint32_t smem_base = smem_u32(smem);
+
+    if (warp == 0) {
+        // ---------------- TMA producer
+        if (lane == 0) {
+            int it = 0;
+            bool ok = true;
+            for (int g = blockIdx.x; g < a.total_tiles && ok; g += gridDim.x) {
+                const int c = g / a.tiles_per_cls, local = g - c * a.tiles_per_cls;
+                const int mt = local / a.tiles_n, n0 = (local - mt * a.tiles_n) * BN;
+                const KClass &k = a.cls[c];
+                const int nb = build_boxes(a.grid, mt, pipe->boxes);
+                for (int t = 0; t < k.taps.n && ok; ++t) {
+                    const int dy = a.s_oy + k.taps.dy[t], dx = a.s_ox + k.taps.dx[t];
+                    const int wcol = (int)k.taps.wt[t] * a.w_tap;
+                    for (int kc = 0; kc < a.kchunks; ++kc, ++it) {
+                        const int s = it % S;
+                        ok = mbar_wait(&pipe->empty[s], ((it / S) & 1) ^ 1, abort_flag, a.status);
+                        if (!ok) break;
+                        mbar_arrive_expect_tx(&pipe->full[s], a.tx_bytes);
+                        const uint32_t sa = smem_base + (uint32_t)s * stage_bytes;
+                        for (int b = 0; b < nb; ++b) {
+                            const Box bx = pipe->boxes[b];
+                            tma_load_4d(sa + (uint32_t)bx.rowoff * rb, &a.mapA[bx.hl], &pipe->full[s], kc * a.CB,
+                                        bx.x * a.s_mul + dx, bx.y * a.s_mul + dy, bx.n);
+                        }
+                        tma_load_2d(sa + a_bytes, &a.mapB, &pipe->full[s], wcol + kc * a.CB, n0);
+                    }
+                }
+            }
+            if (!ok) drain_copies(pipe, it, S);
+        }
+        __syncwarp();
+    } else if (warp == 1) {
+        // ---------------- MMA issue: one thread feeds the tensor core
+        const uint32_t idesc = instr_desc(128, BN, 0, 0);
+        const int nk = a.CB >> 4;  // K = 16 steps per box
+        const uint32_t sbo = 8u * rb;
+        int it = 0, ti = 0;
+        bool ok = true;
+        for (int g = blockIdx.x; g < a.total_tiles && ok; g += gridDim.x, ++ti) {
+            const int c = g / a.tiles_per_cls;
+            const int nkb = a.cls[c].taps.n * a.kchunks;
+            const int acc = ti & 1;
+            ok = mbar_wait(&pipe->tempty[acc], ((ti >> 1) & 1) ^ 1, abort_flag, a.status);
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t tmem_d = tmem_base + acc * acc_cols;
+            for (int kb = 0; kb < nkb; ++kb, ++it) {
+                const int s = it % S;
+                ok = mbar_wait(&pipe->full[s], (it / S) & 1, abort_flag, a.status);
+                if (!ok) break;
+                tc_fence_after();
+                if (lane == 0) {
+                    const uint32_t sa = smem_base + (uint32_t)s * stage_bytes, sb = sa + a_bytes;
+                    for (int kk = 0; kk < nk; ++kk)  // K = 16 elements = 32 bytes along the swizzled row
+                        umma_bf16(tmem_d, smem_desc_sw(sa + kk * 32, 16, sbo, rb), smem_desc_sw(sb + kk * 32, 16, sbo, rb),
+                                  idesc, (kb > 0 || kk > 0) ? 1u : 0u);
+                    umma_commit(&pipe->empty[s]);
+                }
+                __syncwarp();
+            }
+            if (ok && lane == 0) umma_commit(&pipe->tfull[acc]);
+            __syncwarp();
+        }
+    } else {
+        // ---------------- epilogue: warp w reads TMEM lanes 32 (w % 4) .. +31
+        const int lg = warp & 3;
+        const int p = lg * 32 + lane;
+        const RowGrid &gr = a.grid;
+        int ti = 0;
+        bool ok = true;
+        for (int g = blockIdx.x; g < a.total_tiles && ok; g += gridDim.x, ++ti) {
+            const int c = g / a.tiles_per_cls, local = g - c * a.tiles_per_cls;
+            const int mt = local / a.tiles_n, n0 = (local - mt * a.tiles_n) * BN;
+            const KClass &k = a.cls[c];
+            // pixel of tile row p
+            bool row_ok;
+            int n, y, x;
+            if (gr.R == 0) {
+                const int frow = mt / gr.xsegs, xs = mt - frow * gr.xsegs;
+                n = frow / gr.Hr;
+                y = frow - n * gr.Hr;
+                x = xs * 128 + p;
+                row_ok = x < gr.Wr;
+            } else {
+                const int fr = p / gr.Wr;
+                x = p - fr * gr.Wr;
+                const int f = mt * gr.R + fr;
+                n = f / gr.Hr;
+                y = f - n * gr.Hr;
+                row_ok = fr < gr.R && n < gr.Nimg;
+            }
+            const int oy = y * a.o_mul + k.o_oy, ox = x * a.o_mul + k.o_ox;
+            row_ok = row_ok && oy < a.Hout && ox < a.Wout;
+            const long long orow = row_ok ? ((long long)n * a.Hout + oy) * a.Wout + ox : 0;
+            const int acc = ti & 1;
+            ok = mbar_wait(&pipe->tfull[acc], (ti >> 1) & 1, abort_flag, a.status);
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t lane_base = tmem_base + acc * acc_cols + ((uint32_t)(lg * 32) << 16);
+            for (int c0 = 0; c0 < BN; c0 += 16) {
+                if (n0 + c0 >= a.N) break;  // uniform across the warp
+                float v[16];
+                tmem_ld16(lane_base + (uint32_t)c0, v);
+                if (!row_ok) continue;
+                const int nn = n0 + c0;
+                if (a.mode == EPI_HEAD) {
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) {
+                        if (nn + i < a.A) a.mean[orow * a.A + nn + i] = v[i] + a.bias[nn + i];
+                        else if (nn + i == a.A) a.value[orow] = v[i] + a.bias[nn + i];
+                    }
+                    continue;
+                }
+                if (a.mode == EPI_FWD) {
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) {
+                        const float bv = (nn + i < a.N) ? a.bias[nn + i] : 0.f;
+                        v[i] += bv;
+                        if (a.relu) v[i] = fmaxf(v[i], 0.f);
+                    }
+                } else if (a.mask) {
+                    const uint4 *mp = reinterpret_cast<const uint4 *>(a.mask + orow * a.ldo + nn);
+#pragma unroll
+                    for (int hlf = 0; hlf < 2; ++hlf) {
+                        if (nn + hlf * 8 < a.N) {
+                            const uint4 mk = mp[hlf];
+                            const __nv_bfloat162 *m2 = reinterpret_cast<const __nv_bfloat162 *>(&mk);
+#pragma unroll
+                            for (int i = 0; i < 4; ++i) {
+                                const float2 f = __bfloat1622float2(m2[i]);
+                                if (!(f.x > 0.f)) v[hlf * 8 + 2 * i] = 0.f;
+                                if (!(f.y > 0.f)) v[hlf * 8 + 2 * i + 1] = 0.f;
+                            }
+                        }
+                    }
+                }
+                if (a.out) {
+                    uint4 *op = reinterpret_cast<uint4 *>(a.out + orow * a.ldo + nn);
+#pragma unroll
+                    for (int hlf = 0; hlf < 2; ++hlf) {
+                        if (nn + hlf * 8 < a.N) {
+                            __nv_bfloat162 pk[4];
+#pragma unroll
+                            for (int i = 0; i < 4; ++i)
+                                pk[i] = __floats2bfloat162_rn(v[hlf * 8 + 2 * i], v[hlf * 8 + 2 * i + 1]);
+                            op[hlf] = *reinterpret_cast<uint4 *>(pk);
+                        }
+                    }
+                }
+                if (a.out_f32) {
+                    float4 *op = reinterpret_cast<float4 *>(a.out_f32 + orow * a.ldo + nn);
+#pragma unroll
+                    for (int q = 0; q < 4; ++q)
+                        if (nn + q * 4 < a.N) op[q] = make_float4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
+                }
+            }
+            tc_fence_before();
+            mbar_arrive(&pipe->tempty[acc]);
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, ncols);
+    }
+}
+
+// -------------------------------------------------------------------- wgrad ----
+
+struct WArgs {
+    CUtensorMap mapA[kMaxHeights];  // tap boxes of X (traversal stride 2 for a convolution)
+    CUtensorMap mapB[kMaxHeights];  // boxes of dY over the same pixels
+    RowGrid grid;                   // output pixels
+    int s_mul, pad, ksz, ntaps;
+    int CB, rbA, mblocks, kchunks;  // A: channels per box, row bytes, boxes per 128 columns, boxes per tap
+    int CBn, rbB, nblocks, BN;      // B: likewise over the output channels of this tile
+    int Kfwd, Co;
+    int tiles_per_split, nmma, stages;
+    float *dW;                      // [Co][Kfwd], accumulated with atomics
+    int32_t *status;
+};
+
+__global__ void __launch_bounds__(kThreads, 1) tma_wgrad_kernel(const __grid_constant__ WArgs a) {
+    extern __shared__ __align__(1024) uint8_t smem_raw[];
+    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    const int BN = a.BN, S = a.stages;
+    const uint32_t rbA = (uint32_t)a.rbA, rbB = (uint32_t)a.rbB;
+    const uint32_t a_bytes = 128u * 256u;                 // 128 pixel rows x 128 columns of bf16
+    const uint32_t stage_bytes = a_bytes + 128u * 2u * (uint32_t)BN;
+    Pipe *pipe = reinterpret_cast<Pipe *>(smem + (size_t)S * stage_bytes);
+    volatile int *abort_flag = &pipe->abort_flag;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t ncols = tmem_cols_for(BN);
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < S; ++s) {
+            mbar_init(&pipe->full[s], 1);
+            mbar_init(&pipe->empty[s], 1);
+        }
+        mbar_init(&pipe->tfull[0], 1);
+        pipe->abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    // Rows and column blocks no copy ever writes must read as zeros: the pixel index is the reduction.
+    {
+        uint4 *z = reinterpret_cast<uint4 *>(smem);
+        const uint32_t n16 = (uint32_t)S * stage_bytes / 16u;
+        for (uint32_t i = threadIdx.x; i < n16; i += kThreads) z[i] = make_uint4(0, 0, 0, 0);
+        fence_async_smem();
+    }
+    if (warp == 1) tmem_alloc(&pipe->tmem_slot, ncols);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_d = pipe->tmem_slot;
+    const uint32_t smem_base = smem_u32(smem);
+
+    const int jb0 = blockIdx.x * a.mblocks;  // first (tap, channel chunk) box of this column tile
+    const int co0 = blockIdx.y * BN;
+    const int t_lo = blockIdx.z * a.tiles_per_split;
+    const int t_hi = min(a.grid.tiles, t_lo + a.tiles_per_split);
+    const int nkb = max(0, t_hi - t_lo);
+    int nvalid = 0;
+    for (int i = 0; i < a.mblocks; ++i)
+        if ((jb0 + i) / a.kchunks < a.ntaps) ++nvalid;
+    const uint32_t tx_bytes = (uint32_t)a.grid.arows * ((uint32_t)nvalid * rbA + (uint32_t)a.nblocks * rbB);
+
+    if (warp == 0) {
+        if (lane == 0) {
+            bool ok = true;
+            int kb = 0;
+            for (; kb < nkb; ++kb) {
+                const int s = kb % S;
+                ok = mbar_wait(&pipe->empty[s], ((kb / S) & 1) ^ 1, abort_flag, a.status);
+                if (!ok) break;
+                mbar_arrive_expect_tx(&pipe->full[s], tx_bytes);
+                const uint32_t sa = smem_base + (uint32_t)s * stage_bytes, sb = sa + a_bytes;
+                const int nb = build_boxes(a.grid, t_lo + kb, pipe->boxes);
+                for (int b = 0; b < nb; ++b) {
+                    const Box bx = pipe->boxes[b];
+                    for (int i = 0; i < a.mblocks; ++i) {
+                        const int jb = jb0 + i, tap = jb / a.kchunks, kc = jb - tap * a.kchunks;
+                        if (tap >= a.ntaps) break;
+                        const int kh = tap / a.ksz, kw = tap - kh * a.ksz;
+                        tma_load_4d(sa + (uint32_t)i * 128u * rbA + (uint32_t)bx.rowoff * rbA, &a.mapA[bx.hl],
+                                    &pipe->full[s], kc * a.CB, bx.x * a.s_mul - a.pad + kw, bx.y * a.s_mul - a.pad + kh,
+                                    bx.n);
+                    }
+                    for (int i = 0; i < a.nblocks; ++i)
+                        tma_load_4d(sb + (uint32_t)i * 128u * rbB + (uint32_t)bx.rowoff * rbB, &a.mapB[bx.hl],
+                                    &pipe->full[s], co0 + i * a.CBn, bx.x, bx.y, bx.n);
+                }
+            }
+            if (!ok) drain_copies(pipe, kb, S);
+        }
+        __syncwarp();
+    } else if (warp == 1) {
+        const uint32_t idesc = instr_desc(128, BN, 1, 1);
+        bool ok = true;
+        for (int kb = 0; kb < nkb && ok; ++kb) {
+            const int s = kb % S;
+            ok = mbar_wait(&pipe->full[s], (kb / S) & 1, abort_flag, a.status);
+            if (!ok) break;
+            tc_fence_after();
+            if (lane == 0) {
+                const uint32_t sa = smem_base + (uint32_t)s * stage_bytes, sb = sa + a_bytes;
+                for (int k = 0; k < a.nmma; ++k)  // 16 pixel rows per instruction
+                    umma_bf16(tmem_d, smem_desc_sw(sa + (uint32_t)k * 16u * rbA, 128u * rbA, 8u * rbA, rbA),
+                              smem_desc_sw(sb + (uint32_t)k * 16u * rbB, 128u * rbB, 8u * rbB, rbB), idesc,
+                              (kb > 0 || k > 0) ? 1u : 0u);
+                umma_commit(&pipe->empty[s]);
+            }
+            __syncwarp();
+        }
+        if (ok && nkb > 0 && lane == 0) umma_commit(&pipe->tfull[0]);
+        __syncwarp();
+    } else if (nkb > 0) {
+        // ---------------- epilogue: TMEM lane p is column j of dW^T
+        const int lg = warp & 3;
+        const int p = lg * 32 + lane;
+        if (mbar_wait(&pipe->tfull[0], 0, abort_flag, a.status)) {
+            tc_fence_after();
+            const int jj = jb0 * a.CB + p;
+            const uint32_t lane_base = tmem_d + ((uint32_t)(lg * 32) << 16);
+            for (int c0 = 0; c0 < BN; c0 += 16) {
+                if (co0 + c0 >= a.Co) break;
+                float v[16];
+                tmem_ld16(lane_base + (uint32_t)c0, v);
+                if (jj >= a.Kfwd) continue;
+#pragma unroll
+                for (int i = 0; i < 16; ++i) {
+                    const int co = co0 + c0 + i;
+                    if (co < a.Co) atomicAdd(a.dW + (long long)co * a.Kfwd + jj, v[i]);
+                }
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_d, ncols);
+    }
+}
+
+// --------------------------------------------------------------------- host ----
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    static bool tried = false;
+    if (!tried) {
+        tried = true;
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+// Map of a bf16 tensor [d3][d2][d1][d0] whose innermost rows are `ld` elements apart; box and traversal
+// strides innermost first.  `row_bytes` selects the swizzle (box[0] * 2 == row_bytes).
+int make_map(CUtensorMap *m, const void *base, int rank, const long long *dims, long long ld, const int *box,
+             const int *estride, int row_bytes) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return PPO_ERR_CUDA;
+    cuuint64_t gd[4];
+    cuuint64_t gs[3];
+    cuuint32_t bx[4], es[4];
+    for (int i = 0; i < rank; ++i) {
+        gd[i] = (cuuint64_t)dims[i];
+        bx[i] = (cuuint32_t)box[i];
+        es[i] = (cuuint32_t)estride[i];
+        if (box[i] < 1 || box[i] > 256 || dims[i] < 1) return PPO_ERR_UNSUPPORTED;
+    }
+    long long s = ld * 2;
+    for (int i = 0; i + 1 < rank; ++i) {
+        if (s % 16 != 0 || s >= (1ll << 40)) return PPO_ERR_UNSUPPORTED;
+        gs[i] = (cuuint64_t)s;
+        s *= dims[i + 1];
+    }
+    if (box[0] * 2 != row_bytes || !ppo_aligned(base, 16)) return PPO_ERR_UNSUPPORTED;
+    const CUtensorMapSwizzle sw = row_bytes == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B;
+    const CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void *>(base), gd, gs, bx,
+                          es, CU_TENSOR_MAP_INTERLEAVE_NONE, sw, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? PPO_OK : PPO_ERR_CUDA;
+}
+
+// Channels per box for a source of C channels per pixel (`flat`: a 1x1 image, where a ragged last box is
+// completed with zeros by the copy engine), or 0 when the TMA kernels do not cover it.
+int channels_per_box(int C, bool flat) {
+    if (C % 64 == 0) return 64;
+    if (flat) return (C >= 64 && C % 8 == 0) ? 64 : 0;
+    return C % 32 == 0 ? 32 : 0;
+}
+
+bool make_grid(RowGrid &g, int Wr, int Hr, int Nimg, int row_bytes_min) {
+    g.Wr = Wr; g.Hr = Hr; g.Nimg = Nimg;
+    if (Wr <= 128) {
+        const long long rows = (long long)Nimg * Hr;
+        int R = 128 / Wr;
+        if (R > kMaxBoxes) R = kMaxBoxes;
+        if (R > rows) R = (int)rows;
+        g.R = R;
+        g.xsegs = 1;
+        const long long tiles = (rows + R - 1) / R;
+        if (tiles > 0x3fffffff) return false;
+        g.tiles = (int)tiles;
+        g.arows = R * Wr;
+        // every box starts a multiple of Wr rows into the stage; the copy engine wants 128-byte alignment
+        if (((long long)Wr * row_bytes_min) % 128 != 0) return false;
+    } else {
+        g.R = 0;
+        g.xsegs = (Wr + 127) / 128;
+        const long long tiles = (long long)Nimg * Hr * g.xsegs;
+        if (tiles > 0x3fffffff) return false;
+        g.tiles = (int)tiles;
+        g.arows = 128;
+    }
+    return true;
+}
+
+// Maps of an activation tensor [Nimg][Hs][Ws][C, row stride ld] for boxes of CB channels, the tile width of
+// `g` and heights 1 << i, traversal stride es along W and H.
+int make_act_maps(CUtensorMap *maps, const bf16 *base, int C, long long ld, int Ws, int Hs, int Nimg,
+                  const RowGrid &g, int CB, int es) {
+    const long long dims[4] = {C, Ws, Hs, Nimg};
+    const int wbox = (g.R == 0 ? 128 : g.Wr) * es;
+    int maxh = 1;
+    if (g.R > 0) while (maxh * 2 <= g.R && maxh * 2 <= g.Hr) maxh *= 2;
+    for (int i = 0; (1 << i) <= maxh; ++i) {
+        const int box[4] = {CB, wbox, (1 << i) * es, 1};
+        const int estr[4] = {1, es, es, 1};
+        const int s = make_map(&maps[i], base, 4, dims, ld, box, estr, CB * 2);
+        if (s != PPO_OK) return s;
+    }
+    return PPO_OK;
+}
+
+int stages_for(size_t stage_bytes) {
+    int s = (int)(kSmemBudget / stage_bytes);
+    return s > kMaxStages ? kMaxStages : s;
+}
+
+int pick_bn(int N) {  // tile width: N split evenly into tiles of at most 256, rounded up to 16
+    const int tiles = (N + 255) / 256;
+    int bn = ((N + tiles - 1) / tiles + 15) / 16 * 16;
+    return bn < 16 ? 16 : bn;
+}
+
+int ensure_smem_attrs() {
+    static bool attr_set[64] = {false};
+    int dev = 0;
+    PPO_CUDA_CHECK(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) return PPO_ERR_CUDA;
+    if (!attr_set[dev]) {
+        const int mx = (int)(kSmemBudget + sizeof(Pipe) + 1024);
+        PPO_CUDA_CHECK(cudaFuncSetAttribute(tma_kmajor_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, mx));
+        PPO_CUDA_CHECK(cudaFuncSetAttribute(tma_wgrad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, mx));
+        attr_set[dev] = true;
+    }
+    return PPO_OK;
+}
+
+int launch_kmajor(KArgs &a, cudaStream_t st) {
+    int s = ensure_smem_attrs();
+    if (s != PPO_OK) return s;
+    a.tiles_n = (a.N + a.BN - 1) / a.BN;
+    const long long per = (long long)a.grid.tiles * a.tiles_n;
+    const long long total = per * a.ncls;
+    if (total <= 0) return PPO_OK;
+    if (total > 0x7fffffffll) return PPO_ERR_UNSUPPORTED;
+    a.tiles_per_cls = (int)per;
+    a.total_tiles = (int)total;
+    const size_t stage = (size_t)(128 + a.BN) * a.row_bytes;
+    a.stages = stages_for(stage);
+    if (a.stages < 2) return PPO_ERR_UNSUPPORTED;
+    a.tx_bytes = (uint32_t)((a.grid.arows + a.BN) * a.row_bytes);
+    const int sms = ppo_num_sms();
+    const unsigned grid = (unsigned)(total < sms ? total : sms);
+    tma_kmajor_kernel<<<grid, kThreads, (size_t)a.stages * stage + sizeof(Pipe) + 1024, st>>>(a);
+    PPO_LAUNCH_CHECK();
+    return PPO_OK;
+}
+
+bool is_flat(const ConvGeom &g) { return g.Hi == 1 && g.Wi == 1 && g.Ho == 1 && g.Wo == 1 && g.k == 1; }
+
+}  // namespace
+
+int tma_gemm_fwd(const ConvGeom &g, const bf16 *X, const bf16 *W, const FwdEpilogue &e, int32_t *status,
+                 cudaStream_t st) {
+    if (!status || g.taps() > kMaxTaps || g.Ci % 8 != 0) return PPO_ERR_UNSUPPORTED;
+    const bool flat = is_flat(g);
+    const int CB = channels_per_box(g.Ci, flat);
+    if (CB == 0) return PPO_ERR_UNSUPPORTED;
+    KArgs a = {};
+    a.CB = CB;
+    a.row_bytes = CB * 2;
+    a.kchunks = (g.Ci + CB - 1) / CB;
+    a.w_tap = g.Ci;
+    // a fully connected layer is one image with a single row of B pixels
+    const bool ok = flat ? make_grid(a.grid, g.B, 1, 1, a.row_bytes) : make_grid(a.grid, g.Wo, g.Ho, g.B, a.row_bytes);
+    if (!ok) return PPO_ERR_UNSUPPORTED;
+    int s = flat ? make_act_maps(a.mapA, X, g.Ci, g.Ci, g.B, 1, 1, a.grid, CB, 1)
+                 : make_act_maps(a.mapA, X, g.Ci, g.Ci, g.Wi, g.Hi, g.B, a.grid, CB, 2);
+    if (s != PPO_OK) return s;
+    a.N = g.Co;
+    a.BN = pick_bn(g.Co);
+    {
+        const long long dims[2] = {g.K(), g.Co};
+        const int box[2] = {CB, a.BN}, es[2] = {1, 1};
+        s = make_map(&a.mapB, W, 2, dims, g.K(), box, es, a.row_bytes);
+        if (s != PPO_OK) return s;
+    }
+    a.s_mul = flat ? 1 : 2;
+    a.s_oy = a.s_ox = -g.pad;
+    a.o_mul = 1;
+    a.Hout = flat ? 1 : g.Ho;
+    a.Wout = flat ? g.B : g.Wo;
+    a.ldo = g.Co;
+    a.mode = e.out ? EPI_FWD : EPI_HEAD;
+    a.relu = e.relu;
+    a.A = e.A;
+    a.bias = e.bias;
+    a.out = e.out;
+    a.mean = e.out_mean;
+    a.value = e.out_value;
+    a.status = status;
+    if (a.mode == EPI_FWD && g.Co % 8 != 0) return PPO_ERR_UNSUPPORTED;
+    a.ncls = 1;
+    KClass &k = a.cls[0];
+    k.o_oy = k.o_ox = 0;
+    k.taps.n = g.taps();
+    for (int t = 0; t < g.taps(); ++t) {
+        k.taps.dy[t] = (signed char)(t / g.k);
+        k.taps.dx[t] = (signed char)(t % g.k);
+        k.taps.wt[t] = (short)t;
+    }
+    return launch_kmajor(a, st);
+}
+
+int tma_gemm_dgrad(const ConvGeom &g, const bf16 *dY, int ldy, const bf16 *Wt, int wt_ld, const DgradEpilogue &e,
+                   int32_t *status, cudaStream_t st) {
+    if (!status || g.Ci % 8 != 0 || ldy % 8 != 0 || wt_ld % 8 != 0 || ldy < wt_ld) return PPO_ERR_UNSUPPORTED;
+    const bool flat = is_flat(g);
+    if (!flat && (g.k < 3 || g.Hi < 2 || g.Wi < 2)) return PPO_ERR_UNSUPPORTED;
+    const int CB = channels_per_box(g.Co, flat);
+    if (CB == 0 || g.taps() > kMaxTaps || wt_ld < g.Co) return PPO_ERR_UNSUPPORTED;
+    KArgs a = {};
+    a.CB = CB;
+    a.row_bytes = CB * 2;
+    a.kchunks = (g.Co + CB - 1) / CB;
+    a.w_tap = wt_ld;
+    // rows: input pixels of one stride-parity class, (Hi+1)/2 x (Wi+1)/2 of them (classes that have fewer
+    // drop the excess in the epilogue)
+    const int Hr = flat ? 1 : (g.Hi + 1) / 2, Wr = flat ? g.B : (g.Wi + 1) / 2;
+    if (!make_grid(a.grid, Wr, Hr, flat ? 1 : g.B, a.row_bytes)) return PPO_ERR_UNSUPPORTED;
+    int s = flat ? make_act_maps(a.mapA, dY, g.Co, ldy, g.B, 1, 1, a.grid, CB, 1)
+                 : make_act_maps(a.mapA, dY, g.Co, ldy, g.Wo, g.Ho, g.B, a.grid, CB, 1);
+    if (s != PPO_OK) return s;
+    a.N = g.Ci;
+    a.BN = pick_bn(g.Ci);
+    {
+        const long long dims[2] = {(long long)g.taps() * wt_ld, g.Ci};
+        const int box[2] = {CB, a.BN}, es[2] = {1, 1};
+        s = make_map(&a.mapB, Wt, 2, dims, (long long)g.taps() * wt_ld, box, es, a.row_bytes);
+        if (s != PPO_OK) return s;
+    }
+    a.s_mul = 1;
+    a.s_oy = a.s_ox = 0;
+    a.o_mul = flat ? 1 : 2;
+    a.Hout = flat ? 1 : g.Hi;
+    a.Wout = flat ? g.B : g.Wi;
+    a.ldo = g.Ci;
+    a.mode = EPI_DGRAD;
+    a.out = e.out;
+    a.out_f32 = e.out_f32;
+    a.mask = e.mask_act;
+    a.status = status;
+    if (flat) {
+        a.ncls = 1;
+        KClass &k = a.cls[0];
+        k.o_oy = k.o_ox = 0;
+        k.taps.n = 1;
+        k.taps.dy[0] = k.taps.dx[0] = 0;
+        k.taps.wt[0] = 0;
+        return launch_kmajor(a, st);
+    }
+    // One class per stride parity (ih % 2, iw % 2): inside a class every input pixel sees the same kernel
+    // taps, kh = (ph + pad) mod 2, +2, ..., each reading output row (ih + pad - kh) / 2 = y + (ph + pad - kh) / 2.
+    a.ncls = 0;
+    for (int ph = 0; ph < 2; ++ph)
+        for (int pw = 0; pw < 2; ++pw) {
+            KClass &k = a.cls[a.ncls++];
+            k.o_oy = ph;
+            k.o_ox = pw;
+            int nt = 0;
+            for (int kh = (ph + g.pad) & 1; kh < g.k; kh += 2)
+                for (int kw = (pw + g.pad) & 1; kw < g.k; kw += 2) {
+                    k.taps.dy[nt] = (signed char)((ph + g.pad - kh) / 2);
+                    k.taps.dx[nt] = (signed char)((pw + g.pad - kw) / 2);
+                    k.taps.wt[nt] = (short)(kh * g.k + kw);
+                    ++nt;
+                }
+            if (nt == 0) return PPO_ERR_UNSUPPORTED;
+            k.taps.n = nt;
+        }
+    return launch_kmajor(a, st);
+}
+
+int tma_gemm_wgrad(const ConvGeom &g, const bf16 *dY, int ldy, const bf16 *X, float *dW, int32_t *status,
+                   cudaStream_t st) {
+    if (!status || g.Ci % 8 != 0 || ldy % 8 != 0 || g.taps() > kMaxTaps) return PPO_ERR_UNSUPPORTED;
+    const bool flat = is_flat(g);
+    const int CB = channels_per_box(g.Ci, flat);
+    const int CBn = g.Co % 64 == 0 ? 64 : (g.Co % 32 == 0 ? 32 : 0);
+    if (CB == 0 || CBn == 0) return PPO_ERR_UNSUPPORTED;
+    WArgs a = {};
+    a.CB = CB;
+    a.rbA = CB * 2;
+    a.mblocks = 128 / CB;
+    a.kchunks = (g.Ci + CB - 1) / CB;
+    a.CBn = CBn;
+    a.rbB = CBn * 2;
+    a.BN = g.Co < 256 ? g.Co : 256;
+    if (g.Co % a.BN != 0 || a.BN % CBn != 0) return PPO_ERR_UNSUPPORTED;
+    a.nblocks = a.BN / CBn;
+    const int rb_min = a.rbA < a.rbB ? a.rbA : a.rbB;
+    const bool ok = flat ? make_grid(a.grid, g.B, 1, 1, rb_min) : make_grid(a.grid, g.Wo, g.Ho, g.B, rb_min);
+    if (!ok) return PPO_ERR_UNSUPPORTED;
+    int s = flat ? make_act_maps(a.mapA, X, g.Ci, g.Ci, g.B, 1, 1, a.grid, CB, 1)
+                 : make_act_maps(a.mapA, X, g.Ci, g.Ci, g.Wi, g.Hi, g.B, a.grid, CB, 2);
+    if (s != PPO_OK) return s;
+    s = flat ? make_act_maps(a.mapB, dY, g.Co, ldy, g.B, 1, 1, a.grid, CBn, 1)
+             : make_act_maps(a.mapB, dY, g.Co, ldy, g.Wo, g.Ho, g.B, a.grid, CBn, 1);
+    if (s != PPO_OK) return s;
+    a.s_mul = flat ? 1 : 2;
+    a.pad = g.pad;
+    a.ksz = g.k;
+    a.ntaps = g.taps();
+    a.Kfwd = g.K();
+    a.Co = g.Co;
+    a.nmma = (a.grid.arows + 15) / 16;
+    a.dW = dW;
+    a.status = status;
+    const size_t stage = (size_t)128 * 256 + (size_t)128 * 2 * a.BN;
+    a.stages = stages_for(stage);
+    if (a.stages < 2) return PPO_ERR_UNSUPPORTED;
+    s = ensure_smem_attrs();
+    if (s != PPO_OK) return s;
+    const int jtiles = (a.ntaps * a.kchunks + a.mblocks - 1) / a.mblocks, ctiles = g.Co / a.BN;
+    int splits = ppo_num_sms() / (jtiles * ctiles);
+    if (splits < 1) splits = 1;
+    if (splits > a.grid.tiles) splits = a.grid.tiles;
+    a.tiles_per_split = (a.grid.tiles + splits - 1) / splits;
+    splits = (a.grid.tiles + a.tiles_per_split - 1) / a.tiles_per_split;
+    dim3 grid((unsigned)jtiles, (unsigned)ctiles, (unsigned)splits);
+    tma_wgrad_kernel<<<grid, kThreads, (size_t)a.stages * stage + sizeof(Pipe) + 1024, st>>>(a);
+    PPO_LAUNCH_CHECK();
+    return PPO_OK;
+}
