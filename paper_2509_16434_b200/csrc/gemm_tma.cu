@@ -67,12 +67,13 @@ struct Pipe {
     uint64_t tempty[2];
     uint32_t tmem_slot;
     int abort_flag;
+    int nboxes;
     Box boxes[kMaxBoxes];
 };
 
 // Boxes of tile `tile`, in shared-memory row order.  Rows past the last image get an image index >= Nimg,
 // which the copy engine answers with zeros.  Called by one thread.
-__device__ int build_boxes(const RowGrid &g, int tile, Box *out) {
+__host__ __device__ inline int build_boxes(const RowGrid &g, int tile, Box *out) {
     if (g.R == 0) {
         const int frow = tile / g.xsegs, xs = tile - frow * g.xsegs;
         const int n = frow / g.Hr;
@@ -84,9 +85,11 @@ __device__ int build_boxes(const RowGrid &g, int tile, Box *out) {
     while (f < fend) {
         const int n = f / g.Hr;
         int y = f - n * g.Hr;
-        int seg = min(g.Hr - y, fend - f);
+        int seg = g.Hr - y < fend - f ? g.Hr - y : fend - f;
         while (seg > 0) {
-            const int hl = 31 - __clz(seg), h = 1 << hl;
+            int hl = 0;
+            while ((2 << hl) <= seg) ++hl;
+            const int h = 1 << hl;
             out[nb++] = {n, y, 0, hl, off};
             y += h;
             f += h;
@@ -98,10 +101,10 @@ __device__ int build_boxes(const RowGrid &g, int tile, Box *out) {
 }
 
 // After a time-out: bounded wait for the copies of the last `S` armed stages (iterations it-S .. it-1).
-__device__ void drain_copies(Pipe *pipe, int it, int S) {
+__device__ void drain_copies(uint64_t *full, int it, int S) {
     for (int i = max(0, it - S); i < it; ++i) {
         const long long t0 = clock64();
-        while (!mbar_try_wait(&pipe->full[i % S], (i / S) & 1))
+        while (!mbar_try_wait(&full[i % S], (i / S) & 1))
             if (clock64() - t0 > kWaitCycles / 4) break;
     }
 }
@@ -115,6 +118,12 @@ struct KClass {
 
 enum { EPI_FWD = 0, EPI_HEAD = 1, EPI_DGRAD = 2 };
 
+constexpr int kEpiWarps = 8;                      // two warps per TMEM lane quarter, alternating 16-column chunks
+constexpr int kKThreads = (2 + kEpiWarps) * 32;   // warp 0: TMA producer, warp 1: MMA issue and TMEM owner
+constexpr int kMaxBias = 512;
+
+// A pipeline stage carries G sub-blocks; sub-block q of a tile is (tap, channel chunk) = divmod(q, kchunks):
+// the A boxes of that tap (128 rows) followed, unless the weights are resident, by its BN weight rows.
 struct KArgs {
     CUtensorMap mapA[kMaxHeights];
     CUtensorMap mapB;
@@ -123,8 +132,9 @@ struct KArgs {
     int CB, row_bytes;      // channels per box (64 or 32) and bytes of a shared-memory row
     int kchunks;            // boxes along the channels of one tap
     int w_tap;              // elements between taps in a weight row
+    int G, nbmax;           // sub-blocks per stage; most A boxes a tile has
+    int wres, wtaps;        // weights resident in shared memory (all wtaps * kchunks boxes, loaded once)
     int N, BN, tiles_n, tiles_per_cls, total_tiles, ncls, stages;
-    uint32_t tx_bytes;      // bytes one K block brings in
     int o_mul, Hout, Wout, ldo;
     int mode, relu, A;
     const float *bias;
@@ -136,14 +146,29 @@ struct KArgs {
     KClass cls[4];
 };
 
-__global__ void __launch_bounds__(kThreads, 1) tma_kmajor_kernel(const __grid_constant__ KArgs a) {
+struct PipeK {
+    uint64_t full[kMaxStages];
+    uint64_t empty[kMaxStages];
+    uint64_t tfull[2];
+    uint64_t tempty[2];
+    uint64_t wfull;
+    uint32_t tmem_slot;
+    int abort_flag;
+    int nboxes;
+    Box boxes[kMaxBoxes];
+    alignas(16) float bias[kMaxBias];
+};
+
+__global__ void __launch_bounds__(kKThreads, 1) tma_kmajor_kernel(const __grid_constant__ KArgs a) {
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    const int BN = a.BN, S = a.stages;
+    const int BN = a.BN, S = a.stages, G = a.G;
     const uint32_t rb = (uint32_t)a.row_bytes;
-    const uint32_t a_bytes = 128u * rb;
-    const uint32_t stage_bytes = a_bytes + (uint32_t)BN * rb;
-    Pipe *pipe = reinterpret_cast<Pipe *>(smem + (size_t)S * stage_bytes);
+    const uint32_t a_bytes = 128u * rb, b_bytes = (uint32_t)BN * rb;
+    const uint32_t sub_bytes = a_bytes + (a.wres ? 0u : b_bytes);
+    const uint32_t stage_bytes = (uint32_t)G * sub_bytes;
+    const uint32_t res_bytes = a.wres ? (uint32_t)(a.wtaps * a.kchunks) * b_bytes : 0u;
+    PipeK *pipe = reinterpret_cast<PipeK *>(smem + (size_t)S * stage_bytes + res_bytes);
     volatile int *abort_flag = &pipe->abort_flag;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t acc_cols = tmem_cols_for(BN);
@@ -156,48 +181,76 @@ __global__ void __launch_bounds__(kThreads, 1) tma_kmajor_kernel(const __grid_co
         }
         for (int i = 0; i < 2; ++i) {
             mbar_init(&pipe->tfull[i], 1);
-            mbar_init(&pipe->tempty[i], 128);
+            mbar_init(&pipe->tempty[i], kEpiWarps * 32);
         }
+        mbar_init(&pipe->wfull, 1);
         pipe->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
+    if (a.mode != EPI_DGRAD)
+        for (int i = threadIdx.x; i < a.tiles_n * BN; i += kKThreads) pipe->bias[i] = i < a.N ? a.bias[i] : 0.f;
     if (warp == 1) tmem_alloc(&pipe->tmem_slot, ncols);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = pipe->tmem_slot;
     const uint32_t smem_base = smem_u32(smem);
+    const uint32_t res_base = smem_base + (uint32_t)S * stage_bytes;
 
     if (warp == 0) {
-        // ---------------- TMA producer
-        if (lane == 0) {
-            int it = 0;
-            bool ok = true;
-            for (int g = blockIdx.x; g < a.total_tiles && ok; g += gridDim.x) {
-                const int c = g / a.tiles_per_cls, local = g - c * a.tiles_per_cls;
-                const int mt = local / a.tiles_n, n0 = (local - mt * a.tiles_n) * BN;
-                const KClass &k = a.cls[c];
-                const int nb = build_boxes(a.grid, mt, pipe->boxes);
-                for (int t = 0; t < k.taps.n && ok; ++t) {
-                    const int dy = a.s_oy + k.taps.dy[t], dx = a.s_ox + k.taps.dx[t];
-                    const int wcol = (int)k.taps.wt[t] * a.w_tap;
-                    for (int kc = 0; kc < a.kchunks; ++kc, ++it) {
-                        const int s = it % S;
-                        ok = mbar_wait(&pipe->empty[s], ((it / S) & 1) ^ 1, abort_flag, a.status);
-                        if (!ok) break;
-                        mbar_arrive_expect_tx(&pipe->full[s], a.tx_bytes);
-                        const uint32_t sa = smem_base + (uint32_t)s * stage_bytes;
-                        for (int b = 0; b < nb; ++b) {
-                            const Box bx = pipe->boxes[b];
+        // ---------------- TMA producer: the lanes share out the copies of a stage, one thread each
+        if (a.wres) {
+            const int nw = a.wtaps * a.kchunks;
+            if (lane == 0) mbar_arrive_expect_tx(&pipe->wfull, (uint32_t)nw * b_bytes);
+            __syncwarp();
+            for (int q = lane; q < nw; q += 32) {
+                const int tap = q / a.kchunks, kc = q - tap * a.kchunks;
+                tma_load_2d(res_base + (uint32_t)q * b_bytes, &a.mapB, &pipe->wfull, tap * a.w_tap + kc * a.CB, 0);
+            }
+        }
+        const int lps = a.nbmax + (a.wres ? 0 : 1);  // copies per sub-block: its A boxes, then its weight rows
+        const int units = G * lps;
+        int it = 0;
+        bool ok = true;
+        for (int g = blockIdx.x; g < a.total_tiles && ok; g += gridDim.x) {
+            const int c = g / a.tiles_per_cls, local = g - c * a.tiles_per_cls;
+            const int mt = local / a.tiles_n, n0 = (local - mt * a.tiles_n) * BN;
+            const KClass &k = a.cls[c];
+            if (lane == 0) pipe->nboxes = build_boxes(a.grid, mt, pipe->boxes);
+            __syncwarp();
+            const int nb = pipe->nboxes;
+            const int nsub = k.taps.n * a.kchunks;
+            for (int q0 = 0; q0 < nsub; q0 += G, ++it) {
+                const int s = it % S;
+                int okw = 1;
+                if (lane == 0) okw = mbar_wait(&pipe->empty[s], ((it / S) & 1) ^ 1, abort_flag, a.status) ? 1 : 0;
+                ok = __shfl_sync(0xffffffffu, okw, 0) != 0;
+                if (!ok) break;
+                const int nval = min(G, nsub - q0);
+                if (lane == 0) mbar_arrive_expect_tx(&pipe->full[s], (uint32_t)nval * (a.grid.arows * rb + (a.wres ? 0u : b_bytes)));
+                __syncwarp();
+                const uint32_t st = smem_base + (uint32_t)s * stage_bytes;
+                for (int u = lane; u < units; u += 32) {
+                    const int gi = u / lps, j = u - gi * lps;
+                    if (gi >= nval) continue;
+                    const int q = q0 + gi, tap = q / a.kchunks, kc = q - tap * a.kchunks;
+                    const uint32_t sa = st + (uint32_t)gi * sub_bytes;
+                    if (j < a.nbmax) {
+                        if (j < nb) {
+                            const Box bx = pipe->boxes[j];
                             tma_load_4d(sa + (uint32_t)bx.rowoff * rb, &a.mapA[bx.hl], &pipe->full[s], kc * a.CB,
-                                        bx.x * a.s_mul + dx, bx.y * a.s_mul + dy, bx.n);
+                                        bx.x * a.s_mul + a.s_ox + k.taps.dx[tap], bx.y * a.s_mul + a.s_oy + k.taps.dy[tap],
+                                        bx.n);
                         }
-                        tma_load_2d(sa + a_bytes, &a.mapB, &pipe->full[s], wcol + kc * a.CB, n0);
+                    } else {
+                        tma_load_2d(sa + a_bytes, &a.mapB, &pipe->full[s], (int)k.taps.wt[tap] * a.w_tap + kc * a.CB, n0);
                     }
                 }
+                __syncwarp();
             }
-            if (!ok) drain_copies(pipe, it, S);
+            __syncwarp();
         }
+        if (!ok && lane == 0) drain_copies(pipe->full, it, S);
         __syncwarp();
     } else if (warp == 1) {
         // ---------------- MMA issue: one thread feeds the tensor core
@@ -206,24 +259,35 @@ __global__ void __launch_bounds__(kThreads, 1) tma_kmajor_kernel(const __grid_co
         const uint32_t sbo = 8u * rb;
         int it = 0, ti = 0;
         bool ok = true;
+        if (a.wres) ok = mbar_wait(&pipe->wfull, 0, abort_flag, a.status);
         for (int g = blockIdx.x; g < a.total_tiles && ok; g += gridDim.x, ++ti) {
             const int c = g / a.tiles_per_cls;
-            const int nkb = a.cls[c].taps.n * a.kchunks;
+            const KClass &k = a.cls[c];
+            const int nsub = k.taps.n * a.kchunks;
             const int acc = ti & 1;
             ok = mbar_wait(&pipe->tempty[acc], ((ti >> 1) & 1) ^ 1, abort_flag, a.status);
             if (!ok) break;
             tc_fence_after();
             const uint32_t tmem_d = tmem_base + acc * acc_cols;
-            for (int kb = 0; kb < nkb; ++kb, ++it) {
+            for (int q0 = 0; q0 < nsub; q0 += G, ++it) {
                 const int s = it % S;
                 ok = mbar_wait(&pipe->full[s], (it / S) & 1, abort_flag, a.status);
                 if (!ok) break;
                 tc_fence_after();
                 if (lane == 0) {
-                    const uint32_t sa = smem_base + (uint32_t)s * stage_bytes, sb = sa + a_bytes;
-                    for (int kk = 0; kk < nk; ++kk)  // K = 16 elements = 32 bytes along the swizzled row
-                        umma_bf16(tmem_d, smem_desc_sw(sa + kk * 32, 16, sbo, rb), smem_desc_sw(sb + kk * 32, 16, sbo, rb),
-                                  idesc, (kb > 0 || kk > 0) ? 1u : 0u);
+                    const int nval = min(G, nsub - q0);
+                    for (int gi = 0; gi < nval; ++gi) {
+                        const uint32_t sa = smem_base + (uint32_t)s * stage_bytes + (uint32_t)gi * sub_bytes;
+                        uint32_t sb = sa + a_bytes;
+                        if (a.wres) {
+                            const int q = q0 + gi, tap = q / a.kchunks, kc = q - tap * a.kchunks;
+                            sb = res_base + (uint32_t)((int)k.taps.wt[tap] * a.kchunks + kc) * b_bytes;
+                        }
+                        for (int kk = 0; kk < nk; ++kk)  // K = 16 elements = 32 bytes along the swizzled row
+                            umma_bf16(tmem_d, smem_desc_sw(sa + kk * 32, 16, sbo, rb),
+                                      smem_desc_sw(sb + kk * 32, 16, sbo, rb), idesc,
+                                      (q0 > 0 || gi > 0 || kk > 0) ? 1u : 0u);
+                    }
                     umma_commit(&pipe->empty[s]);
                 }
                 __syncwarp();
@@ -232,8 +296,9 @@ __global__ void __launch_bounds__(kThreads, 1) tma_kmajor_kernel(const __grid_co
             __syncwarp();
         }
     } else {
-        // ---------------- epilogue: warp w reads TMEM lanes 32 (w % 4) .. +31
-        const int lg = warp & 3;
+        // ---------------- epilogue: warp w reads TMEM lanes 32 (w % 4) .. +31; the two warps of a lane
+        // quarter take alternate 16-column chunks
+        const int lg = warp & 3, half = (warp - 2) >> 2;
         const int p = lg * 32 + lane;
         const RowGrid &gr = a.grid;
         int ti = 0;
@@ -267,7 +332,7 @@ __global__ void __launch_bounds__(kThreads, 1) tma_kmajor_kernel(const __grid_co
             if (!ok) break;
             tc_fence_after();
             const uint32_t lane_base = tmem_base + acc * acc_cols + ((uint32_t)(lg * 32) << 16);
-            for (int c0 = 0; c0 < BN; c0 += 16) {
+            for (int c0 = half * 16; c0 < BN; c0 += 32) {
                 if (n0 + c0 >= a.N) break;  // uniform across the warp
                 float v[16];
                 tmem_ld16(lane_base + (uint32_t)c0, v);
@@ -276,17 +341,21 @@ __global__ void __launch_bounds__(kThreads, 1) tma_kmajor_kernel(const __grid_co
                 if (a.mode == EPI_HEAD) {
 #pragma unroll
                     for (int i = 0; i < 16; ++i) {
-                        if (nn + i < a.A) a.mean[orow * a.A + nn + i] = v[i] + a.bias[nn + i];
-                        else if (nn + i == a.A) a.value[orow] = v[i] + a.bias[nn + i];
+                        if (nn + i < a.A) a.mean[orow * a.A + nn + i] = v[i] + pipe->bias[nn + i];
+                        else if (nn + i == a.A) a.value[orow] = v[i] + pipe->bias[nn + i];
                     }
                     continue;
                 }
                 if (a.mode == EPI_FWD) {
+                    const float4 *bp = reinterpret_cast<const float4 *>(pipe->bias + nn);
 #pragma unroll
-                    for (int i = 0; i < 16; ++i) {
-                        const float bv = (nn + i < a.N) ? a.bias[nn + i] : 0.f;
-                        v[i] += bv;
-                        if (a.relu) v[i] = fmaxf(v[i], 0.f);
+                    for (int q = 0; q < 4; ++q) {
+                        const float4 bv = bp[q];
+                        v[4 * q] += bv.x; v[4 * q + 1] += bv.y; v[4 * q + 2] += bv.z; v[4 * q + 3] += bv.w;
+                    }
+                    if (a.relu) {
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) v[i] = fmaxf(v[i], 0.f);
                     }
                 } else if (a.mask) {
                     const uint4 *mp = reinterpret_cast<const uint4 *>(a.mask + orow * a.ldo + nn);
@@ -397,33 +466,41 @@ __global__ void __launch_bounds__(kThreads, 1) tma_wgrad_kernel(const __grid_con
     const uint32_t tx_bytes = (uint32_t)a.grid.arows * ((uint32_t)nvalid * rbA + (uint32_t)a.nblocks * rbB);
 
     if (warp == 0) {
-        if (lane == 0) {
-            bool ok = true;
-            int kb = 0;
-            for (; kb < nkb; ++kb) {
-                const int s = kb % S;
-                ok = mbar_wait(&pipe->empty[s], ((kb / S) & 1) ^ 1, abort_flag, a.status);
-                if (!ok) break;
+        // ---------------- TMA producer: the lanes share out the copies of a K block, one thread each
+        const int per_box = nvalid + a.nblocks;
+        bool ok = true;
+        int kb = 0;
+        for (; kb < nkb; ++kb) {
+            const int s = kb % S;
+            int okw = 1;
+            if (lane == 0) okw = mbar_wait(&pipe->empty[s], ((kb / S) & 1) ^ 1, abort_flag, a.status) ? 1 : 0;
+            ok = __shfl_sync(0xffffffffu, okw, 0) != 0;
+            if (!ok) break;
+            if (lane == 0) {
                 mbar_arrive_expect_tx(&pipe->full[s], tx_bytes);
-                const uint32_t sa = smem_base + (uint32_t)s * stage_bytes, sb = sa + a_bytes;
-                const int nb = build_boxes(a.grid, t_lo + kb, pipe->boxes);
-                for (int b = 0; b < nb; ++b) {
-                    const Box bx = pipe->boxes[b];
-                    for (int i = 0; i < a.mblocks; ++i) {
-                        const int jb = jb0 + i, tap = jb / a.kchunks, kc = jb - tap * a.kchunks;
-                        if (tap >= a.ntaps) break;
-                        const int kh = tap / a.ksz, kw = tap - kh * a.ksz;
-                        tma_load_4d(sa + (uint32_t)i * 128u * rbA + (uint32_t)bx.rowoff * rbA, &a.mapA[bx.hl],
-                                    &pipe->full[s], kc * a.CB, bx.x * a.s_mul - a.pad + kw, bx.y * a.s_mul - a.pad + kh,
-                                    bx.n);
-                    }
-                    for (int i = 0; i < a.nblocks; ++i)
-                        tma_load_4d(sb + (uint32_t)i * 128u * rbB + (uint32_t)bx.rowoff * rbB, &a.mapB[bx.hl],
-                                    &pipe->full[s], co0 + i * a.CBn, bx.x, bx.y, bx.n);
+                pipe->nboxes = build_boxes(a.grid, t_lo + kb, pipe->boxes);
+            }
+            __syncwarp();
+            const uint32_t sa = smem_base + (uint32_t)s * stage_bytes, sb = sa + a_bytes;
+            const int units = pipe->nboxes * per_box;
+            for (int u = lane; u < units; u += 32) {
+                const int b = u / per_box, i = u - b * per_box;
+                const Box bx = pipe->boxes[b];
+                if (i < nvalid) {
+                    const int jb = jb0 + i, tap = jb / a.kchunks, kc = jb - tap * a.kchunks;
+                    const int kh = tap / a.ksz, kw = tap - kh * a.ksz;
+                    tma_load_4d(sa + (uint32_t)i * 128u * rbA + (uint32_t)bx.rowoff * rbA, &a.mapA[bx.hl],
+                                &pipe->full[s], kc * a.CB, bx.x * a.s_mul - a.pad + kw, bx.y * a.s_mul - a.pad + kh,
+                                bx.n);
+                } else {
+                    const int ib = i - nvalid;
+                    tma_load_4d(sb + (uint32_t)ib * 128u * rbB + (uint32_t)bx.rowoff * rbB, &a.mapB[bx.hl],
+                                &pipe->full[s], co0 + ib * a.CBn, bx.x, bx.y, bx.n);
                 }
             }
-            if (!ok) drain_copies(pipe, kb, S);
+            __syncwarp();
         }
+        if (!ok && lane == 0) drain_copies(pipe->full, kb, S);
         __syncwarp();
     } else if (warp == 1) {
         const uint32_t idesc = instr_desc(128, BN, 1, 1);
@@ -591,7 +668,7 @@ int ensure_smem_attrs() {
     PPO_CUDA_CHECK(cudaGetDevice(&dev));
     if (dev < 0 || dev >= 64) return PPO_ERR_CUDA;
     if (!attr_set[dev]) {
-        const int mx = (int)(kSmemBudget + sizeof(Pipe) + 1024);
+        const int mx = (int)(kSmemBudget + sizeof(PipeK) + 1024);
         PPO_CUDA_CHECK(cudaFuncSetAttribute(tma_kmajor_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, mx));
         PPO_CUDA_CHECK(cudaFuncSetAttribute(tma_wgrad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, mx));
         attr_set[dev] = true;
@@ -599,23 +676,49 @@ int ensure_smem_attrs() {
     return PPO_OK;
 }
 
+// Most A boxes any tile of the grid is cut into (the cut repeats with the tile's first row modulo Hr).
+int max_boxes(const RowGrid &g) {
+    if (g.R == 0) return 1;
+    Box tmp[kMaxBoxes];
+    int mx = 1;
+    const int lim = g.tiles < g.Hr + 1 ? g.tiles : g.Hr + 1;
+    for (int t = 0; t < lim; ++t) {
+        const int n = build_boxes(g, t, tmp);
+        mx = n > mx ? n : mx;
+    }
+    const int n = build_boxes(g, g.tiles - 1, tmp);
+    return n > mx ? n : mx;
+}
+
+// `a.wtaps` = taps of the whole weight tensor (all classes).
 int launch_kmajor(KArgs &a, cudaStream_t st) {
     int s = ensure_smem_attrs();
     if (s != PPO_OK) return s;
     a.tiles_n = (a.N + a.BN - 1) / a.BN;
+    if (a.tiles_n * a.BN > kMaxBias) return PPO_ERR_UNSUPPORTED;
     const long long per = (long long)a.grid.tiles * a.tiles_n;
     const long long total = per * a.ncls;
     if (total <= 0) return PPO_OK;
     if (total > 0x7fffffffll) return PPO_ERR_UNSUPPORTED;
     a.tiles_per_cls = (int)per;
     a.total_tiles = (int)total;
-    const size_t stage = (size_t)(128 + a.BN) * a.row_bytes;
-    a.stages = stages_for(stage);
+    a.nbmax = max_boxes(a.grid);
+    const size_t b_bytes = (size_t)a.BN * a.row_bytes;
+    const size_t res = (size_t)a.wtaps * a.kchunks * b_bytes;
+    a.wres = (a.tiles_n == 1 && res <= 64 * 1024) ? 1 : 0;
+    const size_t sub = (size_t)128 * a.row_bytes + (a.wres ? 0 : b_bytes);
+    const size_t budget = kSmemBudget - (a.wres ? res : 0);
+    int G = (int)((40 * 1024) / sub);
+    G = G < 1 ? 1 : (G > 4 ? 4 : G);
+    while (G > 1 && budget / (G * sub) < 3) --G;
+    a.G = G;
+    a.stages = (int)(budget / (G * sub));
+    if (a.stages > kMaxStages) a.stages = kMaxStages;
     if (a.stages < 2) return PPO_ERR_UNSUPPORTED;
-    a.tx_bytes = (uint32_t)((a.grid.arows + a.BN) * a.row_bytes);
     const int sms = ppo_num_sms();
     const unsigned grid = (unsigned)(total < sms ? total : sms);
-    tma_kmajor_kernel<<<grid, kThreads, (size_t)a.stages * stage + sizeof(Pipe) + 1024, st>>>(a);
+    const size_t smem = (size_t)a.stages * G * sub + (a.wres ? res : 0) + sizeof(PipeK) + 1024;
+    tma_kmajor_kernel<<<grid, kKThreads, smem, st>>>(a);
     PPO_LAUNCH_CHECK();
     return PPO_OK;
 }
@@ -635,6 +738,7 @@ int tma_gemm_fwd(const ConvGeom &g, const bf16 *X, const bf16 *W, const FwdEpilo
     a.row_bytes = CB * 2;
     a.kchunks = (g.Ci + CB - 1) / CB;
     a.w_tap = g.Ci;
+    a.wtaps = g.taps();
     // a fully connected layer is one image with a single row of B pixels
     const bool ok = flat ? make_grid(a.grid, g.B, 1, 1, a.row_bytes) : make_grid(a.grid, g.Wo, g.Ho, g.B, a.row_bytes);
     if (!ok) return PPO_ERR_UNSUPPORTED;
@@ -688,6 +792,7 @@ int tma_gemm_dgrad(const ConvGeom &g, const bf16 *dY, int ldy, const bf16 *Wt, i
     a.row_bytes = CB * 2;
     a.kchunks = (g.Co + CB - 1) / CB;
     a.w_tap = wt_ld;
+    a.wtaps = g.taps();
     // rows: input pixels of one stride-parity class, (Hi+1)/2 x (Wi+1)/2 of them (classes that have fewer
     // drop the excess in the epilogue)
     const int Hr = flat ? 1 : (g.Hi + 1) / 2, Wr = flat ? g.B : (g.Wi + 1) / 2;
