@@ -8,12 +8,15 @@
 // First layer (C_in = 1): too shallow a reduction (k*k) for a tensor-core tile, and bound by
 // HBM (reads one fp16 frame, writes C1 bf16 maps).  One thread per output pixel; the k*k
 // patch sits in registers, the weights (as the bf16 shadow rounds them) in shared memory.
-template <int KS>
+// With STAGE the 16-byte chunks of a warp's 32 pixels pass through a swizzled shared-memory
+// buffer so that every store instruction of the warp writes 512 contiguous bytes (C1 / 8 a
+// power of two); without it each thread stores its own pixel.
+template <int KS, bool STAGE>
 __global__ void __launch_bounds__(128) conv1_fwd_kernel(const __half *__restrict__ depth,
                                                         const bf16 *__restrict__ W, const float *__restrict__ bias,
                                                         bf16 *__restrict__ out, int rows, int Hi, int Wi, int Ho,
                                                         int Wo, int C1) {
-    extern __shared__ float sm[];  // w[tap][co], then bias[co]
+    extern __shared__ float sm[];  // w[tap][co], then bias[co], then (STAGE) 4 warps x 32 pixels x C1 bf16
     float *w = sm, *bs = sm + KS * KS * C1;
     for (int i = threadIdx.x; i < KS * KS * C1; i += blockDim.x) {
         const int co = i % C1, tap = i / C1;
@@ -23,21 +26,29 @@ __global__ void __launch_bounds__(128) conv1_fwd_kernel(const __half *__restrict
     __syncthreads();
     const long long m = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     const long long M = (long long)rows * Ho * Wo;
-    if (m >= M) return;
-    const int ow = (int)(m % Wo);
-    const long long t = m / Wo;
-    const int oh = (int)(t % Ho);
-    const long long b = t / Ho;
-    const __half *img = depth + b * Hi * Wi;
+    const bool live = m < M;
     constexpr int P = KS / 2;
     float x[KS * KS];
+    if (live) {
+        const int ow = (int)(m % Wo);
+        const long long t = m / Wo;
+        const int oh = (int)(t % Ho);
+        const __half *img = depth + (t / Ho) * Hi * Wi;
 #pragma unroll
-    for (int kh = 0; kh < KS; ++kh)
+        for (int kh = 0; kh < KS; ++kh)
 #pragma unroll
-        for (int kw = 0; kw < KS; ++kw) {
-            const int ih = 2 * oh + kh - P, iw = 2 * ow + kw - P;
-            x[kh * KS + kw] = (ih >= 0 && ih < Hi && iw >= 0 && iw < Wi) ? __half2float(img[ih * Wi + iw]) : 0.f;
-        }
+            for (int kw = 0; kw < KS; ++kw) {
+                const int ih = 2 * oh + kh - P, iw = 2 * ow + kw - P;
+                x[kh * KS + kw] = (ih >= 0 && ih < Hi && iw >= 0 && iw < Wi) ? __half2float(img[ih * Wi + iw]) : 0.f;
+            }
+    } else {
+#pragma unroll
+        for (int i = 0; i < KS * KS; ++i) x[i] = 0.f;
+    }
+    const int CH = C1 >> 3;  // 16-byte chunks per pixel
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    uint4 *stage = reinterpret_cast<uint4 *>(bs + C1) + (size_t)warp * 32 * CH;
+    const int sh = CH == 8 ? 0 : (CH == 4 ? 1 : (CH == 2 ? 2 : 3));
     uint4 *o = reinterpret_cast<uint4 *>(out + m * C1);
     for (int c8 = 0; c8 < C1; c8 += 8) {
         float acc[8];
@@ -50,92 +61,97 @@ __global__ void __launch_bounds__(128) conv1_fwd_kernel(const __half *__restrict
         __nv_bfloat162 p[4];
 #pragma unroll
         for (int j = 0; j < 4; ++j) p[j] = __floats2bfloat162_rn(fmaxf(acc[2 * j], 0.f), fmaxf(acc[2 * j + 1], 0.f));
-        o[c8 / 8] = *reinterpret_cast<uint4 *>(p);
+        if (STAGE) stage[lane * CH + ((c8 >> 3) ^ ((lane >> sh) & (CH - 1)))] = *reinterpret_cast<uint4 *>(p);
+        else if (live) o[c8 >> 3] = *reinterpret_cast<uint4 *>(p);
+    }
+    if (STAGE) {
+        __syncwarp();
+        const long long mw = m - lane;  // first pixel of this warp
+        for (int i = lane; i < 32 * CH; i += 32) {
+            const int px = i / CH, phys = i - px * CH;
+            const int chunk = phys ^ ((px >> sh) & (CH - 1));
+            if (mw + px < M) reinterpret_cast<uint4 *>(out + (mw + px) * C1)[chunk] = stage[i];
+        }
     }
 }
 
 // dW1[co][tap] += sum_m dZ1[m][co] * x(m, tap);  db1[co] += sum_m dZ1[m][co].
-// Register tiling: C1 / CPT threads share one output pixel, each owning CPT channels and all k*k
-// taps (CPT * k*k accumulators); the pixel's gradient row is read once, coalesced, straight from
-// global memory and its input patch through L1.  Partial sums are folded across the pixel groups
-// of a warp by shuffles, across warps through shared memory, then added with one atomic each.
-template <int KS, int CPT>
+// A lane owns one pair of channels; C1 / 2 lanes share a pixel and a warp walks 64 / C1 pixels per
+// step through a contiguous range of output pixels, so that the gradient rows are read once with
+// coalesced 4-byte loads while the k*k input taps of a pixel are one broadcast load each.  Every lane
+// keeps 2 (k*k + 1) accumulators (the last one is the bias gradient); they are folded across the
+// pixel slots of a warp by shuffles, across warps through shared memory, then added with one atomic
+// each.  C1 / 2 must be a power of two <= 32.
+template <int KS>
 __global__ void __launch_bounds__(256) conv1_wgrad_kernel(const __half *__restrict__ depth,
                                                           const bf16 *__restrict__ dZ, float *__restrict__ dW,
                                                           float *__restrict__ db, int rows, int Hi, int Wi, int Ho,
-                                                          int Wo, int C1) {
+                                                          int Wo, int C1, long long px_per_warp) {
     constexpr int K2 = KS * KS, P = KS / 2;
     extern __shared__ float sm[];  // [8 warps][C1 * (K2 + 1)]
-    const int tpp = C1 / CPT;                  // threads per pixel (a power of two <= 32)
-    const int cq = threadIdx.x % tpp;          // channel group
-    const int pg = threadIdx.x / tpp;          // pixel group inside the block
-    const int groups = 256 / tpp;
-    float acc[CPT][K2 + 1];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int lpp = C1 >> 1;       // lanes per pixel
+    const int ppi = 32 / lpp;      // pixels per step
+    const int cp = lane % lpp, ps = lane / lpp;
+    float acc0[K2 + 1], acc1[K2 + 1];
 #pragma unroll
-    for (int c = 0; c < CPT; ++c)
-#pragma unroll
-        for (int t = 0; t <= K2; ++t) acc[c][t] = 0.f;
+    for (int t = 0; t <= K2; ++t) acc0[t] = acc1[t] = 0.f;
     const long long M = (long long)rows * Ho * Wo;
-    for (long long m = (long long)blockIdx.x * groups + pg; m < M; m += (long long)gridDim.x * groups) {
-        float dz[CPT];
-        if (CPT == 4) {
-            const uint2 raw = *reinterpret_cast<const uint2 *>(dZ + m * C1 + cq * 4);
-            const float2 lo = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&raw.x));
-            const float2 hi = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&raw.y));
-            dz[0] = lo.x; dz[1 % CPT] = lo.y; dz[2 % CPT] = hi.x; dz[3 % CPT] = hi.y;
-        } else if (CPT == 2) {
-            const float2 v = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(dZ + m * C1 + cq * 2));
-            dz[0] = v.x; dz[1 % CPT] = v.y;
-        } else {
-            dz[0] = bf2f(dZ[m * C1 + cq]);
-        }
-        bool any = false;
+    const long long gw = (long long)blockIdx.x * 8 + warp;
+    long long m = gw * px_per_warp + ps;
+    const long long m_end = min(M, (gw + 1) * px_per_warp);
+    if (m < m_end) {
+        int ow = (int)(m % Wo);
+        long long t = m / Wo;
+        int oh = (int)(t % Ho);
+        long long b = t / Ho;
+        for (; m < m_end; m += ppi) {
+            const float2 dz = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(dZ + m * C1 + 2 * cp));
+            const __half *img = depth + b * Hi * Wi;
 #pragma unroll
-        for (int c = 0; c < CPT; ++c) any |= dz[c] != 0.f;
-        if (!any) continue;  // ReLU-masked gradient rows are frequent
-        const int ow = (int)(m % Wo);
-        const long long t = m / Wo;
-        const int oh = (int)(t % Ho);
-        const long long b = t / Ho;
-        const __half *img = depth + b * Hi * Wi;
+            for (int kh = 0; kh < KS; ++kh) {
+                const int ih = 2 * oh + kh - P;
 #pragma unroll
-        for (int kh = 0; kh < KS; ++kh) {
-            const int ih = 2 * oh + kh - P;
-            if (ih < 0 || ih >= Hi) continue;
-#pragma unroll
-            for (int kw = 0; kw < KS; ++kw) {
-                const int iw = 2 * ow + kw - P;
-                if (iw < 0 || iw >= Wi) continue;
-                const float xv = __half2float(img[ih * Wi + iw]);
-#pragma unroll
-                for (int c = 0; c < CPT; ++c) acc[c][kh * KS + kw] = fmaf(dz[c], xv, acc[c][kh * KS + kw]);
+                for (int kw = 0; kw < KS; ++kw) {
+                    const int iw = 2 * ow + kw - P;
+                    const float xv =
+                        (ih >= 0 && ih < Hi && iw >= 0 && iw < Wi) ? __half2float(__ldg(img + ih * Wi + iw)) : 0.f;
+                    acc0[kh * KS + kw] = fmaf(dz.x, xv, acc0[kh * KS + kw]);
+                    acc1[kh * KS + kw] = fmaf(dz.y, xv, acc1[kh * KS + kw]);
+                }
+            }
+            acc0[K2] += dz.x;
+            acc1[K2] += dz.y;
+            ow += ppi;
+            while (ow >= Wo) {
+                ow -= Wo;
+                if (++oh == Ho) { oh = 0; ++b; }
             }
         }
-#pragma unroll
-        for (int c = 0; c < CPT; ++c) acc[c][K2] += dz[c];
     }
-    // fold the pixel groups that live in one warp (lanes that differ in bits >= log2(tpp))
+    // fold the pixel slots of the warp (lanes that differ in bits >= log2(lpp))
 #pragma unroll
-    for (int c = 0; c < CPT; ++c)
+    for (int t = 0; t <= K2; ++t) {
+        float v0 = acc0[t], v1 = acc1[t];
+        for (int o = lpp; o < 32; o <<= 1) {
+            v0 += __shfl_xor_sync(0xffffffffu, v0, o);
+            v1 += __shfl_xor_sync(0xffffffffu, v1, o);
+        }
+        acc0[t] = v0;
+        acc1[t] = v1;
+    }
+    const int per = C1 * (K2 + 1);
+    if (lane < lpp) {
 #pragma unroll
         for (int t = 0; t <= K2; ++t) {
-            float v = acc[c][t];
-            for (int o = tpp; o < 32; o <<= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-            acc[c][t] = v;
+            sm[warp * per + (2 * cp) * (K2 + 1) + t] = acc0[t];
+            sm[warp * per + (2 * cp + 1) * (K2 + 1) + t] = acc1[t];
         }
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int per = C1 * (K2 + 1);
-    if (lane < tpp) {
-#pragma unroll
-        for (int c = 0; c < CPT; ++c)
-#pragma unroll
-            for (int t = 0; t <= K2; ++t) sm[warp * per + (cq * CPT + c) * (K2 + 1) + t] = acc[c][t];
     }
     __syncthreads();
-    const int nw = 8;  // every warp holds a full set of channel groups (tpp <= 32)
     for (int i = threadIdx.x; i < per; i += 256) {
         float v = 0.f;
-        for (int w = 0; w < nw; ++w) v += sm[w * per + i];
+        for (int w = 0; w < 8; ++w) v += sm[w * per + i];
         const int co = i / (K2 + 1), t = i % (K2 + 1);
         if (t < K2) atomicAdd(dW + co * K2 + t, v);
         else atomicAdd(db + co, v);
@@ -378,12 +394,21 @@ extern "C" int ppo_encoder_fwd(ppo_model *m, const ppo_minibatch *mb, int row0, 
         const __half *depth = static_cast<const __half *>(mb->depth_f16) + (size_t)row0 * d.H * d.W;
         const int C1 = m->Cs[1], KS = d.conv_k[0];
         const long long M = (long long)rows * m->Hs[1] * m->Ws[1];
-        const size_t smem = (size_t)(KS * KS * C1 + C1) * sizeof(float);
+        const int CH = C1 / 8;
+        const bool stage = CH == 1 || CH == 2 || CH == 4 || CH == 8;
+        const size_t smem = (size_t)(KS * KS * C1 + C1) * sizeof(float) + (stage ? (size_t)4 * 32 * C1 * 2 : 0);
         const bf16 *W = m->shadow + m->tensors[0].off;
         const float *bias = m->master + m->tensors[1].off;
         const int blocks = ppo_cdiv(M, 128);
-#define PPO_CONV1(KS_)                                                                                            \
-    conv1_fwd_kernel<KS_><<<blocks, 128, smem, st>>>(depth, W, bias, m->act[1], rows, d.H, d.W, m->Hs[1], m->Ws[1], C1)
+#define PPO_CONV1(KS_)                                                                                              \
+    do {                                                                                                            \
+        if (stage)                                                                                                  \
+            conv1_fwd_kernel<KS_, true><<<blocks, 128, smem, st>>>(depth, W, bias, m->act[1], rows, d.H, d.W,       \
+                                                                   m->Hs[1], m->Ws[1], C1);                         \
+        else                                                                                                        \
+            conv1_fwd_kernel<KS_, false><<<blocks, 128, smem, st>>>(depth, W, bias, m->act[1], rows, d.H, d.W,      \
+                                                                    m->Hs[1], m->Ws[1], C1);                        \
+    } while (0)
         if (KS == 1) PPO_CONV1(1);
         else if (KS == 3) PPO_CONV1(3);
         else if (KS == 5) PPO_CONV1(5);
@@ -488,27 +513,29 @@ extern "C" int ppo_encoder_bwd(ppo_model *m, const ppo_minibatch *mb, int row0, 
         const __half *depth = static_cast<const __half *>(mb->depth_f16) + (size_t)row0 * d.H * d.W;
         const int C1 = m->Cs[1], KS = d.conv_k[0];
         const long long M = (long long)rows * m->Hs[1] * m->Ws[1];
-        const int cpt = KS <= 3 ? 4 : (KS == 5 ? 2 : 1);
-        const int tpp = C1 / cpt;
-        if (C1 % cpt != 0 || tpp > 32 || (tpp & (tpp - 1)) != 0) return PPO_ERR_UNSUPPORTED;
+        const int lpp = C1 / 2;
+        if (C1 % 2 != 0 || lpp > 32 || (lpp & (lpp - 1)) != 0) return PPO_ERR_UNSUPPORTED;
+        const int ppi = 32 / lpp;
         const size_t smem = (size_t)8 * C1 * (KS * KS + 1) * sizeof(float);
-        int blocks = ppo_cdiv(M, (256 / tpp) * 16);
+        int blocks = ppo_cdiv(M, 8 * 64);
         const int cap = ppo_num_sms() * 4;
         blocks = blocks > cap ? cap : (blocks < 1 ? 1 : blocks);
+        long long per_warp = (M + (long long)blocks * 8 - 1) / ((long long)blocks * 8);
+        per_warp = (per_warp + ppi - 1) / ppi * ppi;
         float *dW = m->grad + m->tensors[0].off, *db = m->grad + m->tensors[1].off;
-#define PPO_CONV1W(KS_, CPT_)                                                                                     \
-    conv1_wgrad_kernel<KS_, CPT_><<<blocks, 256, smem, st>>>(depth, m->dact[1], dW, db, rows, d.H, d.W, m->Hs[1], \
-                                                             m->Ws[1], C1)
+#define PPO_CONV1W(KS_)                                                                                          \
+    conv1_wgrad_kernel<KS_><<<blocks, 256, smem, st>>>(depth, m->dact[1], dW, db, rows, d.H, d.W, m->Hs[1],      \
+                                                       m->Ws[1], C1, per_warp)
         if (smem > 48 * 1024) {
-            if (KS == 5) PPO_CUDA_CHECK(cudaFuncSetAttribute(conv1_wgrad_kernel<5, 2>,
+            if (KS == 5) PPO_CUDA_CHECK(cudaFuncSetAttribute(conv1_wgrad_kernel<5>,
                                                              cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-            if (KS == 7) PPO_CUDA_CHECK(cudaFuncSetAttribute(conv1_wgrad_kernel<7, 1>,
+            if (KS == 7) PPO_CUDA_CHECK(cudaFuncSetAttribute(conv1_wgrad_kernel<7>,
                                                              cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
         }
-        if (KS == 1) PPO_CONV1W(1, 4);
-        else if (KS == 3) PPO_CONV1W(3, 4);
-        else if (KS == 5) PPO_CONV1W(5, 2);
-        else PPO_CONV1W(7, 1);
+        if (KS == 1) PPO_CONV1W(1);
+        else if (KS == 3) PPO_CONV1W(3);
+        else if (KS == 5) PPO_CONV1W(5);
+        else PPO_CONV1W(7);
 #undef PPO_CONV1W
         PPO_LAUNCH_CHECK();
     }

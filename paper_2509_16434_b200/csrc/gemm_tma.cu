@@ -705,7 +705,8 @@ int launch_kmajor(KArgs &a, cudaStream_t st) {
     a.nbmax = max_boxes(a.grid);
     const size_t b_bytes = (size_t)a.BN * a.row_bytes;
     const size_t res = (size_t)a.wtaps * a.kchunks * b_bytes;
-    a.wres = (a.tiles_n == 1 && res <= 64 * 1024) ? 1 : 0;
+    // resident weights when they leave room for at least three stages of A tiles
+    a.wres = (a.tiles_n == 1 && res + 3 * (size_t)128 * a.row_bytes <= kSmemBudget) ? 1 : 0;
     const size_t sub = (size_t)128 * a.row_bytes + (a.wres ? 0 : b_bytes);
     const size_t budget = kSmemBudget - (a.wres ? res : 0);
     int G = (int)((40 * 1024) / sub);
