@@ -16,7 +16,7 @@ __global__ void __launch_bounds__(128) conv1_fwd_kernel(const __half *__restrict
                                                         const bf16 *__restrict__ W, const float *__restrict__ bias,
                                                         bf16 *__restrict__ out, int rows, int Hi, int Wi, int Ho,
                                                         int Wo, int C1) {
-    extern __shared__ float sm[];  // w[tap][co], then bias[co], then (STAGE) 4 warps x 32 pixels x C1 bf16
+    extern __shared__ __align__(16) float sm[];  // w[tap][co], then bias[co], then (STAGE) 4 warps x 32 pixels x C1 bf16
     float *w = sm, *bs = sm + KS * KS * C1;
     for (int i = threadIdx.x; i < KS * KS * C1; i += blockDim.x) {
         const int co = i % C1, tap = i / C1;
@@ -52,12 +52,21 @@ __global__ void __launch_bounds__(128) conv1_fwd_kernel(const __half *__restrict
     uint4 *o = reinterpret_cast<uint4 *>(out + m * C1);
     for (int c8 = 0; c8 < C1; c8 += 8) {
         float acc[8];
+        {
+            const float4 b0 = *reinterpret_cast<const float4 *>(bs + c8), b1 = *reinterpret_cast<const float4 *>(bs + c8 + 4);
+            acc[0] = b0.x; acc[1] = b0.y; acc[2] = b0.z; acc[3] = b0.w;
+            acc[4] = b1.x; acc[5] = b1.y; acc[6] = b1.z; acc[7] = b1.w;
+        }
 #pragma unroll
-        for (int j = 0; j < 8; ++j) acc[j] = bs[c8 + j];
-#pragma unroll
-        for (int tap = 0; tap < KS * KS; ++tap)
-#pragma unroll
-            for (int j = 0; j < 8; ++j) acc[j] = fmaf(w[tap * C1 + c8 + j], x[tap], acc[j]);
+        for (int tap = 0; tap < KS * KS; ++tap) {
+            const float4 w0 = *reinterpret_cast<const float4 *>(w + tap * C1 + c8);
+            const float4 w1 = *reinterpret_cast<const float4 *>(w + tap * C1 + c8 + 4);
+            const float xv = x[tap];
+            acc[0] = fmaf(w0.x, xv, acc[0]); acc[1] = fmaf(w0.y, xv, acc[1]);
+            acc[2] = fmaf(w0.z, xv, acc[2]); acc[3] = fmaf(w0.w, xv, acc[3]);
+            acc[4] = fmaf(w1.x, xv, acc[4]); acc[5] = fmaf(w1.y, xv, acc[5]);
+            acc[6] = fmaf(w1.z, xv, acc[6]); acc[7] = fmaf(w1.w, xv, acc[7]);
+        }
         __nv_bfloat162 p[4];
 #pragma unroll
         for (int j = 0; j < 4; ++j) p[j] = __floats2bfloat162_rn(fmaxf(acc[2 * j], 0.f), fmaxf(acc[2 * j + 1], 0.f));
@@ -101,31 +110,48 @@ __global__ void __launch_bounds__(256) conv1_wgrad_kernel(const __half *__restri
     long long m = gw * px_per_warp + ps;
     const long long m_end = min(M, (gw + 1) * px_per_warp);
     if (m < m_end) {
+        // U steps per trip: all their loads are issued before the first multiply-add
+        constexpr int U = KS <= 3 ? 4 : (KS == 5 ? 2 : 1);
         int ow = (int)(m % Wo);
         long long t = m / Wo;
         int oh = (int)(t % Ho);
         long long b = t / Ho;
-        for (; m < m_end; m += ppi) {
-            const float2 dz = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(dZ + m * C1 + 2 * cp));
-            const __half *img = depth + b * Hi * Wi;
+        for (; m < m_end; m += (long long)U * ppi) {
+            float2 dz[U];
+            float xv[U][K2];
 #pragma unroll
-            for (int kh = 0; kh < KS; ++kh) {
-                const int ih = 2 * oh + kh - P;
+            for (int u = 0; u < U; ++u) {
+                const long long mu = m + (long long)u * ppi;
+                const bool live = mu < m_end;
+                dz[u] = live ? __bfloat1622float2(__ldcs(reinterpret_cast<const __nv_bfloat162 *>(dZ + mu * C1 + 2 * cp)))
+                             : make_float2(0.f, 0.f);
+                const __half *img = depth + b * Hi * Wi;
 #pragma unroll
-                for (int kw = 0; kw < KS; ++kw) {
-                    const int iw = 2 * ow + kw - P;
-                    const float xv =
-                        (ih >= 0 && ih < Hi && iw >= 0 && iw < Wi) ? __half2float(__ldg(img + ih * Wi + iw)) : 0.f;
-                    acc0[kh * KS + kw] = fmaf(dz.x, xv, acc0[kh * KS + kw]);
-                    acc1[kh * KS + kw] = fmaf(dz.y, xv, acc1[kh * KS + kw]);
+                for (int kh = 0; kh < KS; ++kh) {
+                    const int ih = 2 * oh + kh - P;
+#pragma unroll
+                    for (int kw = 0; kw < KS; ++kw) {
+                        const int iw = 2 * ow + kw - P;
+                        xv[u][kh * KS + kw] = (live && ih >= 0 && ih < Hi && iw >= 0 && iw < Wi)
+                                                  ? __half2float(__ldg(img + ih * Wi + iw))
+                                                  : 0.f;
+                    }
+                }
+                ow += ppi;
+                while (ow >= Wo) {
+                    ow -= Wo;
+                    if (++oh == Ho) { oh = 0; ++b; }
                 }
             }
-            acc0[K2] += dz.x;
-            acc1[K2] += dz.y;
-            ow += ppi;
-            while (ow >= Wo) {
-                ow -= Wo;
-                if (++oh == Ho) { oh = 0; ++b; }
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+#pragma unroll
+                for (int k = 0; k < K2; ++k) {
+                    acc0[k] = fmaf(dz[u].x, xv[u][k], acc0[k]);
+                    acc1[k] = fmaf(dz[u].y, xv[u][k], acc1[k]);
+                }
+                acc0[K2] += dz[u].x;
+                acc1[K2] += dz[u].y;
             }
         }
     }

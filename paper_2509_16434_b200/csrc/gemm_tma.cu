@@ -121,6 +121,7 @@ enum { EPI_FWD = 0, EPI_HEAD = 1, EPI_DGRAD = 2 };
 constexpr int kEpiWarps = 8;                      // two warps per TMEM lane quarter, alternating 16-column chunks
 constexpr int kKThreads = (2 + kEpiWarps) * 32;   // warp 0: TMA producer, warp 1: MMA issue and TMEM owner
 constexpr int kMaxBias = 512;
+constexpr int kMaxWtab = 64;
 
 // A pipeline stage carries G sub-blocks; sub-block q of a tile is (tap, channel chunk) = divmod(q, kchunks):
 // the A boxes of that tap (128 rows) followed, unless the weights are resident, by its BN weight rows.
@@ -156,6 +157,7 @@ struct PipeK {
     int abort_flag;
     int nboxes;
     Box boxes[kMaxBoxes];
+    uint32_t wtab[4][kMaxWtab];  // resident weights: (byte offset >> 4) of the box that sub-block q of a class reads
     alignas(16) float bias[kMaxBias];
 };
 
@@ -189,6 +191,13 @@ __global__ void __launch_bounds__(kKThreads, 1) tma_kmajor_kernel(const __grid_c
     }
     if (a.mode != EPI_DGRAD)
         for (int i = threadIdx.x; i < a.tiles_n * BN; i += kKThreads) pipe->bias[i] = i < a.N ? a.bias[i] : 0.f;
+    if (a.wres)
+        for (int i = threadIdx.x; i < a.ncls * kMaxWtab; i += kKThreads) {
+            const int c = i / kMaxWtab, q = i - c * kMaxWtab;
+            const int tap = q / a.kchunks, kc = q - tap * a.kchunks;
+            if (tap < a.cls[c].taps.n)
+                pipe->wtab[c][q] = (uint32_t)((int)a.cls[c].taps.wt[tap] * a.kchunks + kc) * (b_bytes >> 4);
+        }
     if (warp == 1) tmem_alloc(&pipe->tmem_slot, ncols);
     tc_fence_before();
     __syncthreads();
@@ -253,22 +262,29 @@ __global__ void __launch_bounds__(kKThreads, 1) tma_kmajor_kernel(const __grid_c
         if (!ok && lane == 0) drain_copies(pipe->full, it, S);
         __syncwarp();
     } else if (warp == 1) {
-        // ---------------- MMA issue: one thread feeds the tensor core
+        // ---------------- MMA issue: one thread feeds the tensor core.  Its instruction stream is the
+        // ceiling of the whole kernel (a lone thread issues a dependent instruction only every few cycles),
+        // so the descriptors are built once and advanced by adds.
         const uint32_t idesc = instr_desc(128, BN, 0, 0);
-        const int nk = a.CB >> 4;  // K = 16 steps per box
         const uint32_t sbo = 8u * rb;
+        const uint64_t d0 = smem_desc_sw(smem_base, 16, sbo, rb);
+        const uint32_t d_lo0 = (uint32_t)d0, d_hi = (uint32_t)(d0 >> 32);
+        const uint32_t res_lo0 = d_lo0 + ((res_base - smem_base) >> 4);
+        const uint32_t stage16 = stage_bytes >> 4, sub16 = sub_bytes >> 4, ab16 = a_bytes >> 4;
+        const bool four = a.CB == 64;  // 4 or 2 K = 16 steps per box (32 bytes each along the swizzled row)
         int it = 0, ti = 0;
         bool ok = true;
         if (a.wres) ok = mbar_wait(&pipe->wfull, 0, abort_flag, a.status);
         for (int g = blockIdx.x; g < a.total_tiles && ok; g += gridDim.x, ++ti) {
             const int c = g / a.tiles_per_cls;
-            const KClass &k = a.cls[c];
-            const int nsub = k.taps.n * a.kchunks;
+            const int nsub = a.cls[c].taps.n * a.kchunks;
+            const uint32_t *tbl = pipe->wtab[c];
             const int acc = ti & 1;
             ok = mbar_wait(&pipe->tempty[acc], ((ti >> 1) & 1) ^ 1, abort_flag, a.status);
             if (!ok) break;
             tc_fence_after();
             const uint32_t tmem_d = tmem_base + acc * acc_cols;
+            uint32_t accum = 0;
             for (int q0 = 0; q0 < nsub; q0 += G, ++it) {
                 const int s = it % S;
                 ok = mbar_wait(&pipe->full[s], (it / S) & 1, abort_flag, a.status);
@@ -276,17 +292,16 @@ __global__ void __launch_bounds__(kKThreads, 1) tma_kmajor_kernel(const __grid_c
                 tc_fence_after();
                 if (lane == 0) {
                     const int nval = min(G, nsub - q0);
-                    for (int gi = 0; gi < nval; ++gi) {
-                        const uint32_t sa = smem_base + (uint32_t)s * stage_bytes + (uint32_t)gi * sub_bytes;
-                        uint32_t sb = sa + a_bytes;
-                        if (a.wres) {
-                            const int q = q0 + gi, tap = q / a.kchunks, kc = q - tap * a.kchunks;
-                            sb = res_base + (uint32_t)((int)k.taps.wt[tap] * a.kchunks + kc) * b_bytes;
+                    uint32_t la = d_lo0 + (uint32_t)s * stage16;
+                    for (int gi = 0; gi < nval; ++gi, la += sub16) {
+                        const uint32_t lb = a.wres ? res_lo0 + tbl[q0 + gi] : la + ab16;
+                        umma_bf16_lh(tmem_d, la, d_hi, lb, d_hi, idesc, accum);
+                        umma_bf16_lh(tmem_d, la + 2, d_hi, lb + 2, d_hi, idesc, 1u);
+                        if (four) {
+                            umma_bf16_lh(tmem_d, la + 4, d_hi, lb + 4, d_hi, idesc, 1u);
+                            umma_bf16_lh(tmem_d, la + 6, d_hi, lb + 6, d_hi, idesc, 1u);
                         }
-                        for (int kk = 0; kk < nk; ++kk)  // K = 16 elements = 32 bytes along the swizzled row
-                            umma_bf16(tmem_d, smem_desc_sw(sa + kk * 32, 16, sbo, rb),
-                                      smem_desc_sw(sb + kk * 32, 16, sbo, rb), idesc,
-                                      (q0 > 0 || gi > 0 || kk > 0) ? 1u : 0u);
+                        accum = 1u;
                     }
                     umma_commit(&pipe->empty[s]);
                 }
@@ -504,18 +519,23 @@ __global__ void __launch_bounds__(kThreads, 1) tma_wgrad_kernel(const __grid_con
         __syncwarp();
     } else if (warp == 1) {
         const uint32_t idesc = instr_desc(128, BN, 1, 1);
+        const uint64_t dA = smem_desc_sw(smem_base, 128u * rbA, 8u * rbA, rbA);
+        const uint64_t dB = smem_desc_sw(smem_base + a_bytes, 128u * rbB, 8u * rbB, rbB);
+        const uint32_t a_hi = (uint32_t)(dA >> 32), b_hi = (uint32_t)(dB >> 32);
+        const uint32_t stepA = rbA, stepB = rbB;  // 16 pixel rows per instruction: (16 * row bytes) >> 4
         bool ok = true;
+        uint32_t accum = 0;
         for (int kb = 0; kb < nkb && ok; ++kb) {
             const int s = kb % S;
             ok = mbar_wait(&pipe->full[s], (kb / S) & 1, abort_flag, a.status);
             if (!ok) break;
             tc_fence_after();
             if (lane == 0) {
-                const uint32_t sa = smem_base + (uint32_t)s * stage_bytes, sb = sa + a_bytes;
-                for (int k = 0; k < a.nmma; ++k)  // 16 pixel rows per instruction
-                    umma_bf16(tmem_d, smem_desc_sw(sa + (uint32_t)k * 16u * rbA, 128u * rbA, 8u * rbA, rbA),
-                              smem_desc_sw(sb + (uint32_t)k * 16u * rbB, 128u * rbB, 8u * rbB, rbB), idesc,
-                              (kb > 0 || k > 0) ? 1u : 0u);
+                uint32_t la = (uint32_t)dA + (uint32_t)s * (stage_bytes >> 4), lb = (uint32_t)dB + (uint32_t)s * (stage_bytes >> 4);
+                for (int k = 0; k < a.nmma; ++k, la += stepA, lb += stepB) {
+                    umma_bf16_lh(tmem_d, la, a_hi, lb, b_hi, idesc, accum);
+                    accum = 1u;
+                }
                 umma_commit(&pipe->empty[s]);
             }
             __syncwarp();
@@ -706,7 +726,7 @@ int launch_kmajor(KArgs &a, cudaStream_t st) {
     const size_t b_bytes = (size_t)a.BN * a.row_bytes;
     const size_t res = (size_t)a.wtaps * a.kchunks * b_bytes;
     // resident weights when they leave room for at least three stages of A tiles
-    a.wres = (a.tiles_n == 1 && res + 3 * (size_t)128 * a.row_bytes <= kSmemBudget) ? 1 : 0;
+    a.wres = (a.tiles_n == 1 && res + 3 * (size_t)128 * a.row_bytes <= kSmemBudget && a.wtaps * a.kchunks <= kMaxWtab) ? 1 : 0;
     const size_t sub = (size_t)128 * a.row_bytes + (a.wres ? 0 : b_bytes);
     const size_t budget = kSmemBudget - (a.wres ? res : 0);
     int G = (int)((40 * 1024) / sub);
