@@ -217,9 +217,15 @@ __global__ void __launch_bounds__(kKThreads, 1) tma_kmajor_kernel(const __grid_c
                 tma_load_2d(res_base + (uint32_t)q * b_bytes, &a.mapB, &pipe->wfull, tap * a.w_tap + kc * a.CB, 0);
             }
         }
-        const int lps = a.nbmax + (a.wres ? 0 : 1);  // copies per sub-block: its A boxes, then its weight rows
-        const int units = G * lps;
-        int it = 0;
+        // Lane l owns copy j = l % lps of sub-block slot gi = l / lps of every stage (G * lps <= 32): its
+        // A box of the tile, or the weight rows.  Per stage a lane only advances (tap, chunk) and issues.
+        const int lps = a.nbmax + (a.wres ? 0 : 1);
+        const int gi = lane / lps, j = lane - gi * lps;
+        const bool lane_on = gi < G;
+        const bool is_b = !a.wres && j == a.nbmax;
+        const uint32_t tx_sub = (uint32_t)a.grid.arows * rb + (a.wres ? 0u : b_bytes);
+        int it = 0, s = 0;
+        uint32_t ph = 0;
         bool ok = true;
         for (int g = blockIdx.x; g < a.total_tiles && ok; g += gridDim.x) {
             const int c = g / a.tiles_per_cls, local = g - c * a.tiles_per_cls;
@@ -227,37 +233,31 @@ __global__ void __launch_bounds__(kKThreads, 1) tma_kmajor_kernel(const __grid_c
             const KClass &k = a.cls[c];
             if (lane == 0) pipe->nboxes = build_boxes(a.grid, mt, pipe->boxes);
             __syncwarp();
-            const int nb = pipe->nboxes;
-            const int nsub = k.taps.n * a.kchunks;
+            const bool have = lane_on && (is_b || j < pipe->nboxes);
+            Box bx = {0, 0, 0, 0, 0};
+            if (have && !is_b) bx = pipe->boxes[j];
+            __syncwarp();
+            const uint32_t dst_off = (uint32_t)gi * sub_bytes + (is_b ? a_bytes : (uint32_t)bx.rowoff * rb);
+            const int cx = bx.x * a.s_mul + a.s_ox, cy = bx.y * a.s_mul + a.s_oy;
+            const void *map = is_b ? (const void *)&a.mapB : (const void *)&a.mapA[bx.hl];
+            const int ntaps = k.taps.n, nsub = ntaps * a.kchunks;
+            int tap = gi / a.kchunks, kc = gi - tap * a.kchunks;
             for (int q0 = 0; q0 < nsub; q0 += G, ++it) {
-                const int s = it % S;
                 int okw = 1;
-                if (lane == 0) okw = mbar_wait(&pipe->empty[s], ((it / S) & 1) ^ 1, abort_flag, a.status) ? 1 : 0;
+                if (lane == 0) okw = mbar_wait(&pipe->empty[s], ph ^ 1u, abort_flag, a.status) ? 1 : 0;
                 ok = __shfl_sync(0xffffffffu, okw, 0) != 0;
                 if (!ok) break;
-                const int nval = min(G, nsub - q0);
-                if (lane == 0) mbar_arrive_expect_tx(&pipe->full[s], (uint32_t)nval * (a.grid.arows * rb + (a.wres ? 0u : b_bytes)));
+                if (lane == 0) mbar_arrive_expect_tx(&pipe->full[s], (uint32_t)min(G, nsub - q0) * tx_sub);
                 __syncwarp();
-                const uint32_t st = smem_base + (uint32_t)s * stage_bytes;
-                for (int u = lane; u < units; u += 32) {
-                    const int gi = u / lps, j = u - gi * lps;
-                    if (gi >= nval) continue;
-                    const int q = q0 + gi, tap = q / a.kchunks, kc = q - tap * a.kchunks;
-                    const uint32_t sa = st + (uint32_t)gi * sub_bytes;
-                    if (j < a.nbmax) {
-                        if (j < nb) {
-                            const Box bx = pipe->boxes[j];
-                            tma_load_4d(sa + (uint32_t)bx.rowoff * rb, &a.mapA[bx.hl], &pipe->full[s], kc * a.CB,
-                                        bx.x * a.s_mul + a.s_ox + k.taps.dx[tap], bx.y * a.s_mul + a.s_oy + k.taps.dy[tap],
-                                        bx.n);
-                        }
-                    } else {
-                        tma_load_2d(sa + a_bytes, &a.mapB, &pipe->full[s], (int)k.taps.wt[tap] * a.w_tap + kc * a.CB, n0);
-                    }
+                if (have && tap < ntaps) {
+                    const uint32_t dst = smem_base + (uint32_t)s * stage_bytes + dst_off;
+                    if (is_b) tma_load_2d(dst, map, &pipe->full[s], (int)k.taps.wt[tap] * a.w_tap + kc * a.CB, n0);
+                    else tma_load_4d(dst, map, &pipe->full[s], kc * a.CB, cx + k.taps.dx[tap], cy + k.taps.dy[tap], bx.n);
                 }
-                __syncwarp();
+                kc += G;
+                while (kc >= a.kchunks) { kc -= a.kchunks; ++tap; }
+                if (++s == S) { s = 0; ph ^= 1u; }
             }
-            __syncwarp();
         }
         if (!ok && lane == 0) drain_copies(pipe->full, it, S);
         __syncwarp();
@@ -272,7 +272,8 @@ __global__ void __launch_bounds__(kKThreads, 1) tma_kmajor_kernel(const __grid_c
         const uint32_t res_lo0 = d_lo0 + ((res_base - smem_base) >> 4);
         const uint32_t stage16 = stage_bytes >> 4, sub16 = sub_bytes >> 4, ab16 = a_bytes >> 4;
         const bool four = a.CB == 64;  // 4 or 2 K = 16 steps per box (32 bytes each along the swizzled row)
-        int it = 0, ti = 0;
+        int ti = 0, s = 0;
+        uint32_t ph = 0;
         bool ok = true;
         if (a.wres) ok = mbar_wait(&pipe->wfull, 0, abort_flag, a.status);
         for (int g = blockIdx.x; g < a.total_tiles && ok; g += gridDim.x, ++ti) {
@@ -285,9 +286,8 @@ __global__ void __launch_bounds__(kKThreads, 1) tma_kmajor_kernel(const __grid_c
             tc_fence_after();
             const uint32_t tmem_d = tmem_base + acc * acc_cols;
             uint32_t accum = 0;
-            for (int q0 = 0; q0 < nsub; q0 += G, ++it) {
-                const int s = it % S;
-                ok = mbar_wait(&pipe->full[s], (it / S) & 1, abort_flag, a.status);
+            for (int q0 = 0; q0 < nsub; q0 += G) {
+                ok = mbar_wait(&pipe->full[s], ph, abort_flag, a.status);
                 if (!ok) break;
                 tc_fence_after();
                 if (lane == 0) {
@@ -306,6 +306,7 @@ __global__ void __launch_bounds__(kKThreads, 1) tma_kmajor_kernel(const __grid_c
                     umma_commit(&pipe->empty[s]);
                 }
                 __syncwarp();
+                if (++s == S) { s = 0; ph ^= 1u; }
             }
             if (ok && lane == 0) umma_commit(&pipe->tfull[acc]);
             __syncwarp();
@@ -482,13 +483,31 @@ __global__ void __launch_bounds__(kThreads, 1) tma_wgrad_kernel(const __grid_con
 
     if (warp == 0) {
         // ---------------- TMA producer: the lanes share out the copies of a K block, one thread each
+        // Lane l owns copy i = l % per_box (an A column block, then the B blocks) of box l / per_box of every
+        // pixel tile; tiles with more boxes than that go round again.
         const int per_box = nvalid + a.nblocks;
+        const int b_l = lane / per_box, i_l = lane - b_l * per_box;
+        const int boxes_per_round = 32 / per_box;
+        int tap = 0, kc = 0, kh = 0, kw = 0;
+        if (i_l < nvalid) {
+            const int jb = jb0 + i_l;
+            tap = jb / a.kchunks;
+            kc = jb - tap * a.kchunks;
+            kh = tap / a.ksz;
+            kw = tap - kh * a.ksz;
+        }
+        const bool is_a = i_l < nvalid;
+        const uint32_t rbu = is_a ? rbA : rbB;
+        const uint32_t blk_off = is_a ? (uint32_t)i_l * 128u * rbA : a_bytes + (uint32_t)(i_l - nvalid) * 128u * rbB;
+        const int c0 = is_a ? kc * a.CB : co0 + (i_l - nvalid) * a.CBn;
+        const int mul = is_a ? a.s_mul : 1, ox = is_a ? kw - a.pad : 0, oy = is_a ? kh - a.pad : 0;
+        const CUtensorMap *maps = is_a ? a.mapA : a.mapB;
         bool ok = true;
-        int kb = 0;
+        int kb = 0, s = 0;
+        uint32_t ph = 0;
         for (; kb < nkb; ++kb) {
-            const int s = kb % S;
             int okw = 1;
-            if (lane == 0) okw = mbar_wait(&pipe->empty[s], ((kb / S) & 1) ^ 1, abort_flag, a.status) ? 1 : 0;
+            if (lane == 0) okw = mbar_wait(&pipe->empty[s], ph ^ 1u, abort_flag, a.status) ? 1 : 0;
             ok = __shfl_sync(0xffffffffu, okw, 0) != 0;
             if (!ok) break;
             if (lane == 0) {
@@ -496,24 +515,16 @@ __global__ void __launch_bounds__(kThreads, 1) tma_wgrad_kernel(const __grid_con
                 pipe->nboxes = build_boxes(a.grid, t_lo + kb, pipe->boxes);
             }
             __syncwarp();
-            const uint32_t sa = smem_base + (uint32_t)s * stage_bytes, sb = sa + a_bytes;
-            const int units = pipe->nboxes * per_box;
-            for (int u = lane; u < units; u += 32) {
-                const int b = u / per_box, i = u - b * per_box;
-                const Box bx = pipe->boxes[b];
-                if (i < nvalid) {
-                    const int jb = jb0 + i, tap = jb / a.kchunks, kc = jb - tap * a.kchunks;
-                    const int kh = tap / a.ksz, kw = tap - kh * a.ksz;
-                    tma_load_4d(sa + (uint32_t)i * 128u * rbA + (uint32_t)bx.rowoff * rbA, &a.mapA[bx.hl],
-                                &pipe->full[s], kc * a.CB, bx.x * a.s_mul - a.pad + kw, bx.y * a.s_mul - a.pad + kh,
-                                bx.n);
-                } else {
-                    const int ib = i - nvalid;
-                    tma_load_4d(sb + (uint32_t)ib * 128u * rbB + (uint32_t)bx.rowoff * rbB, &a.mapB[bx.hl],
-                                &pipe->full[s], co0 + ib * a.CBn, bx.x, bx.y, bx.n);
+            const int nb = pipe->nboxes;
+            const uint32_t st = smem_base + (uint32_t)s * stage_bytes + blk_off;
+            if (b_l < boxes_per_round)
+                for (int b = b_l; b < nb; b += boxes_per_round) {
+                    const Box bx = pipe->boxes[b];
+                    tma_load_4d(st + (uint32_t)bx.rowoff * rbu, &maps[bx.hl], &pipe->full[s], c0, bx.x * mul + ox,
+                                bx.y * mul + oy, bx.n);
                 }
-            }
             __syncwarp();
+            if (++s == S) { s = 0; ph ^= 1u; }
         }
         if (!ok && lane == 0) drain_copies(pipe->full, kb, S);
         __syncwarp();
@@ -524,10 +535,10 @@ __global__ void __launch_bounds__(kThreads, 1) tma_wgrad_kernel(const __grid_con
         const uint32_t a_hi = (uint32_t)(dA >> 32), b_hi = (uint32_t)(dB >> 32);
         const uint32_t stepA = rbA, stepB = rbB;  // 16 pixel rows per instruction: (16 * row bytes) >> 4
         bool ok = true;
-        uint32_t accum = 0;
+        uint32_t accum = 0, ph = 0;
+        int s = 0;
         for (int kb = 0; kb < nkb && ok; ++kb) {
-            const int s = kb % S;
-            ok = mbar_wait(&pipe->full[s], (kb / S) & 1, abort_flag, a.status);
+            ok = mbar_wait(&pipe->full[s], ph, abort_flag, a.status);
             if (!ok) break;
             tc_fence_after();
             if (lane == 0) {
@@ -539,6 +550,7 @@ __global__ void __launch_bounds__(kThreads, 1) tma_wgrad_kernel(const __grid_con
                 umma_commit(&pipe->empty[s]);
             }
             __syncwarp();
+            if (++s == S) { s = 0; ph ^= 1u; }
         }
         if (ok && nkb > 0 && lane == 0) umma_commit(&pipe->tfull[0]);
         __syncwarp();
@@ -732,6 +744,9 @@ int launch_kmajor(KArgs &a, cudaStream_t st) {
     int G = (int)((40 * 1024) / sub);
     G = G < 1 ? 1 : (G > 4 ? 4 : G);
     while (G > 1 && budget / (G * sub) < 3) --G;
+    const int lps = a.nbmax + (a.wres ? 0 : 1);  // copies per sub-block; one producer lane each
+    if (lps > 32) return PPO_ERR_UNSUPPORTED;
+    while (G > 1 && G * lps > 32) --G;
     a.G = G;
     a.stages = (int)(budget / (G * sub));
     if (a.stages > kMaxStages) a.stages = kMaxStages;
