@@ -85,46 +85,55 @@ __global__ void __launch_bounds__(128) conv1_fwd_kernel(const __half *__restrict
 }
 
 // dW1[co][tap] += sum_m dZ1[m][co] * x(m, tap);  db1[co] += sum_m dZ1[m][co].
-// A lane owns one pair of channels; C1 / 2 lanes share a pixel and a warp walks 64 / C1 pixels per
-// step through a contiguous range of output pixels, so that the gradient rows are read once with
-// coalesced 4-byte loads while the k*k input taps of a pixel are one broadcast load each.  Every lane
-// keeps 2 (k*k + 1) accumulators (the last one is the bias gradient); they are folded across the
-// pixel slots of a warp by shuffles, across warps through shared memory, then added with one atomic
-// each.  C1 / 2 must be a power of two <= 32.
-template <int KS>
-__global__ void __launch_bounds__(256) conv1_wgrad_kernel(const __half *__restrict__ depth,
+// A lane owns CPT consecutive channels; C1 / CPT lanes share a pixel and a warp walks 32 CPT / C1
+// pixels per step through a contiguous range of output pixels: the gradient rows are read once,
+// coalesced, 2 CPT bytes per lane, while a pixel's k*k input taps are one broadcast load each, paid
+// once per CPT * (k*k + 1) multiply-adds.  All loads of a trip (U steps) are issued before the first
+// use.  Every lane keeps CPT (k*k + 1) accumulators (the last of each channel is the bias gradient);
+// they are folded across the pixel slots of a warp by shuffles, across warps through shared memory,
+// then added with one atomic each.  C1 / CPT must be a power of two <= 32.
+template <int KS, int CPT, int U>
+__global__ void __launch_bounds__(128) conv1_wgrad_kernel(const __half *__restrict__ depth,
                                                           const bf16 *__restrict__ dZ, float *__restrict__ dW,
                                                           float *__restrict__ db, int rows, int Hi, int Wi, int Ho,
                                                           int Wo, int C1, long long px_per_warp) {
     constexpr int K2 = KS * KS, P = KS / 2;
-    extern __shared__ float sm[];  // [8 warps][C1 * (K2 + 1)]
+    extern __shared__ float sm[];  // [4 warps][C1 * (K2 + 1)]
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int lpp = C1 >> 1;       // lanes per pixel
+    const int lpp = C1 / CPT;      // lanes per pixel
     const int ppi = 32 / lpp;      // pixels per step
-    const int cp = lane % lpp, ps = lane / lpp;
-    float acc0[K2 + 1], acc1[K2 + 1];
+    const int cq = lane % lpp, ps = lane / lpp;
+    float acc[CPT][K2 + 1];
 #pragma unroll
-    for (int t = 0; t <= K2; ++t) acc0[t] = acc1[t] = 0.f;
+    for (int c = 0; c < CPT; ++c)
+#pragma unroll
+        for (int t = 0; t <= K2; ++t) acc[c][t] = 0.f;
     const long long M = (long long)rows * Ho * Wo;
-    const long long gw = (long long)blockIdx.x * 8 + warp;
+    const long long gw = (long long)blockIdx.x * 4 + warp;
     long long m = gw * px_per_warp + ps;
     const long long m_end = min(M, (gw + 1) * px_per_warp);
     if (m < m_end) {
-        // U steps per trip: all their loads are issued before the first multiply-add
-        constexpr int U = KS <= 3 ? 4 : (KS == 5 ? 2 : 1);
         int ow = (int)(m % Wo);
         long long t = m / Wo;
         int oh = (int)(t % Ho);
         long long b = t / Ho;
         for (; m < m_end; m += (long long)U * ppi) {
-            float2 dz[U];
-            float xv[U][K2];
+            uint32_t dzr[U][CPT / 2];
+            __half xr[U][K2];
 #pragma unroll
             for (int u = 0; u < U; ++u) {
                 const long long mu = m + (long long)u * ppi;
                 const bool live = mu < m_end;
-                dz[u] = live ? __bfloat1622float2(__ldcs(reinterpret_cast<const __nv_bfloat162 *>(dZ + mu * C1 + 2 * cp)))
-                             : make_float2(0.f, 0.f);
+                const bf16 *zp = dZ + mu * C1 + cq * CPT;
+                if (CPT == 8) {
+                    const uint4 r = live ? __ldcs(reinterpret_cast<const uint4 *>(zp)) : make_uint4(0, 0, 0, 0);
+                    dzr[u][0] = r.x; dzr[u][1 % (CPT / 2)] = r.y; dzr[u][2 % (CPT / 2)] = r.z; dzr[u][3 % (CPT / 2)] = r.w;
+                } else if (CPT == 4) {
+                    const uint2 r = live ? __ldcs(reinterpret_cast<const uint2 *>(zp)) : make_uint2(0, 0);
+                    dzr[u][0] = r.x; dzr[u][1 % (CPT / 2)] = r.y;
+                } else {
+                    dzr[u][0] = live ? __ldcs(reinterpret_cast<const uint32_t *>(zp)) : 0u;
+                }
                 const __half *img = depth + b * Hi * Wi;
 #pragma unroll
                 for (int kh = 0; kh < KS; ++kh) {
@@ -132,9 +141,8 @@ __global__ void __launch_bounds__(256) conv1_wgrad_kernel(const __half *__restri
 #pragma unroll
                     for (int kw = 0; kw < KS; ++kw) {
                         const int iw = 2 * ow + kw - P;
-                        xv[u][kh * KS + kw] = (live && ih >= 0 && ih < Hi && iw >= 0 && iw < Wi)
-                                                  ? __half2float(__ldg(img + ih * Wi + iw))
-                                                  : 0.f;
+                        const bool in = live && ih >= 0 && ih < Hi && iw >= 0 && iw < Wi;
+                        xr[u][kh * KS + kw] = in ? __ldg(img + ih * Wi + iw) : __float2half_rn(0.f);
                     }
                 }
                 ow += ppi;
@@ -145,39 +153,43 @@ __global__ void __launch_bounds__(256) conv1_wgrad_kernel(const __half *__restri
             }
 #pragma unroll
             for (int u = 0; u < U; ++u) {
+                float xv[K2];
 #pragma unroll
-                for (int k = 0; k < K2; ++k) {
-                    acc0[k] = fmaf(dz[u].x, xv[u][k], acc0[k]);
-                    acc1[k] = fmaf(dz[u].y, xv[u][k], acc1[k]);
+                for (int k = 0; k < K2; ++k) xv[k] = __half2float(xr[u][k]);
+#pragma unroll
+                for (int c2 = 0; c2 < CPT / 2; ++c2) {
+                    const float2 dz = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&dzr[u][c2]));
+#pragma unroll
+                    for (int k = 0; k < K2; ++k) {
+                        acc[2 * c2][k] = fmaf(dz.x, xv[k], acc[2 * c2][k]);
+                        acc[2 * c2 + 1][k] = fmaf(dz.y, xv[k], acc[2 * c2 + 1][k]);
+                    }
+                    acc[2 * c2][K2] += dz.x;
+                    acc[2 * c2 + 1][K2] += dz.y;
                 }
-                acc0[K2] += dz[u].x;
-                acc1[K2] += dz[u].y;
             }
         }
     }
     // fold the pixel slots of the warp (lanes that differ in bits >= log2(lpp))
 #pragma unroll
-    for (int t = 0; t <= K2; ++t) {
-        float v0 = acc0[t], v1 = acc1[t];
-        for (int o = lpp; o < 32; o <<= 1) {
-            v0 += __shfl_xor_sync(0xffffffffu, v0, o);
-            v1 += __shfl_xor_sync(0xffffffffu, v1, o);
+    for (int c = 0; c < CPT; ++c)
+#pragma unroll
+        for (int t = 0; t <= K2; ++t) {
+            float v = acc[c][t];
+            for (int o = lpp; o < 32; o <<= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+            acc[c][t] = v;
         }
-        acc0[t] = v0;
-        acc1[t] = v1;
-    }
     const int per = C1 * (K2 + 1);
     if (lane < lpp) {
 #pragma unroll
-        for (int t = 0; t <= K2; ++t) {
-            sm[warp * per + (2 * cp) * (K2 + 1) + t] = acc0[t];
-            sm[warp * per + (2 * cp + 1) * (K2 + 1) + t] = acc1[t];
-        }
+        for (int c = 0; c < CPT; ++c)
+#pragma unroll
+            for (int t = 0; t <= K2; ++t) sm[warp * per + (cq * CPT + c) * (K2 + 1) + t] = acc[c][t];
     }
     __syncthreads();
-    for (int i = threadIdx.x; i < per; i += 256) {
+    for (int i = threadIdx.x; i < per; i += 128) {
         float v = 0.f;
-        for (int w = 0; w < 8; ++w) v += sm[w * per + i];
+        for (int w = 0; w < 4; ++w) v += sm[w * per + i];
         const int co = i / (K2 + 1), t = i % (K2 + 1);
         if (t < K2) atomicAdd(dW + co * K2 + t, v);
         else atomicAdd(db + co, v);
@@ -539,29 +551,30 @@ extern "C" int ppo_encoder_bwd(ppo_model *m, const ppo_minibatch *mb, int row0, 
         const __half *depth = static_cast<const __half *>(mb->depth_f16) + (size_t)row0 * d.H * d.W;
         const int C1 = m->Cs[1], KS = d.conv_k[0];
         const long long M = (long long)rows * m->Hs[1] * m->Ws[1];
-        const int lpp = C1 / 2;
-        if (C1 % 2 != 0 || lpp > 32 || (lpp & (lpp - 1)) != 0) return PPO_ERR_UNSUPPORTED;
+        const int cpt = KS <= 3 ? 8 : (KS == 5 ? 4 : 2);
+        const int lpp = C1 / cpt;
+        if (C1 % cpt != 0 || lpp > 32 || (lpp & (lpp - 1)) != 0) return PPO_ERR_UNSUPPORTED;
         const int ppi = 32 / lpp;
-        const size_t smem = (size_t)8 * C1 * (KS * KS + 1) * sizeof(float);
-        int blocks = ppo_cdiv(M, 8 * 64);
-        const int cap = ppo_num_sms() * 4;
+        const size_t smem = (size_t)4 * C1 * (KS * KS + 1) * sizeof(float);
+        int blocks = ppo_cdiv(M, 4 * 256);
+        const int cap = ppo_num_sms() * 6;
         blocks = blocks > cap ? cap : (blocks < 1 ? 1 : blocks);
-        long long per_warp = (M + (long long)blocks * 8 - 1) / ((long long)blocks * 8);
+        long long per_warp = (M + (long long)blocks * 4 - 1) / ((long long)blocks * 4);
         per_warp = (per_warp + ppi - 1) / ppi * ppi;
         float *dW = m->grad + m->tensors[0].off, *db = m->grad + m->tensors[1].off;
-#define PPO_CONV1W(KS_)                                                                                          \
-    conv1_wgrad_kernel<KS_><<<blocks, 256, smem, st>>>(depth, m->dact[1], dW, db, rows, d.H, d.W, m->Hs[1],      \
-                                                       m->Ws[1], C1, per_warp)
+#define PPO_CONV1W(KS_, CPT_, U_)                                                                                 \
+    conv1_wgrad_kernel<KS_, CPT_, U_><<<blocks, 128, smem, st>>>(depth, m->dact[1], dW, db, rows, d.H, d.W,      \
+                                                                 m->Hs[1], m->Ws[1], C1, per_warp)
         if (smem > 48 * 1024) {
-            if (KS == 5) PPO_CUDA_CHECK(cudaFuncSetAttribute(conv1_wgrad_kernel<5>,
+            if (KS == 5) PPO_CUDA_CHECK(cudaFuncSetAttribute(conv1_wgrad_kernel<5, 4, 1>,
                                                              cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-            if (KS == 7) PPO_CUDA_CHECK(cudaFuncSetAttribute(conv1_wgrad_kernel<7>,
+            if (KS == 7) PPO_CUDA_CHECK(cudaFuncSetAttribute(conv1_wgrad_kernel<7, 2, 1>,
                                                              cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
         }
-        if (KS == 1) PPO_CONV1W(1);
-        else if (KS == 3) PPO_CONV1W(3);
-        else if (KS == 5) PPO_CONV1W(5);
-        else PPO_CONV1W(7);
+        if (KS == 1) PPO_CONV1W(1, 8, 2);
+        else if (KS == 3) PPO_CONV1W(3, 8, 2);
+        else if (KS == 5) PPO_CONV1W(5, 4, 1);
+        else PPO_CONV1W(7, 2, 1);
 #undef PPO_CONV1W
         PPO_LAUNCH_CHECK();
     }
