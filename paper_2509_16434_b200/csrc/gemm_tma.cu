@@ -14,11 +14,11 @@
 //      and plain boxes of dY, read with the pixel index as the reduction; split over pixel tiles across
 //      CTAs, fp32 atomics into dW.
 //
-// Tiles follow the pixel grid instead of cutting the flattened pixel index every 128: a tile is R whole
-// rows of the (image, row) sequence (R * width <= 128), fetched as a few boxes of 1, 2, 4, ... rows that
-// never straddle an image, or a 128-pixel segment of one row when rows are longer than 128 (the fully
-// connected layers, whose "row" is the batch).  Rows of the 128-row MMA tile beyond R * width are not
-// written and their results are ignored.
+// Tiles follow the pixel grid instead of cutting the flattened pixel index every 128: a tile is a
+// rectangle of Wt pixels by R rows of the (image, row) sequence (Wt * R <= 128, chosen to fill most of
+// the 128 rows), fetched as a few boxes of 1, 2, 4, ... rows that never straddle an image.  A fully
+// connected layer is one image with a single row of `batch` pixels, cut into 128-pixel tiles.  Rows of
+// the 128-row MMA tile beyond Wt * R are not written and their results are ignored.
 //
 // Shared-memory rows are 128 bytes (64 channels, SWIZZLE_128B) or 64 bytes (32 channels, SWIZZLE_64B).
 // Every wait is bounded: on a time-out the kernel records PPO_ERR_TIMEOUT, waits (bounded) for the
@@ -48,10 +48,11 @@ struct Taps {
 // Pixel grid the rows of a GEMM walk: Nimg images of Hr rows of Wr pixels.
 struct RowGrid {
     int Wr, Hr, Nimg;
-    int R;      // grid rows per tile when Wr <= 128, else 0: a tile is a 128-pixel segment of one row
-    int xsegs;  // segments per row when R == 0
-    int tiles;  // tiles over the whole grid
-    int arows;  // pixel rows a tile fills in shared memory: R * Wr, or 128
+    int Wt;     // pixels of a grid row per tile (Wt <= 128)
+    int xsegs;  // tiles side by side along a grid row: ceil(Wr / Wt)
+    int R;      // grid rows per tile (R * Wt <= 128)
+    int tiles;  // tiles over the whole grid: row groups x xsegs
+    int arows;  // pixel rows a tile fills in shared memory: R * Wt
 };
 
 struct Box {
@@ -74,13 +75,8 @@ struct Pipe {
 // Boxes of tile `tile`, in shared-memory row order.  Rows past the last image get an image index >= Nimg,
 // which the copy engine answers with zeros.  Called by one thread.
 __host__ __device__ inline int build_boxes(const RowGrid &g, int tile, Box *out) {
-    if (g.R == 0) {
-        const int frow = tile / g.xsegs, xs = tile - frow * g.xsegs;
-        const int n = frow / g.Hr;
-        out[0] = {n, frow - n * g.Hr, xs * 128, 0, 0};
-        return 1;
-    }
-    int f = tile * g.R, nb = 0, off = 0;
+    const int rg = tile / g.xsegs, x0 = (tile - rg * g.xsegs) * g.Wt;
+    int f = rg * g.R, nb = 0, off = 0;
     const int fend = f + g.R;
     while (f < fend) {
         const int n = f / g.Hr;
@@ -90,10 +86,10 @@ __host__ __device__ inline int build_boxes(const RowGrid &g, int tile, Box *out)
             int hl = 0;
             while ((2 << hl) <= seg) ++hl;
             const int h = 1 << hl;
-            out[nb++] = {n, y, 0, hl, off};
+            out[nb++] = {n, y, x0, hl, off};
             y += h;
             f += h;
-            off += h * g.Wr;
+            off += h * g.Wt;
             seg -= h;
         }
     }
@@ -110,6 +106,29 @@ __device__ void drain_copies(uint64_t *full, int it, int S) {
 }
 
 // ------------------------------------------------------------------ K-major ----
+
+// Tiles are numbered g = (mt * tiles_n + nt) * ncls + c and every CTA takes one contiguous run of them, so
+// that consecutive tiles of a CTA share their pixel tile (the classes of a dgrad) or at least neighbour it.
+struct TileCursor {
+    int g, g_end, mt, nt, c;
+    __device__ void init(int total, int tiles_n, int ncls) {
+        const int q = total / (int)gridDim.x, r = total - q * (int)gridDim.x, b = (int)blockIdx.x;
+        g = b * q + (b < r ? b : r);
+        g_end = g + q + (b < r ? 1 : 0);
+        c = g % ncls;
+        const int t = g / ncls;
+        nt = t % tiles_n;
+        mt = t / tiles_n;
+    }
+    __device__ bool valid() const { return g < g_end; }
+    __device__ void next(int tiles_n, int ncls) {
+        ++g;
+        if (++c == ncls) {
+            c = 0;
+            if (++nt == tiles_n) { nt = 0; ++mt; }
+        }
+    }
+};
 
 struct KClass {
     int o_oy, o_ox;  // output pixel = (y * o_mul + o_oy, x * o_mul + o_ox)
@@ -135,7 +154,7 @@ struct KArgs {
     int w_tap;              // elements between taps in a weight row
     int G, nbmax;           // sub-blocks per stage; most A boxes a tile has
     int wres, wtaps;        // weights resident in shared memory (all wtaps * kchunks boxes, loaded once)
-    int N, BN, tiles_n, tiles_per_cls, total_tiles, ncls, stages;
+    int N, BN, tiles_n, total_tiles, ncls, stages;  // tile g = ((mt * tiles_n) + nt) * ncls + class
     int o_mul, Hout, Wout, ldo;
     int mode, relu, A;
     const float *bias;
@@ -227,16 +246,21 @@ __global__ void __launch_bounds__(kKThreads, 1) tma_kmajor_kernel(const __grid_c
         int it = 0, s = 0;
         uint32_t ph = 0;
         bool ok = true;
-        for (int g = blockIdx.x; g < a.total_tiles && ok; g += gridDim.x) {
-            const int c = g / a.tiles_per_cls, local = g - c * a.tiles_per_cls;
-            const int mt = local / a.tiles_n, n0 = (local - mt * a.tiles_n) * BN;
-            const KClass &k = a.cls[c];
-            if (lane == 0) pipe->nboxes = build_boxes(a.grid, mt, pipe->boxes);
-            __syncwarp();
-            const bool have = lane_on && (is_b || j < pipe->nboxes);
-            Box bx = {0, 0, 0, 0, 0};
-            if (have && !is_b) bx = pipe->boxes[j];
-            __syncwarp();
+        TileCursor tc_;
+        int last_mt = -1;
+        bool have = false;
+        Box bx = {0, 0, 0, 0, 0};
+        for (tc_.init(a.total_tiles, a.tiles_n, a.ncls); tc_.valid() && ok; tc_.next(a.tiles_n, a.ncls)) {
+            const int n0 = tc_.nt * BN;
+            const KClass &k = a.cls[tc_.c];
+            if (tc_.mt != last_mt) {
+                last_mt = tc_.mt;
+                if (lane == 0) pipe->nboxes = build_boxes(a.grid, tc_.mt, pipe->boxes);
+                __syncwarp();
+                have = lane_on && (is_b || j < pipe->nboxes);
+                if (have && !is_b) bx = pipe->boxes[j];
+                __syncwarp();
+            }
             const uint32_t dst_off = (uint32_t)gi * sub_bytes + (is_b ? a_bytes : (uint32_t)bx.rowoff * rb);
             const int cx = bx.x * a.s_mul + a.s_ox, cy = bx.y * a.s_mul + a.s_oy;
             const void *map = is_b ? (const void *)&a.mapB : (const void *)&a.mapA[bx.hl];
@@ -276,8 +300,9 @@ __global__ void __launch_bounds__(kKThreads, 1) tma_kmajor_kernel(const __grid_c
         uint32_t ph = 0;
         bool ok = true;
         if (a.wres) ok = mbar_wait(&pipe->wfull, 0, abort_flag, a.status);
-        for (int g = blockIdx.x; g < a.total_tiles && ok; g += gridDim.x, ++ti) {
-            const int c = g / a.tiles_per_cls;
+        TileCursor tc_;
+        for (tc_.init(a.total_tiles, a.tiles_n, a.ncls); tc_.valid() && ok; tc_.next(a.tiles_n, a.ncls), ++ti) {
+            const int c = tc_.c;
             const int nsub = a.cls[c].taps.n * a.kchunks;
             const uint32_t *tbl = pipe->wtab[c];
             const int acc = ti & 1;
@@ -319,27 +344,24 @@ __global__ void __launch_bounds__(kKThreads, 1) tma_kmajor_kernel(const __grid_c
         const RowGrid &gr = a.grid;
         int ti = 0;
         bool ok = true;
-        for (int g = blockIdx.x; g < a.total_tiles && ok; g += gridDim.x, ++ti) {
-            const int c = g / a.tiles_per_cls, local = g - c * a.tiles_per_cls;
-            const int mt = local / a.tiles_n, n0 = (local - mt * a.tiles_n) * BN;
-            const KClass &k = a.cls[c];
-            // pixel of tile row p
-            bool row_ok;
-            int n, y, x;
-            if (gr.R == 0) {
-                const int frow = mt / gr.xsegs, xs = mt - frow * gr.xsegs;
-                n = frow / gr.Hr;
-                y = frow - n * gr.Hr;
-                x = xs * 128 + p;
-                row_ok = x < gr.Wr;
-            } else {
-                const int fr = p / gr.Wr;
-                x = p - fr * gr.Wr;
-                const int f = mt * gr.R + fr;
+        TileCursor tc_;
+        int last_mt = -1;
+        bool pix_ok = false;  // tile row p is a pixel of the grid
+        int n = 0, y = 0, x = 0;
+        for (tc_.init(a.total_tiles, a.tiles_n, a.ncls); tc_.valid() && ok; tc_.next(a.tiles_n, a.ncls), ++ti) {
+            const int n0 = tc_.nt * BN;
+            const KClass &k = a.cls[tc_.c];
+            if (tc_.mt != last_mt) {  // pixel of tile row p
+                last_mt = tc_.mt;
+                const int rg = tc_.mt / gr.xsegs, xs = tc_.mt - rg * gr.xsegs;
+                const int fr = p / gr.Wt;
+                x = xs * gr.Wt + (p - fr * gr.Wt);
+                const int f = rg * gr.R + fr;
                 n = f / gr.Hr;
                 y = f - n * gr.Hr;
-                row_ok = fr < gr.R && n < gr.Nimg;
+                pix_ok = fr < gr.R && x < gr.Wr && n < gr.Nimg;
             }
+            bool row_ok = pix_ok;
             const int oy = y * a.o_mul + k.o_oy, ox = x * a.o_mul + k.o_ox;
             row_ok = row_ok && oy < a.Hout && ox < a.Wout;
             const long long orow = row_ok ? ((long long)n * a.Hout + oy) * a.Wout + ox : 0;
@@ -640,29 +662,34 @@ int channels_per_box(int C, bool flat) {
     return C % 32 == 0 ? 32 : 0;
 }
 
+// Chooses the tile rectangle Wt x R (Wt * R <= 128) that fills most of the 128 tile rows with pixels of
+// the grid.  Every box starts a multiple of Wt rows into the stage and the copy engine wants 128-byte
+// alignment there, so Wt * row_bytes_min must be a multiple of 128.
 bool make_grid(RowGrid &g, int Wr, int Hr, int Nimg, int row_bytes_min) {
     g.Wr = Wr; g.Hr = Hr; g.Nimg = Nimg;
-    if (Wr <= 128) {
-        const long long rows = (long long)Nimg * Hr;
-        int R = 128 / Wr;
+    const long long rows = (long long)Nimg * Hr;
+    const int wstep = row_bytes_min >= 128 ? 1 : 128 / row_bytes_min;
+    long long best = -1;
+    for (int xs = (Wr + 127) / 128; xs <= (Wr + 127) / 128 + 7 && xs <= Wr; ++xs) {
+        int Wt = (Wr + xs - 1) / xs;
+        Wt = (Wt + wstep - 1) / wstep * wstep;
+        if (Wt > 128) continue;
+        int R = 128 / Wt;
         if (R > kMaxBoxes) R = kMaxBoxes;
         if (R > rows) R = (int)rows;
-        g.R = R;
-        g.xsegs = 1;
-        const long long tiles = (rows + R - 1) / R;
-        if (tiles > 0x3fffffff) return false;
-        g.tiles = (int)tiles;
-        g.arows = R * Wr;
-        // every box starts a multiple of Wr rows into the stage; the copy engine wants 128-byte alignment
-        if (((long long)Wr * row_bytes_min) % 128 != 0) return false;
-    } else {
-        g.R = 0;
-        g.xsegs = (Wr + 127) / 128;
-        const long long tiles = (long long)Nimg * Hr * g.xsegs;
-        if (tiles > 0x3fffffff) return false;
-        g.tiles = (int)tiles;
-        g.arows = 128;
+        const int xsegs = (Wr + Wt - 1) / Wt;
+        const long long util = (long long)Wr * R * 1000 / ((long long)xsegs * 128);  // useful share of tile rows
+        // narrower tiles mean more and smaller boxes: only worth a clear gain, and never below 16 pixels
+        if (best < 0 || (Wt >= 16 && util * 10 > best * 11)) {
+            best = util;
+            g.Wt = Wt; g.xsegs = xsegs; g.R = R;
+        }
     }
+    if (best < 0) return false;
+    const long long tiles = (rows + g.R - 1) / g.R * g.xsegs;
+    if (tiles > 0x3fffffff) return false;
+    g.tiles = (int)tiles;
+    g.arows = g.R * g.Wt;
     return true;
 }
 
@@ -671,9 +698,9 @@ bool make_grid(RowGrid &g, int Wr, int Hr, int Nimg, int row_bytes_min) {
 int make_act_maps(CUtensorMap *maps, const bf16 *base, int C, long long ld, int Ws, int Hs, int Nimg,
                   const RowGrid &g, int CB, int es) {
     const long long dims[4] = {C, Ws, Hs, Nimg};
-    const int wbox = (g.R == 0 ? 128 : g.Wr) * es;
+    const int wbox = g.Wt * es;
     int maxh = 1;
-    if (g.R > 0) while (maxh * 2 <= g.R && maxh * 2 <= g.Hr) maxh *= 2;
+    while (maxh * 2 <= g.R && maxh * 2 <= g.Hr) maxh *= 2;
     for (int i = 0; (1 << i) <= maxh; ++i) {
         const int box[4] = {CB, wbox, (1 << i) * es, 1};
         const int estr[4] = {1, es, es, 1};
@@ -710,12 +737,12 @@ int ensure_smem_attrs() {
 
 // Most A boxes any tile of the grid is cut into (the cut repeats with the tile's first row modulo Hr).
 int max_boxes(const RowGrid &g) {
-    if (g.R == 0) return 1;
     Box tmp[kMaxBoxes];
     int mx = 1;
-    const int lim = g.tiles < g.Hr + 1 ? g.tiles : g.Hr + 1;
+    const int groups = g.tiles / g.xsegs;  // the cut depends on the row group only
+    const int lim = groups < g.Hr + 1 ? groups : g.Hr + 1;
     for (int t = 0; t < lim; ++t) {
-        const int n = build_boxes(g, t, tmp);
+        const int n = build_boxes(g, t * g.xsegs, tmp);
         mx = n > mx ? n : mx;
     }
     const int n = build_boxes(g, g.tiles - 1, tmp);
@@ -732,7 +759,6 @@ int launch_kmajor(KArgs &a, cudaStream_t st) {
     const long long total = per * a.ncls;
     if (total <= 0) return PPO_OK;
     if (total > 0x7fffffffll) return PPO_ERR_UNSUPPORTED;
-    a.tiles_per_cls = (int)per;
     a.total_tiles = (int)total;
     a.nbmax = max_boxes(a.grid);
     const size_t b_bytes = (size_t)a.BN * a.row_bytes;
