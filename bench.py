@@ -180,6 +180,23 @@ class CallTimer:
         return (sum(xs) / len(xs), len(xs)) if xs else (None, 0)
 
 
+def max_over_ranks(values, device):
+    """Element-wise maximum of a list of per-rank floats over all ranks (identity without a process group)."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return [float(v) for v in values]
+    t = torch.tensor(values, device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return t.tolist()
+
+
+def replicas_throughput(world, units_per_step, steps, ms):
+    """Whole-job units per second of `world` independent replicas that each did `steps` steps in `ms`
+    milliseconds (the slowest rank's time)."""
+    return world * units_per_step * steps / (ms * 1e-3)
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -272,13 +289,10 @@ def run_ours(args):
     barrier()
     e2e_ms = e0.elapsed_time(e1)
 
-    if world > 1:
-        t = torch.tensor([ms, e2e_ms], device=device, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms, e2e_ms = t.tolist()
+    ms, e2e_ms = max_over_ranks([ms, e2e_ms], device)
     env_steps = w.M * w.epochs
-    value = world * env_steps * args.steps / (ms * 1e-3)
-    e2e_value = world * env_steps * e2e_steps / (e2e_ms * 1e-3)
+    value = replicas_throughput(world, env_steps, args.steps, ms)
+    e2e_value = replicas_throughput(world, env_steps, e2e_steps, e2e_ms)
 
     if rank == 0:
         # roofline of the dominant calls: encoder forward+backward (tensor-bound), beside the HBM-bound ones
