@@ -109,6 +109,35 @@ int ppo_buffer_write_step(ppo_buffer *buf, int t, const void *dev_depth_f16, con
 int ppo_compute_gae(ppo_buffer *buf, const float *dev_last_value, float gamma, float lambda, int normalize,
                     float *dev_stats_out, void *stream);
 
+/* No counterpart in the paper: a convenience for callers that are not allowed to allocate device
+ * memory.  Some users of this library run it from places where cudaMalloc is off limits: inside a
+ * host process that hands out one fixed arena and forbids further allocations, under a memory
+ * budget that is fixed before the learner starts, or from code that must not synchronise the
+ * device (cudaMalloc and cudaFree may).  ppo_compute_gae needs a small scratch area for the partial
+ * sums of the advantage moments, which normally comes out of the buffer storage that the caller
+ * allocated for ppo_buffer_alloc.  This variant works on bare arrays and keeps that scratch in a
+ * fixed array inside the library image instead, so it never allocates and never frees: no
+ * cudaMalloc, cudaFree or allocating library routine is called, here or by anything it calls.
+ *
+ * Same arithmetic as ppo_compute_gae, on caller-owned device arrays (time-major, s = t*N + n):
+ *   in : dev_reward, dev_value fp32 [T][N]; dev_done uint8 [T][N]; dev_last_value fp32 [N]
+ *   out: dev_adv, dev_ret fp32 [T][N] (dev_adv 16-byte aligned); dev_stats_out fp32 [2] = {mean, std}
+ *        of the raw advantages when normalize != 0 (may be NULL).
+ * Limits and caveats:
+ *  - at most PPO_GAE_STATIC_MAX_ENVS envs (N); more returns PPO_ERR_UNSUPPORTED and launches nothing.
+ *    The scratch is 64 KiB and every GPU that loads the library holds it until the process exits.
+ *  - the first call on each device looks up the scratch array's device address (with that device
+ *    current); make that first call outside any stream capture.
+ *  - all calls on a device share the one scratch array, and it keeps whatever the last call left in
+ *    it.  Each call overwrites every entry it later reads, so nothing needs clearing, but two calls
+ *    whose kernels can overlap on the GPU (different streams, no dependency) race on it: serialise them.
+ * Errors: NULL pointers, T or N <= 0, gamma or lambda outside [0, 1] -> PPO_ERR_INVALID_ARG;
+ * misaligned dev_adv -> PPO_ERR_ALIGN; failure to find the scratch address -> PPO_ERR_CUDA. */
+#define PPO_GAE_STATIC_MAX_ENVS 524288
+int ppo_gae_static(const float *dev_reward, const float *dev_value, const uint8_t *dev_done,
+                   const float *dev_last_value, int T, int N, float gamma, float lambda, int normalize,
+                   float *dev_adv, float *dev_ret, float *dev_stats_out, void *stream);
+
 /* One gathered minibatch: caller-allocated device arrays of B rows. */
 typedef struct {
     void *depth_f16;  /* [B][H][W] fp16 */

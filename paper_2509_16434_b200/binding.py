@@ -26,7 +26,7 @@ EXPORTS = [
     "ppo_model_create", "ppo_model_destroy", "ppo_model_param_count", "ppo_model_arena_elems",
     "ppo_model_num_tensors", "ppo_model_tensor_info", "ppo_model_workspace_bytes", "ppo_model_bind",
     "ppo_model_sync_shadow", "ppo_encoder_fwd", "ppo_loss_fwd_bwd", "ppo_encoder_bwd", "ppo_model_zero_grad",
-    "ppo_adam_step", "ppo_policy_sample", "ppo_poll_status", "ppo_model_activation_ptr",
+    "ppo_adam_step", "ppo_policy_sample", "ppo_poll_status", "ppo_model_activation_ptr", "ppo_gae_static",
 ]
 
 
@@ -98,6 +98,7 @@ def lib():
         L.ppo_policy_sample.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
                                         C.c_void_p]
         L.ppo_poll_status.argtypes = [C.c_void_p]
+        L.ppo_gae_static.argtypes = [C.c_void_p] * 4 + [C.c_int, C.c_int, C.c_float, C.c_float, C.c_int] + [C.c_void_p] * 4
         L.ppo_model_activation_ptr.argtypes = [C.c_void_p, C.c_int, C.c_int, C.POINTER(C.c_void_p),
                                                C.POINTER(C.c_size_t)]
         _lib = L
@@ -191,6 +192,17 @@ def ppo_compute_gae(buf: Buffer, last_value, gamma: float, lam: float, normalize
                     stream=None):
     _check(lib().ppo_compute_gae(buf.handle, _ptr(last_value), gamma, lam, int(normalize), _ptr(stats_out),
                                  _stream(stream)), "ppo_compute_gae")
+
+
+def ppo_gae_static(reward, value, done, last_value, gamma: float, lam: float, normalize: bool, adv, ret,
+                   stats_out=None, stream=None):
+    """GAE (+ advantage normalisation) on bare [T, N] device tensors without any device allocation by the
+    library: for callers that may not call cudaMalloc (fixed arenas, fixed memory budgets).  At most 524288 envs;
+    calls that could overlap on the GPU must be serialised (they share one scratch array inside the library)."""
+    T, N = reward.shape
+    _check(lib().ppo_gae_static(_ptr(reward), _ptr(value), _ptr(done), _ptr(last_value), T, N, gamma, lam,
+                                int(normalize), _ptr(adv), _ptr(ret), _ptr(stats_out), _stream(stream)),
+           "ppo_gae_static")
 
 
 class MinibatchArrays:

@@ -359,6 +359,54 @@ extern "C" int ppo_compute_gae(ppo_buffer *b, const float *last_value, float gam
     return PPO_OK;
 }
 
+// ------------------------------------------------------------ GAE, no allocation ----
+
+// Scratch of ppo_gae_static: the per-block partial sums the scan leaves for the normalisation pass.
+// Lives in the library image, so every device that loads the library holds these 64 KB until exit.
+static __device__ __align__(256) double g_gae_static_scratch[2 * kMaxGaeBlocks];
+
+// Device address of the scratch array on the current device (nullptr on error).  The array's name is
+// only a host-side handle; kernels must be given the address cudaGetSymbolAddress returns.
+static double *gae_static_scratch_ptr() {
+    static double *ptrs[64] = {nullptr};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    if (!ptrs[dev]) {
+        double *p = nullptr;
+        if (cudaGetSymbolAddress((void **)&p, g_gae_static_scratch) != cudaSuccess) return nullptr;
+        ptrs[dev] = p;
+    }
+    return ptrs[dev];
+}
+
+extern "C" int ppo_gae_static(const float *reward, const float *value, const uint8_t *done, const float *last_value,
+                              int T, int N, float gamma, float lambda, int normalize, float *adv, float *ret,
+                              float *stats_out, void *stream) {
+    if (!reward || !value || !done || !last_value || !adv || !ret) return PPO_ERR_INVALID_ARG;
+    if (T <= 0 || N <= 0 || (long long)T * N >= (1ll << 31)) return PPO_ERR_INVALID_ARG;
+    if (!(gamma >= 0.f && gamma <= 1.f) || !(lambda >= 0.f && lambda <= 1.f)) return PPO_ERR_INVALID_ARG;
+    if (N > PPO_GAE_STATIC_MAX_ENVS) return PPO_ERR_UNSUPPORTED;  // more envs than the fixed scratch covers
+    if (!ppo_aligned(adv, 16)) return PPO_ERR_ALIGN;
+    const int threads = 128;
+    const int blocks = ppo_cdiv(N, threads);
+    double *partials = gae_static_scratch_ptr();
+    if (!partials) return PPO_ERR_CUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    // every partial a later pass reads is written by this launch first: nothing has to start at zero
+    gae_scan_kernel<8><<<blocks, threads, 0, st>>>(reward, value, done, last_value, gamma, gamma * lambda, adv, ret, T, N,
+                                                   partials);
+    PPO_LAUNCH_CHECK();
+    if (normalize) {
+        const long long M = (long long)N * T;
+        int nb = ppo_cdiv(M, 256 * 4 * 4);
+        const int cap = ppo_num_sms() * 8;
+        nb = nb > cap ? cap : (nb < 1 ? 1 : nb);
+        adv_normalize_kernel<<<nb, 256, 0, st>>>(adv, M, partials, blocks, stats_out);
+        PPO_LAUNCH_CHECK();
+    }
+    return PPO_OK;
+}
+
 // ------------------------------------------------------------------ gather ----
 
 struct PermParams {
