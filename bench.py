@@ -377,7 +377,8 @@ def cpu_baseline(w, roll, L, n_samples=None):
     """Times the oracle, as it stands, on this machine's host cores over a bounded sample of the same workload."""
     from oracle import oracle as orc
     import torch
-    n_samples = n_samples or (256 if w.H * w.W <= 64 * 64 else 48 if w.H * w.W <= 120 * 160 else 12)
+    # about 10-30 s of oracle work on a 16-core host: ~0.4 / 7 / 35 ms per row at the three frame sizes
+    n_samples = n_samples or min(w.B, 4096 if w.H * w.W <= 64 * 64 else 2048 if w.H * w.W <= 120 * 160 else 512)
     idx = orc.perm(w.seed, 0, w.M, 0, n_samples).astype(np.int64)
     flat = roll["depth"].view(w.M, w.H, w.W)
     fields = {k: roll[k].cpu().numpy() for k in ("proprio", "action", "logp", "value", "reward", "done",
@@ -401,7 +402,8 @@ def run_reference(args):
     from oracle import oracle as orc
     from paper_2509_16434_b200 import synth
     w = synth.WORKLOADS[args.workload]
-    n_samples = 256 if w.H * w.W <= 64 * 64 else 32 if w.H * w.W <= 120 * 160 else 8
+    # every step is a bounded sample; the default 3 + 5 steps stay within a few minutes of host time
+    n_samples = min(w.B, 1024 if w.H * w.W <= 64 * 64 else 512 if w.H * w.W <= 120 * 160 else 96)
     # a host-generated slice of the workload: all small fields at full size, frames only for the sampled rows
     small = w.scaled(w.N, H=2, W=2)
     roll = synth.rollout_numpy(small, w.seed)
@@ -442,7 +444,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg2")
-    ap.add_argument("--microbatch", type=int, default=512)
+    ap.add_argument("--microbatch", type=int, default=2048)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     if args.impl == "reference":
