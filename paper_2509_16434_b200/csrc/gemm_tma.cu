@@ -16,7 +16,7 @@
 //
 // Tiles follow the pixel grid instead of cutting the flattened pixel index every 128: a tile is a
 // rectangle of Wt pixels by R rows of the (image, row) sequence (Wt * R <= 128, chosen to fill most of
-// the 128 rows), fetched as a few boxes of 1, 2, 4, ... rows that never straddle an image.  A fully
+// the 128 rows), fetched as one box per image it touches (a tensor map per box height).  A fully
 // connected layer is one image with a single row of `batch` pixels, cut into 128-pixel tiles.  Rows of
 // the 128-row MMA tile beyond Wt * R are not written and their results are ignored.
 //
@@ -34,7 +34,8 @@ using namespace tc;
 
 constexpr int kMaxTaps = 49;
 constexpr int kMaxBoxes = 32;    // boxes per tile; rows per tile are capped at 32 so that this always holds
-constexpr int kMaxHeights = 6;   // box heights 1, 2, 4, 8, 16, 32 rows
+constexpr int kMaxHeights = 32;  // one tensor map per box height 1 .. 32 rows (a copy costs ~100 cycles to issue,
+                                 // so a tile is cut into as few boxes as the image boundaries allow)
 constexpr int kMaxStages = 8;
 constexpr int kThreads = 192;    // warp 0: TMA producer, warp 1: MMA issue and TMEM owner, warps 2-5: epilogue
 constexpr size_t kSmemBudget = 200 * 1024;
@@ -57,7 +58,7 @@ struct RowGrid {
 
 struct Box {
     int n, y, x;  // image, first row, first pixel
-    int hl;       // log2 of the box height in rows
+    int hl;       // box height in rows, minus one (index of its tensor map)
     int rowoff;   // first shared-memory row of the box
 };
 
@@ -72,28 +73,50 @@ struct Pipe {
     Box boxes[kMaxBoxes];
 };
 
-// Boxes of tile `tile`, in shared-memory row order.  Rows past the last image get an image index >= Nimg,
-// which the copy engine answers with zeros.  Called by one thread.
-__host__ __device__ inline int build_boxes(const RowGrid &g, int tile, Box *out) {
-    const int rg = tile / g.xsegs, x0 = (tile - rg * g.xsegs) * g.Wt;
-    int f = rg * g.R, nb = 0, off = 0;
-    const int fend = f + g.R;
-    while (f < fend) {
-        const int n = f / g.Hr;
-        int y = f - n * g.Hr;
-        int seg = g.Hr - y < fend - f ? g.Hr - y : fend - f;
-        while (seg > 0) {
-            int hl = 0;
-            while ((2 << hl) <= seg) ++hl;
-            const int h = 1 << hl;
-            out[nb++] = {n, y, x0, hl, off};
-            y += h;
-            f += h;
-            off += h * g.Wt;
-            seg -= h;
-        }
+// Boxes of the pixel tile whose first grid row is row y of image n and whose first pixel is x0, in
+// shared-memory row order.  Rows past the last image get an image index >= Nimg, which the copy engine
+// answers with zeros.  Called by one thread.
+__host__ __device__ inline int build_boxes_at(const RowGrid &g, int n, int y, int x0, Box *out) {
+    int left = g.R, nb = 0, off = 0;
+    while (left > 0) {
+        int seg = g.Hr - y < left ? g.Hr - y : left;
+        left -= seg;
+        out[nb++] = {n, y, x0, seg - 1, off};
+        y += seg;
+        off += seg * g.Wt;
+        if (y >= g.Hr) { y = 0; ++n; }
     }
     return nb;
+}
+
+// First grid row (image n, row y) and x segment xs of pixel tile mt; advanced tile by tile without divisions
+// (a lone thread pays a hundred cycles and more for each).
+struct PixTile {
+    int mt, xs, n, y;
+    __host__ __device__ void init(const RowGrid &g, int mt0) {
+        mt = mt0;
+        const int rg = mt0 / g.xsegs;
+        xs = mt0 - rg * g.xsegs;
+        const long long f = (long long)rg * g.R;
+        n = (int)(f / g.Hr);
+        y = (int)(f - (long long)n * g.Hr);
+    }
+    __host__ __device__ void advance_to(const RowGrid &g, int target) {
+        while (mt < target) {
+            ++mt;
+            if (++xs == g.xsegs) {
+                xs = 0;
+                y += g.R;
+                while (y >= g.Hr) { y -= g.Hr; ++n; }
+            }
+        }
+    }
+};
+
+__host__ __device__ inline int build_boxes(const RowGrid &g, int tile, Box *out) {
+    PixTile pt;
+    pt.init(g, tile);
+    return build_boxes_at(g, pt.n, pt.y, pt.xs * g.Wt, out);
 }
 
 // After a time-out: bounded wait for the copies of the last `S` armed stages (iterations it-S .. it-1).
@@ -247,15 +270,20 @@ __global__ void __launch_bounds__(kKThreads, 1) tma_kmajor_kernel(const __grid_c
         uint32_t ph = 0;
         bool ok = true;
         TileCursor tc_;
+        tc_.init(a.total_tiles, a.tiles_n, a.ncls);
+        PixTile pt;
+        pt.init(a.grid, tc_.mt);
         int last_mt = -1;
         bool have = false;
         Box bx = {0, 0, 0, 0, 0};
-        for (tc_.init(a.total_tiles, a.tiles_n, a.ncls); tc_.valid() && ok; tc_.next(a.tiles_n, a.ncls)) {
+        const int tap0 = gi / a.kchunks, kc0 = gi - tap0 * a.kchunks;
+        for (; tc_.valid() && ok; tc_.next(a.tiles_n, a.ncls)) {
             const int n0 = tc_.nt * BN;
             const KClass &k = a.cls[tc_.c];
             if (tc_.mt != last_mt) {
                 last_mt = tc_.mt;
-                if (lane == 0) pipe->nboxes = build_boxes(a.grid, tc_.mt, pipe->boxes);
+                pt.advance_to(a.grid, tc_.mt);
+                if (lane == 0) pipe->nboxes = build_boxes_at(a.grid, pt.n, pt.y, pt.xs * a.grid.Wt, pipe->boxes);
                 __syncwarp();
                 have = lane_on && (is_b || j < pipe->nboxes);
                 if (have && !is_b) bx = pipe->boxes[j];
@@ -265,7 +293,7 @@ __global__ void __launch_bounds__(kKThreads, 1) tma_kmajor_kernel(const __grid_c
             const int cx = bx.x * a.s_mul + a.s_ox, cy = bx.y * a.s_mul + a.s_oy;
             const void *map = is_b ? (const void *)&a.mapB : (const void *)&a.mapA[bx.hl];
             const int ntaps = k.taps.n, nsub = ntaps * a.kchunks;
-            int tap = gi / a.kchunks, kc = gi - tap * a.kchunks;
+            int tap = tap0, kc = kc0;
             for (int q0 = 0; q0 < nsub; q0 += G, ++it) {
                 int okw = 1;
                 if (lane == 0) okw = mbar_wait(&pipe->empty[s], ph ^ 1u, abort_flag, a.status) ? 1 : 0;
@@ -345,20 +373,23 @@ __global__ void __launch_bounds__(kKThreads, 1) tma_kmajor_kernel(const __grid_c
         int ti = 0;
         bool ok = true;
         TileCursor tc_;
+        tc_.init(a.total_tiles, a.tiles_n, a.ncls);
+        PixTile pt;
+        pt.init(gr, tc_.mt);
         int last_mt = -1;
         bool pix_ok = false;  // tile row p is a pixel of the grid
         int n = 0, y = 0, x = 0;
-        for (tc_.init(a.total_tiles, a.tiles_n, a.ncls); tc_.valid() && ok; tc_.next(a.tiles_n, a.ncls), ++ti) {
+        const int fr = p / gr.Wt, xx = p - fr * gr.Wt;  // row and pixel of tile row p inside the tile rectangle
+        for (; tc_.valid() && ok; tc_.next(a.tiles_n, a.ncls), ++ti) {
             const int n0 = tc_.nt * BN;
             const KClass &k = a.cls[tc_.c];
             if (tc_.mt != last_mt) {  // pixel of tile row p
                 last_mt = tc_.mt;
-                const int rg = tc_.mt / gr.xsegs, xs = tc_.mt - rg * gr.xsegs;
-                const int fr = p / gr.Wt;
-                x = xs * gr.Wt + (p - fr * gr.Wt);
-                const int f = rg * gr.R + fr;
-                n = f / gr.Hr;
-                y = f - n * gr.Hr;
+                pt.advance_to(gr, tc_.mt);
+                x = pt.xs * gr.Wt + xx;
+                n = pt.n;
+                y = pt.y + fr;
+                while (y >= gr.Hr) { y -= gr.Hr; ++n; }
                 pix_ok = fr < gr.R && x < gr.Wr && n < gr.Nimg;
             }
             bool row_ok = pix_ok;
@@ -527,6 +558,8 @@ __global__ void __launch_bounds__(kThreads, 1) tma_wgrad_kernel(const __grid_con
         bool ok = true;
         int kb = 0, s = 0;
         uint32_t ph = 0;
+        PixTile pt;
+        pt.init(a.grid, t_lo);
         for (; kb < nkb; ++kb) {
             int okw = 1;
             if (lane == 0) okw = mbar_wait(&pipe->empty[s], ph ^ 1u, abort_flag, a.status) ? 1 : 0;
@@ -534,7 +567,8 @@ __global__ void __launch_bounds__(kThreads, 1) tma_wgrad_kernel(const __grid_con
             if (!ok) break;
             if (lane == 0) {
                 mbar_arrive_expect_tx(&pipe->full[s], tx_bytes);
-                pipe->nboxes = build_boxes(a.grid, t_lo + kb, pipe->boxes);
+                pt.advance_to(a.grid, t_lo + kb);
+                pipe->nboxes = build_boxes_at(a.grid, pt.n, pt.y, pt.xs * a.grid.Wt, pipe->boxes);
             }
             __syncwarp();
             const int nb = pipe->nboxes;
@@ -694,15 +728,14 @@ bool make_grid(RowGrid &g, int Wr, int Hr, int Nimg, int row_bytes_min) {
 }
 
 // Maps of an activation tensor [Nimg][Hs][Ws][C, row stride ld] for boxes of CB channels, the tile width of
-// `g` and heights 1 << i, traversal stride es along W and H.
+// `g` and heights 1 .. min(R, Hr) rows, traversal stride es along W and H.
 int make_act_maps(CUtensorMap *maps, const bf16 *base, int C, long long ld, int Ws, int Hs, int Nimg,
                   const RowGrid &g, int CB, int es) {
     const long long dims[4] = {C, Ws, Hs, Nimg};
     const int wbox = g.Wt * es;
-    int maxh = 1;
-    while (maxh * 2 <= g.R && maxh * 2 <= g.Hr) maxh *= 2;
-    for (int i = 0; (1 << i) <= maxh; ++i) {
-        const int box[4] = {CB, wbox, (1 << i) * es, 1};
+    const int maxh = g.R < g.Hr ? g.R : g.Hr;
+    for (int i = 0; i < maxh; ++i) {
+        const int box[4] = {CB, wbox, (i + 1) * es, 1};
         const int estr[4] = {1, es, es, 1};
         const int s = make_map(&maps[i], base, 4, dims, ld, box, estr, CB * 2);
         if (s != PPO_OK) return s;
@@ -767,8 +800,8 @@ int launch_kmajor(KArgs &a, cudaStream_t st) {
     a.wres = (a.tiles_n == 1 && res + 3 * (size_t)128 * a.row_bytes <= kSmemBudget && a.wtaps * a.kchunks <= kMaxWtab) ? 1 : 0;
     const size_t sub = (size_t)128 * a.row_bytes + (a.wres ? 0 : b_bytes);
     const size_t budget = kSmemBudget - (a.wres ? res : 0);
-    int G = (int)((40 * 1024) / sub);
-    G = G < 1 ? 1 : (G > 4 ? 4 : G);
+    int G = (int)((48 * 1024) / sub);  // sub-blocks per stage: fewer barrier round trips per byte
+    G = G < 1 ? 1 : (G > 8 ? 8 : G);
     while (G > 1 && budget / (G * sub) < 3) --G;
     const int lps = a.nbmax + (a.wres ? 0 : 1);  // copies per sub-block; one producer lane each
     if (lps > 32) return PPO_ERR_UNSUPPORTED;
