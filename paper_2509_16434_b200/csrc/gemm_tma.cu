@@ -39,6 +39,7 @@ constexpr int kMaxHeights = 32;  // one tensor map per box height 1 .. 32 rows (
 constexpr int kMaxStages = 8;
 constexpr int kThreads = 192;    // warp 0: TMA producer, warp 1: MMA issue and TMEM owner, warps 2-5: epilogue
 constexpr size_t kSmemBudget = 200 * 1024;
+constexpr size_t kMaxResident = 64 * 1024;
 
 struct Taps {
     int n;
@@ -192,8 +193,8 @@ struct KArgs {
 struct PipeK {
     uint64_t full[kMaxStages];
     uint64_t empty[kMaxStages];
-    uint64_t tfull[2];
-    uint64_t tempty[2];
+    uint64_t tfull[4];
+    uint64_t tempty[4];
     uint64_t wfull;
     uint32_t tmem_slot;
     int abort_flag;
@@ -215,15 +216,17 @@ __global__ void __launch_bounds__(kKThreads, 1) tma_kmajor_kernel(const __grid_c
     PipeK *pipe = reinterpret_cast<PipeK *>(smem + (size_t)S * stage_bytes + res_bytes);
     volatile int *abort_flag = &pipe->abort_flag;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    // ring of accumulators in tensor memory: four when they fit in its 512 columns, else two
     const uint32_t acc_cols = tmem_cols_for(BN);
-    const uint32_t ncols = acc_cols * 2;
+    const int nacc_log = acc_cols * 4 <= 512 ? 2 : 1, nacc = 1 << nacc_log;
+    const uint32_t ncols = acc_cols * nacc;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < S; ++s) {
             mbar_init(&pipe->full[s], 1);
             mbar_init(&pipe->empty[s], 1);
         }
-        for (int i = 0; i < 2; ++i) {
+        for (int i = 0; i < nacc; ++i) {
             mbar_init(&pipe->tfull[i], 1);
             mbar_init(&pipe->tempty[i], kEpiWarps * 32);
         }
@@ -333,8 +336,8 @@ __global__ void __launch_bounds__(kKThreads, 1) tma_kmajor_kernel(const __grid_c
             const int c = tc_.c;
             const int nsub = a.cls[c].taps.n * a.kchunks;
             const uint32_t *tbl = pipe->wtab[c];
-            const int acc = ti & 1;
-            ok = mbar_wait(&pipe->tempty[acc], ((ti >> 1) & 1) ^ 1, abort_flag, a.status);
+            const int acc = ti & (nacc - 1);
+            ok = mbar_wait(&pipe->tempty[acc], ((ti >> nacc_log) & 1) ^ 1, abort_flag, a.status);
             if (!ok) break;
             tc_fence_after();
             const uint32_t tmem_d = tmem_base + acc * acc_cols;
@@ -396,12 +399,28 @@ __global__ void __launch_bounds__(kKThreads, 1) tma_kmajor_kernel(const __grid_c
             const int oy = y * a.o_mul + k.o_oy, ox = x * a.o_mul + k.o_ox;
             row_ok = row_ok && oy < a.Hout && ox < a.Wout;
             const long long orow = row_ok ? ((long long)n * a.Hout + oy) * a.Wout + ox : 0;
-            const int acc = ti & 1;
-            ok = mbar_wait(&pipe->tfull[acc], (ti >> 1) & 1, abort_flag, a.status);
+            // the ReLU mask of this warp's first two chunks is fetched before the accumulator is waited for,
+            // so that its memory latency overlaps the tile's MMAs
+            uint4 mpre[2][2];
+            const bool use_mask = a.mode == EPI_DGRAD && a.mask != nullptr;
+            if (use_mask && row_ok) {
+#pragma unroll
+                for (int j = 0; j < 2; ++j) {
+                    const int nn = n0 + half * 16 + j * 32;
+                    if (half * 16 + j * 32 < BN && nn < a.N) {
+                        const uint4 *mp = reinterpret_cast<const uint4 *>(a.mask + orow * a.ldo + nn);
+                        mpre[j][0] = mp[0];
+                        if (nn + 8 < a.N) mpre[j][1] = mp[1];
+                    }
+                }
+            }
+            const int acc = ti & (nacc - 1);
+            ok = mbar_wait(&pipe->tfull[acc], (ti >> nacc_log) & 1, abort_flag, a.status);
             if (!ok) break;
             tc_fence_after();
             const uint32_t lane_base = tmem_base + acc * acc_cols + ((uint32_t)(lg * 32) << 16);
-            for (int c0 = half * 16; c0 < BN; c0 += 32) {
+            int chunk = 0;
+            for (int c0 = half * 16; c0 < BN; c0 += 32, ++chunk) {
                 if (n0 + c0 >= a.N) break;  // uniform across the warp
                 float v[16];
                 tmem_ld16(lane_base + (uint32_t)c0, v);
@@ -426,12 +445,12 @@ __global__ void __launch_bounds__(kKThreads, 1) tma_kmajor_kernel(const __grid_c
 #pragma unroll
                         for (int i = 0; i < 16; ++i) v[i] = fmaxf(v[i], 0.f);
                     }
-                } else if (a.mask) {
+                } else if (use_mask) {
                     const uint4 *mp = reinterpret_cast<const uint4 *>(a.mask + orow * a.ldo + nn);
 #pragma unroll
                     for (int hlf = 0; hlf < 2; ++hlf) {
                         if (nn + hlf * 8 < a.N) {
-                            const uint4 mk = mp[hlf];
+                            const uint4 mk = chunk == 0 ? mpre[0][hlf] : (chunk == 1 ? mpre[1][hlf] : mp[hlf]);
                             const __nv_bfloat162 *m2 = reinterpret_cast<const __nv_bfloat162 *>(&mk);
 #pragma unroll
                             for (int i = 0; i < 4; ++i) {
@@ -796,8 +815,9 @@ int launch_kmajor(KArgs &a, cudaStream_t st) {
     a.nbmax = max_boxes(a.grid);
     const size_t b_bytes = (size_t)a.BN * a.row_bytes;
     const size_t res = (size_t)a.wtaps * a.kchunks * b_bytes;
-    // resident weights when they leave room for at least three stages of A tiles
-    a.wres = (a.tiles_n == 1 && res + 3 * (size_t)128 * a.row_bytes <= kSmemBudget && a.wtaps * a.kchunks <= kMaxWtab) ? 1 : 0;
+    // resident weights only while they leave most of the shared memory to the A stages: the bytes in flight
+    // are what hides the copy latency
+    a.wres = (a.tiles_n == 1 && res <= kMaxResident && a.wtaps * a.kchunks <= kMaxWtab) ? 1 : 0;
     const size_t sub = (size_t)128 * a.row_bytes + (a.wres ? 0 : b_bytes);
     const size_t budget = kSmemBudget - (a.wres ? res : 0);
     int G = (int)((48 * 1024) / sub);  // sub-blocks per stage: fewer barrier round trips per byte
