@@ -71,6 +71,9 @@ struct ppo_model {
     bf16 *wT;                      // transposed bf16 weights Wt[ci][tap][co padded to 8] for the dgrad GEMMs
     int64_t wT_off[2 * PPO_MAX_CONV + 2 * PPO_MAX_FC + 3];  // per tensor index (matrices only)
     size_t wT_elems;
+    bf16 *wC;                      // conv weights regrouped for the merged dgrad: Wc[class*Ci+ci][shift][co]
+    int64_t wC_off[PPO_MAX_CONV + 1];  // per conv layer l (2..L)
+    size_t wC_elems;
     float *loss_partials;
     int loss_partial_blocks;
     bool wT_valid;

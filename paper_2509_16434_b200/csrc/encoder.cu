@@ -368,9 +368,9 @@ static int run_fwd(const ppo_model *m, const ConvGeom &g, const bf16 *X, const b
 }
 
 static int run_dgrad(const ppo_model *m, const ConvGeom &g, const bf16 *dY, int ldy, const bf16 *W, const bf16 *Wt,
-                     int wt_ld, const DgradEpilogue &e, cudaStream_t st) {
+                     int wt_ld, const bf16 *Wc, const DgradEpilogue &e, cudaStream_t st) {
     if (m->impl == 1) return simt_gemm_dgrad(g, dY, ldy, W, e, st);
-    const int s = tma_gemm_dgrad(g, dY, ldy, Wt, wt_ld, e, ppo_device_status_ptr(), st);
+    const int s = tma_gemm_dgrad(g, dY, ldy, Wt, wt_ld, Wc, e, ppo_device_status_ptr(), st);
     if (s != PPO_ERR_UNSUPPORTED) return s;
     return tc_gemm_dgrad(g, dY, ldy, Wt, wt_ld, e, ppo_device_status_ptr(), st);
 }
@@ -490,6 +490,8 @@ static int refresh_transposed(ppo_model *m, cudaStream_t st) {
                                                                      m->wT + m->wT_off[2 * (l - 1)], Co, taps, Ci,
                                                                      wt_ld_of(Co));
         PPO_LAUNCH_CHECK();
+        PPO_TRY(tma_dgrad_weights(m->shadow + m->tensors[2 * (l - 1)].off, m->wC + m->wC_off[l], Co, m->d.conv_k[l - 1], Ci,
+                                  wt_ld_of(Co), st));
     }
     int ti = 2 * m->L;
     for (int l = 1; l <= m->F + 1; ++l, ti += 2) {
@@ -529,7 +531,7 @@ extern "C" int ppo_encoder_bwd(ppo_model *m, const ppo_minibatch *mb, int row0, 
         DgradEpilogue e;
         if (l > 1) e = {m->h[l - 1], m->dh[l - 1], nullptr};
         else e = {nullptr, nullptr, m->dh0_f32};
-        PPO_TRY(run_dgrad(m, g, dY, ldy, m->shadow + m->tensors[ti].off, m->wT + m->wT_off[ti], wt_ld_of(Co), e, st));
+        PPO_TRY(run_dgrad(m, g, dY, ldy, m->shadow + m->tensors[ti].off, m->wT + m->wT_off[ti], wt_ld_of(Co), nullptr, e, st));
     }
     {
         const int npx = m->Hs[L] * m->Ws[L], C = m->Cs[L];
@@ -545,7 +547,7 @@ extern "C" int ppo_encoder_bwd(ppo_model *m, const ppo_minibatch *mb, int row0, 
         PPO_TRY(run_colsum(m->dact[l], g.Co, g.M(), g.Co, m->grad + m->tensors[ti + 1].off, st));
         DgradEpilogue e = {m->act[l - 1], m->dact[l - 1], nullptr};
         PPO_TRY(run_dgrad(m, g, m->dact[l], g.Co, m->shadow + m->tensors[ti].off, m->wT + m->wT_off[ti],
-                          wt_ld_of(g.Co), e, st));
+                          wt_ld_of(g.Co), m->wC + m->wC_off[l], e, st));
     }
     {   // conv1: weight and bias gradients only
         const __half *depth = static_cast<const __half *>(mb->depth_f16) + (size_t)row0 * d.H * d.W;

@@ -41,7 +41,11 @@ int tc_gemm_wgrad(const ConvGeom &g, const bf16 *dY, int ldy, const bf16 *X, flo
 // for anything else they return PPO_ERR_UNSUPPORTED without launching and the caller uses the tc_ versions.
 int tma_gemm_fwd(const ConvGeom &g, const bf16 *X, const bf16 *W, const FwdEpilogue &e, int32_t *status,
                  cudaStream_t st);
-int tma_gemm_dgrad(const ConvGeom &g, const bf16 *dY, int ldy, const bf16 *Wt, int wt_ld, const DgradEpilogue &e,
-                   int32_t *status, cudaStream_t st);
+// Wc: the layer's weights regrouped by tma_dgrad_weights for the merged four-class dgrad (convolutions only;
+// fully connected layers read Wt).
+int tma_gemm_dgrad(const ConvGeom &g, const bf16 *dY, int ldy, const bf16 *Wt, int wt_ld, const bf16 *Wc,
+                   const DgradEpilogue &e, int32_t *status, cudaStream_t st);
+size_t tma_dgrad_weight_elems(int Ci, int k, int wt_ld);
+int tma_dgrad_weights(const bf16 *W, bf16 *Wc, int Co, int k, int Ci, int wt_ld, cudaStream_t st);
 int tma_gemm_wgrad(const ConvGeom &g, const bf16 *dY, int ldy, const bf16 *X, float *dW, int32_t *status,
                    cudaStream_t st);

@@ -154,8 +154,10 @@ struct TileCursor {
     }
 };
 
+// One group of output columns with its own tap list: the whole GEMM for a forward pass; for a merged dgrad
+// one tile of BN columns of the (parity class, input channel) axis, which only some shifts reach.
 struct KClass {
-    int o_oy, o_ox;  // output pixel = (y * o_mul + o_oy, x * o_mul + o_ox)
+    int b_row0;  // first weight row (output column) of the group
     Taps taps;
 };
 
@@ -179,7 +181,8 @@ struct KArgs {
     int G, nbmax;           // sub-blocks per stage; most A boxes a tile has
     int wres, wtaps;        // weights resident in shared memory (all wtaps * kchunks boxes, loaded once)
     int N, BN, tiles_n, total_tiles, ncls, stages;  // tile g = ((mt * tiles_n) + nt) * ncls + class
-    int o_mul, Hout, Wout, ldo;
+    int Hout, Wout, ldo;
+    int nq_ci;  // merged dgrad: channels per parity class (column n = class * nq_ci + channel), else 0
     int mode, relu, A;
     const float *bias;
     bf16 *out;
@@ -306,7 +309,7 @@ __global__ void __launch_bounds__(kKThreads, 1) tma_kmajor_kernel(const __grid_c
                 __syncwarp();
                 if (have && tap < ntaps) {
                     const uint32_t dst = smem_base + (uint32_t)s * stage_bytes + dst_off;
-                    if (is_b) tma_load_2d(dst, map, &pipe->full[s], (int)k.taps.wt[tap] * a.w_tap + kc * a.CB, n0);
+                    if (is_b) tma_load_2d(dst, map, &pipe->full[s], (int)k.taps.wt[tap] * a.w_tap + kc * a.CB, n0 + k.b_row0);
                     else tma_load_4d(dst, map, &pipe->full[s], kc * a.CB, cx + k.taps.dx[tap], cy + k.taps.dy[tap], bx.n);
                 }
                 kc += G;
@@ -395,22 +398,36 @@ __global__ void __launch_bounds__(kKThreads, 1) tma_kmajor_kernel(const __grid_c
                 while (y >= gr.Hr) { y -= gr.Hr; ++n; }
                 pix_ok = fr < gr.R && x < gr.Wr && n < gr.Nimg;
             }
-            bool row_ok = pix_ok;
-            const int oy = y * a.o_mul + k.o_oy, ox = x * a.o_mul + k.o_ox;
-            row_ok = row_ok && oy < a.Hout && ox < a.Wout;
-            const long long orow = row_ok ? ((long long)n * a.Hout + oy) * a.Wout + ox : 0;
+            // Output row and column of this thread's accumulator columns c0 .. c0+15.  Forward and flat GEMMs:
+            // the pixel itself.  Merged dgrad: column class * nq_ci + channel belongs to input pixel
+            // (2y + class / 2, 2x + class % 2).
+            auto locate = [&](int c0, long long &orow, int &col) -> bool {
+                col = n0 + c0;
+                int oy = y, ox = x;
+                if (a.nq_ci) {
+                    const int gc = k.b_row0 + col, q = gc / a.nq_ci;
+                    col = gc - q * a.nq_ci;
+                    oy = 2 * y + (q >> 1);
+                    ox = 2 * x + (q & 1);
+                }
+                orow = ((long long)n * a.Hout + oy) * a.Wout + ox;
+                return pix_ok && oy < a.Hout && ox < a.Wout;
+            };
+            const int ncol = a.nq_ci ? a.nq_ci : a.N;  // columns of an output row
             // the ReLU mask of this warp's first two chunks is fetched before the accumulator is waited for,
             // so that its memory latency overlaps the tile's MMAs
             uint4 mpre[2][2];
             const bool use_mask = a.mode == EPI_DGRAD && a.mask != nullptr;
-            if (use_mask && row_ok) {
+            if (use_mask) {
 #pragma unroll
                 for (int j = 0; j < 2; ++j) {
-                    const int nn = n0 + half * 16 + j * 32;
-                    if (half * 16 + j * 32 < BN && nn < a.N) {
-                        const uint4 *mp = reinterpret_cast<const uint4 *>(a.mask + orow * a.ldo + nn);
+                    const int c0 = half * 16 + j * 32;
+                    long long orow;
+                    int col;
+                    if (c0 < BN && n0 + c0 < a.N && locate(c0, orow, col)) {
+                        const uint4 *mp = reinterpret_cast<const uint4 *>(a.mask + orow * a.ldo + col);
                         mpre[j][0] = mp[0];
-                        if (nn + 8 < a.N) mpre[j][1] = mp[1];
+                        if (col + 8 < ncol) mpre[j][1] = mp[1];
                     }
                 }
             }
@@ -424,8 +441,9 @@ __global__ void __launch_bounds__(kKThreads, 1) tma_kmajor_kernel(const __grid_c
                 if (n0 + c0 >= a.N) break;  // uniform across the warp
                 float v[16];
                 tmem_ld16(lane_base + (uint32_t)c0, v);
-                if (!row_ok) continue;
-                const int nn = n0 + c0;
+                long long orow;
+                int nn;
+                if (!locate(c0, orow, nn)) continue;
                 if (a.mode == EPI_HEAD) {
 #pragma unroll
                     for (int i = 0; i < 16; ++i) {
@@ -449,7 +467,7 @@ __global__ void __launch_bounds__(kKThreads, 1) tma_kmajor_kernel(const __grid_c
                     const uint4 *mp = reinterpret_cast<const uint4 *>(a.mask + orow * a.ldo + nn);
 #pragma unroll
                     for (int hlf = 0; hlf < 2; ++hlf) {
-                        if (nn + hlf * 8 < a.N) {
+                        if (nn + hlf * 8 < ncol) {
                             const uint4 mk = chunk == 0 ? mpre[0][hlf] : (chunk == 1 ? mpre[1][hlf] : mp[hlf]);
                             const __nv_bfloat162 *m2 = reinterpret_cast<const __nv_bfloat162 *>(&mk);
 #pragma unroll
@@ -465,7 +483,7 @@ __global__ void __launch_bounds__(kKThreads, 1) tma_kmajor_kernel(const __grid_c
                     uint4 *op = reinterpret_cast<uint4 *>(a.out + orow * a.ldo + nn);
 #pragma unroll
                     for (int hlf = 0; hlf < 2; ++hlf) {
-                        if (nn + hlf * 8 < a.N) {
+                        if (nn + hlf * 8 < ncol) {
                             __nv_bfloat162 pk[4];
 #pragma unroll
                             for (int i = 0; i < 4; ++i)
@@ -478,7 +496,7 @@ __global__ void __launch_bounds__(kKThreads, 1) tma_kmajor_kernel(const __grid_c
                     float4 *op = reinterpret_cast<float4 *>(a.out_f32 + orow * a.ldo + nn);
 #pragma unroll
                     for (int q = 0; q < 4; ++q)
-                        if (nn + q * 4 < a.N) op[q] = make_float4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
+                        if (nn + q * 4 < ncol) op[q] = make_float4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
                 }
             }
             tc_fence_before();
@@ -817,7 +835,7 @@ int launch_kmajor(KArgs &a, cudaStream_t st) {
     const size_t res = (size_t)a.wtaps * a.kchunks * b_bytes;
     // resident weights only while they leave most of the shared memory to the A stages: the bytes in flight
     // are what hides the copy latency
-    a.wres = (a.tiles_n == 1 && res <= kMaxResident && a.wtaps * a.kchunks <= kMaxWtab) ? 1 : 0;
+    a.wres = (a.tiles_n == 1 && a.ncls == 1 && res <= kMaxResident && a.wtaps * a.kchunks <= kMaxWtab) ? 1 : 0;
     const size_t sub = (size_t)128 * a.row_bytes + (a.wres ? 0 : b_bytes);
     const size_t budget = kSmemBudget - (a.wres ? res : 0);
     int G = (int)((48 * 1024) / sub);  // sub-blocks per stage: fewer barrier round trips per byte
@@ -870,7 +888,6 @@ int tma_gemm_fwd(const ConvGeom &g, const bf16 *X, const bf16 *W, const FwdEpilo
     }
     a.s_mul = flat ? 1 : 2;
     a.s_oy = a.s_ox = -g.pad;
-    a.o_mul = 1;
     a.Hout = flat ? 1 : g.Ho;
     a.Wout = flat ? g.B : g.Wo;
     a.ldo = g.Co;
@@ -885,7 +902,7 @@ int tma_gemm_fwd(const ConvGeom &g, const bf16 *X, const bf16 *W, const FwdEpilo
     if (a.mode == EPI_FWD && g.Co % 8 != 0) return PPO_ERR_UNSUPPORTED;
     a.ncls = 1;
     KClass &k = a.cls[0];
-    k.o_oy = k.o_ox = 0;
+    k.b_row0 = 0;
     k.taps.n = g.taps();
     for (int t = 0; t < g.taps(); ++t) {
         k.taps.dy[t] = (signed char)(t / g.k);
@@ -895,11 +912,23 @@ int tma_gemm_fwd(const ConvGeom &g, const bf16 *X, const bf16 *W, const FwdEpilo
     return launch_kmajor(a, st);
 }
 
-int tma_gemm_dgrad(const ConvGeom &g, const bf16 *dY, int ldy, const bf16 *Wt, int wt_ld, const DgradEpilogue &e,
-                   int32_t *status, cudaStream_t st) {
+static void tma_dgrad_shifts(int k, int *dmin, int *n1) {
+    const int pad = k / 2;
+    *dmin = -((k - 1 - pad) / 2);
+    *n1 = (1 + pad) / 2 - *dmin + 1;
+}
+
+// Fully connected layers: dX[b][ci] = sum_co dY[b][co] Wt[ci][co].  Convolutions: the four stride-parity
+// classes of input pixels are computed together.  Row (y, x) of the GEMM stands for the 2x2 block of input
+// pixels (2y + ph, 2x + pw); column class * Ci + ci; the reduction runs over the shifts (dy, dx) of the
+// output pixel (y + dy, x + dx) and its channels, with the weights Wc[class * Ci + ci][shift][co] (zero
+// where a class has no kernel tap at that shift).  One wide GEMM instead of four narrow ones: the tensor
+// core is fed by one thread, and an instruction costs the same whether it is 32 or 256 columns wide.
+int tma_gemm_dgrad(const ConvGeom &g, const bf16 *dY, int ldy, const bf16 *Wt, int wt_ld, const bf16 *Wc,
+                   const DgradEpilogue &e, int32_t *status, cudaStream_t st) {
     if (!status || g.Ci % 8 != 0 || ldy % 8 != 0 || wt_ld % 8 != 0 || ldy < wt_ld) return PPO_ERR_UNSUPPORTED;
     const bool flat = is_flat(g);
-    if (!flat && (g.k < 3 || g.Hi < 2 || g.Wi < 2)) return PPO_ERR_UNSUPPORTED;
+    if (!flat && (g.k < 3 || g.Hi < 2 || g.Wi < 2 || !Wc || g.Ci % 16 != 0)) return PPO_ERR_UNSUPPORTED;
     const int CB = channels_per_box(g.Co, flat);
     if (CB == 0 || g.taps() > kMaxTaps || wt_ld < g.Co) return PPO_ERR_UNSUPPORTED;
     KArgs a = {};
@@ -907,25 +936,13 @@ int tma_gemm_dgrad(const ConvGeom &g, const bf16 *dY, int ldy, const bf16 *Wt, i
     a.row_bytes = CB * 2;
     a.kchunks = (g.Co + CB - 1) / CB;
     a.w_tap = wt_ld;
-    a.wtaps = g.taps();
-    // rows: input pixels of one stride-parity class, (Hi+1)/2 x (Wi+1)/2 of them (classes that have fewer
-    // drop the excess in the epilogue)
     const int Hr = flat ? 1 : (g.Hi + 1) / 2, Wr = flat ? g.B : (g.Wi + 1) / 2;
     if (!make_grid(a.grid, Wr, Hr, flat ? 1 : g.B, a.row_bytes)) return PPO_ERR_UNSUPPORTED;
     int s = flat ? make_act_maps(a.mapA, dY, g.Co, ldy, g.B, 1, 1, a.grid, CB, 1)
                  : make_act_maps(a.mapA, dY, g.Co, ldy, g.Wo, g.Ho, g.B, a.grid, CB, 1);
     if (s != PPO_OK) return s;
-    a.N = g.Ci;
-    a.BN = pick_bn(g.Ci);
-    {
-        const long long dims[2] = {(long long)g.taps() * wt_ld, g.Ci};
-        const int box[2] = {CB, a.BN}, es[2] = {1, 1};
-        s = make_map(&a.mapB, Wt, 2, dims, (long long)g.taps() * wt_ld, box, es, a.row_bytes);
-        if (s != PPO_OK) return s;
-    }
     a.s_mul = 1;
     a.s_oy = a.s_ox = 0;
-    a.o_mul = flat ? 1 : 2;
     a.Hout = flat ? 1 : g.Hi;
     a.Wout = flat ? g.B : g.Wi;
     a.ldo = g.Ci;
@@ -935,34 +952,91 @@ int tma_gemm_dgrad(const ConvGeom &g, const bf16 *dY, int ldy, const bf16 *Wt, i
     a.mask = e.mask_act;
     a.status = status;
     if (flat) {
+        a.N = g.Ci;
+        a.BN = pick_bn(g.Ci);
+        a.wtaps = 1;
+        const long long dims[2] = {wt_ld, g.Ci};
+        const int box[2] = {CB, a.BN}, es[2] = {1, 1};
+        s = make_map(&a.mapB, Wt, 2, dims, wt_ld, box, es, a.row_bytes);
+        if (s != PPO_OK) return s;
         a.ncls = 1;
         KClass &k = a.cls[0];
-        k.o_oy = k.o_ox = 0;
+        k.b_row0 = 0;
         k.taps.n = 1;
         k.taps.dy[0] = k.taps.dx[0] = 0;
         k.taps.wt[0] = 0;
         return launch_kmajor(a, st);
     }
-    // One class per stride parity (ih % 2, iw % 2): inside a class every input pixel sees the same kernel
-    // taps, kh = (ph + pad) mod 2, +2, ..., each reading output row (ih + pad - kh) / 2 = y + (ph + pad - kh) / 2.
-    a.ncls = 0;
-    for (int ph = 0; ph < 2; ++ph)
-        for (int pw = 0; pw < 2; ++pw) {
-            KClass &k = a.cls[a.ncls++];
-            k.o_oy = ph;
-            k.o_ox = pw;
-            int nt = 0;
-            for (int kh = (ph + g.pad) & 1; kh < g.k; kh += 2)
-                for (int kw = (pw + g.pad) & 1; kw < g.k; kw += 2) {
-                    k.taps.dy[nt] = (signed char)((ph + g.pad - kh) / 2);
-                    k.taps.dx[nt] = (signed char)((pw + g.pad - kw) / 2);
-                    k.taps.wt[nt] = (short)(kh * g.k + kw);
-                    ++nt;
+    int dmin, n1;
+    tma_dgrad_shifts(g.k, &dmin, &n1);
+    const int nshift = n1 * n1, Ntot = 4 * g.Ci;
+    a.BN = pick_bn(Ntot);
+    if (Ntot % a.BN != 0 || Ntot / a.BN > 4 || nshift > kMaxTaps) return PPO_ERR_UNSUPPORTED;
+    a.N = a.BN;  // every group is one full tile of columns
+    a.nq_ci = g.Ci;
+    a.wtaps = nshift;
+    {
+        const long long dims[2] = {(long long)nshift * wt_ld, Ntot};
+        const int box[2] = {CB, a.BN}, es[2] = {1, 1};
+        s = make_map(&a.mapB, Wc, 2, dims, (long long)nshift * wt_ld, box, es, a.row_bytes);
+        if (s != PPO_OK) return s;
+    }
+    a.ncls = Ntot / a.BN;
+    for (int c = 0; c < a.ncls; ++c) {
+        KClass &k = a.cls[c];
+        k.b_row0 = c * a.BN;
+        const int q_lo = c * a.BN / g.Ci, q_hi = ((c + 1) * a.BN - 1) / g.Ci;
+        int nt = 0;
+        for (int sy = 0; sy < n1; ++sy)
+            for (int sx = 0; sx < n1; ++sx) {
+                bool used = false;
+                for (int q = q_lo; q <= q_hi; ++q) {
+                    const int kh = (q >> 1) + g.pad - 2 * (dmin + sy), kw = (q & 1) + g.pad - 2 * (dmin + sx);
+                    used = used || (kh >= 0 && kh < g.k && kw >= 0 && kw < g.k);
                 }
-            if (nt == 0) return PPO_ERR_UNSUPPORTED;
-            k.taps.n = nt;
-        }
+                if (!used) continue;
+                k.taps.dy[nt] = (signed char)(dmin + sy);
+                k.taps.dx[nt] = (signed char)(dmin + sx);
+                k.taps.wt[nt] = (short)(sy * n1 + sx);
+                ++nt;
+            }
+        if (nt == 0) return PPO_ERR_UNSUPPORTED;
+        k.taps.n = nt;
+    }
     return launch_kmajor(a, st);
+}
+
+size_t tma_dgrad_weight_elems(int Ci, int k, int wt_ld) {
+    int dmin, n1;
+    tma_dgrad_shifts(k, &dmin, &n1);
+    return (size_t)4 * Ci * n1 * n1 * wt_ld;
+}
+
+// Wc[class * Ci + ci][shift][co (row stride ld)] = W[co][kh][kw][ci] with kh = ph + pad - 2 dy, kw = pw + pad - 2 dx
+// when that tap exists, else 0.
+__global__ void __launch_bounds__(256) dgrad_weights_kernel(const bf16 *__restrict__ W, bf16 *__restrict__ Wc, int Co,
+                                                            int k, int Ci, int ld, int dmin, int n1) {
+    const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    const long long total = (long long)4 * Ci * n1 * n1 * ld;
+    if (i >= total) return;
+    const int co = (int)(i % ld);
+    long long r = i / ld;
+    const int sh = (int)(r % (n1 * n1));
+    r /= n1 * n1;
+    const int ci = (int)(r % Ci), q = (int)(r / Ci);
+    const int pad = k / 2;
+    const int kh = (q >> 1) + pad - 2 * (dmin + sh / n1), kw = (q & 1) + pad - 2 * (dmin + sh % n1);
+    const bool v = co < Co && kh >= 0 && kh < k && kw >= 0 && kw < k;
+    Wc[i] = v ? W[(((size_t)co * k + kh) * k + kw) * Ci + ci] : __float2bfloat16_rn(0.f);
+}
+
+int tma_dgrad_weights(const bf16 *W, bf16 *Wc, int Co, int k, int Ci, int wt_ld, cudaStream_t st) {
+    int dmin, n1;
+    tma_dgrad_shifts(k, &dmin, &n1);
+    const long long total = (long long)tma_dgrad_weight_elems(Ci, k, wt_ld);
+    dgrad_weights_kernel<<<ppo_cdiv(total, 256), 256, 0, st>>>(W, Wc, Co, k, Ci, wt_ld, dmin, n1);
+    PPO_LAUNCH_CHECK();
+    return PPO_OK;
 }
 
 int tma_gemm_wgrad(const ConvGeom &g, const bf16 *dY, int ldy, const bf16 *X, float *dW, int32_t *status,

@@ -5,6 +5,7 @@
 #include <new>
 
 #include "common.cuh"
+#include "gemm.cuh"
 
 static int conv_out(int in, int k) { return (in + 2 * (k / 2) - k) / 2 + 1; }
 
@@ -70,6 +71,13 @@ extern "C" int ppo_model_create(const ppo_model_desc *d, ppo_model **out) {
         for (int l = 1; l <= m->F + 1; ++l)
             tpush(2 * m->L + 2 * (l - 1), m->hw[l - 1], 1, l <= m->F ? m->hw[l] : d->A + 1);
         m->wT_elems = (size_t)toff;
+        int64_t coff = 0;
+        for (int l = 0; l <= PPO_MAX_CONV; ++l) m->wC_off[l] = 0;
+        for (int l = 2; l <= m->L; ++l) {
+            m->wC_off[l] = coff;
+            coff += ((int64_t)tma_dgrad_weight_elems(m->Cs[l - 1], d->conv_k[l - 1], (m->Cs[l] + 7) / 8 * 8) + 63) / 64 * 64;
+        }
+        m->wC_elems = (size_t)coff;
     }
     m->master = m->grad = m->adam_m = m->adam_v = nullptr;
     m->shadow = nullptr;
@@ -129,6 +137,8 @@ static size_t carve(ppo_model *m, const ppo_model *shape, int mb, char *base) {
         if (m) m->dh0_f32 = (float *)f;
         char *w = take(shape->wT_elems * sizeof(bf16));
         if (m) m->wT = (bf16 *)w;
+        char *wc = take(shape->wC_elems * sizeof(bf16));
+        if (m) m->wC = (bf16 *)wc;
         int blocks = ppo_cdiv(mb, kLossThreads);
         char *lp = take((size_t)blocks * 32 * sizeof(float));
         if (m) { m->loss_partials = (float *)lp; m->loss_partial_blocks = blocks; }
