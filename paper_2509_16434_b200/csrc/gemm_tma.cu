@@ -205,6 +205,7 @@ struct PipeK {
     Box boxes[kMaxBoxes];
     uint32_t wtab[4][kMaxWtab];  // resident weights: (byte offset >> 4) of the box that sub-block q of a class reads
     alignas(16) float bias[kMaxBias];
+    uint4 stage[kEpiWarps][32 * 4];  // per epilogue warp: 32 rows x 32 bf16 columns, 16-byte pieces swizzled
 };
 
 __global__ void __launch_bounds__(kKThreads, 1) tma_kmajor_kernel(const __grid_constant__ KArgs a) {
@@ -414,30 +415,113 @@ __global__ void __launch_bounds__(kKThreads, 1) tma_kmajor_kernel(const __grid_c
                 return pix_ok && oy < a.Hout && ox < a.Wout;
             };
             const int ncol = a.nq_ci ? a.nq_ci : a.N;  // columns of an output row
-            // the ReLU mask of this warp's first two chunks is fetched before the accumulator is waited for,
-            // so that its memory latency overlaps the tile's MMAs
-            uint4 mpre[2][2];
             const bool use_mask = a.mode == EPI_DGRAD && a.mask != nullptr;
-            if (use_mask) {
+            const int acc = ti & (nacc - 1);
+            const uint32_t lane_base = tmem_base + acc * acc_cols + ((uint32_t)(lg * 32) << 16);
+            if (a.out != nullptr && a.out_f32 == nullptr && a.mode != EPI_HEAD) {
+                // ---- bf16 outputs, staged: a thread owns a pixel (its TMEM lane), but a warp that stores 32
+                // pixels with one instruction touches 32 cache lines.  So 32-column groups pass through a small
+                // swizzled shared-memory tile: four lanes then move one pixel's 64 contiguous bytes, and an
+                // instruction covers 8 lines.  The ReLU mask comes in the same way, and the first group's mask
+                // is fetched before the accumulator is waited for, so that its latency overlaps the MMAs.
+                uint4 *stg = pipe->stage[warp - 2];
+                const int sw = (lane >> 1) & 3;
+                const int rr0 = lane >> 2, piece = lane & 3;
+                // this warp's groups: columns half * 32 + 64 g; at most 4 (BN <= 256)
+                int ng = 0;
+                for (int c0 = half * 32; c0 < BN && n0 + c0 < a.N; c0 += 64) ++ng;
+                uint4 mreg[4][4];
+                if (use_mask) {
 #pragma unroll
-                for (int j = 0; j < 2; ++j) {
-                    const int c0 = half * 16 + j * 32;
-                    long long orow;
-                    int col;
-                    if (c0 < BN && n0 + c0 < a.N && locate(c0, orow, col)) {
-                        const uint4 *mp = reinterpret_cast<const uint4 *>(a.mask + orow * a.ldo + col);
-                        mpre[j][0] = mp[0];
-                        if (col + 8 < ncol) mpre[j][1] = mp[1];
+                    for (int g = 0; g < 4; ++g) {
+                        if (g < ng) {
+                            long long orow;
+                            int col;
+                            const int okr = locate(half * 32 + 64 * g, orow, col) ? 1 : 0;
+#pragma unroll
+                            for (int ps = 0; ps < 4; ++ps) {
+                                const int rr = ps * 8 + rr0;
+                                const long long o_r = __shfl_sync(0xffffffffu, orow, rr);
+                                const int ok_r = __shfl_sync(0xffffffffu, okr, rr);
+                                mreg[g][ps] = make_uint4(0, 0, 0, 0);
+                                if (ok_r && col + piece * 8 < ncol)
+                                    mreg[g][ps] = *reinterpret_cast<const uint4 *>(a.mask + o_r * a.ldo + col + piece * 8);
+                            }
+                        }
                     }
                 }
+                ok = mbar_wait(&pipe->tfull[acc], (ti >> nacc_log) & 1, abort_flag, a.status);
+                if (!ok) break;
+                tc_fence_after();
+#pragma unroll
+                for (int g = 0; g < 4; ++g) {
+                    if (g >= ng) break;
+                    const int c0 = half * 32 + 64 * g;
+                    float v[32];
+                    tmem_ld16(lane_base + (uint32_t)c0, v);
+                    if (c0 + 16 < BN) tmem_ld16(lane_base + (uint32_t)c0 + 16u, v + 16);
+                    long long orow;
+                    int col;
+                    const int okr = locate(c0, orow, col) ? 1 : 0;
+                    if (a.mode == EPI_FWD) {
+                        const float4 *bp = reinterpret_cast<const float4 *>(pipe->bias + n0 + c0);
+#pragma unroll
+                        for (int q = 0; q < 8; ++q) {
+                            const float4 bv = bp[q];
+                            v[4 * q] += bv.x; v[4 * q + 1] += bv.y; v[4 * q + 2] += bv.z; v[4 * q + 3] += bv.w;
+                        }
+                        if (a.relu) {
+#pragma unroll
+                            for (int i = 0; i < 32; ++i) v[i] = fmaxf(v[i], 0.f);
+                        }
+                    } else if (use_mask) {
+#pragma unroll
+                        for (int ps = 0; ps < 4; ++ps) {
+                            const int rr = ps * 8 + rr0;
+                            stg[rr * 4 + (piece ^ ((rr >> 1) & 3))] = mreg[g][ps];
+                        }
+                        __syncwarp();
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            const uint4 mk = stg[lane * 4 + (j ^ sw)];
+                            const __nv_bfloat162 *m2 = reinterpret_cast<const __nv_bfloat162 *>(&mk);
+#pragma unroll
+                            for (int i = 0; i < 4; ++i) {
+                                const float2 f = __bfloat1622float2(m2[i]);
+                                if (!(f.x > 0.f)) v[j * 8 + 2 * i] = 0.f;
+                                if (!(f.y > 0.f)) v[j * 8 + 2 * i + 1] = 0.f;
+                            }
+                        }
+                        __syncwarp();
+                    }
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        __nv_bfloat162 pk[4];
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) pk[i] = __floats2bfloat162_rn(v[j * 8 + 2 * i], v[j * 8 + 2 * i + 1]);
+                        stg[lane * 4 + (j ^ sw)] = *reinterpret_cast<uint4 *>(pk);
+                    }
+                    __syncwarp();
+#pragma unroll
+                    for (int ps = 0; ps < 4; ++ps) {
+                        const int rr = ps * 8 + rr0;
+                        const long long o_r = __shfl_sync(0xffffffffu, orow, rr);
+                        const int ok_r = __shfl_sync(0xffffffffu, okr, rr);
+                        if (ok_r && col + piece * 8 < ncol && c0 + piece * 8 < BN)
+                            *reinterpret_cast<uint4 *>(a.out + o_r * a.ldo + col + piece * 8) =
+                                stg[rr * 4 + (piece ^ ((rr >> 1) & 3))];
+                    }
+                    __syncwarp();
+                }
+                tc_fence_before();
+                mbar_arrive(&pipe->tempty[acc]);
+                continue;
             }
-            const int acc = ti & (nacc - 1);
+            // ---- head and fp32 outputs (small): every thread stores its own row
             ok = mbar_wait(&pipe->tfull[acc], (ti >> nacc_log) & 1, abort_flag, a.status);
             if (!ok) break;
             tc_fence_after();
-            const uint32_t lane_base = tmem_base + acc * acc_cols + ((uint32_t)(lg * 32) << 16);
-            int chunk = 0;
-            for (int c0 = half * 16; c0 < BN; c0 += 32, ++chunk) {
+            for (int c0 = half * 16; c0 < BN; c0 += 32) {
                 if (n0 + c0 >= a.N) break;  // uniform across the warp
                 float v[16];
                 tmem_ld16(lane_base + (uint32_t)c0, v);
@@ -452,23 +536,12 @@ __global__ void __launch_bounds__(kKThreads, 1) tma_kmajor_kernel(const __grid_c
                     }
                     continue;
                 }
-                if (a.mode == EPI_FWD) {
-                    const float4 *bp = reinterpret_cast<const float4 *>(pipe->bias + nn);
-#pragma unroll
-                    for (int q = 0; q < 4; ++q) {
-                        const float4 bv = bp[q];
-                        v[4 * q] += bv.x; v[4 * q + 1] += bv.y; v[4 * q + 2] += bv.z; v[4 * q + 3] += bv.w;
-                    }
-                    if (a.relu) {
-#pragma unroll
-                        for (int i = 0; i < 16; ++i) v[i] = fmaxf(v[i], 0.f);
-                    }
-                } else if (use_mask) {
+                if (use_mask) {
                     const uint4 *mp = reinterpret_cast<const uint4 *>(a.mask + orow * a.ldo + nn);
 #pragma unroll
                     for (int hlf = 0; hlf < 2; ++hlf) {
                         if (nn + hlf * 8 < ncol) {
-                            const uint4 mk = chunk == 0 ? mpre[0][hlf] : (chunk == 1 ? mpre[1][hlf] : mp[hlf]);
+                            const uint4 mk = mp[hlf];
                             const __nv_bfloat162 *m2 = reinterpret_cast<const __nv_bfloat162 *>(&mk);
 #pragma unroll
                             for (int i = 0; i < 4; ++i) {
@@ -476,19 +549,6 @@ __global__ void __launch_bounds__(kKThreads, 1) tma_kmajor_kernel(const __grid_c
                                 if (!(f.x > 0.f)) v[hlf * 8 + 2 * i] = 0.f;
                                 if (!(f.y > 0.f)) v[hlf * 8 + 2 * i + 1] = 0.f;
                             }
-                        }
-                    }
-                }
-                if (a.out) {
-                    uint4 *op = reinterpret_cast<uint4 *>(a.out + orow * a.ldo + nn);
-#pragma unroll
-                    for (int hlf = 0; hlf < 2; ++hlf) {
-                        if (nn + hlf * 8 < ncol) {
-                            __nv_bfloat162 pk[4];
-#pragma unroll
-                            for (int i = 0; i < 4; ++i)
-                                pk[i] = __floats2bfloat162_rn(v[hlf * 8 + 2 * i], v[hlf * 8 + 2 * i + 1]);
-                            op[hlf] = *reinterpret_cast<uint4 *>(pk);
                         }
                     }
                 }
@@ -928,7 +988,8 @@ int tma_gemm_dgrad(const ConvGeom &g, const bf16 *dY, int ldy, const bf16 *Wt, i
                    const DgradEpilogue &e, int32_t *status, cudaStream_t st) {
     if (!status || g.Ci % 8 != 0 || ldy % 8 != 0 || wt_ld % 8 != 0 || ldy < wt_ld) return PPO_ERR_UNSUPPORTED;
     const bool flat = is_flat(g);
-    if (!flat && (g.k < 3 || g.Hi < 2 || g.Wi < 2 || !Wc || g.Ci % 16 != 0)) return PPO_ERR_UNSUPPORTED;
+    // a 32-column group of the staged epilogue must lie inside one parity class
+    if (!flat && (g.k < 3 || g.Hi < 2 || g.Wi < 2 || !Wc || g.Ci % 32 != 0)) return PPO_ERR_UNSUPPORTED;
     const int CB = channels_per_box(g.Co, flat);
     if (CB == 0 || g.taps() > kMaxTaps || wt_ld < g.Co) return PPO_ERR_UNSUPPORTED;
     KArgs a = {};
