@@ -246,6 +246,11 @@ int ppo_encoder_bwd(ppo_model *m, const ppo_minibatch *mb, int row0, int rows, c
  * activations between ppo_encoder_fwd and ppo_encoder_bwd. */
 int ppo_model_activation_ptr(const ppo_model *m, int kind, int index, void **dev_ptr, size_t *elems);
 
+/* Recomputes the one-bit-per-element ReLU gates the backward pass reads from the saved conv activations of
+ * the first `rows` rows.  ppo_encoder_fwd keeps them up to date itself; call this only after writing saved
+ * activations from outside (see ppo_model_activation_ptr) and before ppo_encoder_bwd. */
+int ppo_model_sync_masks(ppo_model *m, int rows, void *stream);
+
 /* Zeroes the bound gradient array (start of a minibatch). */
 int ppo_model_zero_grad(ppo_model *m, void *stream);
 

@@ -27,6 +27,7 @@ EXPORTS = [
     "ppo_model_num_tensors", "ppo_model_tensor_info", "ppo_model_workspace_bytes", "ppo_model_bind",
     "ppo_model_sync_shadow", "ppo_encoder_fwd", "ppo_loss_fwd_bwd", "ppo_encoder_bwd", "ppo_model_zero_grad",
     "ppo_adam_step", "ppo_policy_sample", "ppo_poll_status", "ppo_model_activation_ptr", "ppo_gae_static",
+    "ppo_model_sync_masks",
 ]
 
 
@@ -87,6 +88,7 @@ def lib():
         L.ppo_model_bind.argtypes = [C.c_void_p] * 7 + [C.c_size_t, C.c_int]
         L.ppo_model_sync_shadow.argtypes = [C.c_void_p, C.c_void_p]
         L.ppo_model_zero_grad.argtypes = [C.c_void_p, C.c_void_p]
+        L.ppo_model_sync_masks.argtypes = [C.c_void_p, C.c_int, C.c_void_p]
         L.ppo_encoder_fwd.argtypes = [C.c_void_p, C.POINTER(Minibatch), C.c_int, C.c_int, C.c_void_p, C.c_void_p,
                                       C.c_void_p]
         L.ppo_loss_fwd_bwd.argtypes = [C.c_void_p, C.POINTER(Minibatch), C.c_int, C.c_int, C.c_int, C.c_void_p,
@@ -305,6 +307,10 @@ class Model:
 
 def ppo_model_sync_shadow(m: Model, stream=None):
     _check(lib().ppo_model_sync_shadow(m.handle, _stream(stream)), "ppo_model_sync_shadow")
+
+
+def ppo_model_sync_masks(m: Model, rows: int, stream=None):
+    _check(lib().ppo_model_sync_masks(m.handle, rows, _stream(stream)), "ppo_model_sync_masks")
 
 
 def ppo_model_zero_grad(m: Model, stream=None):

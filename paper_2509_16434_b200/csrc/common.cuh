@@ -65,6 +65,7 @@ struct ppo_model {
     // workspace carve
     bf16 *act[PPO_MAX_CONV + 1];   // act[l], l >= 1: [mb][Ho][Wo][C] post-ReLU
     bf16 *dact[PPO_MAX_CONV + 1];  // gradient w.r.t. the pre-activation of act[l]
+    uint32_t *abits[PPO_MAX_CONV + 1];  // ReLU gate of act[l], one bit per element (layers with C % 32 == 0, else null)
     bf16 *h[PPO_MAX_FC + 1];       // h[0] = [pooled, proprio]; h[l] post-ReLU
     bf16 *dh[PPO_MAX_FC + 2];      // dh[l]: gradient w.r.t. pre-activation of h[l]; dh[F+1]: head dout padded to 16
     float *dh0_f32;                // gradient w.r.t. h[0] (pooled part feeds the un-pool)

@@ -14,8 +14,8 @@
 template <int KS, bool STAGE>
 __global__ void __launch_bounds__(128) conv1_fwd_kernel(const __half *__restrict__ depth,
                                                         const bf16 *__restrict__ W, const float *__restrict__ bias,
-                                                        bf16 *__restrict__ out, int rows, int Hi, int Wi, int Ho,
-                                                        int Wo, int C1) {
+                                                        bf16 *__restrict__ out, uint32_t *__restrict__ bits,
+                                                        int rows, int Hi, int Wi, int Ho, int Wo, int C1) {
     extern __shared__ __align__(16) float sm[];  // w[tap][co], then bias[co], then (STAGE) 4 warps x 32 pixels x C1 bf16
     float *w = sm, *bs = sm + KS * KS * C1;
     for (int i = threadIdx.x; i < KS * KS * C1; i += blockDim.x) {
@@ -50,6 +50,7 @@ __global__ void __launch_bounds__(128) conv1_fwd_kernel(const __half *__restrict
     uint4 *stage = reinterpret_cast<uint4 *>(bs + C1) + (size_t)warp * 32 * CH;
     const int sh = CH == 8 ? 0 : (CH == 4 ? 1 : (CH == 2 ? 2 : 3));
     uint4 *o = reinterpret_cast<uint4 *>(out + m * C1);
+    uint32_t gate = 0;  // ReLU gate bits of the current 32 channels
     for (int c8 = 0; c8 < C1; c8 += 8) {
         float acc[8];
         {
@@ -70,6 +71,14 @@ __global__ void __launch_bounds__(128) conv1_fwd_kernel(const __half *__restrict
         __nv_bfloat162 p[4];
 #pragma unroll
         for (int j = 0; j < 4; ++j) p[j] = __floats2bfloat162_rn(fmaxf(acc[2 * j], 0.f), fmaxf(acc[2 * j + 1], 0.f));
+        if (bits) {
+#pragma unroll
+            for (int j = 0; j < 8; ++j) gate |= (acc[j] > 0.f ? 1u : 0u) << ((c8 & 31) + j);
+            if ((c8 & 31) == 24) {
+                if (live) bits[m * (C1 >> 5) + (c8 >> 5)] = gate;
+                gate = 0;
+            }
+        }
         if (STAGE) stage[lane * CH + ((c8 >> 3) ^ ((lane >> sh) & (CH - 1)))] = *reinterpret_cast<uint4 *>(p);
         else if (live) o[c8 >> 3] = *reinterpret_cast<uint4 *>(p);
     }
@@ -197,6 +206,37 @@ __global__ void __launch_bounds__(128) conv1_wgrad_kernel(const __half *__restri
 }
 
 // ------------------------------------------------------------- small kernels ----
+
+// One thread per 32 channels of a pixel: the ReLU gate (act > 0) as a bit mask.
+__global__ void __launch_bounds__(256) relu_bits_kernel(const bf16 *__restrict__ act, uint32_t *__restrict__ bits,
+                                                        long long words) {
+    const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= words) return;
+    const uint4 *p = reinterpret_cast<const uint4 *>(act + i * 32);
+    uint32_t w = 0;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        const uint4 r = p[j];
+        const __nv_bfloat162 *h2 = reinterpret_cast<const __nv_bfloat162 *>(&r);
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const float2 f = __bfloat1622float2(h2[q]);
+            w |= (f.x > 0.f ? 1u : 0u) << (j * 8 + 2 * q);
+            w |= (f.y > 0.f ? 1u : 0u) << (j * 8 + 2 * q + 1);
+        }
+    }
+    bits[i] = w;
+}
+
+int relu_bits(const bf16 *act, uint32_t *bits, long long M, int C, cudaStream_t st) {
+    if (C % 32 != 0) return PPO_ERR_UNSUPPORTED;
+    const long long words = M * (C / 32);
+    if (words <= 0) return PPO_OK;
+    relu_bits_kernel<<<ppo_cdiv(words, 256), 256, 0, st>>>(act, bits, words);
+    PPO_LAUNCH_CHECK();
+    return PPO_OK;
+}
+
 
 // h0[b] = [mean over pixels of act[b][px][c], proprio[b]] as bf16.  One warp per row b; a lane
 // owns 8 channels at a time so that every pixel is read with 128-bit loads.
@@ -361,10 +401,15 @@ static ConvGeom fc_geom(int rows, int in, int out) {
 
 static int run_fwd(const ppo_model *m, const ConvGeom &g, const bf16 *X, const bf16 *W, const FwdEpilogue &e,
                    cudaStream_t st) {
-    if (m->impl == 1) return simt_gemm_fwd(g, X, W, e, st);
-    const int s = tma_gemm_fwd(g, X, W, e, ppo_device_status_ptr(), st);
+    if (m->impl == 1) {
+        const int s = simt_gemm_fwd(g, X, W, e, st);
+        return (s == PPO_OK && e.out_bits) ? relu_bits(e.out, e.out_bits, g.M(), g.Co, st) : s;
+    }
+    int s = tma_gemm_fwd(g, X, W, e, ppo_device_status_ptr(), st);  // writes e.out_bits itself
     if (s != PPO_ERR_UNSUPPORTED) return s;
-    return tc_gemm_fwd(g, X, W, e, ppo_device_status_ptr(), st);
+    s = tc_gemm_fwd(g, X, W, e, ppo_device_status_ptr(), st);
+    if (s == PPO_OK && e.out_bits) s = relu_bits(e.out, e.out_bits, g.M(), g.Co, st);
+    return s;
 }
 
 static int run_dgrad(const ppo_model *m, const ConvGeom &g, const bf16 *dY, int ldy, const bf16 *W, const bf16 *Wt,
@@ -441,10 +486,10 @@ extern "C" int ppo_encoder_fwd(ppo_model *m, const ppo_minibatch *mb, int row0, 
 #define PPO_CONV1(KS_)                                                                                              \
     do {                                                                                                            \
         if (stage)                                                                                                  \
-            conv1_fwd_kernel<KS_, true><<<blocks, 128, smem, st>>>(depth, W, bias, m->act[1], rows, d.H, d.W,       \
+            conv1_fwd_kernel<KS_, true><<<blocks, 128, smem, st>>>(depth, W, bias, m->act[1], m->abits[1], rows, d.H, d.W,       \
                                                                    m->Hs[1], m->Ws[1], C1);                         \
         else                                                                                                        \
-            conv1_fwd_kernel<KS_, false><<<blocks, 128, smem, st>>>(depth, W, bias, m->act[1], rows, d.H, d.W,      \
+            conv1_fwd_kernel<KS_, false><<<blocks, 128, smem, st>>>(depth, W, bias, m->act[1], m->abits[1], rows, d.H, d.W,      \
                                                                     m->Hs[1], m->Ws[1], C1);                        \
     } while (0)
         if (KS == 1) PPO_CONV1(1);
@@ -457,6 +502,7 @@ extern "C" int ppo_encoder_fwd(ppo_model *m, const ppo_minibatch *mb, int row0, 
     for (int l = 2; l <= m->L; ++l) {
         ConvGeom g = conv_geom(m, l, rows);
         FwdEpilogue e = {m->master + m->tensors[2 * (l - 1) + 1].off, 1, m->act[l], nullptr, nullptr, 0};
+        e.out_bits = m->abits[l];
         PPO_TRY(run_fwd(m, g, m->act[l - 1], m->shadow + m->tensors[2 * (l - 1)].off, e, st));
     }
     pool_concat_kernel<<<ppo_cdiv(rows, 8), 256, 0, st>>>(m->act[m->L], mb->proprio + (size_t)row0 * d.P, m->h[0], rows,
@@ -546,6 +592,7 @@ extern "C" int ppo_encoder_bwd(ppo_model *m, const ppo_minibatch *mb, int row0, 
         PPO_TRY(run_wgrad(m, g, m->dact[l], g.Co, m->act[l - 1], m->grad + m->tensors[ti].off, st));
         PPO_TRY(run_colsum(m->dact[l], g.Co, g.M(), g.Co, m->grad + m->tensors[ti + 1].off, st));
         DgradEpilogue e = {m->act[l - 1], m->dact[l - 1], nullptr};
+        e.mask_bits = m->abits[l - 1];
         PPO_TRY(run_dgrad(m, g, m->dact[l], g.Co, m->shadow + m->tensors[ti].off, m->wT + m->wT_off[ti],
                           wt_ld_of(g.Co), m->wC + m->wC_off[l], e, st));
     }

@@ -14,12 +14,15 @@ struct FwdEpilogue {
     float *out_mean;    // head: columns 0..A-1 -> [M][A]
     float *out_value;   // head: column A -> [M]
     int A;
+    uint32_t *out_bits = nullptr;  // optional: gate bits (out > 0) of a ReLU output, [M][Co / 32]; needs Co % 32 == 0
 };
 
 struct DgradEpilogue {
     const bf16 *mask_act;  // [M'][Ci]: output is zeroed where this is <= 0; may be nullptr
     bf16 *out;             // [M'][Ci] bf16, or nullptr
     float *out_f32;        // [M'][Ci] fp32, or nullptr
+    const uint32_t *mask_bits = nullptr;  // the same gate as one bit per element, [M'][Ci / 32] (bit c % 32 of word c / 32);
+                                          // used instead of mask_act by kernels that support it
 };
 
 // ldy: row stride (elements) of Y / dY (>= Co).  wt_ld: row stride of the innermost (co)
@@ -49,3 +52,6 @@ size_t tma_dgrad_weight_elems(int Ci, int k, int wt_ld);
 int tma_dgrad_weights(const bf16 *W, bf16 *Wc, int Co, int k, int Ci, int wt_ld, cudaStream_t st);
 int tma_gemm_wgrad(const ConvGeom &g, const bf16 *dY, int ldy, const bf16 *X, float *dW, int32_t *status,
                    cudaStream_t st);
+
+// bits[m][c / 32] bit (c % 32) = act[m][c] > 0, for C a multiple of 32.
+int relu_bits(const bf16 *act, uint32_t *bits, long long M, int C, cudaStream_t st);

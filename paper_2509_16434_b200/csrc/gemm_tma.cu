@@ -188,6 +188,8 @@ struct KArgs {
     bf16 *out;
     float *out_f32;
     const bf16 *mask;
+    const uint32_t *mask_bits;  // merged dgrad: the gate as bits, [pixels][nq_ci / 32]
+    uint32_t *out_bits;         // forward: gate bits of the ReLU output, [pixels][N / 32]
     float *mean, *value;
     int32_t *status;
     KClass cls[4];
@@ -415,7 +417,8 @@ __global__ void __launch_bounds__(kKThreads, 1) tma_kmajor_kernel(const __grid_c
                 return pix_ok && oy < a.Hout && ox < a.Wout;
             };
             const int ncol = a.nq_ci ? a.nq_ci : a.N;  // columns of an output row
-            const bool use_mask = a.mode == EPI_DGRAD && a.mask != nullptr;
+            const bool use_bits = a.mode == EPI_DGRAD && a.mask_bits != nullptr;
+            const bool use_mask = a.mode == EPI_DGRAD && a.mask != nullptr && !use_bits;
             const int acc = ti & (nacc - 1);
             const uint32_t lane_base = tmem_base + acc * acc_cols + ((uint32_t)(lg * 32) << 16);
             if (a.out != nullptr && a.out_f32 == nullptr && a.mode != EPI_HEAD) {
@@ -431,6 +434,17 @@ __global__ void __launch_bounds__(kKThreads, 1) tma_kmajor_kernel(const __grid_c
                 int ng = 0;
                 for (int c0 = half * 32; c0 < BN && n0 + c0 < a.N; c0 += 64) ++ng;
                 uint4 mreg[4][4];
+                uint32_t gbits[4] = {0u, 0u, 0u, 0u};
+                if (use_bits) {
+#pragma unroll
+                    for (int g = 0; g < 4; ++g) {
+                        if (g < ng) {
+                            long long orow;
+                            int col;
+                            if (locate(half * 32 + 64 * g, orow, col)) gbits[g] = a.mask_bits[orow * (ncol >> 5) + (col >> 5)];
+                        }
+                    }
+                }
                 if (use_mask) {
 #pragma unroll
                     for (int g = 0; g < 4; ++g) {
@@ -474,6 +488,16 @@ __global__ void __launch_bounds__(kKThreads, 1) tma_kmajor_kernel(const __grid_c
 #pragma unroll
                             for (int i = 0; i < 32; ++i) v[i] = fmaxf(v[i], 0.f);
                         }
+                        if (a.out_bits && okr) {
+                            uint32_t w = 0;
+#pragma unroll
+                            for (int i = 0; i < 32; ++i) w |= (v[i] > 0.f ? 1u : 0u) << i;
+                            a.out_bits[orow * (a.N >> 5) + (col >> 5)] = w;
+                        }
+                    } else if (use_bits) {
+#pragma unroll
+                        for (int i = 0; i < 32; ++i)
+                            if (!((gbits[g] >> i) & 1u)) v[i] = 0.f;
                     } else if (use_mask) {
 #pragma unroll
                         for (int ps = 0; ps < 4; ++ps) {
@@ -957,6 +981,8 @@ int tma_gemm_fwd(const ConvGeom &g, const bf16 *X, const bf16 *W, const FwdEpilo
     a.bias = e.bias;
     a.out = e.out;
     a.mean = e.out_mean;
+    a.out_bits = (e.out_bits && e.relu && g.Co % 32 == 0) ? e.out_bits : nullptr;
+    if (e.out_bits && !a.out_bits) return PPO_ERR_UNSUPPORTED;
     a.value = e.out_value;
     a.status = status;
     if (a.mode == EPI_FWD && g.Co % 8 != 0) return PPO_ERR_UNSUPPORTED;
@@ -1011,6 +1037,7 @@ int tma_gemm_dgrad(const ConvGeom &g, const bf16 *dY, int ldy, const bf16 *Wt, i
     a.out = e.out;
     a.out_f32 = e.out_f32;
     a.mask = e.mask_act;
+    a.mask_bits = flat ? nullptr : e.mask_bits;
     a.status = status;
     if (flat) {
         a.N = g.Ci;

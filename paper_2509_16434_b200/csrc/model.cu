@@ -124,6 +124,9 @@ static size_t carve(ppo_model *m, const ppo_model *shape, int mb, char *base) {
         size_t bytes = (size_t)mb * shape->Hs[l] * shape->Ws[l] * shape->Cs[l] * sizeof(bf16);
         char *a = take(bytes), *g = take(bytes);
         if (m) { m->act[l] = (bf16 *)a; m->dact[l] = (bf16 *)g; }
+        const bool bits = shape->Cs[l] % 32 == 0 && l < shape->L;  // gate bits for the dgrad of layer l + 1
+        char *bt = bits ? take(bytes / 16) : nullptr;
+        if (m) m->abits[l] = (uint32_t *)bt;
     }
     for (int l = 0; l <= shape->F; ++l) {
         size_t bytes = (size_t)mb * shape->hw[l] * sizeof(bf16);
@@ -186,6 +189,18 @@ extern "C" int ppo_model_activation_ptr(const ppo_model *m, int kind, int index,
         return PPO_OK;
     }
     return PPO_ERR_INVALID_ARG;
+}
+
+extern "C" int ppo_model_sync_masks(ppo_model *m, int rows, void *stream) {
+    if (!m || !m->ws) return PPO_ERR_STATE;
+    if (rows <= 0 || rows > m->mbmax) return PPO_ERR_SHAPE;
+    for (int l = 1; l < m->L; ++l)
+        if (m->abits[l]) {
+            const int s = relu_bits(m->act[l], m->abits[l], (long long)rows * m->Hs[l] * m->Ws[l], m->Cs[l],
+                                    static_cast<cudaStream_t>(stream));
+            if (s != PPO_OK) return s;
+        }
+    return PPO_OK;
 }
 
 // ------------------------------------------------------------ shadow / zero ----

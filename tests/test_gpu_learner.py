@@ -101,6 +101,7 @@ def test_backward_matches_oracle_on_identical_activations(name):
     L.loss.zero_()
     ppo.ppo_encoder_fwd(L.model, L.mb, 0, B, L.mean, L.value)
     _upload_oracle_activations(L, md, acts, B)
+    ppo.ppo_model_sync_masks(L.model, B)
     L.mean[:B].copy_(torch.as_tensor(mu_o, dtype=torch.float32))
     L.value[:B].copy_(torch.as_tensor(V_o, dtype=torch.float32))
     ppo.ppo_loss_fwd_bwd(L.model, L.mb, 0, B, B, L.mean, L.value, h.clip, h.vf_coef, h.ent_coef, L.loss, L.dmean,
