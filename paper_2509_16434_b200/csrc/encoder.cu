@@ -477,6 +477,11 @@ extern "C" int ppo_encoder_fwd(ppo_model *m, const ppo_minibatch *mb, int row0, 
         const __half *depth = static_cast<const __half *>(mb->depth_f16) + (size_t)row0 * d.H * d.W;
         const int C1 = m->Cs[1], KS = d.conv_k[0];
         const long long M = (long long)rows * m->Hs[1] * m->Ws[1];
+        int tcs = PPO_ERR_UNSUPPORTED;
+        if (m->impl == 0)
+            tcs = conv1_tc_fwd(depth, m->shadow + m->tensors[0].off, m->master + m->tensors[1].off, m->act[1], m->abits[1],
+                               rows, d.H, d.W, m->Hs[1], m->Ws[1], C1, KS, ppo_device_status_ptr(), st);
+        if (tcs != PPO_OK && tcs != PPO_ERR_UNSUPPORTED) return tcs;
         const int CH = C1 / 8;
         const bool stage = CH == 1 || CH == 2 || CH == 4 || CH == 8;
         const size_t smem = (size_t)(KS * KS * C1 + C1) * sizeof(float) + (stage ? (size_t)4 * 32 * C1 * 2 : 0);
@@ -492,7 +497,8 @@ extern "C" int ppo_encoder_fwd(ppo_model *m, const ppo_minibatch *mb, int row0, 
             conv1_fwd_kernel<KS_, false><<<blocks, 128, smem, st>>>(depth, W, bias, m->act[1], m->abits[1], rows, d.H, d.W,      \
                                                                     m->Hs[1], m->Ws[1], C1);                        \
     } while (0)
-        if (KS == 1) PPO_CONV1(1);
+        if (tcs == PPO_OK) { /* done on the tensor cores */ }
+        else if (KS == 1) PPO_CONV1(1);
         else if (KS == 3) PPO_CONV1(3);
         else if (KS == 5) PPO_CONV1(5);
         else PPO_CONV1(7);

@@ -55,3 +55,7 @@ int tma_gemm_wgrad(const ConvGeom &g, const bf16 *dY, int ldy, const bf16 *X, fl
 
 // bits[m][c / 32] bit (c % 32) = act[m][c] > 0, for C a multiple of 32.
 int relu_bits(const bf16 *act, uint32_t *bits, long long M, int C, cudaStream_t st);
+
+// First convolution (C_in = 1) as a tensor-core GEMM over thread-built im2col tiles (conv1_tc.cu).
+int conv1_tc_fwd(const __half *depth, const bf16 *W, const float *bias, bf16 *out, uint32_t *bits, int rows, int Hi,
+                 int Wi, int Ho, int Wo, int C1, int ks, int32_t *status, cudaStream_t st);
