@@ -205,6 +205,158 @@ __global__ void __launch_bounds__(128) conv1_wgrad_kernel(const __half *__restri
     }
 }
 
+// The same reduction on the tensor cores (mma.sync m16n8k16, bf16): per 16 output pixels a warp forms
+// D[tap][co] += X^T[tap][px] dZ[px][co] with the pixel index as K.  The 16 x TP patch tile X (k*k depth taps as
+// bf16, then a column of ones whose product is the bias gradient, zero padded to TP) and the 16 x C1 gradient
+// tile go through per-warp shared memory and come back as fragments with ldmatrix.trans.  About 3 instructions
+// per pixel instead of C1 (k*k + 1) / 32 multiply-adds plus their loads: the kernel becomes a stream over dZ.
+// C1 must be a multiple of 16.
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t addr, uint32_t &r0, uint32_t &r1, uint32_t &r2, uint32_t &r3) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
+                 : "r"(addr));
+}
+__device__ __forceinline__ void mma_bf16_16816(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                               uint32_t b0, uint32_t b1) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+        : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+template <int KS, int NB>  // NB = C1 / 8 column blocks
+__global__ void __launch_bounds__(256) conv1_wgrad_mma_kernel(const __half *__restrict__ depth,
+                                                              const bf16 *__restrict__ dZ, float *__restrict__ dW,
+                                                              float *__restrict__ db, int rows, int Hi, int Wi,
+                                                              int Ho, int Wo, long long px_per_warp) {
+    constexpr int K2 = KS * KS, P = KS / 2, TP = (K2 + 1 + 15) / 16 * 16, MB = TP / 16, C1 = NB * 8;
+    constexpr int kXBytes = 16 * TP * 2, kZBytes = 16 * C1 * 2;
+    extern __shared__ __align__(16) uint8_t smw[];  // per warp: X tile [16 px][TP], dZ tile [16 px][C1]; later the reduction
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    uint8_t *xs = smw + (size_t)warp * (kXBytes + kZBytes), *zs = xs + kXBytes;
+    const uint32_t xs_a = (uint32_t)__cvta_generic_to_shared(xs), zs_a = (uint32_t)__cvta_generic_to_shared(zs);
+    float acc[MB][NB][4];
+#pragma unroll
+    for (int i = 0; i < MB; ++i)
+#pragma unroll
+        for (int j = 0; j < NB; ++j)
+#pragma unroll
+            for (int q = 0; q < 4; ++q) acc[i][j][q] = 0.f;
+    const long long M = (long long)rows * Ho * Wo;
+    const long long gw = (long long)blockIdx.x * 8 + warp;
+    long long m0 = gw * px_per_warp;                       // px_per_warp is a multiple of 16
+    const long long m_end = min(M, m0 + px_per_warp);
+    // this lane's pixel of the patch tile: px = lane % 16, taps [half * TP / 2, +TP / 2)
+    const int pxl = lane & 15, half = lane >> 4;
+    int ow = 0, oh = 0;
+    long long b = 0;
+    if (m0 < m_end) {
+        const long long m = m0 + pxl;
+        ow = (int)(m % Wo);
+        const long long t = m / Wo;
+        oh = (int)(t % Ho);
+        b = t / Ho;
+    }
+    const int d_oh = 16 / Wo, d_ow = 16 % Wo;  // 16 pixels further (Wo >= 1)
+    constexpr int ZP = (16 * C1 / 8 + 31) / 32;  // 16-byte pieces of the gradient tile per lane
+    uint4 xreg[TP / 16], zreg[ZP];
+    // Loads of the tile that starts at pixel mt into registers; they are issued one trip ahead, so that their
+    // latency overlaps the previous tile's MMAs.
+    auto prefetch = [&](long long mt) {
+        const bool live = mt + pxl < m_end;
+        const __half *img = depth + b * Hi * Wi;
+#pragma unroll
+        for (int c = 0; c < TP / 16; ++c) {  // 8 taps = one 16-byte piece
+            const int t0 = half * (TP / 2) + c * 8;
+            __nv_bfloat162 pk[4];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                const int tap = t0 + j;
+                float xv = 0.f;
+                if (tap < K2) {
+                    const int kh = tap / KS, kw = tap - kh * KS;
+                    const int ih = 2 * oh + kh - P, iw = 2 * ow + kw - P;
+                    if (live && ih >= 0 && ih < Hi && iw >= 0 && iw < Wi) xv = __half2float(__ldg(img + ih * Wi + iw));
+                } else if (tap == K2) {
+                    xv = live ? 1.f : 0.f;
+                }
+                if (j & 1) pk[j >> 1].y = __float2bfloat16_rn(xv);
+                else pk[j >> 1].x = __float2bfloat16_rn(xv);
+            }
+            xreg[c] = *reinterpret_cast<uint4 *>(pk);
+        }
+#pragma unroll
+        for (int z = 0; z < ZP; ++z) {
+            const int i = lane + 32 * z;
+            zreg[z] = make_uint4(0, 0, 0, 0);
+            if (i < 16 * C1 / 8 && mt + i / (C1 / 8) < m_end) zreg[z] = __ldcs(reinterpret_cast<const uint4 *>(dZ + mt * C1) + i);
+        }
+    };
+    if (m0 < m_end) prefetch(m0);
+    for (; m0 < m_end; m0 += 16) {
+#pragma unroll
+        for (int c = 0; c < TP / 16; ++c)
+            *reinterpret_cast<uint4 *>(xs + pxl * (TP * 2) + (half * (TP / 2) + c * 8) * 2) = xreg[c];
+#pragma unroll
+        for (int z = 0; z < ZP; ++z)
+            if (lane + 32 * z < 16 * C1 / 8) reinterpret_cast<uint4 *>(zs)[lane + 32 * z] = zreg[z];
+        __syncwarp();
+        ow += d_ow;
+        if (ow >= Wo) { ow -= Wo; ++oh; }
+        oh += d_oh;
+        while (oh >= Ho) { oh -= Ho; ++b; }
+        if (m0 + 16 < m_end) prefetch(m0 + 16);
+        // ---- fragments and MMAs
+        uint32_t af[MB][4];
+#pragma unroll
+        for (int i = 0; i < MB; ++i) {
+            // matrices: (taps 16i..+7, px 0-7), (taps 16i+8.., px 0-7), (taps 16i.., px 8-15), (taps 16i+8.., px 8-15)
+            const int mi = lane >> 3, r = lane & 7;
+            const uint32_t addr = xs_a + (uint32_t)((r + (mi >= 2 ? 8 : 0)) * (TP * 2) + (16 * i + (mi & 1) * 8) * 2);
+            ldmatrix_x4_trans(addr, af[i][0], af[i][1], af[i][2], af[i][3]);
+        }
+#pragma unroll
+        for (int j = 0; j < NB; j += 2) {
+            // matrices: (px 0-7, co 8j..), (px 8-15, co 8j..), (px 0-7, co 8j+8..), (px 8-15, co 8j+8..)
+            const int mi = lane >> 3, r = lane & 7;
+            const uint32_t addr = zs_a + (uint32_t)((r + (mi & 1) * 8) * (C1 * 2) + (8 * j + (mi >> 1) * 8) * 2);
+            uint32_t b0, b1, b2, b3;
+            ldmatrix_x4_trans(addr, b0, b1, b2, b3);
+#pragma unroll
+            for (int i = 0; i < MB; ++i) {
+                mma_bf16_16816(acc[i][j], af[i][0], af[i][1], af[i][2], af[i][3], b0, b1);
+                mma_bf16_16816(acc[i][j + 1], af[i][0], af[i][1], af[i][2], af[i][3], b2, b3);
+            }
+        }
+        __syncwarp();
+    }
+    // ---- block reduction: D element (tap = 16 i + g (+8), co = 8 j + 2 c (+1)) -> [TP][C1] floats per warp
+    __syncthreads();
+    float *red = reinterpret_cast<float *>(smw);
+    constexpr int per = TP * C1;
+    {
+        const int g = lane >> 2, c = lane & 3;
+        float *mine = red + (size_t)warp * per;
+#pragma unroll
+        for (int i = 0; i < MB; ++i)
+#pragma unroll
+            for (int j = 0; j < NB; ++j) {
+                mine[(16 * i + g) * C1 + 8 * j + 2 * c] = acc[i][j][0];
+                mine[(16 * i + g) * C1 + 8 * j + 2 * c + 1] = acc[i][j][1];
+                mine[(16 * i + g + 8) * C1 + 8 * j + 2 * c] = acc[i][j][2];
+                mine[(16 * i + g + 8) * C1 + 8 * j + 2 * c + 1] = acc[i][j][3];
+            }
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < (K2 + 1) * C1; i += 256) {
+        float v = 0.f;
+        for (int w = 0; w < 8; ++w) v += red[(size_t)w * per + i];
+        const int tap = i / C1, co = i - tap * C1;
+        if (tap < K2) atomicAdd(dW + co * K2 + tap, v);
+        else atomicAdd(db + co, v);
+    }
+}
+
 // ------------------------------------------------------------- small kernels ----
 
 // One thread per 32 channels of a pixel: the ReLU gate (act > 0) as a bit mask.
@@ -606,6 +758,38 @@ extern "C" int ppo_encoder_bwd(ppo_model *m, const ppo_minibatch *mb, int row0, 
         const __half *depth = static_cast<const __half *>(mb->depth_f16) + (size_t)row0 * d.H * d.W;
         const int C1 = m->Cs[1], KS = d.conv_k[0];
         const long long M = (long long)rows * m->Hs[1] * m->Ws[1];
+        if (m->impl == 0 && C1 % 16 == 0 && C1 <= 64 && (KS == 3 || KS == 5)) {
+            // tensor-core reduction
+            const int TP = (KS * KS + 1 + 15) / 16 * 16;
+            const size_t tile = (size_t)16 * TP * 2 + (size_t)16 * C1 * 2, redb = (size_t)TP * C1 * sizeof(float);
+            const size_t smem = 8 * (tile > redb ? tile : redb);
+            int blocks = ppo_cdiv(M, 8 * 16 * 8);
+            const int cap = ppo_num_sms() * 4;
+            blocks = blocks > cap ? cap : (blocks < 1 ? 1 : blocks);
+            long long per_warp = (M + (long long)blocks * 8 - 1) / ((long long)blocks * 8);
+            per_warp = (per_warp + 15) / 16 * 16;
+            float *dW = m->grad + m->tensors[0].off, *db = m->grad + m->tensors[1].off;
+#define PPO_C1W(KS_, NB_)                                                                                       \
+    do {                                                                                                        \
+        if (smem > 48 * 1024)                                                                                   \
+            PPO_CUDA_CHECK(cudaFuncSetAttribute(conv1_wgrad_mma_kernel<KS_, NB_>,                               \
+                                                cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));       \
+        conv1_wgrad_mma_kernel<KS_, NB_><<<blocks, 256, smem, st>>>(depth, m->dact[1], dW, db, rows, d.H, d.W, \
+                                                                    m->Hs[1], m->Ws[1], per_warp);              \
+    } while (0)
+            const int nb = C1 / 8;
+            if (KS == 3 && nb == 2) PPO_C1W(3, 2);
+            else if (KS == 3 && nb == 4) PPO_C1W(3, 4);
+            else if (KS == 3 && nb == 6) PPO_C1W(3, 6);
+            else if (KS == 3 && nb == 8) PPO_C1W(3, 8);
+            else if (KS == 5 && nb == 2) PPO_C1W(5, 2);
+            else if (KS == 5 && nb == 4) PPO_C1W(5, 4);
+            else if (KS == 5 && nb == 6) PPO_C1W(5, 6);
+            else PPO_C1W(5, 8);
+#undef PPO_C1W
+            PPO_LAUNCH_CHECK();
+            return PPO_OK;
+        }
         const int cpt = KS <= 3 ? 8 : (KS == 5 ? 4 : 2);
         const int lpp = C1 / cpt;
         if (C1 % cpt != 0 || lpp > 32 || (lpp & (lpp - 1)) != 0) return PPO_ERR_UNSUPPORTED;
