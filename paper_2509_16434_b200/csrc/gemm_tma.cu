@@ -38,7 +38,8 @@ constexpr int kMaxHeights = 32;  // one tensor map per box height 1 .. 32 rows (
                                  // so a tile is cut into as few boxes as the image boundaries allow)
 constexpr int kMaxStages = 8;
 constexpr int kThreads = 192;    // warp 0: TMA producer, warp 1: MMA issue and TMEM owner, warps 2-5: epilogue
-constexpr size_t kSmemBudget = 200 * 1024;
+constexpr size_t kSmemBudget = 200 * 1024;  // operand stages of the wgrad kernel
+constexpr size_t kSmemMax = 227 * 1024;     // dynamic shared memory a CTA may ask for
 constexpr size_t kMaxResident = 64 * 1024;
 
 struct Taps {
@@ -163,7 +164,7 @@ struct KClass {
 
 enum { EPI_FWD = 0, EPI_HEAD = 1, EPI_DGRAD = 2 };
 
-constexpr int kEpiWarps = 8;                      // two warps per TMEM lane quarter, alternating 16-column chunks
+constexpr int kEpiWarps = 16;                     // at most: two or four warps per TMEM lane quarter share out the column groups
 constexpr int kKThreads = (2 + kEpiWarps) * 32;   // warp 0: TMA producer, warp 1: MMA issue and TMEM owner
 constexpr int kMaxBias = 512;
 constexpr int kMaxWtab = 64;
@@ -179,6 +180,7 @@ struct KArgs {
     int kchunks;            // boxes along the channels of one tap
     int w_tap;              // elements between taps in a weight row
     int G, nbmax;           // sub-blocks per stage; most A boxes a tile has
+    int nepi;               // epilogue warps: 8, or 16 where the epilogue is the heavier side (dgrad with gate bits)
     int wres, wtaps;        // weights resident in shared memory (all wtaps * kchunks boxes, loaded once)
     int N, BN, tiles_n, total_tiles, ncls, stages;  // tile g = ((mt * tiles_n) + nt) * ncls + class
     int Hout, Wout, ldo;
@@ -207,7 +209,7 @@ struct PipeK {
     Box boxes[kMaxBoxes];
     uint32_t wtab[4][kMaxWtab];  // resident weights: (byte offset >> 4) of the box that sub-block q of a class reads
     alignas(16) float bias[kMaxBias];
-    uint4 stage[kEpiWarps][32 * 4];  // per epilogue warp: 32 rows x 32 bf16 columns, 16-byte pieces swizzled
+    // followed by the epilogue staging: per epilogue warp 32 rows x 32 bf16 columns (2 KB), 16-byte pieces swizzled
 };
 
 __global__ void __launch_bounds__(kKThreads, 1) tma_kmajor_kernel(const __grid_constant__ KArgs a) {
@@ -234,16 +236,16 @@ __global__ void __launch_bounds__(kKThreads, 1) tma_kmajor_kernel(const __grid_c
         }
         for (int i = 0; i < nacc; ++i) {
             mbar_init(&pipe->tfull[i], 1);
-            mbar_init(&pipe->tempty[i], kEpiWarps * 32);
+            mbar_init(&pipe->tempty[i], a.nepi * 32);
         }
         mbar_init(&pipe->wfull, 1);
         pipe->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (a.mode != EPI_DGRAD)
-        for (int i = threadIdx.x; i < a.tiles_n * BN; i += kKThreads) pipe->bias[i] = i < a.N ? a.bias[i] : 0.f;
+        for (int i = threadIdx.x; i < a.tiles_n * BN; i += (int)blockDim.x) pipe->bias[i] = i < a.N ? a.bias[i] : 0.f;
     if (a.wres)
-        for (int i = threadIdx.x; i < a.ncls * kMaxWtab; i += kKThreads) {
+        for (int i = threadIdx.x; i < a.ncls * kMaxWtab; i += (int)blockDim.x) {
             const int c = i / kMaxWtab, q = i - c * kMaxWtab;
             const int tap = q / a.kchunks, kc = q - tap * a.kchunks;
             if (tap < a.cls[c].taps.n)
@@ -376,7 +378,7 @@ __global__ void __launch_bounds__(kKThreads, 1) tma_kmajor_kernel(const __grid_c
     } else {
         // ---------------- epilogue: warp w reads TMEM lanes 32 (w % 4) .. +31; the two warps of a lane
         // quarter take alternate 16-column chunks
-        const int lg = warp & 3, half = (warp - 2) >> 2;
+        const int lg = warp & 3, ew4 = (warp - 2) >> 2, wq = a.nepi >> 2;  // ew4: which of the quarter's wq warps
         const int p = lg * 32 + lane;
         const RowGrid &gr = a.grid;
         int ti = 0;
@@ -421,19 +423,18 @@ __global__ void __launch_bounds__(kKThreads, 1) tma_kmajor_kernel(const __grid_c
             const bool use_mask = a.mode == EPI_DGRAD && a.mask != nullptr && !use_bits;
             const int acc = ti & (nacc - 1);
             const uint32_t lane_base = tmem_base + acc * acc_cols + ((uint32_t)(lg * 32) << 16);
-            if (a.out != nullptr && a.out_f32 == nullptr && a.mode != EPI_HEAD) {
+            if (a.out != nullptr && a.out_f32 == nullptr && a.mode != EPI_HEAD && !use_mask) {
                 // ---- bf16 outputs, staged: a thread owns a pixel (its TMEM lane), but a warp that stores 32
                 // pixels with one instruction touches 32 cache lines.  So 32-column groups pass through a small
                 // swizzled shared-memory tile: four lanes then move one pixel's 64 contiguous bytes, and an
                 // instruction covers 8 lines.  The ReLU mask comes in the same way, and the first group's mask
                 // is fetched before the accumulator is waited for, so that its latency overlaps the MMAs.
-                uint4 *stg = pipe->stage[warp - 2];
+                uint4 *stg = reinterpret_cast<uint4 *>(pipe + 1) + (size_t)(warp - 2) * 128;
                 const int sw = (lane >> 1) & 3;
                 const int rr0 = lane >> 2, piece = lane & 3;
-                // this warp's groups: columns half * 32 + 64 g; at most 4 (BN <= 256)
+                // this warp's groups: columns (ew4 + wq g) * 32; at most 4 (BN <= 256, wq >= 2)
                 int ng = 0;
-                for (int c0 = half * 32; c0 < BN && n0 + c0 < a.N; c0 += 64) ++ng;
-                uint4 mreg[4][4];
+                for (int c0 = ew4 * 32; c0 < BN && n0 + c0 < a.N; c0 += wq * 32) ++ng;
                 uint32_t gbits[4] = {0u, 0u, 0u, 0u};
                 if (use_bits) {
 #pragma unroll
@@ -441,26 +442,7 @@ __global__ void __launch_bounds__(kKThreads, 1) tma_kmajor_kernel(const __grid_c
                         if (g < ng) {
                             long long orow;
                             int col;
-                            if (locate(half * 32 + 64 * g, orow, col)) gbits[g] = a.mask_bits[orow * (ncol >> 5) + (col >> 5)];
-                        }
-                    }
-                }
-                if (use_mask) {
-#pragma unroll
-                    for (int g = 0; g < 4; ++g) {
-                        if (g < ng) {
-                            long long orow;
-                            int col;
-                            const int okr = locate(half * 32 + 64 * g, orow, col) ? 1 : 0;
-#pragma unroll
-                            for (int ps = 0; ps < 4; ++ps) {
-                                const int rr = ps * 8 + rr0;
-                                const long long o_r = __shfl_sync(0xffffffffu, orow, rr);
-                                const int ok_r = __shfl_sync(0xffffffffu, okr, rr);
-                                mreg[g][ps] = make_uint4(0, 0, 0, 0);
-                                if (ok_r && col + piece * 8 < ncol)
-                                    mreg[g][ps] = *reinterpret_cast<const uint4 *>(a.mask + o_r * a.ldo + col + piece * 8);
-                            }
+                            if (locate((ew4 + wq * g) * 32, orow, col)) gbits[g] = a.mask_bits[orow * (ncol >> 5) + (col >> 5)];
                         }
                     }
                 }
@@ -470,7 +452,7 @@ __global__ void __launch_bounds__(kKThreads, 1) tma_kmajor_kernel(const __grid_c
 #pragma unroll
                 for (int g = 0; g < 4; ++g) {
                     if (g >= ng) break;
-                    const int c0 = half * 32 + 64 * g;
+                    const int c0 = (ew4 + wq * g) * 32;
                     float v[32];
                     tmem_ld16(lane_base + (uint32_t)c0, v);
                     if (c0 + 16 < BN) tmem_ld16(lane_base + (uint32_t)c0 + 16u, v + 16);
@@ -498,25 +480,6 @@ __global__ void __launch_bounds__(kKThreads, 1) tma_kmajor_kernel(const __grid_c
 #pragma unroll
                         for (int i = 0; i < 32; ++i)
                             if (!((gbits[g] >> i) & 1u)) v[i] = 0.f;
-                    } else if (use_mask) {
-#pragma unroll
-                        for (int ps = 0; ps < 4; ++ps) {
-                            const int rr = ps * 8 + rr0;
-                            stg[rr * 4 + (piece ^ ((rr >> 1) & 3))] = mreg[g][ps];
-                        }
-                        __syncwarp();
-#pragma unroll
-                        for (int j = 0; j < 4; ++j) {
-                            const uint4 mk = stg[lane * 4 + (j ^ sw)];
-                            const __nv_bfloat162 *m2 = reinterpret_cast<const __nv_bfloat162 *>(&mk);
-#pragma unroll
-                            for (int i = 0; i < 4; ++i) {
-                                const float2 f = __bfloat1622float2(m2[i]);
-                                if (!(f.x > 0.f)) v[j * 8 + 2 * i] = 0.f;
-                                if (!(f.y > 0.f)) v[j * 8 + 2 * i + 1] = 0.f;
-                            }
-                        }
-                        __syncwarp();
                     }
 #pragma unroll
                     for (int j = 0; j < 4; ++j) {
@@ -545,7 +508,7 @@ __global__ void __launch_bounds__(kKThreads, 1) tma_kmajor_kernel(const __grid_c
             ok = mbar_wait(&pipe->tfull[acc], (ti >> nacc_log) & 1, abort_flag, a.status);
             if (!ok) break;
             tc_fence_after();
-            for (int c0 = half * 16; c0 < BN; c0 += 32) {
+            for (int c0 = ew4 * 16; c0 < BN; c0 += wq * 16) {
                 if (n0 + c0 >= a.N) break;  // uniform across the warp
                 float v[16];
                 tmem_ld16(lane_base + (uint32_t)c0, v);
@@ -573,6 +536,19 @@ __global__ void __launch_bounds__(kKThreads, 1) tma_kmajor_kernel(const __grid_c
                                 if (!(f.x > 0.f)) v[hlf * 8 + 2 * i] = 0.f;
                                 if (!(f.y > 0.f)) v[hlf * 8 + 2 * i + 1] = 0.f;
                             }
+                        }
+                    }
+                }
+                if (a.out) {
+                    uint4 *op = reinterpret_cast<uint4 *>(a.out + orow * a.ldo + nn);
+#pragma unroll
+                    for (int hlf = 0; hlf < 2; ++hlf) {
+                        if (nn + hlf * 8 < ncol) {
+                            __nv_bfloat162 pk[4];
+#pragma unroll
+                            for (int i = 0; i < 4; ++i)
+                                pk[i] = __floats2bfloat162_rn(v[hlf * 8 + 2 * i], v[hlf * 8 + 2 * i + 1]);
+                            op[hlf] = *reinterpret_cast<uint4 *>(pk);
                         }
                     }
                 }
@@ -882,7 +858,7 @@ int ensure_smem_attrs() {
     if (dev < 0 || dev >= 64) return PPO_ERR_CUDA;
     if (!attr_set[dev]) {
         const int mx = (int)(kSmemBudget + sizeof(PipeK) + 1024);
-        PPO_CUDA_CHECK(cudaFuncSetAttribute(tma_kmajor_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, mx));
+        PPO_CUDA_CHECK(cudaFuncSetAttribute(tma_kmajor_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemMax));
         PPO_CUDA_CHECK(cudaFuncSetAttribute(tma_wgrad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, mx));
         attr_set[dev] = true;
     }
@@ -921,7 +897,9 @@ int launch_kmajor(KArgs &a, cudaStream_t st) {
     // are what hides the copy latency
     a.wres = (a.tiles_n == 1 && a.ncls == 1 && res <= kMaxResident && a.wtaps * a.kchunks <= kMaxWtab) ? 1 : 0;
     const size_t sub = (size_t)128 * a.row_bytes + (a.wres ? 0 : b_bytes);
-    const size_t budget = kSmemBudget - (a.wres ? res : 0);
+    a.nepi = (a.mode == EPI_DGRAD && a.mask_bits) ? 16 : 8;
+    const size_t fixed = sizeof(PipeK) + (size_t)a.nepi * 2048 + 1024;  // pipeline state, epilogue staging, alignment slack
+    const size_t budget = kSmemMax - 1024 - fixed - (a.wres ? res : 0);
     int G = (int)((48 * 1024) / sub);  // sub-blocks per stage: fewer barrier round trips per byte
     G = G < 1 ? 1 : (G > 8 ? 8 : G);
     while (G > 1 && budget / (G * sub) < 3) --G;
@@ -934,8 +912,8 @@ int launch_kmajor(KArgs &a, cudaStream_t st) {
     if (a.stages < 2) return PPO_ERR_UNSUPPORTED;
     const int sms = ppo_num_sms();
     const unsigned grid = (unsigned)(total < sms ? total : sms);
-    const size_t smem = (size_t)a.stages * G * sub + (a.wres ? res : 0) + sizeof(PipeK) + 1024;
-    tma_kmajor_kernel<<<grid, kKThreads, smem, st>>>(a);
+    const size_t smem = (size_t)a.stages * G * sub + (a.wres ? res : 0) + fixed;
+    tma_kmajor_kernel<<<grid, (2 + a.nepi) * 32, smem, st>>>(a);
     PPO_LAUNCH_CHECK();
     return PPO_OK;
 }
