@@ -19,7 +19,7 @@ pytestmark = pytest.mark.gpu
 DEV = "cuda"
 GAE_TOL = 1e-5
 ENC_TOL = 2e-2
-BENCH_MICROBATCH = 2048  # bench.py's default
+BENCH_MICROBATCH = 4096  # bench.py's default
 
 
 def _device_rollout(w):
