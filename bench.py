@@ -378,7 +378,7 @@ def cpu_baseline(w, roll, L, n_samples=None):
     from oracle import oracle as orc
     import torch
     # about 10-30 s of oracle work on a 16-core host: ~0.4 / 7 / 35 ms per row at the three frame sizes
-    n_samples = n_samples or min(w.B, 4096 if w.H * w.W <= 64 * 64 else 2048 if w.H * w.W <= 120 * 160 else 512)
+    n_samples = n_samples or min(w.B, 4096 if w.H * w.W <= 120 * 160 else 768)
     idx = orc.perm(w.seed, 0, w.M, 0, n_samples).astype(np.int64)
     flat = roll["depth"].view(w.M, w.H, w.W)
     fields = {k: roll[k].cpu().numpy() for k in ("proprio", "action", "logp", "value", "reward", "done",
@@ -437,6 +437,63 @@ def run_reference(args):
     }))
 
 
+def run_stress(args):
+    """Bandwidth stress (GAE + advantage normalisation + one epoch of minibatch gathers only, T = 32) at
+    1024 / 4096 / 16384 envs: achieved GB/s of the gather and of GAE against the measured HBM copy peak."""
+    import torch
+    from paper_2509_16434_b200 import binding as ppo
+    from paper_2509_16434_b200 import synth
+    torch.cuda.set_device(0)
+    peaks = load_peaks()
+    rows = []
+    for name in ("cfg5_1k", "cfg5_4k", "cfg5_16k"):
+        w = synth.WORKLOADS[name]
+        desc = ppo.buffer_desc(w.N, w.T, w.H, w.W, w.P, w.A)
+        buf = ppo.Buffer(desc)
+        g = torch.Generator(device="cuda")
+        g.manual_seed(w.seed)
+        # fill the slabs in place (the frames of a 20 GB buffer are generated slab by slab)
+        depth = buf.field(ppo.FIELD_DEPTH)
+        for t in range(w.T):
+            u = torch.rand(depth[t].shape, generator=g, device="cuda")
+            z = torch.rand(depth[t].shape, generator=g, device="cuda") < 0.10
+            depth[t].copy_((0.1 + 1.9 * u).to(torch.float16))
+            depth[t][z] = 0
+            del u, z
+        for f in (ppo.FIELD_PROPRIO, ppo.FIELD_ACTION, ppo.FIELD_LOGP, ppo.FIELD_VALUE, ppo.FIELD_REWARD):
+            buf.field(f).copy_(torch.randn(buf.field(f).shape, generator=g, device="cuda"))
+        buf.field(ppo.FIELD_DONE).copy_((torch.rand((w.T, w.N), generator=g, device="cuda") < w.done_rate).to(torch.uint8))
+        last_value = torch.randn(w.N, generator=g, device="cuda")
+        mb = ppo.MinibatchArrays(desc, w.B, with_index=False)
+        ev = lambda: torch.cuda.Event(enable_timing=True)
+        gae_ms, gat_ms = [], []
+        for it in range(args.warmup + args.steps):
+            e0, e1, e2 = ev(), ev(), ev()
+            e0.record()
+            ppo.ppo_compute_gae(buf, last_value, w.gamma, w.lam, True, None)
+            e1.record()
+            for k in range(w.minibatches):
+                ppo.ppo_shuffle_gather_minibatch(buf, it, 0, k, w.minibatches, mb)
+            e2.record()
+            torch.cuda.synchronize()
+            if it >= args.warmup:
+                gae_ms.append(e0.elapsed_time(e1))
+                gat_ms.append(e1.elapsed_time(e2))
+        gae, gat = float(np.median(gae_ms)), float(np.median(gat_ms))
+        gather_gbs = 2 * w.M * record_bytes(w) / (gat * 1e-3) / 1e9
+        gae_gbs = (17 + 8) * w.M / (gae * 1e-3) / 1e9
+        rows.append({"workload": name, "envs": w.N, "T": w.T, "buffer_GB": round(w.M * record_bytes(w) / 1e9, 2),
+                     "gather_ms_per_epoch": round(gat, 3), "gather_GBs": round(gather_gbs, 1),
+                     "gather_frac_of_measured_hbm": round(gather_gbs / peaks["hbm_gbs"], 4),
+                     "gae_norm_ms": round(gae, 4), "gae_norm_GBs": round(gae_gbs, 1),
+                     "gae_norm_frac_of_measured_hbm": round(gae_gbs / peaks["hbm_gbs"], 4)})
+        assert ppo.ppo_poll_status() == 0
+        del buf, mb, depth
+        torch.cuda.empty_cache()
+    print(json.dumps({"metric": "buffer_path_bandwidth", "unit": "GB/s", "peak_hbm_gbs": peaks["hbm_gbs"],
+                      "peak_source": peaks["source"], "rows": rows}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -446,8 +503,11 @@ def main():
     ap.add_argument("--workload", default="cfg2")
     ap.add_argument("--microbatch", type=int, default=4096)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--stress", action="store_true", help="bandwidth stress of the buffer path (GAE + gathers, T = 32)")
     args = ap.parse_args()
-    if args.impl == "reference":
+    if args.stress:
+        run_stress(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_ours(args)
