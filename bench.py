@@ -490,8 +490,49 @@ def run_stress(args):
         assert ppo.ppo_poll_status() == 0
         del buf, mb, depth
         torch.cuda.empty_cache()
+    # Supplementary, HBM-resident inputs (NOT configs): the GAE and Adam kernels on working sets far larger than L2,
+    # to show their asymptotic bandwidth; at config sizes both finish inside a launch latency.
+    extra = []
+    T, N = 128, 524288
+    g = torch.Generator(device="cuda")
+    g.manual_seed(1)
+    reward = torch.randn((T, N), generator=g, device="cuda")
+    value = torch.randn((T, N), generator=g, device="cuda")
+    done = (torch.rand((T, N), generator=g, device="cuda") < 0.01).to(torch.uint8)
+    lastv = torch.randn(N, generator=g, device="cuda")
+    adv, ret = torch.empty_like(reward), torch.empty_like(reward)
+    ms = []
+    for it in range(args.warmup + args.steps):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        ppo.ppo_gae_static(reward, value, done, lastv, 0.99, 0.95, True, adv, ret)
+        e1.record()
+        torch.cuda.synchronize()
+        if it >= args.warmup:
+            ms.append(e0.elapsed_time(e1))
+    t = float(np.median(ms))
+    gbs = (17 + 8) * T * N / (t * 1e-3) / 1e9
+    extra.append({"kernel": "gae_scan + adv_normalize", "input": f"{N} envs x T={T} ({(17 + 8) * T * N / 1e9:.2f} GB moved)",
+                  "ms": round(t, 3), "GBs": round(gbs, 1), "frac_of_measured_hbm": round(gbs / peaks["hbm_gbs"], 4)})
+    del reward, value, done, adv, ret
+    md = ppo.model_desc(16, 16, (8,), (3,), (16384, 16384), 32, 12)
+    model = ppo.Model(md, 1)
+    model.grad.normal_(generator=g)
+    ms = []
+    for it in range(args.warmup + args.steps):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        ppo.ppo_adam_step(model, 3e-4, 0.9, 0.999, 1e-8, it + 1)
+        e1.record()
+        torch.cuda.synchronize()
+        if it >= args.warmup:
+            ms.append(e0.elapsed_time(e1))
+    t = float(np.median(ms))
+    gbs = 30 * model.arena / (t * 1e-3) / 1e9
+    extra.append({"kernel": "adam_kernel", "input": f"{model.arena} parameters ({30 * model.arena / 1e9:.2f} GB moved)",
+                  "ms": round(t, 3), "GBs": round(gbs, 1), "frac_of_measured_hbm": round(gbs / peaks["hbm_gbs"], 4)})
     print(json.dumps({"metric": "buffer_path_bandwidth", "unit": "GB/s", "peak_hbm_gbs": peaks["hbm_gbs"],
-                      "peak_source": peaks["source"], "rows": rows}))
+                      "peak_source": peaks["source"], "rows": rows, "supplementary_scaled_inputs": extra}))
 
 
 def main():
