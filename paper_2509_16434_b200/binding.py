@@ -296,6 +296,8 @@ class Model:
         _check(lib().ppo_model_activation_ptr(self.handle, kind, index, C.byref(p), C.byref(n)),
                "ppo_model_activation_ptr")
         off = p.value - self.workspace.data_ptr()
+        if kind == 2:
+            return self.workspace[off:off + 4 * n.value].view(torch.int32)
         return self.workspace[off:off + 2 * n.value].view(torch.bfloat16)
 
     def load(self, theta, stream=None):

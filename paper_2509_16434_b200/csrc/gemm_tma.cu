@@ -4,12 +4,13 @@
 // activation tensor with a traversal stride of 2 along W and H *is* the im2col tile of one kernel tap
 // of a stride-2 convolution, zero padding included (out-of-range parts of a box arrive as zeros), and
 // it lands in shared memory already in the swizzled image the UMMA descriptors name.  A second thread
-// issues tcgen05.mma into a double-buffered accumulator in tensor memory; four warps read it back with
+// issues tcgen05.mma into a ring of accumulators in tensor memory; 8 or 16 warps read them back with
 // tcgen05.ld for the epilogue.  No thread computes an address per element.
 //
 //  tma_kmajor_kernel : D[m][n] = sum_k A[m][k] B[n][k], both operands K-major.
 //      forward  A = tap boxes of X (row m = output pixel), B = W[co][tap][ci]
-//      dgrad    A = shifted boxes of dY (row m = input pixel of one stride-parity class), B = Wt[ci][tap][co]
+//      dgrad    A = shifted boxes of dY (row m = a 2x2 block of input pixels, all four stride-parity classes
+//               side by side in the columns), B = the weights regrouped per shift
 //  tma_wgrad_kernel  : D[j][co] = sum_m A[m][j] B[m][co], both operands MN-major: the same tap boxes of X
 //      and plain boxes of dY, read with the pixel index as the reduction; split over pixel tiles across
 //      CTAs, fp32 atomics into dW.

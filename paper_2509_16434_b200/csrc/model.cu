@@ -183,6 +183,11 @@ extern "C" int ppo_model_activation_ptr(const ppo_model *m, int kind, int index,
         *elems = (size_t)m->mbmax * m->Hs[index] * m->Ws[index] * m->Cs[index];
         return PPO_OK;
     }
+    if (kind == 2 && index >= 1 && index < m->L && m->abits[index]) {
+        *ptr = m->abits[index];
+        *elems = (size_t)m->mbmax * m->Hs[index] * m->Ws[index] * m->Cs[index] / 32;
+        return PPO_OK;
+    }
     if (kind == 1 && index >= 0 && index <= m->F) {
         *ptr = m->h[index];
         *elems = (size_t)m->mbmax * m->hw[index];

@@ -272,3 +272,31 @@ def test_policy_act_matches_oracle():
     assert rel_l2(a.cpu().numpy(), action[0]) <= ENC_TOL
     assert np.abs(lp.cpu().numpy() - logp[0]).max() <= 1e-4  # log-prob depends on eps and log-sigma only
     assert ppo.ppo_poll_status() == 0
+
+
+def test_forward_writes_the_relu_gate_bits_of_its_activations():
+    """The one-bit gates the backward pass reads must say exactly act > 0, whether the forward kernels wrote them
+    or ppo_model_sync_masks recomputed them."""
+    w = SHAPES["cfg2_twin"]
+    B = w.M // w.minibatches
+    L, md, lay, theta, roll, action, logp, dev = _setup(w, B)
+    L.compute_gae(dev["last_value"])
+    ppo.ppo_shuffle_gather_minibatch(L.buffer, 0, 0, 0, w.minibatches, L.mb)
+    ppo.ppo_encoder_fwd(L.model, L.mb, 0, B, L.mean, L.value)
+    Ho, Wo = orc.conv_shapes(md)
+    checked = 0
+    for l, (h, w_, c) in enumerate(zip(Ho, Wo, md.conv_c), start=1):
+        if l == len(md.conv_c) or c % 32 != 0:
+            continue
+        n = B * h * w_ * c
+        act = L.model.activation(0, l)[:n].float().cpu().numpy().reshape(-1, 32)
+        want = (act > 0).astype(np.uint64)
+        want_words = (want << np.arange(32, dtype=np.uint64)).sum(1).astype(np.uint32)
+        got = L.model.activation(2, l)[:n // 32].cpu().numpy().view(np.uint32)
+        assert np.array_equal(got, want_words), f"layer {l}: forward-written gates"
+        L.model.activation(2, l)[:n // 32].zero_()
+        ppo.ppo_model_sync_masks(L.model, B)
+        got = L.model.activation(2, l)[:n // 32].cpu().numpy().view(np.uint32)
+        assert np.array_equal(got, want_words), f"layer {l}: recomputed gates"
+        checked += 1
+    assert checked >= 2 and ppo.ppo_poll_status() == 0
