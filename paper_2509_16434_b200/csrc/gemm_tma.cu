@@ -181,6 +181,7 @@ struct KArgs {
     int kchunks;            // boxes along the channels of one tap
     int w_tap;              // elements between taps in a weight row
     int G, nbmax;           // sub-blocks per stage; most A boxes a tile has
+    int tmem_cap;           // tensor-memory columns this CTA may take: 512, or 256 when two CTAs share an SM
     int nepi;               // epilogue warps: 8, or 16 where the epilogue is the heavier side (dgrad with gate bits)
     int wres, wtaps;        // weights resident in shared memory (all wtaps * kchunks boxes, loaded once)
     int N, BN, tiles_n, total_tiles, ncls, stages;  // tile g = ((mt * tiles_n) + nt) * ncls + class
@@ -227,7 +228,7 @@ __global__ void __launch_bounds__(kKThreads, 1) tma_kmajor_kernel(const __grid_c
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     // ring of accumulators in tensor memory: four when they fit in its 512 columns, else two
     const uint32_t acc_cols = tmem_cols_for(BN);
-    const int nacc_log = acc_cols * 4 <= 512 ? 2 : 1, nacc = 1 << nacc_log;
+    const int nacc_log = acc_cols * 4 <= (uint32_t)a.tmem_cap ? 2 : 1, nacc = 1 << nacc_log;
     const uint32_t ncols = acc_cols * nacc;
 
     if (threadIdx.x == 0) {
@@ -897,10 +898,17 @@ int launch_kmajor(KArgs &a, cudaStream_t st) {
     // resident weights only while they leave most of the shared memory to the A stages: the bytes in flight
     // are what hides the copy latency
     a.wres = (a.tiles_n == 1 && a.ncls == 1 && res <= kMaxResident && a.wtaps * a.kchunks <= kMaxWtab) ? 1 : 0;
-    const size_t sub = (size_t)128 * a.row_bytes + (a.wres ? 0 : b_bytes);
-    a.nepi = (a.mode == EPI_DGRAD && a.mask_bits) ? 16 : 8;
+    // Narrow tiles (BN <= 128) leave the tensor pipe mostly idle because one thread per CTA cannot issue MMAs
+    // fast enough; two CTAs per SM (half the shared and tensor memory each, 8 epilogue warps each) double the
+    // issue rate.  Wide tiles run at the tensor rate with one CTA and keep the SM to themselves.
+    const bool two = a.BN <= 128;
+    a.tmem_cap = two ? 256 : 512;
+    a.nepi = (!two && a.mode == EPI_DGRAD && a.mask_bits) ? 16 : 8;
     const size_t fixed = sizeof(PipeK) + (size_t)a.nepi * 2048 + 1024;  // pipeline state, epilogue staging, alignment slack
-    const size_t budget = kSmemMax - 1024 - fixed - (a.wres ? res : 0);
+    const size_t cta_max = two ? kSmemMax / 2 : kSmemMax;
+    if (a.wres && res + fixed + 3 * (size_t)128 * a.row_bytes + 1024 > cta_max) a.wres = 0;
+    const size_t sub = (size_t)128 * a.row_bytes + (a.wres ? 0 : b_bytes);
+    const size_t budget = cta_max - 1024 - fixed - (a.wres ? res : 0);
     int G = (int)((48 * 1024) / sub);  // sub-blocks per stage: fewer barrier round trips per byte
     G = G < 1 ? 1 : (G > 8 ? 8 : G);
     while (G > 1 && budget / (G * sub) < 3) --G;
@@ -912,7 +920,8 @@ int launch_kmajor(KArgs &a, cudaStream_t st) {
     if (a.stages > kMaxStages) a.stages = kMaxStages;
     if (a.stages < 2) return PPO_ERR_UNSUPPORTED;
     const int sms = ppo_num_sms();
-    const unsigned grid = (unsigned)(total < sms ? total : sms);
+    const long long ctas = two ? 2ll * sms : sms;
+    const unsigned grid = (unsigned)(total < ctas ? total : ctas);
     const size_t smem = (size_t)a.stages * G * sub + (a.wres ? res : 0) + fixed;
     tma_kmajor_kernel<<<grid, (2 + a.nepi) * 32, smem, st>>>(a);
     PPO_LAUNCH_CHECK();
@@ -1142,12 +1151,16 @@ int tma_gemm_wgrad(const ConvGeom &g, const bf16 *dY, int ldy, const bf16 *X, fl
     a.dW = dW;
     a.status = status;
     const size_t stage = (size_t)128 * 256 + (size_t)128 * 2 * a.BN;
-    a.stages = stages_for(stage);
+    // two CTAs per SM (twice the MMA issue rate) when two stages fit into half of the shared memory
+    const size_t half_budget = kSmemMax / 2 - 1024 - sizeof(Pipe) - 1024;
+    const bool two = 2 * stage <= half_budget && a.BN <= 256;
+    a.stages = two ? (int)(half_budget / stage) : stages_for(stage);
+    if (a.stages > kMaxStages) a.stages = kMaxStages;
     if (a.stages < 2) return PPO_ERR_UNSUPPORTED;
     s = ensure_smem_attrs();
     if (s != PPO_OK) return s;
     const int jtiles = (a.ntaps * a.kchunks + a.mblocks - 1) / a.mblocks, ctiles = g.Co / a.BN;
-    int splits = ppo_num_sms() / (jtiles * ctiles);
+    int splits = (two ? 2 : 1) * ppo_num_sms() / (jtiles * ctiles);
     if (splits < 1) splits = 1;
     if (splits > a.grid.tiles) splits = a.grid.tiles;
     a.tiles_per_split = (a.grid.tiles + splits - 1) / splits;
