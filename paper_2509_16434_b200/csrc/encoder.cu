@@ -206,7 +206,7 @@ __global__ void __launch_bounds__(128) conv1_wgrad_kernel(const __half *__restri
 }
 
 // The same reduction on the tensor cores (mma.sync m16n8k16, bf16): per 16 output pixels a warp forms
-// D[tap][co] += X^T[tap][px] dZ[px][co] with the pixel index as K.  The 16 x TP patch tile X (k*k depth taps as
+// D[tap][co] += X^T[tap][px] dZ[px][co] with the pixel index as K (32 pixels, one per lane, per trip).  The patch tile X (k*k depth taps as
 // bf16, then a column of ones whose product is the bias gradient, zero padded to TP) and the 16 x C1 gradient
 // tile go through per-warp shared memory and come back as fragments with ldmatrix.trans.  About 3 instructions
 // per pixel instead of C1 (k*k + 1) / 32 multiply-adds plus their loads: the kernel becomes a stream over dZ.
@@ -230,8 +230,9 @@ __global__ void __launch_bounds__(256) conv1_wgrad_mma_kernel(const __half *__re
                                                               float *__restrict__ db, int rows, int Hi, int Wi,
                                                               int Ho, int Wo, long long px_per_warp) {
     constexpr int K2 = KS * KS, P = KS / 2, TP = (K2 + 1 + 15) / 16 * 16, MB = TP / 16, C1 = NB * 8;
-    constexpr int kXBytes = 16 * TP * 2, kZBytes = 16 * C1 * 2;
-    extern __shared__ __align__(16) uint8_t smw[];  // per warp: X tile [16 px][TP], dZ tile [16 px][C1]; later the reduction
+    constexpr int PX = 32;  // pixels per trip: one per lane, two K = 16 steps of the MMA
+    constexpr int kXBytes = PX * TP * 2, kZBytes = PX * C1 * 2;
+    extern __shared__ __align__(16) uint8_t smw[];  // per warp: X tile [32 px][TP], dZ tile [32 px][C1]; later the reduction
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     uint8_t *xs = smw + (size_t)warp * (kXBytes + kZBytes), *zs = xs + kXBytes;
     const uint32_t xs_a = (uint32_t)__cvta_generic_to_shared(xs), zs_a = (uint32_t)__cvta_generic_to_shared(zs);
@@ -244,34 +245,31 @@ __global__ void __launch_bounds__(256) conv1_wgrad_mma_kernel(const __half *__re
             for (int q = 0; q < 4; ++q) acc[i][j][q] = 0.f;
     const long long M = (long long)rows * Ho * Wo;
     const long long gw = (long long)blockIdx.x * 8 + warp;
-    long long m0 = gw * px_per_warp;                       // px_per_warp is a multiple of 16
+    long long m0 = gw * px_per_warp;                       // px_per_warp is a multiple of 32
     const long long m_end = min(M, m0 + px_per_warp);
-    // this lane's pixel of the patch tile: px = lane % 16, taps [half * TP / 2, +TP / 2)
-    const int pxl = lane & 15, half = lane >> 4;
-    int ow = 0, oh = 0;
+    int ow = 0, oh = 0;  // this lane's pixel m0 + lane
     long long b = 0;
     if (m0 < m_end) {
-        const long long m = m0 + pxl;
+        const long long m = m0 + lane;
         ow = (int)(m % Wo);
         const long long t = m / Wo;
         oh = (int)(t % Ho);
         b = t / Ho;
     }
-    const int d_oh = 16 / Wo, d_ow = 16 % Wo;  // 16 pixels further (Wo >= 1)
-    constexpr int ZP = (16 * C1 / 8 + 31) / 32;  // 16-byte pieces of the gradient tile per lane
-    uint4 xreg[TP / 16], zreg[ZP];
+    const int d_oh = PX / Wo, d_ow = PX % Wo;  // 32 pixels further (Wo >= 1)
+    constexpr int ZP = PX * C1 / 8 / 32;       // 16-byte pieces of the gradient tile per lane
+    uint4 xreg[TP / 8], zreg[ZP];
     // Loads of the tile that starts at pixel mt into registers; they are issued one trip ahead, so that their
     // latency overlaps the previous tile's MMAs.
     auto prefetch = [&](long long mt) {
-        const bool live = mt + pxl < m_end;
+        const bool live = mt + lane < m_end;
         const __half *img = depth + b * Hi * Wi;
 #pragma unroll
-        for (int c = 0; c < TP / 16; ++c) {  // 8 taps = one 16-byte piece
-            const int t0 = half * (TP / 2) + c * 8;
+        for (int c = 0; c < TP / 8; ++c) {  // 8 taps = one 16-byte piece
             __nv_bfloat162 pk[4];
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
-                const int tap = t0 + j;
+                const int tap = c * 8 + j;
                 float xv = 0.f;
                 if (tap < K2) {
                     const int kh = tap / KS, kw = tap - kh * KS;
@@ -289,43 +287,45 @@ __global__ void __launch_bounds__(256) conv1_wgrad_mma_kernel(const __half *__re
         for (int z = 0; z < ZP; ++z) {
             const int i = lane + 32 * z;
             zreg[z] = make_uint4(0, 0, 0, 0);
-            if (i < 16 * C1 / 8 && mt + i / (C1 / 8) < m_end) zreg[z] = __ldcs(reinterpret_cast<const uint4 *>(dZ + mt * C1) + i);
+            if (mt + i / (C1 / 8) < m_end) zreg[z] = __ldcs(reinterpret_cast<const uint4 *>(dZ + mt * C1) + i);
         }
     };
     if (m0 < m_end) prefetch(m0);
-    for (; m0 < m_end; m0 += 16) {
+    for (; m0 < m_end; m0 += PX) {
 #pragma unroll
-        for (int c = 0; c < TP / 16; ++c)
-            *reinterpret_cast<uint4 *>(xs + pxl * (TP * 2) + (half * (TP / 2) + c * 8) * 2) = xreg[c];
+        for (int c = 0; c < TP / 8; ++c) *reinterpret_cast<uint4 *>(xs + lane * (TP * 2) + c * 16) = xreg[c];
 #pragma unroll
-        for (int z = 0; z < ZP; ++z)
-            if (lane + 32 * z < 16 * C1 / 8) reinterpret_cast<uint4 *>(zs)[lane + 32 * z] = zreg[z];
+        for (int z = 0; z < ZP; ++z) reinterpret_cast<uint4 *>(zs)[lane + 32 * z] = zreg[z];
         __syncwarp();
         ow += d_ow;
         if (ow >= Wo) { ow -= Wo; ++oh; }
         oh += d_oh;
         while (oh >= Ho) { oh -= Ho; ++b; }
-        if (m0 + 16 < m_end) prefetch(m0 + 16);
-        // ---- fragments and MMAs
-        uint32_t af[MB][4];
+        if (m0 + PX < m_end) prefetch(m0 + PX);
+        // ---- fragments and MMAs, 16 pixels per K step
 #pragma unroll
-        for (int i = 0; i < MB; ++i) {
-            // matrices: (taps 16i..+7, px 0-7), (taps 16i+8.., px 0-7), (taps 16i.., px 8-15), (taps 16i+8.., px 8-15)
+        for (int ks = 0; ks < PX / 16; ++ks) {
+            uint32_t af[MB][4];
             const int mi = lane >> 3, r = lane & 7;
-            const uint32_t addr = xs_a + (uint32_t)((r + (mi >= 2 ? 8 : 0)) * (TP * 2) + (16 * i + (mi & 1) * 8) * 2);
-            ldmatrix_x4_trans(addr, af[i][0], af[i][1], af[i][2], af[i][3]);
-        }
-#pragma unroll
-        for (int j = 0; j < NB; j += 2) {
-            // matrices: (px 0-7, co 8j..), (px 8-15, co 8j..), (px 0-7, co 8j+8..), (px 8-15, co 8j+8..)
-            const int mi = lane >> 3, r = lane & 7;
-            const uint32_t addr = zs_a + (uint32_t)((r + (mi & 1) * 8) * (C1 * 2) + (8 * j + (mi >> 1) * 8) * 2);
-            uint32_t b0, b1, b2, b3;
-            ldmatrix_x4_trans(addr, b0, b1, b2, b3);
 #pragma unroll
             for (int i = 0; i < MB; ++i) {
-                mma_bf16_16816(acc[i][j], af[i][0], af[i][1], af[i][2], af[i][3], b0, b1);
-                mma_bf16_16816(acc[i][j + 1], af[i][0], af[i][1], af[i][2], af[i][3], b2, b3);
+                // matrices: (taps 16i..+7, px 0-7), (taps 16i+8.., px 0-7), (taps 16i.., px 8-15), (taps 16i+8.., px 8-15)
+                const uint32_t addr =
+                    xs_a + (uint32_t)((16 * ks + r + (mi >= 2 ? 8 : 0)) * (TP * 2) + (16 * i + (mi & 1) * 8) * 2);
+                ldmatrix_x4_trans(addr, af[i][0], af[i][1], af[i][2], af[i][3]);
+            }
+#pragma unroll
+            for (int j = 0; j < NB; j += 2) {
+                // matrices: (px 0-7, co 8j..), (px 8-15, co 8j..), (px 0-7, co 8j+8..), (px 8-15, co 8j+8..)
+                const uint32_t addr =
+                    zs_a + (uint32_t)((16 * ks + r + (mi & 1) * 8) * (C1 * 2) + (8 * j + (mi >> 1) * 8) * 2);
+                uint32_t b0, b1, b2, b3;
+                ldmatrix_x4_trans(addr, b0, b1, b2, b3);
+#pragma unroll
+                for (int i = 0; i < MB; ++i) {
+                    mma_bf16_16816(acc[i][j], af[i][0], af[i][1], af[i][2], af[i][3], b0, b1);
+                    mma_bf16_16816(acc[i][j + 1], af[i][0], af[i][1], af[i][2], af[i][3], b2, b3);
+                }
             }
         }
         __syncwarp();
@@ -761,13 +761,13 @@ extern "C" int ppo_encoder_bwd(ppo_model *m, const ppo_minibatch *mb, int row0, 
         if (m->impl == 0 && C1 % 16 == 0 && C1 <= 64 && (KS == 3 || KS == 5)) {
             // tensor-core reduction
             const int TP = (KS * KS + 1 + 15) / 16 * 16;
-            const size_t tile = (size_t)16 * TP * 2 + (size_t)16 * C1 * 2, redb = (size_t)TP * C1 * sizeof(float);
+            const size_t tile = (size_t)32 * TP * 2 + (size_t)32 * C1 * 2, redb = (size_t)TP * C1 * sizeof(float);
             const size_t smem = 8 * (tile > redb ? tile : redb);
             int blocks = ppo_cdiv(M, 8 * 16 * 8);
             const int cap = ppo_num_sms() * 4;
             blocks = blocks > cap ? cap : (blocks < 1 ? 1 : blocks);
             long long per_warp = (M + (long long)blocks * 8 - 1) / ((long long)blocks * 8);
-            per_warp = (per_warp + 15) / 16 * 16;
+            per_warp = (per_warp + 31) / 32 * 32;
             float *dW = m->grad + m->tensors[0].off, *db = m->grad + m->tensors[1].off;
 #define PPO_C1W(KS_, NB_)                                                                                       \
     do {                                                                                                        \
