@@ -27,6 +27,7 @@ import numpy as np
 ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
+NCU_DRAM_BYTES_PER_ROW = (1059.7e6 + 333.9e6) / 512
 METRIC = "ppo_learner_env_steps_trained_per_sec"
 UNIT = "env-steps/s"
 
@@ -311,9 +312,15 @@ def run_ours(args):
         gather_gbs = 2 * w.B * record_bytes(w) / (gat_ms * 1e-3) / 1e9
         gae_gbs = (17 + 8) * w.M / (gae_ms * 1e-3) / 1e9
         adam_gbs = 30 * L.model.arena / (adam_ms * 1e-3) / 1e9
-        roofline = {"bound": "tensor", "kernel": "ppo_encoder_fwd + ppo_encoder_bwd (implicit-GEMM convolutions)",
+        # DRAM bytes of the encoder's GEMM and conv1 kernels per sample row (dram__bytes_read + write summed over the 18
+        # launches of one forward + backward, ncu capture of the cfg2 network at 512 rows: profiles/ncu_main_kernels_cfg2_prof.md);
+        # traffic grows in proportion to the rows.  Valid for the cfg2/cfg3 network only, and only while those kernels are unchanged.
+        traffic = NCU_DRAM_BYTES_PER_ROW * mean_rows if w.name in ("cfg2", "cfg3", "cfg2_prof") else None
+        roofline = {"bound": "tensor",
+                    "kernel": "ppo_encoder_fwd + ppo_encoder_bwd: tma_kmajor_kernel / tma_wgrad_kernel (tcgen05 implicit GEMMs) "
+                              "+ conv1 kernels; flops, time and traffic per call pair",
                     "achieved": round(enc_tf, 2), "peak": peak_tf, "unit": "TFLOP/s",
-                    "frac": round(enc_tf / peak_tf, 4), "traffic": None,
+                    "frac": round(enc_tf / peak_tf, 4), "traffic": traffic,
                     "peak_source": peaks["source"] + " (sustained bf16)",
                     "ms_per_call": {"fwd": round(fwd_ms, 4), "bwd": round(bwd_ms, 4), "rows": mean_rows}}
         others = {
