@@ -89,6 +89,8 @@ class Learner:
         ppo.ppo_model_zero_grad(self.model)
         self.loss.zero_()
         self.launches += 3
+        # the first backward after a weight change re-derives the transposed / regrouped weight copies
+        self.launches += 2 * (len(w.conv_c) - 1) + len(w.fc) + 1
         for r0 in range(0, B, self.microbatch):
             rows = min(self.microbatch, B - r0)
             ppo.ppo_encoder_fwd(self.model, self.mb, r0, rows, self.mean, self.value)
