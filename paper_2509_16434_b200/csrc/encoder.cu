@@ -572,12 +572,24 @@ static int run_dgrad(const ppo_model *m, const ConvGeom &g, const bf16 *dY, int 
     return tc_gemm_dgrad(g, dY, ldy, Wt, wt_ld, e, ppo_device_status_ptr(), st);
 }
 
+static int run_colsum(const bf16 *dZ, int ld, long long M, int N, float *db, cudaStream_t st);
+
+// Weight and bias gradients of one layer.  The TMA kernel of a convolution sums the bias gradient on the
+// tensor core on its way; everything else reduces dY in a pass of its own.
 static int run_wgrad(const ppo_model *m, const ConvGeom &g, const bf16 *dY, int ldy, const bf16 *X, float *dW,
-                     cudaStream_t st) {
-    if (m->impl == 1) return simt_gemm_wgrad(g, dY, ldy, X, dW, st);
-    const int s = tma_gemm_wgrad(g, dY, ldy, X, dW, ppo_device_status_ptr(), st);
-    if (s != PPO_ERR_UNSUPPORTED) return s;
-    return tc_gemm_wgrad(g, dY, ldy, X, dW, ppo_device_status_ptr(), st);
+                     float *db, cudaStream_t st) {
+    int s = PPO_ERR_UNSUPPORTED;
+    if (m->impl == 1) {
+        s = simt_gemm_wgrad(g, dY, ldy, X, dW, st);
+    } else {
+        const bool conv = g.k > 1;
+        s = tma_gemm_wgrad(g, dY, ldy, X, dW, conv ? db : nullptr, ppo_device_status_ptr(), st);
+        if (s == PPO_OK && conv) return s;
+        if (s == PPO_ERR_UNSUPPORTED && conv) s = tma_gemm_wgrad(g, dY, ldy, X, dW, nullptr, ppo_device_status_ptr(), st);
+        if (s == PPO_ERR_UNSUPPORTED) s = tc_gemm_wgrad(g, dY, ldy, X, dW, ppo_device_status_ptr(), st);
+    }
+    if (s != PPO_OK) return s;
+    return run_colsum(dY, ldy, g.M(), g.Co, db, st);
 }
 
 static int run_colsum(const bf16 *dZ, int ld, long long M, int N, float *db, cudaStream_t st) {
@@ -730,8 +742,7 @@ extern "C" int ppo_encoder_bwd(ppo_model *m, const ppo_minibatch *mb, int row0, 
         const int ldy = (l <= F) ? Co : 16;
         ConvGeom g = fc_geom(rows, m->hw[l - 1], Co);
         const bf16 *dY = m->dh[l];
-        PPO_TRY(run_wgrad(m, g, dY, ldy, m->h[l - 1], m->grad + m->tensors[ti].off, st));
-        PPO_TRY(run_colsum(dY, ldy, rows, Co, m->grad + m->tensors[ti + 1].off, st));
+        PPO_TRY(run_wgrad(m, g, dY, ldy, m->h[l - 1], m->grad + m->tensors[ti].off, m->grad + m->tensors[ti + 1].off, st));
         DgradEpilogue e;
         if (l > 1) e = {m->h[l - 1], m->dh[l - 1], nullptr};
         else e = {nullptr, nullptr, m->dh0_f32};
@@ -747,8 +758,8 @@ extern "C" int ppo_encoder_bwd(ppo_model *m, const ppo_minibatch *mb, int row0, 
     for (int l = L; l >= 2; --l) {
         const int ti = 2 * (l - 1);
         ConvGeom g = conv_geom(m, l, rows);
-        PPO_TRY(run_wgrad(m, g, m->dact[l], g.Co, m->act[l - 1], m->grad + m->tensors[ti].off, st));
-        PPO_TRY(run_colsum(m->dact[l], g.Co, g.M(), g.Co, m->grad + m->tensors[ti + 1].off, st));
+        PPO_TRY(run_wgrad(m, g, m->dact[l], g.Co, m->act[l - 1], m->grad + m->tensors[ti].off,
+                          m->grad + m->tensors[ti + 1].off, st));
         DgradEpilogue e = {m->act[l - 1], m->dact[l - 1], nullptr};
         e.mask_bits = m->abits[l - 1];
         PPO_TRY(run_dgrad(m, g, m->dact[l], g.Co, m->shadow + m->tensors[ti].off, m->wT + m->wT_off[ti],

@@ -50,7 +50,9 @@ int tma_gemm_dgrad(const ConvGeom &g, const bf16 *dY, int ldy, const bf16 *Wt, i
                    const DgradEpilogue &e, int32_t *status, cudaStream_t st);
 size_t tma_dgrad_weight_elems(int Ci, int k, int wt_ld);
 int tma_dgrad_weights(const bf16 *W, bf16 *Wc, int Co, int k, int Ci, int wt_ld, cudaStream_t st);
-int tma_gemm_wgrad(const ConvGeom &g, const bf16 *dY, int ldy, const bf16 *X, float *dW, int32_t *status,
+// db (may be null; convolutions only): the bias gradient db[co] += sum over pixels of dY[.][co], taken from a
+// column of ones beside the tap columns of X.
+int tma_gemm_wgrad(const ConvGeom &g, const bf16 *dY, int ldy, const bf16 *X, float *dW, float *db, int32_t *status,
                    cudaStream_t st);
 
 // bits[m][c / 32] bit (c % 32) = act[m][c] > 0, for C a multiple of 32.

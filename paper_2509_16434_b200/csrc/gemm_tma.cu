@@ -585,6 +585,11 @@ struct WArgs {
     int Kfwd, Co;
     int tiles_per_split, nmma, stages;
     float *dW;                      // [Co][Kfwd], accumulated with atomics
+    // Bias gradient db[co] += sum over pixels of dY, or null.  The last column tile has an A block that no tap
+    // fills; its first column is set to ones, so row ones_blk * CB of that tile's accumulator is the column
+    // sum of dY: the pass over dY that a separate reduction kernel would make comes for free.
+    float *db;
+    int ones_blk;
     int32_t *status;
 };
 
@@ -614,8 +619,20 @@ __global__ void __launch_bounds__(kThreads, 1) tma_wgrad_kernel(const __grid_con
         uint4 *z = reinterpret_cast<uint4 *>(smem);
         const uint32_t n16 = (uint32_t)S * stage_bytes / 16u;
         for (uint32_t i = threadIdx.x; i < n16; i += kThreads) z[i] = make_uint4(0, 0, 0, 0);
-        fence_async_smem();
     }
+    const bool ones_tile = a.db != nullptr && blockIdx.x == gridDim.x - 1;
+    if (ones_tile) {
+        // channel 0 of block ones_blk, all 128 pixel rows of every stage: the first element of 16-byte piece 0,
+        // which the swizzle moves to piece (row & 7) of a 128-byte row, ((row >> 1) & 3) of a 64-byte row
+        __syncthreads();
+        for (uint32_t i = threadIdx.x; i < (uint32_t)S * 128u; i += kThreads) {
+            const uint32_t s = i >> 7, r = i & 127u;
+            const uint32_t piece = rbA == 128u ? (r & 7u) : ((r >> 1) & 3u);
+            *reinterpret_cast<bf16 *>(smem + (size_t)s * stage_bytes + (size_t)a.ones_blk * 128u * rbA + r * rbA + piece * 16u) =
+                __float2bfloat16_rn(1.f);
+        }
+    }
+    fence_async_smem();
     if (warp == 1) tmem_alloc(&pipe->tmem_slot, ncols);
     tc_fence_before();
     __syncthreads();
@@ -721,6 +738,11 @@ __global__ void __launch_bounds__(kThreads, 1) tma_wgrad_kernel(const __grid_con
                 if (co0 + c0 >= a.Co) break;
                 float v[16];
                 tmem_ld16(lane_base + (uint32_t)c0, v);
+                if (ones_tile && p == a.ones_blk * a.CB) {
+#pragma unroll
+                    for (int i = 0; i < 16; ++i)
+                        if (co0 + c0 + i < a.Co) atomicAdd(a.db + co0 + c0 + i, v[i]);
+                }
                 if (jj >= a.Kfwd) continue;
 #pragma unroll
                 for (int i = 0; i < 16; ++i) {
@@ -1115,7 +1137,7 @@ int tma_dgrad_weights(const bf16 *W, bf16 *Wc, int Co, int k, int Ci, int wt_ld,
     return PPO_OK;
 }
 
-int tma_gemm_wgrad(const ConvGeom &g, const bf16 *dY, int ldy, const bf16 *X, float *dW, int32_t *status,
+int tma_gemm_wgrad(const ConvGeom &g, const bf16 *dY, int ldy, const bf16 *X, float *dW, float *db, int32_t *status,
                    cudaStream_t st) {
     if (!status || g.Ci % 8 != 0 || ldy % 8 != 0 || g.taps() > kMaxTaps) return PPO_ERR_UNSUPPORTED;
     const bool flat = is_flat(g);
@@ -1159,7 +1181,19 @@ int tma_gemm_wgrad(const ConvGeom &g, const bf16 *dY, int ldy, const bf16 *X, fl
     if (a.stages < 2) return PPO_ERR_UNSUPPORTED;
     s = ensure_smem_attrs();
     if (s != PPO_OK) return s;
-    const int jtiles = (a.ntaps * a.kchunks + a.mblocks - 1) / a.mblocks, ctiles = g.Co / a.BN;
+    int jtiles = (a.ntaps * a.kchunks + a.mblocks - 1) / a.mblocks;
+    const int ctiles = g.Co / a.BN;
+    if (db) {
+        // the ones column goes into the first unused block of the last column tile; when every block is
+        // taken, one more tile carries it alone
+        if (flat || g.Ci % CB != 0) return PPO_ERR_UNSUPPORTED;
+        a.db = db;
+        a.ones_blk = a.ntaps * a.kchunks - (jtiles - 1) * a.mblocks;
+        if (a.ones_blk == a.mblocks) {
+            a.ones_blk = 0;
+            ++jtiles;
+        }
+    }
     int splits = (two ? 2 : 1) * ppo_num_sms() / (jtiles * ctiles);
     if (splits < 1) splits = 1;
     if (splits > a.grid.tiles) splits = a.grid.tiles;

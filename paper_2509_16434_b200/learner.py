@@ -97,8 +97,9 @@ class Learner:
             ppo.ppo_loss_fwd_bwd(self.model, self.mb, r0, rows, B, self.mean, self.value, h.clip, h.vf_coef,
                                  h.ent_coef, self.loss, self.dmean, self.dvalue)
             ppo.ppo_encoder_bwd(self.model, self.mb, r0, rows, self.dmean, self.dvalue, True)
-            # fwd: conv1 + GEMMs + pool; loss: 2; bwd: pack + 3 per GEMM layer + unpool + conv1 wgrad
-            self.launches += (1 + n_layers_gemm + 1) + 2 + (1 + 3 * n_layers_gemm + 1 + 1)
+            # fwd: conv1 + GEMMs + pool; loss: 2; bwd: pack + (wgrad, bias sum, dgrad) per GEMM layer + unpool +
+            # conv1 wgrad; the wgrad of a convolution sums the bias gradient itself
+            self.launches += (1 + n_layers_gemm + 1) + 2 + (1 + 3 * n_layers_gemm - (len(w.conv_c) - 1) + 1 + 1)
         self.adam_t += 1
         ppo.ppo_adam_step(self.model, h.lr, h.beta1, h.beta2, h.eps, self.adam_t)
         self.launches += 1
