@@ -333,6 +333,7 @@ def run_ours(args):
                      "frac": round(adam_gbs / peaks["hbm_gbs"], 4), "ms": round(adam_ms, 4),
                      "note": "working set fits L2; launch-latency bound at this size"},
         }
+        rollout = time_rollout_inference(L, roll, w)
         cpu = cpu_baseline(w, roll, L) if world == 1 and not args.no_cpu_baseline else None
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -348,11 +349,30 @@ def run_ours(args):
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": 20,
                     "steps": e2e_steps, "ms_per_step": e2e_ms / e2e_steps},
             "gpu_launches": launches, "clocks": clocks, "roofline": roofline, "roofline_other_kernels": others,
-            "cpu_baseline": cpu, "loss_last_minibatch": loss,
+            "cpu_baseline": cpu, "loss_last_minibatch": loss, "rollout_inference": rollout,
         }
         print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
+
+
+def time_rollout_inference(L, roll, w, calls=8):
+    """The step before the path (Algorithm 2, actions <- pi(obs)): encoder forward over all N envs of one time step
+    plus Gaussian sampling and log-density, outside the timed region of the headline metric."""
+    import torch
+    for t in range(min(2, w.T)):
+        L.act(roll["depth"][t], roll["proprio"][t], roll["eps"][t])
+    s, e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    s.record()
+    for i in range(calls):
+        t = i % w.T
+        L.act(roll["depth"][t], roll["proprio"][t], roll["eps"][t])
+    e.record()
+    torch.cuda.synchronize()
+    ms = s.elapsed_time(e) / calls
+    return {"value": w.N / (ms * 1e-3), "unit": "env-steps acted/s", "ms_per_call": round(ms, 4), "rows": w.N,
+            "note": "ppo_encoder_fwd + ppo_policy_sample over all envs of one time step; not part of `value`"}
 
 
 # ---------------------------------------------------------------- CPU baseline ----
