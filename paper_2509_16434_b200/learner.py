@@ -99,7 +99,9 @@ class Learner:
             ppo.ppo_encoder_bwd(self.model, self.mb, r0, rows, self.dmean, self.dvalue, True)
             # fwd: conv1 + GEMMs + pool; loss: 2; bwd: pack + (wgrad, bias sum, dgrad) per GEMM layer + unpool +
             # conv1 wgrad; the wgrad of a convolution sums the bias gradient itself
-            self.launches += (1 + n_layers_gemm + 1) + 2 + (1 + 3 * n_layers_gemm - (len(w.conv_c) - 1) + 1 + 1)
+            # (a bias sum wider than 256 columns runs one launch per 256-column slab)
+            slabs = sum(o // 256 - 1 for o in w.fc if o > 256 and o % 256 == 0)
+            self.launches += (1 + n_layers_gemm + 1) + 2 + (1 + 3 * n_layers_gemm - (len(w.conv_c) - 1) + slabs + 1 + 1)
         self.adam_t += 1
         ppo.ppo_adam_step(self.model, h.lr, h.beta1, h.beta2, h.eps, self.adam_t)
         self.launches += 1
