@@ -82,6 +82,9 @@ struct ppo_model {
     int last_row0, last_rows;
     bool fwd_valid;
     int impl;  // 0 = tensor-core GEMMs, 1 = CUDA-core reference GEMMs
+    // second stream of the backward pass with its fork and join events (made on first use)
+    cudaStream_t side = nullptr;
+    cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
 };
 
 __device__ __forceinline__ float bf2f(bf16 x) { return __bfloat162float(x); }

@@ -721,6 +721,82 @@ static int refresh_transposed(ppo_model *m, cudaStream_t st) {
     return PPO_OK;
 }
 
+// Second stream and the two events of the fork/join in the backward pass, made on first use.
+static int side_stream(ppo_model *m) {
+    if (m->side) return PPO_OK;
+    PPO_CUDA_CHECK(cudaStreamCreateWithFlags(&m->side, cudaStreamNonBlocking));
+    PPO_CUDA_CHECK(cudaEventCreateWithFlags(&m->ev_fork, cudaEventDisableTiming));
+    PPO_CUDA_CHECK(cudaEventCreateWithFlags(&m->ev_join, cudaEventDisableTiming));
+    return PPO_OK;
+}
+
+// conv1: weight and bias gradients only (there is no dgrad into the depth image).
+static int conv1_wgrad(ppo_model *m, const ppo_minibatch *mb, int row0, int rows, cudaStream_t st) {
+    const ppo_model_desc &d = m->d;
+    const __half *depth = static_cast<const __half *>(mb->depth_f16) + (size_t)row0 * d.H * d.W;
+    const int C1 = m->Cs[1], KS = d.conv_k[0];
+    const long long M = (long long)rows * m->Hs[1] * m->Ws[1];
+    if (m->impl == 0 && C1 % 16 == 0 && C1 <= 64 && (KS == 3 || KS == 5)) {
+        // tensor-core reduction
+        const int TP = (KS * KS + 1 + 15) / 16 * 16;
+        const size_t tile = (size_t)32 * TP * 2 + (size_t)32 * C1 * 2, redb = (size_t)TP * C1 * sizeof(float);
+        const size_t smem = 8 * (tile > redb ? tile : redb);
+        int blocks = ppo_cdiv(M, 8 * 16 * 8);
+        const int cap = ppo_num_sms() * 4;
+        blocks = blocks > cap ? cap : (blocks < 1 ? 1 : blocks);
+        long long per_warp = (M + (long long)blocks * 8 - 1) / ((long long)blocks * 8);
+        per_warp = (per_warp + 31) / 32 * 32;
+        float *dW = m->grad + m->tensors[0].off, *db = m->grad + m->tensors[1].off;
+#define PPO_C1W(KS_, NB_)                                                                                    \
+    do {                                                                                                     \
+        if (smem > 48 * 1024)                                                                                \
+            PPO_CUDA_CHECK(cudaFuncSetAttribute(conv1_wgrad_mma_kernel<KS_, NB_>,                            \
+                                                cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));    \
+        conv1_wgrad_mma_kernel<KS_, NB_><<<blocks, 256, smem, st>>>(depth, m->dact[1], dW, db, rows, d.H,    \
+                                                                    d.W, m->Hs[1], m->Ws[1], per_warp);      \
+    } while (0)
+        const int nb = C1 / 8;
+        if (KS == 3 && nb == 2) PPO_C1W(3, 2);
+        else if (KS == 3 && nb == 4) PPO_C1W(3, 4);
+        else if (KS == 3 && nb == 6) PPO_C1W(3, 6);
+        else if (KS == 3 && nb == 8) PPO_C1W(3, 8);
+        else if (KS == 5 && nb == 2) PPO_C1W(5, 2);
+        else if (KS == 5 && nb == 4) PPO_C1W(5, 4);
+        else if (KS == 5 && nb == 6) PPO_C1W(5, 6);
+        else PPO_C1W(5, 8);
+#undef PPO_C1W
+        PPO_LAUNCH_CHECK();
+        return PPO_OK;
+    }
+    const int cpt = KS <= 3 ? 8 : (KS == 5 ? 4 : 2);
+    const int lpp = C1 / cpt;
+    if (C1 % cpt != 0 || lpp > 32 || (lpp & (lpp - 1)) != 0) return PPO_ERR_UNSUPPORTED;
+    const int ppi = 32 / lpp;
+    const size_t smem = (size_t)4 * C1 * (KS * KS + 1) * sizeof(float);
+    int blocks = ppo_cdiv(M, 4 * 256);
+    const int cap = ppo_num_sms() * 6;
+    blocks = blocks > cap ? cap : (blocks < 1 ? 1 : blocks);
+    long long per_warp = (M + (long long)blocks * 4 - 1) / ((long long)blocks * 4);
+    per_warp = (per_warp + ppi - 1) / ppi * ppi;
+    float *dW = m->grad + m->tensors[0].off, *db = m->grad + m->tensors[1].off;
+#define PPO_CONV1W(KS_, CPT_, U_)                                                                                 \
+    conv1_wgrad_kernel<KS_, CPT_, U_><<<blocks, 128, smem, st>>>(depth, m->dact[1], dW, db, rows, d.H, d.W,      \
+                                                             m->Hs[1], m->Ws[1], C1, per_warp)
+    if (smem > 48 * 1024) {
+        if (KS == 5) PPO_CUDA_CHECK(cudaFuncSetAttribute(conv1_wgrad_kernel<5, 4, 1>,
+                                                         cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        if (KS == 7) PPO_CUDA_CHECK(cudaFuncSetAttribute(conv1_wgrad_kernel<7, 2, 1>,
+                                                         cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    }
+    if (KS == 1) PPO_CONV1W(1, 8, 2);
+    else if (KS == 3) PPO_CONV1W(3, 8, 2);
+    else if (KS == 5) PPO_CONV1W(5, 4, 1);
+    else PPO_CONV1W(7, 2, 1);
+#undef PPO_CONV1W
+    PPO_LAUNCH_CHECK();
+    return PPO_OK;
+}
+
 extern "C" int ppo_encoder_bwd(ppo_model *m, const ppo_minibatch *mb, int row0, int rows, const float *dmean,
                                const float *dvalue, int accumulate, void *stream) {
     PPO_TRY(check_rows(m, mb, row0, rows));
@@ -735,6 +811,26 @@ extern "C" int ppo_encoder_bwd(ppo_model *m, const ppo_minibatch *mb, int row0, 
 
     pack_dout_kernel<<<ppo_cdiv((long long)rows * 16, 256), 256, 0, st>>>(dmean, dvalue, m->dh[F + 1], rows, d.A);
     PPO_LAUNCH_CHECK();
+    // Weight and bias gradients are leaves of the dependency graph: only the chain of dgrads has to run in order.
+    // The leaves of the FC layers (small kernels on a fraction of the SMs) and, further down, conv1's wgrad go to
+    // a second stream that forks from the caller's stream whenever the gradient they read is ready and joins it
+    // at the end of the call.
+    const bool fork = m->impl == 0 && side_stream(m) == PPO_OK;
+    cudaStream_t leaf = fork ? m->side : st;
+    auto fork_here = [&]() -> int {
+        if (!fork) return PPO_OK;
+        PPO_CUDA_CHECK(cudaEventRecord(m->ev_fork, st));
+        PPO_CUDA_CHECK(cudaStreamWaitEvent(m->side, m->ev_fork, 0));
+        return PPO_OK;
+    };
+    auto join = [&](int status) -> int {
+        if (fork) {
+            PPO_CUDA_CHECK(cudaEventRecord(m->ev_join, m->side));
+            PPO_CUDA_CHECK(cudaStreamWaitEvent(st, m->ev_join, 0));
+        }
+        return status;
+    };
+    PPO_TRY(fork_here());
     // head and hidden FC layers, last to first; layer index F+1 is the head
     for (int l = F + 1; l >= 1; --l) {
         const int ti = 2 * L + 2 * (l - 1);
@@ -742,11 +838,14 @@ extern "C" int ppo_encoder_bwd(ppo_model *m, const ppo_minibatch *mb, int row0, 
         const int ldy = (l <= F) ? Co : 16;
         ConvGeom g = fc_geom(rows, m->hw[l - 1], Co);
         const bf16 *dY = m->dh[l];
-        PPO_TRY(run_wgrad(m, g, dY, ldy, m->h[l - 1], m->grad + m->tensors[ti].off, m->grad + m->tensors[ti + 1].off, st));
+        int s = run_wgrad(m, g, dY, ldy, m->h[l - 1], m->grad + m->tensors[ti].off, m->grad + m->tensors[ti + 1].off, leaf);
+        if (s != PPO_OK) return join(s);
         DgradEpilogue e;
         if (l > 1) e = {m->h[l - 1], m->dh[l - 1], nullptr};
         else e = {nullptr, nullptr, m->dh0_f32};
-        PPO_TRY(run_dgrad(m, g, dY, ldy, m->shadow + m->tensors[ti].off, m->wT + m->wT_off[ti], wt_ld_of(Co), nullptr, e, st));
+        s = run_dgrad(m, g, dY, ldy, m->shadow + m->tensors[ti].off, m->wT + m->wT_off[ti], wt_ld_of(Co), nullptr, e, st);
+        if (s == PPO_OK && l > 1) s = fork_here();  // dh[l-1] is ready for the next leaf
+        if (s != PPO_OK) return join(s);
     }
     {
         const int npx = m->Hs[L] * m->Ws[L], C = m->Cs[L];
@@ -755,78 +854,28 @@ extern "C" int ppo_encoder_bwd(ppo_model *m, const ppo_minibatch *mb, int row0, 
                                                            m->hw[0]);
         PPO_LAUNCH_CHECK();
     }
+    // conv2's wgrad and conv1's wgrad are the two kernels of the pass that leave most of an SM idle, and they
+    // do not depend on each other: once conv2's dgrad has produced dZ1 they run side by side.
     for (int l = L; l >= 2; --l) {
         const int ti = 2 * (l - 1);
         ConvGeom g = conv_geom(m, l, rows);
-        PPO_TRY(run_wgrad(m, g, m->dact[l], g.Co, m->act[l - 1], m->grad + m->tensors[ti].off,
-                          m->grad + m->tensors[ti + 1].off, st));
         DgradEpilogue e = {m->act[l - 1], m->dact[l - 1], nullptr};
         e.mask_bits = m->abits[l - 1];
-        PPO_TRY(run_dgrad(m, g, m->dact[l], g.Co, m->shadow + m->tensors[ti].off, m->wT + m->wT_off[ti],
-                          wt_ld_of(g.Co), m->wC + m->wC_off[l], e, st));
-    }
-    {   // conv1: weight and bias gradients only
-        const __half *depth = static_cast<const __half *>(mb->depth_f16) + (size_t)row0 * d.H * d.W;
-        const int C1 = m->Cs[1], KS = d.conv_k[0];
-        const long long M = (long long)rows * m->Hs[1] * m->Ws[1];
-        if (m->impl == 0 && C1 % 16 == 0 && C1 <= 64 && (KS == 3 || KS == 5)) {
-            // tensor-core reduction
-            const int TP = (KS * KS + 1 + 15) / 16 * 16;
-            const size_t tile = (size_t)32 * TP * 2 + (size_t)32 * C1 * 2, redb = (size_t)TP * C1 * sizeof(float);
-            const size_t smem = 8 * (tile > redb ? tile : redb);
-            int blocks = ppo_cdiv(M, 8 * 16 * 8);
-            const int cap = ppo_num_sms() * 4;
-            blocks = blocks > cap ? cap : (blocks < 1 ? 1 : blocks);
-            long long per_warp = (M + (long long)blocks * 8 - 1) / ((long long)blocks * 8);
-            per_warp = (per_warp + 31) / 32 * 32;
-            float *dW = m->grad + m->tensors[0].off, *db = m->grad + m->tensors[1].off;
-#define PPO_C1W(KS_, NB_)                                                                                       \
-    do {                                                                                                        \
-        if (smem > 48 * 1024)                                                                                   \
-            PPO_CUDA_CHECK(cudaFuncSetAttribute(conv1_wgrad_mma_kernel<KS_, NB_>,                               \
-                                                cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));       \
-        conv1_wgrad_mma_kernel<KS_, NB_><<<blocks, 256, smem, st>>>(depth, m->dact[1], dW, db, rows, d.H, d.W, \
-                                                                    m->Hs[1], m->Ws[1], per_warp);              \
-    } while (0)
-            const int nb = C1 / 8;
-            if (KS == 3 && nb == 2) PPO_C1W(3, 2);
-            else if (KS == 3 && nb == 4) PPO_C1W(3, 4);
-            else if (KS == 3 && nb == 6) PPO_C1W(3, 6);
-            else if (KS == 3 && nb == 8) PPO_C1W(3, 8);
-            else if (KS == 5 && nb == 2) PPO_C1W(5, 2);
-            else if (KS == 5 && nb == 4) PPO_C1W(5, 4);
-            else if (KS == 5 && nb == 6) PPO_C1W(5, 6);
-            else PPO_C1W(5, 8);
-#undef PPO_C1W
-            PPO_LAUNCH_CHECK();
-            return PPO_OK;
+        const bool after = fork && l == 2;  // conv2: dgrad first, so that conv1's wgrad can start beside the wgrad
+        int s = PPO_OK;
+        if (!after)
+            s = run_wgrad(m, g, m->dact[l], g.Co, m->act[l - 1], m->grad + m->tensors[ti].off,
+                          m->grad + m->tensors[ti + 1].off, st);
+        if (s == PPO_OK)
+            s = run_dgrad(m, g, m->dact[l], g.Co, m->shadow + m->tensors[ti].off, m->wT + m->wT_off[ti],
+                          wt_ld_of(g.Co), m->wC + m->wC_off[l], e, st);
+        if (s == PPO_OK && after) {
+            s = fork_here();
+            if (s == PPO_OK)
+                s = run_wgrad(m, g, m->dact[l], g.Co, m->act[l - 1], m->grad + m->tensors[ti].off,
+                              m->grad + m->tensors[ti + 1].off, st);
         }
-        const int cpt = KS <= 3 ? 8 : (KS == 5 ? 4 : 2);
-        const int lpp = C1 / cpt;
-        if (C1 % cpt != 0 || lpp > 32 || (lpp & (lpp - 1)) != 0) return PPO_ERR_UNSUPPORTED;
-        const int ppi = 32 / lpp;
-        const size_t smem = (size_t)4 * C1 * (KS * KS + 1) * sizeof(float);
-        int blocks = ppo_cdiv(M, 4 * 256);
-        const int cap = ppo_num_sms() * 6;
-        blocks = blocks > cap ? cap : (blocks < 1 ? 1 : blocks);
-        long long per_warp = (M + (long long)blocks * 4 - 1) / ((long long)blocks * 4);
-        per_warp = (per_warp + ppi - 1) / ppi * ppi;
-        float *dW = m->grad + m->tensors[0].off, *db = m->grad + m->tensors[1].off;
-#define PPO_CONV1W(KS_, CPT_, U_)                                                                                 \
-    conv1_wgrad_kernel<KS_, CPT_, U_><<<blocks, 128, smem, st>>>(depth, m->dact[1], dW, db, rows, d.H, d.W,      \
-                                                                 m->Hs[1], m->Ws[1], C1, per_warp)
-        if (smem > 48 * 1024) {
-            if (KS == 5) PPO_CUDA_CHECK(cudaFuncSetAttribute(conv1_wgrad_kernel<5, 4, 1>,
-                                                             cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-            if (KS == 7) PPO_CUDA_CHECK(cudaFuncSetAttribute(conv1_wgrad_kernel<7, 2, 1>,
-                                                             cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        }
-        if (KS == 1) PPO_CONV1W(1, 8, 2);
-        else if (KS == 3) PPO_CONV1W(3, 8, 2);
-        else if (KS == 5) PPO_CONV1W(5, 4, 1);
-        else PPO_CONV1W(7, 2, 1);
-#undef PPO_CONV1W
-        PPO_LAUNCH_CHECK();
+        if (s != PPO_OK) return join(s);
     }
-    return PPO_OK;
+    return join(conv1_wgrad(m, mb, row0, rows, L >= 2 ? leaf : st));
 }

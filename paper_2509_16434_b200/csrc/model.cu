@@ -96,6 +96,12 @@ extern "C" int ppo_model_create(const ppo_model_desc *d, ppo_model **out) {
 
 extern "C" int ppo_model_destroy(ppo_model *m) {
     if (!m) return PPO_ERR_INVALID_ARG;
+    if (m->side) {
+        cudaStreamSynchronize(m->side);
+        cudaStreamDestroy(m->side);
+        cudaEventDestroy(m->ev_fork);
+        cudaEventDestroy(m->ev_join);
+    }
     delete m;
     return PPO_OK;
 }
