@@ -235,7 +235,10 @@ int ppo_loss_fwd_bwd(ppo_model *m, const ppo_minibatch *mb, int row0, int rows, 
 /* Backward of the rows of the latest ppo_encoder_fwd (same row0/rows, else STATE): adds
  * (accumulate != 0) or writes (accumulate == 0, the log-sigma slot is left as it is)
  * dL/dtheta into the bound gradient array, with respect to the fp32 master (straight
- * through the bf16 rounding). */
+ * through the bf16 rounding).  Weight-gradient kernels that do not feed the chain of
+ * input gradients run on a second stream the model creates at its first backward pass;
+ * that stream forks from `stream` and has joined it again when the call returns, so the
+ * caller sees the ordering of a single stream. */
 int ppo_encoder_bwd(ppo_model *m, const ppo_minibatch *mb, int row0, int rows, const float *dev_dmean,
                     const float *dev_dvalue, int accumulate, void *stream);
 
