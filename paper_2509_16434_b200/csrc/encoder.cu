@@ -854,28 +854,35 @@ extern "C" int ppo_encoder_bwd(ppo_model *m, const ppo_minibatch *mb, int row0, 
                                                            m->hw[0]);
         PPO_LAUNCH_CHECK();
     }
-    // conv2's wgrad and conv1's wgrad are the two kernels of the pass that leave most of an SM idle, and they
-    // do not depend on each other: once conv2's dgrad has produced dZ1 they run side by side.
+    // The chain of dgrads first; then the wgrads of the GEMM layers one after the other on the caller's stream
+    // with conv1's wgrad beside them on the second one.  A wgrad GEMM takes most of an SM's shared memory but
+    // few registers and threads, conv1's wgrad the opposite, and both leave most issue slots and half the DRAM
+    // bandwidth unused on their own, so they share the SMs.  (The dgrad kernels take whole SMs: nothing fits
+    // beside them.)  Without a second stream the order is the plain one: wgrad, dgrad, layer by layer.
     for (int l = L; l >= 2; --l) {
         const int ti = 2 * (l - 1);
         ConvGeom g = conv_geom(m, l, rows);
         DgradEpilogue e = {m->act[l - 1], m->dact[l - 1], nullptr};
         e.mask_bits = m->abits[l - 1];
-        const bool after = fork && l == 2;  // conv2: dgrad first, so that conv1's wgrad can start beside the wgrad
         int s = PPO_OK;
-        if (!after)
+        if (!fork)
             s = run_wgrad(m, g, m->dact[l], g.Co, m->act[l - 1], m->grad + m->tensors[ti].off,
                           m->grad + m->tensors[ti + 1].off, st);
         if (s == PPO_OK)
             s = run_dgrad(m, g, m->dact[l], g.Co, m->shadow + m->tensors[ti].off, m->wT + m->wT_off[ti],
                           wt_ld_of(g.Co), m->wC + m->wC_off[l], e, st);
-        if (s == PPO_OK && after) {
-            s = fork_here();
-            if (s == PPO_OK)
-                s = run_wgrad(m, g, m->dact[l], g.Co, m->act[l - 1], m->grad + m->tensors[ti].off,
-                              m->grad + m->tensors[ti + 1].off, st);
-        }
         if (s != PPO_OK) return join(s);
     }
-    return join(conv1_wgrad(m, mb, row0, rows, L >= 2 ? leaf : st));
+    if (fork && L >= 2) {
+        int s = fork_here();  // dZ1 is ready
+        if (s == PPO_OK) s = conv1_wgrad(m, mb, row0, rows, leaf);
+        for (int l = 2; l <= L && s == PPO_OK; ++l) {  // conv2 first: the longest, and the best partner
+            const int ti = 2 * (l - 1);
+            ConvGeom g = conv_geom(m, l, rows);
+            s = run_wgrad(m, g, m->dact[l], g.Co, m->act[l - 1], m->grad + m->tensors[ti].off,
+                          m->grad + m->tensors[ti + 1].off, st);
+        }
+        return join(s);
+    }
+    return join(conv1_wgrad(m, mb, row0, rows, st));
 }
