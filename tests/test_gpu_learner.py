@@ -300,3 +300,43 @@ def test_forward_writes_the_relu_gate_bits_of_its_activations():
         assert np.array_equal(got, want_words), f"layer {l}: recomputed gates"
         checked += 1
     assert checked >= 2 and ppo.ppo_poll_status() == 0
+
+
+def test_backward_on_a_caller_stream_orders_like_one_stream():
+    """The backward pass forks a second stream for its weight-gradient leaves and joins it before returning: run on a
+    caller's stream (not the default one), twice in a row, it must give the gradients of the default-stream run, and
+    work enqueued behind it on the caller's stream (the copy below) must see all of them."""
+    w = SHAPES["cfg2_twin"]
+    L, md, lay, theta, roll, action, logp, dev = _setup(w, 8)
+    h = L.hyper
+    K = w.minibatches
+    B = w.M // K
+    L.compute_gae(dev["last_value"])
+    ppo.ppo_shuffle_gather_minibatch(L.buffer, 5, 0, 0, K, L.mb)
+
+    def one_pass(out):
+        ppo.ppo_model_zero_grad(L.model)
+        L.loss.zero_()
+        for r0 in range(0, B, L.microbatch):
+            rows = min(L.microbatch, B - r0)
+            ppo.ppo_encoder_fwd(L.model, L.mb, r0, rows, L.mean, L.value)
+            ppo.ppo_loss_fwd_bwd(L.model, L.mb, r0, rows, B, L.mean, L.value, h.clip, h.vf_coef, h.ent_coef, L.loss,
+                                 L.dmean, L.dvalue)
+            ppo.ppo_encoder_bwd(L.model, L.mb, r0, rows, L.dmean, L.dvalue, True)
+        out.copy_(L.model.grad, non_blocking=True)  # same stream: ordered after the join
+
+    ref = torch.empty_like(L.model.grad)
+    one_pass(ref)
+    torch.cuda.synchronize()
+    s = torch.cuda.Stream()
+    s.wait_stream(torch.cuda.current_stream())
+    got = [torch.empty_like(ref), torch.empty_like(ref)]
+    with torch.cuda.stream(s):
+        one_pass(got[0])
+        one_pass(got[1])
+    s.synchronize()
+    assert ppo.ppo_poll_status() == 0
+    r = ref.cpu().numpy()
+    assert np.abs(r).max() > 0
+    for g in got:  # wgrad adds fp32 partial sums with atomics: equal up to their order
+        assert rel_l2(g.cpu().numpy(), r) <= 1e-5
