@@ -1068,10 +1068,11 @@ int tma_gemm_dgrad(const ConvGeom &g, const bf16 *dY, int ldy, const bf16 *Wt, i
     int dmin, n1;
     tma_dgrad_shifts(g.k, &dmin, &n1);
     const int nshift = n1 * n1, Ntot = 4 * g.Ci;
-    // 256 merged columns (C_in = 64) go as two groups of 128: the row-parity-0 group has taps at two of the four
-    // shifts only, so a quarter of the MMAs (all multiplications by zero weights) fall away, and tiles of 128
-    // columns run two CTAs per SM
-    a.BN = Ntot == 256 ? 128 : pick_bn(Ntot);
+    // 256 or 512 merged columns (C_in = 64, 128) go as groups of 128: a group takes only the shifts at which its
+    // parity classes have taps (6 of 8 group-shift pairs for two groups, 9 of 16 for four: one per kernel tap),
+    // so the multiplications by zero weights of a single wide GEMM fall away, at the same operand bytes, and tiles
+    // of 128 columns run two CTAs per SM
+    a.BN = (Ntot == 256 || Ntot == 512) ? 128 : pick_bn(Ntot);
     if (Ntot % a.BN != 0 || Ntot / a.BN > 4 || nshift > kMaxTaps) return PPO_ERR_UNSUPPORTED;
     a.N = a.BN;  // every group is one full tile of columns
     a.nq_ci = g.Ci;
