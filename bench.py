@@ -27,7 +27,7 @@ import numpy as np
 ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
-NCU_DRAM_BYTES_PER_ROW = (1059.8e6 + 334.0e6) / 512
+NCU_DRAM_BYTES_PER_ROW = (1062.2e6 + 333.4e6) / 512
 METRIC = "ppo_learner_env_steps_trained_per_sec"
 UNIT = "env-steps/s"
 
