@@ -7,7 +7,9 @@ encoder forward, fused loss, encoder backward and Adam.  The metric is env-steps
 per second = M * epochs / time, with the buffer resident in HBM (`value`) and with the
 rollout arriving from pinned host memory every step (`e2e`).
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg2] [--impl reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg4] [--impl reference]
+
+The default workload is the largest single-GPU configuration (cfg4: 8192 envs x 16 steps of 320x240 depth).
 
 With N > 1 (torchrun) every rank trains an independent replica on its own buffer: the
 path has no exchange step on one learner GPU, so there is no collective on the data path.
@@ -27,7 +29,10 @@ import numpy as np
 ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
-NCU_DRAM_BYTES_PER_ROW = (1062.2e6 + 333.4e6) / 512
+# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of the encoder kernels of one forward + backward per
+# sample row, from ncu captures of small twins of the workloads (traffic grows in proportion to the rows): workload
+# -> (bytes per row, capture).  An entry is dropped (traffic: null) as soon as a kernel it covers changes.
+NCU_DRAM_BYTES_PER_ROW = {}
 METRIC = "ppo_learner_env_steps_trained_per_sec"
 UNIT = "env-steps/s"
 
@@ -236,7 +241,7 @@ def run_ours(args):
         setattr(ppo, n, timer.wrap(n, originals[n]))
     vis = os.environ.get("CUDA_VISIBLE_DEVICES", "").split(",")
     sampler = ClockSampler(vis[local] if local < len(vis) and vis[local].strip().isdigit() else local)
-    launches0 = L.launches
+    launches0 = ppo.ppo_launch_count()
     if rank == 0:
         sampler.start()
     t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -255,40 +260,69 @@ def run_ours(args):
     status = ppo.ppo_poll_status()
     if status != 0:
         raise RuntimeError(f"device status {status} ({ppo.ppo_status_string(status)})")
-    launches = L.launches - launches0
+    launches = ppo.ppo_launch_count() - launches0
     loss = L.loss.cpu().numpy().tolist()
 
-    # ---- end to end: rollout arrives from pinned host memory every step, loss read back
+    # ---- end to end: every step's rollout arrives from pinned host memory through ppo_buffer_write_step and the loss
+    # scalars are read back.  Two device buffers alternate: the copies of the next rollout run on a second stream
+    # while the learner trains on the current one (the simulator side collects while the learner trains), and a step
+    # only starts once its own rollout has landed.
     host = {k: torch.empty(v.shape, dtype=v.dtype, pin_memory=True) for k, v in roll.items()
             if k in ("depth", "proprio", "action", "logp", "value", "reward", "done", "last_value")}
     for k in host:
         host[k].copy_(roll[k])
-    stage = {k: torch.empty_like(roll[k][0]) for k in host if k != "last_value"}
-    lastv = torch.empty_like(roll["last_value"])
+    del roll["depth"]
+    torch.cuda.empty_cache()
+    stage = [{k: torch.empty_like(host[k][0], device=device) for k in host if k != "last_value"} for _ in range(2)]
+    lastv = [torch.empty_like(roll["last_value"]) for _ in range(2)]
     h2d = sum(v.numel() * v.element_size() for v in host.values())
     loss_host = torch.empty(5, dtype=torch.float32, pin_memory=True)
+    bufs = [L.buffer, ppo.Buffer(L.bdesc, device)]
+    copy_stream = torch.cuda.Stream(device=device)
+    landed = [torch.cuda.Event(), torch.cuda.Event()]
+    trained = [torch.cuda.Event(), torch.cuda.Event()]
+    main = torch.cuda.current_stream()
 
-    def e2e_step(seed):
-        for t in range(w.T):
-            for k in stage:
-                stage[k].copy_(host[k][t], non_blocking=True)
-            ppo.ppo_buffer_write_step(L.buffer, t, stage["depth"], stage["proprio"], stage["action"], stage["logp"],
-                                      stage["value"], stage["reward"], stage["done"])
-        lastv.copy_(host["last_value"], non_blocking=True)
-        L.train(lastv, seed=seed)
-        loss_host.copy_(L.loss, non_blocking=True)
-        torch.cuda.current_stream().synchronize()
+    def upload(i):
+        """Rollout of step i -> buffer i % 2, on the copy stream, once that buffer's previous training is done."""
+        b = i % 2
+        copy_stream.wait_event(trained[b])
+        with torch.cuda.stream(copy_stream):
+            for t in range(w.T):
+                st = stage[t % 2]
+                for k in st:
+                    st[k].copy_(host[k][t], non_blocking=True)
+                ppo.ppo_buffer_write_step(bufs[b], t, st["depth"], st["proprio"], st["action"], st["logp"],
+                                          st["value"], st["reward"], st["done"], stream=copy_stream)
+            lastv[b].copy_(host["last_value"], non_blocking=True)
+            landed[b].record(copy_stream)
 
-    e2e_steps = max(1, min(args.steps, 3))
-    e2e_step(7)
+    def e2e_run(n, seed0):
+        for b in range(2):
+            trained[b].record(main)
+        upload(0)
+        for i in range(n):
+            b = i % 2
+            if i + 1 < n:
+                upload(i + 1)
+            main.wait_event(landed[b])
+            L.buffer = bufs[b]
+            L.train(lastv[b], seed=seed0 + i)
+            trained[b].record(main)
+            loss_host.copy_(L.loss, non_blocking=True)
+            main.synchronize()
+
+    e2e_steps = max(1, min(args.steps, 5))
+    e2e_run(2, 7)
     barrier()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
-    for i in range(e2e_steps):
-        e2e_step(200 + i)
+    e2e_run(e2e_steps, 200)
     e1.record()
     barrier()
     e2e_ms = e0.elapsed_time(e1)
+    L.buffer = bufs[0]
+    del bufs[1]
 
     ms, e2e_ms = max_over_ranks([ms, e2e_ms], device)
     env_steps = w.M * w.epochs
@@ -315,12 +349,13 @@ def run_ours(args):
         # DRAM bytes of the encoder's GEMM and conv1 kernels per sample row (dram__bytes_read + write summed over the 18
         # launches of one forward + backward, ncu capture of the cfg2 network at 512 rows: profiles/ncu_main_kernels_cfg2_prof.md);
         # traffic grows in proportion to the rows.  Valid for the cfg2/cfg3 network only, and only while those kernels are unchanged.
-        traffic = NCU_DRAM_BYTES_PER_ROW * mean_rows if w.name in ("cfg2", "cfg3", "cfg2_prof") else None
+        per_row, capture = NCU_DRAM_BYTES_PER_ROW.get(w.name, (None, "no ncu capture of the current kernels at this workload"))
+        traffic = per_row * mean_rows if per_row else None
         roofline = {"bound": "tensor",
                     "kernel": "ppo_encoder_fwd + ppo_encoder_bwd: tma_kmajor_kernel / tma_wgrad_kernel (tcgen05 implicit GEMMs) "
                               "+ conv1 kernels; flops, time and traffic per call pair",
                     "achieved": round(enc_tf, 2), "peak": peak_tf, "unit": "TFLOP/s",
-                    "frac": round(enc_tf / peak_tf, 4), "traffic": traffic,
+                    "frac": round(enc_tf / peak_tf, 4), "traffic": traffic, "traffic_source": capture,
                     "peak_source": peaks["source"] + " (sustained bf16)",
                     "ms_per_call": {"fwd": round(fwd_ms, 4), "bwd": round(bwd_ms, 4), "rows": mean_rows}}
         others = {
@@ -333,11 +368,14 @@ def run_ours(args):
                      "frac": round(adam_gbs / peaks["hbm_gbs"], 4), "ms": round(adam_ms, 4),
                      "note": "working set fits L2; launch-latency bound at this size"},
         }
-        rollout = time_rollout_inference(L, roll, w)
-        cpu = cpu_baseline(w, roll, L) if world == 1 and not args.no_cpu_baseline else None
+        others["supplementary_scaled_inputs"] = hbm_resident_rows(peaks)
+        rollout = time_rollout_inference(L, host, w)
+        cpu = cpu_baseline(w, host, L) if world == 1 and not args.no_cpu_baseline else None
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-            "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
+            "warmup": args.warmup, "ms_per_step": ms / args.steps,
+            "ms_per_step_x_sm_ghz": (ms / args.steps * clocks["sm_mhz"] / 1e3) if clocks and clocks.get("sm_mhz") else None,
+            "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": {"workload": f"{w.name}: {w.N} envs x T={w.T}, depth 1x{w.H}x{w.W} fp16, conv "
                                    f"{'-'.join(map(str, w.conv_c))}, fc {'-'.join(map(str, w.fc))}, "
@@ -347,7 +385,8 @@ def run_ours(args):
                            w.M * record_bytes(w) / 1e6, L.model.workspace.numel() / 1e6),
                        "parallelism": "replicas only" if world > 1 else "single GPU"},
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": 20,
-                    "steps": e2e_steps, "ms_per_step": e2e_ms / e2e_steps},
+                    "steps": e2e_steps, "ms_per_step": e2e_ms / e2e_steps,
+                    "pipeline": "two device buffers; the next rollout's copies overlap the current step's training"},
             "gpu_launches": launches, "clocks": clocks, "roofline": roofline, "roofline_other_kernels": others,
             "cpu_baseline": cpu, "loss_last_minibatch": loss, "rollout_inference": rollout,
         }
@@ -356,23 +395,76 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
-def time_rollout_inference(L, roll, w, calls=8):
-    """The step before the path (Algorithm 2, actions <- pi(obs)): encoder forward over all N envs of one time step
-    plus Gaussian sampling and log-density, outside the timed region of the headline metric."""
+def time_rollout_inference(L, host, w, calls=8):
+    """The step before the path (Algorithm 2, actions <- pi(obs), D <- D U {...}): the observation of one time step is
+    written into its slab row, the encoder runs on it there and action, log-prob and value land in the same row
+    (ppo_buffer_write_obs + ppo_policy_act over all N envs), outside the timed region of the headline metric."""
     import torch
+    dev = L.device
+    depth = host["depth"][0].to(dev)
+    proprio = host["proprio"][0].to(dev)
+    eps = torch.randn((w.N, w.A), device=dev)
     for t in range(min(2, w.T)):
-        L.act(roll["depth"][t], roll["proprio"][t], roll["eps"][t])
+        L.act_into_buffer(t, depth, proprio, eps)
     s, e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     torch.cuda.synchronize()
     s.record()
     for i in range(calls):
-        t = i % w.T
-        L.act(roll["depth"][t], roll["proprio"][t], roll["eps"][t])
+        L.act_into_buffer(i % w.T, depth, proprio, eps)
     e.record()
     torch.cuda.synchronize()
     ms = s.elapsed_time(e) / calls
     return {"value": w.N / (ms * 1e-3), "unit": "env-steps acted/s", "ms_per_call": round(ms, 4), "rows": w.N,
-            "note": "ppo_encoder_fwd + ppo_policy_sample over all envs of one time step; not part of `value`"}
+            "note": "ppo_buffer_write_obs + ppo_policy_act over all envs of one time step; not part of `value`"}
+
+
+def hbm_resident_rows(peaks, warmup=3, steps=10):
+    """Supplementary, HBM-resident inputs (NOT configs): the GAE and Adam kernels on working sets far larger than L2,
+    to show their asymptotic bandwidth; at config sizes both finish inside a launch latency."""
+    import torch
+    from paper_2509_16434_b200 import binding as ppo
+    extra = []
+    T, N = 128, 524288
+    g = torch.Generator(device="cuda")
+    g.manual_seed(1)
+    reward = torch.randn((T, N), generator=g, device="cuda")
+    value = torch.randn((T, N), generator=g, device="cuda")
+    done = (torch.rand((T, N), generator=g, device="cuda") < 0.01).to(torch.uint8)
+    lastv = torch.randn(N, generator=g, device="cuda")
+    adv, ret = torch.empty_like(reward), torch.empty_like(reward)
+    ms = []
+    for it in range(warmup + steps):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        ppo.ppo_gae_static(reward, value, done, lastv, 0.99, 0.95, True, adv, ret)
+        e1.record()
+        torch.cuda.synchronize()
+        if it >= warmup:
+            ms.append(e0.elapsed_time(e1))
+    t = float(np.median(ms))
+    gbs = (17 + 8) * T * N / (t * 1e-3) / 1e9
+    extra.append({"kernel": "gae_scan + adv_normalize", "input": f"{N} envs x T={T} ({(17 + 8) * T * N / 1e9:.2f} GB moved)",
+                  "ms": round(t, 3), "GBs": round(gbs, 1), "frac_of_measured_hbm": round(gbs / peaks["hbm_gbs"], 4)})
+    del reward, value, done, adv, ret
+    md = ppo.model_desc(16, 16, (8,), (3,), (16384, 16384), 32, 12)
+    model = ppo.Model(md, 1)
+    model.grad.normal_(generator=g)
+    ms = []
+    for it in range(warmup + steps):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        ppo.ppo_adam_step(model, 3e-4, 0.9, 0.999, 1e-8, it + 1)
+        e1.record()
+        torch.cuda.synchronize()
+        if it >= warmup:
+            ms.append(e0.elapsed_time(e1))
+    t = float(np.median(ms))
+    gbs = 30 * model.arena / (t * 1e-3) / 1e9
+    extra.append({"kernel": "adam_kernel", "input": f"{model.arena} parameters ({30 * model.arena / 1e9:.2f} GB moved)",
+                  "ms": round(t, 3), "GBs": round(gbs, 1), "frac_of_measured_hbm": round(gbs / peaks["hbm_gbs"], 4)})
+    del model
+    torch.cuda.empty_cache()
+    return extra
 
 
 # ---------------------------------------------------------------- CPU baseline ----
@@ -400,17 +492,16 @@ def oracle_sample_step(w, fields, theta, n_samples):
     return t_gae, t_mb, out
 
 
-def cpu_baseline(w, roll, L, n_samples=None):
+def cpu_baseline(w, host, L, n_samples=None):
     """Times the oracle, as it stands, on this machine's host cores over a bounded sample of the same workload."""
     from oracle import oracle as orc
     import torch
     # about 10-30 s of oracle work on a 16-core host: ~0.4 / 7 / 35 ms per row at the three frame sizes
     n_samples = n_samples or min(w.B, 4096 if w.H * w.W <= 120 * 160 else 768)
     idx = orc.perm(w.seed, 0, w.M, 0, n_samples).astype(np.int64)
-    flat = roll["depth"].view(w.M, w.H, w.W)
-    fields = {k: roll[k].cpu().numpy() for k in ("proprio", "action", "logp", "value", "reward", "done",
-                                                 "last_value")}
-    fields["depth_rows"] = flat[torch.as_tensor(idx, device=flat.device)].cpu().numpy()
+    flat = host["depth"].view(w.M, w.H, w.W)   # the rollout as it sits in pinned host memory
+    fields = {k: host[k].numpy() for k in ("proprio", "action", "logp", "value", "reward", "done", "last_value")}
+    fields["depth_rows"] = flat[torch.as_tensor(idx)].numpy()
     theta = L.model.master.cpu().numpy()
     t_gae, t_mb, _ = oracle_sample_step(w, fields, theta, n_samples)
     # whole step = GAE once + M*E sample-passes at the measured per-sample minibatch cost
@@ -517,47 +608,7 @@ def run_stress(args):
         assert ppo.ppo_poll_status() == 0
         del buf, mb, depth
         torch.cuda.empty_cache()
-    # Supplementary, HBM-resident inputs (NOT configs): the GAE and Adam kernels on working sets far larger than L2,
-    # to show their asymptotic bandwidth; at config sizes both finish inside a launch latency.
-    extra = []
-    T, N = 128, 524288
-    g = torch.Generator(device="cuda")
-    g.manual_seed(1)
-    reward = torch.randn((T, N), generator=g, device="cuda")
-    value = torch.randn((T, N), generator=g, device="cuda")
-    done = (torch.rand((T, N), generator=g, device="cuda") < 0.01).to(torch.uint8)
-    lastv = torch.randn(N, generator=g, device="cuda")
-    adv, ret = torch.empty_like(reward), torch.empty_like(reward)
-    ms = []
-    for it in range(args.warmup + args.steps):
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record()
-        ppo.ppo_gae_static(reward, value, done, lastv, 0.99, 0.95, True, adv, ret)
-        e1.record()
-        torch.cuda.synchronize()
-        if it >= args.warmup:
-            ms.append(e0.elapsed_time(e1))
-    t = float(np.median(ms))
-    gbs = (17 + 8) * T * N / (t * 1e-3) / 1e9
-    extra.append({"kernel": "gae_scan + adv_normalize", "input": f"{N} envs x T={T} ({(17 + 8) * T * N / 1e9:.2f} GB moved)",
-                  "ms": round(t, 3), "GBs": round(gbs, 1), "frac_of_measured_hbm": round(gbs / peaks["hbm_gbs"], 4)})
-    del reward, value, done, adv, ret
-    md = ppo.model_desc(16, 16, (8,), (3,), (16384, 16384), 32, 12)
-    model = ppo.Model(md, 1)
-    model.grad.normal_(generator=g)
-    ms = []
-    for it in range(args.warmup + args.steps):
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record()
-        ppo.ppo_adam_step(model, 3e-4, 0.9, 0.999, 1e-8, it + 1)
-        e1.record()
-        torch.cuda.synchronize()
-        if it >= args.warmup:
-            ms.append(e0.elapsed_time(e1))
-    t = float(np.median(ms))
-    gbs = 30 * model.arena / (t * 1e-3) / 1e9
-    extra.append({"kernel": "adam_kernel", "input": f"{model.arena} parameters ({30 * model.arena / 1e9:.2f} GB moved)",
-                  "ms": round(t, 3), "GBs": round(gbs, 1), "frac_of_measured_hbm": round(gbs / peaks["hbm_gbs"], 4)})
+    extra = hbm_resident_rows(peaks, args.warmup, args.steps)
     print(json.dumps({"metric": "buffer_path_bandwidth", "unit": "GB/s", "peak_hbm_gbs": peaks["hbm_gbs"],
                       "peak_source": peaks["source"], "rows": rows, "supplementary_scaled_inputs": extra}))
 
@@ -568,7 +619,7 @@ def main():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="cfg2")
+    ap.add_argument("--workload", default="cfg4")
     ap.add_argument("--microbatch", type=int, default=4096)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--stress", action="store_true", help="bandwidth stress of the buffer path (GAE + gathers, T = 32)")

@@ -98,6 +98,14 @@ int ppo_buffer_write_step(ppo_buffer *buf, int t, const void *dev_depth_f16, con
                           const float *dev_action, const float *dev_logp, const float *dev_value,
                           const float *dev_reward, const uint8_t *dev_done, void *stream);
 
+/* The two halves of the same insertion for a rollout whose actions come from ppo_policy_act (Algorithm 2:
+ * obs arrives, actions <- pi(obs), the env step returns rew and done): ppo_buffer_write_obs copies the
+ * observation of step t (depth_f16 [N][H][W] fp16, proprio [N][P]) into slab row t before the policy runs,
+ * ppo_buffer_write_outcome the reward [N] fp32 and done [N] uint8 afterwards; action, log-prob and value of
+ * row t are written in place by ppo_policy_act.  Same errors and invalidation as ppo_buffer_write_step. */
+int ppo_buffer_write_obs(ppo_buffer *buf, int t, const void *dev_depth_f16, const float *dev_proprio, void *stream);
+int ppo_buffer_write_outcome(ppo_buffer *buf, int t, const float *dev_reward, const uint8_t *dev_done, void *stream);
+
 /* First stage of TrainPPO (Algorithm 2): generalised advantage estimation per env by a
  * reverse scan over t,
  *   delta_t = r_t + gamma V_{t+1} (1 - d_t) - V_t,  A_t = delta_t + gamma lambda (1 - d_t) A_{t+1},
@@ -269,6 +277,27 @@ int ppo_adam_step(ppo_model *m, float lr, float beta1, float beta2, float eps, i
  * action = mu + exp(logsigma) * eps, logp = its log-density.  Outputs fp32 [rows][A], [rows]. */
 int ppo_policy_sample(const ppo_model *m, int rows, const float *dev_mean, const float *dev_eps, float *dev_action,
                       float *dev_logp, void *stream);
+
+/* actions <- pi(stack(obs)) followed by D <- D U {...} without a copy in between (Algorithm 2): runs the
+ * encoder on the observation already stored in slab row t of `buf` (all N envs, in micro-batches of the bound
+ * size), draws action = mu + exp(logsigma) * eps from caller-supplied standard-normal noise dev_eps [N][A],
+ * and writes the action, its log-density and the value estimate straight into the ACTION, LOGP and VALUE
+ * slabs at row t (ppo_buffer_field_ptr gives the simulator the address to read the actions from).
+ * Invalidates advantages computed earlier and the saved activations of the last ppo_encoder_fwd.
+ * Errors: t outside [0,T) -> INVALID_ARG; buffer and model shapes (H, W, P, A) differ -> SHAPE. */
+int ppo_policy_act(ppo_model *m, ppo_buffer *buf, int t, const float *dev_eps, void *stream);
+
+/* Number of kernels and memsets the library has enqueued in this process so far (all handles, all
+ * devices).  Instrumentation for benchmarks that report launches per step; no counterpart in the paper. */
+uint64_t ppo_launch_count(void);
+
+/* Self-test of the bounded waits (no counterpart in the paper): every device-side wait of the pipelined
+ * kernels gives up after a cycle limit, records PPO_ERR_TIMEOUT in the status word and lets the kernel
+ * return.  This launches one small kernel whose 64 threads run that same wait, with a limit of
+ * limit_cycles (1 .. 2e9) clock cycles, on a barrier that nothing completes; *dev_gave_up (device int,
+ * zeroed by the caller) receives the number of threads that left the wait unsatisfied.  The next
+ * ppo_poll_status returns PPO_ERR_TIMEOUT and clears it; the device stays usable. */
+int ppo_selftest_wait_timeout(long long limit_cycles, int *dev_gave_up, void *stream);
 
 /* Synchronises `stream`, then returns the first error a kernel recorded in the library's
  * device status word since the last poll (PPO_OK if none), or PPO_ERR_CUDA if the stream

@@ -27,7 +27,8 @@ EXPORTS = [
     "ppo_model_num_tensors", "ppo_model_tensor_info", "ppo_model_workspace_bytes", "ppo_model_bind",
     "ppo_model_sync_shadow", "ppo_encoder_fwd", "ppo_loss_fwd_bwd", "ppo_encoder_bwd", "ppo_model_zero_grad",
     "ppo_adam_step", "ppo_policy_sample", "ppo_poll_status", "ppo_model_activation_ptr", "ppo_gae_static",
-    "ppo_model_sync_masks",
+    "ppo_model_sync_masks", "ppo_buffer_write_obs", "ppo_buffer_write_outcome", "ppo_policy_act", "ppo_launch_count",
+    "ppo_selftest_wait_timeout",
 ]
 
 
@@ -100,6 +101,12 @@ def lib():
         L.ppo_policy_sample.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
                                         C.c_void_p]
         L.ppo_poll_status.argtypes = [C.c_void_p]
+        L.ppo_buffer_write_obs.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p]
+        L.ppo_buffer_write_outcome.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p]
+        L.ppo_policy_act.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.c_void_p]
+        L.ppo_launch_count.restype = C.c_uint64
+        L.ppo_launch_count.argtypes = []
+        L.ppo_selftest_wait_timeout.argtypes = [C.c_longlong, C.c_void_p, C.c_void_p]
         L.ppo_gae_static.argtypes = [C.c_void_p] * 4 + [C.c_int, C.c_int, C.c_float, C.c_float, C.c_int] + [C.c_void_p] * 4
         L.ppo_model_activation_ptr.argtypes = [C.c_void_p, C.c_int, C.c_int, C.POINTER(C.c_void_p),
                                                C.POINTER(C.c_size_t)]
@@ -188,6 +195,25 @@ def ppo_buffer_write_step(buf: Buffer, t: int, depth, proprio, action, logp, val
     _check(lib().ppo_buffer_write_step(buf.handle, t, _ptr(depth), _ptr(proprio), _ptr(action), _ptr(logp),
                                        _ptr(value), _ptr(reward), _ptr(done), _stream(stream)),
            "ppo_buffer_write_step")
+
+
+def ppo_buffer_write_obs(buf: Buffer, t: int, depth, proprio, stream=None):
+    _check(lib().ppo_buffer_write_obs(buf.handle, t, _ptr(depth), _ptr(proprio), _stream(stream)),
+           "ppo_buffer_write_obs")
+
+
+def ppo_buffer_write_outcome(buf: Buffer, t: int, reward, done, stream=None):
+    _check(lib().ppo_buffer_write_outcome(buf.handle, t, _ptr(reward), _ptr(done), _stream(stream)),
+           "ppo_buffer_write_outcome")
+
+
+def ppo_launch_count() -> int:
+    return int(lib().ppo_launch_count())
+
+
+def ppo_selftest_wait_timeout(limit_cycles: int, gave_up, stream=None):
+    _check(lib().ppo_selftest_wait_timeout(limit_cycles, _ptr(gave_up), _stream(stream)),
+           "ppo_selftest_wait_timeout")
 
 
 def ppo_compute_gae(buf: Buffer, last_value, gamma: float, lam: float, normalize: bool = True, stats_out=None,
@@ -339,6 +365,10 @@ def ppo_encoder_bwd(m: Model, mb: MinibatchArrays, row0: int, rows: int, dmean, 
 
 def ppo_adam_step(m: Model, lr: float, beta1: float, beta2: float, eps: float, step: int, stream=None):
     _check(lib().ppo_adam_step(m.handle, lr, beta1, beta2, eps, step, _stream(stream)), "ppo_adam_step")
+
+
+def ppo_policy_act(m: Model, buf: Buffer, t: int, eps, stream=None):
+    _check(lib().ppo_policy_act(m.handle, buf.handle, t, _ptr(eps), _stream(stream)), "ppo_policy_act")
 
 
 def ppo_policy_sample(m: Model, rows: int, mean, eps, action, logp, stream=None):

@@ -1,5 +1,6 @@
 // Rollout buffer D on the learner GPU (Algorithm 2): slab carving, write_step, GAE with
 // advantage normalisation, and the seeded permutation gather.
+#include <atomic>
 #include <new>
 
 #include "common.cuh"
@@ -19,6 +20,12 @@ int32_t *ppo_device_status_ptr() {
     }
     return ptrs[dev];
 }
+
+static std::atomic<unsigned long long> g_launches{0};
+
+void ppo_count_launches(int n) { g_launches.fetch_add((unsigned long long)n, std::memory_order_relaxed); }
+
+extern "C" uint64_t ppo_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 
 int ppo_num_sms() {
     static int sms[64] = {0};
@@ -172,34 +179,59 @@ __global__ void __launch_bounds__(256) write_step_kernel(CopySegs segs) {
     }
 }
 
+// Copies up to 7 per-env arrays of one step into slab row t (null sources are skipped).
+static int write_fields(ppo_buffer *b, int t, const void *const srcs[7], void *stream) {
+    const ppo_buffer_desc &d = b->d;
+    const size_t N = d.N;
+    const int fields[7] = {PPO_FIELD_DEPTH, PPO_FIELD_PROPRIO, PPO_FIELD_ACTION, PPO_FIELD_LOGP,
+                           PPO_FIELD_VALUE, PPO_FIELD_REWARD, PPO_FIELD_DONE};
+    const size_t per_env[7] = {(size_t)d.H * d.W * 2, (size_t)d.P * 4, (size_t)d.A * 4, 4, 4, 4, 1};
+    CopySegs segs;
+    int n = 0;
+    size_t largest = 0;
+    for (int i = 0; i < 7; ++i) {
+        if (!srcs[i]) continue;
+        size_t bytes = N * per_env[i];
+        char *dst = b->base + b->field_off[fields[i]] + (size_t)t * bytes;
+        segs.s[n].src = static_cast<const char *>(srcs[i]);
+        segs.s[n].dst = dst;
+        segs.s[n].bytes = bytes;
+        segs.s[n].vec = (ppo_aligned(srcs[i], 16) && ppo_aligned(dst, 16) && bytes % 16 == 0) ? 16 : 1;
+        largest = bytes > largest ? bytes : largest;
+        ++n;
+    }
+    b->gae_valid = false;
+    if (n == 0) return PPO_OK;
+    // enough blocks to cover the largest segment with ~4 x 16 B per thread, capped at a few waves
+    long long units = (long long)(largest / 16 / 4 / 256) + 1;
+    int gx = (int)(units < (long long)ppo_num_sms() * 16 ? units : (long long)ppo_num_sms() * 16);
+    dim3 grid(gx, n);
+    write_step_kernel<<<grid, 256, 0, static_cast<cudaStream_t>(stream)>>>(segs);
+    PPO_LAUNCH_CHECK();
+    return PPO_OK;
+}
+
 extern "C" int ppo_buffer_write_step(ppo_buffer *b, int t, const void *depth, const float *proprio,
                                      const float *action, const float *logp, const float *value, const float *reward,
                                      const uint8_t *done, void *stream) {
     if (!b || !depth || !proprio || !action || !logp || !value || !reward || !done) return PPO_ERR_INVALID_ARG;
     if (t < 0 || t >= b->d.T) return PPO_ERR_INVALID_ARG;
-    const ppo_buffer_desc &d = b->d;
-    const size_t N = d.N;
     const void *srcs[7] = {depth, proprio, action, logp, value, reward, done};
-    const int fields[7] = {PPO_FIELD_DEPTH, PPO_FIELD_PROPRIO, PPO_FIELD_ACTION, PPO_FIELD_LOGP,
-                           PPO_FIELD_VALUE, PPO_FIELD_REWARD, PPO_FIELD_DONE};
-    const size_t per_env[7] = {(size_t)d.H * d.W * 2, (size_t)d.P * 4, (size_t)d.A * 4, 4, 4, 4, 1};
-    CopySegs segs;
-    for (int i = 0; i < 7; ++i) {
-        size_t bytes = N * per_env[i];
-        char *dst = b->base + b->field_off[fields[i]] + (size_t)t * bytes;
-        segs.s[i].src = static_cast<const char *>(srcs[i]);
-        segs.s[i].dst = dst;
-        segs.s[i].bytes = bytes;
-        segs.s[i].vec = (ppo_aligned(srcs[i], 16) && ppo_aligned(dst, 16) && bytes % 16 == 0) ? 16 : 1;
-    }
-    b->gae_valid = false;
-    // enough blocks to cover the depth segment with ~4 x 16 B per thread, capped at a few waves
-    long long units = (long long)(segs.s[0].bytes / 16 / 4 / 256) + 1;
-    int gx = (int)(units < (long long)ppo_num_sms() * 16 ? units : (long long)ppo_num_sms() * 16);
-    dim3 grid(gx, 7);
-    write_step_kernel<<<grid, 256, 0, static_cast<cudaStream_t>(stream)>>>(segs);
-    PPO_LAUNCH_CHECK();
-    return PPO_OK;
+    return write_fields(b, t, srcs, stream);
+}
+
+extern "C" int ppo_buffer_write_obs(ppo_buffer *b, int t, const void *depth, const float *proprio, void *stream) {
+    if (!b || !depth || !proprio) return PPO_ERR_INVALID_ARG;
+    if (t < 0 || t >= b->d.T) return PPO_ERR_INVALID_ARG;
+    const void *srcs[7] = {depth, proprio, nullptr, nullptr, nullptr, nullptr, nullptr};
+    return write_fields(b, t, srcs, stream);
+}
+
+extern "C" int ppo_buffer_write_outcome(ppo_buffer *b, int t, const float *reward, const uint8_t *done, void *stream) {
+    if (!b || !reward || !done) return PPO_ERR_INVALID_ARG;
+    if (t < 0 || t >= b->d.T) return PPO_ERR_INVALID_ARG;
+    const void *srcs[7] = {nullptr, nullptr, nullptr, nullptr, nullptr, reward, done};
+    return write_fields(b, t, srcs, stream);
 }
 
 // --------------------------------------------------------------------- GAE ----

@@ -18,14 +18,21 @@ typedef __nv_bfloat16 bf16;
         if (_e != cudaSuccess) return PPO_ERR_CUDA; \
     } while (0)
 
-#define PPO_LAUNCH_CHECK() PPO_CUDA_CHECK(cudaGetLastError())
+// After every kernel launch: counts it (ppo_launch_count) and turns a launch error into a status.
+#define PPO_LAUNCH_CHECK()                  \
+    do {                                    \
+        ppo_count_launches(1);              \
+        PPO_CUDA_CHECK(cudaGetLastError()); \
+    } while (0)
 
 static inline bool ppo_aligned(const void *p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
 static inline size_t ppo_align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 static inline int ppo_cdiv(long long a, long long b) { return (int)((a + b - 1) / b); }
 
-// Device status word shared by all kernels (first error wins); lives in status.cu.
+// Device status word shared by all kernels (first error wins); lives in buffer.cu.
 int32_t *ppo_device_status_ptr();
+// Adds n to the process-wide count of kernels and memsets this library has enqueued.
+void ppo_count_launches(int n);
 int ppo_num_sms();
 
 struct ppo_buffer {
@@ -76,12 +83,12 @@ struct ppo_model {
     int64_t wC_off[PPO_MAX_CONV + 1];  // per conv layer l (2..L)
     size_t wC_elems;
     float *loss_partials;
+    float *act_mean;               // [mb][A]: Gaussian mean of ppo_policy_act before sampling
     int loss_partial_blocks;
     bool wT_valid;
     // forward/backward pairing
     int last_row0, last_rows;
     bool fwd_valid;
-    int impl;  // 0 = tensor-core GEMMs, 1 = CUDA-core reference GEMMs
     // second stream of the backward pass with its fork and join events (made on first use)
     cudaStream_t side = nullptr;
     cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
@@ -90,3 +97,29 @@ struct ppo_model {
 __device__ __forceinline__ float bf2f(bf16 x) { return __bfloat162float(x); }
 
 __device__ __forceinline__ void ppo_report(int32_t *status, int code) { atomicCAS(status, 0, code); }
+
+// ReLU and conversion of two fp32 values to a packed pair of bf16 (low half = a) in one instruction.
+__device__ __forceinline__ uint32_t relu_pack_bf16x2(float a, float b) {
+    uint32_t r;
+    asm("cvt.rn.relu.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(b), "f"(a));
+    return r;
+}
+__device__ __forceinline__ uint32_t pack_bf16x2(float a, float b) {
+    uint32_t r;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(b), "f"(a));
+    return r;
+}
+
+// ReLU gates of a group of 32 channels as one word: channel c sits at bit (c >> 1) + 16 (c & 1), i.e. pair j of
+// packed bf16 values owns bits j (its low half, channel 2j) and 16 + j (its high half, channel 2j + 1).  With the
+// halves non-negative (they come out of a ReLU), half + 0x7fff carries into its top bit exactly when it is not
+// zero, so a pair costs an add, a shift and a logic operation; and a pair's two gates come back out as the mask
+// of its two halves with a shift, an and, and a multiply.
+__host__ __device__ __forceinline__ int gate_bit_of_channel(int c) { return ((c & 31) >> 1) + 16 * (c & 1); }
+__device__ __forceinline__ uint32_t gate_bits_add(uint32_t gate, uint32_t pair, int j) {
+    const uint32_t t = pair + 0x7FFF7FFFu;
+    return gate | ((t >> (15 - j)) & (0x00010001u << j));
+}
+__device__ __forceinline__ uint32_t gate_pair_mask(uint32_t gate, int j) {
+    return ((gate >> j) & 0x00010001u) * 0xFFFFu;
+}

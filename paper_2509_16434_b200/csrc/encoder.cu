@@ -553,10 +553,6 @@ static ConvGeom fc_geom(int rows, int in, int out) {
 
 static int run_fwd(const ppo_model *m, const ConvGeom &g, const bf16 *X, const bf16 *W, const FwdEpilogue &e,
                    cudaStream_t st) {
-    if (m->impl == 1) {
-        const int s = simt_gemm_fwd(g, X, W, e, st);
-        return (s == PPO_OK && e.out_bits) ? relu_bits(e.out, e.out_bits, g.M(), g.Co, st) : s;
-    }
     int s = tma_gemm_fwd(g, X, W, e, ppo_device_status_ptr(), st);  // writes e.out_bits itself
     if (s != PPO_ERR_UNSUPPORTED) return s;
     s = tc_gemm_fwd(g, X, W, e, ppo_device_status_ptr(), st);
@@ -566,7 +562,6 @@ static int run_fwd(const ppo_model *m, const ConvGeom &g, const bf16 *X, const b
 
 static int run_dgrad(const ppo_model *m, const ConvGeom &g, const bf16 *dY, int ldy, const bf16 *W, const bf16 *Wt,
                      int wt_ld, const bf16 *Wc, const DgradEpilogue &e, cudaStream_t st) {
-    if (m->impl == 1) return simt_gemm_dgrad(g, dY, ldy, W, e, st);
     const int s = tma_gemm_dgrad(g, dY, ldy, Wt, wt_ld, Wc, e, ppo_device_status_ptr(), st);
     if (s != PPO_ERR_UNSUPPORTED) return s;
     return tc_gemm_dgrad(g, dY, ldy, Wt, wt_ld, e, ppo_device_status_ptr(), st);
@@ -578,16 +573,11 @@ static int run_colsum(const bf16 *dZ, int ld, long long M, int N, float *db, cud
 // tensor core on its way; everything else reduces dY in a pass of its own.
 static int run_wgrad(const ppo_model *m, const ConvGeom &g, const bf16 *dY, int ldy, const bf16 *X, float *dW,
                      float *db, cudaStream_t st) {
-    int s = PPO_ERR_UNSUPPORTED;
-    if (m->impl == 1) {
-        s = simt_gemm_wgrad(g, dY, ldy, X, dW, st);
-    } else {
-        const bool conv = g.k > 1;
-        s = tma_gemm_wgrad(g, dY, ldy, X, dW, conv ? db : nullptr, ppo_device_status_ptr(), st);
-        if (s == PPO_OK && conv) return s;
-        if (s == PPO_ERR_UNSUPPORTED && conv) s = tma_gemm_wgrad(g, dY, ldy, X, dW, nullptr, ppo_device_status_ptr(), st);
-        if (s == PPO_ERR_UNSUPPORTED) s = tc_gemm_wgrad(g, dY, ldy, X, dW, ppo_device_status_ptr(), st);
-    }
+    const bool conv = g.k > 1;
+    int s = tma_gemm_wgrad(g, dY, ldy, X, dW, conv ? db : nullptr, ppo_device_status_ptr(), st);
+    if (s == PPO_OK && conv) return s;
+    if (s == PPO_ERR_UNSUPPORTED && conv) s = tma_gemm_wgrad(g, dY, ldy, X, dW, nullptr, ppo_device_status_ptr(), st);
+    if (s == PPO_ERR_UNSUPPORTED) s = tc_gemm_wgrad(g, dY, ldy, X, dW, ppo_device_status_ptr(), st);
     if (s != PPO_OK) return s;
     return run_colsum(dY, ldy, g.M(), g.Co, db, st);
 }
@@ -606,6 +596,7 @@ static int run_colsum(const bf16 *dZ, int ld, long long M, int N, float *db, cud
             const int cap = ppo_num_sms() * 4;
             blocks = blocks > cap ? cap : (blocks < 1 ? 1 : blocks);
             colsum_kernel<<<blocks, 256, 0, st>>>(dZ + n0, ld, M, 256, db + n0);
+            if (n0 + 256 < N) PPO_LAUNCH_CHECK();
         }
     } else {
         int blocks = ppo_cdiv(M, 2048);
@@ -641,9 +632,8 @@ extern "C" int ppo_encoder_fwd(ppo_model *m, const ppo_minibatch *mb, int row0, 
         const __half *depth = static_cast<const __half *>(mb->depth_f16) + (size_t)row0 * d.H * d.W;
         const int C1 = m->Cs[1], KS = d.conv_k[0];
         const long long M = (long long)rows * m->Hs[1] * m->Ws[1];
-        int tcs = PPO_ERR_UNSUPPORTED;
-        if (m->impl == 0)
-            tcs = conv1_tc_fwd(depth, m->shadow + m->tensors[0].off, m->master + m->tensors[1].off, m->act[1], m->abits[1],
+        const int tcs =
+            conv1_tc_fwd(depth, m->shadow + m->tensors[0].off, m->master + m->tensors[1].off, m->act[1], m->abits[1],
                                rows, d.H, d.W, m->Hs[1], m->Ws[1], C1, KS, ppo_device_status_ptr(), st);
         if (tcs != PPO_OK && tcs != PPO_ERR_UNSUPPORTED) return tcs;
         const int CH = C1 / 8;
@@ -724,9 +714,19 @@ static int refresh_transposed(ppo_model *m, cudaStream_t st) {
 // Second stream and the two events of the fork/join in the backward pass, made on first use.
 static int side_stream(ppo_model *m) {
     if (m->side) return PPO_OK;
-    PPO_CUDA_CHECK(cudaStreamCreateWithFlags(&m->side, cudaStreamNonBlocking));
-    PPO_CUDA_CHECK(cudaEventCreateWithFlags(&m->ev_fork, cudaEventDisableTiming));
-    PPO_CUDA_CHECK(cudaEventCreateWithFlags(&m->ev_join, cudaEventDisableTiming));
+    cudaStream_t s = nullptr;
+    cudaEvent_t ef = nullptr, ej = nullptr;
+    if (cudaStreamCreateWithFlags(&s, cudaStreamNonBlocking) != cudaSuccess ||
+        cudaEventCreateWithFlags(&ef, cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&ej, cudaEventDisableTiming) != cudaSuccess) {
+        if (ej) cudaEventDestroy(ej);
+        if (ef) cudaEventDestroy(ef);
+        if (s) cudaStreamDestroy(s);
+        return PPO_ERR_CUDA;
+    }
+    m->side = s;  // all three exist, or none is kept
+    m->ev_fork = ef;
+    m->ev_join = ej;
     return PPO_OK;
 }
 
@@ -736,7 +736,7 @@ static int conv1_wgrad(ppo_model *m, const ppo_minibatch *mb, int row0, int rows
     const __half *depth = static_cast<const __half *>(mb->depth_f16) + (size_t)row0 * d.H * d.W;
     const int C1 = m->Cs[1], KS = d.conv_k[0];
     const long long M = (long long)rows * m->Hs[1] * m->Ws[1];
-    if (m->impl == 0 && C1 % 16 == 0 && C1 <= 64 && (KS == 3 || KS == 5)) {
+    if (C1 % 16 == 0 && C1 <= 64 && (KS == 3 || KS == 5)) {
         // tensor-core reduction
         const int TP = (KS * KS + 1 + 15) / 16 * 16;
         const size_t tile = (size_t)32 * TP * 2 + (size_t)32 * C1 * 2, redb = (size_t)TP * C1 * sizeof(float);
@@ -806,8 +806,11 @@ extern "C" int ppo_encoder_bwd(ppo_model *m, const ppo_minibatch *mb, int row0, 
     const ppo_model_desc &d = m->d;
     const int L = m->L, F = m->F;
     if (!accumulate)  // everything but the trailing log-sigma slot, which the loss call owns
+    {
         PPO_CUDA_CHECK(cudaMemsetAsync(m->grad, 0, (size_t)m->tensors.back().off * sizeof(float), st));
-    if (m->impl == 0) PPO_TRY(refresh_transposed(m, st));
+        ppo_count_launches(1);
+    }
+    PPO_TRY(refresh_transposed(m, st));
 
     pack_dout_kernel<<<ppo_cdiv((long long)rows * 16, 256), 256, 0, st>>>(dmean, dvalue, m->dh[F + 1], rows, d.A);
     PPO_LAUNCH_CHECK();
@@ -815,7 +818,7 @@ extern "C" int ppo_encoder_bwd(ppo_model *m, const ppo_minibatch *mb, int row0, 
     // The leaves of the FC layers (small kernels on a fraction of the SMs) and, further down, conv1's wgrad go to
     // a second stream that forks from the caller's stream whenever the gradient they read is ready and joins it
     // at the end of the call.
-    const bool fork = m->impl == 0 && side_stream(m) == PPO_OK;
+    const bool fork = side_stream(m) == PPO_OK;
     cudaStream_t leaf = fork ? m->side : st;
     auto fork_here = [&]() -> int {
         if (!fork) return PPO_OK;

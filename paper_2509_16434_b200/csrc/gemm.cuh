@@ -27,11 +27,6 @@ struct DgradEpilogue {
 
 // ldy: row stride (elements) of Y / dY (>= Co).  wt_ld: row stride of the innermost (co)
 // dimension of the transposed weights Wt[ci][tap][wt_ld].
-int simt_gemm_fwd(const ConvGeom &g, const bf16 *X, const bf16 *W, const FwdEpilogue &e, cudaStream_t st);
-int simt_gemm_dgrad(const ConvGeom &g, const bf16 *dY, int ldy, const bf16 *W, const DgradEpilogue &e,
-                    cudaStream_t st);
-int simt_gemm_wgrad(const ConvGeom &g, const bf16 *dY, int ldy, const bf16 *X, float *dW, cudaStream_t st);
-
 int tc_gemm_fwd(const ConvGeom &g, const bf16 *X, const bf16 *W, const FwdEpilogue &e, int32_t *status,
                 cudaStream_t st);
 int tc_gemm_dgrad(const ConvGeom &g, const bf16 *dY, int ldy, const bf16 *Wt, int wt_ld, const DgradEpilogue &e,

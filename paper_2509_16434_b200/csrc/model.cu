@@ -87,9 +87,6 @@ extern "C" int ppo_model_create(const ppo_model_desc *d, ppo_model **out) {
     m->fwd_valid = false;
     m->wT_valid = false;
     m->last_row0 = m->last_rows = -1;
-    m->impl = 0;
-    const char *e = getenv("PPO_B200_ENCODER");
-    if (e && e[0] == 's') m->impl = 1;  // "simt": CUDA-core reference GEMMs (debugging aid)
     *out = m;
     return PPO_OK;
 }
@@ -151,6 +148,8 @@ static size_t carve(ppo_model *m, const ppo_model *shape, int mb, char *base) {
         int blocks = ppo_cdiv(mb, kLossThreads);
         char *lp = take((size_t)blocks * 32 * sizeof(float));
         if (m) { m->loss_partials = (float *)lp; m->loss_partial_blocks = blocks; }
+        char *am = take((size_t)mb * shape->d.A * sizeof(float));
+        if (m) m->act_mean = (float *)am;
     }
     return off;
 }
@@ -241,6 +240,7 @@ extern "C" int ppo_model_sync_shadow(ppo_model *m, void *stream) {
 extern "C" int ppo_model_zero_grad(ppo_model *m, void *stream) {
     if (!m || !m->grad) return PPO_ERR_STATE;
     PPO_CUDA_CHECK(cudaMemsetAsync(m->grad, 0, m->arena * sizeof(float), static_cast<cudaStream_t>(stream)));
+    ppo_count_launches(1);
     return PPO_OK;
 }
 
@@ -436,5 +436,35 @@ extern "C" int ppo_policy_sample(const ppo_model *m, int rows, const float *mean
     sample_kernel<<<ppo_cdiv(rows, 128), 128, 0, static_cast<cudaStream_t>(stream)>>>(
         rows, m->d.A, mean, m->master + m->tensors.back().off, eps, action, logp);
     PPO_LAUNCH_CHECK();
+    return PPO_OK;
+}
+
+// actions <- pi(obs) for time step t of the buffer, in place: the observation is read from slab row t and the
+// action, its log-density and the value estimate are written into slab row t.
+extern "C" int ppo_policy_act(ppo_model *m, ppo_buffer *b, int t, const float *eps, void *stream) {
+    if (!m || !b || !eps) return PPO_ERR_INVALID_ARG;
+    if (!m->master) return PPO_ERR_STATE;
+    const ppo_buffer_desc &d = b->d;
+    if (t < 0 || t >= d.T) return PPO_ERR_INVALID_ARG;
+    if (d.H != m->d.H || d.W != m->d.W || d.P != m->d.P || d.A != m->d.A) return PPO_ERR_SHAPE;
+    const size_t N = (size_t)d.N;
+    char *depth = b->base + b->field_off[PPO_FIELD_DEPTH] + (size_t)t * N * d.H * d.W * 2;
+    float *proprio = reinterpret_cast<float *>(b->base + b->field_off[PPO_FIELD_PROPRIO]) + (size_t)t * N * d.P;
+    float *action = reinterpret_cast<float *>(b->base + b->field_off[PPO_FIELD_ACTION]) + (size_t)t * N * d.A;
+    float *logp = reinterpret_cast<float *>(b->base + b->field_off[PPO_FIELD_LOGP]) + (size_t)t * N;
+    float *value = reinterpret_cast<float *>(b->base + b->field_off[PPO_FIELD_VALUE]) + (size_t)t * N;
+    ppo_minibatch obs = {};
+    obs.depth_f16 = depth;
+    obs.proprio = proprio;
+    obs.B = d.N;
+    b->gae_valid = false;
+    for (int r0 = 0; r0 < d.N; r0 += m->mbmax) {
+        const int rows = d.N - r0 < m->mbmax ? d.N - r0 : m->mbmax;
+        int s = ppo_encoder_fwd(m, &obs, r0, rows, m->act_mean, value + r0, stream);
+        if (s != PPO_OK) return s;
+        s = ppo_policy_sample(m, rows, m->act_mean, eps + (size_t)r0 * d.A, action + (size_t)r0 * d.A, logp + r0, stream);
+        if (s != PPO_OK) return s;
+    }
+    m->fwd_valid = false;  // these activations belong to no minibatch a backward pass could name
     return PPO_OK;
 }

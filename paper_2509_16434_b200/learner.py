@@ -47,7 +47,6 @@ class Learner:
         self.loss = torch.zeros(5, dtype=torch.float32, device=device)
         self.stats = torch.zeros(2, dtype=torch.float32, device=device)
         self.adam_t = 0
-        self.launches = 0  # kernels and memsets enqueued by the library, by this object's count
 
     # ------------------------------------------------------------------ buffer fill
 
@@ -72,39 +71,35 @@ class Learner:
                                   logp[r0:r0 + rows])
         return action, logp, value
 
+    def act_into_buffer(self, t: int, depth: torch.Tensor, proprio: torch.Tensor, eps: torch.Tensor):
+        """One rollout step without intermediate copies: the observation goes into slab row t, the policy reads
+        it there and writes action, log-prob and value into the same row (Algorithm 2, actions <- pi(obs) then
+        D <- D U {...}); ppo_buffer_write_outcome adds reward and done once the env has stepped."""
+        ppo.ppo_buffer_write_obs(self.buffer, t, depth, proprio)
+        ppo.ppo_policy_act(self.model, self.buffer, t, eps)
+
     # ------------------------------------------------------------------ TrainPPO
 
     def compute_gae(self, last_value: torch.Tensor, normalize: bool = True):
         h = self.hyper
         ppo.ppo_compute_gae(self.buffer, last_value, h.gamma, h.lam, normalize, self.stats)
-        self.launches += 2 if normalize else 1
 
     def minibatch_step(self, seed: int, epoch: int, k: int, num_minibatches: Optional[int] = None):
         """gather -> (fwd -> loss -> bwd) per micro-batch -> Adam for minibatch k of this epoch."""
         w, h = self.w, self.hyper
         K = num_minibatches or w.minibatches
         B = w.M // K
-        n_layers_gemm = (len(w.conv_c) - 1) + len(w.fc) + 1
         ppo.ppo_shuffle_gather_minibatch(self.buffer, seed, epoch, k, K, self.mb)
         ppo.ppo_model_zero_grad(self.model)
         self.loss.zero_()
-        self.launches += 3
-        # the first backward after a weight change re-derives the transposed / regrouped weight copies
-        self.launches += 2 * (len(w.conv_c) - 1) + len(w.fc) + 1
         for r0 in range(0, B, self.microbatch):
             rows = min(self.microbatch, B - r0)
             ppo.ppo_encoder_fwd(self.model, self.mb, r0, rows, self.mean, self.value)
             ppo.ppo_loss_fwd_bwd(self.model, self.mb, r0, rows, B, self.mean, self.value, h.clip, h.vf_coef,
                                  h.ent_coef, self.loss, self.dmean, self.dvalue)
             ppo.ppo_encoder_bwd(self.model, self.mb, r0, rows, self.dmean, self.dvalue, True)
-            # fwd: conv1 + GEMMs + pool; loss: 2; bwd: pack + (wgrad, bias sum, dgrad) per GEMM layer + unpool +
-            # conv1 wgrad; the wgrad of a convolution sums the bias gradient itself
-            # (a bias sum wider than 256 columns runs one launch per 256-column slab)
-            slabs = sum(o // 256 - 1 for o in w.fc if o > 256 and o % 256 == 0)
-            self.launches += (1 + n_layers_gemm + 1) + 2 + (1 + 3 * n_layers_gemm - (len(w.conv_c) - 1) + slabs + 1 + 1)
         self.adam_t += 1
         ppo.ppo_adam_step(self.model, h.lr, h.beta1, h.beta2, h.eps, self.adam_t)
-        self.launches += 1
 
     def train(self, last_value: torch.Tensor, seed: int = 0):
         """One TrainPPO call over the current buffer."""

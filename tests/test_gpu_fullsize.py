@@ -31,7 +31,7 @@ def _device_rollout(w):
     return roll, action, logp
 
 
-@pytest.mark.parametrize("name", ["cfg2", "cfg3", "cfg5_4k"])
+@pytest.mark.parametrize("name", ["cfg2", "cfg3", "cfg4", "cfg5_1k", "cfg5_4k", "cfg5_16k"])
 def test_gae_gather_at_full_size(name):
     w = synth.WORKLOADS[name]
     roll, action, logp = _device_rollout(w)
@@ -110,11 +110,16 @@ def test_encoder_forward_sampled_rows_at_bench_shapes(name, rows_checked):
     r = torch.as_tensor(rows, device=DEV)
     depth = L.mb.depth[r].cpu().numpy()
     proprio = L.mb.proprio[r].cpu().numpy()
-    mu_o, V_o, _ = orc.encoder_fwd(md, orc.round_weights(md, theta), depth, proprio, True)
     mu = L.mean[r].cpu().numpy()
     V = L.value[r].cpu().numpy()
-    assert rel_l2(mu, mu_o) <= ENC_TOL, rel_l2(mu, mu_o)
-    assert rel_l2(V, V_o) <= ENC_TOL, rel_l2(V, V_o)
+    # against the oracle that stores its activations as bf16 values like the kernels do, and against the one that
+    # keeps them in fp64 between layers
+    for act_bf16 in (True, False):
+        mu_o, V_o, _ = orc.encoder_fwd(md, orc.round_weights(md, theta), depth, proprio, act_bf16)
+        print(f"[{name}] bench-shape forward, oracle activations {'bf16' if act_bf16 else 'fp64'}: "
+              f"mu {rel_l2(mu, mu_o):.3e}, V {rel_l2(V, V_o):.3e}")
+        assert rel_l2(mu, mu_o) <= ENC_TOL, rel_l2(mu, mu_o)
+        assert rel_l2(V, V_o) <= ENC_TOL, rel_l2(V, V_o)
 
 
 def test_microbatched_gradients_add_up_at_bench_shapes():

@@ -14,14 +14,13 @@ DEV = "cuda"
 ENC_TOL = 2e-2    # relative L2: bf16 operands / activations with fp32 accumulation vs fp64
 LOSS_TOL = 1e-3   # relative error of the loss scalars
 ADAM_TOL = 1e-3   # relative L2 of the parameters after one step
-# End-to-end gradients (GPU forward feeding GPU backward) against the oracle's own forward+backward: a stored activation
-# that lands on the other side of a bf16 rounding boundary (fp32 vs fp64 sums) moves downstream pre-activations by
-# ~1e-4 relative, which flips the ReLU gate of the ~1e-4 fraction of units sitting that close to zero; each flipped
-# gate changes that unit's gradient by its full size, so the relative L2 error of a gradient is ~sqrt(flipped
-# fraction / active fraction) ~ 1-2 % per layer it passes through, not ~eps.  The backward operator itself is
-# held to ENC_TOL in the test that gives both sides identical saved activations.
-E2E_GRAD_TOL_TOTAL = 1e-1
-E2E_GRAD_TOL_TENSOR = 2e-1
+# End-to-end gradients (GPU forward feeding GPU backward) against the oracle's own forward+backward are held to the
+# same 2e-2, in total and per tensor, at these sizes (measured: at most 6e-3).  What separates the two sides beyond
+# the arithmetic is the handful of ReLU gates (measured: fewer than 1 in 10^6) that the two forwards decide
+# differently; test_gpu_parity_wide.py counts them and holds the backward operator to 2e-2 on identical activations.
+E2E_GRAD_TOL_TOTAL = 2e-2
+E2E_GRAD_TOL_TENSOR = 2e-2
+SIGN_AGREEMENT = 0.97  # fraction of clearly moved parameters whose Adam update has the oracle's sign
 
 
 def _setup(w, microbatch, seed=0, jitter=True, theta_scale_head=1.0):
@@ -152,10 +151,12 @@ def test_minibatch_forward_loss_backward_match_oracle(name, microbatch):
     assert rel_l2(V, V_o) <= ENC_TOL, rel_l2(V, V_o)
     out = L.loss.cpu().numpy()
     assert 0.0 < out_o[4] < 1.0, "both clip branches must be exercised"
-    # entropy is exact arithmetic on log-sigma; the others inherit the encoder's bf16 error through mu and V
+    # value loss and entropy to 1e-3 relative; the policy loss and the KL estimate are means of signed terms near
+    # zero, so their errors are measured against the mean magnitude of their terms (|s| ~ |adv|, |log ratio|)
+    assert abs(out[1] - out_o[1]) <= LOSS_TOL * abs(out_o[1])
     assert abs(out[2] - out_o[2]) <= LOSS_TOL * abs(out_o[2])
-    for j, tol in [(0, 2e-2), (1, 2e-2), (3, 2e-2)]:
-        assert abs(out[j] - out_o[j]) <= tol * max(abs(out_o[j]), 0.05), (j, out[j], out_o[j])
+    assert abs(out[0] - out_o[0]) <= LOSS_TOL * float(np.mean(np.abs(f["adv"])))
+    assert abs(out[3] - out_o[3]) <= LOSS_TOL * max(1.0, abs(out_o[3]))
     assert abs(out[4] - out_o[4]) <= 2.0 / B + 1e-6
     _check_grads(lay, L.model.grad.cpu().numpy(), grad_o, E2E_GRAD_TOL_TENSOR, E2E_GRAD_TOL_TOTAL)
 
@@ -262,7 +263,57 @@ def test_whole_learner_step_parameters_match_oracle(name, microbatch):
         got = L.model.master.cpu().numpy()
         assert rel_l2(got, th) <= ADAM_TOL * (k + 1), (k, rel_l2(got, th))
     assert ppo.ppo_poll_status() == 0
-    assert rel_l2(got - theta, th - theta) <= 0.35, rel_l2(got - theta, th - theta)
+    # The update itself: after a few Adam steps from m = v = 0 every parameter has moved by about lr * (steps) *
+    # sign(g), so its relative L2 error is sqrt(4 x the fraction of parameters whose gradient sign differs), and a
+    # sign differs only where |g| is below the gradient's own error.  Measured as that fraction over the parameters
+    # the oracle moved by at least half a step.
+    du_g, du_o = got - theta, th - theta
+    moved = np.abs(du_o) >= 0.5 * h.lr
+    agree = float(np.mean(np.sign(du_g[moved]) == np.sign(du_o[moved])))
+    print(f"[{name}] update after {w.minibatches} Adam steps: sign agreement {agree:.4f} over {int(moved.sum())} "
+          f"parameters, rel L2 {rel_l2(du_g, du_o):.3e}")
+    assert agree >= SIGN_AGREEMENT
+
+
+def test_policy_act_writes_the_rollout_step_into_its_slab_row():
+    """ppo_buffer_write_obs + ppo_policy_act + ppo_buffer_write_outcome fill slab row t like the oracle's rollout:
+    observation, reward and done byte-exact, action / log-prob / value from the policy on that observation."""
+    w = SHAPES["cfg1_twin"]
+    L, md, lay, theta, roll, action, logp, dev = _setup(w, 5, jitter=False)  # 16 envs in micro-batches of 5, 5, 5, 1
+    buf = ppo.Buffer(L.bdesc, DEV)
+    L.buffer = buf
+    for t in range(w.T):
+        L.act_into_buffer(t, dev["depth"][t], dev["proprio"][t], dev["eps"][t])
+        ppo.ppo_buffer_write_outcome(buf, t, dev["reward"][t], dev["done"][t])
+    assert ppo.ppo_poll_status() == 0
+    used = orc.round_weights(md, theta)
+    _, V_o, _ = orc.encoder_fwd(md, used, roll["depth"].reshape(w.M, w.H, w.W), roll["proprio"].reshape(w.M, w.P), True)
+    assert torch.equal(buf.field(ppo.FIELD_DEPTH), dev["depth"])
+    assert torch.equal(buf.field(ppo.FIELD_PROPRIO), dev["proprio"])
+    assert torch.equal(buf.field(ppo.FIELD_REWARD), dev["reward"])
+    assert torch.equal(buf.field(ppo.FIELD_DONE), dev["done"])
+    assert rel_l2(buf.field(ppo.FIELD_ACTION).cpu().numpy(), action) <= ENC_TOL
+    assert np.abs(buf.field(ppo.FIELD_LOGP).cpu().numpy() - logp).max() <= 1e-4
+    assert rel_l2(buf.field(ppo.FIELD_VALUE).cpu().numpy().reshape(-1), V_o) <= ENC_TOL
+    # the model and the buffer must agree on the observation's shape
+    other = ppo.Buffer(ppo.buffer_desc(w.N, w.T, w.H + 2, w.W, w.P, w.A), DEV)
+    assert ppo.lib().ppo_policy_act(L.model.handle, other.handle, 0, ppo._ptr(dev["eps"][0]), ppo._stream()) == 2
+    assert ppo.lib().ppo_policy_act(L.model.handle, buf.handle, w.T, ppo._ptr(dev["eps"][0]), ppo._stream()) == 1
+
+
+def test_a_device_side_wait_that_runs_out_reports_timeout_and_leaves_the_device_usable():
+    gave_up = torch.zeros(1, dtype=torch.int32, device=DEV)
+    ppo.ppo_selftest_wait_timeout(2_000_000, gave_up)   # ~1 ms
+    assert ppo.ppo_poll_status() == 6                   # PPO_ERR_TIMEOUT, cleared by the poll
+    assert gave_up.item() == 64
+    assert ppo.ppo_poll_status() == 0
+    # the context is intact: a real kernel of the library runs and checks out afterwards
+    w = SHAPES["tiny"]
+    L, md, lay, theta, roll, action, logp, dev = _setup(w, 16)
+    L.compute_gae(dev["last_value"])
+    ppo.ppo_shuffle_gather_minibatch(L.buffer, 0, 0, 0, w.minibatches, L.mb)
+    ppo.ppo_encoder_fwd(L.model, L.mb, 0, w.M // w.minibatches, L.mean, L.value)
+    assert ppo.ppo_poll_status() == 0 and bool(torch.isfinite(L.mean).all())
 
 
 def test_policy_act_matches_oracle():
