@@ -25,7 +25,7 @@ class _Model(C.Structure):
         ("H", C.c_int32), ("W", C.c_int32), ("n_conv", C.c_int32),
         ("conv_c", C.c_int32 * 8), ("conv_k", C.c_int32 * 8),
         ("n_fc", C.c_int32), ("fc", C.c_int32 * 4),
-        ("P", C.c_int32), ("A", C.c_int32),
+        ("P", C.c_int32), ("A", C.c_int32), ("norm", C.c_int32), ("embed", C.c_int32),
     ]
 
 
@@ -72,10 +72,13 @@ class ModelDesc:
     fc: Sequence[int]
     P: int = 32
     A: int = 12
+    norm: bool = False   # layer normalisation over the channels of every conv output, before its ReLU
+    embed: int = 0       # > 0: flatten -> FC(embed) -> ReLU instead of the global average pool
 
     def c(self) -> _Model:
         m = _Model()
         m.H, m.W, m.n_conv, m.n_fc, m.P, m.A = self.H, self.W, len(self.conv_c), len(self.fc), self.P, self.A
+        m.norm, m.embed = int(self.norm), int(self.embed)
         for i, v in enumerate(self.conv_c):
             m.conv_c[i] = v
         for i, v in enumerate(self.conv_k):
@@ -99,7 +102,7 @@ def depth_bytes(N, T, H, W, elem) -> int:
 
 
 def param_layout(md: ModelDesc) -> Layout:
-    n_max = 2 * 8 + 2 * 4 + 3
+    n_max = 4 * 8 + 2 * 4 + 5
     offs = (C.c_int64 * n_max)()
     szs = (C.c_int64 * n_max)()
     mat = (C.c_int32 * n_max)()
@@ -111,8 +114,14 @@ def param_layout(md: ModelDesc) -> Layout:
     cin = 1
     for co, kk in zip(md.conv_c, md.conv_k):
         lay.shapes += [(co, kk, kk, cin), (co,)]
+        if md.norm:
+            lay.shapes += [(co,), (co,)]
         cin = co
     i = cin + md.P
+    if md.embed:
+        ho, wo = conv_shapes(md)
+        lay.shapes += [(md.embed, ho[-1] * wo[-1] * cin), (md.embed,)]
+        i = md.embed + md.P
     for o in md.fc:
         lay.shapes += [(o, i), (o,)]
         i = o

@@ -52,7 +52,17 @@ typedef struct {
     int32_t n_fc;
     int32_t fc[ORC_MAX_FC];       /* hidden widths */
     int32_t P, A;                 /* proprio width, action width */
+    /* The depth CNN as Section III-C words it ("layer normalization, and ReLU", "a fully connected layer which
+     * outputs a 32 dimensional embedding"); both 0 for the networks the workloads describe.
+     *   norm != 0 : every conv output is layer-normalised over its channels at each pixel (learned scale gamma and
+     *               shift beta per channel, variance over the channels, eps 1e-5) before the ReLU;
+     *   embed > 0 : the last conv output is flattened (pixel-major, channel innermost) and mapped by a fully
+     *               connected layer with ReLU to `embed` values, which take the place of the pooled vector. */
+    int32_t norm, embed;
 } orc_model;
+
+#define ORC_MAX_TENSORS (4 * ORC_MAX_CONV + 2 * ORC_MAX_FC + 5)
+#define ORC_LN_EPS 1e-5
 
 int orc_num_threads(void) {
 #ifdef _OPENMP
@@ -193,8 +203,10 @@ void orc_conv_shapes(const orc_model *m, int32_t *Ho, int32_t *Wo) {
 /* Parameter vector layout (an interface shared with the caller, restated here):
  * tensors in the order conv W_l [Cout][k][k][Cin], conv b_l, ..., fc W [out][in],
  * fc b, ..., head W [A+1][hid] (rows 0..A-1 mean, row A value), head b [A+1],
- * log-sigma [A]; each tensor starts at a multiple of 64 elements.
- * offsets/sizes must have room for 2*n_conv + 2*n_fc + 3 entries.
+ * log-sigma [A]; each tensor starts at a multiple of 64 elements.  With norm != 0 every conv b_l is followed by
+ * gamma_l [Cout] and beta_l [Cout]; with embed > 0 the conv tensors are followed by embed W [E][Ho*Wo*C_L] and
+ * embed b [E], and the first fc layer reads E + P values.
+ * offsets/sizes must have room for ORC_MAX_TENSORS entries.
  * Returns the total length of the vector; *n_tensors gets the tensor count. */
 int64_t orc_param_layout(const orc_model *m, int64_t *offsets, int64_t *sizes, int32_t *is_matrix, int32_t *n_tensors) {
     int64_t off = 0;
@@ -211,9 +223,20 @@ int64_t orc_param_layout(const orc_model *m, int64_t *offsets, int64_t *sizes, i
     for (int l = 0; l < m->n_conv; ++l) {
         PUSH((int64_t)m->conv_c[l] * m->conv_k[l] * m->conv_k[l] * cin, 1);
         PUSH(m->conv_c[l], 0);
+        if (m->norm) {
+            PUSH(m->conv_c[l], 0);
+            PUSH(m->conv_c[l], 0);
+        }
         cin = m->conv_c[l];
     }
     int in = cin + m->P;
+    if (m->embed > 0) {
+        int32_t Ho[ORC_MAX_CONV], Wo[ORC_MAX_CONV];
+        orc_conv_shapes(m, Ho, Wo);
+        PUSH((int64_t)m->embed * Ho[m->n_conv - 1] * Wo[m->n_conv - 1] * cin, 1);
+        PUSH(m->embed, 0);
+        in = m->embed + m->P;
+    }
     for (int l = 0; l < m->n_fc; ++l) {
         PUSH((int64_t)m->fc[l] * in, 1);
         PUSH(m->fc[l], 0);
@@ -230,8 +253,8 @@ int64_t orc_param_layout(const orc_model *m, int64_t *offsets, int64_t *sizes, i
 /* Weight matrices are used as bf16-rounded copies of the fp32 master; biases
  * and log-sigma are used as they are. */
 void orc_round_weights(const orc_model *m, const double *theta, double *theta_used) {
-    int64_t offs[2 * ORC_MAX_CONV + 2 * ORC_MAX_FC + 3], szs[2 * ORC_MAX_CONV + 2 * ORC_MAX_FC + 3];
-    int32_t mat[2 * ORC_MAX_CONV + 2 * ORC_MAX_FC + 3], n;
+    int64_t offs[ORC_MAX_TENSORS], szs[ORC_MAX_TENSORS];
+    int32_t mat[ORC_MAX_TENSORS], n;
     int64_t total = orc_param_layout(m, offs, szs, mat, &n);
     for (int64_t i = 0; i < total; ++i) theta_used[i] = theta[i];
     for (int t = 0; t < n; ++t)
@@ -239,14 +262,25 @@ void orc_round_weights(const orc_model *m, const double *theta, double *theta_us
             for (int64_t i = 0; i < szs[t]; ++i) theta_used[offs[t] + i] = orc_round_bf16(theta[offs[t] + i]);
 }
 
-/* Per-sample activation record: [image H*W | a_1 | ... | a_L | h_0 = pooled ++ proprio | h_1 | ... | h_F]. */
-int64_t orc_act_stride(const orc_model *m) {
+/* Per-sample activation record: [image H*W | a_1 | ... | a_L | h_0 = pooled (or embedding) ++ proprio | h_1 | ... |
+ * h_F], followed with norm != 0 by what the backward pass of the normalisation needs, layer by layer: the
+ * normalised values xhat_l [Ho*Wo*C] and the reciprocal standard deviations rstd_l [Ho*Wo]. */
+static int64_t act_main_len(const orc_model *m) {
     int32_t Ho[ORC_MAX_CONV], Wo[ORC_MAX_CONV];
     orc_conv_shapes(m, Ho, Wo);
     int64_t s = (int64_t)m->H * m->W;
     for (int l = 0; l < m->n_conv; ++l) s += (int64_t)Ho[l] * Wo[l] * m->conv_c[l];
-    s += m->conv_c[m->n_conv - 1] + m->P;
+    s += (m->embed > 0 ? m->embed : m->conv_c[m->n_conv - 1]) + m->P;
     for (int l = 0; l < m->n_fc; ++l) s += m->fc[l];
+    return s;
+}
+
+int64_t orc_act_stride(const orc_model *m) {
+    int32_t Ho[ORC_MAX_CONV], Wo[ORC_MAX_CONV];
+    orc_conv_shapes(m, Ho, Wo);
+    int64_t s = act_main_len(m);
+    if (m->norm)
+        for (int l = 0; l < m->n_conv; ++l) s += (int64_t)Ho[l] * Wo[l] * (m->conv_c[l] + 1);
     return s;
 }
 
@@ -265,6 +299,7 @@ static void fwd_one(const orc_model *m, const double *th, const int64_t *offs, c
     int32_t Ho[ORC_MAX_CONV], Wo[ORC_MAX_CONV];
     orc_conv_shapes(m, Ho, Wo);
     double *x = act;
+    double *extra = act + act_main_len(m); /* xhat_l, rstd_l of the normalised layers */
     for (int64_t i = 0; i < (int64_t)m->H * m->W; ++i) x[i] = depth[i];
     int hin = m->H, win = m->W, cin = 1;
     int ti = 0;
@@ -272,9 +307,17 @@ static void fwd_one(const orc_model *m, const double *th, const int64_t *offs, c
         int k = m->conv_k[l], p = k / 2, co_n = m->conv_c[l];
         const double *Wt = th + offs[ti], *b = th + offs[ti + 1];
         ti += 2;
+        const double *gam = NULL, *bet = NULL;
+        if (m->norm) {
+            gam = th + offs[ti];
+            bet = th + offs[ti + 1];
+            ti += 2;
+        }
         double *y = x + (int64_t)hin * win * cin;
         for (int oh = 0; oh < Ho[l]; ++oh)
-            for (int ow = 0; ow < Wo[l]; ++ow)
+            for (int ow = 0; ow < Wo[l]; ++ow) {
+                int64_t px = (int64_t)oh * Wo[l] + ow;
+                double *z = y + px * co_n; /* pre-activations of this pixel, then its outputs */
                 for (int co = 0; co < co_n; ++co) {
                     double acc = b[co];
                     for (int kh = 0; kh < k; ++kh) {
@@ -288,24 +331,61 @@ static void fwd_one(const orc_model *m, const double *th, const int64_t *offs, c
                             for (int ci = 0; ci < cin; ++ci) acc += wp[ci] * xp[ci];
                         }
                     }
-                    acc = acc > 0.0 ? acc : 0.0;
-                    y[((int64_t)oh * Wo[l] + ow) * co_n + co] = act_bf16 ? orc_round_bf16(acc) : acc;
+                    z[co] = acc;
                 }
+                if (m->norm) {
+                    /* layer normalisation over the channels of this pixel:
+                     * mean = sum z / C, var = sum (z - mean)^2 / C, xhat = (z - mean) / sqrt(var + eps),
+                     * z <- gamma * xhat + beta */
+                    double mean = 0.0, var = 0.0;
+                    for (int co = 0; co < co_n; ++co) mean += z[co];
+                    mean /= (double)co_n;
+                    for (int co = 0; co < co_n; ++co) var += (z[co] - mean) * (z[co] - mean);
+                    var /= (double)co_n;
+                    double rstd = 1.0 / sqrt(var + ORC_LN_EPS);
+                    double *xh = extra + px * co_n;
+                    extra[(int64_t)Ho[l] * Wo[l] * co_n + px] = rstd;
+                    for (int co = 0; co < co_n; ++co) {
+                        double v = (z[co] - mean) * rstd;
+                        z[co] = gam[co] * v + bet[co];
+                        xh[co] = act_bf16 ? orc_round_bf16(v) : v;
+                    }
+                }
+                for (int co = 0; co < co_n; ++co) {
+                    double acc = z[co] > 0.0 ? z[co] : 0.0;
+                    z[co] = act_bf16 ? orc_round_bf16(acc) : acc;
+                }
+            }
+        if (m->norm) extra += (int64_t)Ho[l] * Wo[l] * (co_n + 1);
         x = y;
         hin = Ho[l];
         win = Wo[l];
         cin = co_n;
     }
-    /* global average pool, then concatenate proprio */
+    /* global average pool (or, with embed > 0, flatten -> fully connected -> ReLU), then concatenate proprio */
     double *h = x + (int64_t)hin * win * cin;
-    for (int c = 0; c < cin; ++c) {
-        double s = 0.0;
-        for (int px = 0; px < hin * win; ++px) s += x[(int64_t)px * cin + c];
-        h[c] = s / (double)(hin * win);
-        if (act_bf16) h[c] = orc_round_bf16(h[c]);
+    int feat = cin;
+    if (m->embed > 0) {
+        const double *We = th + offs[ti], *be = th + offs[ti + 1];
+        ti += 2;
+        int64_t flat = (int64_t)hin * win * cin;
+        feat = m->embed;
+        for (int e = 0; e < feat; ++e) {
+            double acc = be[e];
+            for (int64_t i = 0; i < flat; ++i) acc += We[(int64_t)e * flat + i] * x[i];
+            acc = acc > 0.0 ? acc : 0.0;
+            h[e] = act_bf16 ? orc_round_bf16(acc) : acc;
+        }
+    } else {
+        for (int c = 0; c < cin; ++c) {
+            double s = 0.0;
+            for (int px = 0; px < hin * win; ++px) s += x[(int64_t)px * cin + c];
+            h[c] = s / (double)(hin * win);
+            if (act_bf16) h[c] = orc_round_bf16(h[c]);
+        }
     }
-    for (int j = 0; j < m->P; ++j) h[cin + j] = act_bf16 ? orc_round_bf16(proprio[j]) : proprio[j];
-    int in = cin + m->P;
+    for (int j = 0; j < m->P; ++j) h[feat + j] = act_bf16 ? orc_round_bf16(proprio[j]) : proprio[j];
+    int in = feat + m->P;
     for (int l = 0; l < m->n_fc; ++l) {
         const double *Wt = th + offs[ti], *b = th + offs[ti + 1];
         ti += 2;
@@ -347,7 +427,17 @@ static void bwd_one(const orc_model *m, const double *th, const int64_t *offs, i
     const double *hv[ORC_MAX_FC + 1];
     int hn[ORC_MAX_FC + 1];
     hv[0] = a[L] + (int64_t)hs[L] * ws[L] * cs[L];
-    hn[0] = cs[L] + m->P;
+    hn[0] = (m->embed > 0 ? m->embed : cs[L]) + m->P;
+    /* xhat_l and rstd_l of the normalised layers sit behind the main record */
+    const double *xh[ORC_MAX_CONV + 1], *rs[ORC_MAX_CONV + 1];
+    {
+        const double *e = act + act_main_len(m);
+        for (int l = 1; l <= L; ++l) {
+            xh[l] = e;
+            rs[l] = e + (int64_t)hs[l] * ws[l] * cs[l];
+            e += (int64_t)hs[l] * ws[l] * (cs[l] + 1);
+        }
+    }
     for (int l = 0; l < F; ++l) { hv[l + 1] = hv[l] + hn[l]; hn[l + 1] = m->fc[l]; }
 
     /* scratch: two ping-pong gradient buffers large enough for any activation */
@@ -389,8 +479,24 @@ static void bwd_one(const orc_model *m, const double *th, const int64_t *offs, i
         }
         double *tmp = d_cur; d_cur = d_prev; d_prev = tmp;
     }
-    /* un-pool: every pixel of the last conv output gets dg[c] / (Ho*Wo); the proprio part ends here */
-    {
+    /* un-pool: every pixel of the last conv output gets dg[c] / (Ho*Wo); the proprio part ends here.
+     * With embed > 0: back through ReLU and the fully connected embedding into the flattened conv output. */
+    if (m->embed > 0) {
+        ti -= 2;
+        const double *We = th + offs[ti];
+        double *gW = g + offs[ti], *gb = g + offs[ti + 1];
+        int64_t flat = (int64_t)hs[L] * ws[L] * cs[L];
+        for (int64_t i = 0; i < flat; ++i) d_prev[i] = 0.0;
+        for (int e = 0; e < m->embed; ++e) {
+            double dz = hv[0][e] > 0.0 ? d_cur[e] : 0.0;
+            gb[e] += dz;
+            for (int64_t i = 0; i < flat; ++i) {
+                gW[(int64_t)e * flat + i] += dz * a[L][i];
+                d_prev[i] += We[(int64_t)e * flat + i] * dz;
+            }
+        }
+        double *tmp = d_cur; d_cur = d_prev; d_prev = tmp;
+    } else {
         int npx = hs[L] * ws[L], c_n = cs[L];
         for (int px = 0; px < npx; ++px)
             for (int c = 0; c < c_n; ++c) d_prev[(int64_t)px * c_n + c] = d_cur[c] / (double)npx;
@@ -398,6 +504,14 @@ static void bwd_one(const orc_model *m, const double *th, const int64_t *offs, i
     }
     /* conv layers, last to first; d_cur holds dL/da_l (post-ReLU) */
     for (int l = L; l >= 1; --l) {
+        const double *gam = NULL;
+        double *ggam = NULL, *gbet = NULL;
+        if (m->norm) {
+            ti -= 2;
+            gam = th + offs[ti];
+            ggam = g + offs[ti];
+            gbet = g + offs[ti + 1];
+        }
         ti -= 2;
         int k = m->conv_k[l - 1], p = k / 2, co_n = cs[l], cin = cs[l - 1];
         int hin = hs[l - 1], win = ws[l - 1];
@@ -406,10 +520,30 @@ static void bwd_one(const orc_model *m, const double *th, const int64_t *offs, i
         const double *x = a[l - 1], *y = a[l];
         if (l > 1) for (int64_t i = 0; i < (int64_t)hin * win * cin; ++i) d_prev[i] = 0.0;
         for (int oh = 0; oh < hs[l]; ++oh)
-            for (int ow = 0; ow < ws[l]; ++ow)
+            for (int ow = 0; ow < ws[l]; ++ow) {
+                int64_t px = (int64_t)oh * ws[l] + ow;
+                if (m->norm) {
+                    /* through ReLU and the normalisation of this pixel, in place in d_cur:
+                     * dy = ReLU'(.) d;  dgamma += dy xhat;  dbeta += dy;  t = gamma dy;
+                     * dz = rstd (t - mean(t) - xhat mean(t xhat)) */
+                    double *d = d_cur + px * co_n;
+                    const double *v = xh[l] + px * co_n;
+                    double m1 = 0.0, m2 = 0.0;
+                    for (int co = 0; co < co_n; ++co) {
+                        double dy = y[px * co_n + co] > 0.0 ? d[co] : 0.0;
+                        ggam[co] += dy * v[co];
+                        gbet[co] += dy;
+                        d[co] = gam[co] * dy;
+                        m1 += d[co];
+                        m2 += d[co] * v[co];
+                    }
+                    m1 /= (double)co_n;
+                    m2 /= (double)co_n;
+                    for (int co = 0; co < co_n; ++co) d[co] = rs[l][px] * (d[co] - m1 - v[co] * m2);
+                }
                 for (int co = 0; co < co_n; ++co) {
-                    int64_t oi = ((int64_t)oh * ws[l] + ow) * co_n + co;
-                    double dz = y[oi] > 0.0 ? d_cur[oi] : 0.0;
+                    int64_t oi = px * co_n + co;
+                    double dz = m->norm ? d_cur[oi] : (y[oi] > 0.0 ? d_cur[oi] : 0.0);
                     if (dz == 0.0) continue;
                     gb[co] += dz;
                     for (int kh = 0; kh < k; ++kh) {
@@ -427,6 +561,7 @@ static void bwd_one(const orc_model *m, const double *th, const int64_t *offs, i
                         }
                     }
                 }
+            }
         double *tmp = d_cur; d_cur = d_prev; d_prev = tmp;
     }
 }
@@ -436,7 +571,7 @@ int64_t orc_bwd_scratch_len(const orc_model *m) {
     orc_conv_shapes(m, Ho, Wo);
     int64_t big = (int64_t)m->H * m->W;
     for (int l = 0; l < m->n_conv; ++l) { int64_t s = (int64_t)Ho[l] * Wo[l] * m->conv_c[l]; if (s > big) big = s; }
-    int64_t h0 = m->conv_c[m->n_conv - 1] + m->P;
+    int64_t h0 = (m->embed > 0 ? m->embed : m->conv_c[m->n_conv - 1]) + m->P;
     if (h0 > big) big = h0;
     for (int l = 0; l < m->n_fc; ++l) if (m->fc[l] > big) big = m->fc[l];
     return 2 * big;
@@ -446,8 +581,8 @@ int64_t orc_bwd_scratch_len(const orc_model *m) {
  * bf16-rounded (orc_round_weights).  acts: B * orc_act_stride doubles (kept for backward). */
 void orc_encoder_fwd(const orc_model *m, const double *theta_used, int B, const double *depth, const double *proprio,
                      double *acts, double *mu, double *V, int act_bf16) {
-    int64_t offs[2 * ORC_MAX_CONV + 2 * ORC_MAX_FC + 3], szs[2 * ORC_MAX_CONV + 2 * ORC_MAX_FC + 3];
-    int32_t mat[2 * ORC_MAX_CONV + 2 * ORC_MAX_FC + 3], n;
+    int64_t offs[ORC_MAX_TENSORS], szs[ORC_MAX_TENSORS];
+    int32_t mat[ORC_MAX_TENSORS], n;
     orc_param_layout(m, offs, szs, mat, &n);
     int64_t stride = orc_act_stride(m);
 #pragma omp parallel for schedule(dynamic)
@@ -460,8 +595,8 @@ void orc_encoder_fwd(const orc_model *m, const double *theta_used, int B, const 
  * per-sample gradient, given dL/dmu [B][A] and dL/dV [B]. */
 void orc_encoder_bwd(const orc_model *m, const double *theta_used, int B, const double *acts, const double *dmu,
                      const double *dV, double *grad) {
-    int64_t offs[2 * ORC_MAX_CONV + 2 * ORC_MAX_FC + 3], szs[2 * ORC_MAX_CONV + 2 * ORC_MAX_FC + 3];
-    int32_t mat[2 * ORC_MAX_CONV + 2 * ORC_MAX_FC + 3], n;
+    int64_t offs[ORC_MAX_TENSORS], szs[ORC_MAX_TENSORS];
+    int32_t mat[ORC_MAX_TENSORS], n;
     int64_t total = orc_param_layout(m, offs, szs, mat, &n);
     int64_t stride = orc_act_stride(m);
     int64_t slen = orc_bwd_scratch_len(m);
