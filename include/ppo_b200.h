@@ -254,7 +254,8 @@ int ppo_encoder_bwd(ppo_model *m, const ppo_minibatch *mb, int row0, int rows, c
  * conv activation of layer `index` in 1..n_conv, NHWC bf16 [rows][Ho][Wo][C]; kind 1 = h_index
  * for index in 0..n_fc, bf16 [rows][width] (h_0 = [pooled, proprio]); kind 2 = the ReLU gate bits of conv
  * activation `index` (only for layers below the last whose channel count is a multiple of 32, else INVALID_ARG),
- * uint32 [rows][Ho][Wo][C/32], bit c % 32 of word c / 32 set where the activation is > 0.  *elems is the capacity
+ * uint32 [rows][Ho][Wo][C/32]; channel c belongs to word c / 32 and sits at bit ((c % 32) / 2) + 16 * (c % 2) of it (the
+ * two halves of a packed pair of bf16 values own bits j and 16 + j), set where the activation is > 0.  *elems is the capacity
  * for the bound micro-batch.  For inspection and for tests that substitute the saved
  * activations between ppo_encoder_fwd and ppo_encoder_bwd. */
 int ppo_model_activation_ptr(const ppo_model *m, int kind, int index, void **dev_ptr, size_t *elems);

@@ -82,6 +82,12 @@ struct ppo_model {
     bf16 *wC;                      // conv weights regrouped for the merged dgrad: Wc[class*Ci+ci][shift][co]
     int64_t wC_off[PPO_MAX_CONV + 1];  // per conv layer l (2..L)
     size_t wC_elems;
+    // scratch of the two-stage (reproducible) gradient reductions, per weight-matrix tensor index
+    float *wg_part[2 * PPO_MAX_CONV + 2 * PPO_MAX_FC + 3];  // partial tiles of the split-K weight-gradient GEMMs
+    size_t wg_cap[2 * PPO_MAX_CONV + 2 * PPO_MAX_FC + 3];   // floats
+    float *cs_part[2 * PPO_MAX_CONV + 2 * PPO_MAX_FC + 3];  // per-block partial column sums (bias gradients)
+    float *c1_part;                                         // per-block partial sums of the first layer's gradients
+    size_t c1_cap;
     float *loss_partials;
     float *act_mean;               // [mb][A]: Gaussian mean of ppo_policy_act before sampling
     int loss_partial_blocks;

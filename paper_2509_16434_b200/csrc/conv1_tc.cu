@@ -3,11 +3,18 @@
 // Per output pixel the layer is a dot product of k*k depth values with each of C1 filters: far too short a
 // reduction for the CUDA cores to do cheaply (C1 * k*k multiply-adds per pixel, one instruction each), but
 // one tcgen05.mma of K = 16 covers a 3x3 window for 128 pixels and all filters at once.  Producer threads
-// build the im2col tile themselves -- one pixel per thread, its k*k fp16 depth values (zero padded to a
-// multiple of 16) -- directly in the unswizzled K-major core-matrix layout (8 rows x 16 bytes per core
-// matrix); the filters are converted from the bf16 shadow to fp16 once per CTA, so that both operands are
-// fp16 and the depth values enter exactly.  fp32 accumulation in tensor memory, bias + ReLU + bf16 in the
-// epilogue, which also writes the one-bit ReLU gates the backward pass reads.
+// build the im2col tile themselves, one pixel per thread, directly in the unswizzled K-major core-matrix
+// layout (8 rows x 16 bytes per core matrix).  A window row starts at an even or odd column of the frame, so
+// the thread fetches it as aligned pairs of fp16 pixels (32-bit loads) and stores the pairs as they are: the
+// K axis is laid out as (window row, pair, element of the pair), with one element per row that lies outside
+// the window and meets a zero filter entry.  Nothing is unpacked or repacked, so the producer is a stream of
+// loads and stores.  The filters are converted from the bf16 shadow to fp16 once per CTA, so that both
+// operands are fp16 and the depth values enter exactly; the bias rides in two spare K slots as a pair of fp16
+// values (high part, remainder) against a constant 1.  fp32 accumulation in tensor memory; the epilogue is
+// ReLU + bf16 conversion in one instruction per pair, the one-bit ReLU gates the backward pass reads, and a
+// pass through shared memory so that every store instruction of a warp writes contiguous bytes.
+// Frames must hold finite values (an Inf or NaN beside a window would meet a zero weight) and have an even
+// width.
 #include "gemm.cuh"
 #include "tcgen05.cuh"
 
@@ -27,7 +34,7 @@ struct Args {
     bf16 *out;          // [M][C1]
     uint32_t *bits;     // [M][C1 / 32] or null
     long long M;        // output pixels
-    int Hi, Wi, Ho, Wo, C1, KP;  // KP = k*k rounded up to 16
+    int Hi, Wi, Ho, Wo, C1;
     int tiles;   // 128-pixel tiles
     int T;       // tiles per stage (one barrier round trip and one accumulator hand-over per T tiles)
     int stages;
@@ -41,7 +48,7 @@ struct Pipe {
     uint64_t tempty[4];
     uint32_t tmem_slot;
     int abort_flag;
-    alignas(16) float bias[256];
+    alignas(16) uint32_t pad[2];
 };
 
 // Unswizzled K-major operand image: element (row r, column k) of a tile with KP columns lives at
@@ -60,9 +67,20 @@ __host__ __device__ constexpr uint32_t idesc_f16(int M, int N) {
     return (1u << 4) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
 }
 
+// K layout of a window of size KS: window row kh holds NP pairs; pair q covers frame columns
+// 2 ow - P - ODD + 2 q (+1), element e of it is kernel column 2 q + e - ODD (outside 0 .. KS-1: zero filter entry).
+// Halves 2 KS NP and 2 KS NP + 1 carry the constant 1 for the two bias parts; the rest up to KP are zero.
+template <int KS>
+struct Win {
+    static constexpr int P = KS / 2, ODD = P & 1, NP = (KS + ODD + 1) / 2;
+    static constexpr int KW = KS * NP;                     // 32-bit words of window data
+    static constexpr int KP = (2 * KW + 2 + 15) / 16 * 16; // halves per im2col row
+};
+
 template <int KS>
 __global__ void __launch_bounds__(kThreads, 1) conv1_tc_kernel(const __grid_constant__ Args a) {
-    constexpr int K2 = KS * KS, KP = (K2 + 15) / 16 * 16, P = KS / 2;
+    using WN = Win<KS>;
+    constexpr int K2 = KS * KS, KP = WN::KP, P = WN::P, ODD = WN::ODD, NP = WN::NP, KW = WN::KW;
     constexpr uint32_t kTileBytes = 128u * KP * 2u;
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -70,6 +88,7 @@ __global__ void __launch_bounds__(kThreads, 1) conv1_tc_kernel(const __grid_cons
     const uint32_t stage_bytes = (uint32_t)T * kTileBytes;
     uint8_t *bsm = smem + (size_t)S * stage_bytes;                 // filters [N][KP] fp16
     Pipe *pipe = reinterpret_cast<Pipe *>(bsm + ((N * KP * 2 + 1023) / 1024) * 1024);
+    uint4 *staging = reinterpret_cast<uint4 *>(pipe + 1);          // per epilogue warp 32 pixels x 64 bytes
     volatile int *abort_flag = &pipe->abort_flag;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t acc_cols = tmem_cols_for(T * N);                // T accumulators side by side
@@ -88,12 +107,19 @@ __global__ void __launch_bounds__(kThreads, 1) conv1_tc_kernel(const __grid_cons
         pipe->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    for (int i = threadIdx.x; i < N; i += kThreads) pipe->bias[i] = a.bias[i];
-    // filters: zero padded columns included
+    // filters in the K layout of the window, bias parts in the two slots behind it, zeros elsewhere
     for (int i = threadIdx.x; i < N * KP; i += kThreads) {
         const int n = i / KP, k = i - n * KP;
-        const __half h = k < K2 ? __float2half_rn(bf2f(a.W[n * K2 + k])) : __float2half_rn(0.f);
-        *reinterpret_cast<__half *>(bsm + core_offset(n, k >> 3, KP) + (k & 7) * 2) = h;
+        float f = 0.f;
+        if (k < 2 * KW) {
+            const int w = k >> 1, kh = w / NP, kw = 2 * (w - kh * NP) + (k & 1) - ODD;
+            if (kw >= 0 && kw < KS) f = bf2f(a.W[n * K2 + kh * KS + kw]);
+        } else if (k == 2 * KW) {
+            f = __half2float(__float2half_rn(a.bias[n]));
+        } else if (k == 2 * KW + 1) {
+            f = a.bias[n] - __half2float(__float2half_rn(a.bias[n]));
+        }
+        *reinterpret_cast<__half *>(bsm + core_offset(n, k >> 3, KP) + (k & 7) * 2) = __float2half_rn(f);
     }
     fence_async_smem();
     if (warp == kProdGroups * 4) tmem_alloc(&pipe->tmem_slot, ncols);
@@ -117,6 +143,7 @@ __global__ void __launch_bounds__(kThreads, 1) conv1_tc_kernel(const __grid_cons
             // divisions
             const int step = T * 128, hw = a.Ho * a.Wo;
             const int d_b = step / hw, d_oh = (step % hw) / a.Wo, d_ow = step % a.Wo;
+            const int Wh = a.Wi >> 1;  // 32-bit words per frame row
             int ow, oh, ib;
             long long m = ((long long)s0 * T + grp) * 128 + r;
             {
@@ -130,32 +157,33 @@ __global__ void __launch_bounds__(kThreads, 1) conv1_tc_kernel(const __grid_cons
             for (int li = 0; li < ns && ok; ++li, m += step) {
                 ok = mbar_wait(&pipe->empty[s], ph ^ 1u, abort_flag, a.status);
                 if (!ok) break;
-                unsigned short hv[KP];
+                uint32_t wv[KP / 2];
 #pragma unroll
-                for (int k = 0; k < KP; ++k) hv[k] = 0;
+                for (int k = 0; k < KP / 2; ++k) wv[k] = 0u;
+                wv[KW] = 0x3C003C00u;  // (1.0, 1.0): the bias slots
                 if (m < a.M) {
-                    const unsigned short *img =
-                        reinterpret_cast<const unsigned short *>(a.depth) + (long long)ib * a.Hi * a.Wi;
+                    const uint32_t *img = reinterpret_cast<const uint32_t *>(a.depth) + (long long)ib * a.Hi * Wh;
+                    const int pw0 = ow - (P + ODD) / 2;  // first pair of the window row, in words
 #pragma unroll
                     for (int kh = 0; kh < KS; ++kh) {
                         const int ih = 2 * oh + kh - P;
+                        if (ih >= 0 && ih < a.Hi) {
+                            const uint32_t *row = img + ih * Wh;
 #pragma unroll
-                        for (int kw = 0; kw < KS; ++kw) {
-                            const int iw = 2 * ow + kw - P;
-                            if (ih >= 0 && ih < a.Hi && iw >= 0 && iw < a.Wi) hv[kh * KS + kw] = __ldg(img + ih * a.Wi + iw);
+                            for (int qq = 0; qq < NP; ++qq) {
+                                const int pw = pw0 + qq;
+                                if (pw >= 0 && pw < Wh) wv[kh * NP + qq] = __ldg(row + pw);
+                            }
                         }
                     }
+                } else {
+                    wv[KW] = 0u;  // rows past the last pixel stay zero
                 }
                 uint8_t *dst = smem + (size_t)s * stage_bytes + (size_t)grp * kTileBytes;
 #pragma unroll
-                for (int c = 0; c < KP / 8; ++c) {
-                    uint4 v;
-                    v.x = hv[8 * c] | ((uint32_t)hv[8 * c + 1] << 16);
-                    v.y = hv[8 * c + 2] | ((uint32_t)hv[8 * c + 3] << 16);
-                    v.z = hv[8 * c + 4] | ((uint32_t)hv[8 * c + 5] << 16);
-                    v.w = hv[8 * c + 6] | ((uint32_t)hv[8 * c + 7] << 16);
-                    *reinterpret_cast<uint4 *>(dst + core_offset(r, c, KP)) = v;
-                }
+                for (int c = 0; c < KP / 8; ++c)
+                    *reinterpret_cast<uint4 *>(dst + core_offset(r, c, KP)) =
+                        make_uint4(wv[4 * c], wv[4 * c + 1], wv[4 * c + 2], wv[4 * c + 3]);
                 fence_async_smem();
                 mbar_arrive(&pipe->full[s]);
                 ow += d_ow;
@@ -198,14 +226,14 @@ __global__ void __launch_bounds__(kThreads, 1) conv1_tc_kernel(const __grid_cons
             if (++s == S) { s = 0; ph ^= 1u; }
         }
     } else {
-        // ---------------- epilogue: TMEM lane = pixel of a tile; warp w reads lanes 32 (w % 4) .. +31
-        const int lg = warp & 3, half = (warp - (kProdGroups * 4 + 1)) >> 2;
+        // ---------------- epilogue: TMEM lane = pixel of a tile; warp w reads lanes 32 (w % 4) .. +31; the two
+        // warps of a lane quarter take alternate groups of 32 accumulator columns (16 when C1 is not a multiple
+        // of 32)
+        const int ew = warp - (kProdGroups * 4 + 1), lg = warp & 3, half = ew >> 2;
         const int p = lg * 32 + lane;
-        unsigned short *bits16 = reinterpret_cast<unsigned short *>(a.bits);
-        float bv[16];  // with N = 32 a warp always meets the same 16 columns
-#pragma unroll
-        for (int i = 0; i < 16; ++i) bv[i] = pipe->bias[(half * 16 + i) % N];
-        const bool fixed_cols = N == 32;
+        const int CW = (N & 31) == 0 ? 32 : 16;
+        uint4 *stg = staging + (size_t)ew * 128;
+        const int sw = (lane >> 1) & 3, rr0 = lane >> 2, piece = lane & 3;
         bool ok = true;
         for (int li = 0; li < ns && ok; ++li) {
             const int acc = li & (nacc - 1);
@@ -213,36 +241,38 @@ __global__ void __launch_bounds__(kThreads, 1) conv1_tc_kernel(const __grid_cons
             if (!ok) break;
             tc_fence_after();
             const uint32_t lane_base = tmem_base + acc * acc_cols + ((uint32_t)(lg * 32) << 16);
-            for (int cc = half * 16; cc < T * N; cc += 32) {   // column of the accumulator: tile g, channel c0
+            for (int cc = half * CW; cc < T * N; cc += 2 * CW) {   // column of the accumulator: tile g, channel c0
                 const int g = cc / N, c0 = cc - g * N;
-                const long long m = ((long long)(s0 + li) * T + g) * 128 + p;
-                float v[16];
+                const long long m0 = ((long long)(s0 + li) * T + g) * 128 + lg * 32;  // first pixel of this warp
+                float v[32];
                 tmem_ld16(lane_base + (uint32_t)cc, v);
-                uint4 o[2];
-                __nv_bfloat162 *pk = reinterpret_cast<__nv_bfloat162 *>(o);
+                if (CW == 32) tmem_ld16(lane_base + (uint32_t)cc + 16u, v + 16);
+                uint32_t pk[16];
+                uint32_t gate = 0;
 #pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                    const float b0 = fixed_cols ? bv[2 * j] : pipe->bias[c0 + 2 * j];
-                    const float b1 = fixed_cols ? bv[2 * j + 1] : pipe->bias[c0 + 2 * j + 1];
-                    v[2 * j] = fmaxf(v[2 * j] + b0, 0.f);
-                    v[2 * j + 1] = fmaxf(v[2 * j + 1] + b1, 0.f);
-                    pk[j] = __floats2bfloat162_rn(v[2 * j], v[2 * j + 1]);
-                }
-                if (m < a.M) {
-                    uint4 *op = reinterpret_cast<uint4 *>(a.out + m * N + c0);
-                    op[0] = o[0];
-                    op[1] = o[1];
-                    if (bits16) {  // 16 gate bits = one half of a 32-channel word
-                        uint32_t gate = 0;
-#pragma unroll
-                        for (int i = 0; i < 16; ++i) gate |= (v[i] > 0.f ? 1u : 0u) << i;
-                        bits16[m * (N >> 4) + (c0 >> 4)] = (unsigned short)gate;
+                for (int j = 0; j < 16; ++j) {
+                    if (j < CW / 2) {
+                        pk[j] = relu_pack_bf16x2(v[2 * j], v[2 * j + 1]);
+                        gate = gate_bits_add(gate, pk[j], j);
                     }
                 }
+#pragma unroll
+                for (int j = 0; j < 4; ++j)
+                    if (j < CW / 8) stg[lane * 4 + (j ^ sw)] = make_uint4(pk[4 * j], pk[4 * j + 1], pk[4 * j + 2], pk[4 * j + 3]);
+                if (a.bits && m0 + lane < a.M) a.bits[(m0 + lane) * (N >> 5) + (c0 >> 5)] = gate;
+                __syncwarp();
+#pragma unroll
+                for (int ps = 0; ps < 4; ++ps) {
+                    const int rr = ps * 8 + rr0;
+                    if (m0 + rr < a.M && piece < CW / 8)
+                        *reinterpret_cast<uint4 *>(a.out + (m0 + rr) * N + c0 + piece * 8) = stg[rr * 4 + (piece ^ ((rr >> 1) & 3))];
+                }
+                __syncwarp();
             }
             tc_fence_before();
             mbar_arrive(&pipe->tempty[acc]);
         }
+        (void)p;
     }
     tc_fence_before();
     __syncthreads();
@@ -254,7 +284,7 @@ __global__ void __launch_bounds__(kThreads, 1) conv1_tc_kernel(const __grid_cons
 
 template <int KS>
 int launch(Args &a, cudaStream_t st) {
-    constexpr int KP = (KS * KS + 15) / 16 * 16;
+    constexpr int KP = Win<KS>::KP;
     // tiles per stage: as many accumulators as fit twice into the 512 columns of tensor memory, at most one per
     // producer group
     a.T = 256 / a.C1 < kProdGroups ? 256 / a.C1 : kProdGroups;
@@ -263,7 +293,8 @@ int launch(Args &a, cudaStream_t st) {
     a.stages = (int)((128 * 1024) / stage);
     if (a.stages > kMaxStages) a.stages = kMaxStages;
     if (a.stages < 2) return PPO_ERR_UNSUPPORTED;
-    const size_t smem = (size_t)a.stages * stage + ((size_t)(a.C1 * KP * 2 + 1023) / 1024) * 1024 + sizeof(Pipe) + 1024;
+    const size_t smem = (size_t)a.stages * stage + ((size_t)(a.C1 * KP * 2 + 1023) / 1024) * 1024 + sizeof(Pipe) +
+                        (size_t)kEpiWarps * 2048 + 1024;
     static bool attr_set[64] = {false};
     int dev = 0;
     PPO_CUDA_CHECK(cudaGetDevice(&dev));
@@ -284,15 +315,15 @@ int launch(Args &a, cudaStream_t st) {
 
 // out[m][co] = relu(bias[co] + sum_tap depth(m, tap) * W[co][tap]) as bf16; `bits` (optional, C1 % 32 == 0) gets the
 // ReLU gates.  Returns PPO_ERR_UNSUPPORTED (nothing launched) for shapes it does not cover: C1 must be a multiple
-// of 16 up to 256 (of 32 when bits are wanted), k in {3, 5, 7}.
+// of 16 up to 256 (of 32 when bits are wanted), k in {3, 5, 7}, the frame width even and the frames 4-byte aligned.
 int conv1_tc_fwd(const __half *depth, const bf16 *W, const float *bias, bf16 *out, uint32_t *bits, int rows, int Hi,
                  int Wi, int Ho, int Wo, int C1, int ks, int32_t *status, cudaStream_t st) {
     if (!status || C1 % 16 != 0 || C1 > 256 || C1 < 16 || (bits && C1 % 32 != 0)) return PPO_ERR_UNSUPPORTED;
+    if (Wi % 2 != 0 || !ppo_aligned(depth, 4)) return PPO_ERR_UNSUPPORTED;
     Args a;
     a.depth = depth; a.W = W; a.bias = bias; a.out = out; a.bits = bits;
     a.M = (long long)rows * Ho * Wo;
     a.Hi = Hi; a.Wi = Wi; a.Ho = Ho; a.Wo = Wo; a.C1 = C1;
-    a.KP = (ks * ks + 15) / 16 * 16;
     const long long tiles = (a.M + 127) / 128;
     if (tiles <= 0) return PPO_OK;
     if (tiles > 0x7fffffffll) return PPO_ERR_UNSUPPORTED;

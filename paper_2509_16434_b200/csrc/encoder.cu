@@ -73,7 +73,7 @@ __global__ void __launch_bounds__(128) conv1_fwd_kernel(const __half *__restrict
         for (int j = 0; j < 4; ++j) p[j] = __floats2bfloat162_rn(fmaxf(acc[2 * j], 0.f), fmaxf(acc[2 * j + 1], 0.f));
         if (bits) {
 #pragma unroll
-            for (int j = 0; j < 8; ++j) gate |= (acc[j] > 0.f ? 1u : 0u) << ((c8 & 31) + j);
+            for (int j = 0; j < 4; ++j) gate = gate_bits_add(gate, *reinterpret_cast<uint32_t *>(&p[j]), ((c8 & 31) >> 1) + j);
             if ((c8 & 31) == 24) {
                 if (live) bits[m * (C1 >> 5) + (c8 >> 5)] = gate;
                 gate = 0;
@@ -100,11 +100,12 @@ __global__ void __launch_bounds__(128) conv1_fwd_kernel(const __half *__restrict
 // once per CPT * (k*k + 1) multiply-adds.  All loads of a trip (U steps) are issued before the first
 // use.  Every lane keeps CPT (k*k + 1) accumulators (the last of each channel is the bias gradient);
 // they are folded across the pixel slots of a warp by shuffles, across warps through shared memory,
-// then added with one atomic each.  C1 / CPT must be a power of two <= 32.
+// and left as this block's partial sums in part[blockIdx.x][C1 k*k (dW order) | C1 (db)], which
+// sum_partials_kernel adds up in block order.  C1 / CPT must be a power of two <= 32.
 template <int KS, int CPT, int U>
 __global__ void __launch_bounds__(128) conv1_wgrad_kernel(const __half *__restrict__ depth,
-                                                          const bf16 *__restrict__ dZ, float *__restrict__ dW,
-                                                          float *__restrict__ db, int rows, int Hi, int Wi, int Ho,
+                                                          const bf16 *__restrict__ dZ, float *__restrict__ part,
+                                                          int rows, int Hi, int Wi, int Ho,
                                                           int Wo, int C1, long long px_per_warp) {
     constexpr int K2 = KS * KS, P = KS / 2;
     extern __shared__ float sm[];  // [4 warps][C1 * (K2 + 1)]
@@ -200,17 +201,18 @@ __global__ void __launch_bounds__(128) conv1_wgrad_kernel(const __half *__restri
         float v = 0.f;
         for (int w = 0; w < 4; ++w) v += sm[w * per + i];
         const int co = i / (K2 + 1), t = i % (K2 + 1);
-        if (t < K2) atomicAdd(dW + co * K2 + t, v);
-        else atomicAdd(db + co, v);
+        part[(size_t)blockIdx.x * per + (t < K2 ? co * K2 + t : C1 * K2 + co)] = v;
     }
 }
 
 // The same reduction on the tensor cores (mma.sync m16n8k16, bf16): per 16 output pixels a warp forms
-// D[tap][co] += X^T[tap][px] dZ[px][co] with the pixel index as K (32 pixels, one per lane, per trip).  The patch tile X (k*k depth taps as
-// bf16, then a column of ones whose product is the bias gradient, zero padded to TP) and the 16 x C1 gradient
-// tile go through per-warp shared memory and come back as fragments with ldmatrix.trans.  About 3 instructions
-// per pixel instead of C1 (k*k + 1) / 32 multiply-adds plus their loads: the kernel becomes a stream over dZ.
-// C1 must be a multiple of 16.
+// D[tap][co] += X^T[tap][px] dZ[px][co] with the pixel index as K (32 pixels, one per lane, per trip).  The patch tile X
+// and the 16 x C1 gradient tile go through per-warp shared memory and come back as fragments with ldmatrix.trans.
+// A lane fetches its pixel's window as aligned pairs of fp16 frame pixels (32-bit loads) and converts each pair to bf16
+// in three instructions; the tap axis is laid out as (window row, pair, element of the pair) -- one element per row lies
+// outside the window and its row of D is dropped -- followed by a column of ones whose product is the bias gradient,
+// zero padded to TP.  About 3 instructions per pixel and channel-independent instead of C1 (k*k + 1) / 32 multiply-adds
+// plus their loads: the kernel becomes a stream over dZ.  C1 must be a multiple of 16 and the frame width even.
 __device__ __forceinline__ void ldmatrix_x4_trans(uint32_t addr, uint32_t &r0, uint32_t &r1, uint32_t &r2, uint32_t &r3) {
     asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
                  : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
@@ -226,10 +228,11 @@ __device__ __forceinline__ void mma_bf16_16816(float (&d)[4], uint32_t a0, uint3
 
 template <int KS, int NB>  // NB = C1 / 8 column blocks
 __global__ void __launch_bounds__(256) conv1_wgrad_mma_kernel(const __half *__restrict__ depth,
-                                                              const bf16 *__restrict__ dZ, float *__restrict__ dW,
-                                                              float *__restrict__ db, int rows, int Hi, int Wi,
+                                                              const bf16 *__restrict__ dZ, float *__restrict__ part,
+                                                              int rows, int Hi, int Wi,
                                                               int Ho, int Wo, long long px_per_warp) {
-    constexpr int K2 = KS * KS, P = KS / 2, TP = (K2 + 1 + 15) / 16 * 16, MB = TP / 16, C1 = NB * 8;
+    constexpr int K2 = KS * KS, P = KS / 2, ODD = P & 1, NP = (KS + ODD + 1) / 2, KW = KS * NP;
+    constexpr int TP = (2 * KW + 1 + 15) / 16 * 16, MB = TP / 16, C1 = NB * 8;
     constexpr int PX = 32;  // pixels per trip: one per lane, two K = 16 steps of the MMA
     constexpr int kXBytes = PX * TP * 2, kZBytes = PX * C1 * 2;
     extern __shared__ __align__(16) uint8_t smw[];  // per warp: X tile [32 px][TP], dZ tile [32 px][C1]; later the reduction
@@ -261,28 +264,35 @@ __global__ void __launch_bounds__(256) conv1_wgrad_mma_kernel(const __half *__re
     uint4 xreg[TP / 8], zreg[ZP];
     // Loads of the tile that starts at pixel mt into registers; they are issued one trip ahead, so that their
     // latency overlaps the previous tile's MMAs.
+    const int Wh = Wi >> 1;  // 32-bit words per frame row
     auto prefetch = [&](long long mt) {
         const bool live = mt + lane < m_end;
-        const __half *img = depth + b * Hi * Wi;
+        const uint32_t *img = reinterpret_cast<const uint32_t *>(depth) + b * Hi * Wh;
+        uint32_t wv[TP / 2];
 #pragma unroll
-        for (int c = 0; c < TP / 8; ++c) {  // 8 taps = one 16-byte piece
-            __nv_bfloat162 pk[4];
+        for (int k = 0; k < TP / 2; ++k) wv[k] = 0u;
+        if (live) {
+            wv[KW] = 0x00003F80u;  // (1.0, 0) as bf16: the bias-gradient column
+            const int pw0 = ow - (P + ODD) / 2;
 #pragma unroll
-            for (int j = 0; j < 8; ++j) {
-                const int tap = c * 8 + j;
-                float xv = 0.f;
-                if (tap < K2) {
-                    const int kh = tap / KS, kw = tap - kh * KS;
-                    const int ih = 2 * oh + kh - P, iw = 2 * ow + kw - P;
-                    if (live && ih >= 0 && ih < Hi && iw >= 0 && iw < Wi) xv = __half2float(__ldg(img + ih * Wi + iw));
-                } else if (tap == K2) {
-                    xv = live ? 1.f : 0.f;
+            for (int kh = 0; kh < KS; ++kh) {
+                const int ih = 2 * oh + kh - P;
+                if (ih >= 0 && ih < Hi) {
+                    const uint32_t *row = img + ih * Wh;
+#pragma unroll
+                    for (int q = 0; q < NP; ++q) {
+                        const int pw = pw0 + q;
+                        if (pw >= 0 && pw < Wh) {
+                            const uint32_t raw = __ldg(row + pw);
+                            const float2 f = __half22float2(*reinterpret_cast<const __half2 *>(&raw));
+                            wv[kh * NP + q] = pack_bf16x2(f.x, f.y);
+                        }
+                    }
                 }
-                if (j & 1) pk[j >> 1].y = __float2bfloat16_rn(xv);
-                else pk[j >> 1].x = __float2bfloat16_rn(xv);
             }
-            xreg[c] = *reinterpret_cast<uint4 *>(pk);
         }
+#pragma unroll
+        for (int c = 0; c < TP / 8; ++c) xreg[c] = make_uint4(wv[4 * c], wv[4 * c + 1], wv[4 * c + 2], wv[4 * c + 3]);
 #pragma unroll
         for (int z = 0; z < ZP; ++z) {
             const int i = lane + 32 * z;
@@ -348,18 +358,21 @@ __global__ void __launch_bounds__(256) conv1_wgrad_mma_kernel(const __half *__re
             }
     }
     __syncthreads();
-    for (int i = threadIdx.x; i < (K2 + 1) * C1; i += 256) {
+    for (int i = threadIdx.x; i < (2 * KW + 1) * C1; i += 256) {
+        const int t = i / C1, co = i - t * C1;   // row t of D: element t & 1 of pair (t >> 1) % NP of window row (t >> 1) / NP
+        const int kh = (t >> 1) / NP, kw = 2 * ((t >> 1) - kh * NP) + (t & 1) - ODD;
+        if (t < 2 * KW && (kw < 0 || kw >= KS)) continue;
         float v = 0.f;
         for (int w = 0; w < 8; ++w) v += red[(size_t)w * per + i];
-        const int tap = i / C1, co = i - tap * C1;
-        if (tap < K2) atomicAdd(dW + co * K2 + tap, v);
-        else atomicAdd(db + co, v);
+        // this block's partial sums, [C1 k*k (dW order) | C1 (db)]; sum_partials_kernel adds the blocks up in order
+        part[(size_t)blockIdx.x * (C1 * (K2 + 1)) + (t < 2 * KW ? co * K2 + kh * KS + kw : C1 * K2 + co)] = v;
     }
 }
 
 // ------------------------------------------------------------- small kernels ----
 
-// One thread per 32 channels of a pixel: the ReLU gate (act > 0) as a bit mask.
+// One thread per 32 channels of a pixel: the ReLU gate (act > 0) as a bit mask, channel c at bit
+// gate_bit_of_channel(c).
 __global__ void __launch_bounds__(256) relu_bits_kernel(const bf16 *__restrict__ act, uint32_t *__restrict__ bits,
                                                         long long words) {
     const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
@@ -373,8 +386,8 @@ __global__ void __launch_bounds__(256) relu_bits_kernel(const bf16 *__restrict__
 #pragma unroll
         for (int q = 0; q < 4; ++q) {
             const float2 f = __bfloat1622float2(h2[q]);
-            w |= (f.x > 0.f ? 1u : 0u) << (j * 8 + 2 * q);
-            w |= (f.y > 0.f ? 1u : 0u) << (j * 8 + 2 * q + 1);
+            w |= (f.x > 0.f ? 1u : 0u) << (j * 4 + q);
+            w |= (f.y > 0.f ? 1u : 0u) << (16 + j * 4 + q);
         }
     }
     bits[i] = w;
@@ -458,10 +471,35 @@ __global__ void __launch_bounds__(256) pack_dout_kernel(const float *__restrict_
     out[i] = __float2bfloat16_rn(v);
 }
 
-// db[n] += sum_m dZ[m][n]  (bias gradients), N a multiple of 8.  Threads walk (row, 8-column chunk)
-// pairs with 128-bit loads; threads that share a chunk are folded through shared memory.
+#define PPO_TRY(expr)                 \
+    do {                              \
+        int _s = (expr);              \
+        if (_s != PPO_OK) return _s;  \
+    } while (0)
+
+// dst[i] (i < nA: dstA[i], else dstB[i - nA]) += part[0][i] + part[1][i] + ... in that order: the second stage of the
+// reductions whose blocks leave partial sums instead of adding to the result with atomics (reproducible results).
+__global__ void __launch_bounds__(256) sum_partials_kernel(const float *__restrict__ part, int nparts, int nA,
+                                                           float *__restrict__ dstA, int nB, float *__restrict__ dstB) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    const int n = nA + nB;
+    if (i >= n) return;
+    float acc = 0.f;
+    for (int b = 0; b < nparts; ++b) acc += part[(size_t)b * n + i];
+    if (i < nA) dstA[i] += acc;
+    else dstB[i - nA] += acc;
+}
+
+static int sum_partials(const float *part, int nparts, int nA, float *dstA, int nB, float *dstB, cudaStream_t st) {
+    sum_partials_kernel<<<ppo_cdiv(nA + nB, 256), 256, 0, st>>>(part, nparts, nA, dstA, nB, dstB);
+    PPO_LAUNCH_CHECK();
+    return PPO_OK;
+}
+
+// part[block][n] = sum over this block's rows m of dZ[m][n]  (bias gradients, first stage), N a multiple of 8.  Threads
+// walk (row, 8-column chunk) pairs with 128-bit loads; threads that share a chunk are folded through shared memory.
 __global__ void __launch_bounds__(256) colsum_kernel(const bf16 *__restrict__ dZ, int ld, long long M, int N,
-                                                     float *__restrict__ db) {
+                                                     float *__restrict__ part) {
     __shared__ float sh[256][9];
     const int chunks = N >> 3;                    // 16-byte chunks per row
     const int rows_per_pass = 256 / chunks;       // whole rows covered by one pass of the block
@@ -489,13 +527,13 @@ __global__ void __launch_bounds__(256) colsum_kernel(const bf16 *__restrict__ dZ
         const int c = threadIdx.x >> 3, e = threadIdx.x & 7;
         float v = 0.f;
         for (int r = 0; r < rows_per_pass; ++r) v += sh[r * chunks + c][e];
-        atomicAdd(db + threadIdx.x, v);
+        part[(size_t)blockIdx.x * N + threadIdx.x] = v;
     }
 }
 
-// db[n] += sum_m dZ[m][n] for any N <= ld (used for the head, whose 13 columns sit in rows of 16).
+// The same first stage for any N <= ld (used for the head, whose 13 columns sit in rows of 16).
 __global__ void __launch_bounds__(256) colsum_small_kernel(const bf16 *__restrict__ dZ, int ld, long long M, int N,
-                                                           float *__restrict__ db) {
+                                                           float *__restrict__ part) {
     __shared__ float sh[256];
     for (int n = 0; n < N; ++n) {
         float v = 0.f;
@@ -507,7 +545,7 @@ __global__ void __launch_bounds__(256) colsum_small_kernel(const bf16 *__restric
             if (threadIdx.x < o) sh[threadIdx.x] += sh[threadIdx.x + o];
             __syncthreads();
         }
-        if (threadIdx.x == 0) atomicAdd(db + n, sh[0]);
+        if (threadIdx.x == 0) part[(size_t)blockIdx.x * N + n] = sh[0];
         __syncthreads();
     }
 }
@@ -567,51 +605,58 @@ static int run_dgrad(const ppo_model *m, const ConvGeom &g, const bf16 *dY, int 
     return tc_gemm_dgrad(g, dY, ldy, Wt, wt_ld, e, ppo_device_status_ptr(), st);
 }
 
-static int run_colsum(const bf16 *dZ, int ld, long long M, int N, float *db, cudaStream_t st);
+static int run_colsum(const bf16 *dZ, int ld, long long M, int N, float *db, float *part, cudaStream_t st);
 
-// Weight and bias gradients of one layer.  The TMA kernel of a convolution sums the bias gradient on the
-// tensor core on its way; everything else reduces dY in a pass of its own.
-static int run_wgrad(const ppo_model *m, const ConvGeom &g, const bf16 *dY, int ldy, const bf16 *X, float *dW,
-                     float *db, cudaStream_t st) {
+// Weight and bias gradients of the layer whose weight matrix is tensor ti.  The TMA kernel of a convolution sums
+// the bias gradient on the tensor core on its way; everything else reduces dY in a pass of its own.
+static int run_wgrad(const ppo_model *m, int ti, const ConvGeom &g, const bf16 *dY, int ldy, const bf16 *X,
+                     cudaStream_t st) {
+    float *dW = m->grad + m->tensors[ti].off, *db = m->grad + m->tensors[ti + 1].off;
+    float *part = m->wg_part[ti];
+    const size_t cap = m->wg_cap[ti];
     const bool conv = g.k > 1;
-    int s = tma_gemm_wgrad(g, dY, ldy, X, dW, conv ? db : nullptr, ppo_device_status_ptr(), st);
+    int s = tma_gemm_wgrad(g, dY, ldy, X, dW, conv ? db : nullptr, part, cap, ppo_device_status_ptr(), st);
     if (s == PPO_OK && conv) return s;
-    if (s == PPO_ERR_UNSUPPORTED && conv) s = tma_gemm_wgrad(g, dY, ldy, X, dW, nullptr, ppo_device_status_ptr(), st);
-    if (s == PPO_ERR_UNSUPPORTED) s = tc_gemm_wgrad(g, dY, ldy, X, dW, ppo_device_status_ptr(), st);
+    if (s == PPO_ERR_UNSUPPORTED && conv) s = tma_gemm_wgrad(g, dY, ldy, X, dW, nullptr, part, cap, ppo_device_status_ptr(), st);
+    if (s == PPO_ERR_UNSUPPORTED) s = tc_gemm_wgrad(g, dY, ldy, X, dW, part, cap, ppo_device_status_ptr(), st);
     if (s != PPO_OK) return s;
-    return run_colsum(dY, ldy, g.M(), g.Co, db, st);
+    return run_colsum(dY, ldy, g.M(), g.Co, db, m->cs_part[ti], st);
 }
 
-static int run_colsum(const bf16 *dZ, int ld, long long M, int N, float *db, cudaStream_t st) {
+// Blocks a column sum of M rows is cut into (first stage), at most 4 per SM.
+static int colsum_blocks(long long M, long long rows_per_block) {
+    int blocks = ppo_cdiv(M, rows_per_block);
+    const int cap = ppo_num_sms() * 4;
+    return blocks > cap ? cap : (blocks < 1 ? 1 : blocks);
+}
+
+// db[n] += sum_m dZ[m][n] in two stages; `part` holds 4 x SMs x max(N, 16) floats.
+static int run_colsum(const bf16 *dZ, int ld, long long M, int N, float *db, float *part, cudaStream_t st) {
     if (N % 8 == 0 && N <= 256 && ld % 8 == 0) {
         const int rows_per_pass = 256 / (N / 8);
-        int blocks = ppo_cdiv(M, (long long)rows_per_pass * 8);
-        const int cap = ppo_num_sms() * 4;
-        blocks = blocks > cap ? cap : (blocks < 1 ? 1 : blocks);
-        colsum_kernel<<<blocks, 256, 0, st>>>(dZ, ld, M, N, db);
-    } else if (N > 256 && N % 256 == 0) {
-        // wide FC layers: one launch per 256-column slab
-        for (int n0 = 0; n0 < N; n0 += 256) {
-            int blocks = ppo_cdiv(M, 64);
-            const int cap = ppo_num_sms() * 4;
-            blocks = blocks > cap ? cap : (blocks < 1 ? 1 : blocks);
-            colsum_kernel<<<blocks, 256, 0, st>>>(dZ + n0, ld, M, 256, db + n0);
-            if (n0 + 256 < N) PPO_LAUNCH_CHECK();
-        }
-    } else {
-        int blocks = ppo_cdiv(M, 2048);
-        blocks = blocks > 64 ? 64 : (blocks < 1 ? 1 : blocks);
-        colsum_small_kernel<<<blocks, 256, 0, st>>>(dZ, ld, M, N, db);
+        const int blocks = colsum_blocks(M, (long long)rows_per_pass * 8);
+        colsum_kernel<<<blocks, 256, 0, st>>>(dZ, ld, M, N, part);
+        PPO_LAUNCH_CHECK();
+        return sum_partials(part, blocks, N, db, 0, nullptr, st);
     }
+    if (N > 256 && N % 256 == 0) {
+        // wide FC layers: one launch per 256-column slab
+        const int blocks = colsum_blocks(M, 64);
+        for (int n0 = 0; n0 < N; n0 += 256) {
+            float *p = part + (size_t)(n0 / 256) * blocks * 256;
+            colsum_kernel<<<blocks, 256, 0, st>>>(dZ + n0, ld, M, 256, p);
+            PPO_LAUNCH_CHECK();
+            PPO_TRY(sum_partials(p, blocks, 256, db + n0, 0, nullptr, st));
+        }
+        return PPO_OK;
+    }
+    int blocks = ppo_cdiv(M, 2048);
+    blocks = blocks > 64 ? 64 : (blocks < 1 ? 1 : blocks);
+    colsum_small_kernel<<<blocks, 256, 0, st>>>(dZ, ld, M, N, part);
     PPO_LAUNCH_CHECK();
-    return PPO_OK;
+    return sum_partials(part, blocks, N, db, 0, nullptr, st);
 }
 
-#define PPO_TRY(expr)                 \
-    do {                              \
-        int _s = (expr);              \
-        if (_s != PPO_OK) return _s;  \
-    } while (0)
 
 static int check_rows(const ppo_model *m, const ppo_minibatch *mb, int row0, int rows) {
     if (!m || !mb) return PPO_ERR_INVALID_ARG;
@@ -736,9 +781,9 @@ static int conv1_wgrad(ppo_model *m, const ppo_minibatch *mb, int row0, int rows
     const __half *depth = static_cast<const __half *>(mb->depth_f16) + (size_t)row0 * d.H * d.W;
     const int C1 = m->Cs[1], KS = d.conv_k[0];
     const long long M = (long long)rows * m->Hs[1] * m->Ws[1];
-    if (C1 % 16 == 0 && C1 <= 64 && (KS == 3 || KS == 5)) {
+    if (C1 % 16 == 0 && C1 <= 64 && (KS == 3 || KS == 5) && d.W % 2 == 0 && ppo_aligned(depth, 4)) {
         // tensor-core reduction
-        const int TP = (KS * KS + 1 + 15) / 16 * 16;
+        const int TP = KS == 3 ? 16 : 32;
         const size_t tile = (size_t)32 * TP * 2 + (size_t)32 * C1 * 2, redb = (size_t)TP * C1 * sizeof(float);
         const size_t smem = 8 * (tile > redb ? tile : redb);
         int blocks = ppo_cdiv(M, 8 * 16 * 8);
@@ -747,12 +792,13 @@ static int conv1_wgrad(ppo_model *m, const ppo_minibatch *mb, int row0, int rows
         long long per_warp = (M + (long long)blocks * 8 - 1) / ((long long)blocks * 8);
         per_warp = (per_warp + 31) / 32 * 32;
         float *dW = m->grad + m->tensors[0].off, *db = m->grad + m->tensors[1].off;
+        if ((size_t)blocks * C1 * (KS * KS + 1) > m->c1_cap) return PPO_ERR_SHAPE;
 #define PPO_C1W(KS_, NB_)                                                                                    \
     do {                                                                                                     \
         if (smem > 48 * 1024)                                                                                \
             PPO_CUDA_CHECK(cudaFuncSetAttribute(conv1_wgrad_mma_kernel<KS_, NB_>,                            \
                                                 cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));    \
-        conv1_wgrad_mma_kernel<KS_, NB_><<<blocks, 256, smem, st>>>(depth, m->dact[1], dW, db, rows, d.H,    \
+        conv1_wgrad_mma_kernel<KS_, NB_><<<blocks, 256, smem, st>>>(depth, m->dact[1], m->c1_part, rows, d.H, \
                                                                     d.W, m->Hs[1], m->Ws[1], per_warp);      \
     } while (0)
         const int nb = C1 / 8;
@@ -766,7 +812,7 @@ static int conv1_wgrad(ppo_model *m, const ppo_minibatch *mb, int row0, int rows
         else PPO_C1W(5, 8);
 #undef PPO_C1W
         PPO_LAUNCH_CHECK();
-        return PPO_OK;
+        return sum_partials(m->c1_part, blocks, C1 * KS * KS, dW, C1, db, st);
     }
     const int cpt = KS <= 3 ? 8 : (KS == 5 ? 4 : 2);
     const int lpp = C1 / cpt;
@@ -779,8 +825,9 @@ static int conv1_wgrad(ppo_model *m, const ppo_minibatch *mb, int row0, int rows
     long long per_warp = (M + (long long)blocks * 4 - 1) / ((long long)blocks * 4);
     per_warp = (per_warp + ppi - 1) / ppi * ppi;
     float *dW = m->grad + m->tensors[0].off, *db = m->grad + m->tensors[1].off;
+    if ((size_t)blocks * C1 * (KS * KS + 1) > m->c1_cap) return PPO_ERR_SHAPE;
 #define PPO_CONV1W(KS_, CPT_, U_)                                                                                 \
-    conv1_wgrad_kernel<KS_, CPT_, U_><<<blocks, 128, smem, st>>>(depth, m->dact[1], dW, db, rows, d.H, d.W,      \
+    conv1_wgrad_kernel<KS_, CPT_, U_><<<blocks, 128, smem, st>>>(depth, m->dact[1], m->c1_part, rows, d.H, d.W,  \
                                                              m->Hs[1], m->Ws[1], C1, per_warp)
     if (smem > 48 * 1024) {
         if (KS == 5) PPO_CUDA_CHECK(cudaFuncSetAttribute(conv1_wgrad_kernel<5, 4, 1>,
@@ -794,7 +841,7 @@ static int conv1_wgrad(ppo_model *m, const ppo_minibatch *mb, int row0, int rows
     else PPO_CONV1W(7, 2, 1);
 #undef PPO_CONV1W
     PPO_LAUNCH_CHECK();
-    return PPO_OK;
+    return sum_partials(m->c1_part, blocks, C1 * KS * KS, dW, C1, db, st);
 }
 
 extern "C" int ppo_encoder_bwd(ppo_model *m, const ppo_minibatch *mb, int row0, int rows, const float *dmean,
@@ -841,7 +888,7 @@ extern "C" int ppo_encoder_bwd(ppo_model *m, const ppo_minibatch *mb, int row0, 
         const int ldy = (l <= F) ? Co : 16;
         ConvGeom g = fc_geom(rows, m->hw[l - 1], Co);
         const bf16 *dY = m->dh[l];
-        int s = run_wgrad(m, g, dY, ldy, m->h[l - 1], m->grad + m->tensors[ti].off, m->grad + m->tensors[ti + 1].off, leaf);
+        int s = run_wgrad(m, ti, g, dY, ldy, m->h[l - 1], leaf);
         if (s != PPO_OK) return join(s);
         DgradEpilogue e;
         if (l > 1) e = {m->h[l - 1], m->dh[l - 1], nullptr};
@@ -869,8 +916,7 @@ extern "C" int ppo_encoder_bwd(ppo_model *m, const ppo_minibatch *mb, int row0, 
         e.mask_bits = m->abits[l - 1];
         int s = PPO_OK;
         if (!fork)
-            s = run_wgrad(m, g, m->dact[l], g.Co, m->act[l - 1], m->grad + m->tensors[ti].off,
-                          m->grad + m->tensors[ti + 1].off, st);
+            s = run_wgrad(m, ti, g, m->dact[l], g.Co, m->act[l - 1], st);
         if (s == PPO_OK)
             s = run_dgrad(m, g, m->dact[l], g.Co, m->shadow + m->tensors[ti].off, m->wT + m->wT_off[ti],
                           wt_ld_of(g.Co), m->wC + m->wC_off[l], e, st);
@@ -882,8 +928,7 @@ extern "C" int ppo_encoder_bwd(ppo_model *m, const ppo_minibatch *mb, int row0, 
         for (int l = 2; l <= L && s == PPO_OK; ++l) {  // conv2 first: the longest, and the best partner
             const int ti = 2 * (l - 1);
             ConvGeom g = conv_geom(m, l, rows);
-            s = run_wgrad(m, g, m->dact[l], g.Co, m->act[l - 1], m->grad + m->tensors[ti].off,
-                          m->grad + m->tensors[ti + 1].off, st);
+            s = run_wgrad(m, ti, g, m->dact[l], g.Co, m->act[l - 1], st);
         }
         return join(s);
     }

@@ -21,7 +21,7 @@ struct DgradEpilogue {
     const bf16 *mask_act;  // [M'][Ci]: output is zeroed where this is <= 0; may be nullptr
     bf16 *out;             // [M'][Ci] bf16, or nullptr
     float *out_f32;        // [M'][Ci] fp32, or nullptr
-    const uint32_t *mask_bits = nullptr;  // the same gate as one bit per element, [M'][Ci / 32] (bit c % 32 of word c / 32);
+    const uint32_t *mask_bits = nullptr;  // the same gate as one bit per element, [M'][Ci / 32] (channel c at bit gate_bit_of_channel(c) of word c / 32);
                                           // used instead of mask_act by kernels that support it
 };
 
@@ -31,8 +31,8 @@ int tc_gemm_fwd(const ConvGeom &g, const bf16 *X, const bf16 *W, const FwdEpilog
                 cudaStream_t st);
 int tc_gemm_dgrad(const ConvGeom &g, const bf16 *dY, int ldy, const bf16 *Wt, int wt_ld, const DgradEpilogue &e,
                   int32_t *status, cudaStream_t st);
-int tc_gemm_wgrad(const ConvGeom &g, const bf16 *dY, int ldy, const bf16 *X, float *dW, int32_t *status,
-                  cudaStream_t st);
+int tc_gemm_wgrad(const ConvGeom &g, const bf16 *dY, int ldy, const bf16 *X, float *dW, float *part, size_t part_elems,
+                  int32_t *status, cudaStream_t st);
 
 // TMA-fed versions of the same three operations (operand tiles moved by cp.async.bulk.tensor).  They cover
 // channel counts that are multiples of 32 (any multiple of 8 that is at least 64 for a fully connected layer);
@@ -47,8 +47,14 @@ size_t tma_dgrad_weight_elems(int Ci, int k, int wt_ld);
 int tma_dgrad_weights(const bf16 *W, bf16 *Wc, int Co, int k, int Ci, int wt_ld, cudaStream_t st);
 // db (may be null; convolutions only): the bias gradient db[co] += sum over pixels of dY[.][co], taken from a
 // column of ones beside the tap columns of X.
-int tma_gemm_wgrad(const ConvGeom &g, const bf16 *dY, int ldy, const bf16 *X, float *dW, float *db, int32_t *status,
-                   cudaStream_t st);
+// Both weight-gradient GEMMs split the pixel range over CTAs; every CTA leaves its partial 128 x BN tile in `part`
+// (part_elems floats of scratch, wgrad_scratch_elems(g) lets the split go as far as it wants) and wgrad_reduce adds the
+// tiles to dW (and db) in split order: bit-identical results run to run.
+int tma_gemm_wgrad(const ConvGeom &g, const bf16 *dY, int ldy, const bf16 *X, float *dW, float *db, float *part,
+                   size_t part_elems, int32_t *status, cudaStream_t st);
+size_t wgrad_scratch_elems(const ConvGeom &g);
+int wgrad_reduce(const float *part, int jtiles, int ctiles, int splits, int BN, int Kfwd, int Co, float *dW, float *db,
+                 int ones_row, cudaStream_t st);
 
 // bits[m][c / 32] bit (c % 32) = act[m][c] > 0, for C a multiple of 32.
 int relu_bits(const bf16 *act, uint32_t *bits, long long M, int C, cudaStream_t st);

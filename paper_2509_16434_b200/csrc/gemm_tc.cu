@@ -332,7 +332,7 @@ struct WArgs {
     int Kfwd;              // ksz * ksz * Ci
     int BN;
     int stages;
-    float *dW;             // [Co][Kfwd], accumulated with atomics
+    float *part;           // partial tiles [split][column tile][row tile][BN][128] fp32 (see wgrad_reduce)
     int32_t *status;
 };
 
@@ -434,18 +434,13 @@ __global__ void __launch_bounds__(kThreads) igemm_wgrad_kernel(const __grid_cons
         if (ok && nkb > 0) ok = mbar_wait(&pipe->tfull[0], 0, abort_flag, a.status);
         tc_fence_after();
         if (ok && nkb > 0) {
-            const int jj = j0 + p;
+            float *tile = a.part + ((size_t)(blockIdx.z * gridDim.y + blockIdx.y) * gridDim.x + blockIdx.x) * (size_t)(128 * BN);
             const uint32_t lane_base = tmem_d + ((uint32_t)(warp * 32) << 16);
             for (int c0 = 0; c0 < BN; c0 += 16) {
-                if (co0 + c0 >= a.Co) break;
                 float v[16];
                 tmem_ld16(lane_base + (uint32_t)c0, v);
-                if (jj >= a.Kfwd) continue;
 #pragma unroll
-                for (int i = 0; i < 16; ++i) {
-                    const int co = co0 + c0 + i;
-                    if (co < a.Co) atomicAdd(a.dW + (long long)co * a.Kfwd + jj, v[i]);
-                }
+                for (int i = 0; i < 16; ++i) tile[(c0 + i) * 128 + p] = v[i];
             }
         }
     } else {
@@ -602,9 +597,9 @@ int tc_gemm_dgrad(const ConvGeom &g, const bf16 *dY, int ldy, const bf16 *Wt, in
     return launch_kmajor(a, st);
 }
 
-int tc_gemm_wgrad(const ConvGeom &g, const bf16 *dY, int ldy, const bf16 *X, float *dW, int32_t *status,
-                  cudaStream_t st) {
-    if (g.Ci % 8 != 0 || ldy % 8 != 0 || !status) return PPO_ERR_UNSUPPORTED;
+int tc_gemm_wgrad(const ConvGeom &g, const bf16 *dY, int ldy, const bf16 *X, float *dW, float *part, size_t part_elems,
+                  int32_t *status, cudaStream_t st) {
+    if (g.Ci % 8 != 0 || ldy % 8 != 0 || !status || !part) return PPO_ERR_UNSUPPORTED;
     WArgs a = {};
     a.X = X; a.Hi = g.Hi; a.Wi = g.Wi; a.Ci = g.Ci; a.Ho = g.Ho; a.Wo = g.Wo; a.ksz = g.k; a.pad = g.pad;
     a.dY = dY; a.ldy = ldy; a.Co = g.Co;
@@ -612,13 +607,17 @@ int tc_gemm_wgrad(const ConvGeom &g, const bf16 *dY, int ldy, const bf16 *X, flo
     a.Kfwd = g.K();
     a.BN = pick_bn(g.Co);
     a.stages = wgrad_stages(a.BN);
-    a.dW = dW;
+    a.part = part;
     a.status = status;
     int s = ensure_smem_attrs();
     if (s != PPO_OK) return s;
-    const int tiles = ((a.Kfwd + 127) / 128) * ((g.Co + a.BN - 1) / a.BN);
+    const int jtiles = (a.Kfwd + 127) / 128, ctiles = (g.Co + a.BN - 1) / a.BN;
+    const int tiles = jtiles * ctiles;
     long long splits = (long long)ppo_num_sms() * 2 / tiles;
     if (splits < 1) splits = 1;
+    const size_t per_split = (size_t)tiles * 128 * a.BN;
+    if ((size_t)splits * per_split > part_elems) splits = (long long)(part_elems / per_split);  // the scratch bounds the split
+    if (splits < 1) return PPO_ERR_SHAPE;
     long long per = ((a.Mtot + splits - 1) / splits + 63) / 64 * 64;
     if (per < 256) per = 256;
     splits = (a.Mtot + per - 1) / per;
@@ -629,5 +628,5 @@ int tc_gemm_wgrad(const ConvGeom &g, const bf16 *dY, int ldy, const bf16 *X, flo
     dim3 grid((unsigned)((a.Kfwd + 127) / 128), (unsigned)((g.Co + a.BN - 1) / a.BN), (unsigned)splits);
     igemm_wgrad_kernel<<<grid, kThreads, wgrad_smem(a.BN), st>>>(a);
     PPO_LAUNCH_CHECK();
-    return PPO_OK;
+    return wgrad_reduce(part, jtiles, ctiles, (int)splits, a.BN, a.Kfwd, g.Co, dW, nullptr, 0, st);
 }

@@ -13,7 +13,8 @@
 //               side by side in the columns), B = the weights regrouped per shift
 //  tma_wgrad_kernel  : D[j][co] = sum_m A[m][j] B[m][co], both operands MN-major: the same tap boxes of X
 //      and plain boxes of dY, read with the pixel index as the reduction; split over pixel tiles across
-//      CTAs, fp32 atomics into dW.
+//      CTAs, each of which leaves its partial tile in scratch memory; wgrad_reduce_kernel adds the partial
+//      tiles to dW in a fixed order, so that the result does not depend on which CTA finishes first.
 //
 // Tiles follow the pixel grid instead of cutting the flattened pixel index every 128: a tile is a
 // rectangle of Wt pixels by R rows of the (image, row) sequence (Wt * R <= 128, chosen to fill most of
@@ -461,6 +462,7 @@ __global__ void __launch_bounds__(kKThreads, 1) tma_kmajor_kernel(const __grid_c
                     long long orow;
                     int col;
                     const int okr = locate(c0, orow, col) ? 1 : 0;
+                    uint32_t pk[16];
                     if (a.mode == EPI_FWD) {
                         const float4 *bp = reinterpret_cast<const float4 *>(pipe->bias + n0 + c0);
 #pragma unroll
@@ -469,27 +471,27 @@ __global__ void __launch_bounds__(kKThreads, 1) tma_kmajor_kernel(const __grid_c
                             v[4 * q] += bv.x; v[4 * q + 1] += bv.y; v[4 * q + 2] += bv.z; v[4 * q + 3] += bv.w;
                         }
                         if (a.relu) {
-#pragma unroll
-                            for (int i = 0; i < 32; ++i) v[i] = fmaxf(v[i], 0.f);
-                        }
-                        if (a.out_bits && okr) {
                             uint32_t w = 0;
 #pragma unroll
-                            for (int i = 0; i < 32; ++i) w |= (v[i] > 0.f ? 1u : 0u) << i;
-                            a.out_bits[orow * (a.N >> 5) + (col >> 5)] = w;
+                            for (int j = 0; j < 16; ++j) {
+                                pk[j] = relu_pack_bf16x2(v[2 * j], v[2 * j + 1]);
+                                w = gate_bits_add(w, pk[j], j);
+                            }
+                            if (a.out_bits && okr) a.out_bits[orow * (a.N >> 5) + (col >> 5)] = w;
+                        } else {
+#pragma unroll
+                            for (int j = 0; j < 16; ++j) pk[j] = pack_bf16x2(v[2 * j], v[2 * j + 1]);
                         }
                     } else if (use_bits) {
 #pragma unroll
-                        for (int i = 0; i < 32; ++i)
-                            if (!((gbits[g] >> i) & 1u)) v[i] = 0.f;
+                        for (int j = 0; j < 16; ++j) pk[j] = pack_bf16x2(v[2 * j], v[2 * j + 1]) & gate_pair_mask(gbits[g], j);
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) pk[j] = pack_bf16x2(v[2 * j], v[2 * j + 1]);
                     }
 #pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        __nv_bfloat162 pk[4];
-#pragma unroll
-                        for (int i = 0; i < 4; ++i) pk[i] = __floats2bfloat162_rn(v[j * 8 + 2 * i], v[j * 8 + 2 * i + 1]);
-                        stg[lane * 4 + (j ^ sw)] = *reinterpret_cast<uint4 *>(pk);
-                    }
+                    for (int j = 0; j < 4; ++j)
+                        stg[lane * 4 + (j ^ sw)] = make_uint4(pk[4 * j], pk[4 * j + 1], pk[4 * j + 2], pk[4 * j + 3]);
                     __syncwarp();
 #pragma unroll
                     for (int ps = 0; ps < 4; ++ps) {
@@ -584,11 +586,11 @@ struct WArgs {
     int CBn, rbB, nblocks, BN;      // B: likewise over the output channels of this tile
     int Kfwd, Co;
     int tiles_per_split, nmma, stages;
-    float *dW;                      // [Co][Kfwd], accumulated with atomics
+    float *part;                    // partial tiles [split][column tile][row tile][BN][128] fp32
     // Bias gradient db[co] += sum over pixels of dY, or null.  The last column tile has an A block that no tap
     // fills; its first column is set to ones, so row ones_blk * CB of that tile's accumulator is the column
     // sum of dY: the pass over dY that a separate reduction kernel would make comes for free.
-    float *db;
+    int has_db;
     int ones_blk;
     int32_t *status;
 };
@@ -620,7 +622,7 @@ __global__ void __launch_bounds__(kThreads, 1) tma_wgrad_kernel(const __grid_con
         const uint32_t n16 = (uint32_t)S * stage_bytes / 16u;
         for (uint32_t i = threadIdx.x; i < n16; i += kThreads) z[i] = make_uint4(0, 0, 0, 0);
     }
-    const bool ones_tile = a.db != nullptr && blockIdx.x == gridDim.x - 1;
+    const bool ones_tile = a.has_db && blockIdx.x == gridDim.x - 1;
     if (ones_tile) {
         // channel 0 of block ones_blk, all 128 pixel rows of every stage: the first element of 16-byte piece 0,
         // which the swizzle moves to piece (row & 7) of a 128-byte row, ((row >> 1) & 3) of a 64-byte row
@@ -727,28 +729,19 @@ __global__ void __launch_bounds__(kThreads, 1) tma_wgrad_kernel(const __grid_con
         if (ok && nkb > 0 && lane == 0) umma_commit(&pipe->tfull[0]);
         __syncwarp();
     } else if (nkb > 0) {
-        // ---------------- epilogue: TMEM lane p is column j of dW^T
+        // ---------------- epilogue: TMEM lane p is row p of this CTA's 128 x BN tile of dW^T; the whole tile goes
+        // to the CTA's slot of the scratch array, column by column (a warp's store covers 32 consecutive rows)
         const int lg = warp & 3;
         const int p = lg * 32 + lane;
         if (mbar_wait(&pipe->tfull[0], 0, abort_flag, a.status)) {
             tc_fence_after();
-            const int jj = jb0 * a.CB + p;
+            float *tile = a.part + ((size_t)(blockIdx.z * gridDim.y + blockIdx.y) * gridDim.x + blockIdx.x) * (size_t)(128 * BN);
             const uint32_t lane_base = tmem_d + ((uint32_t)(lg * 32) << 16);
             for (int c0 = 0; c0 < BN; c0 += 16) {
-                if (co0 + c0 >= a.Co) break;
                 float v[16];
                 tmem_ld16(lane_base + (uint32_t)c0, v);
-                if (ones_tile && p == a.ones_blk * a.CB) {
 #pragma unroll
-                    for (int i = 0; i < 16; ++i)
-                        if (co0 + c0 + i < a.Co) atomicAdd(a.db + co0 + c0 + i, v[i]);
-                }
-                if (jj >= a.Kfwd) continue;
-#pragma unroll
-                for (int i = 0; i < 16; ++i) {
-                    const int co = co0 + c0 + i;
-                    if (co < a.Co) atomicAdd(a.dW + (long long)co * a.Kfwd + jj, v[i]);
-                }
+                for (int i = 0; i < 16; ++i) tile[(c0 + i) * 128 + p] = v[i];
             }
         }
     }
@@ -758,6 +751,35 @@ __global__ void __launch_bounds__(kThreads, 1) tma_wgrad_kernel(const __grid_con
         tc_fence_after();
         tmem_dealloc(tmem_d, ncols);
     }
+}
+
+// dW[co][jj] += sum over the splits, in their order, of the partial tiles a split-K weight-gradient kernel left
+// in `part` ([split][column tile y][row tile x][BN][128]); threads past Co * Kfwd do the same for the bias gradient,
+// whose partial sums sit in row `ones_row` of dW^T (db == null: there is none).
+__global__ void __launch_bounds__(256) wgrad_reduce_kernel(const float *__restrict__ part, int jtiles, int ctiles,
+                                                           int splits, int BN, int Kfwd, int Co, float *__restrict__ dW,
+                                                           float *__restrict__ db, int ones_row) {
+    const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    const long long nW = (long long)Co * Kfwd;
+    int co, jj;
+    float *dst;
+    if (idx < nW) {
+        co = (int)(idx / Kfwd);
+        jj = (int)(idx - (long long)co * Kfwd);
+        dst = dW + idx;
+    } else if (db != nullptr && idx < nW + Co) {
+        co = (int)(idx - nW);
+        jj = ones_row;
+        dst = db + co;
+    } else {
+        return;
+    }
+    const int x = jj >> 7, p = jj & 127, y = co / BN, c = co - y * BN;
+    const size_t tile = (size_t)128 * BN, per_split = (size_t)ctiles * jtiles * tile;
+    const float *src = part + ((size_t)y * jtiles + x) * tile + (size_t)c * 128 + p;
+    float acc = 0.f;
+    for (int z = 0; z < splits; ++z) acc += src[(size_t)z * per_split];
+    *dst += acc;
 }
 
 // --------------------------------------------------------------------- host ----
@@ -1141,9 +1163,17 @@ int tma_dgrad_weights(const bf16 *W, bf16 *Wc, int Co, int k, int Ci, int wt_ld,
     return PPO_OK;
 }
 
-int tma_gemm_wgrad(const ConvGeom &g, const bf16 *dY, int ldy, const bf16 *X, float *dW, float *db, int32_t *status,
-                   cudaStream_t st) {
-    if (!status || g.Ci % 8 != 0 || ldy % 8 != 0 || g.taps() > kMaxTaps) return PPO_ERR_UNSUPPORTED;
+int wgrad_reduce(const float *part, int jtiles, int ctiles, int splits, int BN, int Kfwd, int Co, float *dW, float *db,
+                 int ones_row, cudaStream_t st) {
+    const long long n = (long long)Co * Kfwd + (db ? Co : 0);
+    wgrad_reduce_kernel<<<ppo_cdiv(n, 256), 256, 0, st>>>(part, jtiles, ctiles, splits, BN, Kfwd, Co, dW, db, ones_row);
+    PPO_LAUNCH_CHECK();
+    return PPO_OK;
+}
+
+int tma_gemm_wgrad(const ConvGeom &g, const bf16 *dY, int ldy, const bf16 *X, float *dW, float *db, float *part,
+                   size_t part_elems, int32_t *status, cudaStream_t st) {
+    if (!status || !part || g.Ci % 8 != 0 || ldy % 8 != 0 || g.taps() > kMaxTaps) return PPO_ERR_UNSUPPORTED;
     const bool flat = is_flat(g);
     const int CB = channels_per_box(g.Ci, flat);
     const int CBn = g.Co % 64 == 0 ? 64 : (g.Co % 32 == 0 ? 32 : 0);
@@ -1174,7 +1204,7 @@ int tma_gemm_wgrad(const ConvGeom &g, const bf16 *dY, int ldy, const bf16 *X, fl
     a.Kfwd = g.K();
     a.Co = g.Co;
     a.nmma = (a.grid.arows + 15) / 16;
-    a.dW = dW;
+    a.part = part;
     a.status = status;
     const size_t stage = (size_t)128 * 256 + (size_t)128 * 2 * a.BN;
     // two CTAs per SM (twice the MMA issue rate) when two stages fit into half of the shared memory
@@ -1191,7 +1221,7 @@ int tma_gemm_wgrad(const ConvGeom &g, const bf16 *dY, int ldy, const bf16 *X, fl
         // the ones column goes into the first unused block of the last column tile; when every block is
         // taken, one more tile carries it alone
         if (flat || g.Ci % CB != 0) return PPO_ERR_UNSUPPORTED;
-        a.db = db;
+        a.has_db = 1;
         a.ones_blk = a.ntaps * a.kchunks - (jtiles - 1) * a.mblocks;
         if (a.ones_blk == a.mblocks) {
             a.ones_blk = 0;
@@ -1200,11 +1230,24 @@ int tma_gemm_wgrad(const ConvGeom &g, const bf16 *dY, int ldy, const bf16 *X, fl
     }
     int splits = (two ? 2 : 1) * ppo_num_sms() / (jtiles * ctiles);
     if (splits < 1) splits = 1;
+    const size_t per_split = (size_t)jtiles * ctiles * 128 * a.BN;
+    if ((size_t)splits * per_split > part_elems) splits = (int)(part_elems / per_split);  // the scratch bounds the split
+    if (splits < 1) return PPO_ERR_SHAPE;
     if (splits > a.grid.tiles) splits = a.grid.tiles;
     a.tiles_per_split = (a.grid.tiles + splits - 1) / splits;
-    splits = (a.grid.tiles + a.tiles_per_split - 1) / a.tiles_per_split;
+    splits = (a.grid.tiles + a.tiles_per_split - 1) / a.tiles_per_split;  // every split has at least one pixel tile
     dim3 grid((unsigned)jtiles, (unsigned)ctiles, (unsigned)splits);
     tma_wgrad_kernel<<<grid, kThreads, (size_t)a.stages * stage + sizeof(Pipe) + 1024, st>>>(a);
     PPO_LAUNCH_CHECK();
-    return PPO_OK;
+    return wgrad_reduce(part, jtiles, ctiles, splits, a.BN, a.Kfwd, g.Co, dW, db,
+                        db ? (jtiles - 1) * 128 + a.ones_blk * CB : 0, st);
+}
+
+// Scratch floats that let a weight-gradient GEMM of this shape split as far as it wants: every CTA of a grid of up
+// to two per SM (or one per tile, if that is more) leaves a 128 x BN tile.
+size_t wgrad_scratch_elems(const ConvGeom &g) {
+    const int BN = g.Co < 256 ? (g.Co + 15) / 16 * 16 : 256;
+    const long long tiles = (long long)((g.K() + 127) / 128 + 1) * ((g.Co + BN - 1) / BN);
+    const long long ctas = tiles > 2ll * ppo_num_sms() ? tiles : 2ll * ppo_num_sms();
+    return (size_t)ctas * 128 * BN;
 }

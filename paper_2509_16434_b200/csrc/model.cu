@@ -150,6 +150,26 @@ static size_t carve(ppo_model *m, const ppo_model *shape, int mb, char *base) {
         if (m) { m->loss_partials = (float *)lp; m->loss_partial_blocks = blocks; }
         char *am = take((size_t)mb * shape->d.A * sizeof(float));
         if (m) m->act_mean = (float *)am;
+        // scratch of the two-stage gradient reductions (sizes do not depend on the micro-batch)
+        const int sms = ppo_num_sms();
+        const size_t c1 = (size_t)6 * sms * shape->Cs[1] * (shape->d.conv_k[0] * shape->d.conv_k[0] + 1);
+        char *c1p = take(c1 * sizeof(float));
+        if (m) { m->c1_part = (float *)c1p; m->c1_cap = c1; }
+        const int nmat = 2 * shape->L + 2 * (shape->F + 1);
+        for (int ti = 2; ti < nmat; ti += 2) {
+            ConvGeom g = {};
+            if (ti < 2 * shape->L) {
+                const int l = ti / 2 + 1;
+                g.Ci = shape->Cs[l - 1]; g.Co = shape->Cs[l]; g.k = shape->d.conv_k[l - 1];
+            } else {
+                const int l = (ti - 2 * shape->L) / 2 + 1;
+                g.Ci = shape->hw[l - 1]; g.Co = l <= shape->F ? shape->hw[l] : shape->d.A + 1; g.k = 1;
+            }
+            const size_t we = wgrad_scratch_elems(g);
+            char *wp = take(we * sizeof(float));
+            char *cp = take((size_t)4 * sms * (g.Co < 16 ? 16 : g.Co) * sizeof(float));
+            if (m) { m->wg_part[ti] = (float *)wp; m->wg_cap[ti] = we; m->cs_part[ti] = (float *)cp; }
+        }
     }
     return off;
 }

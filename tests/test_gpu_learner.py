@@ -14,12 +14,16 @@ DEV = "cuda"
 ENC_TOL = 2e-2    # relative L2: bf16 operands / activations with fp32 accumulation vs fp64
 LOSS_TOL = 1e-3   # relative error of the loss scalars
 ADAM_TOL = 1e-3   # relative L2 of the parameters after one step
-# End-to-end gradients (GPU forward feeding GPU backward) against the oracle's own forward+backward are held to the
-# same 2e-2, in total and per tensor, at these sizes (measured: at most 6e-3).  What separates the two sides beyond
-# the arithmetic is the handful of ReLU gates (measured: fewer than 1 in 10^6) that the two forwards decide
-# differently; test_gpu_parity_wide.py counts them and holds the backward operator to 2e-2 on identical activations.
-E2E_GRAD_TOL_TOTAL = 2e-2
-E2E_GRAD_TOL_TENSOR = 2e-2
+# End-to-end gradients (GPU forward feeding GPU backward) against the oracle's own forward+backward.  What separates
+# the two sides beyond the arithmetic is the handful of ReLU gates (measured: 0 to 2 in 10^6 of the stored
+# activations) that the two forwards decide differently: a flipped gate of a deep layer removes or adds that unit's
+# whole contribution, and in a minibatch of a few rows one such unit is a visible share of a tensor's gradient
+# (measured: 5.3e-2 of the whole gradient with 4 flipped gates in 4 rows of the cfg4 network, 7e-2 on one tensor in
+# 8 rows of cfg2's, 6e-3 of the whole gradient at 1024 rows).  These bounds therefore only catch gross errors;
+# test_gpu_parity_wide.py counts the flipped gates and holds the backward pass to 2e-2 per tensor against the
+# oracle's backward from the very activations the GPU saved, and on the oracle's activations at up to 1024 rows.
+E2E_GRAD_TOL_TOTAL = 1e-1
+E2E_GRAD_TOL_TENSOR = 2e-1
 SIGN_AGREEMENT = 0.97  # fraction of clearly moved parameters whose Adam update has the oracle's sign
 
 
@@ -151,14 +155,23 @@ def test_minibatch_forward_loss_backward_match_oracle(name, microbatch):
     assert rel_l2(V, V_o) <= ENC_TOL, rel_l2(V, V_o)
     out = L.loss.cpu().numpy()
     assert 0.0 < out_o[4] < 1.0, "both clip branches must be exercised"
-    # value loss and entropy to 1e-3 relative; the policy loss and the KL estimate are means of signed terms near
-    # zero, so their errors are measured against the mean magnitude of their terms (|s| ~ |adv|, |log ratio|)
-    assert abs(out[1] - out_o[1]) <= LOSS_TOL * abs(out_o[1])
+    # Entropy (exact arithmetic on log-sigma) to 1e-3 relative.  The value loss is a mean of squared differences V - R
+    # and the policy loss and the KL estimate are means of signed terms near zero, so their errors are measured
+    # against the mean magnitude of what enters them (V^2 + R^2, |s| ~ |adv|, |log ratio|).  They inherit the encoder's
+    # error in mu and V (2e-3 here, inside its 2e-2): over 8 rows and more it averages below 1e-3
+    # (test_gpu_parity_wide.py holds that), in a minibatch of 2 to 16 rows it shows almost undiminished, so the
+    # bound here is 5e-3 (measured: up to 2e-3).
+    small = 5 * LOSS_TOL
+    assert abs(out[1] - out_o[1]) <= small * max(abs(out_o[1]), float(np.mean(V_o ** 2 + f["ret"] ** 2)))
     assert abs(out[2] - out_o[2]) <= LOSS_TOL * abs(out_o[2])
-    assert abs(out[0] - out_o[0]) <= LOSS_TOL * float(np.mean(np.abs(f["adv"])))
-    assert abs(out[3] - out_o[3]) <= LOSS_TOL * max(1.0, abs(out_o[3]))
+    assert abs(out[0] - out_o[0]) <= small * float(np.mean(np.abs(f["adv"])))
+    assert abs(out[3] - out_o[3]) <= small * max(1.0, abs(out_o[3]))
     assert abs(out[4] - out_o[4]) <= 2.0 / B + 1e-6
-    _check_grads(lay, L.model.grad.cpu().numpy(), grad_o, E2E_GRAD_TOL_TENSOR, E2E_GRAD_TOL_TOTAL)
+    got = L.model.grad.cpu().numpy()
+    errs = [rel_l2(got[o:o + s], grad_o[o:o + s]) for o, s in zip(lay.offsets, lay.sizes)]
+    print(f"[{name}-{microbatch}] end-to-end gradients: max per tensor {max(errs):.3e} (tensor {int(np.argmax(errs))}), "
+          f"total {rel_l2(got, grad_o):.3e}")
+    _check_grads(lay, got, grad_o, E2E_GRAD_TOL_TENSOR, E2E_GRAD_TOL_TOTAL)
 
 
 def test_loss_kernel_alone_matches_oracle_to_1e3():
@@ -342,7 +355,8 @@ def test_forward_writes_the_relu_gate_bits_of_its_activations():
         n = B * h * w_ * c
         act = L.model.activation(0, l)[:n].float().cpu().numpy().reshape(-1, 32)
         want = (act > 0).astype(np.uint64)
-        want_words = (want << np.arange(32, dtype=np.uint64)).sum(1).astype(np.uint32)
+        pos = np.array([(c >> 1) + 16 * (c & 1) for c in range(32)], dtype=np.uint64)  # bit of channel c in its word
+        want_words = (want << pos).sum(1).astype(np.uint32)
         got = L.model.activation(2, l)[:n // 32].cpu().numpy().view(np.uint32)
         assert np.array_equal(got, want_words), f"layer {l}: forward-written gates"
         L.model.activation(2, l)[:n // 32].zero_()
@@ -389,5 +403,33 @@ def test_backward_on_a_caller_stream_orders_like_one_stream():
     assert ppo.ppo_poll_status() == 0
     r = ref.cpu().numpy()
     assert np.abs(r).max() > 0
-    for g in got:  # wgrad adds fp32 partial sums with atomics: equal up to their order
-        assert rel_l2(g.cpu().numpy(), r) <= 1e-5
+    for g in got:  # every reduction adds its partial sums in a fixed order: the same bits on any stream
+        assert np.array_equal(g.cpu().numpy(), r)
+
+
+def test_gradients_are_bit_identical_run_to_run():
+    """Every reduction over rows, pixels or splits (weight gradients of all layers, bias gradients, the loss terms)
+    adds its partial results in a fixed order: the same minibatch processed twice gives the same bits, also when it
+    is accumulated over micro-batches."""
+    w = SHAPES["cfg2_twin"]
+    L, md, lay, theta, roll, action, logp, dev = _setup(w, 3)
+    h = L.hyper
+    K = w.minibatches
+    B = w.M // K
+    L.compute_gae(dev["last_value"])
+    ppo.ppo_shuffle_gather_minibatch(L.buffer, 5, 0, 0, K, L.mb)
+    runs = []
+    for _ in range(3):
+        ppo.ppo_model_zero_grad(L.model)
+        L.loss.zero_()
+        for r0 in range(0, B, L.microbatch):
+            rows = min(L.microbatch, B - r0)
+            ppo.ppo_encoder_fwd(L.model, L.mb, r0, rows, L.mean, L.value)
+            ppo.ppo_loss_fwd_bwd(L.model, L.mb, r0, rows, B, L.mean, L.value, h.clip, h.vf_coef, h.ent_coef, L.loss,
+                                 L.dmean, L.dvalue)
+            ppo.ppo_encoder_bwd(L.model, L.mb, r0, rows, L.dmean, L.dvalue, True)
+        runs.append((L.model.grad.clone(), L.loss.clone()))
+    assert ppo.ppo_poll_status() == 0
+    assert float(runs[0][0].abs().max()) > 0
+    for g, l in runs[1:]:
+        assert torch.equal(g, runs[0][0]) and torch.equal(l, runs[0][1])
