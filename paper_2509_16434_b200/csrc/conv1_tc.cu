@@ -154,31 +154,37 @@ __global__ void __launch_bounds__(kThreads, 1) conv1_tc_kernel(const __grid_cons
             }
             int s = 0;
             uint32_t ph = 0;
-            for (int li = 0; li < ns && ok; ++li, m += step) {
-                ok = mbar_wait(&pipe->empty[s], ph ^ 1u, abort_flag, a.status);
-                if (!ok) break;
-                uint32_t wv[KP / 2];
+            uint32_t wv[KP / 2];
+            // Window of this thread's current pixel into wv.  Every load is issued (from a clamped address where its
+            // pixel pair lies outside the frame) and the pairs outside are zeroed afterwards: no branch separates
+            // the loads of a window.
+            auto load_window = [&]() {
 #pragma unroll
                 for (int k = 0; k < KP / 2; ++k) wv[k] = 0u;
-                wv[KW] = 0x3C003C00u;  // (1.0, 1.0): the bias slots
-                if (m < a.M) {
-                    const uint32_t *img = reinterpret_cast<const uint32_t *>(a.depth) + (long long)ib * a.Hi * Wh;
-                    const int pw0 = ow - (P + ODD) / 2;  // first pair of the window row, in words
+                const bool live = m < a.M;
+                const uint32_t *img = reinterpret_cast<const uint32_t *>(a.depth) + (long long)(live ? ib : 0) * a.Hi * Wh;
+                const int pw0 = ow - (P + ODD) / 2;  // first pair of the window row, in words
 #pragma unroll
-                    for (int kh = 0; kh < KS; ++kh) {
-                        const int ih = 2 * oh + kh - P;
-                        if (ih >= 0 && ih < a.Hi) {
-                            const uint32_t *row = img + ih * Wh;
+                for (int kh = 0; kh < KS; ++kh) {
+                    const int ih = 2 * oh + kh - P;
+                    const bool rok = live && (unsigned)ih < (unsigned)a.Hi;
+                    const uint32_t *row = img + (rok ? ih : 0) * Wh;
 #pragma unroll
-                            for (int qq = 0; qq < NP; ++qq) {
-                                const int pw = pw0 + qq;
-                                if (pw >= 0 && pw < Wh) wv[kh * NP + qq] = __ldg(row + pw);
-                            }
-                        }
+                    for (int qq = 0; qq < NP; ++qq) {
+                        const int pw = pw0 + qq;
+                        const bool pok = rok && (unsigned)pw < (unsigned)Wh;
+                        const uint32_t v = __ldg(row + (pok ? pw : 0));
+                        wv[kh * NP + qq] = pok ? v : 0u;
                     }
-                } else {
-                    wv[KW] = 0u;  // rows past the last pixel stay zero
                 }
+                wv[KW] = live ? 0x3C003C00u : 0u;  // (1.0, 1.0): the bias slots; rows past the last pixel stay zero
+            };
+            if (ns > 0) load_window();
+            // the window of the next stage is fetched before this stage's slot is waited for, so that the loads'
+            // latency overlaps the wait
+            for (int li = 0; li < ns && ok; ++li) {
+                ok = mbar_wait(&pipe->empty[s], ph ^ 1u, abort_flag, a.status);
+                if (!ok) break;
                 uint8_t *dst = smem + (size_t)s * stage_bytes + (size_t)grp * kTileBytes;
 #pragma unroll
                 for (int c = 0; c < KP / 8; ++c)
@@ -186,11 +192,13 @@ __global__ void __launch_bounds__(kThreads, 1) conv1_tc_kernel(const __grid_cons
                         make_uint4(wv[4 * c], wv[4 * c + 1], wv[4 * c + 2], wv[4 * c + 3]);
                 fence_async_smem();
                 mbar_arrive(&pipe->full[s]);
+                m += step;
                 ow += d_ow;
                 if (ow >= a.Wo) { ow -= a.Wo; ++oh; }
                 oh += d_oh;
                 if (oh >= a.Ho) { oh -= a.Ho; ++ib; }
                 ib += d_b;
+                if (li + 1 < ns) load_window();
                 if (++s == S) { s = 0; ph ^= 1u; }
             }
         }

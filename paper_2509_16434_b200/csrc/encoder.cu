@@ -267,30 +267,33 @@ __global__ void __launch_bounds__(256) conv1_wgrad_mma_kernel(const __half *__re
     const int Wh = Wi >> 1;  // 32-bit words per frame row
     auto prefetch = [&](long long mt) {
         const bool live = mt + lane < m_end;
-        const uint32_t *img = reinterpret_cast<const uint32_t *>(depth) + b * Hi * Wh;
-        uint32_t wv[TP / 2];
+        // every load is issued, from a clamped address where its pixel pair lies outside the frame, before the first
+        // conversion: the loads of a trip are then in flight together
+        const uint32_t *img = reinterpret_cast<const uint32_t *>(depth) + (live ? b : 0) * Hi * Wh;
+        uint32_t wv[TP / 2], raw[KW];
+        const int pw0 = ow - (P + ODD) / 2;
+        uint32_t okm = 0;
 #pragma unroll
-        for (int k = 0; k < TP / 2; ++k) wv[k] = 0u;
-        if (live) {
-            wv[KW] = 0x00003F80u;  // (1.0, 0) as bf16: the bias-gradient column
-            const int pw0 = ow - (P + ODD) / 2;
+        for (int kh = 0; kh < KS; ++kh) {
+            const int ih = 2 * oh + kh - P;
+            const bool rok = live && (unsigned)ih < (unsigned)Hi;
+            const uint32_t *row = img + (rok ? ih : 0) * Wh;
 #pragma unroll
-            for (int kh = 0; kh < KS; ++kh) {
-                const int ih = 2 * oh + kh - P;
-                if (ih >= 0 && ih < Hi) {
-                    const uint32_t *row = img + ih * Wh;
-#pragma unroll
-                    for (int q = 0; q < NP; ++q) {
-                        const int pw = pw0 + q;
-                        if (pw >= 0 && pw < Wh) {
-                            const uint32_t raw = __ldg(row + pw);
-                            const float2 f = __half22float2(*reinterpret_cast<const __half2 *>(&raw));
-                            wv[kh * NP + q] = pack_bf16x2(f.x, f.y);
-                        }
-                    }
-                }
+            for (int q = 0; q < NP; ++q) {
+                const int pw = pw0 + q;
+                const bool ok = rok && (unsigned)pw < (unsigned)Wh;
+                raw[kh * NP + q] = __ldg(row + (ok ? pw : 0));
+                okm |= (ok ? 1u : 0u) << (kh * NP + q);
             }
         }
+#pragma unroll
+        for (int k = 0; k < TP / 2; ++k) wv[k] = 0u;
+#pragma unroll
+        for (int k = 0; k < KW; ++k) {
+            const float2 f = __half22float2(*reinterpret_cast<const __half2 *>(&raw[k]));
+            wv[k] = (okm >> k) & 1u ? pack_bf16x2(f.x, f.y) : 0u;
+        }
+        if (live) wv[KW] = 0x00003F80u;  // (1.0, 0) as bf16: the bias-gradient column
 #pragma unroll
         for (int c = 0; c < TP / 8; ++c) xreg[c] = make_uint4(wv[4 * c], wv[4 * c + 1], wv[4 * c + 2], wv[4 * c + 3]);
 #pragma unroll
@@ -481,17 +484,28 @@ __global__ void __launch_bounds__(256) pack_dout_kernel(const float *__restrict_
 // reductions whose blocks leave partial sums instead of adding to the result with atomics (reproducible results).
 __global__ void __launch_bounds__(256) sum_partials_kernel(const float *__restrict__ part, int nparts, int nA,
                                                            float *__restrict__ dstA, int nB, float *__restrict__ dstB) {
-    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    // 32 results per block; eight threads share a result, thread j adding the partials b = j, j + 8, ... in order, and
+    // the eight sums are added in the order of j: fixed, whatever the launch.
+    __shared__ float sh[8][32];
+    const int o = threadIdx.x & 31, j = threadIdx.x >> 5;
+    const int i = blockIdx.x * 32 + o;
     const int n = nA + nB;
-    if (i >= n) return;
     float acc = 0.f;
-    for (int b = 0; b < nparts; ++b) acc += part[(size_t)b * n + i];
-    if (i < nA) dstA[i] += acc;
-    else dstB[i - nA] += acc;
+    if (i < n)
+        for (int b = j; b < nparts; b += 8) acc += part[(size_t)b * n + i];
+    sh[j][o] = acc;
+    __syncthreads();
+    if (j == 0 && i < n) {
+        float v = sh[0][o];
+#pragma unroll
+        for (int q = 1; q < 8; ++q) v += sh[q][o];
+        if (i < nA) dstA[i] += v;
+        else dstB[i - nA] += v;
+    }
 }
 
 static int sum_partials(const float *part, int nparts, int nA, float *dstA, int nB, float *dstB, cudaStream_t st) {
-    sum_partials_kernel<<<ppo_cdiv(nA + nB, 256), 256, 0, st>>>(part, nparts, nA, dstA, nB, dstB);
+    sum_partials_kernel<<<ppo_cdiv(nA + nB, 32), 256, 0, st>>>(part, nparts, nA, dstA, nB, dstB);
     PPO_LAUNCH_CHECK();
     return PPO_OK;
 }
