@@ -66,6 +66,9 @@ def fwd_flops_per_sample(w, skip_conv1=False):
             continue
         f += 2 * cs[l + 1] * hs[l + 1] * ws[l + 1] * cs[l] * k * k
     i = cs[-1] + w.P
+    if getattr(w, "embed", 0):
+        f += 2 * hs[-1] * ws[-1] * cs[-1] * w.embed
+        i = w.embed + w.P
     for o in list(w.fc) + [w.A + 1]:
         f += 2 * i * o
         i = o
@@ -137,17 +140,8 @@ def make_learner(w, microbatch, device):
     from paper_2509_16434_b200.learner import Learner
     L = Learner(w, microbatch, device)
     offs = L.model.tensors()
-    shapes = []
-    cin = 1
-    for c, k in zip(w.conv_c, w.conv_k):
-        shapes += [(c, k, k, cin), (c,)]
-        cin = c
-    i = cin + w.P
-    for o in w.fc:
-        shapes += [(o, i), (o,)]
-        i = o
-    shapes += [(w.A + 1, i), (w.A + 1,), (w.A,)]
-    theta = synth.init_params(L.model.arena, [o for o, _ in offs], shapes, w.seed)
+    shapes, gammas = synth.param_shapes(w)
+    theta = synth.init_params(L.model.arena, [o for o, _ in offs], shapes, w.seed, ones=gammas)
     L.model.load(theta)
     roll = synth.rollout_torch(w, device, w.seed)
     action = torch.empty((w.T, w.N, w.A), dtype=torch.float32, device=device)
@@ -473,7 +467,7 @@ def oracle_sample_step(w, fields, theta, n_samples):
     """The oracle's learner step on a bounded sample: GAE + normalisation at full size, then one minibatch of
     n_samples rows (permutation, gather, forward, loss, backward, Adam).  Returns seconds and samples trained."""
     from oracle import oracle as orc
-    md = orc.ModelDesc(w.H, w.W, tuple(w.conv_c), tuple(w.conv_k), tuple(w.fc), w.P, w.A)
+    md = orc.ModelDesc(w.H, w.W, tuple(w.conv_c), tuple(w.conv_k), tuple(w.fc), w.P, w.A, norm=w.norm, embed=w.embed)
     t0 = time.perf_counter()
     adv, ret = orc.gae(fields["reward"], fields["value"], fields["done"], fields["last_value"], w.gamma, w.lam)
     adv, _, _ = orc.adv_normalize(adv)
@@ -528,9 +522,9 @@ def run_reference(args):
     g = np.random.Generator(np.random.Philox(key=[w.seed, 1234]))
     depth = g.uniform(0.1, 2.0, (n_samples, w.H, w.W)).astype(np.float16)
     depth[g.random(depth.shape) < 0.1] = 0
-    md = orc.ModelDesc(w.H, w.W, tuple(w.conv_c), tuple(w.conv_k), tuple(w.fc), w.P, w.A)
+    md = orc.ModelDesc(w.H, w.W, tuple(w.conv_c), tuple(w.conv_k), tuple(w.fc), w.P, w.A, norm=w.norm, embed=w.embed)
     lay = orc.param_layout(md)
-    theta = synth.init_params(lay.total, lay.offsets, lay.shapes, w.seed)
+    theta = synth.init_params(lay.total, lay.offsets, lay.shapes, w.seed, ones=synth.param_shapes(w)[1])
     fields = {k: roll[k] for k in ("proprio", "value", "reward", "done", "last_value")}
     fields["action"] = roll["eps"]
     fields["logp"] = (-0.5 * (roll["eps"].astype(np.float64) ** 2).sum(-1) - 0.5 * w.A * np.log(2 * np.pi)

@@ -174,12 +174,24 @@ int ppo_shuffle_gather_minibatch(const ppo_buffer *buf, uint64_t seed, uint32_t 
 
 #define PPO_MAX_CONV 8
 #define PPO_MAX_FC 4
+#define PPO_MAX_TENSORS (4 * PPO_MAX_CONV + 2 * PPO_MAX_FC + 5)
 
 /* Policy/value network (Section III-C: CNN with ReLU on the depth image, joined with
  * proprioception, fully connected layers).  Conv l: k x k cross-correlation, stride 2,
  * zero padding k/2, ReLU; global average pool; concat [pooled, proprio]; hidden FC layers
  * with ReLU; one linear head giving the Gaussian mean (A) and the value (1); log-sigma is a
- * free A-vector.  Channel counts of conv layers >= 1 and FC widths must be multiples of 8. */
+ * free A-vector.  Channel counts of conv layers >= 1 and FC widths must be multiples of 8.
+ *
+ * The depth CNN as Section III-C words it ("4-layer CNN ... layer normalization, and ReLU", "a fully connected
+ * layer which outputs a 32 dimensional embedding for the depth") is selected by the last two fields, both 0 for
+ * the plain network above:
+ *   norm != 0 : every conv output is layer-normalised over its channels at each pixel before the ReLU,
+ *               y = ReLU(gamma * (z - mean) / sqrt(var + 1e-5) + beta), mean and (biased) variance over the C
+ *               channels of the pixel, gamma and beta learned per channel.  Needs conv_c[0] in {16, 32}, every
+ *               conv_c <= 256 and an even frame width.
+ *   embed > 0 : instead of the global average pool, the last conv output is flattened (pixel-major, channel
+ *               innermost) and mapped by a fully connected layer with ReLU to `embed` values (a multiple of 32,
+ *               embed + P a multiple of 8), which are concatenated with proprio. */
 typedef struct {
     int32_t H, W;
     int32_t n_conv;
@@ -188,6 +200,7 @@ typedef struct {
     int32_t n_fc;
     int32_t fc[PPO_MAX_FC];
     int32_t P, A;
+    int32_t norm, embed;
 } ppo_model_desc;
 
 typedef struct ppo_model ppo_model;
@@ -196,7 +209,8 @@ int ppo_model_create(const ppo_model_desc *desc, ppo_model **out);
 int ppo_model_destroy(ppo_model *m);
 
 /* Parameter vector ("arena") layout: tensors in the order conv W_l [Cout][k][k][Cin],
- * conv b_l [Cout], ..., fc W [out][in], fc b [out], ..., head W [A+1][hid] (rows 0..A-1
+ * conv b_l [Cout] (with norm: followed by gamma_l [Cout], beta_l [Cout]), ..., (with embed: embed W
+ * [E][Ho*Wo*C_L], embed b [E],) fc W [out][in], fc b [out], ..., head W [A+1][hid] (rows 0..A-1
  * mean, row A value), head b [A+1], log-sigma [A]; every tensor starts at a multiple of 64
  * elements; gaps are zero and stay zero.  The same offsets index master, shadow, gradient
  * and Adam moment arrays. */
@@ -254,7 +268,8 @@ int ppo_encoder_bwd(ppo_model *m, const ppo_minibatch *mb, int row0, int rows, c
  * conv activation of layer `index` in 1..n_conv, NHWC bf16 [rows][Ho][Wo][C]; kind 1 = h_index
  * for index in 0..n_fc, bf16 [rows][width] (h_0 = [pooled, proprio]); kind 2 = the ReLU gate bits of conv
  * activation `index` (only for layers below the last whose channel count is a multiple of 32, else INVALID_ARG),
- * uint32 [rows][Ho][Wo][C/32]; channel c belongs to word c / 32 and sits at bit ((c % 32) / 2) + 16 * (c % 2) of it (the
+ * uint32 [rows][Ho][Wo][C/32] (kind 3 and 4, with norm only: the normalised values xhat of conv layer `index`,
+ * bf16 [rows][Ho][Wo][C], and their reciprocal standard deviations, fp32 [rows][Ho][Wo]); channel c belongs to word c / 32 and sits at bit ((c % 32) / 2) + 16 * (c % 2) of it (the
  * two halves of a packed pair of bf16 values own bits j and 16 + j), set where the activation is > 0.  *elems is the capacity
  * for the bound micro-batch.  For inspection and for tests that substitute the saved
  * activations between ppo_encoder_fwd and ppo_encoder_bwd. */

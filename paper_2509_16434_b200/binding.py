@@ -45,7 +45,7 @@ class BufferDesc(C.Structure):
 class ModelDesc(C.Structure):
     _fields_ = [("H", C.c_int32), ("W", C.c_int32), ("n_conv", C.c_int32), ("conv_c", C.c_int32 * 8),
                 ("conv_k", C.c_int32 * 8), ("n_fc", C.c_int32), ("fc", C.c_int32 * 4), ("P", C.c_int32),
-                ("A", C.c_int32)]
+                ("A", C.c_int32), ("norm", C.c_int32), ("embed", C.c_int32)]
 
 
 class Minibatch(C.Structure):
@@ -261,9 +261,11 @@ def ppo_shuffle_gather_minibatch(buf: Buffer, seed: int, epoch: int, mb_index: i
                                               _stream(stream)), "ppo_shuffle_gather_minibatch")
 
 
-def model_desc(H, W, conv_c: Sequence[int], conv_k: Sequence[int], fc: Sequence[int], P=32, A=12) -> ModelDesc:
+def model_desc(H, W, conv_c: Sequence[int], conv_k: Sequence[int], fc: Sequence[int], P=32, A=12, norm=False,
+               embed=0) -> ModelDesc:
     d = ModelDesc()
     d.H, d.W, d.n_conv, d.n_fc, d.P, d.A = H, W, len(conv_c), len(fc), P, A
+    d.norm, d.embed = int(norm), int(embed)
     for i, v in enumerate(conv_c):
         d.conv_c[i] = v
     for i, v in enumerate(conv_k):
@@ -324,6 +326,8 @@ class Model:
         off = p.value - self.workspace.data_ptr()
         if kind == 2:
             return self.workspace[off:off + 4 * n.value].view(torch.int32)
+        if kind == 4:
+            return self.workspace[off:off + 4 * n.value].view(torch.float32)
         return self.workspace[off:off + 2 * n.value].view(torch.bfloat16)
 
     def load(self, theta, stream=None):

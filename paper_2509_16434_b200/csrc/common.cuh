@@ -62,6 +62,9 @@ struct ppo_model {
     int Hs[PPO_MAX_CONV + 1], Ws[PPO_MAX_CONV + 1], Cs[PPO_MAX_CONV + 1];  // index 0 = input image
     int hw[PPO_MAX_FC + 1];                                                // widths of h_0..h_F
     std::vector<ppo_tensor> tensors;
+    // tensor index of the weight matrix of conv layer l (1..L; bias at +1, with norm gamma at +2 and beta at +3),
+    // of the embedding (-1 without one) and of FC layer l (1..F; F + 1 is the head); log-sigma is the last tensor
+    int ti_conv[PPO_MAX_CONV + 1], ti_embed, ti_fc[PPO_MAX_FC + 2];
     size_t arena, nparams;
     // bound arrays
     float *master, *grad, *adam_m, *adam_v;
@@ -73,19 +76,24 @@ struct ppo_model {
     bf16 *act[PPO_MAX_CONV + 1];   // act[l], l >= 1: [mb][Ho][Wo][C] post-ReLU
     bf16 *dact[PPO_MAX_CONV + 1];  // gradient w.r.t. the pre-activation of act[l]
     uint32_t *abits[PPO_MAX_CONV + 1];  // ReLU gate of act[l], one bit per element (layers with C % 32 == 0, else null)
+    bf16 *xhat[PPO_MAX_CONV + 1];   // with norm: normalised values of conv layer l, [mb][Ho][Wo][C]
+    float *rstd[PPO_MAX_CONV + 1];  // with norm: 1 / sqrt(var + eps) per pixel, [mb][Ho][Wo]
+    bf16 *dze;                      // with embed: gradient w.r.t. the embedding's pre-activation, [mb][E]
+    float *ln_part;                 // with norm: per-block partial sums of the gamma / beta gradients
+    size_t ln_cap;
     bf16 *h[PPO_MAX_FC + 1];       // h[0] = [pooled, proprio]; h[l] post-ReLU
     bf16 *dh[PPO_MAX_FC + 2];      // dh[l]: gradient w.r.t. pre-activation of h[l]; dh[F+1]: head dout padded to 16
     float *dh0_f32;                // gradient w.r.t. h[0] (pooled part feeds the un-pool)
     bf16 *wT;                      // transposed bf16 weights Wt[ci][tap][co padded to 8] for the dgrad GEMMs
-    int64_t wT_off[2 * PPO_MAX_CONV + 2 * PPO_MAX_FC + 3];  // per tensor index (matrices only)
+    int64_t wT_off[PPO_MAX_TENSORS];  // per tensor index (matrices only)
     size_t wT_elems;
     bf16 *wC;                      // conv weights regrouped for the merged dgrad: Wc[class*Ci+ci][shift][co]
     int64_t wC_off[PPO_MAX_CONV + 1];  // per conv layer l (2..L)
     size_t wC_elems;
     // scratch of the two-stage (reproducible) gradient reductions, per weight-matrix tensor index
-    float *wg_part[2 * PPO_MAX_CONV + 2 * PPO_MAX_FC + 3];  // partial tiles of the split-K weight-gradient GEMMs
-    size_t wg_cap[2 * PPO_MAX_CONV + 2 * PPO_MAX_FC + 3];   // floats
-    float *cs_part[2 * PPO_MAX_CONV + 2 * PPO_MAX_FC + 3];  // per-block partial column sums (bias gradients)
+    float *wg_part[PPO_MAX_TENSORS];  // partial tiles of the split-K weight-gradient GEMMs
+    size_t wg_cap[PPO_MAX_TENSORS];   // floats
+    float *cs_part[PPO_MAX_TENSORS];  // per-block partial column sums (bias gradients)
     float *c1_part;                                         // per-block partial sums of the first layer's gradients
     size_t c1_cap;
     float *loss_partials;

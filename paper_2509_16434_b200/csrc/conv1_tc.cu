@@ -33,6 +33,9 @@ struct Args {
     const float *bias;  // [C1]
     bf16 *out;          // [M][C1]
     uint32_t *bits;     // [M][C1 / 32] or null
+    const float *ln_gamma, *ln_beta;  // layer normalisation over the C1 channels of a pixel (null: none; C1 = 16 or 32)
+    bf16 *ln_xhat;      // [M][C1]
+    float *ln_rstd;     // [M]
     long long M;        // output pixels
     int Hi, Wi, Ho, Wo, C1;
     int tiles;   // 128-pixel tiles
@@ -48,7 +51,7 @@ struct Pipe {
     uint64_t tempty[4];
     uint32_t tmem_slot;
     int abort_flag;
-    alignas(16) uint32_t pad[2];
+    alignas(16) float gamma[32], beta[32];
 };
 
 // Unswizzled K-major operand image: element (row r, column k) of a tile with KP columns lives at
@@ -120,6 +123,10 @@ __global__ void __launch_bounds__(kThreads, 1) conv1_tc_kernel(const __grid_cons
             f = a.bias[n] - __half2float(__float2half_rn(a.bias[n]));
         }
         *reinterpret_cast<__half *>(bsm + core_offset(n, k >> 3, KP) + (k & 7) * 2) = __float2half_rn(f);
+    }
+    if (a.ln_gamma && threadIdx.x < 32) {
+        pipe->gamma[threadIdx.x] = (int)threadIdx.x < N ? a.ln_gamma[threadIdx.x] : 0.f;
+        pipe->beta[threadIdx.x] = (int)threadIdx.x < N ? a.ln_beta[threadIdx.x] : 0.f;
     }
     fence_async_smem();
     if (warp == kProdGroups * 4) tmem_alloc(&pipe->tmem_slot, ncols);
@@ -257,6 +264,34 @@ __global__ void __launch_bounds__(kThreads, 1) conv1_tc_kernel(const __grid_cons
                 if (CW == 32) tmem_ld16(lane_base + (uint32_t)cc + 16u, v + 16);
                 uint32_t pk[16];
                 uint32_t gate = 0;
+                if (a.ln_gamma) {
+                    // layer normalisation over the CW = C1 channels this thread holds: two passes in registers; the
+                    // normalised values are stored pixel by pixel (a thread's CW values are contiguous)
+                    float sum = 0.f, sq = 0.f;
+#pragma unroll
+                    for (int i = 0; i < 32; ++i)
+                        if (i < CW) sum += v[i];
+                    const float mean = sum / (float)CW;
+#pragma unroll
+                    for (int i = 0; i < 32; ++i)
+                        if (i < CW) sq += (v[i] - mean) * (v[i] - mean);
+                    const float rs = rsqrtf(sq / (float)CW + kLnEps);
+#pragma unroll
+                    for (int i = 0; i < 32; ++i)
+                        if (i < CW) v[i] = (v[i] - mean) * rs;
+                    if (m0 + lane < a.M) {
+                        uint4 *xp = reinterpret_cast<uint4 *>(a.ln_xhat + (m0 + lane) * N + c0);
+#pragma unroll
+                        for (int j = 0; j < 4; ++j)
+                            if (j < CW / 8)
+                                xp[j] = make_uint4(pack_bf16x2(v[8 * j], v[8 * j + 1]), pack_bf16x2(v[8 * j + 2], v[8 * j + 3]),
+                                                   pack_bf16x2(v[8 * j + 4], v[8 * j + 5]), pack_bf16x2(v[8 * j + 6], v[8 * j + 7]));
+                        a.ln_rstd[m0 + lane] = rs;
+                    }
+#pragma unroll
+                    for (int i = 0; i < 32; ++i)
+                        if (i < CW) v[i] = fmaf(pipe->gamma[c0 + i], v[i], pipe->beta[c0 + i]);
+                }
 #pragma unroll
                 for (int j = 0; j < 16; ++j) {
                     if (j < CW / 2) {
@@ -325,11 +360,14 @@ int launch(Args &a, cudaStream_t st) {
 // ReLU gates.  Returns PPO_ERR_UNSUPPORTED (nothing launched) for shapes it does not cover: C1 must be a multiple
 // of 16 up to 256 (of 32 when bits are wanted), k in {3, 5, 7}, the frame width even and the frames 4-byte aligned.
 int conv1_tc_fwd(const __half *depth, const bf16 *W, const float *bias, bf16 *out, uint32_t *bits, int rows, int Hi,
-                 int Wi, int Ho, int Wo, int C1, int ks, int32_t *status, cudaStream_t st) {
+                 int Wi, int Ho, int Wo, int C1, int ks, const float *ln_gamma, const float *ln_beta, bf16 *ln_xhat,
+                 float *ln_rstd, int32_t *status, cudaStream_t st) {
     if (!status || C1 % 16 != 0 || C1 > 256 || C1 < 16 || (bits && C1 % 32 != 0)) return PPO_ERR_UNSUPPORTED;
+    if (ln_gamma && ((C1 != 16 && C1 != 32) || !ln_beta || !ln_xhat || !ln_rstd)) return PPO_ERR_UNSUPPORTED;
     if (Wi % 2 != 0 || !ppo_aligned(depth, 4)) return PPO_ERR_UNSUPPORTED;
     Args a;
     a.depth = depth; a.W = W; a.bias = bias; a.out = out; a.bits = bits;
+    a.ln_gamma = ln_gamma; a.ln_beta = ln_beta; a.ln_xhat = ln_xhat; a.ln_rstd = ln_rstd;
     a.M = (long long)rows * Ho * Wo;
     a.Hi = Hi; a.Wi = Wi; a.Ho = Ho; a.Wo = Wo; a.C1 = C1;
     const long long tiles = (a.M + 127) / 128;

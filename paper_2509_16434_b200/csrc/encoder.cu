@@ -576,6 +576,102 @@ __global__ void __launch_bounds__(256) transpose_weights_kernel(const bf16 *__re
     Wt[i] = (co < Co) ? W[((size_t)co * taps + tap) * Ci + ci] : __float2bfloat16_rn(0.f);
 }
 
+// h0[b][E .. E+P) = proprio[b] as bf16 (the embedding occupies the first E columns of a row of ld elements).
+__global__ void __launch_bounds__(256) concat_proprio_kernel(const float *__restrict__ proprio, bf16 *__restrict__ h0,
+                                                             int rows, int E, int P, int ld) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= rows * P) return;
+    const int b = i / P, j = i - b * P;
+    h0[(size_t)b * ld + E + j] = __float2bfloat16_rn(proprio[i]);
+}
+
+// dz[b][e] = dh0[b][e] where the embedding h0[b][e] is > 0, else 0 (back through its ReLU), as a bf16 GEMM operand.
+__global__ void __launch_bounds__(256) embed_dz_kernel(const float *__restrict__ dh0, const bf16 *__restrict__ h0,
+                                                       bf16 *__restrict__ dz, int rows, int E, int ld) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= rows * E) return;
+    const int b = i / E, e = i - b * E;
+    const float v = bf2f(h0[(size_t)b * ld + e]) > 0.f ? dh0[(size_t)b * ld + e] : 0.f;
+    dz[i] = __float2bfloat16_rn(v);
+}
+
+// Backward of the layer normalisation of one conv layer, in place on the gradient: d [M][C] holds dL/d(gamma xhat + beta)
+// (already zero where the ReLU was off) and leaves dL/dz,
+//   t = gamma d,  dz = rstd (t - mean_c(t) - xhat mean_c(t xhat)),
+// and every block leaves its partial sums of dgamma = sum d xhat and dbeta = sum d in part[block][2 C].  C / 8 lanes
+// share a pixel (8 channels each, one 128-bit access per array), C a power of two in 16 .. 256.
+__global__ void __launch_bounds__(256) ln_bwd_kernel(bf16 *__restrict__ d, const bf16 *__restrict__ xhat,
+                                                     const float *__restrict__ rstd, const float *__restrict__ gamma,
+                                                     long long M, int C, float *__restrict__ part) {
+    __shared__ float sh[16][256];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int lpp = C >> 3, ppw = 32 / lpp;
+    const int cq = lane % lpp, slot = lane / lpp;
+    float gm[8], dg[8], db[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        gm[i] = gamma[cq * 8 + i];
+        dg[i] = 0.f;
+        db[i] = 0.f;
+    }
+    const float inv_c = 1.f / (float)C;
+    for (long long px0 = ((long long)blockIdx.x * 8 + warp) * ppw; px0 < M; px0 += (long long)gridDim.x * 8 * ppw) {
+        const long long px = px0 + slot;
+        const bool live = px < M;
+        float dv[8], xv[8], t[8];
+        uint4 rd = make_uint4(0, 0, 0, 0), rx = make_uint4(0, 0, 0, 0);
+        float rs = 0.f;
+        if (live) {
+            rd = *reinterpret_cast<const uint4 *>(d + px * C + cq * 8);
+            rx = *reinterpret_cast<const uint4 *>(xhat + px * C + cq * 8);
+            rs = rstd[px];
+        }
+        const __nv_bfloat162 *d2 = reinterpret_cast<const __nv_bfloat162 *>(&rd);
+        const __nv_bfloat162 *x2 = reinterpret_cast<const __nv_bfloat162 *>(&rx);
+        float s1 = 0.f, s2 = 0.f;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const float2 a = __bfloat1622float2(d2[i]), b = __bfloat1622float2(x2[i]);
+            dv[2 * i] = a.x; dv[2 * i + 1] = a.y;
+            xv[2 * i] = b.x; xv[2 * i + 1] = b.y;
+        }
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            t[i] = gm[i] * dv[i];
+            s1 += t[i];
+            s2 += t[i] * xv[i];
+            dg[i] += dv[i] * xv[i];
+            db[i] += dv[i];
+        }
+        for (int o = 1; o < lpp; o <<= 1) {  // the lanes of a pixel are adjacent
+            s1 += __shfl_xor_sync(0xffffffffu, s1, o);
+            s2 += __shfl_xor_sync(0xffffffffu, s2, o);
+        }
+        const float m1 = s1 * inv_c, m2 = s2 * inv_c;
+        if (live) {
+            uint4 o4;
+            o4.x = pack_bf16x2(rs * (t[0] - m1 - xv[0] * m2), rs * (t[1] - m1 - xv[1] * m2));
+            o4.y = pack_bf16x2(rs * (t[2] - m1 - xv[2] * m2), rs * (t[3] - m1 - xv[3] * m2));
+            o4.z = pack_bf16x2(rs * (t[4] - m1 - xv[4] * m2), rs * (t[5] - m1 - xv[5] * m2));
+            o4.w = pack_bf16x2(rs * (t[6] - m1 - xv[6] * m2), rs * (t[7] - m1 - xv[7] * m2));
+            *reinterpret_cast<uint4 *>(d + px * C + cq * 8) = o4;
+        }
+    }
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        sh[i][threadIdx.x] = dg[i];
+        sh[8 + i][threadIdx.x] = db[i];
+    }
+    __syncthreads();
+    // channel ch of kind k (0: dgamma, 1: dbeta): the threads whose lane % lpp == ch / 8, in thread order
+    for (int o = threadIdx.x; o < 2 * C; o += 256) {
+        const int k = o / C, ch = o - k * C, q = ch >> 3, e = k * 8 + (ch & 7);
+        float v = 0.f;
+        for (int tdx = q; tdx < 256; tdx += lpp) v += sh[e][tdx];
+        part[(size_t)blockIdx.x * 2 * C + o] = v;
+    }
+}
+
 // ------------------------------------------------------------ orchestration ----
 
 static ConvGeom conv_geom(const ppo_model *m, int l, int rows) {  // conv layer l in 1..L
@@ -691,10 +787,13 @@ extern "C" int ppo_encoder_fwd(ppo_model *m, const ppo_minibatch *mb, int row0, 
         const __half *depth = static_cast<const __half *>(mb->depth_f16) + (size_t)row0 * d.H * d.W;
         const int C1 = m->Cs[1], KS = d.conv_k[0];
         const long long M = (long long)rows * m->Hs[1] * m->Ws[1];
-        const int tcs =
-            conv1_tc_fwd(depth, m->shadow + m->tensors[0].off, m->master + m->tensors[1].off, m->act[1], m->abits[1],
-                               rows, d.H, d.W, m->Hs[1], m->Ws[1], C1, KS, ppo_device_status_ptr(), st);
-        if (tcs != PPO_OK && tcs != PPO_ERR_UNSUPPORTED) return tcs;
+        const bool norm = d.norm != 0;
+        const int tcs = conv1_tc_fwd(depth, m->shadow + m->tensors[0].off, m->master + m->tensors[1].off, m->act[1],
+                                     m->abits[1], rows, d.H, d.W, m->Hs[1], m->Ws[1], C1, KS,
+                                     norm ? m->master + m->tensors[2].off : nullptr,
+                                     norm ? m->master + m->tensors[3].off : nullptr, norm ? m->xhat[1] : nullptr,
+                                     norm ? m->rstd[1] : nullptr, ppo_device_status_ptr(), st);
+        if (tcs != PPO_OK && (tcs != PPO_ERR_UNSUPPORTED || norm)) return tcs;  // only the tensor-core kernel normalises
         const int CH = C1 / 8;
         const bool stage = CH == 1 || CH == 2 || CH == 4 || CH == 8;
         const size_t smem = (size_t)(KS * KS * C1 + C1) * sizeof(float) + (stage ? (size_t)4 * 32 * C1 * 2 : 0);
@@ -720,14 +819,31 @@ extern "C" int ppo_encoder_fwd(ppo_model *m, const ppo_minibatch *mb, int row0, 
     }
     for (int l = 2; l <= m->L; ++l) {
         ConvGeom g = conv_geom(m, l, rows);
-        FwdEpilogue e = {m->master + m->tensors[2 * (l - 1) + 1].off, 1, m->act[l], nullptr, nullptr, 0};
+        const int tc = m->ti_conv[l];
+        FwdEpilogue e = {m->master + m->tensors[tc + 1].off, 1, m->act[l], nullptr, nullptr, 0};
         e.out_bits = m->abits[l];
-        PPO_TRY(run_fwd(m, g, m->act[l - 1], m->shadow + m->tensors[2 * (l - 1)].off, e, st));
+        if (d.norm) {
+            e.ln_gamma = m->master + m->tensors[tc + 2].off;
+            e.ln_beta = m->master + m->tensors[tc + 3].off;
+            e.ln_xhat = m->xhat[l];
+            e.ln_rstd = m->rstd[l];
+        }
+        PPO_TRY(run_fwd(m, g, m->act[l - 1], m->shadow + m->tensors[tc].off, e, st));
     }
-    pool_concat_kernel<<<ppo_cdiv(rows, 8), 256, 0, st>>>(m->act[m->L], mb->proprio + (size_t)row0 * d.P, m->h[0], rows,
-                                                          m->Hs[m->L] * m->Ws[m->L], m->Cs[m->L], d.P);
+    if (m->ti_embed >= 0) {
+        // flatten -> fully connected -> ReLU into the first E columns of h_0, proprio behind them
+        ConvGeom g = fc_geom(rows, m->Hs[m->L] * m->Ws[m->L] * m->Cs[m->L], d.embed);
+        FwdEpilogue e = {m->master + m->tensors[m->ti_embed + 1].off, 1, m->h[0], nullptr, nullptr, 0};
+        e.ldo = m->hw[0];
+        PPO_TRY(run_fwd(m, g, m->act[m->L], m->shadow + m->tensors[m->ti_embed].off, e, st));
+        concat_proprio_kernel<<<ppo_cdiv((long long)rows * d.P, 256), 256, 0, st>>>(mb->proprio + (size_t)row0 * d.P, m->h[0],
+                                                                                  rows, d.embed, d.P, m->hw[0]);
+    } else {
+        pool_concat_kernel<<<ppo_cdiv(rows, 8), 256, 0, st>>>(m->act[m->L], mb->proprio + (size_t)row0 * d.P, m->h[0], rows,
+                                                              m->Hs[m->L] * m->Ws[m->L], m->Cs[m->L], d.P);
+    }
     PPO_LAUNCH_CHECK();
-    int ti = 2 * m->L;
+    int ti = m->ti_fc[1];
     for (int l = 1; l <= m->F; ++l, ti += 2) {
         ConvGeom g = fc_geom(rows, m->hw[l - 1], m->hw[l]);
         FwdEpilogue e = {m->master + m->tensors[ti + 1].off, 1, m->h[l], nullptr, nullptr, 0};
@@ -750,15 +866,22 @@ static int refresh_transposed(ppo_model *m, cudaStream_t st) {
     if (m->wT_valid) return PPO_OK;
     for (int l = 2; l <= m->L; ++l) {
         const int Co = m->Cs[l], Ci = m->Cs[l - 1], taps = m->d.conv_k[l - 1] * m->d.conv_k[l - 1];
+        const int tc = m->ti_conv[l];
         const long long total = (long long)Ci * taps * wt_ld_of(Co);
-        transpose_weights_kernel<<<ppo_cdiv(total, 256), 256, 0, st>>>(m->shadow + m->tensors[2 * (l - 1)].off,
-                                                                     m->wT + m->wT_off[2 * (l - 1)], Co, taps, Ci,
-                                                                     wt_ld_of(Co));
+        transpose_weights_kernel<<<ppo_cdiv(total, 256), 256, 0, st>>>(m->shadow + m->tensors[tc].off,
+                                                                     m->wT + m->wT_off[tc], Co, taps, Ci, wt_ld_of(Co));
         PPO_LAUNCH_CHECK();
-        PPO_TRY(tma_dgrad_weights(m->shadow + m->tensors[2 * (l - 1)].off, m->wC + m->wC_off[l], Co, m->d.conv_k[l - 1], Ci,
+        PPO_TRY(tma_dgrad_weights(m->shadow + m->tensors[tc].off, m->wC + m->wC_off[l], Co, m->d.conv_k[l - 1], Ci,
                                   wt_ld_of(Co), st));
     }
-    int ti = 2 * m->L;
+    if (m->ti_embed >= 0) {
+        const int Ci = m->Hs[m->L] * m->Ws[m->L] * m->Cs[m->L], Co = m->d.embed;
+        const long long total = (long long)Ci * wt_ld_of(Co);
+        transpose_weights_kernel<<<ppo_cdiv(total, 256), 256, 0, st>>>(m->shadow + m->tensors[m->ti_embed].off,
+                                                                     m->wT + m->wT_off[m->ti_embed], Co, 1, Ci, wt_ld_of(Co));
+        PPO_LAUNCH_CHECK();
+    }
+    int ti = m->ti_fc[1];
     for (int l = 1; l <= m->F + 1; ++l, ti += 2) {
         const int Ci = m->hw[l - 1], Co = (l <= m->F) ? m->hw[l] : m->d.A + 1;
         const long long total = (long long)Ci * wt_ld_of(Co);
@@ -897,7 +1020,7 @@ extern "C" int ppo_encoder_bwd(ppo_model *m, const ppo_minibatch *mb, int row0, 
     PPO_TRY(fork_here());
     // head and hidden FC layers, last to first; layer index F+1 is the head
     for (int l = F + 1; l >= 1; --l) {
-        const int ti = 2 * L + 2 * (l - 1);
+        const int ti = m->ti_fc[l];
         const int Co = (l <= F) ? m->hw[l] : d.A + 1;
         const int ldy = (l <= F) ? Co : 16;
         ConvGeom g = fc_geom(rows, m->hw[l - 1], Co);
@@ -911,36 +1034,70 @@ extern "C" int ppo_encoder_bwd(ppo_model *m, const ppo_minibatch *mb, int row0, 
         if (s == PPO_OK && l > 1) s = fork_here();  // dh[l-1] is ready for the next leaf
         if (s != PPO_OK) return join(s);
     }
-    {
+    if (m->ti_embed >= 0) {
+        // back through the embedding: its ReLU, then weight gradient (a leaf) and input gradient (masked by the
+        // ReLU of the last conv output, which the flattened vector is)
+        const int te = m->ti_embed, E = d.embed;
+        ConvGeom g = fc_geom(rows, m->Hs[L] * m->Ws[L] * m->Cs[L], E);
+        embed_dz_kernel<<<ppo_cdiv((long long)rows * E, 256), 256, 0, st>>>(m->dh0_f32, m->h[0], m->dze, rows, E, m->hw[0]);
+        PPO_LAUNCH_CHECK();
+        int s = fork_here();
+        if (s == PPO_OK) s = run_wgrad(m, te, g, m->dze, E, m->act[L], leaf);
+        DgradEpilogue e = {m->act[L], m->dact[L], nullptr};
+        if (s == PPO_OK)
+            s = run_dgrad(m, g, m->dze, E, m->shadow + m->tensors[te].off, m->wT + m->wT_off[te], wt_ld_of(E), nullptr, e, st);
+        if (s != PPO_OK) return join(s);
+    } else {
         const int npx = m->Hs[L] * m->Ws[L], C = m->Cs[L];
         const long long total8 = (long long)rows * npx * C / 8;
         unpool_kernel<<<ppo_cdiv(total8, 256), 256, 0, st>>>(m->dh0_f32, m->act[L], m->dact[L], total8, npx, C,
                                                            m->hw[0]);
         PPO_LAUNCH_CHECK();
     }
+    // With layer normalisation dact[l] arrives as the gradient of the normalised, scaled and shifted value; ln_bwd
+    // turns it in place into the gradient of the convolution's output and adds the gamma and beta gradients.
+    auto ln_bwd = [&](int l) -> int {
+        if (!d.norm) return PPO_OK;
+        const int C = m->Cs[l], tc = m->ti_conv[l];
+        const long long M = (long long)rows * m->Hs[l] * m->Ws[l];
+        const int lpp = C / 8;
+        if (C < 16 || C > 256 || (C & (C - 1)) != 0) return PPO_ERR_UNSUPPORTED;
+        int blocks = ppo_cdiv(M, (long long)8 * (32 / lpp) * 4);
+        const int cap = ppo_num_sms() * 4;
+        blocks = blocks > cap ? cap : (blocks < 1 ? 1 : blocks);
+        if ((size_t)blocks * 2 * C > m->ln_cap) return PPO_ERR_SHAPE;
+        ln_bwd_kernel<<<blocks, 256, 0, st>>>(m->dact[l], m->xhat[l], m->rstd[l], m->master + m->tensors[tc + 2].off, M, C,
+                                              m->ln_part);
+        PPO_LAUNCH_CHECK();
+        return sum_partials(m->ln_part, blocks, C, m->grad + m->tensors[tc + 2].off, C, m->grad + m->tensors[tc + 3].off, st);
+    };
     // The chain of dgrads first; then the wgrads of the GEMM layers one after the other on the caller's stream
     // with conv1's wgrad beside them on the second one.  A wgrad GEMM takes most of an SM's shared memory but
     // few registers and threads, conv1's wgrad the opposite, and both leave most issue slots and half the DRAM
     // bandwidth unused on their own, so they share the SMs.  (The dgrad kernels take whole SMs: nothing fits
     // beside them.)  Without a second stream the order is the plain one: wgrad, dgrad, layer by layer.
     for (int l = L; l >= 2; --l) {
-        const int ti = 2 * (l - 1);
+        const int ti = m->ti_conv[l];
         ConvGeom g = conv_geom(m, l, rows);
         DgradEpilogue e = {m->act[l - 1], m->dact[l - 1], nullptr};
         e.mask_bits = m->abits[l - 1];
-        int s = PPO_OK;
-        if (!fork)
+        int s = ln_bwd(l);
+        if (s == PPO_OK && !fork)
             s = run_wgrad(m, ti, g, m->dact[l], g.Co, m->act[l - 1], st);
         if (s == PPO_OK)
             s = run_dgrad(m, g, m->dact[l], g.Co, m->shadow + m->tensors[ti].off, m->wT + m->wT_off[ti],
                           wt_ld_of(g.Co), m->wC + m->wC_off[l], e, st);
         if (s != PPO_OK) return join(s);
     }
+    {
+        const int s = ln_bwd(1);
+        if (s != PPO_OK) return join(s);
+    }
     if (fork && L >= 2) {
         int s = fork_here();  // dZ1 is ready
         if (s == PPO_OK) s = conv1_wgrad(m, mb, row0, rows, leaf);
         for (int l = 2; l <= L && s == PPO_OK; ++l) {  // conv2 first: the longest, and the best partner
-            const int ti = 2 * (l - 1);
+            const int ti = m->ti_conv[l];
             ConvGeom g = conv_geom(m, l, rows);
             s = run_wgrad(m, ti, g, m->dact[l], g.Co, m->act[l - 1], st);
         }

@@ -15,7 +15,16 @@ struct FwdEpilogue {
     float *out_value;   // head: column A -> [M]
     int A;
     uint32_t *out_bits = nullptr;  // optional: gate bits (out > 0) of a ReLU output, [M][Co / 32]; needs Co % 32 == 0
+    int ldo = 0;                   // row stride of `out` in elements (0: Co)
+    // Layer normalisation over the Co channels of every output row, between the bias and the ReLU (all null: none):
+    // xhat = (z - mean) / sqrt(var + 1e-5), out = act(gamma * xhat + beta); xhat [M][Co] bf16 and rstd [M] fp32 are
+    // kept for the backward pass.  Needs Co <= 256 (one column tile) and ldo == Co.
+    const float *ln_gamma = nullptr, *ln_beta = nullptr;
+    bf16 *ln_xhat = nullptr;
+    float *ln_rstd = nullptr;
 };
+
+constexpr float kLnEps = 1e-5f;
 
 struct DgradEpilogue {
     const bf16 *mask_act;  // [M'][Ci]: output is zeroed where this is <= 0; may be nullptr
@@ -60,5 +69,7 @@ int wgrad_reduce(const float *part, int jtiles, int ctiles, int splits, int BN, 
 int relu_bits(const bf16 *act, uint32_t *bits, long long M, int C, cudaStream_t st);
 
 // First convolution (C_in = 1) as a tensor-core GEMM over thread-built im2col tiles (conv1_tc.cu).
+// ln_* as in FwdEpilogue (all null: no normalisation); with them C1 must be 16 or 32.
 int conv1_tc_fwd(const __half *depth, const bf16 *W, const float *bias, bf16 *out, uint32_t *bits, int rows, int Hi,
-                 int Wi, int Ho, int Wo, int C1, int ks, int32_t *status, cudaStream_t st);
+                 int Wi, int Ho, int Wo, int C1, int ks, const float *ln_gamma, const float *ln_beta, bf16 *ln_xhat,
+                 float *ln_rstd, int32_t *status, cudaStream_t st);

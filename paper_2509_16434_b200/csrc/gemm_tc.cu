@@ -64,6 +64,9 @@ struct KArgs {
     float *out_f32;
     const bf16 *mask;
     float *mean, *value;
+    const float *ln_gamma, *ln_beta;  // forward with layer normalisation over the N columns of a row (null: none)
+    bf16 *ln_xhat;
+    float *ln_rstd;
     int32_t *status;
     int ncls, total_tiles;
     KClass cls[4];
@@ -245,6 +248,31 @@ __global__ void __launch_bounds__(kKThreads, 1) igemm_kmajor_kernel(const __grid
             if (!ok) break;
             tc_fence_after();
             const uint32_t lane_base = tmem_base + acc * acc_cols + ((uint32_t)(lg * 32) << 16);
+            // Layer normalisation: the row of this thread holds all N channels of its pixel (one column tile), so it
+            // walks the row twice (mean, then variance about it) before the pass that writes.
+            float ln_mean = 0.f, ln_rs = 0.f;
+            if (a.ln_gamma && nkb > 0) {
+                float sum = 0.f;
+                for (int c0 = 0; c0 < a.N; c0 += 16) {
+                    float t[16];
+                    tmem_ld16(lane_base + (uint32_t)c0, t);
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) sum += t[i] + a.bias[c0 + i];
+                }
+                ln_mean = sum / (float)a.N;
+                float sq = 0.f;
+                for (int c0 = 0; c0 < a.N; c0 += 16) {
+                    float t[16];
+                    tmem_ld16(lane_base + (uint32_t)c0, t);
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) {
+                        const float dlt = t[i] + a.bias[c0 + i] - ln_mean;
+                        sq += dlt * dlt;
+                    }
+                }
+                ln_rs = rsqrtf(sq / (float)a.N + kLnEps);
+                if (row_ok) a.ln_rstd[orow] = ln_rs;
+            }
             for (int c0 = 0; c0 < BN; c0 += 16) {
                 if (n0 + c0 >= a.N) break;  // uniform across the warp
                 float v[16];
@@ -269,7 +297,22 @@ __global__ void __launch_bounds__(kKThreads, 1) igemm_kmajor_kernel(const __grid
                     for (int i = 0; i < 16; ++i) {
                         const float bv = (n + i < a.N) ? a.bias[n + i] : 0.f;
                         v[i] += bv;
-                        if (a.relu) v[i] = fmaxf(v[i], 0.f);
+                    }
+                    if (a.ln_gamma) {
+                        uint4 *xp = reinterpret_cast<uint4 *>(a.ln_xhat + orow * a.ldo + n);
+                        uint32_t pk[8];
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) v[i] = (v[i] - ln_mean) * ln_rs;
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) pk[i] = pack_bf16x2(v[2 * i], v[2 * i + 1]);
+                        xp[0] = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                        xp[1] = make_uint4(pk[4], pk[5], pk[6], pk[7]);
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) v[i] = fmaf(a.ln_gamma[n + i], v[i], a.ln_beta[n + i]);
+                    }
+                    if (a.relu) {
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) v[i] = fmaxf(v[i], 0.f);
                     }
                 } else if (a.mask) {
                     const uint4 *mp = reinterpret_cast<const uint4 *>(a.mask + orow * a.ldo + n);
@@ -543,8 +586,12 @@ int tc_gemm_fwd(const ConvGeom &g, const bf16 *X, const bf16 *W, const FwdEpilog
     a.Wm = W; a.w_row = g.K(); a.w_tap = g.Ci; a.ck = g.Ci / 8;
     a.s_mul = 2; a.s_oy = a.s_ox = -g.pad;
     a.o_mul = 1; a.Hout = g.Ho; a.Wout = g.Wo;
-    a.N = g.Co; a.BN = pick_bn(g.Co); a.ldo = g.Co;
+    a.N = g.Co; a.BN = pick_bn(g.Co); a.ldo = e.ldo ? e.ldo : g.Co;
     a.mode = e.out ? EPI_FWD : EPI_HEAD; a.relu = e.relu; a.A = e.A;
+    if (e.ln_gamma) {
+        if (!e.ln_beta || !e.ln_xhat || !e.ln_rstd || !e.out || g.Co > 256 || g.Co % 16 != 0 || a.ldo != g.Co) return PPO_ERR_UNSUPPORTED;
+        a.ln_gamma = e.ln_gamma; a.ln_beta = e.ln_beta; a.ln_xhat = e.ln_xhat; a.ln_rstd = e.ln_rstd;
+    }
     a.bias = e.bias; a.out = e.out; a.out_f32 = nullptr; a.mask = nullptr; a.mean = e.out_mean; a.value = e.out_value;
     a.status = status;
     a.ncls = 1;

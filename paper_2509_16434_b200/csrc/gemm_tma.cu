@@ -196,6 +196,9 @@ struct KArgs {
     const uint32_t *mask_bits;  // merged dgrad: the gate as bits, [pixels][nq_ci / 32]
     uint32_t *out_bits;         // forward: gate bits of the ReLU output, [pixels][N / 32]
     float *mean, *value;
+    const float *ln_gamma, *ln_beta;  // forward with layer normalisation over the N columns of a row (null: none)
+    bf16 *ln_xhat;
+    float *ln_rstd;
     int32_t *status;
     KClass cls[4];
 };
@@ -212,6 +215,7 @@ struct PipeK {
     Box boxes[kMaxBoxes];
     uint32_t wtab[4][kMaxWtab];  // resident weights: (byte offset >> 4) of the box that sub-block q of a class reads
     alignas(16) float bias[kMaxBias];
+    alignas(16) float gamma[256], beta[256];  // layer normalisation (N <= 256)
     // followed by the epilogue staging: per epilogue warp 32 rows x 32 bf16 columns (2 KB), 16-byte pieces swizzled
 };
 
@@ -247,6 +251,11 @@ __global__ void __launch_bounds__(kKThreads, 1) tma_kmajor_kernel(const __grid_c
     }
     if (a.mode != EPI_DGRAD)
         for (int i = threadIdx.x; i < a.tiles_n * BN; i += (int)blockDim.x) pipe->bias[i] = i < a.N ? a.bias[i] : 0.f;
+    if (a.ln_gamma)
+        for (int i = threadIdx.x; i < 256; i += (int)blockDim.x) {
+            pipe->gamma[i] = i < a.N ? a.ln_gamma[i] : 0.f;
+            pipe->beta[i] = i < a.N ? a.ln_beta[i] : 0.f;
+        }
     if (a.wres)
         for (int i = threadIdx.x; i < a.ncls * kMaxWtab; i += (int)blockDim.x) {
             const int c = i / kMaxWtab, q = i - c * kMaxWtab;
@@ -452,6 +461,31 @@ __global__ void __launch_bounds__(kKThreads, 1) tma_kmajor_kernel(const __grid_c
                 ok = mbar_wait(&pipe->tfull[acc], (ti >> nacc_log) & 1, abort_flag, a.status);
                 if (!ok) break;
                 tc_fence_after();
+                // Layer normalisation: this thread's row holds all N channels of its pixel in the accumulator, so
+                // every warp of the lane quarter walks the whole row twice (mean, then variance about it) before it
+                // normalises its own column groups.
+                float ln_mean = 0.f, ln_rs = 0.f;
+                if (a.ln_gamma) {
+                    float sum = 0.f;
+                    for (int c0 = 0; c0 < a.N; c0 += 16) {
+                        float t[16];
+                        tmem_ld16(lane_base + (uint32_t)c0, t);
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) sum += t[i] + pipe->bias[c0 + i];
+                    }
+                    ln_mean = sum / (float)a.N;
+                    float sq = 0.f;
+                    for (int c0 = 0; c0 < a.N; c0 += 16) {
+                        float t[16];
+                        tmem_ld16(lane_base + (uint32_t)c0, t);
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) {
+                            const float dlt = t[i] + pipe->bias[c0 + i] - ln_mean;
+                            sq += dlt * dlt;
+                        }
+                    }
+                    ln_rs = rsqrtf(sq / (float)a.N + kLnEps);
+                }
 #pragma unroll
                 for (int g = 0; g < 4; ++g) {
                     if (g >= ng) break;
@@ -469,6 +503,30 @@ __global__ void __launch_bounds__(kKThreads, 1) tma_kmajor_kernel(const __grid_c
                         for (int q = 0; q < 8; ++q) {
                             const float4 bv = bp[q];
                             v[4 * q] += bv.x; v[4 * q + 1] += bv.y; v[4 * q + 2] += bv.z; v[4 * q + 3] += bv.w;
+                        }
+                        if (a.ln_gamma) {
+                            // the normalised values go out first (same staging, same store pattern), then v becomes
+                            // gamma * xhat + beta and takes the usual path
+#pragma unroll
+                            for (int i = 0; i < 32; ++i) v[i] = (v[i] - ln_mean) * ln_rs;
+#pragma unroll
+                            for (int j = 0; j < 4; ++j)
+                                stg[lane * 4 + (j ^ sw)] = make_uint4(pack_bf16x2(v[8 * j], v[8 * j + 1]), pack_bf16x2(v[8 * j + 2], v[8 * j + 3]),
+                                                                       pack_bf16x2(v[8 * j + 4], v[8 * j + 5]), pack_bf16x2(v[8 * j + 6], v[8 * j + 7]));
+                            __syncwarp();
+#pragma unroll
+                            for (int ps = 0; ps < 4; ++ps) {
+                                const int rr = ps * 8 + rr0;
+                                const long long o_r = __shfl_sync(0xffffffffu, orow, rr);
+                                const int ok_r = __shfl_sync(0xffffffffu, okr, rr);
+                                if (ok_r && col + piece * 8 < ncol && c0 + piece * 8 < BN)
+                                    *reinterpret_cast<uint4 *>(a.ln_xhat + o_r * a.ldo + col + piece * 8) =
+                                        stg[rr * 4 + (piece ^ ((rr >> 1) & 3))];
+                            }
+                            __syncwarp();
+                            if (okr && c0 == 0) a.ln_rstd[orow] = ln_rs;
+#pragma unroll
+                            for (int i = 0; i < 32; ++i) v[i] = fmaf(pipe->gamma[c0 + i], v[i], pipe->beta[c0 + i]);
                         }
                         if (a.relu) {
                             uint32_t w = 0;
@@ -835,7 +893,7 @@ int make_map(CUtensorMap *m, const void *base, int rank, const long long *dims, 
 // completed with zeros by the copy engine), or 0 when the TMA kernels do not cover it.
 int channels_per_box(int C, bool flat) {
     if (C % 64 == 0) return 64;
-    if (flat) return (C >= 64 && C % 8 == 0) ? 64 : 0;
+    if (flat) return (C >= 64 && C % 8 == 0) ? 64 : (C % 32 == 0 ? 32 : 0);
     return C % 32 == 0 ? 32 : 0;
 }
 
@@ -930,7 +988,7 @@ int launch_kmajor(KArgs &a, cudaStream_t st) {
     int s = ensure_smem_attrs();
     if (s != PPO_OK) return s;
     a.tiles_n = (a.N + a.BN - 1) / a.BN;
-    if (a.tiles_n * a.BN > kMaxBias) return PPO_ERR_UNSUPPORTED;
+    if (a.mode != EPI_DGRAD && a.tiles_n * a.BN > kMaxBias) return PPO_ERR_UNSUPPORTED;  // bias staged in shared memory
     const long long per = (long long)a.grid.tiles * a.tiles_n;
     const long long total = per * a.ncls;
     if (total <= 0) return PPO_OK;
@@ -1006,8 +1064,15 @@ int tma_gemm_fwd(const ConvGeom &g, const bf16 *X, const bf16 *W, const FwdEpilo
     a.s_oy = a.s_ox = -g.pad;
     a.Hout = flat ? 1 : g.Ho;
     a.Wout = flat ? g.B : g.Wo;
-    a.ldo = g.Co;
+    a.ldo = e.ldo ? e.ldo : g.Co;
     a.mode = e.out ? EPI_FWD : EPI_HEAD;
+    if (e.ln_gamma) {
+        if (!e.ln_beta || !e.ln_xhat || !e.ln_rstd || !e.out || g.Co > 256 || g.Co % 32 != 0 || a.ldo != g.Co) return PPO_ERR_UNSUPPORTED;
+        a.ln_gamma = e.ln_gamma;
+        a.ln_beta = e.ln_beta;
+        a.ln_xhat = e.ln_xhat;
+        a.ln_rstd = e.ln_rstd;
+    }
     a.relu = e.relu;
     a.A = e.A;
     a.bias = e.bias;

@@ -24,7 +24,15 @@ extern "C" int ppo_model_create(const ppo_model_desc *d, ppo_model **out) {
     if (d->conv_c[0] * (d->conv_k[0] * d->conv_k[0] + 1) > 2048) return PPO_ERR_UNSUPPORTED;
     for (int l = 0; l < d->n_fc; ++l)
         if (d->fc[l] <= 0 || d->fc[l] % 8 != 0) return PPO_ERR_UNSUPPORTED;
-    if ((d->conv_c[d->n_conv - 1] + d->P) % 8 != 0) return PPO_ERR_UNSUPPORTED;
+    if (d->embed < 0) return PPO_ERR_INVALID_ARG;
+    if (d->embed > 0 && (d->embed % 32 != 0 || (d->embed + d->P) % 8 != 0 || d->embed > 256)) return PPO_ERR_UNSUPPORTED;
+    if (d->embed == 0 && (d->conv_c[d->n_conv - 1] + d->P) % 8 != 0) return PPO_ERR_UNSUPPORTED;
+    if (d->norm) {
+        // the normalisation runs in the forward kernels' epilogues, where one thread owns all channels of a pixel
+        if ((d->conv_c[0] != 16 && d->conv_c[0] != 32) || d->W % 2 != 0 || d->conv_k[0] == 1) return PPO_ERR_UNSUPPORTED;
+        for (int l = 0; l < d->n_conv; ++l)  // 16, 32, 64, 128 or 256 channels: a pixel's channels split evenly over lanes
+            if (d->conv_c[l] > 256 || d->conv_c[l] < 16 || (d->conv_c[l] & (d->conv_c[l] - 1)) != 0) return PPO_ERR_UNSUPPORTED;
+    }
     ppo_model *m = new (std::nothrow) ppo_model();
     if (!m) return PPO_ERR_INVALID_ARG;
     m->d = *d;
@@ -38,7 +46,7 @@ extern "C" int ppo_model_create(const ppo_model_desc *d, ppo_model **out) {
         m->Ws[l + 1] = conv_out(m->Ws[l], d->conv_k[l]);
         m->Cs[l + 1] = d->conv_c[l];
     }
-    m->hw[0] = m->Cs[m->L] + d->P;
+    m->hw[0] = (d->embed > 0 ? d->embed : m->Cs[m->L]) + d->P;
     for (int l = 0; l < m->F; ++l) m->hw[l + 1] = d->fc[l];
     int64_t off = 0;
     size_t count = 0;
@@ -48,13 +56,26 @@ extern "C" int ppo_model_create(const ppo_model_desc *d, ppo_model **out) {
         count += (size_t)sz;
     };
     for (int l = 0; l < m->L; ++l) {
+        m->ti_conv[l + 1] = (int)m->tensors.size();
         push((int64_t)m->Cs[l + 1] * d->conv_k[l] * d->conv_k[l] * m->Cs[l]);
         push(m->Cs[l + 1]);
+        if (d->norm) {
+            push(m->Cs[l + 1]);
+            push(m->Cs[l + 1]);
+        }
+    }
+    m->ti_embed = -1;
+    if (d->embed > 0) {
+        m->ti_embed = (int)m->tensors.size();
+        push((int64_t)d->embed * m->Hs[m->L] * m->Ws[m->L] * m->Cs[m->L]);
+        push(d->embed);
     }
     for (int l = 0; l < m->F; ++l) {
+        m->ti_fc[l + 1] = (int)m->tensors.size();
         push((int64_t)m->hw[l + 1] * m->hw[l]);
         push(m->hw[l + 1]);
     }
+    m->ti_fc[m->F + 1] = (int)m->tensors.size();
     push((int64_t)(d->A + 1) * m->hw[m->F]);
     push(d->A + 1);
     push(d->A);
@@ -67,9 +88,9 @@ extern "C" int ppo_model_create(const ppo_model_desc *d, ppo_model **out) {
             m->wT_off[ti] = toff;
             toff += (Ci * taps * ((Co + 7) / 8 * 8) + 63) / 64 * 64;
         };
-        for (int l = 2; l <= m->L; ++l) tpush(2 * (l - 1), m->Cs[l - 1], d->conv_k[l - 1] * d->conv_k[l - 1], m->Cs[l]);
-        for (int l = 1; l <= m->F + 1; ++l)
-            tpush(2 * m->L + 2 * (l - 1), m->hw[l - 1], 1, l <= m->F ? m->hw[l] : d->A + 1);
+        for (int l = 2; l <= m->L; ++l) tpush(m->ti_conv[l], m->Cs[l - 1], d->conv_k[l - 1] * d->conv_k[l - 1], m->Cs[l]);
+        if (m->ti_embed >= 0) tpush(m->ti_embed, (int64_t)m->Hs[m->L] * m->Ws[m->L] * m->Cs[m->L], 1, d->embed);
+        for (int l = 1; l <= m->F + 1; ++l) tpush(m->ti_fc[l], m->hw[l - 1], 1, l <= m->F ? m->hw[l] : d->A + 1);
         m->wT_elems = (size_t)toff;
         int64_t coff = 0;
         for (int l = 0; l <= PPO_MAX_CONV; ++l) m->wC_off[l] = 0;
@@ -130,6 +151,9 @@ static size_t carve(ppo_model *m, const ppo_model *shape, int mb, char *base) {
         const bool bits = shape->Cs[l] % 32 == 0 && l < shape->L;  // gate bits for the dgrad of layer l + 1
         char *bt = bits ? take(bytes / 16) : nullptr;
         if (m) m->abits[l] = (uint32_t *)bt;
+        char *xh = shape->d.norm ? take(bytes) : nullptr;
+        char *rs = shape->d.norm ? take((size_t)mb * shape->Hs[l] * shape->Ws[l] * sizeof(float)) : nullptr;
+        if (m) { m->xhat[l] = (bf16 *)xh; m->rstd[l] = (float *)rs; }
     }
     for (int l = 0; l <= shape->F; ++l) {
         size_t bytes = (size_t)mb * shape->hw[l] * sizeof(bf16);
@@ -155,20 +179,29 @@ static size_t carve(ppo_model *m, const ppo_model *shape, int mb, char *base) {
         const size_t c1 = (size_t)6 * sms * shape->Cs[1] * (shape->d.conv_k[0] * shape->d.conv_k[0] + 1);
         char *c1p = take(c1 * sizeof(float));
         if (m) { m->c1_part = (float *)c1p; m->c1_cap = c1; }
-        const int nmat = 2 * shape->L + 2 * (shape->F + 1);
-        for (int ti = 2; ti < nmat; ti += 2) {
+        auto scratch_for = [&](int ti, int Ci, int Co, int k) {
             ConvGeom g = {};
-            if (ti < 2 * shape->L) {
-                const int l = ti / 2 + 1;
-                g.Ci = shape->Cs[l - 1]; g.Co = shape->Cs[l]; g.k = shape->d.conv_k[l - 1];
-            } else {
-                const int l = (ti - 2 * shape->L) / 2 + 1;
-                g.Ci = shape->hw[l - 1]; g.Co = l <= shape->F ? shape->hw[l] : shape->d.A + 1; g.k = 1;
-            }
+            g.Ci = Ci; g.Co = Co; g.k = k;
             const size_t we = wgrad_scratch_elems(g);
             char *wp = take(we * sizeof(float));
-            char *cp = take((size_t)4 * sms * (g.Co < 16 ? 16 : g.Co) * sizeof(float));
+            char *cp = take((size_t)4 * sms * (Co < 16 ? 16 : Co) * sizeof(float));
             if (m) { m->wg_part[ti] = (float *)wp; m->wg_cap[ti] = we; m->cs_part[ti] = (float *)cp; }
+        };
+        for (int l = 2; l <= shape->L; ++l) scratch_for(shape->ti_conv[l], shape->Cs[l - 1], shape->Cs[l], shape->d.conv_k[l - 1]);
+        if (shape->ti_embed >= 0)
+            scratch_for(shape->ti_embed, shape->Hs[shape->L] * shape->Ws[shape->L] * shape->Cs[shape->L], shape->d.embed, 1);
+        for (int l = 1; l <= shape->F + 1; ++l)
+            scratch_for(shape->ti_fc[l], shape->hw[l - 1], l <= shape->F ? shape->hw[l] : shape->d.A + 1, 1);
+        if (shape->d.embed > 0) {
+            char *dz = take((size_t)mb * shape->d.embed * sizeof(bf16));
+            if (m) m->dze = (bf16 *)dz;
+        }
+        if (shape->d.norm) {
+            int cmax = 0;
+            for (int l = 1; l <= shape->L; ++l) cmax = shape->Cs[l] > cmax ? shape->Cs[l] : cmax;
+            const size_t lc = (size_t)4 * sms * 2 * cmax;
+            char *lp2 = take(lc * sizeof(float));
+            if (m) { m->ln_part = (float *)lp2; m->ln_cap = lc; }
         }
     }
     return off;
@@ -206,6 +239,16 @@ extern "C" int ppo_model_activation_ptr(const ppo_model *m, int kind, int index,
     if (kind == 0 && index >= 1 && index <= m->L) {
         *ptr = m->act[index];
         *elems = (size_t)m->mbmax * m->Hs[index] * m->Ws[index] * m->Cs[index];
+        return PPO_OK;
+    }
+    if (kind == 3 && index >= 1 && index <= m->L && m->xhat[index]) {
+        *ptr = m->xhat[index];
+        *elems = (size_t)m->mbmax * m->Hs[index] * m->Ws[index] * m->Cs[index];
+        return PPO_OK;
+    }
+    if (kind == 4 && index >= 1 && index <= m->L && m->rstd[index]) {
+        *ptr = m->rstd[index];
+        *elems = (size_t)m->mbmax * m->Hs[index] * m->Ws[index];
         return PPO_OK;
     }
     if (kind == 2 && index >= 1 && index < m->L && m->abits[index]) {

@@ -35,7 +35,7 @@ class Learner:
         self.hyper = hyper or Hyper(gamma=w.gamma, lam=w.lam, clip=w.clip)
         self.bdesc = ppo.buffer_desc(w.N, w.T, w.H, w.W, w.P, w.A)
         self.buffer = ppo.Buffer(self.bdesc, device)
-        self.mdesc = ppo.model_desc(w.H, w.W, w.conv_c, w.conv_k, w.fc, w.P, w.A)
+        self.mdesc = ppo.model_desc(w.H, w.W, w.conv_c, w.conv_k, w.fc, w.P, w.A, norm=w.norm, embed=w.embed)
         self.microbatch = min(microbatch, w.B)
         self.model = ppo.Model(self.mdesc, self.microbatch, device)
         self.mb = ppo.MinibatchArrays(self.bdesc, w.B, device, with_index=with_index)

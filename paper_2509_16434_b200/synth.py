@@ -38,6 +38,8 @@ class Workload:
     lam: float = 0.95
     clip: float = 0.2
     seed: int = 0
+    norm: bool = False  # layer normalisation over the channels of every conv output, before its ReLU
+    embed: int = 0      # > 0: flatten -> fully connected (embed) -> ReLU instead of the global average pool
 
     @property
     def M(self) -> int:
@@ -59,6 +61,10 @@ WORKLOADS: Dict[str, Workload] = {
     "cfg3": Workload("cfg3", 4096, 16, 120, 160, (32, 64, 128, 256), (3, 3, 3, 3), (512, 512), 5, 4),
     "cfg4": Workload("cfg4", 8192, 16, 240, 320, (32, 64, 128, 256, 256), (5, 3, 3, 3, 3), (512, 512), 5, 8,
                      done_rate=0.005),
+    # the depth CNN of Section III-C on 160x120 frames: [16, 32, 64, 128] filters with layer normalisation and ReLU, a
+    # 32-d embedding of the flattened map, joined with proprioception, fully connected [512, 512, 256]
+    "paper_cnn": Workload("paper_cnn", 1024, 16, 120, 160, (16, 32, 64, 128), (3, 3, 3, 3), (512, 512, 256), 1, 4,
+                          norm=True, embed=32),
     # profiling-sized twin of cfg2: same frames, network and micro-batch shapes, 1/8 of the envs
     "cfg2_prof": Workload("cfg2_prof", 128, 16, 120, 160, (32, 64, 128, 256), (3, 3, 3, 3), (512, 512), 1, 4),
     "cfg5_1k": Workload("cfg5_1k", 1024, 32, 120, 160, (32, 64, 128, 256), (3, 3, 3, 3), (512, 512), 1, 4),
@@ -141,14 +147,39 @@ def rollout_torch(w: Workload, device, seed: int | None = None, chunk_t: int = 1
     }
 
 
-def init_params(total: int, offsets: List[int], shapes: List[tuple], seed: int) -> np.ndarray:
+def param_shapes(w: Workload):
+    """Shapes of the parameter tensors of a workload's network in arena order, and the indices of the layer
+    normalisation scales (which start at 1, not 0)."""
+    shapes, gammas = [], []
+    cin, h, wd = 1, w.H, w.W
+    for c, k in zip(w.conv_c, w.conv_k):
+        shapes += [(c, k, k, cin), (c,)]
+        if w.norm:
+            gammas.append(len(shapes))
+            shapes += [(c,), (c,)]
+        cin = c
+        h, wd = (h + 2 * (k // 2) - k) // 2 + 1, (wd + 2 * (k // 2) - k) // 2 + 1
+    i = cin + w.P
+    if w.embed:
+        shapes += [(w.embed, h * wd * cin), (w.embed,)]
+        i = w.embed + w.P
+    for o in w.fc:
+        shapes += [(o, i), (o,)]
+        i = o
+    shapes += [(w.A + 1, i), (w.A + 1,), (w.A,)]
+    return shapes, gammas
+
+
+def init_params(total: int, offsets: List[int], shapes: List[tuple], seed: int, ones: Sequence[int] = ()) -> np.ndarray:
     """Random initial fp32 parameter vector for a given tensor layout.
 
     Weight tensors (rank >= 2) ~ U(+-sqrt(6 / fan_in)); the last weight tensor (the mean/value head) is
-    scaled by 0.01 so that the initial policy mean is near zero; rank-1 tensors (biases, log-sigma) are 0.
-    Gaps between tensors stay 0.
+    scaled by 0.01 so that the initial policy mean is near zero; rank-1 tensors (biases, log-sigma) are 0,
+    except those listed in `ones` (layer normalisation scales), which are 1.  Gaps between tensors stay 0.
     """
     theta = np.zeros(total, np.float32)
+    for i in ones:
+        theta[offsets[i]: offsets[i] + int(np.prod(shapes[i]))] = 1.0
     g = np.random.Generator(np.random.Philox(key=[seed + 1, 99]))
     mats = [i for i, s in enumerate(shapes) if len(s) >= 2]
     for i in mats:

@@ -19,7 +19,7 @@ def max_abs_scaled(x, ref):
 
 
 def oracle_model(w):
-    return orc.ModelDesc(w.H, w.W, tuple(w.conv_c), tuple(w.conv_k), tuple(w.fc), w.P, w.A)
+    return orc.ModelDesc(w.H, w.W, tuple(w.conv_c), tuple(w.conv_k), tuple(w.fc), w.P, w.A, norm=w.norm, embed=w.embed)
 
 
 def oracle_rollout_actions(md, theta, roll):

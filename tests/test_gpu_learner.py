@@ -39,6 +39,8 @@ def _setup(w, microbatch, seed=0, jitter=True, theta_scale_head=1.0):
     for off, sz, shp in zip(lay.offsets, lay.sizes, lay.shapes):
         if len(shp) == 1:
             theta[off:off + sz] = (0.05 * g.standard_normal(sz)).astype(np.float32)
+    for i in synth.param_shapes(w)[1]:  # layer-normalisation scales sit around 1
+        theta[lay.offsets[i]:lay.offsets[i] + lay.sizes[i]] += 1.0
     roll = synth.rollout_numpy(w, seed)
     action, logp = oracle_rollout_actions(md, theta, roll)
     if jitter:
@@ -81,10 +83,17 @@ def _upload_oracle_activations(L, md, acts, B):
         n = h * w_ * c
         L.model.activation(0, l)[:B * n].copy_(torch.as_tensor(acts[:, off:off + n].reshape(-1)).to(torch.bfloat16))
         off += n
-    widths = [md.conv_c[-1] + md.P] + list(md.fc)
+    widths = [(md.embed or md.conv_c[-1]) + md.P] + list(md.fc)
     for l, n in enumerate(widths):
         L.model.activation(1, l)[:B * n].copy_(torch.as_tensor(acts[:, off:off + n].reshape(-1)).to(torch.bfloat16))
         off += n
+    if md.norm:  # the normalised values and reciprocal standard deviations the backward pass reads
+        for l, (h, w_, c) in enumerate(zip(Ho, Wo, md.conv_c), start=1):
+            n = h * w_ * c
+            L.model.activation(3, l)[:B * n].copy_(torch.as_tensor(acts[:, off:off + n].reshape(-1)).to(torch.bfloat16))
+            off += n
+            L.model.activation(4, l)[:B * h * w_].copy_(torch.as_tensor(acts[:, off:off + h * w_].reshape(-1)).float())
+            off += h * w_
     assert off == acts.shape[1]
 
 
