@@ -22,7 +22,8 @@
 // connected layer is one image with a single row of `batch` pixels, cut into 128-pixel tiles.  Rows of
 // the 128-row MMA tile beyond Wt * R are not written and their results are ignored.
 //
-// Shared-memory rows are 128 bytes (64 channels, SWIZZLE_128B) or 64 bytes (32 channels, SWIZZLE_64B).
+// Shared-memory rows are 128 bytes (64 channels, SWIZZLE_128B), 64 bytes (32 channels, SWIZZLE_64B) or 32 bytes
+// (16 channels, SWIZZLE_32B).
 // Every wait is bounded: on a time-out the kernel records PPO_ERR_TIMEOUT, waits (bounded) for the
 // copies it has in flight, frees its tensor memory and returns.
 #include <cuda.h>  // CUtensorMap and its enums; the encoder is reached through the runtime's entry-point query
@@ -178,7 +179,7 @@ struct KArgs {
     CUtensorMap mapB;
     RowGrid grid;
     int s_mul, s_oy, s_ox;  // source pixel of tap t: (y * s_mul + s_oy + dy[t], x * s_mul + s_ox + dx[t])
-    int CB, row_bytes;      // channels per box (64 or 32) and bytes of a shared-memory row
+    int CB, row_bytes;      // channels per box (64, 32 or 16) and bytes of a shared-memory row
     int kchunks;            // boxes along the channels of one tap
     int w_tap;              // elements between taps in a weight row
     int G, nbmax;           // sub-blocks per stage; most A boxes a tile has
@@ -346,7 +347,7 @@ __global__ void __launch_bounds__(kKThreads, 1) tma_kmajor_kernel(const __grid_c
         const uint32_t d_lo0 = (uint32_t)d0, d_hi = (uint32_t)(d0 >> 32);
         const uint32_t res_lo0 = d_lo0 + ((res_base - smem_base) >> 4);
         const uint32_t stage16 = stage_bytes >> 4, sub16 = sub_bytes >> 4, ab16 = a_bytes >> 4;
-        const bool four = a.CB == 64;  // 4 or 2 K = 16 steps per box (32 bytes each along the swizzled row)
+        const int ksteps = a.CB >> 4;  // 4, 2 or 1 K = 16 steps per box (32 bytes each along the swizzled row)
         int ti = 0, s = 0;
         uint32_t ph = 0;
         bool ok = true;
@@ -372,8 +373,8 @@ __global__ void __launch_bounds__(kKThreads, 1) tma_kmajor_kernel(const __grid_c
                     for (int gi = 0; gi < nval; ++gi, la += sub16) {
                         const uint32_t lb = a.wres ? res_lo0 + tbl[q0 + gi] : la + ab16;
                         umma_bf16_lh(tmem_d, la, d_hi, lb, d_hi, idesc, accum);
-                        umma_bf16_lh(tmem_d, la + 2, d_hi, lb + 2, d_hi, idesc, 1u);
-                        if (four) {
+                        if (ksteps >= 2) umma_bf16_lh(tmem_d, la + 2, d_hi, lb + 2, d_hi, idesc, 1u);
+                        if (ksteps == 4) {
                             umma_bf16_lh(tmem_d, la + 4, d_hi, lb + 4, d_hi, idesc, 1u);
                             umma_bf16_lh(tmem_d, la + 6, d_hi, lb + 6, d_hi, idesc, 1u);
                         }
@@ -683,11 +684,12 @@ __global__ void __launch_bounds__(kThreads, 1) tma_wgrad_kernel(const __grid_con
     const bool ones_tile = a.has_db && blockIdx.x == gridDim.x - 1;
     if (ones_tile) {
         // channel 0 of block ones_blk, all 128 pixel rows of every stage: the first element of 16-byte piece 0,
-        // which the swizzle moves to piece (row & 7) of a 128-byte row, ((row >> 1) & 3) of a 64-byte row
+        // which the swizzle moves to piece (row & 7) of a 128-byte row, ((row >> 1) & 3) of a 64-byte row,
+        // ((row >> 2) & 1) of a 32-byte row
         __syncthreads();
         for (uint32_t i = threadIdx.x; i < (uint32_t)S * 128u; i += kThreads) {
             const uint32_t s = i >> 7, r = i & 127u;
-            const uint32_t piece = rbA == 128u ? (r & 7u) : ((r >> 1) & 3u);
+            const uint32_t piece = rbA == 128u ? (r & 7u) : (rbA == 64u ? ((r >> 1) & 3u) : ((r >> 2) & 1u));
             *reinterpret_cast<bf16 *>(smem + (size_t)s * stage_bytes + (size_t)a.ones_blk * 128u * rbA + r * rbA + piece * 16u) =
                 __float2bfloat16_rn(1.f);
         }
@@ -882,7 +884,8 @@ int make_map(CUtensorMap *m, const void *base, int rank, const long long *dims, 
         s *= dims[i + 1];
     }
     if (box[0] * 2 != row_bytes || !ppo_aligned(base, 16)) return PPO_ERR_UNSUPPORTED;
-    const CUtensorMapSwizzle sw = row_bytes == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B;
+    const CUtensorMapSwizzle sw = row_bytes == 128 ? CU_TENSOR_MAP_SWIZZLE_128B
+                                  : (row_bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B);
     const CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void *>(base), gd, gs, bx,
                           es, CU_TENSOR_MAP_INTERLEAVE_NONE, sw, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
@@ -894,7 +897,7 @@ int make_map(CUtensorMap *m, const void *base, int rank, const long long *dims, 
 int channels_per_box(int C, bool flat) {
     if (C % 64 == 0) return 64;
     if (flat) return (C >= 64 && C % 8 == 0) ? 64 : (C % 32 == 0 ? 32 : 0);
-    return C % 32 == 0 ? 32 : 0;
+    return C % 32 == 0 ? 32 : (C % 16 == 0 ? 16 : 0);
 }
 
 // Chooses the tile rectangle Wt x R (Wt * R <= 128) that fills most of the 128 tile rows with pixels of
@@ -1111,8 +1114,10 @@ int tma_gemm_dgrad(const ConvGeom &g, const bf16 *dY, int ldy, const bf16 *Wt, i
                    const DgradEpilogue &e, int32_t *status, cudaStream_t st) {
     if (!status || g.Ci % 8 != 0 || ldy % 8 != 0 || wt_ld % 8 != 0 || ldy < wt_ld) return PPO_ERR_UNSUPPORTED;
     const bool flat = is_flat(g);
-    // a 32-column group of the staged epilogue must lie inside one parity class
-    if (!flat && (g.k < 3 || g.Hi < 2 || g.Wi < 2 || !Wc || g.Ci % 32 != 0)) return PPO_ERR_UNSUPPORTED;
+    // a 32-column group of the staged epilogue must lie inside one parity class; with 16 input channels the
+    // per-thread epilogue (16 columns = one class at a time) takes over, which needs the bf16 gate
+    if (!flat && (g.k < 3 || g.Hi < 2 || g.Wi < 2 || !Wc)) return PPO_ERR_UNSUPPORTED;
+    if (!flat && g.Ci % 32 != 0 && (g.Ci % 16 != 0 || !e.mask_act || e.mask_bits || !e.out)) return PPO_ERR_UNSUPPORTED;
     const int CB = channels_per_box(g.Co, flat);
     if (CB == 0 || g.taps() > kMaxTaps || wt_ld < g.Co) return PPO_ERR_UNSUPPORTED;
     KArgs a = {};

@@ -157,11 +157,11 @@ __device__ __forceinline__ uint32_t tmem_cols_for(int bn) {
 }
 
 
-// Shared-memory matrix descriptor for a swizzled image with rows of `row_bytes` (128 or 64): layout
-// type 2 (SWIZZLE_128B) or 4 (SWIZZLE_64B) in bits 61-63; offsets as in smem_desc.
+// Shared-memory matrix descriptor for a swizzled image with rows of `row_bytes` (128, 64 or 32): layout
+// type 2 (SWIZZLE_128B), 4 (SWIZZLE_64B) or 6 (SWIZZLE_32B) in bits 61-63; offsets as in smem_desc.
 __device__ __forceinline__ uint64_t smem_desc_sw(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes,
                                                  uint32_t row_bytes) {
-    const uint64_t type = row_bytes == 128u ? 2ull : 4ull;
+    const uint64_t type = row_bytes == 128u ? 2ull : (row_bytes == 64u ? 4ull : 6ull);
     return (uint64_t)((addr >> 4) & 0x3FFFu) | ((uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16) |
            ((uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32) | (1ull << 46) | (type << 61);
 }
