@@ -106,6 +106,19 @@ int ppo_buffer_write_step(ppo_buffer *buf, int t, const void *dev_depth_f16, con
 int ppo_buffer_write_obs(ppo_buffer *buf, int t, const void *dev_depth_f16, const float *dev_proprio, void *stream);
 int ppo_buffer_write_outcome(ppo_buffer *buf, int t, const float *dev_reward, const uint8_t *dev_done, void *stream);
 
+/* Synthetic depth producer, standing in for the simulator's depth rendering (Section III-C; Algorithm 1 renders,
+ * Algorithm 2 receives): ray-casts one small analytic scene per env straight into the DEPTH slab at row t, as fp16.
+ * Pinhole camera at the origin looking along +z with horizontal field of view hfov (radians); pixel (v, u) sees the
+ * ray through ((u + 0.5 - W/2) / f, (v + 0.5 - H/2) / f, 1), f = (W/2) / tan(hfov/2).  The scene of env n is the
+ * plane normal . p = offset (dev_plane [N][4] = {nx, ny, nz, offset}, unit normal) and n_prims (<= 32) primitives,
+ * dev_prims [N][n_prims][8] = {type, x, y, z, p0, p1, p2, p3}: type 0 sphere (centre, radius p0), 1 axis-aligned box
+ * (centre, half extents p0..p2), 2 capsule (segment from (x,y,z) to (x,y,z) + (p0,p1,p2), radius p3).  A pixel gets
+ * the z coordinate of the nearest hit if it lies in [near, far], else 0 (no return).  fp32 arithmetic.
+ * Invalidates advantages computed earlier.  Errors: t outside [0,T), n_prims outside [0,32], bad camera values ->
+ * INVALID_ARG. */
+int ppo_buffer_render_depth(ppo_buffer *buf, int t, float hfov, float near, float far, const float *dev_plane,
+                            int n_prims, const float *dev_prims, void *stream);
+
 /* First stage of TrainPPO (Algorithm 2): generalised advantage estimation per env by a
  * reverse scan over t,
  *   delta_t = r_t + gamma V_{t+1} (1 - d_t) - V_t,  A_t = delta_t + gamma lambda (1 - d_t) A_{t+1},

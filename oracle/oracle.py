@@ -292,3 +292,23 @@ def total_loss_and_grad(md: ModelDesc, theta, depth, proprio, action, logp_old, 
     grad[lay.offsets[-1]: lay.offsets[-1] + md.A] += dls
     L = out[0] + c_v * out[1] - c_e * out[2]
     return L, out, grad, mu, V
+
+
+# -------------------------------------------------------- depth producer ----
+
+def round_fp16(x: float) -> float:
+    lib().orc_round_fp16.restype = C.c_double
+    lib().orc_round_fp16.argtypes = [C.c_double]
+    return float(lib().orc_round_fp16(float(x)))
+
+
+def render_depth(H: int, W: int, hfov: float, near: float, far: float, plane, prims) -> np.ndarray:
+    """plane [N,4] (unit normal, offset), prims [N,K,8] ({type, x, y, z, p0..p3}) -> depth [N,H,W] float64 holding
+    fp16 values (0 where nothing is seen within [near, far])."""
+    plane = _f64(plane)
+    prims = _f64(prims)
+    N, K = prims.shape[0], prims.shape[1]
+    out = np.empty((N, H, W), np.float64)
+    lib().orc_render_depth(C.c_int(N), C.c_int(H), C.c_int(W), C.c_double(hfov), C.c_double(near), C.c_double(far),
+                           _p(plane), C.c_int(K), _p(prims), _p(out))
+    return out

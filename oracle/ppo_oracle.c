@@ -697,3 +697,134 @@ void orc_adam(int64_t n, double *theta, double *m, double *v, const double *g, d
         theta[i] = (double)(float)(theta[i] - lr * mhat / (sqrt(vhat) + eps));
     }
 }
+
+/* ------------------------------------------------------------ depth producer -- */
+
+/* A stand-in for the simulator's tiled depth rendering (Section III-C renders a depth image per environment; the
+ * paper gives no formulas, so the camera and the scene are a reading): one pinhole camera per env at the origin,
+ * looking along +z, pixel (v, u) of an H x W image sees the ray through ((u + 0.5 - W/2) / f, (v + 0.5 - H/2) / f, 1)
+ * with f = (W/2) / tan(hfov/2).  The scene of an env is the plane n . p = d (unit n in params[0..2], d in params[3]) and
+ * n_prims primitives of 8 doubles each: {type, x, y, z, p0, p1, p2, p3}
+ *   type 0 sphere : centre (x,y,z), radius p0
+ *   type 1 box    : centre (x,y,z), half extents (p0,p1,p2), axis aligned
+ *   type 2 capsule: segment from (x,y,z) to (x,y,z) + (p0,p1,p2), radius p3
+ * The depth of a pixel is the z coordinate of the nearest intersection in front of the camera; it is kept when it
+ * lies in [near, far] and is 0 (no return) otherwise, then rounded to fp16 (nearest even) and returned as a double. */
+static double round_fp16(double x) {
+    if (x == 0.0) return 0.0;
+    int e;
+    double m = frexp(fabs(x), &e);          /* |x| = m 2^e, m in [0.5, 1) */
+    int emin = -13;                          /* smallest normal 2^-14 = 0.5 * 2^-13 */
+    int shift = (e < emin ? emin : e) - 11;  /* 11 significant bits above 2^shift */
+    double q = ldexp(fabs(x), -shift);
+    double r = nearbyint(q);                 /* ties to even in the default rounding mode */
+    (void)m;
+    double y = ldexp(r, shift);
+    if (y > 65504.0) y = INFINITY;
+    return x < 0 ? -y : y;
+}
+
+static double hit_sphere(const double o[3], const double d[3], const double c[3], double r) {
+    /* |o + t d - c|^2 = r^2, nearest t > 0 */
+    double oc[3] = {o[0] - c[0], o[1] - c[1], o[2] - c[2]};
+    double a = d[0] * d[0] + d[1] * d[1] + d[2] * d[2];
+    double b = oc[0] * d[0] + oc[1] * d[1] + oc[2] * d[2];
+    double cc = oc[0] * oc[0] + oc[1] * oc[1] + oc[2] * oc[2] - r * r;
+    double disc = b * b - a * cc;
+    if (disc < 0.0) return INFINITY;
+    double s = sqrt(disc);
+    double t = (-b - s) / a;
+    if (t > 0.0) return t;
+    t = (-b + s) / a;
+    return t > 0.0 ? t : INFINITY;
+}
+
+static double hit_box(const double d[3], const double c[3], const double h[3]) {
+    /* slabs, ray from the origin */
+    double t0 = 0.0, t1 = INFINITY;
+    for (int i = 0; i < 3; ++i) {
+        double lo = c[i] - h[i], hi = c[i] + h[i];
+        if (d[i] == 0.0) {
+            if (lo > 0.0 || hi < 0.0) return INFINITY;
+            continue;
+        }
+        double a = lo / d[i], b = hi / d[i];
+        if (a > b) { double tmp = a; a = b; b = tmp; }
+        if (a > t0) t0 = a;
+        if (b < t1) t1 = b;
+    }
+    if (t0 > t1) return INFINITY;
+    return t0 > 0.0 ? t0 : (t1 > 0.0 && t1 < INFINITY ? t1 : INFINITY);
+}
+
+static double hit_capsule(const double d[3], const double pa[3], const double ab[3], double r) {
+    /* cylinder around the segment plus the two end spheres; ray from the origin */
+    double best = INFINITY;
+    const double o[3] = {0.0, 0.0, 0.0};
+    double pb[3] = {pa[0] + ab[0], pa[1] + ab[1], pa[2] + ab[2]};
+    double t = hit_sphere(o, d, pa, r);
+    if (t < best) best = t;
+    t = hit_sphere(o, d, pb, r);
+    if (t < best) best = t;
+    double l2 = ab[0] * ab[0] + ab[1] * ab[1] + ab[2] * ab[2];
+    if (l2 > 0.0) {
+        /* components perpendicular to the axis: |(t d - pa)_perp|^2 = r^2 */
+        double dd = (d[0] * ab[0] + d[1] * ab[1] + d[2] * ab[2]) / l2;
+        double pp = (-(pa[0] * ab[0] + pa[1] * ab[1] + pa[2] * ab[2])) / l2; /* axis coordinate of the origin */
+        double dp[3], op[3];
+        for (int i = 0; i < 3; ++i) {
+            dp[i] = d[i] - dd * ab[i];
+            op[i] = -pa[i] - pp * ab[i];
+        }
+        double a = dp[0] * dp[0] + dp[1] * dp[1] + dp[2] * dp[2];
+        double b = op[0] * dp[0] + op[1] * dp[1] + op[2] * dp[2];
+        double c = op[0] * op[0] + op[1] * op[1] + op[2] * op[2] - r * r;
+        double disc = b * b - a * c;
+        if (a > 0.0 && disc >= 0.0) {
+            double s = sqrt(disc);
+            double ts[2] = {(-b - s) / a, (-b + s) / a};
+            for (int k = 0; k < 2; ++k) {
+                double u = pp + ts[k] * dd; /* position along the axis in units of its length */
+                if (ts[k] > 0.0 && u >= 0.0 && u <= 1.0 && ts[k] < best) best = ts[k];
+            }
+        }
+    }
+    return best;
+}
+
+void orc_render_depth(int N, int H, int W, double hfov, double near, double far, const double *plane /*[N][4]*/,
+                      int n_prims, const double *prims /*[N][n_prims][8]*/, double *depth /*[N][H][W]*/) {
+    double f = (0.5 * W) / tan(0.5 * hfov);
+#pragma omp parallel for schedule(static)
+    for (int n = 0; n < N; ++n) {
+        const double *pl = plane + 4 * (int64_t)n;
+        for (int v = 0; v < H; ++v)
+            for (int u = 0; u < W; ++u) {
+                double d[3] = {(u + 0.5 - 0.5 * W) / f, (v + 0.5 - 0.5 * H) / f, 1.0};
+                double best = INFINITY;
+                double nd = pl[0] * d[0] + pl[1] * d[1] + pl[2] * d[2];
+                if (nd != 0.0) {
+                    double t = pl[3] / nd;
+                    if (t > 0.0) best = t;
+                }
+                for (int p = 0; p < n_prims; ++p) {
+                    const double *q = prims + ((int64_t)n * n_prims + p) * 8;
+                    int type = (int)q[0];
+                    double t = INFINITY;
+                    if (type == 0) {
+                        const double o[3] = {0.0, 0.0, 0.0};
+                        t = hit_sphere(o, d, q + 1, q[4]);
+                    } else if (type == 1) {
+                        t = hit_box(d, q + 1, q + 4);
+                    } else if (type == 2) {
+                        t = hit_capsule(d, q + 1, q + 4, q[7]);
+                    }
+                    if (t < best) best = t;
+                }
+                double z = best; /* d has z = 1: the ray parameter is the depth */
+                depth[((int64_t)n * H + v) * W + u] = (z >= near && z <= far) ? round_fp16(z) : 0.0;
+            }
+    }
+}
+
+double orc_round_fp16(double x) { return round_fp16(x); }

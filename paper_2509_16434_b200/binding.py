@@ -28,7 +28,7 @@ EXPORTS = [
     "ppo_model_sync_shadow", "ppo_encoder_fwd", "ppo_loss_fwd_bwd", "ppo_encoder_bwd", "ppo_model_zero_grad",
     "ppo_adam_step", "ppo_policy_sample", "ppo_poll_status", "ppo_model_activation_ptr", "ppo_gae_static",
     "ppo_model_sync_masks", "ppo_buffer_write_obs", "ppo_buffer_write_outcome", "ppo_policy_act", "ppo_launch_count",
-    "ppo_selftest_wait_timeout",
+    "ppo_selftest_wait_timeout", "ppo_buffer_render_depth",
 ]
 
 
@@ -104,6 +104,8 @@ def lib():
         L.ppo_buffer_write_obs.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p]
         L.ppo_buffer_write_outcome.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p]
         L.ppo_policy_act.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.c_void_p]
+        L.ppo_buffer_render_depth.argtypes = [C.c_void_p, C.c_int, C.c_float, C.c_float, C.c_float, C.c_void_p, C.c_int,
+                                              C.c_void_p, C.c_void_p]
         L.ppo_launch_count.restype = C.c_uint64
         L.ppo_launch_count.argtypes = []
         L.ppo_selftest_wait_timeout.argtypes = [C.c_longlong, C.c_void_p, C.c_void_p]
@@ -205,6 +207,12 @@ def ppo_buffer_write_obs(buf: Buffer, t: int, depth, proprio, stream=None):
 def ppo_buffer_write_outcome(buf: Buffer, t: int, reward, done, stream=None):
     _check(lib().ppo_buffer_write_outcome(buf.handle, t, _ptr(reward), _ptr(done), _stream(stream)),
            "ppo_buffer_write_outcome")
+
+
+def ppo_buffer_render_depth(buf: Buffer, t: int, hfov: float, near: float, far: float, plane, prims, stream=None):
+    """plane [N,4] fp32, prims [N,K,8] fp32 device tensors: renders the scenes into slab row t of the depth field."""
+    _check(lib().ppo_buffer_render_depth(buf.handle, t, hfov, near, far, _ptr(plane), prims.shape[1], _ptr(prims),
+                                         _stream(stream)), "ppo_buffer_render_depth")
 
 
 def ppo_launch_count() -> int:

@@ -170,6 +170,26 @@ def param_shapes(w: Workload):
     return shapes, gammas
 
 
+def scenes_numpy(N: int, n_prims: int, seed: int):
+    """Seeded scene parameters for the depth producer: per env a table-like plane below the camera and n_prims
+    spheres, boxes and capsules in front of it.  Returns (plane [N,4], prims [N,n_prims,8]) as float32."""
+    g = np.random.Generator(np.random.Philox(key=[seed, 4242]))
+    nrm = np.stack([0.1 * g.standard_normal(N), -np.ones(N), -0.3 + 0.1 * g.standard_normal(N)], 1)
+    nrm /= np.linalg.norm(nrm, axis=1, keepdims=True)
+    plane = np.concatenate([nrm, -(0.4 + 0.2 * g.random((N, 1)))], 1).astype(np.float32)
+    prims = np.zeros((N, n_prims, 8), np.float32)
+    prims[:, :, 0] = g.integers(0, 3, (N, n_prims))
+    prims[:, :, 1] = g.uniform(-0.5, 0.5, (N, n_prims))
+    prims[:, :, 2] = g.uniform(-0.3, 0.4, (N, n_prims))
+    prims[:, :, 3] = g.uniform(0.5, 1.8, (N, n_prims))
+    size = g.uniform(0.05, 0.2, (N, n_prims, 4)).astype(np.float32)
+    prims[:, :, 4:8] = size
+    cap = prims[:, :, 0] == 2  # capsules: p0..p2 is the segment vector, p3 the radius
+    prims[:, :, 4:7][cap] = g.uniform(-0.25, 0.25, (int(cap.sum()), 3))
+    prims[:, :, 7][cap] = g.uniform(0.03, 0.1, int(cap.sum()))
+    return plane, prims
+
+
 def init_params(total: int, offsets: List[int], shapes: List[tuple], seed: int, ones: Sequence[int] = ()) -> np.ndarray:
     """Random initial fp32 parameter vector for a given tensor layout.
 
