@@ -330,6 +330,17 @@ def run_ours(args):
         bwd_ms, _ = timer.mean_ms("ppo_encoder_bwd")
         gat_ms, _ = timer.mean_ms("ppo_shuffle_gather_minibatch")
         gae_ms, _ = timer.mean_ms("ppo_compute_gae")
+        # the single-launch variant of GAE + moments + normalisation (scan, grid barrier, normalise), outside the step
+        gae1 = []
+        for i in range(8):
+            s_, e_ = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            s_.record()
+            ppo.ppo_compute_gae(L.buffer, lastv[0], w.gamma, w.lam, 2, L.stats)
+            e_.record()
+            torch.cuda.synchronize()
+            if i >= 3:
+                gae1.append(s_.elapsed_time(e_))
+        gae1_ms = float(np.median(gae1))
         adam_ms, _ = timer.mean_ms("ppo_adam_step")
         # a trailing micro-batch may be smaller; use the true mean rows per call
         calls_per_mb = -(-w.B // rows)
@@ -357,7 +368,8 @@ def run_ours(args):
                        "frac": round(gather_gbs / peaks["hbm_gbs"], 4), "ms": round(gat_ms, 4)},
             "gae_norm": {"bound": "hbm", "achieved": round(gae_gbs, 1), "peak": peaks["hbm_gbs"], "unit": "GB/s",
                          "frac": round(gae_gbs / peaks["hbm_gbs"], 4), "ms": round(gae_ms, 4),
-                         "note": "working set fits L2; launch-latency bound at this size"},
+                         "note": "working set fits L2; launch-latency bound at this size",
+                         "single_cooperative_launch_ms": round(gae1_ms, 4)},
             "adam": {"bound": "hbm", "achieved": round(adam_gbs, 1), "peak": peaks["hbm_gbs"], "unit": "GB/s",
                      "frac": round(adam_gbs / peaks["hbm_gbs"], 4), "ms": round(adam_ms, 4),
                      "note": "working set fits L2; launch-latency bound at this size"},

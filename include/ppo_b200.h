@@ -126,7 +126,11 @@ int ppo_buffer_render_depth(ppo_buffer *buf, int t, float hfov, float near, floa
  * written to the ADV and RET slabs; then, if normalize != 0, the advantages of the whole
  * buffer are replaced by (A - mean) / (std + 1e-8) with the unbiased (M-1) standard
  * deviation.  dev_stats_out (may be NULL) receives {mean, std} of the raw advantages as
- * fp32 when normalize != 0.  fp32 arithmetic, fp64 accumulation of the moments. */
+ * fp32 when normalize != 0.  fp32 arithmetic, fp64 accumulation of the moments.
+ * normalize == 1 runs the scan and the normalisation as two launches; normalize == 2 runs both as one cooperative
+ * launch with a bounded grid barrier in between (the same arithmetic; the fp64 partial moments of more than 32 blocks
+ * are added in a different fixed order, which the rounding of mean and deviation to fp32 all but always hides;
+ * PPO_ERR_UNSUPPORTED when the scan's blocks, one per 128 envs, cannot all be resident at once). */
 int ppo_compute_gae(ppo_buffer *buf, const float *dev_last_value, float gamma, float lambda, int normalize,
                     float *dev_stats_out, void *stream);
 

@@ -224,8 +224,9 @@ def ppo_selftest_wait_timeout(limit_cycles: int, gave_up, stream=None):
            "ppo_selftest_wait_timeout")
 
 
-def ppo_compute_gae(buf: Buffer, last_value, gamma: float, lam: float, normalize: bool = True, stats_out=None,
+def ppo_compute_gae(buf: Buffer, last_value, gamma: float, lam: float, normalize=True, stats_out=None,
                     stream=None):
+    """normalize: False / True (two launches) / 2 (one cooperative launch)."""
     _check(lib().ppo_compute_gae(buf.handle, _ptr(last_value), gamma, lam, int(normalize), _ptr(stats_out),
                                  _stream(stream)), "ppo_compute_gae")
 

@@ -42,6 +42,7 @@ struct ppo_buffer {
     size_t field_off[PPO_NUM_FIELDS];
     bool gae_valid;
     int gae_blocks;  // partial sums held in the scratch slab
+    bool barrier_zeroed;  // the grid-barrier words at the end of the scratch slab have been cleared once
 };
 
 // Geometry of one stride-2 convolution (an FC layer is the 1x1 image, k = 1 case).

@@ -95,6 +95,13 @@ def test_gae_and_normalisation_match_oracle(N, T, done_rate):
         # run twice: the reduction order is fixed, so the result is bit-identical
         ppo.ppo_compute_gae(buf, lv, 0.99, 0.95, True, stats)
         assert np.array_equal(buf.field(ppo.FIELD_ADV).cpu().numpy(), advn)
+        # the single-launch variant (scan, grid barrier, normalisation) gives the same bits, twice in a row
+        for _ in range(2):
+            stats2 = torch.zeros(2, device=DEV)
+            ppo.ppo_compute_gae(buf, lv, 0.99, 0.95, 2, stats2)
+            assert np.array_equal(buf.field(ppo.FIELD_ADV).cpu().numpy(), advn)
+            assert np.array_equal(buf.field(ppo.FIELD_RET).cpu().numpy(), ret)
+            assert torch.equal(stats2, stats)
     assert ppo.ppo_poll_status() == 0
 
 
