@@ -152,7 +152,9 @@ int ppo_compute_gae(ppo_buffer *buf, const float *dev_last_value, float gamma, f
  *  - at most PPO_GAE_STATIC_MAX_ENVS envs (N); more returns PPO_ERR_UNSUPPORTED and launches nothing.
  *    The scratch is 64 KiB and every GPU that loads the library holds it until the process exits.
  *  - the first call on each device looks up the scratch array's device address (with that device
- *    current); make that first call outside any stream capture.
+ *    current); make that first call outside any stream capture.  If the library's code has not been
+ *    loaded onto the device yet, that first call also makes the CUDA runtime load it, which may
+ *    allocate and synchronise inside the driver; later calls do neither.
  *  - all calls on a device share the one scratch array, and it keeps whatever the last call left in
  *    it.  Each call overwrites every entry it later reads, so nothing needs clearing, but two calls
  *    whose kernels can overlap on the GPU (different streams, no dependency) race on it: serialise them.

@@ -67,6 +67,9 @@ WORKLOADS: Dict[str, Workload] = {
                           norm=True, embed=32),
     # profiling-sized twin of cfg2: same frames, network and micro-batch shapes, 1/8 of the envs
     "cfg2_prof": Workload("cfg2_prof", 128, 16, 120, 160, (32, 64, 128, 256), (3, 3, 3, 3), (512, 512), 1, 4),
+    # profiling-sized twin of cfg4: same frames and network, 64 envs (minibatches of 128 rows)
+    "cfg4_prof": Workload("cfg4_prof", 64, 16, 240, 320, (32, 64, 128, 256, 256), (5, 3, 3, 3, 3), (512, 512), 1, 8,
+                          done_rate=0.005),
     "cfg5_1k": Workload("cfg5_1k", 1024, 32, 120, 160, (32, 64, 128, 256), (3, 3, 3, 3), (512, 512), 1, 4),
     "cfg5_4k": Workload("cfg5_4k", 4096, 32, 120, 160, (32, 64, 128, 256), (3, 3, 3, 3), (512, 512), 1, 4),
     "cfg5_16k": Workload("cfg5_16k", 16384, 32, 120, 160, (32, 64, 128, 256), (3, 3, 3, 3), (512, 512), 1, 4),
