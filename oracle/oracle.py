@@ -26,6 +26,7 @@ class _Model(C.Structure):
         ("conv_c", C.c_int32 * 8), ("conv_k", C.c_int32 * 8),
         ("n_fc", C.c_int32), ("fc", C.c_int32 * 4),
         ("P", C.c_int32), ("A", C.c_int32), ("norm", C.c_int32), ("embed", C.c_int32),
+        ("n_lstm", C.c_int32), ("lstm_h", C.c_int32),
     ]
 
 
@@ -74,11 +75,14 @@ class ModelDesc:
     A: int = 12
     norm: bool = False   # layer normalisation over the channels of every conv output, before its ReLU
     embed: int = 0       # > 0: flatten -> FC(embed) -> ReLU instead of the global average pool
+    n_lstm: int = 0      # stacked LSTM layers between h_0 and the fully connected layers
+    lstm_h: int = 0      # their width
 
     def c(self) -> _Model:
         m = _Model()
         m.H, m.W, m.n_conv, m.n_fc, m.P, m.A = self.H, self.W, len(self.conv_c), len(self.fc), self.P, self.A
         m.norm, m.embed = int(self.norm), int(self.embed)
+        m.n_lstm, m.lstm_h = int(self.n_lstm), int(self.lstm_h)
         for i, v in enumerate(self.conv_c):
             m.conv_c[i] = v
         for i, v in enumerate(self.conv_k):
@@ -102,7 +106,7 @@ def depth_bytes(N, T, H, W, elem) -> int:
 
 
 def param_layout(md: ModelDesc) -> Layout:
-    n_max = 4 * 8 + 2 * 4 + 5
+    n_max = 4 * 8 + 2 * 4 + 3 * 4 + 5
     offs = (C.c_int64 * n_max)()
     szs = (C.c_int64 * n_max)()
     mat = (C.c_int32 * n_max)()
@@ -122,6 +126,9 @@ def param_layout(md: ModelDesc) -> Layout:
         ho, wo = conv_shapes(md)
         lay.shapes += [(md.embed, ho[-1] * wo[-1] * cin), (md.embed,)]
         i = md.embed + md.P
+    for _ in range(md.n_lstm):
+        lay.shapes += [(4 * md.lstm_h, i), (4 * md.lstm_h, md.lstm_h), (4 * md.lstm_h,)]
+        i = md.lstm_h
     for o in md.fc:
         lay.shapes += [(o, i), (o,)]
         i = o
@@ -312,3 +319,57 @@ def render_depth(H: int, W: int, hfov: float, near: float, far: float, plane, pr
     lib().orc_render_depth(C.c_int(N), C.c_int(H), C.c_int(W), C.c_double(hfov), C.c_double(near), C.c_double(far),
                            _p(plane), C.c_int(K), _p(prims), _p(out))
     return out
+
+
+# ------------------------------------------------------ recurrent trunk ----
+
+def lstm_rec_len(md: ModelDesc) -> int:
+    lib().orc_lstm_rec_len.restype = C.c_int64
+    m = md.c()
+    return int(lib().orc_lstm_rec_len(C.byref(m)))
+
+
+def encoder_fwd_seq(md: ModelDesc, theta_used, depth, proprio, done, h_init, c_init, act_bf16: bool = False):
+    """Sequence minibatch, rows time-major: depth [T,Be,H,W], proprio [T,Be,P], done uint8 [T,Be], h_init / c_init
+    [n_lstm,Be,lstm_h] -> mu [T*Be,A], V [T*Be], acts, lrec (the trunk's per-row record, kept for the backward)."""
+    T, Be = done.shape
+    depth = _f64(depth).reshape(T * Be, md.H, md.W)
+    proprio = _f64(proprio).reshape(T * Be, md.P)
+    done = np.ascontiguousarray(done, dtype=np.uint8)
+    h_init, c_init, theta_used = _f64(h_init), _f64(c_init), _f64(theta_used)
+    R = T * Be
+    acts = np.zeros((R, act_stride(md)), np.float64)
+    lrec = np.zeros((R, lstm_rec_len(md)), np.float64)
+    mu = np.empty((R, md.A), np.float64)
+    V = np.empty((R,), np.float64)
+    m = md.c()
+    lib().orc_encoder_fwd_seq(C.byref(m), _p(theta_used), C.c_int(T), C.c_int(Be), _p(depth), _p(proprio), _p(done),
+                              _p(h_init), _p(c_init), _p(acts), _p(lrec), _p(mu), _p(V), C.c_int(int(act_bf16)))
+    return mu, V, acts, lrec
+
+
+def encoder_bwd_seq(md: ModelDesc, theta_used, done, acts, lrec, dmu, dV, grad=None) -> np.ndarray:
+    T, Be = done.shape
+    done = np.ascontiguousarray(done, dtype=np.uint8)
+    theta_used, dmu, dV = _f64(theta_used), _f64(dmu), _f64(dV)
+    if grad is None:
+        grad = np.zeros_like(theta_used)
+    m = md.c()
+    lib().orc_encoder_bwd_seq(C.byref(m), _p(theta_used), C.c_int(T), C.c_int(Be), _p(done), _p(acts), _p(lrec),
+                              _p(dmu), _p(dV), _p(grad))
+    return grad
+
+
+def total_loss_and_grad_seq(md: ModelDesc, theta, depth, proprio, done, h_init, c_init, action, logp_old, adv, ret,
+                            clip, c_v, c_e, act_bf16: bool = False):
+    """One sequence minibatch (rows time-major, T*Be of them): as total_loss_and_grad, through the recurrent trunk."""
+    lay = param_layout(md)
+    theta = _f64(theta)
+    used = round_weights(md, theta)
+    logsigma = theta[lay.offsets[-1]: lay.offsets[-1] + md.A]
+    mu, V, acts, lrec = encoder_fwd_seq(md, used, depth, proprio, done, h_init, c_init, act_bf16)
+    out, dmu, dV, dls = loss(mu, V, logsigma, action, logp_old, adv, ret, clip, c_v, c_e)
+    grad = encoder_bwd_seq(md, used, done, acts, lrec, dmu, dV)
+    grad[lay.offsets[-1]: lay.offsets[-1] + md.A] += dls
+    L = out[0] + c_v * out[1] - c_e * out[2]
+    return L, out, grad, mu, V

@@ -59,9 +59,14 @@ typedef struct {
      *   embed > 0 : the last conv output is flattened (pixel-major, channel innermost) and mapped by a fully
      *               connected layer with ReLU to `embed` values, which take the place of the pooled vector. */
     int32_t norm, embed;
+    /* The recurrent trunk of Section III-C ("fed into two LSTM layers with 1024 units, the output of which is fed
+     * into a 3 layer fully-connected network"): n_lstm stacked LSTM layers of lstm_h units between h_0 (the depth
+     * feature joined with proprioception) and the fully connected layers; 0 layers for the feed-forward networks. */
+    int32_t n_lstm, lstm_h;
 } orc_model;
 
-#define ORC_MAX_TENSORS (4 * ORC_MAX_CONV + 2 * ORC_MAX_FC + 5)
+#define ORC_MAX_LSTM 4
+#define ORC_MAX_TENSORS (4 * ORC_MAX_CONV + 2 * ORC_MAX_FC + 3 * ORC_MAX_LSTM + 5)
 #define ORC_LN_EPS 1e-5
 
 int orc_num_threads(void) {
@@ -237,6 +242,13 @@ int64_t orc_param_layout(const orc_model *m, int64_t *offsets, int64_t *sizes, i
         PUSH(m->embed, 0);
         in = m->embed + m->P;
     }
+    /* LSTM layer: W_x [4H][in], W_h [4H][H] (gate blocks in the order input, forget, cell, output), b [4H] */
+    for (int l = 0; l < m->n_lstm; ++l) {
+        PUSH((int64_t)4 * m->lstm_h * in, 1);
+        PUSH((int64_t)4 * m->lstm_h * m->lstm_h, 1);
+        PUSH((int64_t)4 * m->lstm_h, 0);
+        in = m->lstm_h;
+    }
     for (int l = 0; l < m->n_fc; ++l) {
         PUSH((int64_t)m->fc[l] * in, 1);
         PUSH(m->fc[l], 0);
@@ -294,10 +306,43 @@ int64_t orc_act_stride(const orc_model *m) {
  *   h_l = ReLU(W_l h_{l-1} + b_l);  out = W_head h_F + b_head; mu = out[0..A), V = out[A].
  * With act_bf16 != 0 every conv output, h_0 and every hidden h_l is rounded to bf16 where it
  * is stored (the next layer's operand); the head output is not rounded. */
+/* phase 0: the whole feed-forward network.  With a recurrent trunk the sample is processed in two phases around
+ * it: phase 1 stops after h_0; phase 2 runs the fully connected layers and the head on `trunk_out` (the top LSTM
+ * layer's output for this sample, lstm_h values) and stores h_1.. behind h_0 as usual. */
 static void fwd_one(const orc_model *m, const double *th, const int64_t *offs, const double *depth,
-                    const double *proprio, double *act, double *mu, double *V, int act_bf16) {
+                    const double *proprio, double *act, double *mu, double *V, int act_bf16, int phase,
+                    const double *trunk_out) {
     int32_t Ho[ORC_MAX_CONV], Wo[ORC_MAX_CONV];
     orc_conv_shapes(m, Ho, Wo);
+    if (phase == 2) {
+        int ti = 2 * m->n_conv + (m->norm ? 2 * m->n_conv : 0) + (m->embed > 0 ? 2 : 0) + 3 * m->n_lstm;
+        int h0w = (m->embed > 0 ? m->embed : m->conv_c[m->n_conv - 1]) + m->P;
+        double *y = act + act_main_len(m);
+        for (int l = 0; l < m->n_fc; ++l) y -= m->fc[l]; /* h_1 sits right behind h_0 */
+        (void)h0w;
+        const double *h = trunk_out;
+        int in = m->lstm_h;
+        for (int l = 0; l < m->n_fc; ++l) {
+            const double *Wt = th + offs[ti], *b = th + offs[ti + 1];
+            ti += 2;
+            for (int o = 0; o < m->fc[l]; ++o) {
+                double acc = b[o];
+                for (int i = 0; i < in; ++i) acc += Wt[(int64_t)o * in + i] * h[i];
+                acc = acc > 0.0 ? acc : 0.0;
+                y[o] = act_bf16 ? orc_round_bf16(acc) : acc;
+            }
+            h = y;
+            in = m->fc[l];
+            y += m->fc[l];
+        }
+        const double *Wh = th + offs[ti], *bh = th + offs[ti + 1];
+        for (int o = 0; o <= m->A; ++o) {
+            double acc = bh[o];
+            for (int i = 0; i < in; ++i) acc += Wh[(int64_t)o * in + i] * h[i];
+            if (o < m->A) mu[o] = acc; else *V = acc;
+        }
+        return;
+    }
     double *x = act;
     double *extra = act + act_main_len(m); /* xhat_l, rstd_l of the normalised layers */
     for (int64_t i = 0; i < (int64_t)m->H * m->W; ++i) x[i] = depth[i];
@@ -385,6 +430,7 @@ static void fwd_one(const orc_model *m, const double *th, const int64_t *offs, c
         }
     }
     for (int j = 0; j < m->P; ++j) h[feat + j] = act_bf16 ? orc_round_bf16(proprio[j]) : proprio[j];
+    if (phase == 1) return;
     int in = feat + m->P;
     for (int l = 0; l < m->n_fc; ++l) {
         const double *Wt = th + offs[ti], *b = th + offs[ti + 1];
@@ -411,8 +457,13 @@ static void fwd_one(const orc_model *m, const double *th, const int64_t *offs, c
  * (same layout as the parameter vector).  ReLU' = 1 where the stored output is
  * > 0 (equivalently the pre-activation is > 0), else 0.  The log-sigma slot of g
  * is not touched here (it has no path through the network). */
+/* phase 0: the whole feed-forward network.  Around a recurrent trunk: phase 2 goes from the head down through the
+ * fully connected layers, whose first input was `trunk_out`, and leaves dL/d(trunk_out) in d_trunk [lstm_h];
+ * phase 1 starts from d_trunk = dL/dh_0 [width of h_0] and goes down through the pooling or embedding and the
+ * convolutions. */
 static void bwd_one(const orc_model *m, const double *th, const int64_t *offs, int n_tensors, const double *act,
-                    const double *dmu, double dV, double *g, double *scratch) {
+                    const double *dmu, double dV, double *g, double *scratch, int phase, const double *trunk_out,
+                    double *d_trunk) {
     int32_t Ho[ORC_MAX_CONV], Wo[ORC_MAX_CONV];
     orc_conv_shapes(m, Ho, Wo);
     /* locate activations */
@@ -439,16 +490,26 @@ static void bwd_one(const orc_model *m, const double *th, const int64_t *offs, i
         }
     }
     for (int l = 0; l < F; ++l) { hv[l + 1] = hv[l] + hn[l]; hn[l + 1] = m->fc[l]; }
+    const int h0w = hn[0];
+    if (phase == 2) { /* the fully connected layers read the trunk's output, not h_0 */
+        hv[0] = trunk_out;
+        hn[0] = m->lstm_h;
+    }
 
     /* scratch: two ping-pong gradient buffers large enough for any activation */
     int64_t big = (int64_t)m->H * m->W;
     for (int l = 1; l <= L; ++l) { int64_t s = (int64_t)hs[l] * ws[l] * cs[l]; if (s > big) big = s; }
     for (int l = 0; l <= F; ++l) if (hn[l] > big) big = hn[l];
+    if (h0w > big) big = h0w;
     double *d_cur = scratch, *d_prev = scratch + big;
 
     /* head */
     int ti = n_tensors - 3; /* head W, head b, log-sigma */
-    {
+    if (phase == 1) {
+        for (int i = 0; i < h0w; ++i) d_cur[i] = d_trunk[i];
+        ti -= 2 * F + 3 * m->n_lstm; /* past the fully connected and the LSTM tensors */
+    }
+    if (phase != 1) {
         const double *Wh = th + offs[ti];
         double *gW = g + offs[ti], *gb = g + offs[ti + 1];
         int in = hn[F];
@@ -463,7 +524,7 @@ static void bwd_one(const orc_model *m, const double *th, const int64_t *offs, i
         }
     }
     /* hidden fc layers, last to first; d_cur holds dL/dh_l (post-ReLU) */
-    for (int l = F; l >= 1; --l) {
+    for (int l = F; l >= 1 && phase != 1; --l) {
         ti -= 2;
         const double *Wt = th + offs[ti];
         double *gW = g + offs[ti], *gb = g + offs[ti + 1];
@@ -478,6 +539,10 @@ static void bwd_one(const orc_model *m, const double *th, const int64_t *offs, i
             }
         }
         double *tmp = d_cur; d_cur = d_prev; d_prev = tmp;
+    }
+    if (phase == 2) {
+        for (int i = 0; i < m->lstm_h; ++i) d_trunk[i] = d_cur[i];
+        return;
     }
     /* un-pool: every pixel of the last conv output gets dg[c] / (Ho*Wo); the proprio part ends here.
      * With embed > 0: back through ReLU and the fully connected embedding into the flattened conv output. */
@@ -573,6 +638,7 @@ int64_t orc_bwd_scratch_len(const orc_model *m) {
     for (int l = 0; l < m->n_conv; ++l) { int64_t s = (int64_t)Ho[l] * Wo[l] * m->conv_c[l]; if (s > big) big = s; }
     int64_t h0 = (m->embed > 0 ? m->embed : m->conv_c[m->n_conv - 1]) + m->P;
     if (h0 > big) big = h0;
+    if (m->n_lstm > 0 && m->lstm_h > big) big = m->lstm_h;
     for (int l = 0; l < m->n_fc; ++l) if (m->fc[l] > big) big = m->fc[l];
     return 2 * big;
 }
@@ -588,7 +654,7 @@ void orc_encoder_fwd(const orc_model *m, const double *theta_used, int B, const 
 #pragma omp parallel for schedule(dynamic)
     for (int b = 0; b < B; ++b)
         fwd_one(m, theta_used, offs, depth + (int64_t)b * m->H * m->W, proprio + (int64_t)b * m->P,
-                acts + b * stride, mu + (int64_t)b * m->A, V + b, act_bf16);
+                acts + b * stride, mu + (int64_t)b * m->A, V + b, act_bf16, 0, NULL);
 }
 
 /* Backward of B samples: grad (length = parameter vector) += sum over samples of the
@@ -606,7 +672,8 @@ void orc_encoder_bwd(const orc_model *m, const double *theta_used, int B, const 
         double *scratch = (double *)malloc((size_t)slen * sizeof(double));
 #pragma omp for schedule(dynamic)
         for (int b = 0; b < B; ++b)
-            bwd_one(m, theta_used, offs, n, acts + b * stride, dmu + (int64_t)b * m->A, dV[b], g_local, scratch);
+            bwd_one(m, theta_used, offs, n, acts + b * stride, dmu + (int64_t)b * m->A, dV[b], g_local, scratch, 0, NULL,
+                    NULL);
 #pragma omp critical
         for (int64_t i = 0; i < total; ++i) grad[i] += g_local[i];
         free(g_local);
@@ -828,3 +895,177 @@ void orc_render_depth(int N, int H, int W, double hfov, double near, double far,
 }
 
 double orc_round_fp16(double x) { return round_fp16(x); }
+
+/* ------------------------------------------------------- recurrent trunk -- */
+
+/* Length of the per-row record of the recurrent trunk: for every LSTM layer the gate activations i, f, g, o
+ * (4H), the cell state c (H), the output h (H) and the state the step started from, h_prev (H) and c_prev (H). */
+int64_t orc_lstm_rec_len(const orc_model *m) { return (int64_t)m->n_lstm * 8 * m->lstm_h; }
+
+static double sigmoid(double x) { return 1.0 / (1.0 + exp(-x)); }
+
+/* Forward over a minibatch of sequences (Section III-C: CNN embedding joined with proprioception -> LSTM layers ->
+ * fully connected layers -> heads).  Rows are time-major: row r = t * Be + e is env e of the minibatch at step t.
+ * Per LSTM layer, with x_t the layer's input (h_0 of the row, or the output of the layer below):
+ *   (i, f, g, o) = (sigmoid, sigmoid, tanh, sigmoid)(W_x x_t + W_h h_prev + b),   c_t = f c_prev + i g,
+ *   h_t = o tanh(c_t),
+ * the state a step starts from being the caller's (h_init, c_init) [L][Be][H] at t = 0 and afterwards the previous
+ * step's (h, c), zeroed where done[t-1][e] != 0 (the episode ended: Algorithm 2 stores done with the step that
+ * returned it).  With act_bf16 the stored h (the operand of the next contractions) is rounded to bf16; c is not.
+ * acts [R][orc_act_stride] and lrec [R][orc_lstm_rec_len] are kept for the backward pass. */
+void orc_encoder_fwd_seq(const orc_model *m, const double *theta_used, int T, int Be, const double *depth,
+                         const double *proprio, const uint8_t *done, const double *h_init, const double *c_init,
+                         double *acts, double *lrec, double *mu, double *V, int act_bf16) {
+    int64_t offs[ORC_MAX_TENSORS], szs[ORC_MAX_TENSORS];
+    int32_t mat[ORC_MAX_TENSORS], n;
+    orc_param_layout(m, offs, szs, mat, &n);
+    const int64_t stride = orc_act_stride(m), lstride = orc_lstm_rec_len(m);
+    const int R = T * Be, H = m->lstm_h, L = m->n_lstm;
+    const int h0w = (m->embed > 0 ? m->embed : m->conv_c[m->n_conv - 1]) + m->P;
+    int64_t h0_off = act_main_len(m) - h0w;
+    for (int l = 0; l < m->n_fc; ++l) h0_off -= m->fc[l];
+#pragma omp parallel for schedule(dynamic)
+    for (int r = 0; r < R; ++r)
+        fwd_one(m, theta_used, offs, depth + (int64_t)r * m->H * m->W, proprio + (int64_t)r * m->P, acts + r * stride,
+                NULL, NULL, act_bf16, 1, NULL);
+    const int ti0 = 2 * m->n_conv + (m->norm ? 2 * m->n_conv : 0) + (m->embed > 0 ? 2 : 0);
+    for (int l = 0; l < L; ++l) {
+        const int in = l == 0 ? h0w : H;
+        const double *Wx = theta_used + offs[ti0 + 3 * l], *Wh = theta_used + offs[ti0 + 3 * l + 1];
+        const double *b = theta_used + offs[ti0 + 3 * l + 2];
+        for (int t = 0; t < T; ++t) {
+#pragma omp parallel for schedule(static)
+            for (int e = 0; e < Be; ++e) {
+                const int r = t * Be + e;
+                double *rec = lrec + r * lstride + (int64_t)l * 8 * H;
+                double *gi = rec, *gf = rec + H, *gg = rec + 2 * H, *go = rec + 3 * H;
+                double *c = rec + 4 * H, *h = rec + 5 * H, *hp = rec + 6 * H, *cp = rec + 7 * H;
+                const double *x = l == 0 ? acts + r * stride + h0_off : lrec + r * lstride + (int64_t)(l - 1) * 8 * H + 5 * H;
+                if (t == 0) {
+                    for (int j = 0; j < H; ++j) {
+                        hp[j] = h_init[((int64_t)l * Be + e) * H + j];
+                        cp[j] = c_init[((int64_t)l * Be + e) * H + j];
+                    }
+                } else {
+                    const double *prev = lrec + (int64_t)(r - Be) * lstride + (int64_t)l * 8 * H;
+                    const double keep = done[(t - 1) * Be + e] ? 0.0 : 1.0;
+                    for (int j = 0; j < H; ++j) {
+                        hp[j] = keep * prev[5 * H + j];
+                        cp[j] = keep * prev[4 * H + j];
+                    }
+                }
+                for (int j = 0; j < 4 * H; ++j) {
+                    double acc = b[j];
+                    for (int k = 0; k < in; ++k) acc += Wx[(int64_t)j * in + k] * x[k];
+                    for (int k = 0; k < H; ++k) acc += Wh[(int64_t)j * H + k] * hp[k];
+                    rec[j] = (j >= 2 * H && j < 3 * H) ? tanh(acc) : sigmoid(acc);
+                }
+                for (int j = 0; j < H; ++j) {
+                    c[j] = gf[j] * cp[j] + gi[j] * gg[j];
+                    const double hv = go[j] * tanh(c[j]);
+                    h[j] = act_bf16 ? orc_round_bf16(hv) : hv;
+                }
+            }
+        }
+    }
+#pragma omp parallel for schedule(dynamic)
+    for (int r = 0; r < R; ++r)
+        fwd_one(m, theta_used, offs, NULL, NULL, acts + r * stride, mu + (int64_t)r * m->A, V + r, act_bf16, 2,
+                lrec + r * lstride + (int64_t)(L - 1) * 8 * H + 5 * H);
+}
+
+/* Backward through orc_encoder_fwd_seq (back-propagation through time over the T steps of the minibatch; the
+ * initial states are constants).  grad += dL/dtheta. */
+void orc_encoder_bwd_seq(const orc_model *m, const double *theta_used, int T, int Be, const uint8_t *done,
+                         const double *acts, const double *lrec, const double *dmu, const double *dV, double *grad) {
+    int64_t offs[ORC_MAX_TENSORS], szs[ORC_MAX_TENSORS];
+    int32_t mat[ORC_MAX_TENSORS], n;
+    const int64_t total = orc_param_layout(m, offs, szs, mat, &n);
+    const int64_t stride = orc_act_stride(m), lstride = orc_lstm_rec_len(m), slen = orc_bwd_scratch_len(m);
+    const int R = T * Be, H = m->lstm_h, L = m->n_lstm;
+    const int h0w = (m->embed > 0 ? m->embed : m->conv_c[m->n_conv - 1]) + m->P;
+    int64_t h0_off = act_main_len(m) - h0w;
+    for (int l = 0; l < m->n_fc; ++l) h0_off -= m->fc[l];
+    const int wmax = H > h0w ? H : h0w;
+    double *dx = (double *)calloc((size_t)R * wmax, sizeof(double));   /* gradient w.r.t. a layer's output rows */
+    double *dxl = (double *)calloc((size_t)R * wmax, sizeof(double));  /* gradient w.r.t. the layer's input rows */
+    /* fully connected layers and head, row by row */
+#pragma omp parallel
+    {
+        double *g_local = (double *)calloc((size_t)total, sizeof(double));
+        double *scratch = (double *)malloc((size_t)slen * sizeof(double));
+#pragma omp for schedule(dynamic)
+        for (int r = 0; r < R; ++r)
+            bwd_one(m, theta_used, offs, n, acts + r * stride, dmu + (int64_t)r * m->A, dV[r], g_local, scratch, 2,
+                    lrec + r * lstride + (int64_t)(L - 1) * 8 * H + 5 * H, dx + (int64_t)r * wmax);
+#pragma omp critical
+        for (int64_t i = 0; i < total; ++i) grad[i] += g_local[i];
+        free(g_local);
+        free(scratch);
+    }
+    const int ti0 = 2 * m->n_conv + (m->norm ? 2 * m->n_conv : 0) + (m->embed > 0 ? 2 : 0);
+    double *dh_carry = (double *)malloc((size_t)Be * H * sizeof(double));
+    double *dc_carry = (double *)malloc((size_t)Be * H * sizeof(double));
+    double *dgate = (double *)malloc((size_t)4 * H * sizeof(double));
+    for (int l = L - 1; l >= 0; --l) {
+        const int in = l == 0 ? h0w : H;
+        const double *Wx = theta_used + offs[ti0 + 3 * l], *Wh = theta_used + offs[ti0 + 3 * l + 1];
+        double *gWx = grad + offs[ti0 + 3 * l], *gWh = grad + offs[ti0 + 3 * l + 1], *gb = grad + offs[ti0 + 3 * l + 2];
+        for (int64_t i = 0; i < (int64_t)Be * H; ++i) dh_carry[i] = dc_carry[i] = 0.0;
+        for (int64_t i = 0; i < (int64_t)R * wmax; ++i) dxl[i] = 0.0;
+        for (int t = T - 1; t >= 0; --t)
+            for (int e = 0; e < Be; ++e) {
+                const int r = t * Be + e;
+                const double *rec = lrec + r * lstride + (int64_t)l * 8 * H;
+                const double *gi = rec, *gf = rec + H, *gg = rec + 2 * H, *go = rec + 3 * H;
+                const double *c = rec + 4 * H, *hp = rec + 6 * H, *cp = rec + 7 * H;
+                const double *x = l == 0 ? acts + r * stride + h0_off : lrec + r * lstride + (int64_t)(l - 1) * 8 * H + 5 * H;
+                double *dhc = dh_carry + (int64_t)e * H, *dcc = dc_carry + (int64_t)e * H;
+                for (int j = 0; j < H; ++j) {
+                    const double dh = dx[(int64_t)r * wmax + j] + dhc[j];
+                    const double tc = tanh(c[j]);
+                    const double dc = dcc[j] + dh * go[j] * (1.0 - tc * tc);
+                    dgate[j] = dc * gg[j] * gi[j] * (1.0 - gi[j]);             /* input gate, pre-activation */
+                    dgate[H + j] = dc * cp[j] * gf[j] * (1.0 - gf[j]);         /* forget gate */
+                    dgate[2 * H + j] = dc * gi[j] * (1.0 - gg[j] * gg[j]);     /* cell candidate */
+                    dgate[3 * H + j] = dh * tc * go[j] * (1.0 - go[j]);        /* output gate */
+                    dcc[j] = dc * gf[j];                                       /* into c_prev */
+                }
+                for (int j = 0; j < H; ++j) dhc[j] = 0.0;
+                double *dxr = dxl + (int64_t)r * wmax;
+                for (int j = 0; j < 4 * H; ++j) {
+                    const double d = dgate[j];
+                    gb[j] += d;
+                    for (int k = 0; k < in; ++k) {
+                        gWx[(int64_t)j * in + k] += d * x[k];
+                        dxr[k] += Wx[(int64_t)j * in + k] * d;
+                    }
+                    for (int k = 0; k < H; ++k) {
+                        gWh[(int64_t)j * H + k] += d * hp[k];
+                        dhc[k] += Wh[(int64_t)j * H + k] * d;
+                    }
+                }
+                /* the state this step started from was the previous step's, zeroed after a done */
+                const double keep = (t > 0 && !done[(t - 1) * Be + e]) ? 1.0 : 0.0;
+                for (int j = 0; j < H; ++j) {
+                    dhc[j] *= keep;
+                    dcc[j] *= keep;
+                }
+            }
+        double *tmp = dx; dx = dxl; dxl = tmp;
+    }
+    /* h_0 and below, row by row */
+#pragma omp parallel
+    {
+        double *g_local = (double *)calloc((size_t)total, sizeof(double));
+        double *scratch = (double *)malloc((size_t)slen * sizeof(double));
+#pragma omp for schedule(dynamic)
+        for (int r = 0; r < R; ++r)
+            bwd_one(m, theta_used, offs, n, acts + r * stride, NULL, 0.0, g_local, scratch, 1, NULL, dx + (int64_t)r * wmax);
+#pragma omp critical
+        for (int64_t i = 0; i < total; ++i) grad[i] += g_local[i];
+        free(g_local);
+        free(scratch);
+    }
+    free(dx); free(dxl); free(dh_carry); free(dc_carry); free(dgate);
+}
