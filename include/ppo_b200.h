@@ -193,7 +193,8 @@ int ppo_shuffle_gather_minibatch(const ppo_buffer *buf, uint64_t seed, uint32_t 
 
 #define PPO_MAX_CONV 8
 #define PPO_MAX_FC 4
-#define PPO_MAX_TENSORS (4 * PPO_MAX_CONV + 2 * PPO_MAX_FC + 5)
+#define PPO_MAX_LSTM 4
+#define PPO_MAX_TENSORS (4 * PPO_MAX_CONV + 2 * PPO_MAX_FC + 3 * PPO_MAX_LSTM + 5)
 
 /* Policy/value network (Section III-C: CNN with ReLU on the depth image, joined with
  * proprioception, fully connected layers).  Conv l: k x k cross-correlation, stride 2,
@@ -210,7 +211,14 @@ int ppo_shuffle_gather_minibatch(const ppo_buffer *buf, uint64_t seed, uint32_t 
  *               conv_c <= 256 and an even frame width.
  *   embed > 0 : instead of the global average pool, the last conv output is flattened (pixel-major, channel
  *               innermost) and mapped by a fully connected layer with ReLU to `embed` values (a multiple of 32,
- *               embed + P a multiple of 8), which are concatenated with proprio. */
+ *               embed + P a multiple of 8), which are concatenated with proprio.
+ *
+ * The recurrent trunk of Section III-C ("two LSTM layers with 1024 units" between that joined feature and the fully
+ * connected layers) is selected by n_lstm > 0 (up to 4 layers of lstm_h units, lstm_h a multiple of 64):
+ *   (i, f, g, o) = (sigmoid, sigmoid, tanh, sigmoid)(W_x x_t + W_h h_prev + b),  c_t = f c_prev + i g,  h_t = o tanh(c_t)
+ * per layer and time step.  Such a model works on sequence minibatches (ppo_shuffle_gather_sequences) whose rows are
+ * time-major, row = t * Be + e, announced with ppo_model_set_sequence; ppo_encoder_fwd / ppo_encoder_bwd then take
+ * the whole minibatch (rows == T * Be), the backward pass being back-propagation through the T steps. */
 typedef struct {
     int32_t H, W;
     int32_t n_conv;
@@ -220,6 +228,7 @@ typedef struct {
     int32_t fc[PPO_MAX_FC];
     int32_t P, A;
     int32_t norm, embed;
+    int32_t n_lstm, lstm_h;
 } ppo_model_desc;
 
 typedef struct ppo_model ppo_model;
@@ -229,7 +238,8 @@ int ppo_model_destroy(ppo_model *m);
 
 /* Parameter vector ("arena") layout: tensors in the order conv W_l [Cout][k][k][Cin],
  * conv b_l [Cout] (with norm: followed by gamma_l [Cout], beta_l [Cout]), ..., (with embed: embed W
- * [E][Ho*Wo*C_L], embed b [E],) fc W [out][in], fc b [out], ..., head W [A+1][hid] (rows 0..A-1
+ * [E][Ho*Wo*C_L], embed b [E],) (per LSTM layer: W_x [4H][in], W_h [4H][H], b [4H], gate blocks in the order input,
+ * forget, cell, output,) fc W [out][in], fc b [out], ..., head W [A+1][hid] (rows 0..A-1
  * mean, row A value), head b [A+1], log-sigma [A]; every tensor starts at a multiple of 64
  * elements; gaps are zero and stay zero.  The same offsets index master, shadow, gradient
  * and Adam moment arrays. */
@@ -247,6 +257,14 @@ size_t ppo_model_workspace_bytes(const ppo_model *m, int microbatch);
  * ppo_model_workspace_bytes(m, microbatch). */
 int ppo_model_bind(ppo_model *m, float *dev_master, void *dev_shadow_bf16, float *dev_grad, float *dev_adam_m,
                    float *dev_adam_v, void *dev_workspace, size_t ws_bytes, int microbatch);
+
+/* Describes the sequence minibatch the next ppo_encoder_fwd / ppo_encoder_bwd of a recurrent model work on: T time
+ * steps of Be envs, rows time-major; dev_done uint8 [T][Be] (the flags stored with the steps: a set flag zeroes the
+ * state the NEXT step starts from); dev_h_init, dev_c_init fp32 [n_lstm][Be][lstm_h], the state the first step starts
+ * from (constants of the backward pass).  The pointers are read by those calls, not copied.  T * Be must not
+ * exceed the bound micro-batch.  Errors: model without LSTM layers -> STATE; bad sizes -> SHAPE. */
+int ppo_model_set_sequence(ppo_model *m, int T, int Be, const uint8_t *dev_done, const float *dev_h_init,
+                           const float *dev_c_init);
 
 /* shadow <- bf16(master) (round to nearest even); call after writing master from outside. */
 int ppo_model_sync_shadow(ppo_model *m, void *stream);
@@ -288,7 +306,10 @@ int ppo_encoder_bwd(ppo_model *m, const ppo_minibatch *mb, int row0, int rows, c
  * for index in 0..n_fc, bf16 [rows][width] (h_0 = [pooled, proprio]); kind 2 = the ReLU gate bits of conv
  * activation `index` (only for layers below the last whose channel count is a multiple of 32, else INVALID_ARG),
  * uint32 [rows][Ho][Wo][C/32] (kind 3 and 4, with norm only: the normalised values xhat of conv layer `index`,
- * bf16 [rows][Ho][Wo][C], and their reciprocal standard deviations, fp32 [rows][Ho][Wo]); channel c belongs to word c / 32 and sits at bit ((c % 32) / 2) + 16 * (c % 2) of it (the
+ * bf16 [rows][Ho][Wo][C], and their reciprocal standard deviations, fp32 [rows][Ho][Wo]; kind 5, 6, 7, 8, with
+ * LSTM layers only, index = layer 0..n_lstm-1: the layer's outputs h bf16 [rows][lstm_h], its cell states c fp32
+ * [rows][lstm_h], its gate activations fp32 [rows][4 lstm_h], and the states its steps started from, h_prev bf16
+ * [rows][lstm_h] (c_prev fp32 [rows][lstm_h] follows the cell states: kind 6 has 2 rows lstm_h elements)); channel c belongs to word c / 32 and sits at bit ((c % 32) / 2) + 16 * (c % 2) of it (the
  * two halves of a packed pair of bf16 values own bits j and 16 + j), set where the activation is > 0.  *elems is the capacity
  * for the bound micro-batch.  For inspection and for tests that substitute the saved
  * activations between ppo_encoder_fwd and ppo_encoder_bwd. */
@@ -306,6 +327,15 @@ int ppo_model_zero_grad(ppo_model *m, void *stream);
  * weight decay), step >= 1:  m <- b1 m + (1-b1) g;  v <- b2 v + (1-b2) g^2;
  * theta <- theta - lr (m/(1-b1^step)) / (sqrt(v/(1-b2^step)) + eps); shadow <- bf16(theta). */
 int ppo_adam_step(ppo_model *m, float lr, float beta1, float beta2, float eps, int64_t step, void *stream);
+
+/* Sequence minibatch mb_index of num_minibatches for (seed, epoch), for recurrent policies (Section III-C: the LSTM
+ * needs every env's steps in order): the ENVS are permuted with the same seeded bijection, now on [0, N), and a
+ * minibatch holds Be = N / num_minibatches envs with all their T steps, rows time-major: row t * Be + e is an exact
+ * copy of sample t * N + pi(mb_index * Be + e).  out->B must be T * Be; dev_done_out uint8 [T][Be] receives the done
+ * flags of the rows; out->index (optional) the sample numbers.  Requires N % num_minibatches == 0 (else SHAPE) and a
+ * prior ppo_compute_gae (else STATE). */
+int ppo_shuffle_gather_sequences(const ppo_buffer *buf, uint64_t seed, uint32_t epoch, int mb_index, int num_minibatches,
+                                 const ppo_minibatch *out, uint8_t *dev_done_out, void *stream);
 
 /* Rollout-time action of the policy (Algorithm 2, actions <- pi(obs)) given the mean from
  * ppo_encoder_fwd and caller-supplied standard-normal noise dev_eps [rows][A]:

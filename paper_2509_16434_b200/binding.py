@@ -28,7 +28,7 @@ EXPORTS = [
     "ppo_model_sync_shadow", "ppo_encoder_fwd", "ppo_loss_fwd_bwd", "ppo_encoder_bwd", "ppo_model_zero_grad",
     "ppo_adam_step", "ppo_policy_sample", "ppo_poll_status", "ppo_model_activation_ptr", "ppo_gae_static",
     "ppo_model_sync_masks", "ppo_buffer_write_obs", "ppo_buffer_write_outcome", "ppo_policy_act", "ppo_launch_count",
-    "ppo_selftest_wait_timeout", "ppo_buffer_render_depth",
+    "ppo_selftest_wait_timeout", "ppo_buffer_render_depth", "ppo_model_set_sequence", "ppo_shuffle_gather_sequences",
 ]
 
 
@@ -45,7 +45,8 @@ class BufferDesc(C.Structure):
 class ModelDesc(C.Structure):
     _fields_ = [("H", C.c_int32), ("W", C.c_int32), ("n_conv", C.c_int32), ("conv_c", C.c_int32 * 8),
                 ("conv_k", C.c_int32 * 8), ("n_fc", C.c_int32), ("fc", C.c_int32 * 4), ("P", C.c_int32),
-                ("A", C.c_int32), ("norm", C.c_int32), ("embed", C.c_int32)]
+                ("A", C.c_int32), ("norm", C.c_int32), ("embed", C.c_int32), ("n_lstm", C.c_int32),
+                ("lstm_h", C.c_int32)]
 
 
 class Minibatch(C.Structure):
@@ -106,6 +107,9 @@ def lib():
         L.ppo_policy_act.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.c_void_p]
         L.ppo_buffer_render_depth.argtypes = [C.c_void_p, C.c_int, C.c_float, C.c_float, C.c_float, C.c_void_p, C.c_int,
                                               C.c_void_p, C.c_void_p]
+        L.ppo_model_set_sequence.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p]
+        L.ppo_shuffle_gather_sequences.argtypes = [C.c_void_p, C.c_uint64, C.c_uint32, C.c_int, C.c_int,
+                                                   C.POINTER(Minibatch), C.c_void_p, C.c_void_p]
         L.ppo_launch_count.restype = C.c_uint64
         L.ppo_launch_count.argtypes = []
         L.ppo_selftest_wait_timeout.argtypes = [C.c_longlong, C.c_void_p, C.c_void_p]
@@ -271,10 +275,10 @@ def ppo_shuffle_gather_minibatch(buf: Buffer, seed: int, epoch: int, mb_index: i
 
 
 def model_desc(H, W, conv_c: Sequence[int], conv_k: Sequence[int], fc: Sequence[int], P=32, A=12, norm=False,
-               embed=0) -> ModelDesc:
+               embed=0, n_lstm=0, lstm_h=0) -> ModelDesc:
     d = ModelDesc()
     d.H, d.W, d.n_conv, d.n_fc, d.P, d.A = H, W, len(conv_c), len(fc), P, A
-    d.norm, d.embed = int(norm), int(embed)
+    d.norm, d.embed, d.n_lstm, d.lstm_h = int(norm), int(embed), int(n_lstm), int(lstm_h)
     for i, v in enumerate(conv_c):
         d.conv_c[i] = v
     for i, v in enumerate(conv_k):
@@ -335,7 +339,7 @@ class Model:
         off = p.value - self.workspace.data_ptr()
         if kind == 2:
             return self.workspace[off:off + 4 * n.value].view(torch.int32)
-        if kind == 4:
+        if kind in (4, 6, 7):
             return self.workspace[off:off + 4 * n.value].view(torch.float32)
         return self.workspace[off:off + 2 * n.value].view(torch.bfloat16)
 
@@ -344,6 +348,17 @@ class Model:
         t = torch.as_tensor(theta, dtype=torch.float32)
         self.master.copy_(t.to(self.master.device))
         ppo_model_sync_shadow(self, stream)
+
+
+def ppo_model_set_sequence(m: Model, T: int, Be: int, done, h_init, c_init):
+    """done uint8 [T,Be], h_init / c_init fp32 [n_lstm,Be,lstm_h]: the tensors must stay alive until the backward pass."""
+    _check(lib().ppo_model_set_sequence(m.handle, T, Be, _ptr(done), _ptr(h_init), _ptr(c_init)), "ppo_model_set_sequence")
+
+
+def ppo_shuffle_gather_sequences(buf: Buffer, seed: int, epoch: int, mb_index: int, num_minibatches: int,
+                                 out: "MinibatchArrays", done_out, stream=None):
+    _check(lib().ppo_shuffle_gather_sequences(buf.handle, seed, epoch, mb_index, num_minibatches, C.byref(out.c),
+                                              _ptr(done_out), _stream(stream)), "ppo_shuffle_gather_sequences")
 
 
 def ppo_model_sync_shadow(m: Model, stream=None):

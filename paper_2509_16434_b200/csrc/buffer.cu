@@ -630,6 +630,11 @@ struct GatherArgs {
     uint32_t frame16;    // frame length in copy units (16 B, or 2 B for odd frame sizes)
     uint32_t chunks;     // CTAs per row
     int P, A;
+    // sequence minibatches: envs are permuted, not samples; row = t * seq_Be + e holds sample t * N + pi(start + e)
+    uint32_t seq_Be;     // 0: flat minibatch
+    uint32_t N;
+    const uint8_t *done;
+    uint8_t *o_done;
 };
 
 // One CTA copies one chunk of one row's depth frame with 128-bit loads (no L1 allocation,
@@ -639,7 +644,13 @@ template <typename VecT>
 __global__ void __launch_bounds__(256) gather_kernel(GatherArgs g, PermParams p) {
     const uint32_t row = blockIdx.x / g.chunks;
     const uint32_t chunk = blockIdx.x - row * g.chunks;
-    const uint32_t s = perm_apply(p, g.start + row);
+    uint32_t s;
+    if (g.seq_Be) {
+        const uint32_t t = row / g.seq_Be, e = row - t * g.seq_Be;
+        s = t * g.N + perm_apply(p, g.start + e);
+    } else {
+        s = perm_apply(p, g.start + row);
+    }
     const VecT *src = reinterpret_cast<const VecT *>(g.depth) + (size_t)s * g.frame16;
     VecT *dst = reinterpret_cast<VecT *>(g.o_depth) + (size_t)row * g.frame16;
     const uint32_t per = (g.frame16 + g.chunks - 1) / g.chunks;
@@ -663,16 +674,33 @@ __global__ void __launch_bounds__(256) gather_kernel(GatherArgs g, PermParams p)
         if (t == 130) g.o_adv[row] = g.adv[s];
         if (t == 131) g.o_ret[row] = g.ret[s];
         if (t == 132 && g.o_index) g.o_index[row] = s;
+        if (t == 133 && g.o_done) g.o_done[row] = g.done[s];
     }
 }
 
+static int gather_impl(const ppo_buffer *b, uint64_t seed, uint32_t epoch, int mb_index, int num_minibatches,
+                       const ppo_minibatch *out, uint8_t *done_out, bool sequences, void *stream);
+
 extern "C" int ppo_shuffle_gather_minibatch(const ppo_buffer *b, uint64_t seed, uint32_t epoch, int mb_index,
                                             int num_minibatches, const ppo_minibatch *out, void *stream) {
+    return gather_impl(b, seed, epoch, mb_index, num_minibatches, out, nullptr, false, stream);
+}
+
+extern "C" int ppo_shuffle_gather_sequences(const ppo_buffer *b, uint64_t seed, uint32_t epoch, int mb_index,
+                                            int num_minibatches, const ppo_minibatch *out, uint8_t *done_out, void *stream) {
+    if (!done_out) return PPO_ERR_INVALID_ARG;
+    return gather_impl(b, seed, epoch, mb_index, num_minibatches, out, done_out, true, stream);
+}
+
+static int gather_impl(const ppo_buffer *b, uint64_t seed, uint32_t epoch, int mb_index, int num_minibatches,
+                       const ppo_minibatch *out, uint8_t *done_out, bool sequences, void *stream) {
     if (!b || !out) return PPO_ERR_INVALID_ARG;
     if (num_minibatches <= 0 || mb_index < 0 || mb_index >= num_minibatches) return PPO_ERR_INVALID_ARG;
-    const long long M = (long long)b->d.N * b->d.T;
+    // what is permuted and cut into minibatches: the samples, or the envs (each with all its T steps)
+    const long long M = sequences ? (long long)b->d.N : (long long)b->d.N * b->d.T;
     if (M % num_minibatches != 0) return PPO_ERR_SHAPE;
-    const long long B = M / num_minibatches;
+    const long long per = M / num_minibatches;
+    const long long B = sequences ? per * b->d.T : per;
     if (out->B != B) return PPO_ERR_SHAPE;
     if (!out->depth_f16 || !out->proprio || !out->action || !out->logp_old || !out->value_old || !out->adv ||
         !out->ret)
@@ -698,8 +726,12 @@ extern "C" int ppo_shuffle_gather_minibatch(const ppo_buffer *b, uint64_t seed, 
     g.o_adv = out->adv;
     g.o_ret = out->ret;
     g.o_index = out->index;
-    g.start = (uint32_t)(mb_index * B);
+    g.start = (uint32_t)(mb_index * per);
     g.rows = (uint32_t)B;
+    g.seq_Be = sequences ? (uint32_t)per : 0u;
+    g.N = (uint32_t)b->d.N;
+    g.done = slab<uint8_t>(b, PPO_FIELD_DONE);
+    g.o_done = done_out;
     g.frame16 = (uint32_t)(vec16 ? frame / 16 : frame / 2);
     // 16 KB per CTA: 4 x 128-bit per thread, so a frame of 38 400 B becomes 3 CTAs
     g.chunks = (uint32_t)((frame + 16383) / 16384);

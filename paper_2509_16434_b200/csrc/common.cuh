@@ -66,6 +66,20 @@ struct ppo_model {
     // tensor index of the weight matrix of conv layer l (1..L; bias at +1, with norm gamma at +2 and beta at +3),
     // of the embedding (-1 without one) and of FC layer l (1..F; F + 1 is the head); log-sigma is the last tensor
     int ti_conv[PPO_MAX_CONV + 1], ti_embed, ti_fc[PPO_MAX_FC + 2];
+    int ti_lstm[PPO_MAX_LSTM];     // W_x of LSTM layer l (W_h at +1, b at +2)
+    int fc_in_w;                   // width of the first FC layer's input: hw[0], or lstm_h behind a recurrent trunk
+    // recurrent trunk: the sequence the next forward/backward work on, and the workspace carve
+    int seq_T, seq_Be;
+    const uint8_t *seq_done;
+    const float *seq_h_init, *seq_c_init;
+    bf16 *lstm_hs[PPO_MAX_LSTM];     // outputs h [mb][H]
+    bf16 *lstm_hprev[PPO_MAX_LSTM];  // state each step started from (after done-resets) [mb][H]
+    float *lstm_c[PPO_MAX_LSTM];     // cell states [mb][H], followed by c_prev [mb][H]
+    float *lstm_gates[PPO_MAX_LSTM]; // gate activations i, f, g, o [mb][4H]
+    float *lstm_xg, *lstm_hg;        // W_x x of all rows [mb][4H]; W_h h_prev of one step [mb][4H]
+    bf16 *lstm_dg;                   // gradient w.r.t. the gate pre-activations [mb][4H]
+    float *lstm_dtop;                // gradient w.r.t. a layer's outputs [mb][H] (from the FC layers or the layer above)
+    float *lstm_dhc, *lstm_dcc;      // gradients carried to the previous step [mb][H]
     size_t arena, nparams;
     // bound arrays
     float *master, *grad, *adam_m, *adam_v;

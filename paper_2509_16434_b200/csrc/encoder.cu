@@ -672,6 +672,78 @@ __global__ void __launch_bounds__(256) ln_bwd_kernel(bf16 *__restrict__ d, const
     }
 }
 
+// ------------------------------------------------------------ recurrent trunk ----
+
+__device__ __forceinline__ float sigmoidf_(float x) { return 1.f / (1.f + __expf(-x)); }
+
+// State the first step of a sequence starts from: h_prev[0] = bf16(h_init), c_prev[0] = c_init (rows of one step, Be x H).
+__global__ void __launch_bounds__(256) lstm_init_kernel(const float *__restrict__ h_init, const float *__restrict__ c_init,
+                                                        bf16 *__restrict__ hprev, float *__restrict__ cprev, int n) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n) return;
+    hprev[i] = __float2bfloat16_rn(h_init[i]);
+    cprev[i] = c_init[i];
+}
+
+// One time step of one LSTM layer for Be envs, element-wise part: gate pre-activations = xg + hg + b,
+//   (i, f, g, o) = (sigmoid, sigmoid, tanh, sigmoid)(.),  c = f c_prev + i g,  h = o tanh(c).
+// Keeps the gate activations and c for the backward pass, writes h as bf16 (the operand of the next contractions) and,
+// unless this is the last step, the state the next step starts from: (h, c) or zeros where done != 0.
+__global__ void __launch_bounds__(256) lstm_cell_fwd_kernel(const float *__restrict__ xg, const float *__restrict__ hg,
+                                                            const float *__restrict__ bias, const float *__restrict__ cprev,
+                                                            const uint8_t *__restrict__ done, float *__restrict__ gates,
+                                                            float *__restrict__ c, bf16 *__restrict__ h,
+                                                            bf16 *__restrict__ hprev_next, float *__restrict__ cprev_next,
+                                                            int Be, int H) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= Be * H) return;
+    const int e = i / H, j = i - e * H;
+    const size_t g0 = (size_t)e * 4 * H + j;
+    const float gi = sigmoidf_(xg[g0] + hg[g0] + bias[j]);
+    const float gf = sigmoidf_(xg[g0 + H] + hg[g0 + H] + bias[H + j]);
+    const float gg = tanhf(xg[g0 + 2 * H] + hg[g0 + 2 * H] + bias[2 * H + j]);
+    const float go = sigmoidf_(xg[g0 + 3 * H] + hg[g0 + 3 * H] + bias[3 * H + j]);
+    const float cv = gf * cprev[i] + gi * gg;
+    const float hv = go * tanhf(cv);
+    gates[g0] = gi;
+    gates[g0 + H] = gf;
+    gates[g0 + 2 * H] = gg;
+    gates[g0 + 3 * H] = go;
+    c[i] = cv;
+    const bf16 hb = __float2bfloat16_rn(hv);
+    h[i] = hb;
+    if (hprev_next) {
+        const bool reset = done[e] != 0;
+        hprev_next[i] = reset ? __float2bfloat16_rn(0.f) : hb;
+        cprev_next[i] = reset ? 0.f : cv;
+    }
+}
+
+// The same step backwards.  dtop: gradient w.r.t. this step's h from above; dhc, dcc: gradients w.r.t. the state the
+// NEXT step started from (raw: they count only where this step's done flag is clear).  Writes the gradient of the gate
+// pre-activations as bf16 (a GEMM operand) and the raw gradient of c_prev; the raw gradient of h_prev comes out of the
+// GEMM dg W_h that follows.  last != 0: no step follows, nothing is carried.
+__global__ void __launch_bounds__(256) lstm_cell_bwd_kernel(const float *__restrict__ dtop, const float *__restrict__ dhc,
+                                                            float *__restrict__ dcc, const uint8_t *__restrict__ done,
+                                                            const float *__restrict__ gates, const float *__restrict__ c,
+                                                            const float *__restrict__ cprev, bf16 *__restrict__ dg,
+                                                            int Be, int H, int last) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= Be * H) return;
+    const int e = i / H, j = i - e * H;
+    const size_t g0 = (size_t)e * 4 * H + j;
+    const bool carry = !last && done[e] == 0;
+    const float dh = dtop[i] + (carry ? dhc[i] : 0.f);
+    const float gi = gates[g0], gf = gates[g0 + H], gg = gates[g0 + 2 * H], go = gates[g0 + 3 * H];
+    const float tc = tanhf(c[i]);
+    const float dc = (carry ? dcc[i] : 0.f) + dh * go * (1.f - tc * tc);
+    dg[g0] = __float2bfloat16_rn(dc * gg * gi * (1.f - gi));
+    dg[g0 + H] = __float2bfloat16_rn(dc * cprev[i] * gf * (1.f - gf));
+    dg[g0 + 2 * H] = __float2bfloat16_rn(dc * gi * (1.f - gg * gg));
+    dg[g0 + 3 * H] = __float2bfloat16_rn(dh * tc * go * (1.f - go));
+    dcc[i] = dc * gf;
+}
+
 // ------------------------------------------------------------ orchestration ----
 
 static ConvGeom conv_geom(const ppo_model *m, int l, int rows) {  // conv layer l in 1..L
@@ -720,8 +792,8 @@ static int run_colsum(const bf16 *dZ, int ld, long long M, int N, float *db, flo
 // Weight and bias gradients of the layer whose weight matrix is tensor ti.  The TMA kernel of a convolution sums
 // the bias gradient on the tensor core on its way; everything else reduces dY in a pass of its own.
 static int run_wgrad(const ppo_model *m, int ti, const ConvGeom &g, const bf16 *dY, int ldy, const bf16 *X,
-                     cudaStream_t st) {
-    float *dW = m->grad + m->tensors[ti].off, *db = m->grad + m->tensors[ti + 1].off;
+                     cudaStream_t st, bool with_bias = true) {
+    float *dW = m->grad + m->tensors[ti].off, *db = with_bias ? m->grad + m->tensors[ti + 1].off : nullptr;
     float *part = m->wg_part[ti];
     const size_t cap = m->wg_cap[ti];
     const bool conv = g.k > 1;
@@ -729,7 +801,7 @@ static int run_wgrad(const ppo_model *m, int ti, const ConvGeom &g, const bf16 *
     if (s == PPO_OK && conv) return s;
     if (s == PPO_ERR_UNSUPPORTED && conv) s = tma_gemm_wgrad(g, dY, ldy, X, dW, nullptr, part, cap, ppo_device_status_ptr(), st);
     if (s == PPO_ERR_UNSUPPORTED) s = tc_gemm_wgrad(g, dY, ldy, X, dW, part, cap, ppo_device_status_ptr(), st);
-    if (s != PPO_OK) return s;
+    if (s != PPO_OK || !with_bias) return s;
     return run_colsum(dY, ldy, g.M(), g.Co, db, m->cs_part[ti], st);
 }
 
@@ -773,6 +845,82 @@ static int check_rows(const ppo_model *m, const ppo_minibatch *mb, int row0, int
     if (!m->master) return PPO_ERR_STATE;
     if (row0 < 0 || rows <= 0 || row0 + rows > mb->B || rows > m->mbmax) return PPO_ERR_SHAPE;
     if (!mb->depth_f16 || !mb->proprio) return PPO_ERR_INVALID_ARG;
+    return PPO_OK;
+}
+
+// Input of FC layer l (1..F; F + 1 is the head): the layer below, and for the first one h_0 or, behind a recurrent
+// trunk, the top LSTM layer's outputs.
+static const bf16 *fc_input(const ppo_model *m, int l) {
+    if (l > 1) return m->h[l - 1];
+    return m->d.n_lstm > 0 ? m->lstm_hs[m->d.n_lstm - 1] : m->h[0];
+}
+static int fc_input_width(const ppo_model *m, int l) { return l > 1 ? m->hw[l - 1] : m->fc_in_w; }
+
+static int wt_ld_of(int Co) { return (Co + 7) / 8 * 8; }
+
+// out [rows][N] (fp32, row stride N) = A [rows][K] (bf16, row stride lda) . Wn [N][K]^T: the plain product behind every
+// contraction of the recurrent trunk, through the flat (1x1-image) input-gradient GEMM.
+static int gemm_nt_f32(const ppo_model *m, int rows, int N, int K, const bf16 *A, int lda, const bf16 *Wn, float *out,
+                       cudaStream_t st) {
+    ConvGeom g = fc_geom(rows, N, K);
+    DgradEpilogue e = {nullptr, nullptr, out};
+    return run_dgrad(m, g, A, lda, Wn, Wn, K, nullptr, e, st);
+}
+
+// Forward of the recurrent trunk over the announced sequence (rows = T * Be, time-major): per layer one GEMM for
+// W_x x of all rows, then per step the GEMM W_h h_prev and the element-wise cell.
+static int lstm_forward(ppo_model *m, int rows, cudaStream_t st) {
+    const ppo_model_desc &d = m->d;
+    const int T = m->seq_T, Be = m->seq_Be, H = d.lstm_h;
+    if (T <= 0 || T * Be != rows || !m->seq_done) return PPO_ERR_STATE;
+    for (int l = 0; l < d.n_lstm; ++l) {
+        const int in = l == 0 ? m->hw[0] : H, ti = m->ti_lstm[l];
+        const bf16 *X = l == 0 ? m->h[0] : m->lstm_hs[l - 1];
+        float *cprev = m->lstm_c[l] + (size_t)m->mbmax * H;
+        PPO_TRY(gemm_nt_f32(m, rows, 4 * H, in, X, in, m->shadow + m->tensors[ti].off, m->lstm_xg, st));
+        lstm_init_kernel<<<ppo_cdiv((long long)Be * H, 256), 256, 0, st>>>(m->seq_h_init + (size_t)l * Be * H,
+                                                                          m->seq_c_init + (size_t)l * Be * H,
+                                                                          m->lstm_hprev[l], cprev, Be * H);
+        PPO_LAUNCH_CHECK();
+        for (int t = 0; t < T; ++t) {
+            const size_t r0 = (size_t)t * Be;
+            PPO_TRY(gemm_nt_f32(m, Be, 4 * H, H, m->lstm_hprev[l] + r0 * H, H, m->shadow + m->tensors[ti + 1].off, m->lstm_hg, st));
+            const bool last = t == T - 1;
+            lstm_cell_fwd_kernel<<<ppo_cdiv((long long)Be * H, 256), 256, 0, st>>>(
+                m->lstm_xg + r0 * 4 * H, m->lstm_hg, m->master + m->tensors[ti + 2].off, cprev + r0 * H, m->seq_done + r0,
+                m->lstm_gates[l] + r0 * 4 * H, m->lstm_c[l] + r0 * H, m->lstm_hs[l] + r0 * H,
+                last ? nullptr : m->lstm_hprev[l] + (r0 + Be) * H, last ? nullptr : cprev + (r0 + Be) * H, Be, H);
+            PPO_LAUNCH_CHECK();
+        }
+    }
+    return PPO_OK;
+}
+
+// Back-propagation through time.  In: lstm_dtop = dL/d(top layer's outputs) [rows][H] fp32.  Out: dh0_f32 = dL/dh_0 and
+// the gradients of every layer's W_x, W_h and b.
+static int lstm_backward(ppo_model *m, int rows, cudaStream_t st) {
+    const ppo_model_desc &d = m->d;
+    const int T = m->seq_T, Be = m->seq_Be, H = d.lstm_h;
+    if (T <= 0 || T * Be != rows || !m->seq_done) return PPO_ERR_STATE;
+    for (int l = d.n_lstm - 1; l >= 0; --l) {
+        const int in = l == 0 ? m->hw[0] : H, ti = m->ti_lstm[l];
+        const bf16 *X = l == 0 ? m->h[0] : m->lstm_hs[l - 1];
+        const float *cprev = m->lstm_c[l] + (size_t)m->mbmax * H;
+        for (int t = T - 1; t >= 0; --t) {
+            const size_t r0 = (size_t)t * Be;
+            lstm_cell_bwd_kernel<<<ppo_cdiv((long long)Be * H, 256), 256, 0, st>>>(
+                m->lstm_dtop + r0 * H, m->lstm_dhc, m->lstm_dcc, m->seq_done + r0, m->lstm_gates[l] + r0 * 4 * H,
+                m->lstm_c[l] + r0 * H, cprev + r0 * H, m->lstm_dg + r0 * 4 * H, Be, H, t == T - 1 ? 1 : 0);
+            PPO_LAUNCH_CHECK();
+            if (t > 0)  // raw gradient of the state this step started from: dg W_h
+                PPO_TRY(gemm_nt_f32(m, Be, H, 4 * H, m->lstm_dg + r0 * 4 * H, 4 * H, m->wT + m->wT_off[ti + 1], m->lstm_dhc, st));
+        }
+        // over all steps at once: the weight gradients, the bias gradient and the gradient of the layer's input
+        PPO_TRY(run_wgrad(m, ti, fc_geom(rows, in, 4 * H), m->lstm_dg, 4 * H, X, st, false));
+        PPO_TRY(run_wgrad(m, ti + 1, fc_geom(rows, H, 4 * H), m->lstm_dg, 4 * H, m->lstm_hprev[l], st, false));
+        PPO_TRY(run_colsum(m->lstm_dg, 4 * H, rows, 4 * H, m->grad + m->tensors[ti + 2].off, m->cs_part[ti], st));
+        PPO_TRY(gemm_nt_f32(m, rows, in, 4 * H, m->lstm_dg, 4 * H, m->wT + m->wT_off[ti], l == 0 ? m->dh0_f32 : m->lstm_dtop, st));
+    }
     return PPO_OK;
 }
 
@@ -843,24 +991,23 @@ extern "C" int ppo_encoder_fwd(ppo_model *m, const ppo_minibatch *mb, int row0, 
                                                               m->Hs[m->L] * m->Ws[m->L], m->Cs[m->L], d.P);
     }
     PPO_LAUNCH_CHECK();
+    if (d.n_lstm > 0) PPO_TRY(lstm_forward(m, rows, st));
     int ti = m->ti_fc[1];
     for (int l = 1; l <= m->F; ++l, ti += 2) {
-        ConvGeom g = fc_geom(rows, m->hw[l - 1], m->hw[l]);
+        ConvGeom g = fc_geom(rows, fc_input_width(m, l), m->hw[l]);
         FwdEpilogue e = {m->master + m->tensors[ti + 1].off, 1, m->h[l], nullptr, nullptr, 0};
-        PPO_TRY(run_fwd(m, g, m->h[l - 1], m->shadow + m->tensors[ti].off, e, st));
+        PPO_TRY(run_fwd(m, g, fc_input(m, l), m->shadow + m->tensors[ti].off, e, st));
     }
     {
-        ConvGeom g = fc_geom(rows, m->hw[m->F], d.A + 1);
+        ConvGeom g = fc_geom(rows, fc_input_width(m, m->F + 1), d.A + 1);
         FwdEpilogue e = {m->master + m->tensors[ti + 1].off, 0, nullptr, mean, value, d.A};
-        PPO_TRY(run_fwd(m, g, m->h[m->F], m->shadow + m->tensors[ti].off, e, st));
+        PPO_TRY(run_fwd(m, g, fc_input(m, m->F + 1), m->shadow + m->tensors[ti].off, e, st));
     }
     m->fwd_valid = true;
     m->last_row0 = row0;
     m->last_rows = rows;
     return PPO_OK;
 }
-
-static int wt_ld_of(int Co) { return (Co + 7) / 8 * 8; }
 
 static int refresh_transposed(ppo_model *m, cudaStream_t st) {
     if (m->wT_valid) return PPO_OK;
@@ -881,9 +1028,18 @@ static int refresh_transposed(ppo_model *m, cudaStream_t st) {
                                                                      m->wT + m->wT_off[m->ti_embed], Co, 1, Ci, wt_ld_of(Co));
         PPO_LAUNCH_CHECK();
     }
+    for (int l = 0; l < m->d.n_lstm; ++l) {
+        const int H = m->d.lstm_h, in = l == 0 ? m->hw[0] : H, tl = m->ti_lstm[l];
+        transpose_weights_kernel<<<ppo_cdiv((long long)in * 4 * H, 256), 256, 0, st>>>(m->shadow + m->tensors[tl].off,
+                                                                                     m->wT + m->wT_off[tl], 4 * H, 1, in, 4 * H);
+        PPO_LAUNCH_CHECK();
+        transpose_weights_kernel<<<ppo_cdiv((long long)H * 4 * H, 256), 256, 0, st>>>(m->shadow + m->tensors[tl + 1].off,
+                                                                                    m->wT + m->wT_off[tl + 1], 4 * H, 1, H, 4 * H);
+        PPO_LAUNCH_CHECK();
+    }
     int ti = m->ti_fc[1];
     for (int l = 1; l <= m->F + 1; ++l, ti += 2) {
-        const int Ci = m->hw[l - 1], Co = (l <= m->F) ? m->hw[l] : m->d.A + 1;
+        const int Ci = fc_input_width(m, l), Co = (l <= m->F) ? m->hw[l] : m->d.A + 1;
         const long long total = (long long)Ci * wt_ld_of(Co);
         transpose_weights_kernel<<<ppo_cdiv(total, 256), 256, 0, st>>>(m->shadow + m->tensors[ti].off,
                                                                      m->wT + m->wT_off[ti], Co, 1, Ci, wt_ld_of(Co));
@@ -1023,15 +1179,19 @@ extern "C" int ppo_encoder_bwd(ppo_model *m, const ppo_minibatch *mb, int row0, 
         const int ti = m->ti_fc[l];
         const int Co = (l <= F) ? m->hw[l] : d.A + 1;
         const int ldy = (l <= F) ? Co : 16;
-        ConvGeom g = fc_geom(rows, m->hw[l - 1], Co);
+        ConvGeom g = fc_geom(rows, fc_input_width(m, l), Co);
         const bf16 *dY = m->dh[l];
-        int s = run_wgrad(m, ti, g, dY, ldy, m->h[l - 1], leaf);
+        int s = run_wgrad(m, ti, g, dY, ldy, fc_input(m, l), leaf);
         if (s != PPO_OK) return join(s);
         DgradEpilogue e;
         if (l > 1) e = {m->h[l - 1], m->dh[l - 1], nullptr};
-        else e = {nullptr, nullptr, m->dh0_f32};
+        else e = {nullptr, nullptr, d.n_lstm > 0 ? m->lstm_dtop : m->dh0_f32};
         s = run_dgrad(m, g, dY, ldy, m->shadow + m->tensors[ti].off, m->wT + m->wT_off[ti], wt_ld_of(Co), nullptr, e, st);
         if (s == PPO_OK && l > 1) s = fork_here();  // dh[l-1] is ready for the next leaf
+        if (s != PPO_OK) return join(s);
+    }
+    if (d.n_lstm > 0) {  // through the recurrent trunk: lstm_dtop -> dh0_f32
+        const int s = lstm_backward(m, rows, st);
         if (s != PPO_OK) return join(s);
     }
     if (m->ti_embed >= 0) {

@@ -33,6 +33,10 @@ extern "C" int ppo_model_create(const ppo_model_desc *d, ppo_model **out) {
         for (int l = 0; l < d->n_conv; ++l)  // 16, 32, 64, 128 or 256 channels: a pixel's channels split evenly over lanes
             if (d->conv_c[l] > 256 || d->conv_c[l] < 16 || (d->conv_c[l] & (d->conv_c[l] - 1)) != 0) return PPO_ERR_UNSUPPORTED;
     }
+    if (d->n_lstm < 0 || d->n_lstm > PPO_MAX_LSTM) return PPO_ERR_INVALID_ARG;
+    if (d->n_lstm > 0 && (d->lstm_h <= 0 || d->lstm_h % 64 != 0 || d->lstm_h > 4096)) return PPO_ERR_UNSUPPORTED;
+    if (d->n_lstm > 0 && ((d->embed > 0 ? d->embed : d->conv_c[d->n_conv - 1]) + d->P) % 64 != 0)
+        return PPO_ERR_UNSUPPORTED;  // the trunk's input rows feed 64-channel boxes
     ppo_model *m = new (std::nothrow) ppo_model();
     if (!m) return PPO_ERR_INVALID_ARG;
     m->d = *d;
@@ -70,13 +74,21 @@ extern "C" int ppo_model_create(const ppo_model_desc *d, ppo_model **out) {
         push((int64_t)d->embed * m->Hs[m->L] * m->Ws[m->L] * m->Cs[m->L]);
         push(d->embed);
     }
+    m->fc_in_w = m->hw[0];
+    for (int l = 0; l < d->n_lstm; ++l) {
+        m->ti_lstm[l] = (int)m->tensors.size();
+        push((int64_t)4 * d->lstm_h * m->fc_in_w);
+        push((int64_t)4 * d->lstm_h * d->lstm_h);
+        push((int64_t)4 * d->lstm_h);
+        m->fc_in_w = d->lstm_h;
+    }
     for (int l = 0; l < m->F; ++l) {
         m->ti_fc[l + 1] = (int)m->tensors.size();
-        push((int64_t)m->hw[l + 1] * m->hw[l]);
+        push((int64_t)m->hw[l + 1] * (l == 0 ? m->fc_in_w : m->hw[l]));
         push(m->hw[l + 1]);
     }
     m->ti_fc[m->F + 1] = (int)m->tensors.size();
-    push((int64_t)(d->A + 1) * m->hw[m->F]);
+    push((int64_t)(d->A + 1) * (m->F == 0 ? m->fc_in_w : m->hw[m->F]));
     push(d->A + 1);
     push(d->A);
     m->arena = (size_t)off;
@@ -90,7 +102,12 @@ extern "C" int ppo_model_create(const ppo_model_desc *d, ppo_model **out) {
         };
         for (int l = 2; l <= m->L; ++l) tpush(m->ti_conv[l], m->Cs[l - 1], d->conv_k[l - 1] * d->conv_k[l - 1], m->Cs[l]);
         if (m->ti_embed >= 0) tpush(m->ti_embed, (int64_t)m->Hs[m->L] * m->Ws[m->L] * m->Cs[m->L], 1, d->embed);
-        for (int l = 1; l <= m->F + 1; ++l) tpush(m->ti_fc[l], m->hw[l - 1], 1, l <= m->F ? m->hw[l] : d->A + 1);
+        for (int l = 0; l < d->n_lstm; ++l) {  // W_x^T [in][4H] and W_h^T [H][4H]
+            tpush(m->ti_lstm[l], 4 * d->lstm_h, 1, l == 0 ? m->hw[0] : d->lstm_h);
+            tpush(m->ti_lstm[l] + 1, 4 * d->lstm_h, 1, d->lstm_h);
+        }
+        for (int l = 1; l <= m->F + 1; ++l)
+            tpush(m->ti_fc[l], l == 1 ? m->fc_in_w : m->hw[l - 1], 1, l <= m->F ? m->hw[l] : d->A + 1);
         m->wT_elems = (size_t)toff;
         int64_t coff = 0;
         for (int l = 0; l <= PPO_MAX_CONV; ++l) m->wC_off[l] = 0;
@@ -108,6 +125,9 @@ extern "C" int ppo_model_create(const ppo_model_desc *d, ppo_model **out) {
     m->fwd_valid = false;
     m->wT_valid = false;
     m->last_row0 = m->last_rows = -1;
+    m->seq_T = m->seq_Be = 0;
+    m->seq_done = nullptr;
+    m->seq_h_init = m->seq_c_init = nullptr;
     *out = m;
     return PPO_OK;
 }
@@ -191,7 +211,27 @@ static size_t carve(ppo_model *m, const ppo_model *shape, int mb, char *base) {
         if (shape->ti_embed >= 0)
             scratch_for(shape->ti_embed, shape->Hs[shape->L] * shape->Ws[shape->L] * shape->Cs[shape->L], shape->d.embed, 1);
         for (int l = 1; l <= shape->F + 1; ++l)
-            scratch_for(shape->ti_fc[l], shape->hw[l - 1], l <= shape->F ? shape->hw[l] : shape->d.A + 1, 1);
+            scratch_for(shape->ti_fc[l], l == 1 ? shape->fc_in_w : shape->hw[l - 1], l <= shape->F ? shape->hw[l] : shape->d.A + 1, 1);
+        if (shape->d.n_lstm > 0) {
+            const size_t H = (size_t)shape->d.lstm_h, R = (size_t)mb;
+            for (int l = 0; l < shape->d.n_lstm; ++l) {
+                scratch_for(shape->ti_lstm[l], l == 0 ? shape->hw[0] : (int)H, 4 * (int)H, 1);
+                scratch_for(shape->ti_lstm[l] + 1, (int)H, 4 * (int)H, 1);
+                char *a = take(R * H * sizeof(bf16)), *b = take(R * H * sizeof(bf16));
+                char *c = take(2 * R * H * sizeof(float)), *g = take(4 * R * H * sizeof(float));
+                if (m) {
+                    m->lstm_hs[l] = (bf16 *)a; m->lstm_hprev[l] = (bf16 *)b;
+                    m->lstm_c[l] = (float *)c; m->lstm_gates[l] = (float *)g;
+                }
+            }
+            char *xg = take(4 * R * H * sizeof(float)), *hg = take(4 * R * H * sizeof(float));
+            char *dg = take(4 * R * H * sizeof(bf16)), *dt = take(R * H * sizeof(float));
+            char *dh = take(R * H * sizeof(float)), *dc = take(R * H * sizeof(float));
+            if (m) {
+                m->lstm_xg = (float *)xg; m->lstm_hg = (float *)hg; m->lstm_dg = (bf16 *)dg;
+                m->lstm_dtop = (float *)dt; m->lstm_dhc = (float *)dh; m->lstm_dcc = (float *)dc;
+            }
+        }
         if (shape->d.embed > 0) {
             char *dz = take((size_t)mb * shape->d.embed * sizeof(bf16));
             if (m) m->dze = (bf16 *)dz;
@@ -251,6 +291,13 @@ extern "C" int ppo_model_activation_ptr(const ppo_model *m, int kind, int index,
         *elems = (size_t)m->mbmax * m->Hs[index] * m->Ws[index];
         return PPO_OK;
     }
+    if (kind >= 5 && kind <= 8 && index >= 0 && index < m->d.n_lstm) {
+        const size_t H = (size_t)m->d.lstm_h, R = (size_t)m->mbmax;
+        *ptr = kind == 5 ? (void *)m->lstm_hs[index] : kind == 6 ? (void *)m->lstm_c[index]
+               : kind == 7 ? (void *)m->lstm_gates[index] : (void *)m->lstm_hprev[index];
+        *elems = kind == 6 ? 2 * R * H : kind == 7 ? 4 * R * H : R * H;
+        return PPO_OK;
+    }
     if (kind == 2 && index >= 1 && index < m->L && m->abits[index]) {
         *ptr = m->abits[index];
         *elems = (size_t)m->mbmax * m->Hs[index] * m->Ws[index] * m->Cs[index] / 32;
@@ -262,6 +309,20 @@ extern "C" int ppo_model_activation_ptr(const ppo_model *m, int kind, int index,
         return PPO_OK;
     }
     return PPO_ERR_INVALID_ARG;
+}
+
+extern "C" int ppo_model_set_sequence(ppo_model *m, int T, int Be, const uint8_t *done, const float *h_init,
+                                      const float *c_init) {
+    if (!m || !done || !h_init || !c_init) return PPO_ERR_INVALID_ARG;
+    if (m->d.n_lstm == 0 || !m->ws) return PPO_ERR_STATE;
+    if (T <= 0 || Be <= 0 || (long long)T * Be > m->mbmax) return PPO_ERR_SHAPE;
+    m->seq_T = T;
+    m->seq_Be = Be;
+    m->seq_done = done;
+    m->seq_h_init = h_init;
+    m->seq_c_init = c_init;
+    m->fwd_valid = false;
+    return PPO_OK;
 }
 
 extern "C" int ppo_model_sync_masks(ppo_model *m, int rows, void *stream) {
@@ -510,6 +571,7 @@ extern "C" int ppo_policy_act(ppo_model *m, ppo_buffer *b, int t, const float *e
     const ppo_buffer_desc &d = b->d;
     if (t < 0 || t >= d.T) return PPO_ERR_INVALID_ARG;
     if (d.H != m->d.H || d.W != m->d.W || d.P != m->d.P || d.A != m->d.A) return PPO_ERR_SHAPE;
+    if (m->d.n_lstm > 0) return PPO_ERR_UNSUPPORTED;  // a recurrent policy acts through ppo_model_set_sequence + ppo_encoder_fwd
     const size_t N = (size_t)d.N;
     char *depth = b->base + b->field_off[PPO_FIELD_DEPTH] + (size_t)t * N * d.H * d.W * 2;
     float *proprio = reinterpret_cast<float *>(b->base + b->field_off[PPO_FIELD_PROPRIO]) + (size_t)t * N * d.P;

@@ -35,10 +35,26 @@ class Learner:
         self.hyper = hyper or Hyper(gamma=w.gamma, lam=w.lam, clip=w.clip)
         self.bdesc = ppo.buffer_desc(w.N, w.T, w.H, w.W, w.P, w.A)
         self.buffer = ppo.Buffer(self.bdesc, device)
-        self.mdesc = ppo.model_desc(w.H, w.W, w.conv_c, w.conv_k, w.fc, w.P, w.A, norm=w.norm, embed=w.embed)
+        self.mdesc = ppo.model_desc(w.H, w.W, w.conv_c, w.conv_k, w.fc, w.P, w.A, norm=w.norm, embed=w.embed,
+                                    n_lstm=w.n_lstm, lstm_h=w.lstm_h)
         self.microbatch = min(microbatch, w.B)
+        self.recurrent = w.n_lstm > 0
+        if self.recurrent:
+            # a minibatch is N / minibatches whole env sequences; a micro-batch is a group of them, time-major
+            envs = w.N // w.minibatches
+            if w.N % w.minibatches:
+                raise ValueError("a recurrent minibatch holds whole env sequences: N must divide by minibatches")
+            self.seq_envs = max(1, min(self.microbatch // w.T, envs))
+            while envs % self.seq_envs:
+                self.seq_envs -= 1
+            self.microbatch = self.seq_envs * w.T
         self.model = ppo.Model(self.mdesc, self.microbatch, device)
-        self.mb = ppo.MinibatchArrays(self.bdesc, w.B, device, with_index=with_index)
+        self.mb = ppo.MinibatchArrays(self.bdesc, self.microbatch if self.recurrent else w.B, device,
+                                      with_index=with_index)
+        if self.recurrent:
+            self.seq_done = torch.zeros((w.T, self.seq_envs), dtype=torch.uint8, device=device)
+            self.h_init = torch.zeros((w.n_lstm, self.seq_envs, w.lstm_h), dtype=torch.float32, device=device)
+            self.c_init = torch.zeros_like(self.h_init)
         mbs = self.microbatch
         self.mean = torch.empty((mbs, w.A), dtype=torch.float32, device=device)
         self.value = torch.empty(mbs, dtype=torch.float32, device=device)
@@ -89,6 +105,8 @@ class Learner:
         w, h = self.w, self.hyper
         K = num_minibatches or w.minibatches
         B = w.M // K
+        if self.recurrent:
+            return self._sequence_step(seed, epoch, k, K)
         ppo.ppo_shuffle_gather_minibatch(self.buffer, seed, epoch, k, K, self.mb)
         ppo.ppo_model_zero_grad(self.model)
         self.loss.zero_()
@@ -98,6 +116,25 @@ class Learner:
             ppo.ppo_loss_fwd_bwd(self.model, self.mb, r0, rows, B, self.mean, self.value, h.clip, h.vf_coef,
                                  h.ent_coef, self.loss, self.dmean, self.dvalue)
             ppo.ppo_encoder_bwd(self.model, self.mb, r0, rows, self.dmean, self.dvalue, True)
+        self.adam_t += 1
+        ppo.ppo_adam_step(self.model, h.lr, h.beta1, h.beta2, h.eps, self.adam_t)
+
+    def _sequence_step(self, seed: int, epoch: int, k: int, K: int):
+        """Recurrent minibatch k: the env permutation is cut into K * S groups of seq_envs envs, groups k*S .. k*S+S-1
+        are this minibatch's micro-batches; each runs forward through time from a zero state (reset again wherever
+        the previous step ended an episode), then backward through time."""
+        w, h = self.w, self.hyper
+        S = (w.N // K) // self.seq_envs
+        rows, B = self.microbatch, (w.N // K) * w.T
+        ppo.ppo_model_zero_grad(self.model)
+        self.loss.zero_()
+        for j in range(S):
+            ppo.ppo_shuffle_gather_sequences(self.buffer, seed, epoch, k * S + j, K * S, self.mb, self.seq_done)
+            ppo.ppo_model_set_sequence(self.model, w.T, self.seq_envs, self.seq_done, self.h_init, self.c_init)
+            ppo.ppo_encoder_fwd(self.model, self.mb, 0, rows, self.mean, self.value)
+            ppo.ppo_loss_fwd_bwd(self.model, self.mb, 0, rows, B, self.mean, self.value, h.clip, h.vf_coef,
+                                 h.ent_coef, self.loss, self.dmean, self.dvalue)
+            ppo.ppo_encoder_bwd(self.model, self.mb, 0, rows, self.dmean, self.dvalue, True)
         self.adam_t += 1
         ppo.ppo_adam_step(self.model, h.lr, h.beta1, h.beta2, h.eps, self.adam_t)
 

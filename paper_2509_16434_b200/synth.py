@@ -40,6 +40,8 @@ class Workload:
     seed: int = 0
     norm: bool = False  # layer normalisation over the channels of every conv output, before its ReLU
     embed: int = 0      # > 0: flatten -> fully connected (embed) -> ReLU instead of the global average pool
+    n_lstm: int = 0     # LSTM layers between the joined feature and the fully connected layers
+    lstm_h: int = 0     # their width
 
     @property
     def M(self) -> int:
@@ -65,6 +67,10 @@ WORKLOADS: Dict[str, Workload] = {
     # 32-d embedding of the flattened map, joined with proprioception, fully connected [512, 512, 256]
     "paper_cnn": Workload("paper_cnn", 1024, 16, 120, 160, (16, 32, 64, 128), (3, 3, 3, 3), (512, 512, 256), 1, 4,
                           norm=True, embed=32),
+    # the paper's whole policy: that CNN and embedding, two LSTM layers of 1024 units, fully connected [512, 512, 256];
+    # minibatches are sequences (256 envs x 16 steps)
+    "paper_policy": Workload("paper_policy", 1024, 16, 120, 160, (16, 32, 64, 128), (3, 3, 3, 3), (512, 512, 256), 1, 4,
+                             norm=True, embed=32, n_lstm=2, lstm_h=1024),
     # profiling-sized twin of cfg2: same frames, network and micro-batch shapes, 1/8 of the envs
     "cfg2_prof": Workload("cfg2_prof", 128, 16, 120, 160, (32, 64, 128, 256), (3, 3, 3, 3), (512, 512), 1, 4),
     # profiling-sized twin of cfg4: same frames and network, 64 envs (minibatches of 128 rows)
@@ -166,6 +172,9 @@ def param_shapes(w: Workload):
     if w.embed:
         shapes += [(w.embed, h * wd * cin), (w.embed,)]
         i = w.embed + w.P
+    for _ in range(w.n_lstm):
+        shapes += [(4 * w.lstm_h, i), (4 * w.lstm_h, w.lstm_h), (4 * w.lstm_h,)]
+        i = w.lstm_h
     for o in w.fc:
         shapes += [(o, i), (o,)]
         i = o

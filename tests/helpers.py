@@ -19,7 +19,8 @@ def max_abs_scaled(x, ref):
 
 
 def oracle_model(w):
-    return orc.ModelDesc(w.H, w.W, tuple(w.conv_c), tuple(w.conv_k), tuple(w.fc), w.P, w.A, norm=w.norm, embed=w.embed)
+    return orc.ModelDesc(w.H, w.W, tuple(w.conv_c), tuple(w.conv_k), tuple(w.fc), w.P, w.A, norm=w.norm, embed=w.embed,
+                         n_lstm=w.n_lstm, lstm_h=w.lstm_h)
 
 
 def oracle_rollout_actions(md, theta, roll):

@@ -78,13 +78,16 @@ def test_buffer_alloc_rejects_bad_arguments(lib):
     assert lib.ppo_buffer_free(h) == 0
 
 
-@pytest.mark.parametrize("name", ["cfg1", "cfg2", "cfg4"])
+@pytest.mark.parametrize("name", ["cfg1", "cfg2", "cfg4", "paper_cnn", "paper_policy"])
 def test_model_layout_matches_the_oracles(lib, name):
     w = synth.WORKLOADS[name]
-    md = ppo.model_desc(w.H, w.W, w.conv_c, w.conv_k, w.fc, w.P, w.A)
+    md = ppo.model_desc(w.H, w.W, w.conv_c, w.conv_k, w.fc, w.P, w.A, norm=w.norm, embed=w.embed, n_lstm=w.n_lstm,
+                        lstm_h=w.lstm_h)
     h = C.c_void_p()
     assert lib.ppo_model_create(C.byref(md), C.byref(h)) == 0
-    lay = orc.param_layout(orc.ModelDesc(w.H, w.W, w.conv_c, w.conv_k, w.fc, w.P, w.A))
+    lay = orc.param_layout(orc.ModelDesc(w.H, w.W, w.conv_c, w.conv_k, w.fc, w.P, w.A, norm=w.norm, embed=w.embed,
+                                         n_lstm=w.n_lstm, lstm_h=w.lstm_h))
+    assert [tuple(s) for s in lay.shapes] == [tuple(s) for s in synth.param_shapes(w)[0]]
     assert lib.ppo_model_param_count(h) == sum(lay.sizes)
     assert lib.ppo_model_arena_elems(h) == lay.total
     assert lib.ppo_model_num_tensors(h) == len(lay.offsets)
@@ -92,7 +95,18 @@ def test_model_layout_matches_the_oracles(lib, name):
         off, sz = C.c_int64(), C.c_int64()
         assert lib.ppo_model_tensor_info(h, i, C.byref(off), C.byref(sz)) == 0
         assert (off.value, sz.value) == (o, s)
-    assert lib.ppo_model_param_count(h) == {"cfg1": 51_481, "cfg2": 805_145, "cfg4": 1_395_737}[name]
+    closed = {"cfg1": 51_481, "cfg2": 805_145, "cfg4": 1_395_737}
+    if name in closed:
+        assert lib.ppo_model_param_count(h) == closed[name]
+    if w.n_lstm:  # W_x, W_h and b of each layer: 4H (in + H + 1)
+        H, ins = w.lstm_h, [w.embed + w.P] + [w.lstm_h] * (w.n_lstm - 1)
+        i0 = len(lay.sizes) - 3 - 2 * len(w.fc) - 3 * w.n_lstm
+        assert sum(lay.sizes[i0:i0 + 3 * w.n_lstm]) == sum(4 * H * (i + H + 1) for i in ins)
+        # a sequence must be announced with sane arguments
+        assert lib.ppo_model_set_sequence(h, 4, 4, C.c_void_p(0x100), C.c_void_p(0x100), C.c_void_p(0x100)) == 4  # unbound
+        assert lib.ppo_model_set_sequence(h, 4, 4, None, C.c_void_p(0x100), C.c_void_p(0x100)) == 1
+    else:
+        assert lib.ppo_model_set_sequence(h, 4, 4, C.c_void_p(0x100), C.c_void_p(0x100), C.c_void_p(0x100)) != 0
     ws1, ws2 = lib.ppo_model_workspace_bytes(h, 64), lib.ppo_model_workspace_bytes(h, 128)
     assert 0 < ws1 < ws2
     # calls before bind are refused
@@ -117,10 +131,14 @@ def test_model_create_rejects_unsupported_shapes(lib):
     bad = [ppo.model_desc(64, 64, (16, 30), (3, 3), (64,)),      # channels not a multiple of 8
            ppo.model_desc(64, 64, (16, 32), (3, 4), (64,)),      # even kernel
            ppo.model_desc(64, 64, (16, 32), (3, 3), (60,)),      # fc width
-           ppo.model_desc(64, 64, (16, 32), (3, 3), (64,), P=3)]  # pooled + proprio width
+           ppo.model_desc(64, 64, (16, 32), (3, 3), (64,), P=3),  # pooled + proprio width
+           ppo.model_desc(64, 64, (16, 32), (3, 3), (64,), n_lstm=1, lstm_h=48),   # LSTM width
+           ppo.model_desc(64, 64, (16, 32), (3, 3), (64,), P=8, n_lstm=1, lstm_h=64),]  # LSTM input width
     for md in bad:
         assert lib.ppo_model_create(C.byref(md), C.byref(h)) == 7
     assert lib.ppo_model_create(None, C.byref(h)) == 1
+    many = ppo.model_desc(64, 64, (16, 32), (3, 3), (64,), n_lstm=5, lstm_h=64)  # more layers than the descriptor holds
+    assert lib.ppo_model_create(C.byref(many), C.byref(h)) == 1
 
 
 def test_synth_is_seeded_and_shaped():
