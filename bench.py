@@ -75,6 +75,9 @@ def fwd_flops_per_sample(w, skip_conv1=False):
     if getattr(w, "embed", 0):
         f += 2 * hs[-1] * ws[-1] * cs[-1] * w.embed
         i = w.embed + w.P
+    for _ in range(getattr(w, "n_lstm", 0)):  # W_x x and W_h h_prev of the four gates
+        f += 2 * 4 * w.lstm_h * (i + w.lstm_h)
+        i = w.lstm_h
     for o in list(w.fc) + [w.A + 1]:
         f += 2 * i * o
         i = o
@@ -221,8 +224,8 @@ def run_ours(args):
     L, roll = make_learner(w, args.microbatch, device)
 
     timer = CallTimer()
-    names = ["ppo_compute_gae", "ppo_shuffle_gather_minibatch", "ppo_encoder_fwd", "ppo_loss_fwd_bwd",
-             "ppo_encoder_bwd", "ppo_adam_step"]
+    gather_name = "ppo_shuffle_gather_sequences" if w.n_lstm else "ppo_shuffle_gather_minibatch"
+    names = ["ppo_compute_gae", gather_name, "ppo_encoder_fwd", "ppo_loss_fwd_bwd", "ppo_encoder_bwd", "ppo_adam_step"]
     originals = {n: getattr(ppo, n) for n in names}
 
     def barrier():
@@ -334,7 +337,7 @@ def run_ours(args):
         rows = L.microbatch
         fwd_ms, n_fwd = timer.mean_ms("ppo_encoder_fwd")
         bwd_ms, _ = timer.mean_ms("ppo_encoder_bwd")
-        gat_ms, _ = timer.mean_ms("ppo_shuffle_gather_minibatch")
+        gat_ms, _ = timer.mean_ms(gather_name)
         gae_ms, _ = timer.mean_ms("ppo_compute_gae")
         # the single-launch variant of GAE + moments + normalisation (scan, grid barrier, normalise), outside the step
         gae1 = []
@@ -354,7 +357,7 @@ def run_ours(args):
         enc_flops = (fwd_flops_per_sample(w) + bwd_flops_per_sample(w)) * mean_rows
         enc_tf = enc_flops / ((fwd_ms + bwd_ms) * 1e-3) / 1e12
         peak_tf = peaks["bf16_tflops_sustained"]
-        gather_gbs = 2 * w.B * record_bytes(w) / (gat_ms * 1e-3) / 1e9
+        gather_gbs = 2 * (rows if w.n_lstm else w.B) * record_bytes(w) / (gat_ms * 1e-3) / 1e9
         gae_gbs = (17 + 8) * w.M / (gae_ms * 1e-3) / 1e9
         adam_gbs = 30 * L.model.arena / (adam_ms * 1e-3) / 1e9
         # DRAM bytes of the encoder's GEMM and conv1 kernels per sample row (dram__bytes_read + write summed over the 18
@@ -381,7 +384,7 @@ def run_ours(args):
                      "note": "working set fits L2; launch-latency bound at this size"},
         }
         others["supplementary_scaled_inputs"] = hbm_resident_rows(peaks)
-        rollout = time_rollout_inference(L, host, w)
+        rollout = None if w.n_lstm else time_rollout_inference(L, host, w)
         cpu = cpu_baseline(w, host, L) if world == 1 and not args.no_cpu_baseline else None
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -390,7 +393,9 @@ def run_ours(args):
             "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": {"workload": f"{w.name}: {w.N} envs x T={w.T}, depth 1x{w.H}x{w.W} fp16, conv "
-                                   f"{'-'.join(map(str, w.conv_c))}, fc {'-'.join(map(str, w.fc))}, "
+                                   f"{'-'.join(map(str, w.conv_c))}, "
+                                   + (f"{w.n_lstm} x LSTM({w.lstm_h}), " if w.n_lstm else "") +
+                                   f"fc {'-'.join(map(str, w.fc))}, "
                                    f"{w.epochs} epoch(s) x {w.minibatches} minibatches",
                        "env_steps_per_step": env_steps, "minibatch": w.B, "microbatch": L.microbatch,
                        "l2_policy": "inputs_larger_than_l2 (buffer %.0f MB, minibatch activations %.0f MB)" % (
@@ -481,23 +486,42 @@ def hbm_resident_rows(peaks, warmup=3, steps=10):
 
 # ---------------------------------------------------------------- CPU baseline ----
 
+def sample_rows(w, n_samples):
+    """Buffer rows (t * N + n) of the bounded sample, in the order the oracle trains on them: the first n_samples of the
+    sample permutation, or, for a recurrent policy, the first n_samples / T envs of the env permutation, time-major."""
+    from oracle import oracle as orc
+    if not w.n_lstm:
+        return orc.perm(w.seed, 0, w.M, 0, n_samples).astype(np.int64)
+    envs = orc.perm(w.seed, 0, w.N, 0, n_samples // w.T).astype(np.int64)
+    return (np.arange(w.T, dtype=np.int64)[:, None] * w.N + envs[None, :]).reshape(-1)
+
+
 def oracle_sample_step(w, fields, theta, n_samples):
     """The oracle's learner step on a bounded sample: GAE + normalisation at full size, then one minibatch of
     n_samples rows (permutation, gather, forward, loss, backward, Adam).  Returns seconds and samples trained."""
     from oracle import oracle as orc
-    md = orc.ModelDesc(w.H, w.W, tuple(w.conv_c), tuple(w.conv_k), tuple(w.fc), w.P, w.A, norm=w.norm, embed=w.embed)
+    md = orc.ModelDesc(w.H, w.W, tuple(w.conv_c), tuple(w.conv_k), tuple(w.fc), w.P, w.A, norm=w.norm, embed=w.embed,
+                       n_lstm=w.n_lstm, lstm_h=w.lstm_h)
     t0 = time.perf_counter()
     adv, ret = orc.gae(fields["reward"], fields["value"], fields["done"], fields["last_value"], w.gamma, w.lam)
     adv, _, _ = orc.adv_normalize(adv)
     t_gae = time.perf_counter() - t0
     t0 = time.perf_counter()
-    idx = orc.perm(w.seed, 0, w.M, 0, n_samples)
-    tt, nn = np.divmod(idx.astype(np.int64), w.N)
+    idx = sample_rows(w, n_samples)
+    tt, nn = np.divmod(idx, w.N)
     depth = fields["depth_rows"]            # the sampled rows' frames, gathered on the device side of the bench
     g = {"proprio": fields["proprio"][tt, nn], "action": fields["action"][tt, nn], "logp": fields["logp"][tt, nn],
          "adv": adv[tt, nn], "ret": ret[tt, nn]}
-    _, out, grad, _, _ = orc.total_loss_and_grad(md, theta, depth, g["proprio"], g["action"], g["logp"], g["adv"],
-                                                 g["ret"], w.clip, 0.5, 0.01, act_bf16=True)
+    if w.n_lstm:
+        ne = n_samples // w.T
+        zero = np.zeros((w.n_lstm, ne, w.lstm_h))
+        _, out, grad, _, _ = orc.total_loss_and_grad_seq(
+            md, theta, depth.reshape(w.T, ne, w.H, w.W), g["proprio"].reshape(w.T, ne, w.P),
+            fields["done"][tt, nn].reshape(w.T, ne), zero, zero, g["action"], g["logp"], g["adv"], g["ret"], w.clip, 0.5,
+            0.01, act_bf16=True)
+    else:
+        _, out, grad, _, _ = orc.total_loss_and_grad(md, theta, depth, g["proprio"], g["action"], g["logp"], g["adv"],
+                                                     g["ret"], w.clip, 0.5, 0.01, act_bf16=True)
     th = np.asarray(theta, np.float64).copy()
     orc.adam(th, np.zeros_like(th), np.zeros_like(th), grad, 3e-4, 0.9, 0.999, 1e-8, 1)
     t_mb = time.perf_counter() - t0
@@ -510,7 +534,9 @@ def cpu_baseline(w, host, L, n_samples=None):
     import torch
     # about 10-30 s of oracle work on a 16-core host: ~0.4 / 7 / 35 ms per row at the three frame sizes
     n_samples = n_samples or min(w.B, 4096 if w.H * w.W <= 120 * 160 else 768)
-    idx = orc.perm(w.seed, 0, w.M, 0, n_samples).astype(np.int64)
+    if w.n_lstm:  # whole env sequences; the recurrent layers cost the oracle several times the CNN's time per row
+        n_samples = max(1, min(n_samples, 1024) // w.T) * w.T
+    idx = sample_rows(w, n_samples)
     flat = host["depth"].view(w.M, w.H, w.W)   # the rollout as it sits in pinned host memory
     fields = {k: host[k].numpy() for k in ("proprio", "action", "logp", "value", "reward", "done", "last_value")}
     fields["depth_rows"] = flat[torch.as_tensor(idx)].numpy()
@@ -534,13 +560,16 @@ def run_reference(args):
     w = synth.WORKLOADS[args.workload]
     # every step is a bounded sample; the default 3 + 5 steps stay within a few minutes of host time
     n_samples = min(w.B, 1024 if w.H * w.W <= 64 * 64 else 512 if w.H * w.W <= 120 * 160 else 96)
+    if w.n_lstm:
+        n_samples = max(1, n_samples // w.T) * w.T  # whole env sequences
     # a host-generated slice of the workload: all small fields at full size, frames only for the sampled rows
     small = w.scaled(w.N, H=2, W=2)
     roll = synth.rollout_numpy(small, w.seed)
     g = np.random.Generator(np.random.Philox(key=[w.seed, 1234]))
     depth = g.uniform(0.1, 2.0, (n_samples, w.H, w.W)).astype(np.float16)
     depth[g.random(depth.shape) < 0.1] = 0
-    md = orc.ModelDesc(w.H, w.W, tuple(w.conv_c), tuple(w.conv_k), tuple(w.fc), w.P, w.A, norm=w.norm, embed=w.embed)
+    md = orc.ModelDesc(w.H, w.W, tuple(w.conv_c), tuple(w.conv_k), tuple(w.fc), w.P, w.A, norm=w.norm, embed=w.embed,
+                       n_lstm=w.n_lstm, lstm_h=w.lstm_h)
     lay = orc.param_layout(md)
     theta = synth.init_params(lay.total, lay.offsets, lay.shapes, w.seed, ones=synth.param_shapes(w)[1])
     fields = {k: roll[k] for k in ("proprio", "value", "reward", "done", "last_value")}

@@ -490,6 +490,8 @@ __global__ void __launch_bounds__(256) sum_partials_kernel(const float *__restri
     const int o = threadIdx.x & 31, j = threadIdx.x >> 5;
     const int i = blockIdx.x * 32 + o;
     const int n = nA + nB;
+    part += (size_t)blockIdx.y * nparts * n;  // blockIdx.y: one of several independent reductions of nA results (nB = 0)
+    dstA += (size_t)blockIdx.y * nA;
     float acc = 0.f;
     if (i < n)
         for (int b = j; b < nparts; b += 8) acc += part[(size_t)b * n + i];
@@ -504,8 +506,9 @@ __global__ void __launch_bounds__(256) sum_partials_kernel(const float *__restri
     }
 }
 
-static int sum_partials(const float *part, int nparts, int nA, float *dstA, int nB, float *dstB, cudaStream_t st) {
-    sum_partials_kernel<<<ppo_cdiv(nA + nB, 32), 256, 0, st>>>(part, nparts, nA, dstA, nB, dstB);
+static int sum_partials(const float *part, int nparts, int nA, float *dstA, int nB, float *dstB, cudaStream_t st,
+                        int slabs = 1) {
+    sum_partials_kernel<<<dim3(ppo_cdiv(nA + nB, 32), slabs), 256, 0, st>>>(part, nparts, nA, dstA, nB, dstB);
     PPO_LAUNCH_CHECK();
     return PPO_OK;
 }
@@ -518,6 +521,8 @@ __global__ void __launch_bounds__(256) colsum_kernel(const bf16 *__restrict__ dZ
     const int chunks = N >> 3;                    // 16-byte chunks per row
     const int rows_per_pass = 256 / chunks;       // whole rows covered by one pass of the block
     const int tc = threadIdx.x % chunks, tr = threadIdx.x / chunks;
+    dZ += (size_t)blockIdx.y * N;  // blockIdx.y: slab of N columns of a wider matrix
+    part += (size_t)blockIdx.y * gridDim.x * N;
     float acc[8];
 #pragma unroll
     for (int i = 0; i < 8; ++i) acc[i] = 0.f;
@@ -822,15 +827,11 @@ static int run_colsum(const bf16 *dZ, int ld, long long M, int N, float *db, flo
         return sum_partials(part, blocks, N, db, 0, nullptr, st);
     }
     if (N > 256 && N % 256 == 0) {
-        // wide FC layers: one launch per 256-column slab
+        // wide layers: slabs of 256 columns along the grid's second axis
         const int blocks = colsum_blocks(M, 64);
-        for (int n0 = 0; n0 < N; n0 += 256) {
-            float *p = part + (size_t)(n0 / 256) * blocks * 256;
-            colsum_kernel<<<blocks, 256, 0, st>>>(dZ + n0, ld, M, 256, p);
-            PPO_LAUNCH_CHECK();
-            PPO_TRY(sum_partials(p, blocks, 256, db + n0, 0, nullptr, st));
-        }
-        return PPO_OK;
+        colsum_kernel<<<dim3(blocks, N / 256), 256, 0, st>>>(dZ, ld, M, 256, part);
+        PPO_LAUNCH_CHECK();
+        return sum_partials(part, blocks, 256, db, 0, nullptr, st, N / 256);
     }
     int blocks = ppo_cdiv(M, 2048);
     blocks = blocks > 64 ? 64 : (blocks < 1 ? 1 : blocks);

@@ -958,6 +958,15 @@ int pick_bn(int N) {  // tile width: N split evenly into tiles of at most 256, r
     return bn < 16 ? 16 : bn;
 }
 
+// Tile width of a flat GEMM (rows x N): as pick_bn, then halved while the tiles would leave SMs without work (few rows,
+// as in the per-step products of a recurrent layer) and the halves still divide N.
+static int flat_bn(int N, long long rows) {
+    int bn = pick_bn(N);
+    const long long mt = (rows + 127) / 128;
+    while (bn >= 64 && bn % 32 == 0 && N % (bn / 2) == 0 && mt * ((N + bn - 1) / bn) < ppo_num_sms()) bn /= 2;
+    return bn;
+}
+
 int ensure_smem_attrs() {
     static bool attr_set[64] = {false};
     int dev = 0;
@@ -1056,7 +1065,7 @@ int tma_gemm_fwd(const ConvGeom &g, const bf16 *X, const bf16 *W, const FwdEpilo
                  : make_act_maps(a.mapA, X, g.Ci, g.Ci, g.Wi, g.Hi, g.B, a.grid, CB, 2);
     if (s != PPO_OK) return s;
     a.N = g.Co;
-    a.BN = pick_bn(g.Co);
+    a.BN = flat && e.out ? flat_bn(g.Co, g.B) : pick_bn(g.Co);
     {
         const long long dims[2] = {g.K(), g.Co};
         const int box[2] = {CB, a.BN}, es[2] = {1, 1};
@@ -1143,7 +1152,7 @@ int tma_gemm_dgrad(const ConvGeom &g, const bf16 *dY, int ldy, const bf16 *Wt, i
     a.status = status;
     if (flat) {
         a.N = g.Ci;
-        a.BN = pick_bn(g.Ci);
+        a.BN = flat_bn(g.Ci, g.B);
         a.wtaps = 1;
         const long long dims[2] = {wt_ld, g.Ci};
         const int box[2] = {CB, a.BN}, es[2] = {1, 1};

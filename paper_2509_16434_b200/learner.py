@@ -55,6 +55,7 @@ class Learner:
             self.seq_done = torch.zeros((w.T, self.seq_envs), dtype=torch.uint8, device=device)
             self.h_init = torch.zeros((w.n_lstm, self.seq_envs, w.lstm_h), dtype=torch.float32, device=device)
             self.c_init = torch.zeros_like(self.h_init)
+        self.roll_h = self.roll_c = self.roll_done = None
         mbs = self.microbatch
         self.mean = torch.empty((mbs, w.A), dtype=torch.float32, device=device)
         self.value = torch.empty(mbs, dtype=torch.float32, device=device)
@@ -80,17 +81,42 @@ class Learner:
         logp = torch.empty(n, dtype=torch.float32, device=self.device)
         value = torch.empty(n, dtype=torch.float32, device=self.device)
         obs = ppo.Minibatch(depth.data_ptr(), proprio.data_ptr(), None, None, None, None, None, None, n)
+        if self.recurrent and (self.roll_h is None or self.roll_h.shape[1] != n):
+            self.reset_rollout_state(n)
         for r0 in range(0, n, self.microbatch):
             rows = min(self.microbatch, n - r0)
+            if self.recurrent:  # a one-step sequence from the state the envs carry
+                h_in = self.roll_h[:, r0:r0 + rows].contiguous()
+                c_in = self.roll_c[:, r0:r0 + rows].contiguous()
+                ppo.ppo_model_set_sequence(self.model, 1, rows, self.roll_done[r0:r0 + rows], h_in, c_in)
             ppo.ppo_encoder_fwd(self.model, obs, r0, rows, self.mean, value[r0:r0 + rows])
             ppo.ppo_policy_sample(self.model, rows, self.mean, eps[r0:r0 + rows], action[r0:r0 + rows],
                                   logp[r0:r0 + rows])
+            if self.recurrent:
+                H = self.w.lstm_h
+                for l in range(self.w.n_lstm):
+                    self.roll_h[l, r0:r0 + rows] = self.model.activation(5, l)[:rows * H].view(rows, H).float()
+                    self.roll_c[l, r0:r0 + rows] = self.model.activation(6, l)[:rows * H].view(rows, H)
         return action, logp, value
+
+    def reset_rollout_state(self, n: int, done: Optional[torch.Tensor] = None):
+        """Recurrent state the rollout policy carries per env: all zeros (done None), or zeroed where done != 0."""
+        w = self.w
+        if done is None or self.roll_h is None:
+            self.roll_h = torch.zeros((w.n_lstm, n, w.lstm_h), dtype=torch.float32, device=self.device)
+            self.roll_c = torch.zeros_like(self.roll_h)
+            self.roll_done = torch.zeros(n, dtype=torch.uint8, device=self.device)
+        else:
+            keep = (done == 0).to(torch.float32).view(1, n, 1)
+            self.roll_h *= keep
+            self.roll_c *= keep
 
     def act_into_buffer(self, t: int, depth: torch.Tensor, proprio: torch.Tensor, eps: torch.Tensor):
         """One rollout step without intermediate copies: the observation goes into slab row t, the policy reads
         it there and writes action, log-prob and value into the same row (Algorithm 2, actions <- pi(obs) then
         D <- D U {...}); ppo_buffer_write_outcome adds reward and done once the env has stepped."""
+        if self.recurrent:
+            raise NotImplementedError("a recurrent policy acts through act(), which carries the state")
         ppo.ppo_buffer_write_obs(self.buffer, t, depth, proprio)
         ppo.ppo_policy_act(self.model, self.buffer, t, eps)
 
