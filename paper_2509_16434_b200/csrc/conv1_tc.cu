@@ -23,8 +23,8 @@ namespace {
 using namespace tc;
 
 constexpr int kMaxStages = 8;
-constexpr int kProdGroups = 4;  // groups of 128 producer threads; group g builds sub-tile g of every stage
-constexpr int kEpiWarps = 8;    // two per TMEM lane quarter, alternate 16-column chunks
+constexpr int kProdGroups = 3;  // groups of 128 producer threads; group g builds sub-tile g of every stage
+constexpr int kEpiWarps = 12;   // three per TMEM lane quarter, which take the column groups in turn
 constexpr int kThreads = (kProdGroups * 4 + 1 + kEpiWarps) * 32;
 
 struct Args {
@@ -256,7 +256,7 @@ __global__ void __launch_bounds__(kThreads, 1) conv1_tc_kernel(const __grid_cons
             if (!ok) break;
             tc_fence_after();
             const uint32_t lane_base = tmem_base + acc * acc_cols + ((uint32_t)(lg * 32) << 16);
-            for (int cc = half * CW; cc < T * N; cc += 2 * CW) {   // column of the accumulator: tile g, channel c0
+            for (int cc = half * CW; cc < T * N; cc += (kEpiWarps / 4) * CW) {   // column of the accumulator: tile g, channel c0
                 const int g = cc / N, c0 = cc - g * N;
                 const long long m0 = ((long long)(s0 + li) * T + g) * 128 + lg * 32;  // first pixel of this warp
                 float v[32];
