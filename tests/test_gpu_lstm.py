@@ -22,6 +22,8 @@ REC = {
                                 embed=32, n_lstm=2, lstm_h=128),
     # the paper's policy (CNN, embedding, 2 x LSTM(1024), fully connected [512, 512, 256]) on few envs
     "paper_twin": synth.WORKLOADS["paper_policy"].scaled(8, T=3, minibatches=2),
+    # the same at the paper's horizon of 16 steps: 256-row sequence minibatches (two row tiles in the all-step GEMMs)
+    "paper_h16": synth.WORKLOADS["paper_policy"].scaled(32, T=16, minibatches=2),
 }
 
 
@@ -113,7 +115,7 @@ def _forward(L, w, f, h0, c0):
 
 
 @pytest.mark.parametrize("name,zero_state", [("rec_pool", False), ("rec_embed", False), ("rec_embed", True),
-                                             ("paper_twin", False)])
+                                             ("paper_twin", False), ("paper_h16", False)])
 def test_forward_through_time_matches_oracle(name, zero_state):
     w = REC[name]
     K = w.minibatches
@@ -175,7 +177,7 @@ def _oracle_step(md, theta, f, h0, c0, h):
                                        np.float32(h.ent_coef), act_bf16=True)
 
 
-@pytest.mark.parametrize("name", ["rec_pool", "rec_embed", "paper_twin"])
+@pytest.mark.parametrize("name", ["rec_pool", "rec_embed", "paper_twin", "paper_h16"])
 def test_backward_through_time_matches_oracle_on_identical_state(name):
     """Both sides start from the oracle's saved activations, recurrent state, mean and value."""
     w = REC[name]
