@@ -1118,7 +1118,8 @@ static void tma_dgrad_shifts(int k, int *dmin, int *n1) {
 // pixels (2y + ph, 2x + pw); column class * Ci + ci; the reduction runs over the shifts (dy, dx) of the
 // output pixel (y + dy, x + dx) and its channels, with the weights Wc[class * Ci + ci][shift][co] (zero
 // where a class has no kernel tap at that shift).  One wide GEMM instead of four narrow ones: the tensor
-// core is fed by one thread, and an instruction costs the same whether it is 32 or 256 columns wide.
+// core is fed by one thread, and an instruction of 64 columns or fewer occupies it as long as one of 128
+// (~55 cycles per issue at best; 128 columns run at the tensor rate of 64 cycles, 256 at 128).
 int tma_gemm_dgrad(const ConvGeom &g, const bf16 *dY, int ldy, const bf16 *Wt, int wt_ld, const bf16 *Wc,
                    const DgradEpilogue &e, int32_t *status, cudaStream_t st) {
     if (!status || g.Ci % 8 != 0 || ldy % 8 != 0 || wt_ld % 8 != 0 || ldy < wt_ld) return PPO_ERR_UNSUPPORTED;
