@@ -958,12 +958,12 @@ int pick_bn(int N) {  // tile width: N split evenly into tiles of at most 256, r
     return bn < 16 ? 16 : bn;
 }
 
-// Tile width of a flat GEMM (rows x N): as pick_bn, then halved while the tiles would leave SMs without work (few rows,
-// as in the per-step products of a recurrent layer) and the halves still divide N.
+// Tile width of a flat GEMM (rows x N): as pick_bn, then halved while the tiles would leave more than half of the SMs
+// without work (few rows, as in the per-step products of a recurrent layer) and the halves still divide N.
 static int flat_bn(int N, long long rows) {
     int bn = pick_bn(N);
     const long long mt = (rows + 127) / 128;
-    while (bn >= 64 && bn % 32 == 0 && N % (bn / 2) == 0 && mt * ((N + bn - 1) / bn) < ppo_num_sms()) bn /= 2;
+    while (bn >= 64 && bn % 32 == 0 && N % (bn / 2) == 0 && mt * ((N + bn - 1) / bn) < ppo_num_sms() / 2) bn /= 2;
     return bn;
 }
 
@@ -1015,7 +1015,10 @@ int launch_kmajor(KArgs &a, cudaStream_t st) {
     // Narrow tiles (BN <= 128) leave the tensor pipe mostly idle because one thread per CTA cannot issue MMAs
     // fast enough; two CTAs per SM (half the shared and tensor memory each, 8 epilogue warps each) double the
     // issue rate.  Wide tiles run at the tensor rate with one CTA and keep the SM to themselves.
-    const bool two = a.BN <= 128;
+    // A GEMM of a few row tiles gives a CTA one or two tiles: nothing amortises the copy latency, so such a CTA takes the
+    // SM alone, with stages of up to 96 KB (fewer, larger hand-overs), and the narrow-tile rule below does not apply.
+    const bool small_m = a.grid.tiles <= 4 && a.ncls == 1;
+    const bool two = a.BN <= 128 && !small_m;
     a.tmem_cap = two ? 256 : 512;
     a.nepi = (!two && a.mode == EPI_DGRAD && a.mask_bits) ? 16 : 8;
     const size_t fixed = sizeof(PipeK) + (size_t)a.nepi * 2048 + 1024;  // pipeline state, epilogue staging, alignment slack
@@ -1023,9 +1026,9 @@ int launch_kmajor(KArgs &a, cudaStream_t st) {
     if (a.wres && res + fixed + 3 * (size_t)128 * a.row_bytes + 1024 > cta_max) a.wres = 0;
     const size_t sub = (size_t)128 * a.row_bytes + (a.wres ? 0 : b_bytes);
     const size_t budget = cta_max - 1024 - fixed - (a.wres ? res : 0);
-    int G = (int)((48 * 1024) / sub);  // sub-blocks per stage: fewer barrier round trips per byte
+    int G = (int)(((small_m ? 96 : 48) * 1024) / sub);  // sub-blocks per stage: fewer barrier round trips per byte
     G = G < 1 ? 1 : (G > 8 ? 8 : G);
-    while (G > 1 && budget / (G * sub) < 3) --G;
+    while (G > 1 && budget / (G * sub) < (small_m ? 2 : 3)) --G;
     const int lps = a.nbmax + (a.wres ? 0 : 1);  // copies per sub-block; one producer lane each
     if (lps > 32) return PPO_ERR_UNSUPPORTED;
     while (G > 1 && G * lps > 32) --G;
