@@ -266,6 +266,14 @@ int ppo_model_bind(ppo_model *m, float *dev_master, void *dev_shadow_bf16, float
 int ppo_model_set_sequence(ppo_model *m, int T, int Be, const uint8_t *dev_done, const float *dev_h_init,
                            const float *dev_c_init);
 
+/* The recurrent state the step AFTER the announced sequence starts from (Algorithm 2 keeps acting with the policy from
+ * one buffer fill to the next): dev_h_out, dev_c_out fp32 [n_lstm][Be][lstm_h] receive h and c of the last time step of
+ * the latest ppo_encoder_fwd (h as the layers pass it on, i.e. rounded to bf16), zeroed where that step's done flag is
+ * set.  They may be the arrays a later ppo_model_set_sequence names as the initial state, but not the ones the
+ * current sequence was announced with while its backward pass is still to run.  Errors: no forward since the sequence
+ * was announced, or a model without LSTM layers -> STATE. */
+int ppo_model_read_state(const ppo_model *m, float *dev_h_out, float *dev_c_out, void *stream);
+
 /* shadow <- bf16(master) (round to nearest even); call after writing master from outside. */
 int ppo_model_sync_shadow(ppo_model *m, void *stream);
 

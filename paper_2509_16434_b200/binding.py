@@ -29,6 +29,7 @@ EXPORTS = [
     "ppo_adam_step", "ppo_policy_sample", "ppo_poll_status", "ppo_model_activation_ptr", "ppo_gae_static",
     "ppo_model_sync_masks", "ppo_buffer_write_obs", "ppo_buffer_write_outcome", "ppo_policy_act", "ppo_launch_count",
     "ppo_selftest_wait_timeout", "ppo_buffer_render_depth", "ppo_model_set_sequence", "ppo_shuffle_gather_sequences",
+    "ppo_model_read_state",
 ]
 
 
@@ -110,6 +111,7 @@ def lib():
         L.ppo_model_set_sequence.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p]
         L.ppo_shuffle_gather_sequences.argtypes = [C.c_void_p, C.c_uint64, C.c_uint32, C.c_int, C.c_int,
                                                    C.POINTER(Minibatch), C.c_void_p, C.c_void_p]
+        L.ppo_model_read_state.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         L.ppo_launch_count.restype = C.c_uint64
         L.ppo_launch_count.argtypes = []
         L.ppo_selftest_wait_timeout.argtypes = [C.c_longlong, C.c_void_p, C.c_void_p]
@@ -353,6 +355,11 @@ class Model:
 def ppo_model_set_sequence(m: Model, T: int, Be: int, done, h_init, c_init):
     """done uint8 [T,Be], h_init / c_init fp32 [n_lstm,Be,lstm_h]: the tensors must stay alive until the backward pass."""
     _check(lib().ppo_model_set_sequence(m.handle, T, Be, _ptr(done), _ptr(h_init), _ptr(c_init)), "ppo_model_set_sequence")
+
+
+def ppo_model_read_state(m: Model, h_out, c_out, stream=None):
+    """fp32 [n_lstm,Be,lstm_h] each: the state after the last step of the latest forward, zero where that step was done."""
+    _check(lib().ppo_model_read_state(m.handle, _ptr(h_out), _ptr(c_out), _stream(stream)), "ppo_model_read_state")
 
 
 def ppo_shuffle_gather_sequences(buf: Buffer, seed: int, epoch: int, mb_index: int, num_minibatches: int,

@@ -325,6 +325,31 @@ extern "C" int ppo_model_set_sequence(ppo_model *m, int T, int Be, const uint8_t
     return PPO_OK;
 }
 
+// h (bf16 -> fp32) and c of the last time step, zero where done: one thread per state element of a layer.
+__global__ void __launch_bounds__(256) lstm_read_state_kernel(const bf16 *__restrict__ h, const float *__restrict__ c,
+                                                              const uint8_t *__restrict__ done, float *__restrict__ h_out,
+                                                              float *__restrict__ c_out, int Be, int H) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= Be * H) return;
+    const bool reset = done[i / H] != 0;
+    h_out[i] = reset ? 0.f : __bfloat162float(h[i]);
+    c_out[i] = reset ? 0.f : c[i];
+}
+
+extern "C" int ppo_model_read_state(const ppo_model *m, float *h_out, float *c_out, void *stream) {
+    if (!m || !h_out || !c_out) return PPO_ERR_INVALID_ARG;
+    if (m->d.n_lstm == 0 || !m->ws || m->seq_T <= 0 || !m->fwd_valid) return PPO_ERR_STATE;
+    const int Be = m->seq_Be, H = m->d.lstm_h;
+    const size_t last = (size_t)(m->seq_T - 1) * Be;
+    for (int l = 0; l < m->d.n_lstm; ++l) {
+        lstm_read_state_kernel<<<ppo_cdiv((long long)Be * H, 256), 256, 0, static_cast<cudaStream_t>(stream)>>>(
+            m->lstm_hs[l] + last * H, m->lstm_c[l] + last * H, m->seq_done + last, h_out + (size_t)l * Be * H,
+            c_out + (size_t)l * Be * H, Be, H);
+        PPO_LAUNCH_CHECK();
+    }
+    return PPO_OK;
+}
+
 extern "C" int ppo_model_sync_masks(ppo_model *m, int rows, void *stream) {
     if (!m || !m->ws) return PPO_ERR_STATE;
     if (rows <= 0 || rows > m->mbmax) return PPO_ERR_SHAPE;

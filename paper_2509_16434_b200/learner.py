@@ -92,11 +92,10 @@ class Learner:
             ppo.ppo_encoder_fwd(self.model, obs, r0, rows, self.mean, value[r0:r0 + rows])
             ppo.ppo_policy_sample(self.model, rows, self.mean, eps[r0:r0 + rows], action[r0:r0 + rows],
                                   logp[r0:r0 + rows])
-            if self.recurrent:
-                H = self.w.lstm_h
-                for l in range(self.w.n_lstm):
-                    self.roll_h[l, r0:r0 + rows] = self.model.activation(5, l)[:rows * H].view(rows, H).float()
-                    self.roll_c[l, r0:r0 + rows] = self.model.activation(6, l)[:rows * H].view(rows, H)
+            if self.recurrent:  # the state these envs carry into their next step
+                ppo.ppo_model_read_state(self.model, h_in, c_in)
+                self.roll_h[:, r0:r0 + rows] = h_in
+                self.roll_c[:, r0:r0 + rows] = c_in
         return action, logp, value
 
     def reset_rollout_state(self, n: int, done: Optional[torch.Tensor] = None):

@@ -251,3 +251,40 @@ def test_recurrent_model_rejects_calls_without_a_sequence():
     eps = torch.zeros((w.N, w.A), device=DEV)
     with pytest.raises(ppo.PpoError):  # the one-step rollout call has no recurrent state to carry
         ppo.ppo_policy_act(L.model, L.buffer, 0, eps)
+
+
+def test_state_after_a_sequence_matches_oracle_and_chains():
+    """ppo_model_read_state: h and c of the last step (zero where that step was done) against the oracle's record, and
+    a sequence run in one piece against the same sequence run step by step through the returned state."""
+    w = REC["rec_embed"]
+    K = w.minibatches
+    L, md, lay, theta, roll, action, logp, dev = _setup(w, (w.N // K) * w.T)
+    L.compute_gae(dev["last_value"])
+    Be, R, H = L.seq_envs, L.seq_envs * w.T, w.lstm_h
+    _gather_group(L, w, 4, 0, 0, K)
+    envs, f = _oracle_sequences(w, roll, action, logp, L.hyper, 4, 0, 0, K)
+    L.seq_done[w.T - 1, ::2] = 1  # some envs end their episode on the last step
+    f["done"][w.T - 1, ::2] = 1
+    h0, c0 = _states(w, Be, 3)
+    _forward(L, w, f, h0, c0)
+    h_out, c_out = torch.empty_like(L.h_init), torch.empty_like(L.c_init)
+    ppo.ppo_model_read_state(L.model, h_out, c_out)
+    mu_all = L.mean[:R].clone()
+    _, _, _, lrec = orc.encoder_fwd_seq(md, orc.round_weights(md, theta), f["depth"], f["proprio"], f["done"], h0, c0, True)
+    last = lrec[(w.T - 1) * Be:]
+    keep = (f["done"][w.T - 1] == 0)[:, None]
+    for l in range(w.n_lstm):
+        h_o, c_o = last[:, l * 8 * H + 5 * H:l * 8 * H + 6 * H] * keep, last[:, l * 8 * H + 4 * H:l * 8 * H + 5 * H] * keep
+        assert rel_l2(h_out[l].cpu().numpy(), h_o) <= ENC_TOL and rel_l2(c_out[l].cpu().numpy(), c_o) <= ENC_TOL
+        assert np.all(h_out[l].cpu().numpy()[::2] == 0) and np.all(c_out[l].cpu().numpy()[::2] == 0)
+    # step by step: T one-step sequences, each started from the state the previous one returned
+    hs, cs = torch.as_tensor(h0).to(DEV), torch.as_tensor(c0).to(DEV)
+    one = ppo.Minibatch(L.mb.depth.data_ptr(), L.mb.proprio.data_ptr(), None, None, None, None, None, None, R)
+    for t in range(w.T):
+        ppo.ppo_model_set_sequence(L.model, 1, Be, L.seq_done[t], hs, cs)
+        ppo.ppo_encoder_fwd(L.model, one, t * Be, Be, L.mean, L.value)
+        assert torch.equal(L.mean[:Be], mu_all[t * Be:(t + 1) * Be]), t
+        hs, cs = torch.empty_like(hs), torch.empty_like(cs)
+        ppo.ppo_model_read_state(L.model, hs, cs)
+    assert torch.equal(hs, h_out) and torch.equal(cs, c_out)
+    assert ppo.ppo_poll_status() == 0

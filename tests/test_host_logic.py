@@ -105,6 +105,8 @@ def test_model_layout_matches_the_oracles(lib, name):
         # a sequence must be announced with sane arguments
         assert lib.ppo_model_set_sequence(h, 4, 4, C.c_void_p(0x100), C.c_void_p(0x100), C.c_void_p(0x100)) == 4  # unbound
         assert lib.ppo_model_set_sequence(h, 4, 4, None, C.c_void_p(0x100), C.c_void_p(0x100)) == 1
+        assert lib.ppo_model_read_state(h, C.c_void_p(0x100), C.c_void_p(0x100), None) == 4  # nothing was run yet
+        assert lib.ppo_model_read_state(h, None, C.c_void_p(0x100), None) == 1
     else:
         assert lib.ppo_model_set_sequence(h, 4, 4, C.c_void_p(0x100), C.c_void_p(0x100), C.c_void_p(0x100)) != 0
     ws1, ws2 = lib.ppo_model_workspace_bytes(h, 64), lib.ppo_model_workspace_bytes(h, 128)
