@@ -725,20 +725,24 @@ __global__ void __launch_bounds__(256) lstm_cell_fwd_kernel(const float *__restr
 }
 
 // The same step backwards.  dtop: gradient w.r.t. this step's h from above; dhc, dcc: gradients w.r.t. the state the
-// NEXT step started from (raw: they count only where this step's done flag is clear).  Writes the gradient of the gate
-// pre-activations as bf16 (a GEMM operand) and the raw gradient of c_prev; the raw gradient of h_prev comes out of the
-// GEMM dg W_h that follows.  last != 0: no step follows, nothing is carried.
+// NEXT step started from (raw: they count only where this step's done flag is clear; dhc arrives as nsplit partial
+// products, Be * H floats apart, that are added in order).  Writes the gradient of the gate pre-activations as bf16 (a
+// GEMM operand) and the raw gradient of c_prev; the raw gradient of h_prev comes out of the GEMM dg W_h that follows.
+// last != 0: no step follows, nothing is carried.
 __global__ void __launch_bounds__(256) lstm_cell_bwd_kernel(const float *__restrict__ dtop, const float *__restrict__ dhc,
                                                             float *__restrict__ dcc, const uint8_t *__restrict__ done,
                                                             const float *__restrict__ gates, const float *__restrict__ c,
                                                             const float *__restrict__ cprev, bf16 *__restrict__ dg,
-                                                            int Be, int H, int last) {
+                                                            int Be, int H, int last, int nsplit) {
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= Be * H) return;
     const int e = i / H, j = i - e * H;
     const size_t g0 = (size_t)e * 4 * H + j;
     const bool carry = !last && done[e] == 0;
-    const float dh = dtop[i] + (carry ? dhc[i] : 0.f);
+    float dhn = 0.f;
+    if (carry)
+        for (int s = 0; s < nsplit; ++s) dhn += dhc[(size_t)s * Be * H + i];
+    const float dh = dtop[i] + dhn;
     const float gi = gates[g0], gf = gates[g0 + H], gg = gates[g0 + 2 * H], go = gates[g0 + 3 * H];
     const float tc = tanhf(c[i]);
     const float dc = (carry ? dcc[i] : 0.f) + dh * go * (1.f - tc * tc);
@@ -861,10 +865,14 @@ static int wt_ld_of(int Co) { return (Co + 7) / 8 * 8; }
 
 // out [rows][N] (fp32, row stride N) = A [rows][K] (bf16, row stride lda) . Wn [N][K]^T: the plain product behind every
 // contraction of the recurrent trunk, through the flat (1x1-image) input-gradient GEMM.
+// ksplit > 1: the reduction is cut into that many slabs and `out` receives their partial products one after another
+// (rows * N floats each), for the reader to add in order.
 static int gemm_nt_f32(const ppo_model *m, int rows, int N, int K, const bf16 *A, int lda, const bf16 *Wn, float *out,
-                       cudaStream_t st) {
+                       cudaStream_t st, int ksplit = 1) {
     ConvGeom g = fc_geom(rows, N, K);
     DgradEpilogue e = {nullptr, nullptr, out};
+    e.ksplit = ksplit;
+    if (ksplit > 1) return tma_gemm_dgrad(g, A, lda, Wn, K, nullptr, e, ppo_device_status_ptr(), st);
     return run_dgrad(m, g, A, lda, Wn, Wn, K, nullptr, e, st);
 }
 
@@ -907,14 +915,25 @@ static int lstm_backward(ppo_model *m, int rows, cudaStream_t st) {
         const int in = l == 0 ? m->hw[0] : H, ti = m->ti_lstm[l];
         const bf16 *X = l == 0 ? m->h[0] : m->lstm_hs[l - 1];
         const float *cprev = m->lstm_c[l] + (size_t)m->mbmax * H;
+        // dg W_h reduces over 4H columns into few output tiles: with few envs the reduction is cut into four slabs that
+        // as many CTAs work on, and the next cell kernel adds their partial products (dhc holds rows * H floats)
+        int nsplit = (T >= 4 && Be <= 512) ? 4 : 1;
         for (int t = T - 1; t >= 0; --t) {
             const size_t r0 = (size_t)t * Be;
             lstm_cell_bwd_kernel<<<ppo_cdiv((long long)Be * H, 256), 256, 0, st>>>(
                 m->lstm_dtop + r0 * H, m->lstm_dhc, m->lstm_dcc, m->seq_done + r0, m->lstm_gates[l] + r0 * 4 * H,
-                m->lstm_c[l] + r0 * H, cprev + r0 * H, m->lstm_dg + r0 * 4 * H, Be, H, t == T - 1 ? 1 : 0);
+                m->lstm_c[l] + r0 * H, cprev + r0 * H, m->lstm_dg + r0 * 4 * H, Be, H, t == T - 1 ? 1 : 0, nsplit);
             PPO_LAUNCH_CHECK();
-            if (t > 0)  // raw gradient of the state this step started from: dg W_h
-                PPO_TRY(gemm_nt_f32(m, Be, H, 4 * H, m->lstm_dg + r0 * 4 * H, 4 * H, m->wT + m->wT_off[ti + 1], m->lstm_dhc, st));
+            if (t > 0) {  // raw gradient of the state this step started from: dg W_h
+                int s = PPO_ERR_UNSUPPORTED;
+                if (nsplit > 1)
+                    s = gemm_nt_f32(m, Be, H, 4 * H, m->lstm_dg + r0 * 4 * H, 4 * H, m->wT + m->wT_off[ti + 1], m->lstm_dhc, st, nsplit);
+                if (s == PPO_ERR_UNSUPPORTED) {
+                    nsplit = 1;
+                    s = gemm_nt_f32(m, Be, H, 4 * H, m->lstm_dg + r0 * 4 * H, 4 * H, m->wT + m->wT_off[ti + 1], m->lstm_dhc, st);
+                }
+                PPO_TRY(s);
+            }
         }
         // over all steps at once: the weight gradients, the bias gradient and the gradient of the layer's input
         PPO_TRY(run_wgrad(m, ti, fc_geom(rows, in, 4 * H), m->lstm_dg, 4 * H, X, st, false));

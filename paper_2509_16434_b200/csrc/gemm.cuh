@@ -32,6 +32,8 @@ struct DgradEpilogue {
     float *out_f32;        // [M'][Ci] fp32, or nullptr
     const uint32_t *mask_bits = nullptr;  // the same gate as one bit per element, [M'][Ci / 32] (channel c at bit gate_bit_of_channel(c) of word c / 32);
                                           // used instead of mask_act by kernels that support it
+    int ksplit = 1;  // flat GEMMs with out_f32 only: the reduction is cut into ksplit (<= 4) equal slabs and slab s leaves
+                     // its partial product in out_f32 + s * M' * Ci; the reader adds the slabs in order
 };
 
 // ldy: row stride (elements) of Y / dY (>= Co).  wt_ld: row stride of the innermost (co)

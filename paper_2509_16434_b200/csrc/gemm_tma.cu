@@ -189,6 +189,7 @@ struct KArgs {
     int N, BN, tiles_n, total_tiles, ncls, stages;  // tile g = ((mt * tiles_n) + nt) * ncls + class
     int Hout, Wout, ldo;
     int nq_ci;  // merged dgrad: channels per parity class (column n = class * nq_ci + channel), else 0
+    long long cls_orows;  // output rows between the classes' results (split reduction of a flat GEMM), else 0
     int mode, relu, A;
     const float *bias;
     bf16 *out;
@@ -428,7 +429,7 @@ __global__ void __launch_bounds__(kKThreads, 1) tma_kmajor_kernel(const __grid_c
                     oy = 2 * y + (q >> 1);
                     ox = 2 * x + (q & 1);
                 }
-                orow = ((long long)n * a.Hout + oy) * a.Wout + ox;
+                orow = ((long long)n * a.Hout + oy) * a.Wout + ox + tc_.c * a.cls_orows;
                 return pix_ok && oy < a.Hout && ox < a.Wout;
             };
             const int ncol = a.nq_ci ? a.nq_ci : a.N;  // columns of an output row
@@ -1017,7 +1018,7 @@ int launch_kmajor(KArgs &a, cudaStream_t st) {
     // issue rate.  Wide tiles run at the tensor rate with one CTA and keep the SM to themselves.
     // A GEMM of a few row tiles gives a CTA one or two tiles: nothing amortises the copy latency, so such a CTA takes the
     // SM alone, with stages of up to 96 KB (fewer, larger hand-overs), and the narrow-tile rule below does not apply.
-    const bool small_m = a.grid.tiles <= 4 && a.ncls == 1;
+    const bool small_m = a.grid.tiles <= 4 && (a.ncls == 1 || a.cls_orows != 0);
     const bool two = a.BN <= 128 && !small_m;
     a.tmem_cap = two ? 256 : 512;
     a.nepi = (!two && a.mode == EPI_DGRAD && a.mask_bits) ? 16 : 8;
@@ -1154,6 +1155,43 @@ int tma_gemm_dgrad(const ConvGeom &g, const bf16 *dY, int ldy, const bf16 *Wt, i
     a.mask = e.mask_act;
     a.mask_bits = flat ? nullptr : e.mask_bits;
     a.status = status;
+    const int ks = flat && e.ksplit > 1 ? e.ksplit : 1;
+    if (ks > 1) {
+        // Split reduction: the Co columns of dY are seen as an image of ks rows of Co / ks channels (row y of pixel x
+        // starts at x * ldy + y * Co / ks), class s reads row s against the weight columns s * Co / ks .. and
+        // leaves its product in its own copy of the output.
+        if (ks > 4 || g.Co % (ks * 64) != 0 || !e.out_f32 || e.out || e.mask_act) return PPO_ERR_UNSUPPORTED;
+        const int Kc = g.Co / ks;
+        a.kchunks = Kc / CB;
+        a.w_tap = Kc;
+        EncodeTiledFn fn = encode_fn();
+        if (!fn || !ppo_aligned(dY, 16)) return PPO_ERR_UNSUPPORTED;
+        const cuuint64_t gd[4] = {(cuuint64_t)Kc, (cuuint64_t)g.B, (cuuint64_t)ks, 1};
+        const cuuint64_t gs[3] = {(cuuint64_t)ldy * 2, (cuuint64_t)Kc * 2, (cuuint64_t)ldy * 2 * (cuuint64_t)g.B};
+        const cuuint32_t bx[4] = {(cuuint32_t)CB, (cuuint32_t)a.grid.Wt, 1, 1}, es[4] = {1, 1, 1, 1};
+        if (a.grid.R != 1 ||
+            fn(&a.mapA[0], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<bf16 *>(dY), gd, gs, bx, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+               CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return PPO_ERR_UNSUPPORTED;
+        a.N = g.Ci;
+        a.BN = flat_bn(g.Ci, (long long)g.B * ks);
+        a.wtaps = ks;
+        const long long dims[2] = {wt_ld, g.Ci};
+        const int box[2] = {CB, a.BN}, esb[2] = {1, 1};
+        s = make_map(&a.mapB, Wt, 2, dims, wt_ld, box, esb, a.row_bytes);
+        if (s != PPO_OK) return s;
+        a.ncls = ks;
+        a.cls_orows = g.B;
+        for (int c = 0; c < ks; ++c) {
+            KClass &k = a.cls[c];
+            k.b_row0 = 0;
+            k.taps.n = 1;
+            k.taps.dy[0] = (int8_t)c;
+            k.taps.dx[0] = 0;
+            k.taps.wt[0] = (decltype(k.taps.wt[0]))c;
+        }
+        return launch_kmajor(a, st);
+    }
     if (flat) {
         a.N = g.Ci;
         a.BN = flat_bn(g.Ci, g.B);
