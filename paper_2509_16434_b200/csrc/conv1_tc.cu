@@ -23,9 +23,10 @@ namespace {
 using namespace tc;
 
 constexpr int kMaxStages = 8;
-constexpr int kProdGroups = 3;  // groups of 128 producer threads; group g builds sub-tile g of every stage
-constexpr int kEpiWarps = 12;   // three per TMEM lane quarter, which take the column groups in turn
-constexpr int kThreads = (kProdGroups * 4 + 1 + kEpiWarps) * 32;
+constexpr int kProdWarps = 4;    // 128 producer threads; thread r fills row r of every tile of a stage with asynchronous copies
+constexpr int kMaxT = 5;         // tiles per stage at most
+constexpr int kEpiWarps = 20;    // five per TMEM lane quarter, which take the column groups in turn
+constexpr int kThreads = (kProdWarps + 1 + kEpiWarps) * 32;
 
 struct Args {
     const __half *depth;
@@ -58,6 +59,12 @@ struct Pipe {
 // (r / 8) * (KP / 8) * 128 + (k / 8) * 128 + (r % 8) * 16 + (k % 8) * 2 bytes.
 __device__ __forceinline__ uint32_t core_offset(int r, int kchunk, int KP) {
     return (uint32_t)(r >> 3) * (uint32_t)(KP >> 3) * 128u + (uint32_t)kchunk * 128u + (uint32_t)(r & 7) * 16u;
+}
+
+// Four bytes global -> shared without passing through registers; !valid writes zeros (no source byte is read).
+__device__ __forceinline__ void cp_async4(uint32_t dst, const void *src, bool valid) {
+    const uint32_t n = valid ? 4u : 0u;
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;" ::"r"(dst), "l"(src), "r"(n) : "memory");
 }
 
 __device__ __forceinline__ uint64_t desc_nosw(uint32_t addr, uint32_t lbo, uint32_t sbo) {
@@ -100,7 +107,7 @@ __global__ void __launch_bounds__(kThreads, 1) conv1_tc_kernel(const __grid_cons
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < S; ++s) {
-            mbar_init(&pipe->full[s], T * 128);
+            mbar_init(&pipe->full[s], kProdWarps * 32);
             mbar_init(&pipe->empty[s], 1);
         }
         for (int i = 0; i < nacc; ++i) {
@@ -124,12 +131,20 @@ __global__ void __launch_bounds__(kThreads, 1) conv1_tc_kernel(const __grid_cons
         }
         *reinterpret_cast<__half *>(bsm + core_offset(n, k >> 3, KP) + (k & 7) * 2) = __float2half_rn(f);
     }
+    // The constant part of every im2col row of every stage: the two bias slots hold 1.0 (as fp16), the padding behind
+    // them zero.  The producers' copies only ever write the window words in front of it.
+    for (int i = threadIdx.x; i < S * T * 128; i += kThreads) {
+        uint8_t *row = smem + (size_t)(i >> 7) * kTileBytes;
+#pragma unroll
+        for (int k = KW; k < KP / 2; ++k)
+            *reinterpret_cast<uint32_t *>(row + core_offset(i & 127, k >> 2, KP) + (k & 3) * 4) = k == KW ? 0x3C003C00u : 0u;
+    }
     if (a.ln_gamma && threadIdx.x < 32) {
         pipe->gamma[threadIdx.x] = (int)threadIdx.x < N ? a.ln_gamma[threadIdx.x] : 0.f;
         pipe->beta[threadIdx.x] = (int)threadIdx.x < N ? a.ln_beta[threadIdx.x] : 0.f;
     }
     fence_async_smem();
-    if (warp == kProdGroups * 4) tmem_alloc(&pipe->tmem_slot, ncols);
+    if (warp == kProdWarps) tmem_alloc(&pipe->tmem_slot, ncols);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -141,35 +156,35 @@ __global__ void __launch_bounds__(kThreads, 1) conv1_tc_kernel(const __grid_cons
     const int q = nstage_all / (int)gridDim.x, rem = nstage_all - q * (int)gridDim.x, b = (int)blockIdx.x;
     const int s0 = b * q + (b < rem ? b : rem), ns = q + (b < rem ? 1 : 0);
 
-    if (warp < kProdGroups * 4) {
-        // ---------------- producers: one output pixel per thread and stage
-        const int grp = warp >> 2, r = threadIdx.x & 127;
-        if (grp < T) {
-            bool ok = true;
-            // output pixel of this thread in its first stage, then advanced by T * 128 pixels per stage without
-            // divisions
-            const int step = T * 128, hw = a.Ho * a.Wo;
-            const int d_b = step / hw, d_oh = (step % hw) / a.Wo, d_ow = step % a.Wo;
-            const int Wh = a.Wi >> 1;  // 32-bit words per frame row
-            int ow, oh, ib;
-            long long m = ((long long)s0 * T + grp) * 128 + r;
-            {
-                ow = (int)(m % a.Wo);
-                const long long t = m / a.Wo;
-                oh = (int)(t % a.Ho);
-                ib = (int)(t / a.Ho);
-            }
-            int s = 0;
-            uint32_t ph = 0;
-            uint32_t wv[KP / 2];
-            // Window of this thread's current pixel into wv.  Every load is issued (from a clamped address where its
-            // pixel pair lies outside the frame) and the pairs outside are zeroed afterwards: no branch separates
-            // the loads of a window.
-            auto load_window = [&]() {
-#pragma unroll
-                for (int k = 0; k < KP / 2; ++k) wv[k] = 0u;
+    if (warp < kProdWarps) {
+        // ---------------- producers: thread r owns row r of each of the stage's T tiles.  A window goes from the frame
+        // straight into its im2col row as aligned pairs of fp16 pixels, one 4-byte asynchronous copy per pair (zeros
+        // where the pair lies outside the frame or the pixel past the end); the copies of up to S stages are in flight
+        // while the thread moves on, and the stage's barrier counts them in as they land.
+        const int r = threadIdx.x;
+        bool ok = true;
+        const int hw = a.Ho * a.Wo;
+        const int d_b = 128 / hw, d_oh = (128 % hw) / a.Wo, d_ow = 128 % a.Wo;  // 128 pixels further, without divisions
+        const int Wh = a.Wi >> 1;  // 32-bit words per frame row
+        const uint32_t *frames = reinterpret_cast<const uint32_t *>(a.depth);
+        long long m = (long long)s0 * T * 128 + r;
+        int ow = (int)(m % a.Wo);
+        int oh, ib;
+        {
+            const long long t = m / a.Wo;
+            oh = (int)(t % a.Ho);
+            ib = (int)(t / a.Ho);
+        }
+        const uint32_t row_off = core_offset(r, 0, KP);
+        int s = 0;
+        uint32_t ph = 0;
+        for (int li = 0; li < ns && ok; ++li) {
+            ok = mbar_wait(&pipe->empty[s], ph ^ 1u, abort_flag, a.status);
+            if (!ok) break;
+            uint32_t dst = smem_base + (uint32_t)s * stage_bytes + row_off;
+            for (int g = 0; g < T; ++g, dst += kTileBytes) {
                 const bool live = m < a.M;
-                const uint32_t *img = reinterpret_cast<const uint32_t *>(a.depth) + (long long)(live ? ib : 0) * a.Hi * Wh;
+                const uint32_t *img = frames + (long long)(live ? ib : 0) * a.Hi * Wh;
                 const int pw0 = ow - (P + ODD) / 2;  // first pair of the window row, in words
 #pragma unroll
                 for (int kh = 0; kh < KS; ++kh) {
@@ -178,38 +193,23 @@ __global__ void __launch_bounds__(kThreads, 1) conv1_tc_kernel(const __grid_cons
                     const uint32_t *row = img + (rok ? ih : 0) * Wh;
 #pragma unroll
                     for (int qq = 0; qq < NP; ++qq) {
-                        const int pw = pw0 + qq;
+                        const int pw = pw0 + qq, k = kh * NP + qq;
                         const bool pok = rok && (unsigned)pw < (unsigned)Wh;
-                        const uint32_t v = __ldg(row + (pok ? pw : 0));
-                        wv[kh * NP + qq] = pok ? v : 0u;
+                        cp_async4(dst + (uint32_t)(k >> 2) * 128u + (uint32_t)(k & 3) * 4u, row + (pok ? pw : 0), pok);
                     }
                 }
-                wv[KW] = live ? 0x3C003C00u : 0u;  // (1.0, 1.0): the bias slots; rows past the last pixel stay zero
-            };
-            if (ns > 0) load_window();
-            // the window of the next stage is fetched before this stage's slot is waited for, so that the loads'
-            // latency overlaps the wait
-            for (int li = 0; li < ns && ok; ++li) {
-                ok = mbar_wait(&pipe->empty[s], ph ^ 1u, abort_flag, a.status);
-                if (!ok) break;
-                uint8_t *dst = smem + (size_t)s * stage_bytes + (size_t)grp * kTileBytes;
-#pragma unroll
-                for (int c = 0; c < KP / 8; ++c)
-                    *reinterpret_cast<uint4 *>(dst + core_offset(r, c, KP)) =
-                        make_uint4(wv[4 * c], wv[4 * c + 1], wv[4 * c + 2], wv[4 * c + 3]);
-                fence_async_smem();
-                mbar_arrive(&pipe->full[s]);
-                m += step;
+                m += 128;
                 ow += d_ow;
                 if (ow >= a.Wo) { ow -= a.Wo; ++oh; }
                 oh += d_oh;
                 if (oh >= a.Ho) { oh -= a.Ho; ++ib; }
                 ib += d_b;
-                if (li + 1 < ns) load_window();
-                if (++s == S) { s = 0; ph ^= 1u; }
             }
+            cp_async_arrive(&pipe->full[s]);
+            if (++s == S) { s = 0; ph ^= 1u; }
         }
-    } else if (warp == kProdGroups * 4) {
+        cp_async_wait<0>();
+    } else if (warp == kProdWarps) {
         // ---------------- MMA issue: T tiles per stage, each into its own columns of the accumulator
         const uint32_t idesc = idesc_f16(128, N);
         const uint32_t sbo = (uint32_t)(KP >> 3) * 128u;
@@ -225,6 +225,7 @@ __global__ void __launch_bounds__(kThreads, 1) conv1_tc_kernel(const __grid_cons
             if (!ok) break;
             ok = mbar_wait(&pipe->full[s], ph, abort_flag, a.status);
             if (!ok) break;
+            fence_async_smem();  // the producers' copies were ordinary shared-memory writes; the tensor core reads through the async proxy
             tc_fence_after();
             if (lane == 0) {
                 uint32_t la = (uint32_t)dA0 + (uint32_t)s * (stage_bytes >> 4);
@@ -241,10 +242,10 @@ __global__ void __launch_bounds__(kThreads, 1) conv1_tc_kernel(const __grid_cons
             if (++s == S) { s = 0; ph ^= 1u; }
         }
     } else {
-        // ---------------- epilogue: TMEM lane = pixel of a tile; warp w reads lanes 32 (w % 4) .. +31; the two
-        // warps of a lane quarter take alternate groups of 32 accumulator columns (16 when C1 is not a multiple
+        // ---------------- epilogue: TMEM lane = pixel of a tile; warp w reads lanes 32 (w % 4) .. +31; the
+        // warps of a lane quarter take the groups of 32 accumulator columns in turn (16 when C1 is not a multiple
         // of 32)
-        const int ew = warp - (kProdGroups * 4 + 1), lg = warp & 3, half = ew >> 2;
+        const int ew = warp - (kProdWarps + 1), lg = warp & 3, half = ew >> 2;
         const int p = lg * 32 + lane;
         const int CW = (N & 31) == 0 ? 32 : 16;
         uint4 *stg = staging + (size_t)ew * 128;
@@ -319,7 +320,7 @@ __global__ void __launch_bounds__(kThreads, 1) conv1_tc_kernel(const __grid_cons
     }
     tc_fence_before();
     __syncthreads();
-    if (warp == kProdGroups * 4) {
+    if (warp == kProdWarps) {
         tc_fence_after();
         tmem_dealloc(tmem_base, ncols);
     }
@@ -328,9 +329,8 @@ __global__ void __launch_bounds__(kThreads, 1) conv1_tc_kernel(const __grid_cons
 template <int KS>
 int launch(Args &a, cudaStream_t st) {
     constexpr int KP = Win<KS>::KP;
-    // tiles per stage: as many accumulators as fit twice into the 512 columns of tensor memory, at most one per
-    // producer group
-    a.T = 256 / a.C1 < kProdGroups ? 256 / a.C1 : kProdGroups;
+    // tiles per stage: as many accumulators as fit twice into the 512 columns of tensor memory, at most kMaxT
+    a.T = 256 / a.C1 < kMaxT ? 256 / a.C1 : kMaxT;
     if (a.T < 1) a.T = 1;
     const size_t stage = (size_t)a.T * 128 * KP * 2;
     a.stages = (int)((128 * 1024) / stage);
