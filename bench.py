@@ -33,11 +33,11 @@ sys.path.insert(0, ROOT)
 # sample row, from ncu captures of small twins of the workloads (traffic grows in proportion to the rows): workload
 # -> (bytes per row, capture).  An entry is dropped (traffic: null) as soon as a kernel it covers changes.
 NCU_DRAM_BYTES_PER_ROW = {
-    "cfg2": (2.7473e6, "ncu capture of cfg2_prof at 512 rows, scaled by rows: profiles/ncu_main_kernels_cfg2_prof.md"),
-    "cfg3": (2.7473e6, "ncu capture of cfg2_prof at 512 rows, scaled by rows: profiles/ncu_main_kernels_cfg2_prof.md"),
-    "cfg2_prof": (2.7473e6, "ncu capture of cfg2_prof at 512 rows: profiles/ncu_main_kernels_cfg2_prof.md"),
-    "cfg4": (11.3844e6, "ncu capture of cfg4_prof at 128 rows, scaled by rows: profiles/ncu_main_kernels_cfg4_prof.md"),
-    "cfg4_prof": (11.3844e6, "ncu capture of cfg4_prof at 128 rows: profiles/ncu_main_kernels_cfg4_prof.md"),
+    "cfg2": (2.7490e6, "ncu capture of cfg2_prof at 512 rows, scaled by rows: profiles/ncu_main_kernels_cfg2_prof.md"),
+    "cfg3": (2.7490e6, "ncu capture of cfg2_prof at 512 rows, scaled by rows: profiles/ncu_main_kernels_cfg2_prof.md"),
+    "cfg2_prof": (2.7490e6, "ncu capture of cfg2_prof at 512 rows: profiles/ncu_main_kernels_cfg2_prof.md"),
+    "cfg4": (11.4461e6, "ncu capture of cfg4_prof at 128 rows, scaled by rows: profiles/ncu_main_kernels_cfg4_prof.md"),
+    "cfg4_prof": (11.4461e6, "ncu capture of cfg4_prof at 128 rows: profiles/ncu_main_kernels_cfg4_prof.md"),
 }
 METRIC = "ppo_learner_env_steps_trained_per_sec"
 UNIT = "env-steps/s"
